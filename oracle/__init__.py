@@ -1,0 +1,25 @@
+"""CPU oracle of the Beagle cross-attention draft head.
+
+TEST INFRASTRUCTURE ONLY.  Nothing here is on the product path: the CUDA
+library never imports, links or calls this package, and this package never
+imports the CUDA binding.  Only the tests, the smoke check and the benchmark's
+CPU-baseline / reference legs may use it.
+"""
+from .beagle_oracle import (  # noqa: F401
+    HeadConfig,
+    OracleHead,
+    OracleSequence,
+    rms_norm,
+    silu,
+    visible_true_count,
+    project_kv,
+    attention_weights,
+    cross_attention,
+    draft_block,
+    prefill_kv,
+    rollback,
+    draft_step,
+    block_forward,
+    argmax_lowest,
+    verify_greedy,
+)

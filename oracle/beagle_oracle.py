@@ -1,0 +1,400 @@
+"""Plain fp64 CPU statement of the Beagle draft head (cross-attention speculative decoding).
+
+TEST INFRASTRUCTURE ONLY -- slow, obvious, independent of the CUDA library.
+Every floating-point operation runs in numpy float64; the only library
+primitives are matrix products, exp, sqrt and argmax.  Inputs arrive already
+rounded to whatever storage type the caller studies (bf16 values are exactly
+representable in float64), so the oracle itself never rounds.
+
+Notation follows the paper (Section 3 "Preliminaries", Section 4.1
+"Cross-Attention Draft Modeling", Section 4.2 "Two-Stage Block-Attention
+Training"):
+
+  * positions are 1-based; ``h_j`` is the higher-level state at position j
+    (it predicts token j+1); the query at position p is built from ``e(t_p)``;
+  * Eq. 1:  y_p = CrossAttn(h_{1:p-1}, e(t_p)) + e(t_p);  h_p = MLP(y_p) + y_p;
+  * Eq. 2:  Q = W_Q^T e(t_p), K_j = W_K^T h_j, V_j = W_V^T h_j, softmax over
+    the visible keys of <Q, K_j>/sqrt(d_h), o = sum_j s_j V_j, y = W_O^T[o^1..o^H];
+  * the cross mask hides every key j >= p (the diagonal too);
+  * logits z_p = e^{-1}(h_p) is a plain linear map to the vocabulary.
+
+Arrays are 0-based: ``tokens[p-1]`` is t_p and ``hidden[j-1]`` is h_j.
+Weights use the [out, in] row-major layout, i.e. the stored matrix is the
+paper's W^T; per-head matrices are consecutive row blocks of w_q / w_k / w_v
+and consecutive column blocks of w_o.
+
+Readings taken where the paper is silent (all are the caller's config flags or
+stated in the function that uses them):
+  * the mask is applied before the softmax (rows over visible keys sum to one);
+  * RMSNorm (gain g, eps) on the query input and on the MLP input, residuals
+    add the un-normalised vectors, no norm on key/value inputs, none before the
+    LM head;
+  * the MLP is SiLU-gated without biases: W_down( SiLU(W_gate n) * (W_up n) );
+  * grouped-query attention: query head h reads key/value head h // (Hq/Hkv);
+  * a query with no visible key gets o = 0;
+  * argmax ties go to the lowest index, NaN never wins.
+
+Pins (tests/test_oracle_*.py, all CPU): hand-worked tiny head, softmax row
+sums, single-key / identical-key special cases, GQA==MHA with repeated heads,
+mask brute force against the literal window rule, block forward == step-by-step
+drafting, greedy losslessness, the tail-sum closed form for the expected
+acceptance length, and a library cross-check (torch scaled-dot-product
+attention, F.silu, F.linear).  The paper prints no numeric example of the
+layer; its tokens/s and acceptance-length tables need trained weights and
+public evaluation suites, so those figures are "parity unpinned".
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Dict, Iterable, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+F64 = np.float64
+
+
+@dataclass(frozen=True)
+class HeadConfig:
+    hidden: int          # d
+    n_q_heads: int       # Hq
+    n_kv_heads: int      # Hkv (Hq % Hkv == 0)
+    head_dim: int        # d_h
+    mlp_dim: int         # m
+    vocab: int           # V
+    rms_eps: float = 1e-5
+    norm_q: bool = True
+    norm_mlp: bool = True
+
+    @property
+    def group(self) -> int:
+        return self.n_q_heads // self.n_kv_heads
+
+
+_WEIGHT_SHAPES = {
+    "embed": lambda c: (c.vocab, c.hidden),
+    "g_q": lambda c: (c.hidden,),
+    "w_q": lambda c: (c.n_q_heads * c.head_dim, c.hidden),
+    "w_k": lambda c: (c.n_kv_heads * c.head_dim, c.hidden),
+    "w_v": lambda c: (c.n_kv_heads * c.head_dim, c.hidden),
+    "w_o": lambda c: (c.hidden, c.n_q_heads * c.head_dim),
+    "g_mlp": lambda c: (c.hidden,),
+    "w_gate": lambda c: (c.mlp_dim, c.hidden),
+    "w_up": lambda c: (c.mlp_dim, c.hidden),
+    "w_down": lambda c: (c.hidden, c.mlp_dim),
+    "w_lm": lambda c: (c.vocab, c.hidden),
+}
+
+
+class OracleHead:
+    """The draft head's parameters, widened to float64."""
+
+    def __init__(self, cfg: HeadConfig, weights: Dict[str, np.ndarray]):
+        if cfg.n_q_heads % cfg.n_kv_heads != 0:
+            raise ValueError("n_q_heads must be a multiple of n_kv_heads")
+        self.cfg = cfg
+        for name, shape_of in _WEIGHT_SHAPES.items():
+            w = np.asarray(weights[name], dtype=F64)
+            if w.shape != shape_of(cfg):
+                raise ValueError(f"{name}: shape {w.shape}, expected {shape_of(cfg)}")
+            setattr(self, name, w)
+
+
+# --------------------------------------------------------------------------- primitives
+
+def rms_norm(v: np.ndarray, g: np.ndarray, eps: float) -> np.ndarray:
+    """RMSNorm over the last axis: g * v / sqrt(mean(v^2) + eps)."""
+    v = np.asarray(v, dtype=F64)
+    ms = np.mean(v * v, axis=-1, keepdims=True)
+    return g * (v / np.sqrt(ms + eps))
+
+
+def silu(u: np.ndarray) -> np.ndarray:
+    """SiLU(u) = u / (1 + exp(-u))."""
+    u = np.asarray(u, dtype=F64)
+    return u / (1.0 + np.exp(-u))
+
+
+def argmax_lowest(z: np.ndarray) -> np.ndarray:
+    """Arg-max over the last axis; ties go to the lowest index, NaN never wins
+    (a row of NaNs gives 0)."""
+    z = np.asarray(z, dtype=F64)
+    z = np.where(np.isnan(z), -np.inf, z)
+    return np.argmax(z, axis=-1).astype(np.int64)
+
+
+def visible_true_count(p: int, block: int, offset: int) -> int:
+    """Number of true states the query at (1-based) position p may read under
+    the inverse block mask of Section 4.2 combined with the strict cross mask
+    of Section 4.1.
+
+    Positions p <= offset lie before the first window and are plain strict
+    causal: keys 1..p-1.  Windows of size ``block`` tile the positions from
+    ``offset`` on; a window that starts at n holds the queries n+1..n+block,
+    and hides the keys n+1..n+block from all of them, so each of those queries
+    reads keys 1..n.
+    """
+    if block < 1 or offset < 0 or p < 1:
+        raise ValueError("bad mask arguments")
+    if p <= offset:
+        return p - 1
+    return offset + block * ((p - 1 - offset) // block)
+
+
+# --------------------------------------------------------------------------- Eq. 2
+
+def project_kv(head: OracleHead, states: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """K_j = W_K^T h_j, V_j = W_V^T h_j for every row of ``states`` [n, d].
+    Returns K, V of shape [n, Hkv, d_h]  (Eq. 2, first line)."""
+    c = head.cfg
+    s = np.asarray(states, dtype=F64).reshape(-1, c.hidden)
+    k = s @ head.w_k.T
+    v = s @ head.w_v.T
+    return (k.reshape(-1, c.n_kv_heads, c.head_dim), v.reshape(-1, c.n_kv_heads, c.head_dim))
+
+
+def attention_weights(head: OracleHead, q: np.ndarray, k_vis: np.ndarray) -> np.ndarray:
+    """Softmax over the visible keys of <Q^h, K_j^h> / sqrt(d_h)  (Eq. 2, second
+    line; only visible keys enter the softmax).  q: [Hq, d_h]; k_vis:
+    [nv, Hkv, d_h]; returns [Hq, nv]."""
+    c = head.cfg
+    nv = k_vis.shape[0]
+    w = np.zeros((c.n_q_heads, nv), dtype=F64)
+    if nv == 0:
+        return w
+    for h in range(c.n_q_heads):
+        kh = h // c.group
+        a = (k_vis[:, kh, :] @ q[h]) / np.sqrt(F64(c.head_dim))
+        a = a - np.max(a)
+        e = np.exp(a)
+        w[h] = e / np.sum(e)
+    return w
+
+
+def cross_attention(head: OracleHead, q: np.ndarray, k_vis: np.ndarray,
+                    v_vis: np.ndarray) -> np.ndarray:
+    """o^h = sum_j s^h_j V^h_j over the visible keys (Eq. 2, third line),
+    heads concatenated to [Hq*d_h].  No visible key: o = 0."""
+    c = head.cfg
+    w = attention_weights(head, q, k_vis)
+    o = np.zeros((c.n_q_heads, c.head_dim), dtype=F64)
+    for h in range(c.n_q_heads):
+        kh = h // c.group
+        if k_vis.shape[0]:
+            o[h] = w[h] @ v_vis[:, kh, :]
+    return o.reshape(-1)
+
+
+# --------------------------------------------------------------------------- Eq. 1
+
+def draft_block(head: OracleHead, tokens: Sequence[int],
+                kv_vis: Sequence[Tuple[np.ndarray, np.ndarray]]) -> Dict[str, np.ndarray]:
+    """The draft Transformer block (Eq. 1) and the LM head for a set of
+    independent query rows.  Row r has token ``tokens[r]`` and reads the
+    visible keys/values ``kv_vis[r] = (K [nv,Hkv,d_h], V [nv,Hkv,d_h])``.
+
+    Returns x (embeddings), q, o, y, h (the block output, also the state that
+    is re-used as key/value input when drafting continues), logits z and the
+    greedy token argmax z.
+    """
+    c = head.cfg
+    tok = np.asarray(tokens, dtype=np.int64).reshape(-1)
+    if np.any(tok < 0) or np.any(tok >= c.vocab):
+        raise ValueError("token id out of range")
+    x = head.embed[tok]                                         # e(t_p)
+    xq = rms_norm(x, head.g_q, c.rms_eps) if c.norm_q else x
+    q = xq @ head.w_q.T                                         # Q = W_Q^T e(t_p)
+    o = np.zeros((len(tok), c.n_q_heads * c.head_dim), dtype=F64)
+    for r in range(len(tok)):
+        k_vis, v_vis = kv_vis[r]
+        o[r] = cross_attention(head, q[r].reshape(c.n_q_heads, c.head_dim), k_vis, v_vis)
+    y = o @ head.w_o.T + x                                      # y = W_O^T[o] + e(t_p)
+    yn = rms_norm(y, head.g_mlp, c.rms_eps) if c.norm_mlp else y
+    mlp = (silu(yn @ head.w_gate.T) * (yn @ head.w_up.T)) @ head.w_down.T
+    h = mlp + y                                                 # h = MLP(y) + y
+    z = h @ head.w_lm.T                                         # z = e^{-1}(h)
+    return {"x": x, "q": q, "o": o, "y": y, "h": h, "logits": z, "argmax": argmax_lowest(z)}
+
+
+# --------------------------------------------------------------------------- serve-time drafting
+
+class OracleSequence:
+    """Key/value cache of one sequence: a prefix made from true (target)
+    states and a tail made from the draft's own states (Section 4.1, last
+    paragraphs: reuse cached K_j,V_j, append the new state's K,V when the next
+    state is queried, reset to true states at the end of the SD iteration)."""
+
+    def __init__(self, head: OracleHead):
+        c = head.cfg
+        self.k_true = np.zeros((0, c.n_kv_heads, c.head_dim), dtype=F64)
+        self.v_true = np.zeros((0, c.n_kv_heads, c.head_dim), dtype=F64)
+        self.k_draft: List[np.ndarray] = []
+        self.v_draft: List[np.ndarray] = []
+        self.pending_h: Optional[np.ndarray] = None   # previous step's h, not yet appended
+        self.pending_token: Optional[int] = None      # previous step's greedy token
+
+    @property
+    def n_true(self) -> int:
+        return self.k_true.shape[0]
+
+    @property
+    def n_draft(self) -> int:
+        return len(self.k_draft)
+
+
+def rollback(seq: OracleSequence) -> None:
+    """Reset the cache to true states only."""
+    seq.k_draft, seq.v_draft = [], []
+    seq.pending_h, seq.pending_token = None, None
+
+
+def prefill_kv(head: OracleHead, seq: OracleSequence, hidden_rows: np.ndarray) -> None:
+    """Drop the draft tail, then append K/V of new true states [r, d]."""
+    rollback(seq)
+    rows = np.asarray(hidden_rows, dtype=F64).reshape(-1, head.cfg.hidden)
+    if rows.shape[0] == 0:
+        return
+    k, v = project_kv(head, rows)
+    seq.k_true = np.concatenate([seq.k_true, k], axis=0)
+    seq.v_true = np.concatenate([seq.v_true, v], axis=0)
+
+
+def draft_step(head: OracleHead, seqs: Sequence[OracleSequence],
+               tokens_in: Optional[Sequence[int]] = None, concat: bool = True) -> Dict[str, np.ndarray]:
+    """One drafted token for each sequence.
+
+    ``tokens_in`` None: each sequence continues from its previous step's greedy
+    token.  ``concat`` true: the previous step's state h is projected and
+    appended to the cache tail before attending (the paper's default); false:
+    only true states are read and the previous state is discarded.
+    """
+    toks: List[int] = []
+    kv: List[Tuple[np.ndarray, np.ndarray]] = []
+    for b, seq in enumerate(seqs):
+        if tokens_in is None:
+            if seq.pending_token is None:
+                raise ValueError("no previous draft token for this sequence")
+            toks.append(int(seq.pending_token))
+        else:
+            toks.append(int(tokens_in[b]))
+        if seq.pending_h is not None and concat:
+            k, v = project_kv(head, seq.pending_h[None, :])
+            seq.k_draft.append(k[0])
+            seq.v_draft.append(v[0])
+        seq.pending_h = None
+        if seq.k_draft:
+            k_vis = np.concatenate([seq.k_true, np.stack(seq.k_draft)], axis=0)
+            v_vis = np.concatenate([seq.v_true, np.stack(seq.v_draft)], axis=0)
+        else:
+            k_vis, v_vis = seq.k_true, seq.v_true
+        kv.append((k_vis, v_vis))
+    out = draft_block(head, toks, kv)
+    for b, seq in enumerate(seqs):
+        seq.pending_h = out["h"][b].copy()
+        seq.pending_token = int(out["argmax"][b])
+    return out
+
+
+# --------------------------------------------------------------------------- block-attention forward
+
+def block_forward(head: OracleHead, tokens: Sequence[int], hidden: np.ndarray, block: int,
+                  offset: int, sim_steps: int = 1,
+                  positions: Optional[Iterable[int]] = None) -> Dict[str, np.ndarray]:
+    """Block-attention forward over one sequence of S tokens and S true states
+    (Section 4.2 and its mask figure).
+
+    Simulation step 1 is the early-stage inverse block mask: the query at
+    position p reads the true states 1..n, n = visible_true_count(p).  At
+    simulation step i > 1 the state predicted at step i-1 for window slot i-1
+    (position n+i-1) has been written into the key/value memory at that
+    position, and the queries of the same window with slot >= i are recomputed
+    with true states 1..n plus predicted states n+1..n+i-1.  No new queries are
+    made: every query is the data token's embedding.  The reported output of a
+    position is that of its last recomputation (step min(slot, sim_steps)).
+
+    ``positions``: optional subset of 1-based positions to report (their
+    window predecessors are computed as needed).  Returns arrays over the
+    reported positions in ascending order: 'positions', 'hidden', 'logits',
+    'argmax'.
+    """
+    c = head.cfg
+    tok = np.asarray(tokens, dtype=np.int64).reshape(-1)
+    S = tok.shape[0]
+    hid = np.asarray(hidden, dtype=F64).reshape(S, c.hidden)
+    if not (1 <= sim_steps <= block):
+        raise ValueError("sim_steps must be in [1, block]")
+    if not (0 <= offset < max(S, 1)):
+        raise ValueError("offset must be in [0, S)")
+    want = sorted(set(range(1, S + 1) if positions is None else (int(p) for p in positions)))
+    if want and (want[0] < 1 or want[-1] > S):
+        raise ValueError("position out of range")
+
+    def slot_of(p: int) -> int:
+        return p - visible_true_count(p, block, offset)   # 1 for p <= offset
+
+    # closure: a reported position needs the predicted states of the earlier slots of its window
+    need = set()
+    for p in want:
+        n, i = visible_true_count(p, block, offset), slot_of(p)
+        for r in range(1, min(i, sim_steps)):
+            need.add(n + r)
+        need.add(p)
+    active = sorted(need)
+
+    k_true, v_true = project_kv(head, hid)                       # K_j, V_j of every true state
+    k_pred: Dict[int, np.ndarray] = {}                           # position -> [Hkv, d_h]
+    v_pred: Dict[int, np.ndarray] = {}
+    result: Dict[int, Tuple[np.ndarray, np.ndarray, int]] = {}
+
+    for step in range(1, sim_steps + 1):
+        rows = [p for p in active if slot_of(p) >= step]
+        if not rows:
+            break
+        kv = []
+        for p in rows:
+            n = visible_true_count(p, block, offset)
+            ks = [k_true[:n]] + [k_pred[n + r][None] for r in range(1, step)]
+            vs = [v_true[:n]] + [v_pred[n + r][None] for r in range(1, step)]
+            kv.append((np.concatenate(ks, axis=0), np.concatenate(vs, axis=0)))
+        out = draft_block(head, tok[[p - 1 for p in rows]], kv)
+        for r, p in enumerate(rows):
+            result[p] = (out["h"][r], out["logits"][r], int(out["argmax"][r]))
+            if slot_of(p) == step and step < sim_steps:
+                k, v = project_kv(head, out["h"][r][None, :])    # saved predicted state
+                k_pred[p], v_pred[p] = k[0], v[0]
+
+    pos = np.asarray(want, dtype=np.int64)
+    return {
+        "positions": pos,
+        "hidden": np.stack([result[p][0] for p in want]) if want else np.zeros((0, c.hidden)),
+        "logits": np.stack([result[p][1] for p in want]) if want else np.zeros((0, c.vocab)),
+        "argmax": np.asarray([result[p][2] for p in want], dtype=np.int64),
+    }
+
+
+# --------------------------------------------------------------------------- greedy verification
+
+def verify_greedy(draft_tokens: np.ndarray, target_logits: Optional[np.ndarray] = None,
+                  target_ids: Optional[np.ndarray] = None) -> Tuple[np.ndarray, np.ndarray]:
+    """Greedy draft/verify acceptance (Section 3): with target top-1 tokens
+    g_1..g_{gamma+1} and drafts t_1..t_gamma, accept the longest prefix with
+    t_r == g_r; emit g_1..g_{a+1} (the accepted drafts equal the target's
+    tokens, plus the one extra target token).  Returns accept_len [B] and
+    out_tokens [B, gamma+1] padded with -1; tau = accept_len + 1.
+    """
+    draft = np.asarray(draft_tokens, dtype=np.int64)
+    B, gamma = draft.shape
+    if (target_logits is None) == (target_ids is None):
+        raise ValueError("give exactly one of target_logits / target_ids")
+    if target_ids is None:
+        g = argmax_lowest(np.asarray(target_logits, dtype=F64).reshape(B, gamma + 1, -1))
+    else:
+        g = np.asarray(target_ids, dtype=np.int64).reshape(B, gamma + 1)
+    accept = np.zeros(B, dtype=np.int64)
+    out = np.full((B, gamma + 1), -1, dtype=np.int64)
+    for b in range(B):
+        a = 0
+        while a < gamma and draft[b, a] == g[b, a]:
+            a += 1
+        accept[b] = a
+        out[b, : a + 1] = g[b, : a + 1]
+    return accept, out

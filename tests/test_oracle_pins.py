@@ -1,0 +1,439 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+None of these tests touches the CUDA library.  Each one names the passage it
+leans on; together they are chosen so that a dropped term, a wrong sign or
+index, or a transposed operand in the oracle fails at least one of them.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+
+import oracle as O
+from paper_2505_24544_b200 import workloads as WL
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def small_head(seed=0, d=32, hq=4, hkv=2, dh=8, m=48, V=50, std=0.3, **kw):
+    rng = np.random.default_rng(seed)
+    cfg = O.HeadConfig(d, hq, hkv, dh, m, V, **kw)
+    w = {
+        "embed": rng.normal(0, 1.0, (V, d)),
+        "g_q": 1 + rng.normal(0, 0.1, d),
+        "w_q": rng.normal(0, std, (hq * dh, d)),
+        "w_k": rng.normal(0, std, (hkv * dh, d)),
+        "w_v": rng.normal(0, std, (hkv * dh, d)),
+        "w_o": rng.normal(0, std, (d, hq * dh)),
+        "g_mlp": 1 + rng.normal(0, 0.1, d),
+        "w_gate": rng.normal(0, std, (m, d)),
+        "w_up": rng.normal(0, std, (m, d)),
+        "w_down": rng.normal(0, std, (d, m)),
+        "w_lm": rng.normal(0, std, (V, d)),
+    }
+    return O.OracleHead(cfg, w), w, rng
+
+
+# ----------------------------------------------------------------------------- hand-worked case
+
+def read_golden(name):
+    out = {}
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            key, *vals = line.split()
+            out[key] = np.array([float(v) for v in vals])
+    return out
+
+
+def tiny_head():
+    ln3, ln7, s2 = math.log(3.0), math.log(7.0), math.sqrt(2.0)
+    cfg = O.HeadConfig(hidden=2, n_q_heads=2, n_kv_heads=1, head_dim=2, mlp_dim=2, vocab=3, rms_eps=0.0)
+    w = {
+        "embed": [[1, 1], [1, -1], [s2, 0]],
+        "g_q": [2, 0.5],
+        "w_q": [[1, 4], [ln3 / (2 * s2), 0], [s2 * ln7 / 2, 0], [1, 4]],
+        "w_k": [[0, 1], [2, 0]],
+        "w_v": [[1, 2], [3, 4]],
+        "w_o": [[1, -1, 0, 0], [0, 0, -1, 1]],
+        "g_mlp": [0.5, 2],
+        "w_gate": [[0, ln3 / 2], [2 * ln3, 0]],
+        "w_up": [[2, 1], [4, 0]],
+        "w_down": [[1, 1], [2, -2]],
+        "w_lm": [[1, 0], [0, 1], [1, 1]],
+    }
+    return O.OracleHead(cfg, {k: np.array(v, dtype=float) for k, v in w.items()})
+
+
+def test_hand_worked_draft_step_matches_golden():
+    """Eq. 1-2 and the LM head on the pencil-and-paper instance (serve-time path)."""
+    g = read_golden("tiny_head.txt")
+    head = tiny_head()
+    seq = O.OracleSequence(head)
+    O.prefill_kv(head, seq, np.array([[1.0, 0.0], [0.0, 1.0]]))
+    out = O.draft_step(head, [seq], tokens_in=[1])
+    q = out["q"][0].reshape(2, 2)
+    w = O.attention_weights(head, q, seq.k_true)
+    np.testing.assert_allclose(w[0], g["attn_head1"], atol=1e-15)
+    np.testing.assert_allclose(w[1], g["attn_head2"], atol=1e-15)
+    np.testing.assert_allclose(out["o"][0], g["o"], atol=1e-14)
+    np.testing.assert_allclose(out["y"][0], g["y"], atol=1e-14)
+    np.testing.assert_allclose(out["h"][0], g["h"], atol=1e-14)
+    np.testing.assert_allclose(out["logits"][0], g["z"], atol=1e-14)
+    assert int(out["argmax"][0]) == int(g["argmax"][0])
+
+
+def test_hand_worked_block_forward_hides_diagonal():
+    """Same instance through the block path: the query at position 3 must not
+    read h_3 (Mask_{i,j} = 0 for j >= i, Section 4.1)."""
+    g = read_golden("tiny_head.txt")
+    head = tiny_head()
+    hidden = np.array([[1.0, 0.0], [0.0, 1.0], [5.0, 5.0]])
+    out = O.block_forward(head, tokens=[0, 2, 1], hidden=hidden, block=1, offset=0, sim_steps=1, positions=[3])
+    np.testing.assert_allclose(out["hidden"][0], g["h"], atol=1e-14)
+    np.testing.assert_allclose(out["logits"][0], g["z"], atol=1e-14)
+    assert int(out["argmax"][0]) == 2
+
+
+# ----------------------------------------------------------------------------- softmax invariants
+
+def test_attention_rows_sum_to_one_and_shift_invariance():
+    """Rows of s_{i,j} over the visible keys are probability vectors; adding
+    one vector to every key shifts every score of a head by the same amount and
+    so leaves the softmax unchanged (Eq. 2, second line)."""
+    head, _, rng = small_head(1)
+    c = head.cfg
+    q = rng.normal(0, 2.0, (c.n_q_heads, c.head_dim))
+    k = rng.normal(0, 2.0, (37, c.n_kv_heads, c.head_dim))
+    w = O.attention_weights(head, q, k)
+    assert w.shape == (c.n_q_heads, 37)
+    assert np.all(w >= 0)
+    np.testing.assert_allclose(w.sum(axis=1), 1.0, atol=1e-12)
+    shift = rng.normal(0, 3.0, (1, c.n_kv_heads, c.head_dim))
+    np.testing.assert_allclose(O.attention_weights(head, q, k + shift), w, atol=1e-12)
+    # the scale 1/sqrt(d_h): a single dominating score ratio, checked against the scalar formula
+    q1 = np.zeros_like(q); q1[0, 0] = 1.0
+    k2 = np.zeros((2, c.n_kv_heads, c.head_dim)); k2[0, 0, 0] = 3.0
+    w2 = O.attention_weights(head, q1, k2)
+    expect = 1.0 / (1.0 + math.exp(-3.0 / math.sqrt(c.head_dim)))
+    assert abs(w2[0, 0] - expect) < 1e-15
+
+
+def test_single_key_and_identical_keys():
+    """One visible key: o = V_1.  Identical keys: o = mean of the values."""
+    head, _, rng = small_head(2)
+    c = head.cfg
+    q = rng.normal(size=(c.n_q_heads, c.head_dim))
+    k = rng.normal(size=(1, c.n_kv_heads, c.head_dim))
+    v = rng.normal(size=(1, c.n_kv_heads, c.head_dim))
+    o = O.cross_attention(head, q, k, v).reshape(c.n_q_heads, c.head_dim)
+    for h in range(c.n_q_heads):
+        np.testing.assert_allclose(o[h], v[0, h // c.group], atol=1e-15)
+    k5 = np.repeat(k, 5, axis=0)
+    v5 = rng.normal(size=(5, c.n_kv_heads, c.head_dim))
+    o5 = O.cross_attention(head, q, k5, v5).reshape(c.n_q_heads, c.head_dim)
+    for h in range(c.n_q_heads):
+        np.testing.assert_allclose(o5[h], v5[:, h // c.group].mean(axis=0), atol=1e-14)
+
+
+def test_no_visible_key_gives_embedding_path_only():
+    """Position 1 has no key: o = 0, y = e(t)."""
+    head, w, rng = small_head(3)
+    seq = O.OracleSequence(head)
+    out = O.draft_step(head, [seq], tokens_in=[7])
+    np.testing.assert_array_equal(out["o"][0], 0.0)
+    np.testing.assert_allclose(out["y"][0], w["embed"][7], atol=0)
+
+
+def test_zero_output_projections_reduce_to_embedding_times_lm_head():
+    """W_O = 0 and W_down = 0 remove both sub-layers: z = W_lm e(t) (Eq. 1 residual paths)."""
+    head, w, rng = small_head(4)
+    w = dict(w); w["w_o"] = np.zeros_like(w["w_o"]); w["w_down"] = np.zeros_like(w["w_down"])
+    head0 = O.OracleHead(head.cfg, w)
+    seq = O.OracleSequence(head0)
+    O.prefill_kv(head0, seq, rng.normal(size=(9, head.cfg.hidden)))
+    out = O.draft_step(head0, [seq], tokens_in=[11])
+    np.testing.assert_allclose(out["logits"][0], w["w_lm"] @ w["embed"][11], atol=1e-13)
+
+
+def test_gqa_equals_mha_with_repeated_kv_heads():
+    """Grouped-query attention equals multi-head attention whose key/value
+    head weights are each repeated Hq/Hkv times."""
+    head, w, rng = small_head(5, hq=6, hkv=2, dh=4)
+    c = head.cfg
+    rep = lambda a: np.repeat(a.reshape(c.n_kv_heads, c.head_dim, c.hidden), c.group, axis=0).reshape(-1, c.hidden)
+    w_mha = dict(w); w_mha["w_k"] = rep(w["w_k"]); w_mha["w_v"] = rep(w["w_v"])
+    head_mha = O.OracleHead(O.HeadConfig(c.hidden, c.n_q_heads, c.n_q_heads, c.head_dim, c.mlp_dim, c.vocab), w_mha)
+    states = rng.normal(size=(13, c.hidden))
+    outs = []
+    for hd in (head, head_mha):
+        seq = O.OracleSequence(hd)
+        O.prefill_kv(hd, seq, states)
+        outs.append(O.draft_step(hd, [seq], tokens_in=[3]))
+    np.testing.assert_allclose(outs[0]["logits"], outs[1]["logits"], atol=1e-12)
+    np.testing.assert_allclose(outs[0]["o"], outs[1]["o"], atol=1e-13)
+
+
+def test_norm_flags_and_rmsnorm_definition():
+    """RMSNorm(v) has unit mean square when g = 1, eps = 0; flags switch it off."""
+    rng = np.random.default_rng(6)
+    v = rng.normal(size=(5, 17)) * 3.0
+    n = O.rms_norm(v, np.ones(17), 0.0)
+    np.testing.assert_allclose((n * n).mean(axis=1), 1.0, atol=1e-13)
+    np.testing.assert_allclose(n * np.sqrt((v * v).mean(axis=1, keepdims=True)), v, atol=1e-12)
+    # eps enters under the root: v = 0 stays 0 and a constant vector c gives c/sqrt(c^2+eps)
+    assert abs(O.rms_norm(np.full(4, 2.0), np.ones(4), 5.0)[0] - 2.0 / 3.0) < 1e-15
+    head, w, _ = small_head(7, norm_q=False, norm_mlp=False)
+    w1 = dict(w); w1["g_q"] = w["g_q"] * 9.0; w1["g_mlp"] = w["g_mlp"] * -2.0
+    a = O.draft_block(head, [1], [(np.zeros((0, 2, 8)), np.zeros((0, 2, 8)))])
+    b = O.draft_block(O.OracleHead(head.cfg, w1), [1], [(np.zeros((0, 2, 8)), np.zeros((0, 2, 8)))])
+    np.testing.assert_array_equal(a["logits"], b["logits"])
+
+
+def test_silu_values():
+    """SiLU(u) = u * sigmoid(u): SiLU(0) = 0, SiLU(ln 3) = 3/4 ln 3, SiLU(-ln 3) = -1/4 ln 3."""
+    l3 = math.log(3.0)
+    np.testing.assert_allclose(O.silu(np.array([0.0, l3, -l3])), [0.0, 0.75 * l3, -0.25 * l3], atol=1e-15)
+
+
+# ----------------------------------------------------------------------------- the mask
+
+def literal_visible_keys(S, block, offset):
+    """The mask built literally from the text: key j is visible to query i iff
+    j < i (Section 4.1) and not (i and j lie in the same window) (Section 4.2,
+    a window starting at n holds positions n+1..n+block; windows tile from
+    ``offset``)."""
+    def window(p):
+        return None if p <= offset else (p - 1 - offset) // block
+    vis = {}
+    for i in range(1, S + 1):
+        vis[i] = [j for j in range(1, S + 1)
+                  if j < i and not (window(i) is not None and window(i) == window(j))]
+    return vis
+
+
+def test_mask_brute_force():
+    for S in (1, 2, 7, 16):
+        for block in (1, 2, 3, 4, 5):
+            for offset in range(0, S):
+                vis = literal_visible_keys(S, block, offset)
+                for p in range(1, S + 1):
+                    n = O.visible_true_count(p, block, offset)
+                    assert vis[p] == list(range(1, n + 1)), (S, block, offset, p)
+
+
+def test_block_of_one_is_strict_causal():
+    for p in range(1, 20):
+        for offset in (0, 3, 11):
+            assert O.visible_true_count(p, 1, offset) == p - 1
+
+
+# ----------------------------------------------------------------------------- block forward == sequential drafting
+
+def sequential_reference(head, tokens, hidden, block, offset, sim_steps):
+    """Step-by-step serve-time drafting that the block forward has to reproduce
+    (the mask figure's caption: the unrolled states simulate inference): from
+    every window start n, prefill the n true states and draft the window's
+    tokens one at a time, feeding the DATA tokens."""
+    S = len(tokens)
+    hid_out = np.zeros((S, head.cfg.hidden)); logits = np.zeros((S, head.cfg.vocab))
+    p = 1
+    while p <= S:
+        n = O.visible_true_count(p, block, offset)
+        width = 1 if p <= offset else min(block, S - n)
+        seq = O.OracleSequence(head)
+        O.prefill_kv(head, seq, hidden[:n])
+        for i in range(1, width + 1):
+            out = O.draft_step(head, [seq], tokens_in=[tokens[n + i - 1]], concat=(i <= sim_steps))
+            hid_out[n + i - 1] = out["h"][0]; logits[n + i - 1] = out["logits"][0]
+        p = n + width + 1
+    return hid_out, logits
+
+
+@pytest.mark.parametrize("block,offset,sim_steps", [(4, 0, 1), (4, 0, 4), (4, 3, 1), (4, 3, 4), (3, 2, 2), (5, 1, 3), (1, 0, 1)])
+def test_block_forward_equals_sequential_drafting(block, offset, sim_steps):
+    head, _, rng = small_head(10 + block)
+    S = 19
+    tokens = rng.integers(0, head.cfg.vocab, S)
+    hidden = rng.normal(size=(S, head.cfg.hidden))
+    out = O.block_forward(head, tokens, hidden, block, offset, sim_steps)
+    ref_h, ref_z = sequential_reference(head, tokens, hidden, block, offset, sim_steps)
+    np.testing.assert_allclose(out["hidden"], ref_h, atol=1e-10)
+    np.testing.assert_allclose(out["logits"], ref_z, atol=1e-10)
+    # a subset of positions reports the same rows
+    sub = O.block_forward(head, tokens, hidden, block, offset, sim_steps, positions=[S, 6, 1])
+    np.testing.assert_allclose(sub["logits"], out["logits"][[0, 5, S - 1]], atol=1e-12)
+
+
+def test_simulation_changes_only_later_slots():
+    """Slot-1 queries never read a predicted state, so their outputs do not
+    depend on sim_steps; later slots do change."""
+    head, _, rng = small_head(21)
+    S, k = 16, 4
+    tokens = rng.integers(0, head.cfg.vocab, S); hidden = rng.normal(size=(S, head.cfg.hidden))
+    a = O.block_forward(head, tokens, hidden, k, 0, 1)["logits"]
+    b = O.block_forward(head, tokens, hidden, k, 0, k)["logits"]
+    np.testing.assert_allclose(a[0::k], b[0::k], atol=1e-12)
+    assert np.max(np.abs(a[5] - b[5])) > 1e-6      # slot 2 of window 2 reads a predicted state
+
+
+# ----------------------------------------------------------------------------- cache semantics
+
+def test_cache_reset_drops_draft_tail_and_order_is_irrelevant():
+    """The cache is reset to true states at the end of an iteration; with no
+    positional term the order of visible keys cannot matter (Eq. 2)."""
+    head, _, rng = small_head(30)
+    d = head.cfg.hidden
+    states = rng.normal(size=(10, d))
+    seq = O.OracleSequence(head)
+    O.prefill_kv(head, seq, states)
+    first = O.draft_step(head, [seq], tokens_in=[4])
+    O.draft_step(head, [seq])                     # continues from its own token, appends a draft state
+    assert seq.n_draft == 1
+    O.prefill_kv(head, seq, np.zeros((0, d)))     # reset only
+    assert seq.n_draft == 0 and seq.n_true == 10
+    again = O.draft_step(head, [seq], tokens_in=[4])
+    np.testing.assert_array_equal(first["logits"], again["logits"])
+    perm = rng.permutation(10)
+    seq2 = O.OracleSequence(head)
+    O.prefill_kv(head, seq2, states[perm])
+    other = O.draft_step(head, [seq2], tokens_in=[4])
+    np.testing.assert_allclose(other["logits"], first["logits"], atol=1e-12)
+
+
+def test_sequences_are_independent_and_chain_feeds_own_token():
+    head, _, rng = small_head(31)
+    d = head.cfg.hidden
+    sa, sb = rng.normal(size=(6, d)), rng.normal(size=(9, d))
+    seqs = [O.OracleSequence(head), O.OracleSequence(head)]
+    O.prefill_kv(head, seqs[0], sa); O.prefill_kv(head, seqs[1], sb)
+    both1 = O.draft_step(head, seqs, tokens_in=[1, 2])
+    both2 = O.draft_step(head, seqs)
+    alone = O.OracleSequence(head)
+    O.prefill_kv(head, alone, sb)
+    one1 = O.draft_step(head, [alone], tokens_in=[2])
+    one2 = O.draft_step(head, [alone], tokens_in=[int(one1["argmax"][0])])
+    np.testing.assert_allclose(both1["logits"][1], one1["logits"][0], atol=1e-12)
+    np.testing.assert_allclose(both2["logits"][1], one2["logits"][0], atol=1e-12)
+    # concat off ignores the draft's own state
+    seqs2 = [O.OracleSequence(head)]
+    O.prefill_kv(head, seqs2[0], sb)
+    O.draft_step(head, seqs2, tokens_in=[2], concat=False)
+    off2 = O.draft_step(head, seqs2, concat=False)
+    plain = O.OracleSequence(head); O.prefill_kv(head, plain, sb)
+    ref = O.draft_step(head, [plain], tokens_in=[int(one1["argmax"][0])])
+    np.testing.assert_allclose(off2["logits"], ref["logits"], atol=1e-12)
+    assert np.max(np.abs(off2["logits"] - one2["logits"])) > 1e-9
+
+
+# ----------------------------------------------------------------------------- verification
+
+def test_greedy_verify_is_lossless_and_bounded():
+    """Accepted drafts equal the target's top-1 tokens, one more target token is
+    always emitted, and 1 <= tau <= gamma + 1 (Section 3)."""
+    rng = np.random.default_rng(40)
+    B, gamma, V = 200, 6, 11
+    logits = rng.normal(size=(B, gamma + 1, V))
+    g = np.argmax(logits, axis=-1)
+    draft = np.where(rng.random((B, gamma)) < 0.6, g[:, :gamma], rng.integers(0, V, (B, gamma)))
+    acc, out = O.verify_greedy(draft, target_logits=logits)
+    acc2, out2 = O.verify_greedy(draft, target_ids=g)
+    np.testing.assert_array_equal(acc, acc2); np.testing.assert_array_equal(out, out2)
+    for b in range(B):
+        a = int(acc[b])
+        assert 0 <= a <= gamma
+        np.testing.assert_array_equal(out[b, : a + 1], g[b, : a + 1])
+        assert np.all(out[b, a + 1:] == -1)
+        np.testing.assert_array_equal(draft[b, :a], g[b, :a])
+        if a < gamma:
+            assert draft[b, a] != g[b, a]
+    # the extremes
+    acc, out = O.verify_greedy(g[:, :gamma], target_ids=g)
+    assert np.all(acc == gamma) and np.all(out == g)
+    acc, out = O.verify_greedy((g[:, :gamma] + 1) % V, target_ids=g)
+    assert np.all(acc == 0) and np.all(out[:, 0] == g[:, 0]) and np.all(out[:, 1:] == -1)
+
+
+def test_argmax_ties_and_nan():
+    z = np.array([[1.0, 3.0, 3.0, 2.0], [np.nan, -5.0, np.nan, -7.0], [np.nan] * 4])
+    np.testing.assert_array_equal(O.argmax_lowest(z), [1, 1, 0])
+
+
+@pytest.mark.parametrize("gamma,expect", [(8, 3.1988), (6, 3.0588)])
+def test_expected_tau_matches_tail_sum_closed_form(gamma, expect):
+    """Appendix tail-sum: E[L] = sum_i prod_{j<=i} alpha^(j).  With a constant
+    rate alpha the iteration emits E[tau] = 1 + sum_{i=1}^{gamma} alpha^i tokens."""
+    alpha = 0.7
+    closed = 1.0 + sum(alpha ** i for i in range(1, gamma + 1))
+    assert abs(closed - expect) < 5e-5
+    w = WL.WORKLOADS["c3_llama3_8b_b1"].scaled(batch=200_000, gamma=gamma)
+    rng = np.random.default_rng(41)
+    draft = rng.integers(0, w.vocab, (w.batch, gamma))
+    target = WL.make_target_stream(w, rng, draft)
+    acc, _ = O.verify_greedy(draft, target_ids=target)
+    tau = acc + 1
+    sigma = tau.std() / math.sqrt(w.batch)
+    assert abs(tau.mean() - closed) < 3.5 * sigma
+
+
+# ----------------------------------------------------------------------------- library cross-check
+
+def test_against_torch_library_routines():
+    """The block reduces to library routines: F.linear, F.rms_norm-free formula,
+    scaled_dot_product_attention with a boolean mask, F.silu."""
+    torch = pytest.importorskip("torch")
+    F = torch.nn.functional
+    head, w, rng = small_head(50, d=48, hq=6, hkv=3, dh=8, m=40, V=31)
+    c = head.cfg
+    S, k, offset = 13, 3, 2
+    tokens = rng.integers(0, c.vocab, S); hidden = rng.normal(size=(S, c.hidden))
+    ours = O.block_forward(head, tokens, hidden, k, offset, 1)
+    T = {n: torch.tensor(np.asarray(v), dtype=torch.float64) for n, v in w.items()}
+    x = T["embed"][torch.tensor(tokens)]
+    rms = lambda v, g: v * torch.rsqrt(v.pow(2).mean(-1, keepdim=True) + c.rms_eps) * g
+    q = F.linear(rms(x, T["g_q"]), T["w_q"]).view(S, c.n_q_heads, c.head_dim).transpose(0, 1)
+    hs = torch.tensor(hidden)
+    kk = F.linear(hs, T["w_k"]).view(S, c.n_kv_heads, c.head_dim).transpose(0, 1).repeat_interleave(c.group, 0)
+    vv = F.linear(hs, T["w_v"]).view(S, c.n_kv_heads, c.head_dim).transpose(0, 1).repeat_interleave(c.group, 0)
+    mask = torch.zeros(S, S, dtype=torch.bool)
+    vis = literal_visible_keys(S, k, offset)
+    for i in range(1, S + 1):
+        for j in vis[i]:
+            mask[i - 1, j - 1] = True
+    keep = mask.any(-1)
+    mask_safe = mask.clone(); mask_safe[~keep, 0] = True           # SDPA needs a non-empty row
+    o = F.scaled_dot_product_attention(q[None], kk[None], vv[None], attn_mask=mask_safe[None, None])[0]
+    o = o.transpose(0, 1).reshape(S, -1) * keep[:, None]
+    y = F.linear(o, T["w_o"]) + x
+    yn = rms(y, T["g_mlp"])
+    h = F.linear(F.silu(F.linear(yn, T["w_gate"])) * F.linear(yn, T["w_up"]), T["w_down"]) + y
+    z = F.linear(h, T["w_lm"])
+    np.testing.assert_allclose(ours["hidden"], h.numpy(), atol=1e-11)
+    np.testing.assert_allclose(ours["logits"], z.numpy(), atol=1e-11)
+    np.testing.assert_array_equal(ours["argmax"], z.argmax(-1).numpy())
+
+
+# ----------------------------------------------------------------------------- generators
+
+def test_bf16_rounding_of_generator_matches_torch():
+    torch = pytest.importorskip("torch")
+    rng = np.random.default_rng(60)
+    a = rng.normal(size=10000).astype(np.float32) * 3
+    a[:4] = [1.00390625, 1.01171875, -1.00390625, 0.0]      # exact halves round to even
+    r = WL.round_to_storage(a, "bf16")
+    t = torch.from_numpy(a).to(torch.bfloat16).to(torch.float32).numpy()
+    np.testing.assert_array_equal(r, t)
+    np.testing.assert_array_equal(WL.round_to_storage(a, "fp32"), a)
+
+
+def test_workload_shapes_and_determinism():
+    w = WL.WORKLOADS["c1_tiny_fp32"]
+    a, b = WL.make_weights(w), WL.make_weights(w)
+    for k in a:
+        np.testing.assert_array_equal(a[k], b[k])
+    assert a["w_gate"].shape == (688, 256) and a["w_lm"].shape == (1024, 256)
+    w4 = WL.WORKLOADS["c4_llama3_8b_b32"]
+    n = WL.make_context_lengths(w4, WL.data_rng(w4))
+    assert n.shape == (32,) and n.min() >= 512 and n.max() <= 8192
