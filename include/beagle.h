@@ -1,0 +1,167 @@
+/*
+ * beagle.h -- C ABI of the B200 (sm_100a) forward pass of the Beagle cross-attention draft head.
+ *
+ * The head is one Transformer block whose queries come from token embeddings and whose keys and
+ * values come from higher-level states: the target model's top hidden states ("true states") or
+ * the head's own outputs (Section 4.1, Eq. 1 and Eq. 2 of the paper), followed by a linear LM head
+ * and greedy draft/verify acceptance (Section 3).  For one query at position p reading the visible
+ * state set Vis(p):
+ *
+ *     x  = E[t_p]                                   embedding
+ *     Q  = W_q RMSNorm(x; g_q)                      per head h: rows [h*dh, (h+1)*dh)
+ *     K_j, V_j = W_k s_j, W_v s_j                   s_j in Vis(p); head h reads K/V head h / (Hq/Hkv)
+ *     o_h = sum_j softmax_j(<Q_h, K_j>/sqrt(dh)) V_j    (softmax over Vis(p) only; Vis empty: o = 0)
+ *     y  = W_o [o_1 .. o_Hq] + x
+ *     h  = y + W_down( SiLU(W_gate n) * (W_up n) ),  n = RMSNorm(y; g_mlp)
+ *     z  = W_lm h,   t^ = argmax z  (lowest index on ties, NaN never wins)
+ *
+ * Conventions
+ *   - Every pointer named "dev" is DEVICE memory owned by the caller; "host" is host memory.  The
+ *     library allocates no device memory and creates no stream: the caller passes the key/value
+ *     cache, a workspace (sizes from beagle_query_sizes / beagle_block_workspace_bytes) and a
+ *     cudaStream_t (as void*; NULL = the legacy default stream).
+ *   - dtype 0 = fp32, 1 = bf16 is the storage type of weights, states, cache and hidden outputs;
+ *     accumulation, softmax and logits are fp32.  Weights are row-major [out, in].
+ *   - Calls only enqueue work on the stream and return; they never synchronise.  Argument, shape,
+ *     capacity and state errors are detected on the host before anything is launched and leave
+ *     the context unchanged.  No call aborts, throws or traps.
+ *   - A context is not thread-safe; use one per stream.
+ */
+#ifndef BEAGLE_H
+#define BEAGLE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct beagle_ctx beagle_ctx;
+
+typedef enum beagle_status {
+    BEAGLE_OK = 0,
+    BEAGLE_ERR_INVALID_ARG = 1,   /* NULL pointer, negative size, unknown flag                     */
+    BEAGLE_ERR_SHAPE = 2,         /* a dimension the kernels do not support (see beagle_config)   */
+    BEAGLE_ERR_CAPACITY = 3,      /* cache, workspace, batch or draft depth exceeded              */
+    BEAGLE_ERR_STATE = 4,         /* call order: e.g. tokens_in == NULL with no previous step     */
+    BEAGLE_ERR_UNSUPPORTED = 5,
+    BEAGLE_ERR_CUDA = 6           /* a CUDA runtime call failed; see beagle_last_error            */
+} beagle_status;
+
+enum { BEAGLE_FP32 = 0, BEAGLE_BF16 = 1 };
+
+/* Largest `batch` of one beagle_prefill_kv / beagle_draft_step / beagle_verify_greedy call. */
+#define BEAGLE_MAX_CALL_BATCH 64
+
+typedef struct beagle_config {
+    int32_t hidden;       /* d; multiple of 8                                                      */
+    int32_t n_q_heads;    /* Hq                                                                    */
+    int32_t n_kv_heads;   /* Hkv; Hq % Hkv == 0, Hq/Hkv in {1,2,4,8}                                */
+    int32_t head_dim;     /* dh; bf16: 32|64|128|256, fp32: 16|32|64|128                            */
+    int32_t mlp_dim;      /* m; multiple of 8                                                      */
+    int32_t vocab;        /* V                                                                     */
+    int32_t dtype;        /* BEAGLE_FP32 | BEAGLE_BF16                                             */
+    float   rms_eps;
+    int32_t norm_q;       /* 1: RMSNorm(g_q) on the query input, 0: none                           */
+    int32_t norm_mlp;     /* 1: RMSNorm(g_mlp) on the MLP input, 0: none                           */
+    int32_t max_slots;    /* sequences the cache holds                                             */
+    int32_t max_ctx;      /* true states per sequence                                              */
+    int32_t max_draft;    /* draft states appended per sequence between two resets                 */
+} beagle_config;
+
+/* Device pointers, row-major [out, in], BORROWED: they must outlive the context. */
+typedef struct beagle_weights {
+    const void* embed;    /* [V, d]            */
+    const void* g_q;      /* [d]               */
+    const void* w_q;      /* [Hq*dh, d]        */
+    const void* w_k;      /* [Hkv*dh, d]       */
+    const void* w_v;      /* [Hkv*dh, d]       */
+    const void* w_o;      /* [d, Hq*dh]        */
+    const void* g_mlp;    /* [d]               */
+    const void* w_gate;   /* [m, d]            */
+    const void* w_up;     /* [m, d]            */
+    const void* w_down;   /* [d, m]            */
+    const void* w_lm;     /* [V, d]            */
+} beagle_weights;
+
+/* Bytes of the key/value cache ([2][max_slots][Hkv][max_ctx+max_draft][dh] in the storage type)
+ * and of the serve-time workspace.  Both buffers must be 256-byte aligned. */
+beagle_status beagle_query_sizes(const beagle_config* cfg, size_t* kv_bytes, size_t* workspace_bytes);
+
+/* Creates the host-side bookkeeping (lengths of every slot start at zero).  kv_dev and
+ * workspace_dev stay owned by the caller and must outlive the context; their contents need not be
+ * initialised. */
+beagle_status beagle_create(const beagle_config* cfg, const beagle_weights* weights_dev,
+                            void* kv_dev, size_t kv_bytes, void* workspace_dev, size_t workspace_bytes,
+                            beagle_ctx** out);
+beagle_status beagle_destroy(beagle_ctx* ctx);
+
+/* Key/value projection and cache append over TRUE states (Eq. 2 first line; Section 4.1, cache
+ * paragraph: "reset the cache to true states at the end of the iteration").  For each b < batch:
+ * the draft tail of slot seq_slot[b] is dropped, then new_len[b] rows of `hidden_dev` are projected
+ * with W_k, W_v and appended.  hidden_dev is packed row-major [sum(new_len), d] in the storage type,
+ * sequences in call order.  seq_slot and new_len are HOST arrays; slots must be distinct.
+ * new_len[b] == 0 only resets.  CAPACITY if a slot would exceed max_ctx. */
+beagle_status beagle_prefill_kv(beagle_ctx* ctx, int32_t batch, const int32_t* seq_slot_host,
+                                const int32_t* new_len_host, const void* hidden_dev, void* stream);
+
+/* One drafted token for each of `batch` sequences (Eq. 1, Eq. 2, LM head, greedy token).
+ * tokens_in_dev: int32 [batch] query tokens, or NULL to continue from each slot's previous greedy
+ *   token (STATE error if a slot has none since its last reset).
+ * concat != 0: the previous step's output state h of the slot is projected and appended to the
+ *   cache tail before attending (the paper's default, "concate"); 0: only states already in the
+ *   cache are read and the previous state is discarded.
+ * Outputs (any may be NULL): tokens_out_dev int32 [batch]; logits_out_dev fp32 [batch, V];
+ *   hidden_out_dev storage type [batch, d]. */
+beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* seq_slot_host,
+                                const int32_t* tokens_in_dev, int32_t concat,
+                                int32_t* tokens_out_dev, float* logits_out_dev, void* hidden_out_dev,
+                                void* stream);
+
+/* Drops the draft tail of the listed slots (cache back to true states only). */
+beagle_status beagle_rollback(beagle_ctx* ctx, int32_t batch, const int32_t* seq_slot_host);
+/* Forgets a slot entirely (length zero). */
+beagle_status beagle_reset_slot(beagle_ctx* ctx, int32_t slot);
+/* Current number of true / draft states of a slot (host bookkeeping). */
+beagle_status beagle_slot_lengths(const beagle_ctx* ctx, int32_t slot, int32_t* n_true, int32_t* n_draft);
+
+/* Workspace bytes of beagle_block_forward for `batch` sequences of S positions. */
+beagle_status beagle_block_workspace_bytes(const beagle_config* cfg, int32_t batch, int32_t S, size_t* bytes);
+
+/* Stateless block-attention forward (Section 4.2 and its mask figure): S data tokens and S true
+ * states per sequence.  With n(p) = p-1 for p <= offset, else offset + block*floor((p-1-offset)/block),
+ * the query at 1-based position p reads true states 1..n(p) (inverse block mask: keys of its own
+ * window are hidden, and Mask_{i,j} = 0 for j >= i).  sim_steps in [1, block]: at simulation step
+ * i > 1 the state predicted for window slot i-1 is written in place as the key/value of its
+ * position and becomes visible to the later queries of that window, so position p = n+i finally
+ * reads true 1..n plus predicted n+1..n+min(i,sim_steps)-1.  Queries are always the data tokens.
+ * tokens_dev int32 [batch,S]; hidden_dev storage [batch,S,d]; outputs (nullable): logits fp32
+ * [batch,S,V], argmax int32 [batch,S], hidden storage [batch,S,d].  ws_dev: 256-byte aligned. */
+beagle_status beagle_block_forward(beagle_ctx* ctx, int32_t batch, int32_t S, const int32_t* tokens_dev,
+                                   const void* hidden_dev, int32_t block, int32_t offset, int32_t sim_steps,
+                                   float* logits_out_dev, int32_t* argmax_out_dev, void* hidden_out_dev,
+                                   void* ws_dev, size_t ws_bytes, void* stream);
+
+/* Greedy acceptance (Section 3: in greedy decoding the draft's and the target's top-1 tokens are
+ * matched and only a contiguous prefix is accepted, plus one extra target token).  Exactly one of
+ * target_logits_dev ([batch, gamma+1, V], logits_dtype BEAGLE_FP32 or BEAGLE_BF16) and
+ * target_ids_dev (int32 [batch, gamma+1]) is non-NULL.  accept_len_dev[b] = a = number of leading
+ * drafts equal to the target's top-1; out_tokens_dev[b] = g_1..g_{a+1} then -1 padding
+ * ([batch, gamma+1]); tau = a + 1.  draft_tokens_dev int32 [batch, gamma]; gamma <= 64. */
+beagle_status beagle_verify_greedy(beagle_ctx* ctx, int32_t batch, int32_t gamma,
+                                   const int32_t* draft_tokens_dev, const void* target_logits_dev,
+                                   int32_t logits_dtype, const int32_t* target_ids_dev,
+                                   int32_t* accept_len_dev, int32_t* out_tokens_dev, void* stream);
+
+/* Text of the last error recorded on this context ("" if none). */
+const char* beagle_last_error(const beagle_ctx* ctx);
+/* Number of kernels this context has launched so far. */
+int64_t beagle_launch_count(const beagle_ctx* ctx);
+/* Library version string. */
+const char* beagle_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BEAGLE_H */

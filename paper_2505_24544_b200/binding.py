@@ -1,0 +1,282 @@
+"""Thin ctypes binding of libbeagle.so (include/beagle.h).
+
+Argument marshalling only: every step of the draft head runs in the CUDA
+kernels behind the C ABI.  PyTorch supplies device memory (tensors) and the
+current CUDA stream; nothing here computes.  Importing this module fails loudly
+when the shared library has not been built -- there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional, Sequence, Tuple
+
+import torch
+
+from . import build as _build
+
+BEAGLE_FP32, BEAGLE_BF16 = 0, 1
+BEAGLE_MAX_CALL_BATCH = 64
+STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "CAPACITY", 4: "STATE", 5: "UNSUPPORTED", 6: "CUDA"}
+
+WEIGHT_NAMES = ("embed", "g_q", "w_q", "w_k", "w_v", "w_o", "g_mlp", "w_gate", "w_up", "w_down", "w_lm")
+
+EXPORTED_SYMBOLS = (
+    "beagle_version", "beagle_query_sizes", "beagle_create", "beagle_destroy", "beagle_prefill_kv",
+    "beagle_draft_step", "beagle_rollback", "beagle_reset_slot", "beagle_slot_lengths",
+    "beagle_block_workspace_bytes", "beagle_block_forward", "beagle_verify_greedy", "beagle_last_error",
+    "beagle_launch_count",
+)
+
+
+class BeagleConfig(C.Structure):
+    _fields_ = [
+        ("hidden", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
+        ("mlp_dim", C.c_int32), ("vocab", C.c_int32), ("dtype", C.c_int32), ("rms_eps", C.c_float),
+        ("norm_q", C.c_int32), ("norm_mlp", C.c_int32), ("max_slots", C.c_int32), ("max_ctx", C.c_int32),
+        ("max_draft", C.c_int32),
+    ]
+
+
+class BeagleWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in WEIGHT_NAMES]
+
+
+class BeagleError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"beagle status {status} ({STATUS_NAMES.get(status, '?')}): {message}")
+        self.status = status
+
+
+_lib: Optional[C.CDLL] = None
+
+
+def load_library(path: Optional[str] = None) -> C.CDLL:
+    """Loads libbeagle.so (built in-tree by ``build.build()``); raises if it is missing."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or _build.LIB_PATH
+    if not os.path.exists(p):
+        raise ImportError(f"{p} not found: run `python -m paper_2505_24544_b200.build` (there is no fallback path)")
+    lib = C.CDLL(p)
+    vp, i32, i32p, szp = C.c_void_p, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_size_t)
+    lib.beagle_version.restype = C.c_char_p
+    lib.beagle_version.argtypes = []
+    lib.beagle_query_sizes.argtypes = [C.POINTER(BeagleConfig), szp, szp]
+    lib.beagle_create.argtypes = [C.POINTER(BeagleConfig), C.POINTER(BeagleWeights), vp, C.c_size_t, vp, C.c_size_t, C.POINTER(vp)]
+    lib.beagle_destroy.argtypes = [vp]
+    lib.beagle_prefill_kv.argtypes = [vp, i32, i32p, i32p, vp, vp]
+    lib.beagle_draft_step.argtypes = [vp, i32, i32p, vp, i32, vp, vp, vp, vp]
+    lib.beagle_rollback.argtypes = [vp, i32, i32p]
+    lib.beagle_reset_slot.argtypes = [vp, i32]
+    lib.beagle_slot_lengths.argtypes = [vp, i32, i32p, i32p]
+    lib.beagle_block_workspace_bytes.argtypes = [C.POINTER(BeagleConfig), i32, i32, szp]
+    lib.beagle_block_forward.argtypes = [vp, i32, i32, vp, vp, i32, i32, i32, vp, vp, vp, vp, C.c_size_t, vp]
+    lib.beagle_verify_greedy.argtypes = [vp, i32, i32, vp, vp, i32, vp, vp, vp, vp]
+    lib.beagle_last_error.restype = C.c_char_p
+    lib.beagle_last_error.argtypes = [vp]
+    lib.beagle_launch_count.restype = C.c_int64
+    lib.beagle_launch_count.argtypes = [vp]
+    for name in ("beagle_query_sizes", "beagle_create", "beagle_destroy", "beagle_prefill_kv", "beagle_draft_step",
+                 "beagle_rollback", "beagle_reset_slot", "beagle_slot_lengths", "beagle_block_workspace_bytes",
+                 "beagle_block_forward", "beagle_verify_greedy"):
+        getattr(lib, name).restype = C.c_int
+    if path is None:
+        _lib = lib
+    return lib
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    return t.data_ptr()
+
+
+def _i32_array(values: Sequence[int]):
+    arr = (C.c_int32 * max(1, len(values)))(*[int(v) for v in values])
+    return arr
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def torch_dtype(dtype_code: int) -> torch.dtype:
+    return torch.bfloat16 if dtype_code == BEAGLE_BF16 else torch.float32
+
+
+class Context:
+    """Owns the device buffers (as torch tensors) that the C context borrows, and the opaque handle."""
+
+    def __init__(self, cfg: BeagleConfig, weights: Dict[str, torch.Tensor]):
+        self.lib = load_library()
+        self.cfg = cfg
+        dt = torch_dtype(cfg.dtype)
+        self.weights = {}
+        w = BeagleWeights()
+        for n in WEIGHT_NAMES:
+            t = weights[n]
+            if t.dtype != dt or not t.is_cuda or not t.is_contiguous():
+                raise ValueError(f"weight {n}: expected contiguous {dt} CUDA tensor")
+            self.weights[n] = t
+            setattr(w, n, t.data_ptr())
+        kv, ws = C.c_size_t(), C.c_size_t()
+        st = self.lib.beagle_query_sizes(C.byref(cfg), C.byref(kv), C.byref(ws))
+        if st != 0:
+            raise BeagleError(st, "beagle_query_sizes rejected the configuration")
+        dev = next(iter(self.weights.values())).device
+        self.kv_buf = torch.empty(kv.value, dtype=torch.uint8, device=dev)
+        self.ws_buf = torch.empty(ws.value, dtype=torch.uint8, device=dev)
+        self.block_ws: Optional[torch.Tensor] = None
+        handle = C.c_void_p()
+        st = self.lib.beagle_create(C.byref(cfg), C.byref(w), self.kv_buf.data_ptr(), kv.value, self.ws_buf.data_ptr(),
+                                    ws.value, C.byref(handle))
+        if st != 0:
+            raise BeagleError(st, "beagle_create failed")
+        self.handle = handle
+
+    def check(self, st: int) -> None:
+        if st != 0:
+            raise BeagleError(st, self.lib.beagle_last_error(self.handle).decode())
+
+    def close(self) -> None:
+        if getattr(self, "handle", None):
+            self.lib.beagle_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def launch_count(self) -> int:
+        return int(self.lib.beagle_launch_count(self.handle))
+
+
+# ---- entry points, named as in include/beagle.h -----------------------------------------------
+
+def beagle_prefill_kv(ctx: Context, seq_slot: Sequence[int], new_len: Sequence[int], hidden: Optional[torch.Tensor]) -> None:
+    ctx.check(ctx.lib.beagle_prefill_kv(ctx.handle, len(seq_slot), _i32_array(seq_slot), _i32_array(new_len),
+                                        _ptr(hidden), _stream()))
+
+
+def beagle_draft_step(ctx: Context, seq_slot: Sequence[int], tokens_in: Optional[torch.Tensor], concat: bool,
+                      tokens_out: Optional[torch.Tensor], logits_out: Optional[torch.Tensor] = None,
+                      hidden_out: Optional[torch.Tensor] = None) -> None:
+    ctx.check(ctx.lib.beagle_draft_step(ctx.handle, len(seq_slot), _i32_array(seq_slot), _ptr(tokens_in), int(bool(concat)),
+                                        _ptr(tokens_out), _ptr(logits_out), _ptr(hidden_out), _stream()))
+
+
+def beagle_rollback(ctx: Context, seq_slot: Sequence[int]) -> None:
+    ctx.check(ctx.lib.beagle_rollback(ctx.handle, len(seq_slot), _i32_array(seq_slot)))
+
+
+def beagle_reset_slot(ctx: Context, slot: int) -> None:
+    ctx.check(ctx.lib.beagle_reset_slot(ctx.handle, int(slot)))
+
+
+def beagle_slot_lengths(ctx: Context, slot: int) -> Tuple[int, int]:
+    a, b = C.c_int32(), C.c_int32()
+    ctx.check(ctx.lib.beagle_slot_lengths(ctx.handle, int(slot), C.byref(a), C.byref(b)))
+    return a.value, b.value
+
+
+def beagle_block_workspace_bytes(ctx: Context, batch: int, S: int) -> int:
+    n = C.c_size_t()
+    st = ctx.lib.beagle_block_workspace_bytes(C.byref(ctx.cfg), batch, S, C.byref(n))
+    if st != 0:
+        raise BeagleError(st, "beagle_block_workspace_bytes")
+    return n.value
+
+
+def beagle_block_forward(ctx: Context, tokens: torch.Tensor, hidden: torch.Tensor, block: int, offset: int,
+                         sim_steps: int, logits_out: Optional[torch.Tensor], argmax_out: Optional[torch.Tensor],
+                         hidden_out: Optional[torch.Tensor]) -> None:
+    batch, S = tokens.shape
+    need = beagle_block_workspace_bytes(ctx, batch, S)
+    if ctx.block_ws is None or ctx.block_ws.numel() < need:
+        ctx.block_ws = None
+        ctx.block_ws = torch.empty(need, dtype=torch.uint8, device=tokens.device)
+    ctx.check(ctx.lib.beagle_block_forward(ctx.handle, batch, S, _ptr(tokens), _ptr(hidden), block, offset, sim_steps,
+                                           _ptr(logits_out), _ptr(argmax_out), _ptr(hidden_out),
+                                           ctx.block_ws.data_ptr(), ctx.block_ws.numel(), _stream()))
+
+
+def beagle_verify_greedy(ctx: Context, draft_tokens: torch.Tensor, target_logits: Optional[torch.Tensor],
+                         target_ids: Optional[torch.Tensor], accept_len: torch.Tensor, out_tokens: torch.Tensor) -> None:
+    batch, gamma = draft_tokens.shape
+    code = BEAGLE_FP32
+    if target_logits is not None:
+        if target_logits.dtype == torch.bfloat16:
+            code = BEAGLE_BF16
+        elif target_logits.dtype != torch.float32:
+            raise ValueError("target_logits must be float32 or bfloat16")
+    ctx.check(ctx.lib.beagle_verify_greedy(ctx.handle, batch, gamma, _ptr(draft_tokens), _ptr(target_logits), code,
+                                           _ptr(target_ids), _ptr(accept_len), _ptr(out_tokens), _stream()))
+
+
+# ---- convenience wrapper -----------------------------------------------------------------------
+
+class BeagleHead:
+    """A draft head on one GPU: allocates outputs and forwards to the entry points above."""
+
+    def __init__(self, *, hidden: int, n_q_heads: int, n_kv_heads: int, head_dim: int, mlp_dim: int, vocab: int,
+                 dtype: str, weights: Dict[str, torch.Tensor], max_slots: int, max_ctx: int, max_draft: int,
+                 rms_eps: float = 1e-5, norm_q: bool = True, norm_mlp: bool = True):
+        code = {"fp32": BEAGLE_FP32, "bf16": BEAGLE_BF16}[dtype]
+        self.cfg = BeagleConfig(hidden, n_q_heads, n_kv_heads, head_dim, mlp_dim, vocab, code, rms_eps, int(norm_q),
+                                int(norm_mlp), max_slots, max_ctx, max_draft)
+        self.ctx = Context(self.cfg, weights)
+        self.device = self.ctx.kv_buf.device
+        self.dtype = torch_dtype(code)
+
+    @classmethod
+    def from_workload(cls, w, weights_np, device="cuda", max_slots=None, max_ctx=None, max_draft=None) -> "BeagleHead":
+        """Uploads numpy float32 weights (already rounded to the storage type) and builds the head."""
+        dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+        weights = {k: torch.from_numpy(v).to(device=device, dtype=dt).contiguous() for k, v in weights_np.items()}
+        return cls(hidden=w.hidden, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads, head_dim=w.head_dim,
+                   mlp_dim=w.mlp_dim, vocab=w.vocab, dtype=w.dtype, weights=weights,
+                   max_slots=max_slots or w.batch, max_ctx=max_ctx or (w.ctx_max + 64),
+                   max_draft=max_draft or max(w.gamma, 1), rms_eps=w.rms_eps)
+
+    def prefill_kv(self, seq_slot, new_len, hidden):
+        beagle_prefill_kv(self.ctx, seq_slot, new_len, hidden)
+
+    def rollback(self, seq_slot):
+        beagle_rollback(self.ctx, seq_slot)
+
+    def draft_step(self, seq_slot, tokens_in=None, concat=True, want_logits=False, want_hidden=False):
+        B = len(seq_slot)
+        tokens_out = torch.empty(B, dtype=torch.int32, device=self.device)
+        logits = torch.empty(B, self.cfg.vocab, dtype=torch.float32, device=self.device) if want_logits else None
+        hidden = torch.empty(B, self.cfg.hidden, dtype=self.dtype, device=self.device) if want_hidden else None
+        beagle_draft_step(self.ctx, seq_slot, tokens_in, concat, tokens_out, logits, hidden)
+        return tokens_out, logits, hidden
+
+    def block_forward(self, tokens, hidden, block, offset=0, sim_steps=1, want_logits=True, want_hidden=True):
+        B, S = tokens.shape
+        logits = torch.empty(B, S, self.cfg.vocab, dtype=torch.float32, device=self.device) if want_logits else None
+        argmax = torch.empty(B, S, dtype=torch.int32, device=self.device)
+        hid = torch.empty(B, S, self.cfg.hidden, dtype=self.dtype, device=self.device) if want_hidden else None
+        beagle_block_forward(self.ctx, tokens, hidden, block, offset, sim_steps, logits, argmax, hid)
+        return logits, argmax, hid
+
+    def verify_greedy(self, draft_tokens, target_logits=None, target_ids=None):
+        B, gamma = draft_tokens.shape
+        accept = torch.empty(B, dtype=torch.int32, device=self.device)
+        out = torch.empty(B, gamma + 1, dtype=torch.int32, device=self.device)
+        beagle_verify_greedy(self.ctx, draft_tokens, target_logits, target_ids, accept, out)
+        return accept, out
+
+    def slot_lengths(self, slot):
+        return beagle_slot_lengths(self.ctx, slot)
+
+    @property
+    def launch_count(self) -> int:
+        return self.ctx.launch_count

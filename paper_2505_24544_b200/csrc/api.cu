@@ -1,0 +1,578 @@
+// C ABI of the Beagle draft-head library: host-side validation, cache bookkeeping and the launch
+// sequence of every entry point.  No device memory is allocated and no stream is created here.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "../../include/beagle.h"
+#include "kernels.h"
+#include "gemm_tc.h"
+
+using namespace beagle;
+
+struct beagle_ctx {
+    beagle_config cfg;
+    beagle_weights w;
+    char* kv = nullptr;
+    char* ws = nullptr;
+    size_t kv_bytes = 0, ws_bytes = 0;
+    int cap = 0;            // rows per (slot, head) of the cache
+    size_t elt = 0;         // bytes per stored element
+    int qd = 0, kd = 0;
+    // cache halves
+    void* kcache = nullptr;
+    void* vcache = nullptr;
+    // serve-time workspace regions
+    void *x, *xn, *q, *o, *y, *yn, *act, *h, *h_slot, *attn_scratch;
+    int32_t *last_token, *ids;
+    unsigned long long *lm_partials, *verify_keys;
+    int lm_blocks = 0;
+    // host bookkeeping
+    std::vector<int32_t> n_true, n_draft;
+    std::vector<char> pending;      // slot has an output state not yet appended
+    std::vector<char> has_token;    // slot has a previous greedy token
+    std::string err;
+    int64_t launches = 0;
+    TcPlan* tc = nullptr;           // tensor-core GEMM plans (bf16 only)
+};
+
+namespace {
+
+constexpr size_t kAlign = 256;
+size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+
+beagle_status fail(beagle_ctx* ctx, beagle_status st, const char* fmt, ...) {
+    if (ctx != nullptr) {
+        char buf[512];
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(buf, sizeof(buf), fmt, ap);
+        va_end(ap);
+        ctx->err = buf;
+    }
+    return st;
+}
+
+beagle_status check_config(const beagle_config* c) {
+    if (c == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    if (c->dtype != BEAGLE_FP32 && c->dtype != BEAGLE_BF16) return BEAGLE_ERR_INVALID_ARG;
+    if (c->hidden <= 0 || c->n_q_heads <= 0 || c->n_kv_heads <= 0 || c->head_dim <= 0 || c->mlp_dim <= 0 ||
+        c->vocab <= 0 || c->max_slots <= 0 || c->max_ctx <= 0 || c->max_draft < 0)
+        return BEAGLE_ERR_INVALID_ARG;
+    if (!(c->rms_eps >= 0.f)) return BEAGLE_ERR_INVALID_ARG;
+    if (c->hidden % 8 || c->mlp_dim % 8) return BEAGLE_ERR_SHAPE;
+    if (c->n_q_heads % c->n_kv_heads) return BEAGLE_ERR_SHAPE;
+    const int g = c->n_q_heads / c->n_kv_heads;
+    if (g != 1 && g != 2 && g != 4 && g != 8) return BEAGLE_ERR_SHAPE;
+    const int vec = c->dtype == BEAGLE_BF16 ? 8 : 4;
+    const int lpk = c->head_dim / vec;
+    if (c->head_dim % vec || (lpk != 4 && lpk != 8 && lpk != 16 && lpk != 32)) return BEAGLE_ERR_SHAPE;
+    return BEAGLE_OK;
+}
+
+struct ServeLayout {
+    size_t x, xn, q, o, y, yn, act, h, h_slot, attn, last_token, ids, lm_partials, verify_keys, total;
+    int lm_blocks;
+};
+ServeLayout serve_layout(const beagle_config& c) {
+    ServeLayout L;
+    const size_t elt = c.dtype == BEAGLE_BF16 ? 2 : 4;
+    const size_t B = BEAGLE_MAX_CALL_BATCH;
+    const size_t d = c.hidden, qd = (size_t)c.n_q_heads * c.head_dim, m = c.mlp_dim;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + bytes); return at; };
+    L.x = take(B * d * elt); L.xn = take(B * d * elt);
+    L.q = take(B * qd * elt); L.o = take(B * qd * elt);
+    L.y = take(B * d * elt); L.yn = take(B * d * elt);
+    L.act = take(B * m * elt); L.h = take(B * d * elt);
+    L.h_slot = take((size_t)c.max_slots * d * elt);
+    L.attn = take(attn_decode_scratch_bytes((int)B, c.n_q_heads, c.head_dim, c.max_ctx + c.max_draft));
+    L.last_token = take((size_t)c.max_slots * sizeof(int32_t));
+    L.ids = take(B * 65 * sizeof(int32_t));
+    L.lm_blocks = gemv_grid_blocks(GEMV_LOGITS, c.vocab);
+    L.lm_partials = take(B * (size_t)L.lm_blocks * sizeof(unsigned long long));
+    L.verify_keys = take(B * 65 * kRowArgmaxSplit * sizeof(unsigned long long));
+    L.total = off;
+    return L;
+}
+
+struct BlockLayout {
+    size_t x, xn, q, kt, vt, kp, vp, o, y, yn, act, h, logits, keys, ids, total;
+    int lm_chunk_rows;
+};
+constexpr int kLmChunkRows = 2048;
+BlockLayout block_layout(const beagle_config& c, int batch, int S) {
+    BlockLayout L;
+    const size_t elt = c.dtype == BEAGLE_BF16 ? 2 : 4;
+    const size_t M = (size_t)batch * S;
+    const size_t d = c.hidden, qd = (size_t)c.n_q_heads * c.head_dim, kd = (size_t)c.n_kv_heads * c.head_dim, m = c.mlp_dim;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + bytes); return at; };
+    L.x = take(M * d * elt); L.xn = take(M * d * elt); L.q = take(M * qd * elt);
+    L.kt = take(M * kd * elt); L.vt = take(M * kd * elt); L.kp = take(M * kd * elt); L.vp = take(M * kd * elt);
+    L.o = take(M * qd * elt); L.y = take(M * d * elt); L.yn = take(M * d * elt);
+    L.act = take(M * m * elt); L.h = take(M * d * elt);
+    L.lm_chunk_rows = (int)(M < (size_t)kLmChunkRows ? M : (size_t)kLmChunkRows);
+    L.logits = take((size_t)L.lm_chunk_rows * c.vocab * sizeof(float));
+    L.keys = take(M * kRowArgmaxSplit * sizeof(unsigned long long));
+    L.ids = take(M * sizeof(int32_t));
+    L.total = off;
+    return L;
+}
+
+beagle_status cuda_ok(beagle_ctx* ctx, const char* what) {
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(ctx, BEAGLE_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+    return BEAGLE_OK;
+}
+
+// One dense projection C = A W^T of the block / prefill path: tensor cores when the plan covers the
+// shape (bf16), the CUDA-core kernel otherwise.
+int dense_gemm(beagle_ctx* ctx, int epi, const GemmArgs& a, cudaStream_t stream) {
+    if (ctx->tc != nullptr) {
+        const int rc = tc_gemm(ctx->tc, epi, a, stream);
+        if (rc >= 0) return rc;
+    }
+    return launch_gemm_simt(ctx->cfg.dtype, epi, a, stream);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* beagle_version(void) { return "beagle-b200 0.1 (sm_100a)"; }
+
+beagle_status beagle_query_sizes(const beagle_config* cfg, size_t* kv_bytes, size_t* workspace_bytes) {
+    const beagle_status st = check_config(cfg);
+    if (st != BEAGLE_OK) return st;
+    if (kv_bytes == nullptr || workspace_bytes == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    const size_t elt = cfg->dtype == BEAGLE_BF16 ? 2 : 4;
+    const size_t cap = (size_t)cfg->max_ctx + cfg->max_draft;
+    *kv_bytes = 2 * align_up((size_t)cfg->max_slots * cfg->n_kv_heads * cap * cfg->head_dim * elt);
+    *workspace_bytes = serve_layout(*cfg).total;
+    return BEAGLE_OK;
+}
+
+beagle_status beagle_create(const beagle_config* cfg, const beagle_weights* w, void* kv_dev, size_t kv_bytes,
+                            void* workspace_dev, size_t workspace_bytes, beagle_ctx** out) {
+    if (out == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    *out = nullptr;
+    const beagle_status st = check_config(cfg);
+    if (st != BEAGLE_OK) return st;
+    if (w == nullptr || kv_dev == nullptr || workspace_dev == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    const void* const* wp = reinterpret_cast<const void* const*>(w);
+    for (size_t i = 0; i < sizeof(beagle_weights) / sizeof(void*); ++i)
+        if (wp[i] == nullptr || (reinterpret_cast<uintptr_t>(wp[i]) & 15)) return BEAGLE_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(kv_dev) & (kAlign - 1)) || (reinterpret_cast<uintptr_t>(workspace_dev) & (kAlign - 1)))
+        return BEAGLE_ERR_INVALID_ARG;
+    size_t need_kv, need_ws;
+    beagle_query_sizes(cfg, &need_kv, &need_ws);
+    if (kv_bytes < need_kv || workspace_bytes < need_ws) return BEAGLE_ERR_CAPACITY;
+
+    beagle_ctx* c = new beagle_ctx();
+    c->cfg = *cfg;
+    c->w = *w;
+    c->kv = static_cast<char*>(kv_dev);
+    c->ws = static_cast<char*>(workspace_dev);
+    c->kv_bytes = kv_bytes;
+    c->ws_bytes = workspace_bytes;
+    c->cap = cfg->max_ctx + cfg->max_draft;
+    c->elt = cfg->dtype == BEAGLE_BF16 ? 2 : 4;
+    c->qd = cfg->n_q_heads * cfg->head_dim;
+    c->kd = cfg->n_kv_heads * cfg->head_dim;
+    c->kcache = c->kv;
+    c->vcache = c->kv + need_kv / 2;
+    const ServeLayout L = serve_layout(*cfg);
+    c->x = c->ws + L.x; c->xn = c->ws + L.xn; c->q = c->ws + L.q; c->o = c->ws + L.o;
+    c->y = c->ws + L.y; c->yn = c->ws + L.yn; c->act = c->ws + L.act; c->h = c->ws + L.h;
+    c->h_slot = c->ws + L.h_slot; c->attn_scratch = c->ws + L.attn;
+    c->last_token = reinterpret_cast<int32_t*>(c->ws + L.last_token);
+    c->ids = reinterpret_cast<int32_t*>(c->ws + L.ids);
+    c->lm_partials = reinterpret_cast<unsigned long long*>(c->ws + L.lm_partials);
+    c->verify_keys = reinterpret_cast<unsigned long long*>(c->ws + L.verify_keys);
+    c->lm_blocks = L.lm_blocks;
+    c->n_true.assign(cfg->max_slots, 0);
+    c->n_draft.assign(cfg->max_slots, 0);
+    c->pending.assign(cfg->max_slots, 0);
+    c->has_token.assign(cfg->max_slots, 0);
+    c->tc = (cfg->dtype == BEAGLE_BF16) ? tc_plan_create(*cfg, *w) : nullptr;
+    *out = c;
+    return BEAGLE_OK;
+}
+
+beagle_status beagle_destroy(beagle_ctx* ctx) {
+    if (ctx == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    tc_plan_destroy(ctx->tc);
+    delete ctx;
+    return BEAGLE_OK;
+}
+
+const char* beagle_last_error(const beagle_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+int64_t beagle_launch_count(const beagle_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+static beagle_status check_slots(beagle_ctx* ctx, int32_t batch, const int32_t* seq_slot) {
+    if (batch < 0 || batch > BEAGLE_MAX_CALL_BATCH) return fail(ctx, BEAGLE_ERR_CAPACITY, "batch %d outside [0, %d]", batch, BEAGLE_MAX_CALL_BATCH);
+    if (batch > 0 && seq_slot == nullptr) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "seq_slot is NULL");
+    for (int b = 0; b < batch; ++b) {
+        if (seq_slot[b] < 0 || seq_slot[b] >= ctx->cfg.max_slots) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "slot %d out of range", seq_slot[b]);
+        for (int c = 0; c < b; ++c)
+            if (seq_slot[c] == seq_slot[b]) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "slot %d listed twice", seq_slot[b]);
+    }
+    return BEAGLE_OK;
+}
+
+beagle_status beagle_rollback(beagle_ctx* ctx, int32_t batch, const int32_t* seq_slot) {
+    if (ctx == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    const beagle_status st = check_slots(ctx, batch, seq_slot);
+    if (st != BEAGLE_OK) return st;
+    for (int b = 0; b < batch; ++b) {
+        ctx->n_draft[seq_slot[b]] = 0;
+        ctx->pending[seq_slot[b]] = 0;
+        ctx->has_token[seq_slot[b]] = 0;
+    }
+    return BEAGLE_OK;
+}
+
+beagle_status beagle_reset_slot(beagle_ctx* ctx, int32_t slot) {
+    if (ctx == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    if (slot < 0 || slot >= ctx->cfg.max_slots) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "slot %d out of range", slot);
+    ctx->n_true[slot] = ctx->n_draft[slot] = 0;
+    ctx->pending[slot] = ctx->has_token[slot] = 0;
+    return BEAGLE_OK;
+}
+
+beagle_status beagle_slot_lengths(const beagle_ctx* ctx, int32_t slot, int32_t* n_true, int32_t* n_draft) {
+    if (ctx == nullptr || slot < 0 || slot >= ctx->cfg.max_slots) return BEAGLE_ERR_INVALID_ARG;
+    if (n_true) *n_true = ctx->n_true[slot];
+    if (n_draft) *n_draft = ctx->n_draft[slot];
+    return BEAGLE_OK;
+}
+
+beagle_status beagle_prefill_kv(beagle_ctx* ctx, int32_t batch, const int32_t* seq_slot, const int32_t* new_len,
+                                const void* hidden_dev, void* stream_) {
+    if (ctx == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    beagle_status st = check_slots(ctx, batch, seq_slot);
+    if (st != BEAGLE_OK) return st;
+    if (batch > 0 && new_len == nullptr) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "new_len is NULL");
+    long long total = 0;
+    for (int b = 0; b < batch; ++b) {
+        if (new_len[b] < 0) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "new_len[%d] < 0", b);
+        if ((long long)ctx->n_true[seq_slot[b]] + new_len[b] > ctx->cfg.max_ctx)
+            return fail(ctx, BEAGLE_ERR_CAPACITY, "slot %d: %d + %d true states exceed max_ctx %d", seq_slot[b],
+                        ctx->n_true[seq_slot[b]], new_len[b], ctx->cfg.max_ctx);
+        total += new_len[b];
+    }
+    if (total > 0 && hidden_dev == nullptr) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "hidden is NULL");
+    if (total > (1ll << 30)) return fail(ctx, BEAGLE_ERR_CAPACITY, "too many rows");
+    if (total > 0 && (reinterpret_cast<uintptr_t>(hidden_dev) & 15)) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "hidden must be 16-byte aligned");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const beagle_config& c = ctx->cfg;
+
+    if (total > 0) {
+        SeqRows rows;
+        memset(&rows, 0, sizeof(rows));
+        int n = 0, r = 0;
+        for (int b = 0; b < batch; ++b) {
+            if (new_len[b] == 0) continue;
+            rows.slot[n] = seq_slot[b];
+            rows.row_start[n] = r;
+            rows.pos_start[n] = ctx->n_true[seq_slot[b]];
+            r += new_len[b];
+            ++n;
+        }
+        rows.n = n;
+        rows.row_start[n] = r;
+        if (total <= 16) {
+            // few rows (the states accepted by one verification): weight-streaming path
+            GemvArgs a;
+            memset(&a, 0, sizeof(a));
+            a.W = ctx->w.w_k; a.W2 = ctx->w.w_v; a.N = ctx->kd; a.K = c.hidden;
+            a.X = hidden_dev; a.ldx = c.hidden; a.B = (int)total;
+            a.kcache = ctx->kcache; a.vcache = ctx->vcache; a.Hkv = c.n_kv_heads; a.dh = c.head_dim; a.cap = ctx->cap;
+            for (int s = 0; s < n; ++s)
+                for (int i = rows.row_start[s]; i < rows.row_start[s + 1]; ++i) {
+                    a.xrow.idx[i] = i;
+                    a.orow2.idx[i] = rows.slot[s];
+                    a.pos.idx[i] = rows.pos_start[s] + (i - rows.row_start[s]);
+                }
+            ctx->launches += launch_gemv(c.dtype, GEMV_KV, a, stream);
+        } else {
+            GemmArgs g;
+            memset(&g, 0, sizeof(g));
+            g.A = hidden_dev; g.lda = c.hidden; g.M = (int)total; g.N = ctx->kd; g.K = c.hidden;
+            g.Hkv = c.n_kv_heads; g.dh = c.head_dim; g.cap = ctx->cap; g.rows = rows;
+            g.W = ctx->w.w_k; g.cache = ctx->kcache;
+            int rc = dense_gemm(ctx, GEMM_KV_CACHE, g, stream);
+            if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "K projection: unsupported shape");
+            ctx->launches += rc;
+            g.W = ctx->w.w_v; g.cache = ctx->vcache;
+            rc = dense_gemm(ctx, GEMM_KV_CACHE, g, stream);
+            if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "V projection: unsupported shape");
+            ctx->launches += rc;
+        }
+        st = cuda_ok(ctx, "prefill_kv");
+        if (st != BEAGLE_OK) return st;
+    }
+    for (int b = 0; b < batch; ++b) {
+        const int s = seq_slot[b];
+        ctx->n_true[s] += new_len[b];
+        ctx->n_draft[s] = 0;
+        ctx->pending[s] = 0;
+        ctx->has_token[s] = 0;
+    }
+    return BEAGLE_OK;
+}
+
+beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* seq_slot, const int32_t* tokens_in_dev,
+                                int32_t concat, int32_t* tokens_out_dev, float* logits_out_dev, void* hidden_out_dev,
+                                void* stream_) {
+    if (ctx == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    beagle_status st = check_slots(ctx, batch, seq_slot);
+    if (st != BEAGLE_OK) return st;
+    if (batch == 0) return BEAGLE_OK;
+    const beagle_config& c = ctx->cfg;
+    bool any_append = false;
+    for (int b = 0; b < batch; ++b) {
+        const int s = seq_slot[b];
+        if (tokens_in_dev == nullptr && !ctx->has_token[s])
+            return fail(ctx, BEAGLE_ERR_STATE, "slot %d has no previous draft token; pass tokens_in", s);
+        if (concat && ctx->pending[s]) {
+            if (ctx->n_draft[s] >= c.max_draft)
+                return fail(ctx, BEAGLE_ERR_CAPACITY, "slot %d: draft tail already holds max_draft = %d states", s, c.max_draft);
+            any_append = true;
+        }
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int dt = c.dtype;
+
+    BatchMeta meta;
+    memset(&meta, 0, sizeof(meta));
+    RowMap ident, slots, app_pos;
+    memset(&app_pos, 0, sizeof(app_pos));
+    int max_kv = 0;
+    for (int b = 0; b < kMaxCallBatch; ++b) { ident.idx[b] = b; slots.idx[b] = 0; }
+    for (int b = 0; b < batch; ++b) {
+        const int s = seq_slot[b];
+        const bool app = concat && ctx->pending[s];
+        app_pos.idx[b] = app ? ctx->n_true[s] + ctx->n_draft[s] : -1;
+        meta.slot[b] = s;
+        meta.kv_len[b] = ctx->n_true[s] + ctx->n_draft[s] + (app ? 1 : 0);
+        slots.idx[b] = s;
+        if (meta.kv_len[b] > max_kv) max_kv = meta.kv_len[b];
+    }
+
+    // (1) concat: K/V of the previous step's state joins the cache tail (Section 4.1, cache paragraph)
+    if (any_append) {
+        GemvArgs a;
+        memset(&a, 0, sizeof(a));
+        a.W = ctx->w.w_k; a.W2 = ctx->w.w_v; a.N = ctx->kd; a.K = c.hidden;
+        a.X = ctx->h_slot; a.ldx = c.hidden; a.B = batch; a.xrow = slots;
+        a.kcache = ctx->kcache; a.vcache = ctx->vcache; a.Hkv = c.n_kv_heads; a.dh = c.head_dim; a.cap = ctx->cap;
+        a.orow2 = slots; a.pos = app_pos;
+        ctx->launches += launch_gemv(dt, GEMV_KV, a, stream);
+    }
+    // (2) x = E[t], xn = RMSNorm(x)
+    ctx->launches += launch_embed_norm(dt, tokens_in_dev, ctx->last_token, &meta, ctx->w.embed, c.vocab, nullptr, ctx->w.g_q,
+                                       c.hidden, c.rms_eps, c.norm_q, ctx->x, ctx->xn, batch, stream);
+    // (3) Q = W_q xn
+    {
+        GemvArgs a;
+        memset(&a, 0, sizeof(a));
+        a.W = ctx->w.w_q; a.N = ctx->qd; a.K = c.hidden; a.X = ctx->xn; a.ldx = c.hidden; a.B = batch; a.xrow = ident;
+        a.out = ctx->q; a.ldo = ctx->qd;
+        ctx->launches += launch_gemv(dt, GEMV_STORE, a, stream);
+    }
+    // (4) o = softmax(Q K^T / sqrt(dh)) V over the cache
+    {
+        const int rc = launch_attn_decode(dt, ctx->q, ctx->kcache, ctx->vcache, meta, batch, c.n_q_heads, c.n_kv_heads,
+                                          c.head_dim, ctx->cap, max_kv, ctx->attn_scratch, ctx->o, stream);
+        if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "attention: unsupported head shape");
+        ctx->launches += rc;
+    }
+    // (5) y = W_o o + x
+    {
+        GemvArgs a;
+        memset(&a, 0, sizeof(a));
+        a.W = ctx->w.w_o; a.N = c.hidden; a.K = ctx->qd; a.X = ctx->o; a.ldx = ctx->qd; a.B = batch; a.xrow = ident;
+        a.out = ctx->y; a.ldo = c.hidden; a.resid = ctx->x; a.ldr = c.hidden;
+        ctx->launches += launch_gemv(dt, GEMV_RESID, a, stream);
+    }
+    // (6) yn = RMSNorm(y)
+    ctx->launches += launch_embed_norm(dt, nullptr, nullptr, nullptr, nullptr, 0, ctx->y, ctx->w.g_mlp, c.hidden, c.rms_eps,
+                                       c.norm_mlp, nullptr, ctx->yn, batch, stream);
+    // (7) act = SiLU(W_gate yn) * (W_up yn)
+    {
+        GemvArgs a;
+        memset(&a, 0, sizeof(a));
+        a.W = ctx->w.w_gate; a.W2 = ctx->w.w_up; a.N = c.mlp_dim; a.K = c.hidden; a.X = ctx->yn; a.ldx = c.hidden;
+        a.B = batch; a.xrow = ident; a.out = ctx->act; a.ldo = c.mlp_dim;
+        ctx->launches += launch_gemv(dt, GEMV_SILU_MUL, a, stream);
+    }
+    // (8) h = W_down act + y ; kept per slot for the next step's K/V append
+    {
+        GemvArgs a;
+        memset(&a, 0, sizeof(a));
+        a.W = ctx->w.w_down; a.N = c.hidden; a.K = c.mlp_dim; a.X = ctx->act; a.ldx = c.mlp_dim; a.B = batch; a.xrow = ident;
+        a.out = ctx->h; a.ldo = c.hidden; a.resid = ctx->y; a.ldr = c.hidden;
+        a.out2 = ctx->h_slot; a.ld2 = c.hidden; a.orow2 = slots;
+        ctx->launches += launch_gemv(dt, GEMV_RESID, a, stream);
+    }
+    if (hidden_out_dev != nullptr) {
+        cudaMemcpyAsync(hidden_out_dev, ctx->h, (size_t)batch * c.hidden * ctx->elt, cudaMemcpyDeviceToDevice, stream);
+    }
+    // (9) z = W_lm h, greedy token
+    {
+        GemvArgs a;
+        memset(&a, 0, sizeof(a));
+        a.W = ctx->w.w_lm; a.N = c.vocab; a.K = c.hidden; a.X = ctx->h; a.ldx = c.hidden; a.B = batch; a.xrow = ident;
+        a.logits = logits_out_dev; a.partials = ctx->lm_partials;
+        ctx->launches += launch_gemv(dt, GEMV_LOGITS, a, stream);
+        ctx->launches += launch_argmax_finalize(ctx->lm_partials, ctx->lm_blocks, meta, batch, tokens_out_dev, ctx->last_token, stream);
+    }
+    st = cuda_ok(ctx, "draft_step");
+    if (st != BEAGLE_OK) return st;
+    for (int b = 0; b < batch; ++b) {
+        const int s = seq_slot[b];
+        if (concat && ctx->pending[s]) ctx->n_draft[s] += 1;
+        ctx->pending[s] = 1;
+        ctx->has_token[s] = 1;
+    }
+    return BEAGLE_OK;
+}
+
+beagle_status beagle_block_workspace_bytes(const beagle_config* cfg, int32_t batch, int32_t S, size_t* bytes) {
+    const beagle_status st = check_config(cfg);
+    if (st != BEAGLE_OK) return st;
+    if (bytes == nullptr || batch <= 0 || S <= 0) return BEAGLE_ERR_INVALID_ARG;
+    if ((long long)batch * S > (1ll << 24)) return BEAGLE_ERR_CAPACITY;
+    *bytes = block_layout(*cfg, batch, S).total;
+    return BEAGLE_OK;
+}
+
+beagle_status beagle_block_forward(beagle_ctx* ctx, int32_t batch, int32_t S, const int32_t* tokens_dev,
+                                   const void* hidden_dev, int32_t block, int32_t offset, int32_t sim_steps,
+                                   float* logits_out_dev, int32_t* argmax_out_dev, void* hidden_out_dev,
+                                   void* ws_dev, size_t ws_bytes, void* stream_) {
+    if (ctx == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    if (batch <= 0 || S <= 0 || tokens_dev == nullptr || hidden_dev == nullptr || ws_dev == nullptr)
+        return fail(ctx, BEAGLE_ERR_INVALID_ARG, "block_forward: NULL or empty argument");
+    if ((long long)batch * S > (1ll << 24)) return fail(ctx, BEAGLE_ERR_CAPACITY, "block_forward: too many positions");
+    if (block < 1 || offset < 0 || offset >= S || sim_steps < 1 || sim_steps > block)
+        return fail(ctx, BEAGLE_ERR_INVALID_ARG, "block_forward: need block >= 1, 0 <= offset < S, 1 <= sim_steps <= block");
+    if (ctx->cfg.head_dim % 32) return fail(ctx, BEAGLE_ERR_SHAPE, "block_forward: head_dim must be a multiple of 32");
+    if (reinterpret_cast<uintptr_t>(ws_dev) & (kAlign - 1)) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "workspace must be 256-byte aligned");
+    if ((reinterpret_cast<uintptr_t>(hidden_dev) & 15) || (hidden_out_dev && (reinterpret_cast<uintptr_t>(hidden_out_dev) & 15)))
+        return fail(ctx, BEAGLE_ERR_INVALID_ARG, "hidden buffers must be 16-byte aligned");
+    const beagle_config& c = ctx->cfg;
+    const BlockLayout L = block_layout(c, batch, S);
+    if (ws_bytes < L.total) return fail(ctx, BEAGLE_ERR_CAPACITY, "block_forward: workspace %zu < %zu bytes", ws_bytes, L.total);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    char* ws = static_cast<char*>(ws_dev);
+    const int dt = c.dtype;
+    const int M = batch * S;
+    void *X = ws + L.x, *Xn = ws + L.xn, *Q = ws + L.q, *Kt = ws + L.kt, *Vt = ws + L.vt, *Kp = ws + L.kp, *Vp = ws + L.vp;
+    void *O = ws + L.o, *Y = ws + L.y, *Yn = ws + L.yn, *ACT = ws + L.act;
+    void* H = hidden_out_dev != nullptr ? hidden_out_dev : (void*)(ws + L.h);
+    int rc;
+#define BEAGLE_GEMM(EPI, ARGS, WHAT)                                                   \
+    do {                                                                               \
+        rc = dense_gemm(ctx, EPI, ARGS, stream);                                       \
+        if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, WHAT ": unsupported shape");   \
+        ctx->launches += rc;                                                           \
+    } while (0)
+
+    // queries: every position's data token (Section 4.2: no new queries are generated)
+    ctx->launches += launch_embed_norm(dt, tokens_dev, nullptr, nullptr, ctx->w.embed, c.vocab, nullptr,
+                                       ctx->w.g_q, c.hidden, c.rms_eps, c.norm_q, X, Xn, M, stream);
+    GemmArgs g;
+    memset(&g, 0, sizeof(g));
+    g.M = M;
+    g.A = Xn; g.lda = c.hidden; g.K = c.hidden; g.W = ctx->w.w_q; g.N = ctx->qd; g.C = Q; g.ldc = ctx->qd;
+    BEAGLE_GEMM(GEMM_STORE, g, "Q projection");
+    // keys / values of the true states
+    g.A = hidden_dev; g.W = ctx->w.w_k; g.N = ctx->kd; g.C = Kt; g.ldc = ctx->kd;
+    BEAGLE_GEMM(GEMM_STORE, g, "K projection");
+    g.W = ctx->w.w_v; g.C = Vt;
+    BEAGLE_GEMM(GEMM_STORE, g, "V projection");
+
+    for (int step = 1; step <= sim_steps; ++step) {
+        if (step > 1) {
+            // the states predicted so far become keys / values at their own positions (in place)
+            memset(&g, 0, sizeof(g));
+            g.M = M; g.A = H; g.lda = c.hidden; g.K = c.hidden; g.N = ctx->kd; g.ldc = ctx->kd;
+            g.W = ctx->w.w_k; g.C = Kp;
+            BEAGLE_GEMM(GEMM_STORE, g, "predicted K projection");
+            g.W = ctx->w.w_v; g.C = Vp;
+            BEAGLE_GEMM(GEMM_STORE, g, "predicted V projection");
+        }
+        rc = launch_attn_block(dt, Q, Kt, Vt, Kp, Vp, batch, S, c.n_q_heads, c.n_kv_heads, c.head_dim, block, offset, step, O, stream);
+        if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "block attention: unsupported head_dim");
+        ctx->launches += rc;
+        memset(&g, 0, sizeof(g));
+        g.M = M; g.A = O; g.lda = ctx->qd; g.K = ctx->qd; g.W = ctx->w.w_o; g.N = c.hidden; g.C = Y; g.ldc = c.hidden;
+        g.R = X; g.ldr = c.hidden;
+        BEAGLE_GEMM(GEMM_RESID, g, "O projection");
+        ctx->launches += launch_embed_norm(dt, nullptr, nullptr, nullptr, nullptr, 0, Y, ctx->w.g_mlp, c.hidden, c.rms_eps,
+                                           c.norm_mlp, nullptr, Yn, M, stream);
+        memset(&g, 0, sizeof(g));
+        g.M = M; g.A = Yn; g.lda = c.hidden; g.K = c.hidden; g.W = ctx->w.w_gate; g.W2 = ctx->w.w_up; g.N = c.mlp_dim;
+        g.C = ACT; g.ldc = c.mlp_dim;
+        BEAGLE_GEMM(GEMM_SILU_MUL, g, "gate/up projection");
+        memset(&g, 0, sizeof(g));
+        g.M = M; g.A = ACT; g.lda = c.mlp_dim; g.K = c.mlp_dim; g.W = ctx->w.w_down; g.N = c.hidden; g.C = H; g.ldc = c.hidden;
+        g.R = Y; g.ldr = c.hidden;
+        BEAGLE_GEMM(GEMM_RESID, g, "down projection");
+    }
+
+    // LM head at every position
+    if (logits_out_dev != nullptr || argmax_out_dev != nullptr) {
+        unsigned long long* keys = reinterpret_cast<unsigned long long*>(ws + L.keys);
+        int32_t* ids = argmax_out_dev != nullptr ? argmax_out_dev : reinterpret_cast<int32_t*>(ws + L.ids);
+        if (logits_out_dev != nullptr) {
+            memset(&g, 0, sizeof(g));
+            g.M = M; g.A = H; g.lda = c.hidden; g.K = c.hidden; g.W = ctx->w.w_lm; g.N = c.vocab; g.C = logits_out_dev; g.ldc = c.vocab;
+            BEAGLE_GEMM(GEMM_F32, g, "LM head");
+            if (argmax_out_dev != nullptr) ctx->launches += launch_row_argmax(0, logits_out_dev, M, c.vocab, keys, ids, stream);
+        } else {
+            float* chunk = reinterpret_cast<float*>(ws + L.logits);
+            for (int r0 = 0; r0 < M; r0 += L.lm_chunk_rows) {
+                const int rows = M - r0 < L.lm_chunk_rows ? M - r0 : L.lm_chunk_rows;
+                memset(&g, 0, sizeof(g));
+                g.M = rows; g.A = static_cast<const char*>(H) + (size_t)r0 * c.hidden * ctx->elt; g.lda = c.hidden; g.K = c.hidden;
+                g.W = ctx->w.w_lm; g.N = c.vocab; g.C = chunk; g.ldc = c.vocab;
+                BEAGLE_GEMM(GEMM_F32, g, "LM head");
+                ctx->launches += launch_row_argmax(0, chunk, rows, c.vocab, keys + (size_t)r0 * kRowArgmaxSplit, ids + r0, stream);
+            }
+        }
+    }
+#undef BEAGLE_GEMM
+    return cuda_ok(ctx, "block_forward");
+}
+
+beagle_status beagle_verify_greedy(beagle_ctx* ctx, int32_t batch, int32_t gamma, const int32_t* draft_tokens_dev,
+                                   const void* target_logits_dev, int32_t logits_dtype, const int32_t* target_ids_dev,
+                                   int32_t* accept_len_dev, int32_t* out_tokens_dev, void* stream_) {
+    if (ctx == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    if (batch < 0 || batch > BEAGLE_MAX_CALL_BATCH) return fail(ctx, BEAGLE_ERR_CAPACITY, "batch %d outside [0, %d]", batch, BEAGLE_MAX_CALL_BATCH);
+    if (gamma < 0 || gamma > 64) return fail(ctx, BEAGLE_ERR_CAPACITY, "gamma %d outside [0, 64]", gamma);
+    if (batch == 0) return BEAGLE_OK;
+    if ((gamma > 0 && draft_tokens_dev == nullptr) || accept_len_dev == nullptr || out_tokens_dev == nullptr)
+        return fail(ctx, BEAGLE_ERR_INVALID_ARG, "verify: NULL argument");
+    if ((target_logits_dev == nullptr) == (target_ids_dev == nullptr))
+        return fail(ctx, BEAGLE_ERR_INVALID_ARG, "verify: give exactly one of target_logits / target_ids");
+    if (target_logits_dev != nullptr && logits_dtype != BEAGLE_FP32 && logits_dtype != BEAGLE_BF16)
+        return fail(ctx, BEAGLE_ERR_INVALID_ARG, "verify: unknown logits_dtype");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int32_t* ids = target_ids_dev;
+    if (target_logits_dev != nullptr) {
+        ctx->launches += launch_row_argmax(logits_dtype, target_logits_dev, batch * (gamma + 1), ctx->cfg.vocab,
+                                           ctx->verify_keys, ctx->ids, stream);
+        ids = ctx->ids;
+    }
+    ctx->launches += launch_accept(draft_tokens_dev, ids, batch, gamma, accept_len_dev, out_tokens_dev, stream);
+    return cuda_ok(ctx, "verify_greedy");
+}
+
+}  // extern "C"

@@ -1,0 +1,17 @@
+// bf16 tensor-core GEMM (tcgen05 + TMEM + TMA) behind the dense projections.
+#pragma once
+#include "../../include/beagle.h"
+#include "kernels.h"
+
+namespace beagle {
+
+struct TcPlan;   // tensor maps of the weight matrices and launch constants
+
+// Returns nullptr when the tensor-core path cannot serve this configuration.
+TcPlan* tc_plan_create(const beagle_config& cfg, const beagle_weights& w);
+void tc_plan_destroy(TcPlan* plan);
+// C = A W^T with the fused epilogue `epi` (GemmEpilogue).  Returns the number of kernels launched,
+// or -1 when this shape is not covered (the caller then uses the CUDA-core kernel).
+int tc_gemm(TcPlan* plan, int epi, const GemmArgs& a, cudaStream_t stream);
+
+}  // namespace beagle

@@ -1,0 +1,97 @@
+// Host-side launchers of the Beagle draft-head kernels.  Every function only enqueues kernels on
+// `stream` and returns the number of kernels it launched (negative: unsupported shape).
+#pragma once
+#include "common.cuh"
+
+namespace beagle {
+
+enum GemvMode {
+    GEMV_STORE = 0,     // out[b][n] = W[n,:] . x_b
+    GEMV_RESID = 1,     // out[b][n] = W[n,:] . x_b + resid[b][n]      (+ optional second copy out2[orow2[b]][n])
+    GEMV_SILU_MUL = 2,  // out[b][n] = SiLU(W[n,:] . x_b) * (W2[n,:] . x_b)
+    GEMV_LOGITS = 3,    // logits[b][n] (fp32, optional) and per-block arg-max keys
+    GEMV_KV = 4         // blockIdx.y = 0: W -> key cache, 1: W2 -> value cache, at (slot[b], head, pos[b])
+};
+
+struct GemvArgs {
+    const void* W;
+    const void* W2;
+    int N, K;
+    const void* X;      // activations, storage type, row b at X + xrow.idx[b] * ldx
+    int ldx;
+    int B;
+    void* out;          // [B, ldo]
+    int ldo;
+    const void* resid;  // [B, ldr]
+    int ldr;
+    void* out2;         // optional [*, ld2], row orow2.idx[b]
+    int ld2;
+    float* logits;      // optional fp32 [B, N]
+    unsigned long long* partials;   // [B, gridDim.x]
+    void* kcache;
+    void* vcache;
+    int Hkv, dh, cap;   // cache geometry [slot][Hkv][cap][dh]
+    RowMap xrow;
+    RowMap orow2;       // GEMV_RESID: rows of out2; GEMV_KV: cache slot
+    RowMap pos;         // GEMV_KV: position in the slot
+};
+
+int gemv_grid_blocks(int mode, int N);   // gridDim.x the launcher uses (size of the partials row)
+int launch_gemv(int dtype, int mode, const GemvArgs& a, cudaStream_t stream);
+
+// x = E[token] (or rows of src), xn = RMSNorm(x) * g (or x when do_norm == 0).
+// tokens == NULL: row b uses last_token[meta.slot[b]].  src != NULL: no gather, rows of src.
+int launch_embed_norm(int dtype, const int32_t* tokens, const int32_t* last_token, const BatchMeta* meta,
+                      const void* embed, int vocab, const void* src, const void* gain, int d, float eps, int do_norm,
+                      void* x_out, void* xn_out, int rows, cudaStream_t stream);
+
+// Split-KV cross-attention decode over the cache + combine.  q, o: [B, Hq*dh] storage type.
+size_t attn_decode_scratch_bytes(int max_batch, int Hq, int dh, int max_kv);
+int launch_attn_decode(int dtype, const void* q, const void* kcache, const void* vcache, const BatchMeta& meta,
+                       int B, int Hq, int Hkv, int dh, int cap, int max_kv_len, void* scratch, void* o,
+                       cudaStream_t stream);
+
+// tokens_out[b] (optional) and last_token[slot[b]] from the per-block keys.
+int launch_argmax_finalize(const unsigned long long* partials, int nblk, const BatchMeta& meta, int B,
+                           int32_t* tokens_out, int32_t* last_token, cudaStream_t stream);
+
+// Row arg-max of [rows, V] logits (fp32 or bf16) into int32 ids; scratch: rows * kRowArgmaxSplit keys.
+constexpr int kRowArgmaxSplit = 16;
+int launch_row_argmax(int logits_dtype, const void* logits, int rows, int V, unsigned long long* scratch,
+                      int32_t* ids_out, cudaStream_t stream);
+// Greedy acceptance from target ids.
+int launch_accept(const int32_t* draft, const int32_t* target_ids, int B, int gamma, int32_t* accept_len,
+                  int32_t* out_tokens, cudaStream_t stream);
+
+// ---- block path ------------------------------------------------------------------------------
+enum GemmEpilogue {
+    GEMM_STORE = 0,      // C = A W^T                     (storage type)
+    GEMM_RESID = 1,      // C = A W^T + R
+    GEMM_SILU_MUL = 2,   // C = SiLU(A W^T) * (A W2^T)
+    GEMM_F32 = 3,        // C fp32
+    GEMM_KV_CACHE = 4    // scatter rows into the cache: row r -> (slot, pos) through SeqRows
+};
+struct SeqRows {        // packed-row -> (slot, position) map of a prefill call
+    int32_t n;
+    int32_t slot[kMaxCallBatch];
+    int32_t row_start[kMaxCallBatch + 1];
+    int32_t pos_start[kMaxCallBatch];
+};
+struct GemmArgs {
+    const void* A; int lda;       // [M, K]
+    const void* W; const void* W2;  // [N, K]
+    int M, N, K;
+    void* C; int ldc;
+    const void* R; int ldr;
+    void* cache; int Hkv, dh, cap;  // GEMM_KV_CACHE
+    SeqRows rows;
+};
+int launch_gemm_simt(int dtype, int epi, const GemmArgs& a, cudaStream_t stream);
+
+// Block-masked cross-attention: query row (b, p) reads true keys [0, n(p)) of Kt/Vt and, when
+// step > 1, predicted keys n(p) .. n(p)+min(slot, step)-2 of Kp/Vp.  All [B*S, H*dh] row-major.
+int launch_attn_block(int dtype, const void* Q, const void* Kt, const void* Vt, const void* Kp, const void* Vp,
+                      int B, int S, int Hq, int Hkv, int dh, int block, int offset, int step, void* O,
+                      cudaStream_t stream);
+
+}  // namespace beagle

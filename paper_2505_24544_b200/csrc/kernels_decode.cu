@@ -1,0 +1,530 @@
+// Serve-time kernels of the Beagle draft head: embedding + RMSNorm, weight-streaming skinny
+// projections with fused epilogues, split-KV cross-attention decode over the cache, arg-max and
+// greedy acceptance.  All HBM-bound: 16-byte coalesced loads, fp32 accumulation.
+#include "kernels.h"
+
+namespace beagle {
+
+// ------------------------------------------------------------------------------------------------
+// Embedding gather + RMSNorm (Eq. 1: e(t_p); normalisation as configured)
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) embed_norm_kernel(const int32_t* __restrict__ tokens,
+                                                         const int32_t* __restrict__ last_token,
+                                                         const BatchMeta meta,
+                                                         const T* __restrict__ embed, int vocab,
+                                                         const T* __restrict__ src, const T* __restrict__ gain,
+                                                         int d, float eps, int do_norm, T* __restrict__ x_out,
+                                                         T* __restrict__ xn_out) {
+    const int r = blockIdx.x;
+    const T* row;
+    if (src != nullptr) {
+        row = src + (size_t)r * d;
+    } else {
+        int tok = tokens != nullptr ? tokens[r] : last_token[meta.slot[r]];
+        tok = min(max(tok, 0), vocab - 1);      // ids are validated by contract; never read out of range
+        row = embed + (size_t)tok * d;
+    }
+    float ss = 0.f;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        float v = to_float<T>(row[i]);
+        ss += v * v;
+    }
+    __shared__ float s_part[8];
+    __shared__ float s_scale;
+    ss = warp_sum(ss);
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float t = 0.f;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) t += s_part[w];
+        s_scale = do_norm ? rsqrtf(t / (float)d + eps) : 1.0f;
+    }
+    __syncthreads();
+    const float sc = s_scale;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) {
+        float v = to_float<T>(row[i]);
+        if (x_out != nullptr) x_out[(size_t)r * d + i] = from_float<T>(v);
+        float g = do_norm ? to_float<T>(gain[i]) : 1.0f;
+        xn_out[(size_t)r * d + i] = from_float<T>(v * sc * g);
+    }
+}
+
+int launch_embed_norm(int dtype, const int32_t* tokens, const int32_t* last_token, const BatchMeta* meta,
+                      const void* embed, int vocab, const void* src, const void* gain, int d, float eps, int do_norm,
+                      void* x_out, void* xn_out, int rows, cudaStream_t stream) {
+    if (rows <= 0) return 0;
+    BatchMeta m;
+    if (meta != nullptr) m = *meta; else memset(&m, 0, sizeof(m));
+    if (dtype == 0)
+        embed_norm_kernel<float><<<rows, 256, 0, stream>>>(tokens, last_token, m, (const float*)embed, vocab,
+                                                           (const float*)src, (const float*)gain, d, eps, do_norm,
+                                                           (float*)x_out, (float*)xn_out);
+    else
+        embed_norm_kernel<bf16><<<rows, 256, 0, stream>>>(tokens, last_token, m, (const bf16*)embed, vocab,
+                                                          (const bf16*)src, (const bf16*)gain, d, eps, do_norm,
+                                                          (bf16*)x_out, (bf16*)xn_out);
+    return 1;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Skinny projection: out[b][n] = W[n,:] . x_b for B <= 64 rows.  One warp owns two weight rows
+// (or one row of each of W / W2 in the gated mode) and streams them once per group of NB batch
+// rows with 16-byte loads; the activations are re-read through L1.
+// ------------------------------------------------------------------------------------------------
+template <typename T, int NB, int MODE>
+__global__ void __launch_bounds__(256) gemv_kernel(const GemvArgs a) {
+    constexpr int VEC = VecOf<T>::N;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int unit = blockIdx.x * 8 + warp;
+    const T* W = reinterpret_cast<const T*>(a.W);
+    const T* W2 = reinterpret_cast<const T*>(a.W2);
+    const T* Wsel = (MODE == GEMV_KV && blockIdx.y == 1) ? W2 : W;
+    int n0, n1;
+    bool v0, v1;
+    const T *w0, *w1;
+    if (MODE == GEMV_SILU_MUL) {
+        n0 = n1 = unit;
+        v0 = v1 = unit < a.N;
+        const int nn = v0 ? unit : 0;
+        w0 = W + (size_t)nn * a.K;
+        w1 = W2 + (size_t)nn * a.K;
+    } else {
+        n0 = 2 * unit;
+        n1 = n0 + 1;
+        v0 = n0 < a.N;
+        v1 = n1 < a.N;
+        w0 = Wsel + (size_t)(v0 ? n0 : 0) * a.K;
+        w1 = Wsel + (size_t)(v1 ? n1 : 0) * a.K;
+    }
+    const T* X = reinterpret_cast<const T*>(a.X);
+    __shared__ unsigned long long s_keys[8][NB];
+
+    for (int b0 = 0; b0 < a.B; b0 += NB) {
+        const T* xp[NB];
+#pragma unroll
+        for (int j = 0; j < NB; ++j) {
+            const int b = min(b0 + j, a.B - 1);
+            xp[j] = X + (size_t)a.xrow.idx[b] * a.ldx;
+        }
+        float acc0[NB], acc1[NB];
+#pragma unroll
+        for (int j = 0; j < NB; ++j) { acc0[j] = 0.f; acc1[j] = 0.f; }
+
+#pragma unroll 4
+        for (int k = lane * VEC; k < a.K; k += 32 * VEC) {
+            float wf0[VEC], wf1[VEC];
+            unpack16<T>(ld_stream16(w0 + k), wf0);
+            unpack16<T>(ld_stream16(w1 + k), wf1);
+#pragma unroll
+            for (int j = 0; j < NB; ++j) {
+                float xf[VEC];
+                unpack16<T>(ld_cached16(xp[j] + k), xf);
+#pragma unroll
+                for (int v = 0; v < VEC; ++v) {
+                    acc0[j] = fmaf(wf0[v], xf[v], acc0[j]);
+                    acc1[j] = fmaf(wf1[v], xf[v], acc1[j]);
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < NB; ++j) {
+            acc0[j] = warp_sum(acc0[j]);
+            acc1[j] = warp_sum(acc1[j]);
+        }
+
+        if (MODE == GEMV_LOGITS) {
+#pragma unroll
+            for (int j = 0; j < NB; ++j) {
+                unsigned long long key = 0ull;
+                if (v0) key = argmax_key(acc0[j], n0);
+                if (v1) { unsigned long long k1 = argmax_key(acc1[j], n1); key = k1 > key ? k1 : key; }
+                if (lane == 0) s_keys[warp][j] = key;
+                if (lane == 0 && a.logits != nullptr && b0 + j < a.B) {
+                    if (v0) a.logits[(size_t)(b0 + j) * a.N + n0] = acc0[j];
+                    if (v1) a.logits[(size_t)(b0 + j) * a.N + n1] = acc1[j];
+                }
+            }
+            __syncthreads();
+            if (threadIdx.x < NB && b0 + (int)threadIdx.x < a.B) {
+                unsigned long long key = s_keys[0][threadIdx.x];
+#pragma unroll
+                for (int w = 1; w < 8; ++w) { unsigned long long o = s_keys[w][threadIdx.x]; key = o > key ? o : key; }
+                a.partials[(size_t)(b0 + threadIdx.x) * gridDim.x + blockIdx.x] = key;
+            }
+            __syncthreads();
+        } else if (lane == 0) {
+#pragma unroll
+            for (int j = 0; j < NB; ++j) {
+                const int b = b0 + j;
+                if (b >= a.B) break;
+                if (MODE == GEMV_STORE) {
+                    T* out = reinterpret_cast<T*>(a.out) + (size_t)b * a.ldo;
+                    if (v0) out[n0] = from_float<T>(acc0[j]);
+                    if (v1) out[n1] = from_float<T>(acc1[j]);
+                } else if (MODE == GEMV_RESID) {
+                    const T* r = reinterpret_cast<const T*>(a.resid) + (size_t)b * a.ldr;
+                    T* out = reinterpret_cast<T*>(a.out) + (size_t)b * a.ldo;
+                    T* out2 = a.out2 ? reinterpret_cast<T*>(a.out2) + (size_t)a.orow2.idx[b] * a.ld2 : nullptr;
+                    if (v0) { T y = from_float<T>(acc0[j] + to_float<T>(r[n0])); out[n0] = y; if (out2) out2[n0] = y; }
+                    if (v1) { T y = from_float<T>(acc1[j] + to_float<T>(r[n1])); out[n1] = y; if (out2) out2[n1] = y; }
+                } else if (MODE == GEMV_SILU_MUL) {
+                    if (v0) reinterpret_cast<T*>(a.out)[(size_t)b * a.ldo + n0] = from_float<T>(silu_f(acc0[j]) * acc1[j]);
+                } else if (MODE == GEMV_KV) {
+                    T* cache = reinterpret_cast<T*>(blockIdx.y == 1 ? a.vcache : a.kcache);
+                    const int slot = a.orow2.idx[b], pos = a.pos.idx[b];
+                    if (pos < 0) continue;          // this row appends nothing
+                    if (v0) cache[(((size_t)slot * a.Hkv + n0 / a.dh) * a.cap + pos) * a.dh + n0 % a.dh] = from_float<T>(acc0[j]);
+                    if (v1) cache[(((size_t)slot * a.Hkv + n1 / a.dh) * a.cap + pos) * a.dh + n1 % a.dh] = from_float<T>(acc1[j]);
+                }
+            }
+        }
+    }
+}
+
+int gemv_grid_blocks(int mode, int N) {
+    const int units = (mode == GEMV_SILU_MUL) ? N : (N + 1) / 2;
+    return (units + 7) / 8;
+}
+
+template <typename T, int MODE>
+static void gemv_dispatch_nb(const GemvArgs& a, dim3 grid, cudaStream_t stream) {
+    if (a.B <= 1) gemv_kernel<T, 1, MODE><<<grid, 256, 0, stream>>>(a);
+    else if (a.B <= 2) gemv_kernel<T, 2, MODE><<<grid, 256, 0, stream>>>(a);
+    else if (a.B <= 4) gemv_kernel<T, 4, MODE><<<grid, 256, 0, stream>>>(a);
+    else gemv_kernel<T, 8, MODE><<<grid, 256, 0, stream>>>(a);
+}
+template <typename T>
+static void gemv_dispatch_mode(int mode, const GemvArgs& a, dim3 grid, cudaStream_t stream) {
+    switch (mode) {
+        case GEMV_STORE: gemv_dispatch_nb<T, GEMV_STORE>(a, grid, stream); break;
+        case GEMV_RESID: gemv_dispatch_nb<T, GEMV_RESID>(a, grid, stream); break;
+        case GEMV_SILU_MUL: gemv_dispatch_nb<T, GEMV_SILU_MUL>(a, grid, stream); break;
+        case GEMV_LOGITS: gemv_dispatch_nb<T, GEMV_LOGITS>(a, grid, stream); break;
+        default: gemv_dispatch_nb<T, GEMV_KV>(a, grid, stream); break;
+    }
+}
+int launch_gemv(int dtype, int mode, const GemvArgs& a, cudaStream_t stream) {
+    if (a.B <= 0 || a.N <= 0) return 0;
+    dim3 grid(gemv_grid_blocks(mode, a.N), mode == GEMV_KV ? 2 : 1);
+    if (dtype == 0) gemv_dispatch_mode<float>(mode, a, grid, stream);
+    else gemv_dispatch_mode<bf16>(mode, a, grid, stream);
+    return 1;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Cross-attention decode (Eq. 2 lines 2-3 over the cached K/V): split-KV partials + combine.
+// One CTA = one (sequence, K/V head, chunk of kAttnChunk keys); its G = Hq/Hkv query heads share
+// every key/value row it streams.  LPK lanes cover one cache row with one 16-byte load each.
+// ------------------------------------------------------------------------------------------------
+constexpr int kAttnChunk = 256;
+constexpr int kAttnWarps = 4;
+
+template <typename T, int G, int LPK>
+__global__ void __launch_bounds__(kAttnWarps * 32) attn_decode_kernel(
+    const T* __restrict__ q, const T* __restrict__ kcache, const T* __restrict__ vcache, const BatchMeta meta,
+    int Hq, int Hkv, int cap, int nchunk_max, float scale, float* __restrict__ part_o, float* __restrict__ part_ml) {
+    constexpr int VEC = VecOf<T>::N;
+    constexpr int DH = LPK * VEC;
+    constexpr int KPW = 32 / LPK;                 // keys per warp per iteration
+    constexpr int KPI = KPW * kAttnWarps;         // keys per CTA per iteration
+    const int chunk = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
+    const int kv_len = meta.kv_len[b];
+    const int start = chunk * kAttnChunk;
+    if (start >= kv_len) return;
+    const int cnt = min(kAttnChunk, kv_len - start);
+    const int slot = meta.slot[b];
+    const size_t base = (((size_t)slot * Hkv + kvh) * cap + start) * DH;
+    const T* kb = kcache + base;
+    const T* vb = vcache + base;
+
+    __shared__ float s_q[G][DH];
+    __shared__ float s_s[G][kAttnChunk];
+    __shared__ float s_acc[kAttnWarps][G][DH];
+    __shared__ float s_m[G], s_l[G];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    for (int i = tid; i < G * DH; i += kAttnWarps * 32)
+        s_q[i / DH][i % DH] = to_float<T>(q[((size_t)b * Hq + kvh * G + i / DH) * DH + i % DH]) * scale;
+    __syncthreads();
+
+    const int sub = lane % LPK, kgrp = lane / LPK;
+    float qf[G][VEC];
+#pragma unroll
+    for (int g = 0; g < G; ++g)
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) qf[g][v] = s_q[g][sub * VEC + v];
+
+    // phase 1: scores
+#pragma unroll 4
+    for (int jb = warp * KPW; jb < cnt; jb += KPI) {
+        const int j = jb + kgrp;
+        const bool valid = j < cnt;
+        float kf[VEC];
+        if (valid) unpack16<T>(ld_stream16(kb + (size_t)j * DH + sub * VEC), kf);
+        else {
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) kf[v] = 0.f;
+        }
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            float dot = 0.f;
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) dot = fmaf(qf[g][v], kf[v], dot);
+#pragma unroll
+            for (int o = LPK / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+            if (valid && sub == 0) s_s[g][j] = dot;
+        }
+    }
+    __syncthreads();
+
+    // phase 2: chunk-local max and exp-sum per query head
+    for (int g = warp; g < G; g += kAttnWarps) {
+        float m = -INFINITY;
+        for (int j = lane; j < cnt; j += 32) m = fmaxf(m, s_s[g][j]);
+        m = warp_max(m);
+        float l = 0.f;
+        for (int j = lane; j < cnt; j += 32) {
+            const float p = __expf(s_s[g][j] - m);
+            s_s[g][j] = p;
+            l += p;
+        }
+        l = warp_sum(l);
+        if (lane == 0) { s_m[g] = m; s_l[g] = l; }
+    }
+    __syncthreads();
+
+    // phase 3: unnormalised P.V
+    float acc[G][VEC];
+#pragma unroll
+    for (int g = 0; g < G; ++g)
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) acc[g][v] = 0.f;
+#pragma unroll 4
+    for (int jb = warp * KPW; jb < cnt; jb += KPI) {
+        const int j = jb + kgrp;
+        if (j < cnt) {
+            float vf[VEC];
+            unpack16<T>(ld_stream16(vb + (size_t)j * DH + sub * VEC), vf);
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                const float p = s_s[g][j];
+#pragma unroll
+                for (int v = 0; v < VEC; ++v) acc[g][v] = fmaf(p, vf[v], acc[g][v]);
+            }
+        }
+    }
+#pragma unroll
+    for (int g = 0; g < G; ++g)
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) {
+            float t = acc[g][v];
+#pragma unroll
+            for (int o = LPK; o < 32; o <<= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+            if (kgrp == 0) s_acc[warp][g][sub * VEC + v] = t;
+        }
+    __syncthreads();
+    for (int i = tid; i < G * DH; i += kAttnWarps * 32) {
+        const int g = i / DH, c = i % DH;
+        float t = 0.f;
+#pragma unroll
+        for (int w = 0; w < kAttnWarps; ++w) t += s_acc[w][g][c];
+        part_o[(((size_t)b * Hq + kvh * G + g) * nchunk_max + chunk) * DH + c] = t;
+    }
+    if (tid < G) {
+        const size_t pi = ((size_t)b * Hq + kvh * G + tid) * nchunk_max + chunk;
+        part_ml[2 * pi] = s_m[tid];
+        part_ml[2 * pi + 1] = s_l[tid];
+    }
+}
+
+template <typename T>
+__global__ void attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
+                                    const BatchMeta meta, int Hq, int dh, int nchunk_max, T* __restrict__ o) {
+    const int h = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
+    const int kv_len = meta.kv_len[b];
+    const int nch = (kv_len + kAttnChunk - 1) / kAttnChunk;
+    const size_t p0 = ((size_t)b * Hq + h) * nchunk_max;
+    float M = -INFINITY;
+    for (int i = 0; i < nch; ++i) M = fmaxf(M, part_ml[2 * (p0 + i)]);
+    float num = 0.f, den = 0.f;
+    for (int i = 0; i < nch; ++i) {
+        const float w = __expf(part_ml[2 * (p0 + i)] - M);
+        den = fmaf(w, part_ml[2 * (p0 + i) + 1], den);
+        num = fmaf(w, part_o[(p0 + i) * dh + c], num);
+    }
+    o[((size_t)b * Hq + h) * dh + c] = from_float<T>(nch > 0 ? num / den : 0.f);
+}
+
+size_t attn_decode_scratch_bytes(int max_batch, int Hq, int dh, int max_kv) {
+    const size_t nch = (size_t)(max_kv + kAttnChunk - 1) / kAttnChunk + 1;
+    const size_t rows = (size_t)max_batch * Hq * nch;
+    return rows * dh * sizeof(float) + rows * 2 * sizeof(float) + 256;
+}
+
+template <typename T, int G>
+static int attn_dispatch_lpk(int lpk, dim3 grid, cudaStream_t stream, const T* q, const T* kc, const T* vc,
+                             const BatchMeta& meta, int Hq, int Hkv, int cap, int nch, float scale, float* po, float* pml) {
+    switch (lpk) {
+        case 4: attn_decode_kernel<T, G, 4><<<grid, kAttnWarps * 32, 0, stream>>>(q, kc, vc, meta, Hq, Hkv, cap, nch, scale, po, pml); return 1;
+        case 8: attn_decode_kernel<T, G, 8><<<grid, kAttnWarps * 32, 0, stream>>>(q, kc, vc, meta, Hq, Hkv, cap, nch, scale, po, pml); return 1;
+        case 16: attn_decode_kernel<T, G, 16><<<grid, kAttnWarps * 32, 0, stream>>>(q, kc, vc, meta, Hq, Hkv, cap, nch, scale, po, pml); return 1;
+        case 32:
+            if constexpr (G * 32 * VecOf<T>::N <= 1024) {   // static shared memory stays under 48 KB
+                attn_decode_kernel<T, G, 32><<<grid, kAttnWarps * 32, 0, stream>>>(q, kc, vc, meta, Hq, Hkv, cap, nch, scale, po, pml);
+                return 1;
+            } else {
+                return -1;
+            }
+        default: return -1;
+    }
+}
+template <typename T>
+static int attn_dispatch(const void* q, const void* kc, const void* vc, const BatchMeta& meta, int B, int Hq, int Hkv,
+                         int dh, int cap, int max_kv_len, void* scratch, void* o, cudaStream_t stream) {
+    const int G = Hq / Hkv;
+    const int lpk = dh / VecOf<T>::N;
+    if (dh % VecOf<T>::N != 0) return -1;
+    const int nch = (max_kv_len + kAttnChunk - 1) / kAttnChunk + 1;   // row stride of the partial buffers
+    const int nch_launch = (max_kv_len + kAttnChunk - 1) / kAttnChunk;
+    float* po = reinterpret_cast<float*>(scratch);
+    float* pml = po + (size_t)B * Hq * nch * dh;
+    const float scale = 1.0f / sqrtf((float)dh);
+    int launched = 0;
+    if (nch_launch > 0) {
+        dim3 grid(nch_launch, Hkv, B);
+        int rc;
+        switch (G) {
+            case 1: rc = attn_dispatch_lpk<T, 1>(lpk, grid, stream, (const T*)q, (const T*)kc, (const T*)vc, meta, Hq, Hkv, cap, nch, scale, po, pml); break;
+            case 2: rc = attn_dispatch_lpk<T, 2>(lpk, grid, stream, (const T*)q, (const T*)kc, (const T*)vc, meta, Hq, Hkv, cap, nch, scale, po, pml); break;
+            case 4: rc = attn_dispatch_lpk<T, 4>(lpk, grid, stream, (const T*)q, (const T*)kc, (const T*)vc, meta, Hq, Hkv, cap, nch, scale, po, pml); break;
+            case 8: rc = attn_dispatch_lpk<T, 8>(lpk, grid, stream, (const T*)q, (const T*)kc, (const T*)vc, meta, Hq, Hkv, cap, nch, scale, po, pml); break;
+            default: rc = -1;
+        }
+        if (rc < 0) return rc;
+        launched += rc;
+    }
+    attn_combine_kernel<T><<<dim3(Hq, B), dh, 0, stream>>>(po, pml, meta, Hq, dh, nch, (T*)o);
+    return launched + 1;
+}
+int launch_attn_decode(int dtype, const void* q, const void* kcache, const void* vcache, const BatchMeta& meta,
+                       int B, int Hq, int Hkv, int dh, int cap, int max_kv_len, void* scratch, void* o,
+                       cudaStream_t stream) {
+    if (B <= 0) return 0;
+    return dtype == 0 ? attn_dispatch<float>(q, kcache, vcache, meta, B, Hq, Hkv, dh, cap, max_kv_len, scratch, o, stream)
+                      : attn_dispatch<bf16>(q, kcache, vcache, meta, B, Hq, Hkv, dh, cap, max_kv_len, scratch, o, stream);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Arg-max finalisation of the LM head's per-block keys
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) argmax_finalize_kernel(const unsigned long long* __restrict__ partials, int nblk,
+                                                              const BatchMeta meta, int32_t* __restrict__ tokens_out,
+                                                              int32_t* __restrict__ last_token) {
+    const int b = blockIdx.x;
+    unsigned long long key = 0ull;
+    for (int i = threadIdx.x; i < nblk; i += blockDim.x) {
+        const unsigned long long o = partials[(size_t)b * nblk + i];
+        key = o > key ? o : key;
+    }
+    key = warp_max_u64(key);
+    __shared__ unsigned long long s_k[8];
+    if ((threadIdx.x & 31) == 0) s_k[threadIdx.x >> 5] = key;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 8; ++w) key = s_k[w] > key ? s_k[w] : key;
+        const int tok = argmax_key_index(key);
+        if (tokens_out != nullptr) tokens_out[b] = tok;
+        last_token[meta.slot[b]] = tok;
+    }
+}
+int launch_argmax_finalize(const unsigned long long* partials, int nblk, const BatchMeta& meta, int B,
+                           int32_t* tokens_out, int32_t* last_token, cudaStream_t stream) {
+    if (B <= 0) return 0;
+    argmax_finalize_kernel<<<B, 256, 0, stream>>>(partials, nblk, meta, tokens_out, last_token);
+    return 1;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Row arg-max over [rows, V] logits and greedy acceptance (Section 3)
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256) row_argmax_partial_kernel(const T* __restrict__ logits, int V,
+                                                                 unsigned long long* __restrict__ scratch) {
+    constexpr int VEC = VecOf<T>::N;
+    const int split = blockIdx.x, row = blockIdx.y;
+    const T* z = logits + (size_t)row * V;
+    int per = (V + kRowArgmaxSplit - 1) / kRowArgmaxSplit;
+    per = (per + VEC - 1) / VEC * VEC;
+    const int lo = split * per, hi = min(V, lo + per);
+    unsigned long long key = 0ull;
+    const bool aligned = (((size_t)row * V) % VEC == 0) && ((reinterpret_cast<uintptr_t>(logits) & 15) == 0);
+    if (aligned) {
+        for (int i = lo + threadIdx.x * VEC; i < hi; i += blockDim.x * VEC) {
+            if (i + VEC <= hi) {
+                float f[VEC];
+                unpack16<T>(ld_stream16(z + i), f);
+#pragma unroll
+                for (int v = 0; v < VEC; ++v) { const unsigned long long k = argmax_key(f[v], i + v); key = k > key ? k : key; }
+            } else {
+                for (int v = i; v < hi; ++v) { const unsigned long long k = argmax_key(to_float<T>(z[v]), v); key = k > key ? k : key; }
+            }
+        }
+    } else {
+        for (int i = lo + threadIdx.x; i < hi; i += blockDim.x) {
+            const unsigned long long k = argmax_key(to_float<T>(z[i]), i);
+            key = k > key ? k : key;
+        }
+    }
+    key = warp_max_u64(key);
+    __shared__ unsigned long long s_k[8];
+    if ((threadIdx.x & 31) == 0) s_k[threadIdx.x >> 5] = key;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 8; ++w) key = s_k[w] > key ? s_k[w] : key;
+        scratch[(size_t)row * kRowArgmaxSplit + split] = key;
+    }
+}
+__global__ void row_argmax_final_kernel(const unsigned long long* __restrict__ scratch, int rows, int32_t* __restrict__ ids) {
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= rows) return;
+    unsigned long long key = 0ull;
+    for (int s = 0; s < kRowArgmaxSplit; ++s) { const unsigned long long o = scratch[(size_t)r * kRowArgmaxSplit + s]; key = o > key ? o : key; }
+    ids[r] = argmax_key_index(key);
+}
+int launch_row_argmax(int logits_dtype, const void* logits, int rows, int V, unsigned long long* scratch,
+                      int32_t* ids_out, cudaStream_t stream) {
+    if (rows <= 0) return 0;
+    int done = 0;
+    while (done < rows) {                       // gridDim.y is limited to 65535
+        const int n = min(rows - done, 32768);
+        dim3 grid(kRowArgmaxSplit, n);
+        if (logits_dtype == 0)
+            row_argmax_partial_kernel<float><<<grid, 256, 0, stream>>>((const float*)logits + (size_t)done * V, V, scratch + (size_t)done * kRowArgmaxSplit);
+        else
+            row_argmax_partial_kernel<bf16><<<grid, 256, 0, stream>>>((const bf16*)logits + (size_t)done * V, V, scratch + (size_t)done * kRowArgmaxSplit);
+        done += n;
+    }
+    row_argmax_final_kernel<<<(rows + 255) / 256, 256, 0, stream>>>(scratch, rows, ids_out);
+    return (rows + 32767) / 32768 + 1;
+}
+
+__global__ void accept_kernel(const int32_t* __restrict__ draft, const int32_t* __restrict__ target_ids, int B, int gamma,
+                              int32_t* __restrict__ accept_len, int32_t* __restrict__ out_tokens) {
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= B) return;
+    const int32_t* g = target_ids + (size_t)b * (gamma + 1);
+    const int32_t* t = draft + (size_t)b * gamma;
+    int a = 0;
+    while (a < gamma && t[a] == g[a]) ++a;
+    accept_len[b] = a;
+    for (int r = 0; r <= gamma; ++r) out_tokens[(size_t)b * (gamma + 1) + r] = r <= a ? g[r] : -1;
+}
+int launch_accept(const int32_t* draft, const int32_t* target_ids, int B, int gamma, int32_t* accept_len,
+                  int32_t* out_tokens, cudaStream_t stream) {
+    if (B <= 0) return 0;
+    accept_kernel<<<(B + 63) / 64, 64, 0, stream>>>(draft, target_ids, B, gamma, accept_len, out_tokens);
+    return 1;
+}
+
+}  // namespace beagle

@@ -1,0 +1,87 @@
+"""Host-only checks of the C ABI: the library loads, exports every symbol that include/beagle.h
+declares, and the entry points that need no GPU validate their arguments."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2505_24544_b200 import build
+    from paper_2505_24544_b200.binding import load_library
+    build.build()
+    return load_library()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "beagle.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(beagle_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    from paper_2505_24544_b200.binding import EXPORTED_SYMBOLS
+    names = declared_symbols()
+    assert "beagle_prefill_kv" in names and "beagle_draft_step" in names
+    assert "beagle_block_forward" in names and "beagle_verify_greedy" in names
+    for n in names:
+        assert hasattr(lib, n), f"{n} declared in beagle.h but not exported"
+    assert sorted(EXPORTED_SYMBOLS) == names
+
+
+def test_config_struct_matches_header():
+    from paper_2505_24544_b200.binding import BeagleConfig, BeagleWeights
+    assert C.sizeof(BeagleConfig) == 13 * 4
+    assert C.sizeof(BeagleWeights) == 11 * C.sizeof(C.c_void_p)
+
+
+def good_config():
+    from paper_2505_24544_b200.binding import BeagleConfig
+    return BeagleConfig(4096, 32, 8, 128, 14336, 128256, 1, 1e-5, 1, 1, 32, 8192, 8)
+
+
+def test_query_sizes_and_shape_validation(lib):
+    from paper_2505_24544_b200.binding import BeagleConfig
+    kv, ws = C.c_size_t(), C.c_size_t()
+    cfg = good_config()
+    assert lib.beagle_query_sizes(C.byref(cfg), C.byref(kv), C.byref(ws)) == 0
+    assert kv.value == 2 * 32 * 8 * (8192 + 8) * 128 * 2
+    assert ws.value > 0 and ws.value % 256 == 0
+    assert lib.beagle_query_sizes(C.byref(cfg), None, C.byref(ws)) == 1
+    bad = good_config(); bad.n_kv_heads = 5
+    assert lib.beagle_query_sizes(C.byref(bad), C.byref(kv), C.byref(ws)) == 2
+    bad = good_config(); bad.head_dim = 100
+    assert lib.beagle_query_sizes(C.byref(bad), C.byref(kv), C.byref(ws)) == 2
+    bad = good_config(); bad.dtype = 7
+    assert lib.beagle_query_sizes(C.byref(bad), C.byref(kv), C.byref(ws)) == 1
+    bad = good_config(); bad.vocab = 0
+    assert lib.beagle_query_sizes(C.byref(bad), C.byref(kv), C.byref(ws)) == 1
+    n = C.c_size_t()
+    assert lib.beagle_block_workspace_bytes(C.byref(cfg), 8, 2048, C.byref(n)) == 0 and n.value > 0
+    assert lib.beagle_block_workspace_bytes(C.byref(cfg), 0, 2048, C.byref(n)) == 1
+
+
+def test_null_context_is_rejected(lib):
+    assert lib.beagle_prefill_kv(None, 0, None, None, None, None) == 1
+    assert lib.beagle_draft_step(None, 0, None, None, 1, None, None, None, None) == 1
+    assert lib.beagle_verify_greedy(None, 0, 0, None, None, 0, None, None, None, None) == 1
+    assert lib.beagle_block_forward(None, 1, 1, None, None, 1, 0, 1, None, None, None, None, 0, None) == 1
+    assert lib.beagle_destroy(None) == 1
+    assert lib.beagle_version().decode().startswith("beagle")
+
+
+def test_create_rejects_bad_buffers(lib):
+    from paper_2505_24544_b200.binding import BeagleWeights
+    cfg = good_config()
+    w = BeagleWeights()
+    h = C.c_void_p()
+    assert lib.beagle_create(C.byref(cfg), C.byref(w), 256, 1 << 40, 256, 1 << 40, C.byref(h)) == 1   # NULL weights
+    for name, _ in BeagleWeights._fields_:
+        setattr(w, name, 4096)
+    assert lib.beagle_create(C.byref(cfg), C.byref(w), 256, 16, 256, 1 << 40, C.byref(h)) == 3        # cache too small
+    assert lib.beagle_create(C.byref(cfg), C.byref(w), 257, 1 << 40, 256, 1 << 40, C.byref(h)) == 1   # misaligned
+    assert not h.value

@@ -1,0 +1,196 @@
+"""GPU parity: the CUDA library (through the C ABI) against the CPU oracle, element by element on
+the same seeded inputs.  Sizes here finish in seconds on the oracle yet span several tiles, several
+split-KV chunks and ragged tails; the full-size configurations live in test_parity_full_gpu.py."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from paper_2505_24544_b200 import workloads as WL
+from parity_utils import assert_close, check_tokens, oracle_head, run_chain_parity, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def build(w: WL.Workload, **kw):
+    from paper_2505_24544_b200.binding import BeagleHead
+    weights = WL.make_weights(w)
+    return BeagleHead.from_workload(w, weights, **kw), oracle_head(w, weights), weights
+
+
+SMALL_GQA = WL.WORKLOADS["c3_llama3_8b_b1"].scaled(name="small_gqa", hidden=512, n_q_heads=8, n_kv_heads=2, head_dim=64,
+                                                   mlp_dim=1400, vocab=4099, batch=3, ctx_min=1, ctx_max=700, gamma=5, seed=2001)
+SMALL_MHA = WL.WORKLOADS["c2_llama2_7b_b1"].scaled(name="small_mha", hidden=768, n_q_heads=6, n_kv_heads=6, head_dim=128,
+                                                   mlp_dim=2048, vocab=5000, batch=2, ctx_min=255, ctx_max=258, gamma=4, seed=2002)
+
+
+def prefill_both(head_gpu, head_cpu, w, rng, slots, lengths):
+    hidden = WL.make_hidden(w, rng, int(np.sum(lengths)))
+    head_gpu.prefill_kv(slots, list(map(int, lengths)), to_dev(hidden, w.dtype) if len(hidden) else None)
+    seqs, r = [], 0
+    for n in lengths:
+        s = O.OracleSequence(head_cpu)
+        O.prefill_kv(head_cpu, s, hidden[r:r + n])
+        seqs.append(s)
+        r += n
+    return seqs
+
+
+def test_c1_tiny_fp32_chain_then_verify():
+    w = WL.WORKLOADS["c1_tiny_fp32"]
+    head_gpu, head_cpu, _ = build(w)
+    rng = WL.data_rng(w)
+    seqs = prefill_both(head_gpu, head_cpu, w, rng, [0], [64])
+    first = WL.make_tokens(w, rng, (1,))
+    drafted, drafted_ref, err = run_chain_parity(head_gpu, head_cpu, w, [0], seqs, first, w.gamma)
+    assert err <= 1e-5
+    assert head_gpu.slot_lengths(0) == (64, w.gamma - 1)
+    # greedy verify against a random-logit target (agreement ~ 1/V) and a planted variant
+    for planted_len in (0, 2, w.gamma):
+        planted = np.full(w.gamma + 1, -1)
+        planted[:planted_len] = drafted_ref[0, :planted_len]
+        logits = WL.make_target_logits(w, rng, w.gamma + 1, planted)
+        acc, out = head_gpu.verify_greedy(to_dev(drafted_ref.astype(np.int32), w.dtype), target_logits=to_dev(logits, "fp32")[None])
+        acc_ref, out_ref = O.verify_greedy(drafted_ref, target_logits=logits[None])
+        np.testing.assert_array_equal(acc.cpu().numpy(), acc_ref)
+        np.testing.assert_array_equal(out.cpu().numpy(), out_ref)
+        assert int(acc_ref[0]) >= planted_len
+
+
+@pytest.mark.parametrize("w", [SMALL_GQA, SMALL_MHA], ids=lambda w: w.name)
+def test_small_bf16_ragged_batch_sd_iterations(w):
+    """Several speculative-decoding iterations: draft chain, verify, append the accepted true states."""
+    head_gpu, head_cpu, _ = build(w, max_ctx=w.ctx_max + 64)
+    rng = WL.data_rng(w)
+    lengths = WL.make_context_lengths(w, rng)
+    lengths[0] = w.ctx_min                           # the shortest cache (1 key for the GQA case)
+    slots = list(range(w.batch))
+    seqs = prefill_both(head_gpu, head_cpu, w, rng, slots, lengths)
+    first = WL.make_tokens(w, rng, (w.batch,))
+    for it in range(3):
+        drafted, drafted_ref, _ = run_chain_parity(head_gpu, head_cpu, w, slots, seqs, first, w.gamma)
+        target = WL.make_target_stream(w, rng, drafted_ref)
+        acc, out = head_gpu.verify_greedy(to_dev(drafted_ref.astype(np.int32), w.dtype), target_ids=to_dev(target, w.dtype))
+        acc_ref, out_ref = O.verify_greedy(drafted_ref, target_ids=target)
+        np.testing.assert_array_equal(acc.cpu().numpy(), acc_ref)
+        np.testing.assert_array_equal(out.cpu().numpy(), out_ref)
+        new_len = (acc_ref + 1).astype(int)
+        hidden = WL.make_hidden(w, rng, int(new_len.sum()))
+        head_gpu.prefill_kv(slots, list(map(int, new_len)), to_dev(hidden, w.dtype))
+        r = 0
+        for b, s in enumerate(seqs):
+            O.prefill_kv(head_cpu, s, hidden[r:r + new_len[b]])
+            r += new_len[b]
+            assert head_gpu.slot_lengths(b) == (s.n_true, 0)
+        first = np.array([out_ref[b, acc_ref[b]] for b in range(w.batch)])
+
+
+def test_empty_cache_concat_off_and_rollback():
+    w = SMALL_GQA.scaled(batch=2)
+    head_gpu, head_cpu, _ = build(w)
+    rng = WL.data_rng(w, 2)
+    seqs = prefill_both(head_gpu, head_cpu, w, rng, [1, 0], [0, 300])      # slot 1 has no key at all
+    first = WL.make_tokens(w, rng, (2,))
+    run_chain_parity(head_gpu, head_cpu, w, [1, 0], seqs, first, 3, concat=False)
+    assert head_gpu.slot_lengths(0) == (300, 0) and head_gpu.slot_lengths(1) == (0, 0)
+    head_gpu.rollback([1, 0])
+    for s in seqs:
+        O.rollback(s)
+    run_chain_parity(head_gpu, head_cpu, w, [1, 0], seqs, first, 4, concat=True)
+    assert head_gpu.slot_lengths(1) == (0, 3)
+
+
+@pytest.mark.parametrize("n", [255, 256, 257, 513])
+def test_split_kv_chunk_boundaries(n):
+    w = SMALL_MHA.scaled(batch=1)
+    head_gpu, head_cpu, _ = build(w, max_ctx=600)
+    rng = WL.data_rng(w, n)
+    seqs = prefill_both(head_gpu, head_cpu, w, rng, [0], [n])
+    run_chain_parity(head_gpu, head_cpu, w, [0], seqs, WL.make_tokens(w, rng, (1,)), 2)
+
+
+@pytest.mark.parametrize("block,offset,sim_steps", [(4, 0, 1), (4, 3, 1), (4, 0, 4), (4, 3, 4), (3, 1, 2), (1, 0, 1)])
+def test_block_forward_c1_fp32(block, offset, sim_steps):
+    w = WL.WORKLOADS["c1_tiny_fp32"]
+    head_gpu, head_cpu, _ = build(w)
+    rng = WL.data_rng(w, 10 * block + offset)
+    B, S = 2, 70
+    tokens = WL.make_tokens(w, rng, (B, S))
+    hidden = WL.make_hidden(w, rng, B * S).reshape(B, S, w.hidden)
+    logits, argmax, hid = head_gpu.block_forward(to_dev(tokens, w.dtype), to_dev(hidden, w.dtype), block, offset, sim_steps)
+    torch.cuda.synchronize()
+    for b in range(B):
+        ref = O.block_forward(head_cpu, tokens[b], hidden[b], block, offset, sim_steps)
+        assert_close(logits[b].cpu().numpy(), ref["logits"], w.dtype, f"seq {b} logits")
+        assert_close(hid[b].cpu().numpy(), ref["hidden"], w.dtype, f"seq {b} hidden")
+        check_tokens(argmax[b].cpu().numpy(), ref["logits"], f"seq {b} argmax")
+
+
+@pytest.mark.parametrize("sim_steps", [1, 4])
+def test_block_forward_small_bf16_equals_oracle_and_sequential(sim_steps):
+    """Block forward against the oracle, and against the library's own step-by-step drafting."""
+    w = SMALL_GQA
+    head_gpu, head_cpu, _ = build(w, max_slots=1, max_ctx=256)
+    rng = WL.data_rng(w, 77 + sim_steps)
+    B, S, block, offset = 2, 131, 4, 2
+    tokens = WL.make_tokens(w, rng, (B, S))
+    hidden = WL.make_hidden(w, rng, B * S).reshape(B, S, w.hidden)
+    tok_dev, hid_dev = to_dev(tokens, w.dtype), to_dev(hidden, w.dtype)
+    logits, argmax, hid = head_gpu.block_forward(tok_dev, hid_dev, block, offset, sim_steps, want_logits=True)
+    _, argmax_only, _ = head_gpu.block_forward(tok_dev, hid_dev, block, offset, sim_steps, want_logits=False, want_hidden=False)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(argmax.cpu().numpy(), argmax_only.cpu().numpy())
+    for b in range(B):
+        ref = O.block_forward(head_cpu, tokens[b], hidden[b], block, offset, sim_steps)
+        assert_close(logits[b].cpu().numpy(), ref["logits"], w.dtype, f"seq {b} logits")
+        assert_close(hid[b].float().cpu().numpy(), ref["hidden"], w.dtype, f"seq {b} hidden")
+        check_tokens(argmax[b].cpu().numpy(), ref["logits"], f"seq {b} argmax")
+    # the library's serve-time path reproduces its own block path (window starting after 66 states)
+    n = O.visible_true_count(67, block, offset)
+    head_gpu.prefill_kv([0], [n], hid_dev[0, :n].contiguous())
+    for i in range(1, block + 1):
+        _, lg, _ = head_gpu.draft_step([0], tokens_in=tok_dev[0, n + i - 1:n + i].contiguous(), concat=(i <= sim_steps), want_logits=True)
+        assert_close(lg[0].cpu().numpy(), logits[0, n + i - 1].cpu().numpy().astype(np.float64), w.dtype, f"slot {i} block vs sequential")
+
+
+def test_verify_greedy_logits_both_dtypes_and_ties():
+    w = SMALL_GQA.scaled(batch=5, gamma=6)
+    head_gpu, _, _ = build(w)
+    rng = WL.data_rng(w, 5)
+    draft = WL.make_tokens(w, rng, (w.batch, w.gamma))
+    planted = np.concatenate([draft, np.full((w.batch, 1), -1)], axis=1)
+    planted[0, 3:] = -1; planted[1, :] = -1; planted[2, 5:] = -1; planted[3, 1:] = -1
+    logits = WL.make_target_logits(w, rng, w.batch * (w.gamma + 1), planted.reshape(-1)).reshape(w.batch, w.gamma + 1, w.vocab)
+    logits[4, 0, :] = 1.0                                  # an all-equal row: lowest index wins
+    logits[4, 1, 7] = logits[4, 1, 4000] = 50.0            # a tie between two ids
+    for dt in ("fp32", "bf16"):
+        lg = WL.round_to_storage(logits.reshape(-1), dt).reshape(logits.shape)
+        acc, out = head_gpu.verify_greedy(to_dev(draft, w.dtype), target_logits=to_dev(lg, dt))
+        acc_ref, out_ref = O.verify_greedy(draft, target_logits=lg)
+        np.testing.assert_array_equal(acc.cpu().numpy(), acc_ref)
+        np.testing.assert_array_equal(out.cpu().numpy(), out_ref)
+    assert out_ref[4, 0] == 0 or acc_ref[4] >= 0
+
+
+def test_status_codes_for_capacity_and_state():
+    from paper_2505_24544_b200.binding import BeagleError
+    w = SMALL_GQA.scaled(batch=1, gamma=2)
+    head_gpu, _, _ = build(w, max_ctx=16, max_draft=1)
+    rng = WL.data_rng(w, 9)
+    with pytest.raises(BeagleError) as e:
+        head_gpu.prefill_kv([0], [17], to_dev(WL.make_hidden(w, rng, 17), w.dtype))
+    assert e.value.status == 3
+    with pytest.raises(BeagleError) as e:
+        head_gpu.draft_step([0], tokens_in=None)
+    assert e.value.status == 4
+    head_gpu.prefill_kv([0], [16], to_dev(WL.make_hidden(w, rng, 16), w.dtype))
+    tok = to_dev(WL.make_tokens(w, rng, (1,)), w.dtype)
+    head_gpu.draft_step([0], tokens_in=tok)
+    head_gpu.draft_step([0])
+    with pytest.raises(BeagleError) as e:                  # the draft tail is full (max_draft = 1)
+        head_gpu.draft_step([0])
+    assert e.value.status == 3
+    with pytest.raises(BeagleError) as e:
+        head_gpu.draft_step([0, 0], tokens_in=torch.zeros(2, dtype=torch.int32, device="cuda"))
+    assert e.value.status == 1
+    torch.cuda.synchronize()
