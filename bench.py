@@ -1,0 +1,626 @@
+#!/usr/bin/env python
+"""Benchmark of the Beagle draft-head hot path on B200.
+
+A "step" is one speculative-decoding iteration over the whole batch of the serving workload:
+append K/V of the true states accepted by the previous verification (beagle_prefill_kv), draft
+gamma tokens (beagle_draft_step x gamma, concat on, tokens fed device-to-device) and run the
+greedy acceptance (beagle_verify_greedy) against a seeded synthetic target stream that agrees with
+the draft at ~70 % per position.  value = drafted tokens per second = batch * gamma * steps / time.
+
+One JSON line is printed by rank 0.  Besides the headline (batched serving, batch 32) the line
+carries the batch-1 workloads, the block-attention forward, the roofline of the dominant kernel
+(from per-stage CUDA events), the end-to-end figure with host buffers and the CPU oracle baseline.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2505_24544_b200 import workloads as WL  # noqa: E402
+
+METRIC = "draft_tokens_per_s"
+UNIT = "draft tokens/s"
+HEADLINE = "c4_llama3_8b_b32"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+# ------------------------------------------------------------------------------------------------ helpers
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS if k in p} | {"source": "measured"}
+    return dict(FALLBACK_PEAKS) | {"source": "fallback"}
+
+
+def load_ncu_traffic():
+    """Per-launch DRAM bytes of the profiled kernels, from the committed ncu summaries."""
+    path = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f)
+    return {}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed regions run."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,utilization.gpu,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(prefix="beagle_clocks_", suffix=".csv")
+            os.close(fd)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.out,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        res = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return res
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        rows = []
+        try:
+            with open(self.path) as f:
+                for line in f:
+                    parts = [p.strip() for p in line.split(",")]
+                    if len(parts) == 8:
+                        rows.append(parts)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if not rows:
+            return res
+        def num(s):
+            try:
+                return float(s)
+            except ValueError:
+                return None
+        busy = [r for r in rows if (num(r[3]) or 0) >= 50] or rows
+        clocks = sorted(c for c in (num(r[0]) for r in busy) if c is not None)
+        res["samples"] = len(busy)
+        if clocks:
+            res["sm_mhz"] = clocks[len(clocks) // 2]
+        mx = [num(r[1]) for r in rows if num(r[1]) is not None]
+        res["sm_max_mhz"] = max(mx) if mx else None
+        pw = [num(r[2]) for r in busy if num(r[2]) is not None]
+        res["power_w_max"] = max(pw) if pw else None
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for i, n in enumerate(names):
+            if any(r[4 + i].lower().startswith("active") for r in busy):
+                res["reasons"].append(n)
+        return res
+
+
+def physical_gpu_index(local: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",")
+    if local < len(vis) and vis[local].strip().isdigit():
+        return int(vis[local])
+    return local
+
+
+def dist_info():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def max_over_ranks(ms: float, world: int, device=None, backend_is_gloo: bool = False) -> float:
+    """The slowest rank's time (MAX all-reduce); identity on one rank."""
+    if world == 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device="cpu" if backend_is_gloo else device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+# ------------------------------------------------------------------------------------------------ serving scenario
+
+class ServeScenario:
+    """Pre-generated, device-resident inputs of `iters` speculative-decoding iterations."""
+
+    def __init__(self, head, w: WL.Workload, iters: int, device):
+        import torch
+        self.torch = torch
+        self.head, self.w, self.iters, self.device = head, w, iters, device
+        self.slots = list(range(w.batch))
+        rng = WL.data_rng(w, 7)
+        self.lengths = WL.make_context_lengths(w, rng)
+        g = torch.Generator(device=device)
+        g.manual_seed(w.seed)
+        dt = head.dtype
+        # context states ~ N(0,1), generated on the device (values are bf16/fp32 representable by construction)
+        self.ctx_hidden = torch.randn(int(self.lengths.sum()), w.hidden, generator=g, device=device, dtype=torch.float32).to(dt)
+        self.new_hidden = torch.randn(iters, w.batch * (w.gamma + 1), w.hidden, generator=g, device=device, dtype=torch.float32).to(dt)
+        self.first_tokens = torch.from_numpy(WL.make_tokens(w, rng, (iters, w.batch))).to(device)
+        self.draft = torch.zeros(iters, w.batch, w.gamma, dtype=torch.int32, device=device)
+        self.accept = torch.zeros(iters, w.batch, dtype=torch.int32, device=device)
+        self.out_tokens = torch.zeros(iters, w.batch, w.gamma + 1, dtype=torch.int32, device=device)
+        self.target_ids = torch.zeros(iters, w.batch, w.gamma + 1, dtype=torch.int32, device=device)
+        self.new_len = [[1] * w.batch for _ in range(iters)]      # rows appended at the START of iteration it
+        self.rng = rng
+
+    def reset(self):
+        from paper_2505_24544_b200 import binding as B
+        for s in self.slots:
+            B.beagle_reset_slot(self.head.ctx, s)
+        self.head.prefill_kv(self.slots, [int(n) for n in self.lengths], self.ctx_hidden)
+
+    def iteration(self, it: int, new_len=None, hidden=None, first=None, target=None):
+        """Enqueues one SD iteration; nothing here synchronises."""
+        from paper_2505_24544_b200 import binding as B
+        w, head = self.w, self.head
+        nl = self.new_len[it] if new_len is None else new_len
+        hid = self.new_hidden[it] if hidden is None else hidden
+        if it > 0:
+            B.beagle_prefill_kv(head.ctx, self.slots, nl, hid)
+        first = self.first_tokens[it] if first is None else first
+        for s in range(w.gamma):
+            B.beagle_draft_step(head.ctx, self.slots, first if s == 0 else None, True, self.draft[it, :, s])
+        B.beagle_verify_greedy(head.ctx, self.draft[it], None, self.target_ids[it] if target is None else target,
+                               self.accept[it], self.out_tokens[it])
+
+    def rehearse(self):
+        """Runs every iteration once (untimed) to learn the draft tokens, builds the ~70 %-agreement
+        target stream from them and records how many true states each iteration appends."""
+        torch = self.torch
+        self.reset()
+        for it in range(self.iters):
+            w = self.w
+            from paper_2505_24544_b200 import binding as B
+            if it > 0:
+                B.beagle_prefill_kv(self.head.ctx, self.slots, self.new_len[it], self.new_hidden[it])
+            for s in range(w.gamma):
+                B.beagle_draft_step(self.head.ctx, self.slots, self.first_tokens[it] if s == 0 else None, True, self.draft[it, :, s])
+            torch.cuda.synchronize()
+            draft = self.draft[it].cpu().numpy()
+            target = WL.make_target_stream(w, self.rng, draft)
+            self.target_ids[it].copy_(torch.from_numpy(target))
+            a = 0
+            acc = np.zeros(w.batch, dtype=np.int64)
+            for b in range(w.batch):
+                a = 0
+                while a < w.gamma and draft[b, a] == target[b, a]:
+                    a += 1
+                acc[b] = a
+            if it + 1 < self.iters:
+                self.new_len[it + 1] = [int(a) + 1 for a in acc]
+        self.mean_tau = float(np.mean([np.mean(n) for n in self.new_len[1:]])) if self.iters > 1 else None
+
+
+def time_serve(scn: ServeScenario, steps: int, warmup: int, world: int):
+    """Device-resident timing: W untimed + K timed iterations, CUDA events, barrier on both sides."""
+    import torch
+    scn.reset()
+    for it in range(warmup):
+        scn.iteration(it)
+    torch.cuda.synchronize()
+    if world > 1:
+        torch.distributed.barrier()
+    l0 = scn.head.launch_count
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for it in range(warmup, warmup + steps):
+        scn.iteration(it)
+    e1.record()
+    torch.cuda.synchronize()
+    if world > 1:
+        torch.distributed.barrier()
+    return e0.elapsed_time(e1), scn.head.launch_count - l0
+
+
+def profile_serve(scn: ServeScenario, steps: int, warmup: int):
+    """Same iterations with every stage bracketed by CUDA events inside the library."""
+    import torch
+    from paper_2505_24544_b200 import binding as B
+    scn.reset()
+    for it in range(warmup):
+        scn.iteration(it)
+    torch.cuda.synchronize()
+    B.beagle_profile_enable(scn.head.ctx, True)
+    for it in range(warmup, warmup + steps):
+        scn.iteration(it)
+    torch.cuda.synchronize()
+    stages = B.beagle_profile_read(scn.head.ctx)
+    B.beagle_profile_enable(scn.head.ctx, False)
+    return stages
+
+
+def time_serve_e2e(scn: ServeScenario, steps: int, warmup: int, world: int):
+    """End to end through the binding with HOST buffers: every iteration copies its new true
+    states, first tokens and target ids from pinned host memory and reads accept lengths and
+    emitted tokens back; the host's bookkeeping uses the values it read."""
+    import torch
+    w = scn.w
+    dev = scn.device
+    rows = w.batch * (w.gamma + 1)
+    host_hidden = scn.new_hidden.cpu().pin_memory()
+    host_first = scn.first_tokens.cpu().pin_memory()
+    host_target = scn.target_ids.cpu().pin_memory()
+    stage_h = torch.empty(rows, w.hidden, dtype=scn.head.dtype).pin_memory()
+    dev_h = torch.empty(rows, w.hidden, dtype=scn.head.dtype, device=dev)
+    dev_first = torch.empty(w.batch, dtype=torch.int32, device=dev)
+    dev_target = torch.empty(w.batch, w.gamma + 1, dtype=torch.int32, device=dev)
+    host_acc = torch.empty(w.batch, dtype=torch.int32).pin_memory()
+    host_out = torch.empty(w.batch, w.gamma + 1, dtype=torch.int32).pin_memory()
+    scn.reset()
+    new_len = [1] * w.batch
+    h2d = d2h = 0
+
+    def one(it, count):
+        nonlocal new_len, h2d, d2h
+        if it > 0:
+            r = 0
+            for b in range(w.batch):                       # pack the accepted rows of every sequence
+                n = new_len[b]
+                stage_h[r:r + n].copy_(host_hidden[it, b * (w.gamma + 1): b * (w.gamma + 1) + n])
+                r += n
+            dev_h[:r].copy_(stage_h[:r], non_blocking=True)
+            if count:
+                h2d += r * w.hidden * stage_h.element_size()
+        dev_first.copy_(host_first[it], non_blocking=True)
+        dev_target.copy_(host_target[it], non_blocking=True)
+        if count:
+            h2d += dev_first.numel() * 4 + dev_target.numel() * 4
+        scn.iteration(it, new_len=new_len, hidden=dev_h, first=dev_first, target=dev_target)
+        host_acc.copy_(scn.accept[it], non_blocking=True)
+        host_out.copy_(scn.out_tokens[it], non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        if count:
+            d2h += (host_acc.numel() + host_out.numel()) * 4
+        new_len = [int(a) + 1 for a in host_acc.tolist()]
+
+    for it in range(warmup):
+        one(it, False)
+    torch.cuda.synchronize()
+    if world > 1:
+        torch.distributed.barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for it in range(warmup, warmup + steps):
+        one(it, True)
+    e1.record()
+    torch.cuda.synchronize()
+    if world > 1:
+        torch.distributed.barrier()
+    return e0.elapsed_time(e1), h2d / steps, d2h / steps
+
+
+# ------------------------------------------------------------------------------------------------ byte / flop accounting
+
+def elt(w):
+    return 2 if w.dtype == "bf16" else 4
+
+
+def step_bytes(w: WL.Workload, mean_ctx: float):
+    """Algorithmic HBM bytes of one draft step of the whole batch (weights once + K/V per sequence)."""
+    e, d, qd, kd, m, V = elt(w), w.hidden, w.n_q_heads * w.head_dim, w.n_kv_heads * w.head_dim, w.mlp_dim, w.vocab
+    weights = e * (2 * d * qd + 2 * d * kd + 3 * d * m + V * d)
+    kv = w.batch * 2 * kd * mean_ctx * e
+    return weights + kv
+
+
+def stage_bytes(w: WL.Workload, stage: str, mean_ctx: float):
+    e, d, qd, kd, m, V, B = elt(w), w.hidden, w.n_q_heads * w.head_dim, w.n_kv_heads * w.head_dim, w.mlp_dim, w.vocab, w.batch
+    return {
+        "lm_head": e * (V * d + B * d),
+        "gate_up": e * (2 * m * d + B * d + B * m),
+        "down_proj": e * (d * m + B * m + 2 * B * d),
+        "q_proj": e * (qd * d + B * d + B * qd),
+        "o_proj": e * (d * qd + B * qd + 2 * B * d),
+        "kv_append": e * (2 * kd * d + B * d + 2 * B * kd),
+        "attn_decode": e * (B * 2 * kd * mean_ctx + 2 * B * qd),
+    }.get(stage)
+
+
+# ------------------------------------------------------------------------------------------------ CPU oracle legs
+
+def oracle_sample(w: WL.Workload, n_seq: int, iters: int, warm: int = 0):
+    """Times the CPU oracle, as it stands, on `n_seq` sequences of the workload for `iters` SD
+    iterations (context prefill untimed).  Returns (draft tokens/s, seconds, threads)."""
+    import oracle as O
+    weights = WL.make_weights(w)
+    head = O.OracleHead(O.HeadConfig(w.hidden, w.n_q_heads, w.n_kv_heads, w.head_dim, w.mlp_dim, w.vocab, rms_eps=w.rms_eps), weights)
+    del weights
+    rng = WL.data_rng(w, 7)
+    lengths = WL.make_context_lengths(w, rng)[:n_seq]
+    seqs = []
+    for n in lengths:
+        s = O.OracleSequence(head)
+        O.prefill_kv(head, s, WL.make_hidden(w, rng, int(n)))
+        seqs.append(s)
+    new_len = [1] * n_seq
+    first = WL.make_tokens(w, rng, (n_seq,))
+    t0 = time.perf_counter()
+    for it in range(-warm, iters):
+        if it == 0:
+            t0 = time.perf_counter()
+        if it != -warm:
+            for b, s in enumerate(seqs):
+                O.prefill_kv(head, s, WL.make_hidden(w, rng, new_len[b]))
+        drafted = np.zeros((n_seq, w.gamma), dtype=np.int64)
+        for st in range(w.gamma):
+            out = O.draft_step(head, seqs, tokens_in=list(first) if st == 0 else None, concat=True)
+            drafted[:, st] = out["argmax"]
+        target = WL.make_target_stream(w, rng, drafted)
+        acc, out_tok = O.verify_greedy(drafted, target_ids=target)
+        new_len = [int(a) + 1 for a in acc]
+        first = np.array([out_tok[b, acc[b]] for b in range(n_seq)])
+    dt = time.perf_counter() - t0
+    threads = os.cpu_count() or 1
+    try:
+        from threadpoolctl import threadpool_info
+        nt = [p.get("num_threads") for p in threadpool_info() if p.get("user_api") == "blas"]
+        if nt:
+            threads = max(nt)
+    except Exception:
+        pass
+    return n_seq * w.gamma * iters / dt, dt, threads
+
+
+def run_reference(args):
+    """`--impl reference`: the CPU oracle, unmodified, on the host cores (rank 0 only)."""
+    rank, world, _ = dist_info()
+    if rank != 0:
+        return
+    w = WL.WORKLOADS[args.workload]
+    n_seq = min(2, w.batch)
+    steps = max(1, min(args.steps, 3))
+    warm = 1 if args.warmup > 0 else 0
+    t0 = time.perf_counter()
+    val, sec, threads = oracle_sample(w, n_seq, steps, warm)
+    sample = f"{n_seq} of {w.batch} sequences x {steps} SD iteration(s) of {w.gamma} draft tokens, context prefill untimed"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+        "warmup": warm, "ms_per_step": 1e3 * sec / steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "batch": w.batch, "gamma": w.gamma, "ctx": [w.ctx_min, w.ctx_max], "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0, "wall_s": time.perf_counter() - t0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------ block forward
+
+def bench_block(head, w: WL.Workload, steps: int, warmup: int, peaks):
+    import torch
+    from paper_2505_24544_b200 import binding as B
+    dev = head.device
+    g = torch.Generator(device=dev)
+    g.manual_seed(w.seed)
+    S = w.ctx_max
+    tokens = torch.randint(0, w.vocab, (w.batch, S), generator=g, device=dev, dtype=torch.int32)
+    hidden = torch.randn(w.batch, S, w.hidden, generator=g, device=dev, dtype=torch.float32).to(head.dtype)
+    argmax = torch.empty(w.batch, S, dtype=torch.int32, device=dev)
+
+    def run():
+        B.beagle_block_forward(head.ctx, tokens, hidden, w.block, 0, 1, None, argmax, None)
+
+    for _ in range(warmup):
+        run()
+    torch.cuda.synchronize()
+    l0 = head.launch_count
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        run()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    launches = (head.launch_count - l0) // steps
+    B.beagle_profile_enable(head.ctx, True)
+    run()
+    torch.cuda.synchronize()
+    stages = B.beagle_profile_read(head.ctx)
+    B.beagle_profile_enable(head.ctx, False)
+    M = w.batch * S
+    d, qd, kd, m, V = w.hidden, w.n_q_heads * w.head_dim, w.n_kv_heads * w.head_dim, w.mlp_dim, w.vocab
+    flops = {"blk_lm_head": 2.0 * M * V * d, "blk_gate_up": 4.0 * M * m * d, "blk_down": 2.0 * M * m * d,
+             "blk_qkv": 2.0 * M * d * (qd + 2 * kd), "blk_o_proj": 2.0 * M * d * qd}
+    vis = sum(WL_vis(p, w.block) for p in range(1, S + 1)) * w.batch
+    flops["blk_attn"] = 4.0 * w.head_dim * w.n_q_heads * vis
+    total = sum(flops.values())
+    st = {k: {"ms": v[0], "tflops": (flops[k] / (v[0] * 1e-3) / 1e12) if k in flops and v[0] > 0 else None} for k, v in stages.items()}
+    lm = st.get("blk_lm_head", {})
+    peak = peaks["bf16_tflops_sustained"]
+    return {
+        "workload": w.name, "positions_per_s": M / (ms * 1e-3), "ms_per_forward": ms, "tflop_per_forward": total / 1e12,
+        "tflops": total / (ms * 1e-3) / 1e12, "gpu_launches": launches, "stages": st,
+        "roofline": {"bound": "tensor", "kernel": "blk_lm_head", "achieved": lm.get("tflops"), "peak": peak, "unit": "TFLOP/s",
+                     "frac": (lm.get("tflops") / peak) if lm.get("tflops") else None, "traffic": None,
+                     "peak_source": peaks["source"] + " (sustained)"},
+    }
+
+
+def WL_vis(p: int, block: int, offset: int = 0) -> int:
+    """Visible true keys of position p under the inverse block mask (flop accounting only)."""
+    return p - 1 if p <= offset else offset + block * ((p - 1 - offset) // block)
+
+
+# ------------------------------------------------------------------------------------------------ main
+
+def serve_result(scn, w, ms, steps, world):
+    total_tokens = world * w.batch * w.gamma * steps
+    return total_tokens / (ms * 1e-3)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=HEADLINE, choices=[k for k in WL.WORKLOADS if not k.startswith("c5")])
+    ap.add_argument("--only-headline", action="store_true", help="skip the batch-1, block-forward and CPU legs")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+    args.warmup = max(args.warmup, 3)
+
+    import torch
+    from paper_2505_24544_b200 import build as _build
+    _build.build()
+    from paper_2505_24544_b200 import binding as B
+    from paper_2505_24544_b200.binding import BeagleHead
+
+    rank, world, local = dist_info()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        torch.distributed.init_process_group("nccl", device_id=device)
+    peaks = load_peaks()
+    traffic = load_ncu_traffic()
+    t_wall = time.perf_counter()
+
+    w = WL.WORKLOADS[args.workload]
+    iters = args.steps + args.warmup
+    extra = iters * (w.gamma + 1) + 64
+    max_draft = max(x.gamma for x in WL.WORKLOADS.values())
+    weights = WL.make_weights(w)
+    head = BeagleHead.from_workload(w, weights, device=device, max_slots=w.batch, max_ctx=w.ctx_max + extra, max_draft=max_draft)
+    del weights
+
+    sampler = ClockSampler(physical_gpu_index(local))
+    scn = ServeScenario(head, w, iters, device)
+    scn.rehearse()
+    sampler.start()
+    ms, launches = time_serve(scn, args.steps, args.warmup, world)
+    ms = max_over_ranks(ms, world, device)
+    value = serve_result(scn, w, ms, args.steps, world)
+    stages = profile_serve(scn, args.steps, args.warmup)
+    e2e_ms, h2d, d2h = time_serve_e2e(scn, args.steps, args.warmup, world)
+    e2e_ms = max_over_ranks(e2e_ms, world, device)
+    e2e_value = serve_result(scn, w, e2e_ms, args.steps, world)
+    mean_ctx = float(scn.lengths.mean()) + (args.warmup + args.steps / 2) * (scn.mean_tau or 1.0)
+
+    stage_out = {}
+    for name, (sms, cnt) in stages.items():
+        per = sms / cnt
+        by = stage_bytes(w, name, mean_ctx)
+        stage_out[name] = {"us_per_launch": 1e3 * per, "launches": cnt, "share": sms / max(1e-9, sum(v[0] for v in stages.values())),
+                           "gbs": (by / (per * 1e-3) / 1e9) if by else None}
+    dom = max((k for k in stage_out if stage_out[k]["gbs"]), key=lambda k: stage_out[k]["share"])
+    achieved = stage_out[dom]["gbs"]
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": achieved / peaks["hbm_gbs"], "traffic": traffic.get(f"{dom}@{w.name}"),
+                "algorithmic_bytes_per_launch": stage_bytes(w, dom, mean_ctx), "peak_source": peaks["source"],
+                "attn_decode_gbs": stage_out.get("attn_decode", {}).get("gbs"),
+                "attn_decode_frac": (stage_out["attn_decode"]["gbs"] / peaks["hbm_gbs"]) if stage_out.get("attn_decode", {}).get("gbs") else None}
+    step_gb = step_bytes(w, mean_ctx) * w.gamma / 1e9
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": w.name, "batch": w.batch, "gamma": w.gamma, "ctx": [w.ctx_min, w.ctx_max],
+                   "hidden": w.hidden, "heads": [w.n_q_heads, w.n_kv_heads, w.head_dim], "mlp": w.mlp_dim, "vocab": w.vocab,
+                   "step": "one SD iteration: prefill_kv(accepted states) + gamma x draft_step(concat) + verify_greedy",
+                   "l2": "inputs larger than L2 (weights %.2f GB + K/V per draft step)" % (step_bytes(w, mean_ctx) / 1e9),
+                   "mean_tau": scn.mean_tau, "parallelism": "replicas" if world > 1 else "single"},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps},
+        "gpu_launches": launches,
+        "roofline": roofline,
+        "step_hbm": {"algorithmic_gb_per_step": step_gb, "achieved_gbs": step_gb / (ms / args.steps * 1e-3),
+                     "frac_of_peak": step_gb / (ms / args.steps * 1e-3) / peaks["hbm_gbs"]},
+        "stages": stage_out,
+    }
+
+    if not args.only_headline and world == 1:
+        # batch-1 serving on the same head (Llama-3-8B shape) and on the Llama-2-7B shaped head
+        others = {}
+        if w.name == HEADLINE:
+            w3 = WL.WORKLOADS["c3_llama3_8b_b1"]
+            scn3 = ServeScenario(head, w3, iters, device)
+            scn3.rehearse()
+            ms3, l3 = time_serve(scn3, args.steps, args.warmup, 1)
+            st3 = profile_serve(scn3, args.steps, args.warmup)
+            others[w3.name] = summarize_b1(w3, scn3, ms3, l3, st3, args, peaks)
+            del scn3
+        del scn
+        head.ctx.close()
+        del head
+        torch.cuda.empty_cache()
+        w2 = WL.WORKLOADS["c2_llama2_7b_b1"]
+        w5 = WL.WORKLOADS["c5_block_llama2_7b"]
+        weights2 = WL.make_weights(w2)
+        head2 = BeagleHead.from_workload(w2, weights2, device=device, max_slots=1, max_ctx=w2.ctx_max + extra, max_draft=max_draft)
+        del weights2
+        scn2 = ServeScenario(head2, w2, iters, device)
+        scn2.rehearse()
+        ms2, l2 = time_serve(scn2, args.steps, args.warmup, 1)
+        st2 = profile_serve(scn2, args.steps, args.warmup)
+        others[w2.name] = summarize_b1(w2, scn2, ms2, l2, st2, args, peaks)
+        line["batch1"] = others
+        del scn2
+        line["block_forward"] = bench_block(head2, w5, steps=max(2, min(5, args.steps)), warmup=3, peaks=peaks)
+        head2.ctx.close()
+        del head2
+        torch.cuda.empty_cache()
+    line["clocks"] = sampler.stop()
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.only_headline:
+        n_seq = min(2, w.batch)
+        val, sec, threads = oracle_sample(w, n_seq, 1)
+        line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": sec,
+                                "sample": f"{n_seq} of {w.batch} sequences x 1 SD iteration of {w.gamma} draft tokens, context prefill untimed"}
+    line["wall_s"] = time.perf_counter() - t_wall
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def summarize_b1(w, scn, ms, launches, stages, args, peaks):
+    mean_ctx = float(scn.lengths.mean()) + (args.warmup + args.steps / 2) * (scn.mean_tau or 1.0)
+    gb = step_bytes(w, mean_ctx) * w.gamma / 1e9
+    per_step = ms / args.steps
+    out = {"value": w.batch * w.gamma * args.steps / (ms * 1e-3), "unit": UNIT, "ms_per_step": per_step, "gpu_launches": launches,
+           "mean_tau": scn.mean_tau, "algorithmic_gb_per_step": gb, "achieved_gbs": gb / (per_step * 1e-3),
+           "frac_of_hbm_peak": gb / (per_step * 1e-3) / peaks["hbm_gbs"], "stages": {}}
+    tot = sum(v[0] for v in stages.values())
+    for name, (sms, cnt) in stages.items():
+        by = stage_bytes(w, name, mean_ctx)
+        per = sms / cnt
+        out["stages"][name] = {"us_per_launch": 1e3 * per, "share": sms / tot, "gbs": (by / (per * 1e-3) / 1e9) if by else None}
+    return out
+
+
+if __name__ == "__main__":
+    main()

@@ -112,12 +112,14 @@ beagle_status beagle_prefill_kv(beagle_ctx* ctx, int32_t batch, const int32_t* s
  * concat != 0: the previous step's output state h of the slot is projected and appended to the
  *   cache tail before attending (the paper's default, "concate"); 0: only states already in the
  *   cache are read and the previous state is discarded.
- * Outputs (any may be NULL): tokens_out_dev int32 [batch]; logits_out_dev fp32 [batch, V];
+ * Outputs (any may be NULL): tokens_out_dev int32, row b at tokens_out_dev[b * tokens_out_stride]
+ *   (stride 1 = dense [batch]; stride gamma with a base of draft + s fills column s of a
+ *   [batch, gamma] draft matrix for beagle_verify_greedy); logits_out_dev fp32 [batch, V];
  *   hidden_out_dev storage type [batch, d]. */
 beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* seq_slot_host,
                                 const int32_t* tokens_in_dev, int32_t concat,
-                                int32_t* tokens_out_dev, float* logits_out_dev, void* hidden_out_dev,
-                                void* stream);
+                                int32_t* tokens_out_dev, int32_t tokens_out_stride,
+                                float* logits_out_dev, void* hidden_out_dev, void* stream);
 
 /* Drops the draft tail of the listed slots (cache back to true states only). */
 beagle_status beagle_rollback(beagle_ctx* ctx, int32_t batch, const int32_t* seq_slot_host);
@@ -153,6 +155,16 @@ beagle_status beagle_verify_greedy(beagle_ctx* ctx, int32_t batch, int32_t gamma
                                    const int32_t* draft_tokens_dev, const void* target_logits_dev,
                                    int32_t logits_dtype, const int32_t* target_ids_dev,
                                    int32_t* accept_len_dev, int32_t* out_tokens_dev, void* stream);
+
+/* Optional per-stage timing (no counterpart in the paper; measurement support).  While enabled,
+ * every stage of every entry point is bracketed by a pair of CUDA events recorded on the call's
+ * stream.  beagle_profile_read waits for the recorded events, writes the accumulated milliseconds
+ * and the number of bracketed stage instances into two HOST arrays of beagle_profile_stage_count()
+ * entries, and clears the record.  Stage names: beagle_profile_stage_name(i). */
+beagle_status beagle_profile_enable(beagle_ctx* ctx, int32_t on);
+beagle_status beagle_profile_read(beagle_ctx* ctx, float* ms_out_host, int32_t* count_out_host);
+int32_t beagle_profile_stage_count(void);
+const char* beagle_profile_stage_name(int32_t stage);
 
 /* Text of the last error recorded on this context ("" if none). */
 const char* beagle_last_error(const beagle_ctx* ctx);

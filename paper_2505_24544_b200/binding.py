@@ -25,7 +25,8 @@ EXPORTED_SYMBOLS = (
     "beagle_version", "beagle_query_sizes", "beagle_create", "beagle_destroy", "beagle_prefill_kv",
     "beagle_draft_step", "beagle_rollback", "beagle_reset_slot", "beagle_slot_lengths",
     "beagle_block_workspace_bytes", "beagle_block_forward", "beagle_verify_greedy", "beagle_last_error",
-    "beagle_launch_count",
+    "beagle_launch_count", "beagle_profile_enable", "beagle_profile_read", "beagle_profile_stage_count",
+    "beagle_profile_stage_name",
 )
 
 
@@ -67,7 +68,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.beagle_create.argtypes = [C.POINTER(BeagleConfig), C.POINTER(BeagleWeights), vp, C.c_size_t, vp, C.c_size_t, C.POINTER(vp)]
     lib.beagle_destroy.argtypes = [vp]
     lib.beagle_prefill_kv.argtypes = [vp, i32, i32p, i32p, vp, vp]
-    lib.beagle_draft_step.argtypes = [vp, i32, i32p, vp, i32, vp, vp, vp, vp]
+    lib.beagle_draft_step.argtypes = [vp, i32, i32p, vp, i32, vp, i32, vp, vp, vp]
     lib.beagle_rollback.argtypes = [vp, i32, i32p]
     lib.beagle_reset_slot.argtypes = [vp, i32]
     lib.beagle_slot_lengths.argtypes = [vp, i32, i32p, i32p]
@@ -76,6 +77,14 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.beagle_verify_greedy.argtypes = [vp, i32, i32, vp, vp, i32, vp, vp, vp, vp]
     lib.beagle_last_error.restype = C.c_char_p
     lib.beagle_last_error.argtypes = [vp]
+    lib.beagle_profile_enable.argtypes = [vp, i32]
+    lib.beagle_profile_enable.restype = C.c_int
+    lib.beagle_profile_read.argtypes = [vp, C.POINTER(C.c_float), i32p]
+    lib.beagle_profile_read.restype = C.c_int
+    lib.beagle_profile_stage_count.argtypes = []
+    lib.beagle_profile_stage_count.restype = C.c_int32
+    lib.beagle_profile_stage_name.argtypes = [i32]
+    lib.beagle_profile_stage_name.restype = C.c_char_p
     lib.beagle_launch_count.restype = C.c_int64
     lib.beagle_launch_count.argtypes = [vp]
     for name in ("beagle_query_sizes", "beagle_create", "beagle_destroy", "beagle_prefill_kv", "beagle_draft_step",
@@ -168,8 +177,14 @@ def beagle_prefill_kv(ctx: Context, seq_slot: Sequence[int], new_len: Sequence[i
 def beagle_draft_step(ctx: Context, seq_slot: Sequence[int], tokens_in: Optional[torch.Tensor], concat: bool,
                       tokens_out: Optional[torch.Tensor], logits_out: Optional[torch.Tensor] = None,
                       hidden_out: Optional[torch.Tensor] = None) -> None:
+    """tokens_out may be a dense [batch] tensor or one column of a [batch, gamma] draft matrix."""
+    stride, out_ptr = 1, None
+    if tokens_out is not None:
+        if tokens_out.dim() != 1 or tokens_out.dtype != torch.int32:
+            raise ValueError("tokens_out must be a 1-D int32 tensor (a column view is fine)")
+        stride, out_ptr = int(tokens_out.stride(0)), tokens_out.data_ptr()
     ctx.check(ctx.lib.beagle_draft_step(ctx.handle, len(seq_slot), _i32_array(seq_slot), _ptr(tokens_in), int(bool(concat)),
-                                        _ptr(tokens_out), _ptr(logits_out), _ptr(hidden_out), _stream()))
+                                        out_ptr, stride, _ptr(logits_out), _ptr(hidden_out), _stream()))
 
 
 def beagle_rollback(ctx: Context, seq_slot: Sequence[int]) -> None:
@@ -218,6 +233,18 @@ def beagle_verify_greedy(ctx: Context, draft_tokens: torch.Tensor, target_logits
             raise ValueError("target_logits must be float32 or bfloat16")
     ctx.check(ctx.lib.beagle_verify_greedy(ctx.handle, batch, gamma, _ptr(draft_tokens), _ptr(target_logits), code,
                                            _ptr(target_ids), _ptr(accept_len), _ptr(out_tokens), _stream()))
+
+
+def beagle_profile_enable(ctx: Context, on: bool) -> None:
+    ctx.check(ctx.lib.beagle_profile_enable(ctx.handle, int(bool(on))))
+
+
+def beagle_profile_read(ctx: Context) -> Dict[str, Tuple[float, int]]:
+    """{stage name: (accumulated ms, bracketed instances)} since the last read; synchronises."""
+    n = ctx.lib.beagle_profile_stage_count()
+    ms, cnt = (C.c_float * n)(), (C.c_int32 * n)()
+    ctx.check(ctx.lib.beagle_profile_read(ctx.handle, ms, cnt))
+    return {ctx.lib.beagle_profile_stage_name(i).decode(): (float(ms[i]), int(cnt[i])) for i in range(n) if cnt[i]}
 
 
 # ---- convenience wrapper -----------------------------------------------------------------------

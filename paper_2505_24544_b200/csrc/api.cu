@@ -12,6 +12,18 @@
 
 using namespace beagle;
 
+enum Stage {
+    ST_KV_APPEND = 0, ST_EMBED_NORM, ST_Q_PROJ, ST_ATTN_DECODE, ST_O_PROJ, ST_MLP_NORM, ST_GATE_UP, ST_DOWN, ST_LM_HEAD,
+    ST_ARGMAX, ST_PREFILL, ST_VERIFY, ST_BLK_EMBED, ST_BLK_QKV, ST_BLK_PRED_KV, ST_BLK_ATTN, ST_BLK_O, ST_BLK_NORM,
+    ST_BLK_GATE_UP, ST_BLK_DOWN, ST_BLK_LM_HEAD, ST_BLK_ARGMAX, ST_COUNT
+};
+static const char* const kStageNames[ST_COUNT] = {
+    "kv_append", "embed_norm", "q_proj", "attn_decode", "o_proj", "mlp_norm", "gate_up", "down_proj", "lm_head",
+    "argmax_finalize", "prefill_kv", "verify", "blk_embed", "blk_qkv", "blk_pred_kv", "blk_attn", "blk_o_proj", "blk_norm",
+    "blk_gate_up", "blk_down", "blk_lm_head", "blk_argmax"};
+
+struct StageRecord { int stage; cudaEvent_t start, stop; };
+
 struct beagle_ctx {
     beagle_config cfg;
     beagle_weights w;
@@ -36,7 +48,39 @@ struct beagle_ctx {
     std::string err;
     int64_t launches = 0;
     TcPlan* tc = nullptr;           // tensor-core GEMM plans (bf16 only)
+    // optional per-stage timing with CUDA events (off by default)
+    bool profiling = false;
+    std::vector<StageRecord> records;
+    std::vector<std::pair<cudaEvent_t, cudaEvent_t>> free_events;
 };
+
+namespace {
+// Brackets one stage with events on the call's stream while profiling is on.
+struct StageTimer {
+    beagle_ctx* ctx;
+    cudaStream_t stream;
+    StageRecord rec;
+    bool on;
+    StageTimer(beagle_ctx* c, int stage, cudaStream_t s) : ctx(c), stream(s), on(c->profiling) {
+        if (!on) return;
+        rec.stage = stage;
+        if (!ctx->free_events.empty()) {
+            rec.start = ctx->free_events.back().first;
+            rec.stop = ctx->free_events.back().second;
+            ctx->free_events.pop_back();
+        } else if (cudaEventCreate(&rec.start) != cudaSuccess || cudaEventCreate(&rec.stop) != cudaSuccess) {
+            on = false;
+            return;
+        }
+        cudaEventRecord(rec.start, stream);
+    }
+    ~StageTimer() {
+        if (!on) return;
+        cudaEventRecord(rec.stop, stream);
+        ctx->records.push_back(rec);
+    }
+};
+}  // namespace
 
 namespace {
 
@@ -202,8 +246,40 @@ beagle_status beagle_create(const beagle_config* cfg, const beagle_weights* w, v
     return BEAGLE_OK;
 }
 
+static void release_events(beagle_ctx* ctx) {
+    for (auto& r : ctx->records) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
+    for (auto& e : ctx->free_events) { cudaEventDestroy(e.first); cudaEventDestroy(e.second); }
+    ctx->records.clear();
+    ctx->free_events.clear();
+}
+
+beagle_status beagle_profile_enable(beagle_ctx* ctx, int32_t on) {
+    if (ctx == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    ctx->profiling = on != 0;
+    return BEAGLE_OK;
+}
+
+int32_t beagle_profile_stage_count(void) { return ST_COUNT; }
+const char* beagle_profile_stage_name(int32_t stage) { return (stage >= 0 && stage < ST_COUNT) ? kStageNames[stage] : ""; }
+
+beagle_status beagle_profile_read(beagle_ctx* ctx, float* ms_out, int32_t* count_out) {
+    if (ctx == nullptr || ms_out == nullptr || count_out == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    for (int i = 0; i < ST_COUNT; ++i) { ms_out[i] = 0.f; count_out[i] = 0; }
+    for (auto& r : ctx->records) {
+        if (cudaEventSynchronize(r.stop) != cudaSuccess) return fail(ctx, BEAGLE_ERR_CUDA, "profile_read: event sync failed");
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, r.start, r.stop) != cudaSuccess) return fail(ctx, BEAGLE_ERR_CUDA, "profile_read: elapsed time failed");
+        ms_out[r.stage] += ms;
+        count_out[r.stage] += 1;
+        ctx->free_events.emplace_back(r.start, r.stop);
+    }
+    ctx->records.clear();
+    return BEAGLE_OK;
+}
+
 beagle_status beagle_destroy(beagle_ctx* ctx) {
     if (ctx == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    release_events(ctx);
     tc_plan_destroy(ctx->tc);
     delete ctx;
     return BEAGLE_OK;
@@ -271,6 +347,7 @@ beagle_status beagle_prefill_kv(beagle_ctx* ctx, int32_t batch, const int32_t* s
     const beagle_config& c = ctx->cfg;
 
     if (total > 0) {
+        StageTimer timer_(ctx, ST_PREFILL, stream);
         SeqRows rows;
         memset(&rows, 0, sizeof(rows));
         int n = 0, r = 0;
@@ -326,12 +403,13 @@ beagle_status beagle_prefill_kv(beagle_ctx* ctx, int32_t batch, const int32_t* s
 }
 
 beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* seq_slot, const int32_t* tokens_in_dev,
-                                int32_t concat, int32_t* tokens_out_dev, float* logits_out_dev, void* hidden_out_dev,
-                                void* stream_) {
+                                int32_t concat, int32_t* tokens_out_dev, int32_t tokens_out_stride, float* logits_out_dev,
+                                void* hidden_out_dev, void* stream_) {
     if (ctx == nullptr) return BEAGLE_ERR_INVALID_ARG;
     beagle_status st = check_slots(ctx, batch, seq_slot);
     if (st != BEAGLE_OK) return st;
     if (batch == 0) return BEAGLE_OK;
+    if (tokens_out_dev != nullptr && tokens_out_stride < 1) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "tokens_out_stride must be >= 1");
     const beagle_config& c = ctx->cfg;
     bool any_append = false;
     for (int b = 0; b < batch; ++b) {
@@ -365,6 +443,7 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
 
     // (1) concat: K/V of the previous step's state joins the cache tail (Section 4.1, cache paragraph)
     if (any_append) {
+        StageTimer timer_(ctx, ST_KV_APPEND, stream);
         GemvArgs a;
         memset(&a, 0, sizeof(a));
         a.W = ctx->w.w_k; a.W2 = ctx->w.w_v; a.N = ctx->kd; a.K = c.hidden;
@@ -374,10 +453,14 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
         ctx->launches += launch_gemv(dt, GEMV_KV, a, stream);
     }
     // (2) x = E[t], xn = RMSNorm(x)
-    ctx->launches += launch_embed_norm(dt, tokens_in_dev, ctx->last_token, &meta, ctx->w.embed, c.vocab, nullptr, ctx->w.g_q,
-                                       c.hidden, c.rms_eps, c.norm_q, ctx->x, ctx->xn, batch, stream);
+    {
+        StageTimer timer_(ctx, ST_EMBED_NORM, stream);
+        ctx->launches += launch_embed_norm(dt, tokens_in_dev, ctx->last_token, &meta, ctx->w.embed, c.vocab, nullptr, ctx->w.g_q,
+                                           c.hidden, c.rms_eps, c.norm_q, ctx->x, ctx->xn, batch, stream);
+    }
     // (3) Q = W_q xn
     {
+        StageTimer timer_(ctx, ST_Q_PROJ, stream);
         GemvArgs a;
         memset(&a, 0, sizeof(a));
         a.W = ctx->w.w_q; a.N = ctx->qd; a.K = c.hidden; a.X = ctx->xn; a.ldx = c.hidden; a.B = batch; a.xrow = ident;
@@ -386,6 +469,7 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
     }
     // (4) o = softmax(Q K^T / sqrt(dh)) V over the cache
     {
+        StageTimer timer_(ctx, ST_ATTN_DECODE, stream);
         const int rc = launch_attn_decode(dt, ctx->q, ctx->kcache, ctx->vcache, meta, batch, c.n_q_heads, c.n_kv_heads,
                                           c.head_dim, ctx->cap, max_kv, ctx->attn_scratch, ctx->o, stream);
         if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "attention: unsupported head shape");
@@ -393,6 +477,7 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
     }
     // (5) y = W_o o + x
     {
+        StageTimer timer_(ctx, ST_O_PROJ, stream);
         GemvArgs a;
         memset(&a, 0, sizeof(a));
         a.W = ctx->w.w_o; a.N = c.hidden; a.K = ctx->qd; a.X = ctx->o; a.ldx = ctx->qd; a.B = batch; a.xrow = ident;
@@ -400,10 +485,14 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
         ctx->launches += launch_gemv(dt, GEMV_RESID, a, stream);
     }
     // (6) yn = RMSNorm(y)
-    ctx->launches += launch_embed_norm(dt, nullptr, nullptr, nullptr, nullptr, 0, ctx->y, ctx->w.g_mlp, c.hidden, c.rms_eps,
-                                       c.norm_mlp, nullptr, ctx->yn, batch, stream);
+    {
+        StageTimer timer_(ctx, ST_MLP_NORM, stream);
+        ctx->launches += launch_embed_norm(dt, nullptr, nullptr, nullptr, nullptr, 0, ctx->y, ctx->w.g_mlp, c.hidden, c.rms_eps,
+                                           c.norm_mlp, nullptr, ctx->yn, batch, stream);
+    }
     // (7) act = SiLU(W_gate yn) * (W_up yn)
     {
+        StageTimer timer_(ctx, ST_GATE_UP, stream);
         GemvArgs a;
         memset(&a, 0, sizeof(a));
         a.W = ctx->w.w_gate; a.W2 = ctx->w.w_up; a.N = c.mlp_dim; a.K = c.hidden; a.X = ctx->yn; a.ldx = c.hidden;
@@ -412,6 +501,7 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
     }
     // (8) h = W_down act + y ; kept per slot for the next step's K/V append
     {
+        StageTimer timer_(ctx, ST_DOWN, stream);
         GemvArgs a;
         memset(&a, 0, sizeof(a));
         a.W = ctx->w.w_down; a.N = c.hidden; a.K = c.mlp_dim; a.X = ctx->act; a.ldx = c.mlp_dim; a.B = batch; a.xrow = ident;
@@ -428,8 +518,12 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
         memset(&a, 0, sizeof(a));
         a.W = ctx->w.w_lm; a.N = c.vocab; a.K = c.hidden; a.X = ctx->h; a.ldx = c.hidden; a.B = batch; a.xrow = ident;
         a.logits = logits_out_dev; a.partials = ctx->lm_partials;
-        ctx->launches += launch_gemv(dt, GEMV_LOGITS, a, stream);
-        ctx->launches += launch_argmax_finalize(ctx->lm_partials, ctx->lm_blocks, meta, batch, tokens_out_dev, ctx->last_token, stream);
+        {
+            StageTimer timer_(ctx, ST_LM_HEAD, stream);
+            ctx->launches += launch_gemv(dt, GEMV_LOGITS, a, stream);
+        }
+        StageTimer timer_(ctx, ST_ARGMAX, stream);
+        ctx->launches += launch_argmax_finalize(ctx->lm_partials, ctx->lm_blocks, meta, batch, tokens_out_dev, tokens_out_stride, ctx->last_token, stream);
     }
     st = cuda_ok(ctx, "draft_step");
     if (st != BEAGLE_OK) return st;
@@ -476,26 +570,30 @@ beagle_status beagle_block_forward(beagle_ctx* ctx, int32_t batch, int32_t S, co
     void *O = ws + L.o, *Y = ws + L.y, *Yn = ws + L.yn, *ACT = ws + L.act;
     void* H = hidden_out_dev != nullptr ? hidden_out_dev : (void*)(ws + L.h);
     int rc;
-#define BEAGLE_GEMM(EPI, ARGS, WHAT)                                                   \
+#define BEAGLE_GEMM(STAGE, EPI, ARGS, WHAT)                                            \
     do {                                                                               \
+        StageTimer timer_(ctx, STAGE, stream);                                         \
         rc = dense_gemm(ctx, EPI, ARGS, stream);                                       \
         if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, WHAT ": unsupported shape");   \
         ctx->launches += rc;                                                           \
     } while (0)
 
     // queries: every position's data token (Section 4.2: no new queries are generated)
-    ctx->launches += launch_embed_norm(dt, tokens_dev, nullptr, nullptr, ctx->w.embed, c.vocab, nullptr,
-                                       ctx->w.g_q, c.hidden, c.rms_eps, c.norm_q, X, Xn, M, stream);
+    {
+        StageTimer timer_(ctx, ST_BLK_EMBED, stream);
+        ctx->launches += launch_embed_norm(dt, tokens_dev, nullptr, nullptr, ctx->w.embed, c.vocab, nullptr,
+                                           ctx->w.g_q, c.hidden, c.rms_eps, c.norm_q, X, Xn, M, stream);
+    }
     GemmArgs g;
     memset(&g, 0, sizeof(g));
     g.M = M;
     g.A = Xn; g.lda = c.hidden; g.K = c.hidden; g.W = ctx->w.w_q; g.N = ctx->qd; g.C = Q; g.ldc = ctx->qd;
-    BEAGLE_GEMM(GEMM_STORE, g, "Q projection");
+    BEAGLE_GEMM(ST_BLK_QKV, GEMM_STORE, g, "Q projection");
     // keys / values of the true states
     g.A = hidden_dev; g.W = ctx->w.w_k; g.N = ctx->kd; g.C = Kt; g.ldc = ctx->kd;
-    BEAGLE_GEMM(GEMM_STORE, g, "K projection");
+    BEAGLE_GEMM(ST_BLK_QKV, GEMM_STORE, g, "K projection");
     g.W = ctx->w.w_v; g.C = Vt;
-    BEAGLE_GEMM(GEMM_STORE, g, "V projection");
+    BEAGLE_GEMM(ST_BLK_QKV, GEMM_STORE, g, "V projection");
 
     for (int step = 1; step <= sim_steps; ++step) {
         if (step > 1) {
@@ -503,27 +601,33 @@ beagle_status beagle_block_forward(beagle_ctx* ctx, int32_t batch, int32_t S, co
             memset(&g, 0, sizeof(g));
             g.M = M; g.A = H; g.lda = c.hidden; g.K = c.hidden; g.N = ctx->kd; g.ldc = ctx->kd;
             g.W = ctx->w.w_k; g.C = Kp;
-            BEAGLE_GEMM(GEMM_STORE, g, "predicted K projection");
+            BEAGLE_GEMM(ST_BLK_PRED_KV, GEMM_STORE, g, "predicted K projection");
             g.W = ctx->w.w_v; g.C = Vp;
-            BEAGLE_GEMM(GEMM_STORE, g, "predicted V projection");
+            BEAGLE_GEMM(ST_BLK_PRED_KV, GEMM_STORE, g, "predicted V projection");
         }
-        rc = launch_attn_block(dt, Q, Kt, Vt, Kp, Vp, batch, S, c.n_q_heads, c.n_kv_heads, c.head_dim, block, offset, step, O, stream);
-        if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "block attention: unsupported head_dim");
-        ctx->launches += rc;
+        {
+            StageTimer timer_(ctx, ST_BLK_ATTN, stream);
+            rc = launch_attn_block(dt, Q, Kt, Vt, Kp, Vp, batch, S, c.n_q_heads, c.n_kv_heads, c.head_dim, block, offset, step, O, stream);
+            if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "block attention: unsupported head_dim");
+            ctx->launches += rc;
+        }
         memset(&g, 0, sizeof(g));
         g.M = M; g.A = O; g.lda = ctx->qd; g.K = ctx->qd; g.W = ctx->w.w_o; g.N = c.hidden; g.C = Y; g.ldc = c.hidden;
         g.R = X; g.ldr = c.hidden;
-        BEAGLE_GEMM(GEMM_RESID, g, "O projection");
-        ctx->launches += launch_embed_norm(dt, nullptr, nullptr, nullptr, nullptr, 0, Y, ctx->w.g_mlp, c.hidden, c.rms_eps,
-                                           c.norm_mlp, nullptr, Yn, M, stream);
+        BEAGLE_GEMM(ST_BLK_O, GEMM_RESID, g, "O projection");
+        {
+            StageTimer timer_(ctx, ST_BLK_NORM, stream);
+            ctx->launches += launch_embed_norm(dt, nullptr, nullptr, nullptr, nullptr, 0, Y, ctx->w.g_mlp, c.hidden, c.rms_eps,
+                                               c.norm_mlp, nullptr, Yn, M, stream);
+        }
         memset(&g, 0, sizeof(g));
         g.M = M; g.A = Yn; g.lda = c.hidden; g.K = c.hidden; g.W = ctx->w.w_gate; g.W2 = ctx->w.w_up; g.N = c.mlp_dim;
         g.C = ACT; g.ldc = c.mlp_dim;
-        BEAGLE_GEMM(GEMM_SILU_MUL, g, "gate/up projection");
+        BEAGLE_GEMM(ST_BLK_GATE_UP, GEMM_SILU_MUL, g, "gate/up projection");
         memset(&g, 0, sizeof(g));
         g.M = M; g.A = ACT; g.lda = c.mlp_dim; g.K = c.mlp_dim; g.W = ctx->w.w_down; g.N = c.hidden; g.C = H; g.ldc = c.hidden;
         g.R = Y; g.ldr = c.hidden;
-        BEAGLE_GEMM(GEMM_RESID, g, "down projection");
+        BEAGLE_GEMM(ST_BLK_DOWN, GEMM_RESID, g, "down projection");
     }
 
     // LM head at every position
@@ -533,8 +637,11 @@ beagle_status beagle_block_forward(beagle_ctx* ctx, int32_t batch, int32_t S, co
         if (logits_out_dev != nullptr) {
             memset(&g, 0, sizeof(g));
             g.M = M; g.A = H; g.lda = c.hidden; g.K = c.hidden; g.W = ctx->w.w_lm; g.N = c.vocab; g.C = logits_out_dev; g.ldc = c.vocab;
-            BEAGLE_GEMM(GEMM_F32, g, "LM head");
-            if (argmax_out_dev != nullptr) ctx->launches += launch_row_argmax(0, logits_out_dev, M, c.vocab, keys, ids, stream);
+            BEAGLE_GEMM(ST_BLK_LM_HEAD, GEMM_F32, g, "LM head");
+            if (argmax_out_dev != nullptr) {
+                StageTimer timer_(ctx, ST_BLK_ARGMAX, stream);
+                ctx->launches += launch_row_argmax(0, logits_out_dev, M, c.vocab, keys, ids, stream);
+            }
         } else {
             float* chunk = reinterpret_cast<float*>(ws + L.logits);
             for (int r0 = 0; r0 < M; r0 += L.lm_chunk_rows) {
@@ -542,7 +649,8 @@ beagle_status beagle_block_forward(beagle_ctx* ctx, int32_t batch, int32_t S, co
                 memset(&g, 0, sizeof(g));
                 g.M = rows; g.A = static_cast<const char*>(H) + (size_t)r0 * c.hidden * ctx->elt; g.lda = c.hidden; g.K = c.hidden;
                 g.W = ctx->w.w_lm; g.N = c.vocab; g.C = chunk; g.ldc = c.vocab;
-                BEAGLE_GEMM(GEMM_F32, g, "LM head");
+                BEAGLE_GEMM(ST_BLK_LM_HEAD, GEMM_F32, g, "LM head");
+                StageTimer timer_(ctx, ST_BLK_ARGMAX, stream);
                 ctx->launches += launch_row_argmax(0, chunk, rows, c.vocab, keys + (size_t)r0 * kRowArgmaxSplit, ids + r0, stream);
             }
         }
@@ -566,6 +674,7 @@ beagle_status beagle_verify_greedy(beagle_ctx* ctx, int32_t batch, int32_t gamma
         return fail(ctx, BEAGLE_ERR_INVALID_ARG, "verify: unknown logits_dtype");
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const int32_t* ids = target_ids_dev;
+    StageTimer timer_(ctx, ST_VERIFY, stream);
     if (target_logits_dev != nullptr) {
         ctx->launches += launch_row_argmax(logits_dtype, target_logits_dev, batch * (gamma + 1), ctx->cfg.vocab,
                                            ctx->verify_keys, ctx->ids, stream);

@@ -53,7 +53,7 @@ int launch_attn_decode(int dtype, const void* q, const void* kcache, const void*
 
 // tokens_out[b] (optional) and last_token[slot[b]] from the per-block keys.
 int launch_argmax_finalize(const unsigned long long* partials, int nblk, const BatchMeta& meta, int B,
-                           int32_t* tokens_out, int32_t* last_token, cudaStream_t stream);
+                           int32_t* tokens_out, int tokens_out_stride, int32_t* last_token, cudaStream_t stream);
 
 // Row arg-max of [rows, V] logits (fp32 or bf16) into int32 ids; scratch: rows * kRowArgmaxSplit keys.
 constexpr int kRowArgmaxSplit = 16;

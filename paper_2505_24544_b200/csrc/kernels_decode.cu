@@ -420,7 +420,7 @@ int launch_attn_decode(int dtype, const void* q, const void* kcache, const void*
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) argmax_finalize_kernel(const unsigned long long* __restrict__ partials, int nblk,
                                                               const BatchMeta meta, int32_t* __restrict__ tokens_out,
-                                                              int32_t* __restrict__ last_token) {
+                                                              int tokens_out_stride, int32_t* __restrict__ last_token) {
     const int b = blockIdx.x;
     unsigned long long key = 0ull;
     for (int i = threadIdx.x; i < nblk; i += blockDim.x) {
@@ -434,14 +434,14 @@ __global__ void __launch_bounds__(256) argmax_finalize_kernel(const unsigned lon
     if (threadIdx.x == 0) {
         for (int w = 1; w < 8; ++w) key = s_k[w] > key ? s_k[w] : key;
         const int tok = argmax_key_index(key);
-        if (tokens_out != nullptr) tokens_out[b] = tok;
+        if (tokens_out != nullptr) tokens_out[(size_t)b * tokens_out_stride] = tok;
         last_token[meta.slot[b]] = tok;
     }
 }
 int launch_argmax_finalize(const unsigned long long* partials, int nblk, const BatchMeta& meta, int B,
-                           int32_t* tokens_out, int32_t* last_token, cudaStream_t stream) {
+                           int32_t* tokens_out, int tokens_out_stride, int32_t* last_token, cudaStream_t stream) {
     if (B <= 0) return 0;
-    argmax_finalize_kernel<<<B, 256, 0, stream>>>(partials, nblk, meta, tokens_out, last_token);
+    argmax_finalize_kernel<<<B, 256, 0, stream>>>(partials, nblk, meta, tokens_out, tokens_out_stride, last_token);
     return 1;
 }
 

@@ -67,7 +67,7 @@ def test_query_sizes_and_shape_validation(lib):
 
 def test_null_context_is_rejected(lib):
     assert lib.beagle_prefill_kv(None, 0, None, None, None, None) == 1
-    assert lib.beagle_draft_step(None, 0, None, None, 1, None, None, None, None) == 1
+    assert lib.beagle_draft_step(None, 0, None, None, 1, None, 1, None, None, None) == 1
     assert lib.beagle_verify_greedy(None, 0, 0, None, None, 0, None, None, None, None) == 1
     assert lib.beagle_block_forward(None, 1, 1, None, None, 1, 0, 1, None, None, None, None, 0, None) == 1
     assert lib.beagle_destroy(None) == 1
