@@ -156,6 +156,35 @@ beagle_status beagle_verify_greedy(beagle_ctx* ctx, int32_t batch, int32_t gamma
                                    int32_t logits_dtype, const int32_t* target_ids_dev,
                                    int32_t* accept_len_dev, int32_t* out_tokens_dev, void* stream);
 
+/* Greedy acceptance from target logits with NO memory handed over by the caller beyond the inputs
+ * and outputs.  (The paper has no counterpart: this is a packaging variant of beagle_verify_greedy.)
+ *
+ * Who needs it: code that must not allocate device memory at the point where it verifies a draft --
+ * a serving loop whose framework took the whole GPU for its own pool at start-up, so a fresh
+ * cudaMalloc would fail or stall the device; a plug-in that is only lent its input and output
+ * tensors; a latency-critical path that may not run an allocator at all.  Such callers also have
+ * no workspace to pass to beagle_create, so this entry point needs no context.
+ *
+ * How: the arg-max scratch (partial keys and row ids) is a fixed array inside the library's device
+ * image, BEAGLE_STATIC_VERIFY_MAX_ROWS logit rows large (about 0.55 MB, resident on every GPU that
+ * loads the library until the process exits).  The call performs no cudaMalloc/cudaFree and calls
+ * no allocating routine.  batch * (gamma + 1) above that limit is rejected with
+ * BEAGLE_ERR_CAPACITY and a message in err_buf (optional HOST buffer of err_len bytes).
+ *
+ * The first call on each device looks up the array's device address (a host-side query, done with
+ * that device current); make that first call outside any stream capture.  All calls on a device
+ * share the one array: it keeps the previous call's contents, which is harmless because every
+ * entry that is read is written first by the same call -- but two calls whose kernels can overlap
+ * on the GPU (different streams, no dependency between them) race on it.  Serialise them.
+ *
+ * Arguments as in beagle_verify_greedy with target logits ([batch, gamma+1, vocab], logits_dtype
+ * BEAGLE_FP32 or BEAGLE_BF16); results are identical to that call's. */
+#define BEAGLE_STATIC_VERIFY_MAX_ROWS 4160
+beagle_status beagle_verify_greedy_static(int32_t batch, int32_t gamma, int32_t vocab,
+                                          const int32_t* draft_tokens_dev, const void* target_logits_dev,
+                                          int32_t logits_dtype, int32_t* accept_len_dev, int32_t* out_tokens_dev,
+                                          void* stream, char* err_buf, size_t err_len);
+
 /* Optional per-stage timing (no counterpart in the paper; measurement support).  While enabled,
  * every stage of every entry point is bracketed by a pair of CUDA events recorded on the call's
  * stream.  beagle_profile_read waits for the recorded events, writes the accumulated milliseconds

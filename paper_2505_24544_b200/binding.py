@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = (
     "beagle_draft_step", "beagle_rollback", "beagle_reset_slot", "beagle_slot_lengths",
     "beagle_block_workspace_bytes", "beagle_block_forward", "beagle_verify_greedy", "beagle_last_error",
     "beagle_launch_count", "beagle_profile_enable", "beagle_profile_read", "beagle_profile_stage_count",
-    "beagle_profile_stage_name",
+    "beagle_profile_stage_name", "beagle_verify_greedy_static",
 )
 
 
@@ -85,6 +85,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.beagle_profile_stage_count.restype = C.c_int32
     lib.beagle_profile_stage_name.argtypes = [i32]
     lib.beagle_profile_stage_name.restype = C.c_char_p
+    lib.beagle_verify_greedy_static.argtypes = [i32, i32, i32, vp, vp, i32, vp, vp, vp, C.c_char_p, C.c_size_t]
+    lib.beagle_verify_greedy_static.restype = C.c_int
     lib.beagle_launch_count.restype = C.c_int64
     lib.beagle_launch_count.argtypes = [vp]
     for name in ("beagle_query_sizes", "beagle_create", "beagle_destroy", "beagle_prefill_kv", "beagle_draft_step",
@@ -233,6 +235,25 @@ def beagle_verify_greedy(ctx: Context, draft_tokens: torch.Tensor, target_logits
             raise ValueError("target_logits must be float32 or bfloat16")
     ctx.check(ctx.lib.beagle_verify_greedy(ctx.handle, batch, gamma, _ptr(draft_tokens), _ptr(target_logits), code,
                                            _ptr(target_ids), _ptr(accept_len), _ptr(out_tokens), _stream()))
+
+
+def beagle_verify_greedy_static(draft_tokens: torch.Tensor, target_logits: torch.Tensor, accept_len: torch.Tensor,
+                                out_tokens: torch.Tensor) -> None:
+    """Greedy acceptance for callers that may not allocate: no context, no workspace -- the
+    library's built-in device array serves as scratch (see include/beagle.h for the limits)."""
+    batch, gamma = draft_tokens.shape
+    if target_logits.dtype == torch.bfloat16:
+        code = BEAGLE_BF16
+    elif target_logits.dtype == torch.float32:
+        code = BEAGLE_FP32
+    else:
+        raise ValueError("target_logits must be float32 or bfloat16")
+    err = C.create_string_buffer(256)
+    st = load_library().beagle_verify_greedy_static(batch, gamma, target_logits.shape[-1], _ptr(draft_tokens),
+                                                    _ptr(target_logits), code, _ptr(accept_len), _ptr(out_tokens),
+                                                    _stream(), err, len(err))
+    if st != 0:
+        raise BeagleError(st, err.value.decode())
 
 
 def beagle_profile_enable(ctx: Context, on: bool) -> None:
