@@ -46,7 +46,8 @@ typedef enum beagle_status {
     BEAGLE_ERR_CAPACITY = 3,      /* cache, workspace, batch or draft depth exceeded              */
     BEAGLE_ERR_STATE = 4,         /* call order: e.g. tokens_in == NULL with no previous step     */
     BEAGLE_ERR_UNSUPPORTED = 5,
-    BEAGLE_ERR_CUDA = 6           /* a CUDA runtime call failed; see beagle_last_error            */
+    BEAGLE_ERR_CUDA = 6,          /* a CUDA runtime call failed; see beagle_last_error            */
+    BEAGLE_ERR_DEVICE = 7         /* a kernel gave up on one of its bounded waits (beagle_check_device) */
 } beagle_status;
 
 enum { BEAGLE_FP32 = 0, BEAGLE_BF16 = 1 };
@@ -194,6 +195,10 @@ beagle_status beagle_profile_enable(beagle_ctx* ctx, int32_t on);
 beagle_status beagle_profile_read(beagle_ctx* ctx, float* ms_out_host, int32_t* count_out_host);
 int32_t beagle_profile_stage_count(void);
 const char* beagle_profile_stage_name(int32_t stage);
+
+/* Waits for the stream, then reports BEAGLE_ERR_DEVICE if any kernel of this context abandoned a
+ * bounded wait (its outputs are then undefined).  The only call that synchronises. */
+beagle_status beagle_check_device(beagle_ctx* ctx, void* stream);
 
 /* Text of the last error recorded on this context ("" if none). */
 const char* beagle_last_error(const beagle_ctx* ctx);

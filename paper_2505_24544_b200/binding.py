@@ -17,7 +17,7 @@ from . import build as _build
 
 BEAGLE_FP32, BEAGLE_BF16 = 0, 1
 BEAGLE_MAX_CALL_BATCH = 64
-STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "CAPACITY", 4: "STATE", 5: "UNSUPPORTED", 6: "CUDA"}
+STATUS_NAMES = {0: "OK", 1: "INVALID_ARG", 2: "SHAPE", 3: "CAPACITY", 4: "STATE", 5: "UNSUPPORTED", 6: "CUDA", 7: "DEVICE"}
 
 WEIGHT_NAMES = ("embed", "g_q", "w_q", "w_k", "w_v", "w_o", "g_mlp", "w_gate", "w_up", "w_down", "w_lm")
 
@@ -26,7 +26,7 @@ EXPORTED_SYMBOLS = (
     "beagle_draft_step", "beagle_rollback", "beagle_reset_slot", "beagle_slot_lengths",
     "beagle_block_workspace_bytes", "beagle_block_forward", "beagle_verify_greedy", "beagle_last_error",
     "beagle_launch_count", "beagle_profile_enable", "beagle_profile_read", "beagle_profile_stage_count",
-    "beagle_profile_stage_name", "beagle_verify_greedy_static",
+    "beagle_profile_stage_name", "beagle_verify_greedy_static", "beagle_check_device",
 )
 
 
@@ -87,6 +87,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.beagle_profile_stage_name.restype = C.c_char_p
     lib.beagle_verify_greedy_static.argtypes = [i32, i32, i32, vp, vp, i32, vp, vp, vp, C.c_char_p, C.c_size_t]
     lib.beagle_verify_greedy_static.restype = C.c_int
+    lib.beagle_check_device.argtypes = [vp, vp]
+    lib.beagle_check_device.restype = C.c_int
     lib.beagle_launch_count.restype = C.c_int64
     lib.beagle_launch_count.argtypes = [vp]
     for name in ("beagle_query_sizes", "beagle_create", "beagle_destroy", "beagle_prefill_kv", "beagle_draft_step",
@@ -254,6 +256,11 @@ def beagle_verify_greedy_static(draft_tokens: torch.Tensor, target_logits: torch
                                                     _stream(), err, len(err))
     if st != 0:
         raise BeagleError(st, err.value.decode())
+
+
+def beagle_check_device(ctx: Context) -> None:
+    """Synchronises the current stream and raises if a kernel abandoned a bounded wait."""
+    ctx.check(ctx.lib.beagle_check_device(ctx.handle, _stream()))
 
 
 def beagle_profile_enable(ctx: Context, on: bool) -> None:

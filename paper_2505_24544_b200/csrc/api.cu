@@ -40,6 +40,8 @@ struct beagle_ctx {
     void *x, *xn, *q, *o, *y, *yn, *act, *h, *h_slot, *attn_scratch;
     int32_t *last_token, *ids;
     unsigned long long *lm_partials, *verify_keys;
+    int* dev_error = nullptr;       // device word raised by a kernel whose bounded wait ran out
+    bool dev_error_cleared = false;
     int lm_blocks = 0;
     // host bookkeeping
     std::vector<int32_t> n_true, n_draft;
@@ -117,7 +119,7 @@ beagle_status check_config(const beagle_config* c) {
 }
 
 struct ServeLayout {
-    size_t x, xn, q, o, y, yn, act, h, h_slot, attn, last_token, ids, lm_partials, verify_keys, total;
+    size_t x, xn, q, o, y, yn, act, h, h_slot, attn, last_token, ids, lm_partials, verify_keys, dev_error, total;
     int lm_blocks;
 };
 ServeLayout serve_layout(const beagle_config& c) {
@@ -138,6 +140,7 @@ ServeLayout serve_layout(const beagle_config& c) {
     L.lm_blocks = gemv_grid_blocks(GEMV_LOGITS, c.vocab);
     L.lm_partials = take(B * (size_t)L.lm_blocks * sizeof(unsigned long long));
     L.verify_keys = take(B * 65 * kRowArgmaxSplit * sizeof(unsigned long long));
+    L.dev_error = take(256);
     L.total = off;
     return L;
 }
@@ -160,7 +163,8 @@ BlockLayout block_layout(const beagle_config& c, int batch, int S) {
     L.act = take(M * m * elt); L.h = take(M * d * elt);
     L.lm_chunk_rows = (int)(M < (size_t)kLmChunkRows ? M : (size_t)kLmChunkRows);
     L.logits = take((size_t)L.lm_chunk_rows * c.vocab * sizeof(float));
-    L.keys = take(M * kRowArgmaxSplit * sizeof(unsigned long long));
+    const size_t key_cols = (size_t)(tc_argmax_tiles(c.vocab) > kRowArgmaxSplit ? tc_argmax_tiles(c.vocab) : kRowArgmaxSplit);
+    L.keys = take(M * key_cols * sizeof(unsigned long long));
     L.ids = take(M * sizeof(int32_t));
     L.total = off;
     return L;
@@ -174,11 +178,22 @@ beagle_status cuda_ok(beagle_ctx* ctx, const char* what) {
 
 // One dense projection C = A W^T of the block / prefill path: tensor cores when the plan covers the
 // shape (bf16), the CUDA-core kernel otherwise.
+void clear_error_word_once(beagle_ctx* ctx, cudaStream_t stream) {
+    if (!ctx->dev_error_cleared) {
+        cudaMemsetAsync(ctx->dev_error, 0, sizeof(int), stream);
+        ctx->dev_error_cleared = true;
+    }
+}
+
 int dense_gemm(beagle_ctx* ctx, int epi, const GemmArgs& a, cudaStream_t stream) {
     if (ctx->tc != nullptr) {
-        const int rc = tc_gemm(ctx->tc, epi, a, stream);
+        clear_error_word_once(ctx, stream);
+        GemmArgs t = a;
+        t.error_word = ctx->dev_error;
+        const int rc = tc_gemm(ctx->tc, epi, t, stream);
         if (rc >= 0) return rc;
     }
+    if (epi == GEMM_ARGMAX_KEYS) return -1;
     return launch_gemm_simt(ctx->cfg.dtype, epi, a, stream);
 }
 
@@ -236,12 +251,18 @@ beagle_status beagle_create(const beagle_config* cfg, const beagle_weights* w, v
     c->ids = reinterpret_cast<int32_t*>(c->ws + L.ids);
     c->lm_partials = reinterpret_cast<unsigned long long*>(c->ws + L.lm_partials);
     c->verify_keys = reinterpret_cast<unsigned long long*>(c->ws + L.verify_keys);
+    c->dev_error = reinterpret_cast<int*>(c->ws + L.dev_error);
     c->lm_blocks = L.lm_blocks;
     c->n_true.assign(cfg->max_slots, 0);
     c->n_draft.assign(cfg->max_slots, 0);
     c->pending.assign(cfg->max_slots, 0);
     c->has_token.assign(cfg->max_slots, 0);
-    c->tc = (cfg->dtype == BEAGLE_BF16) ? tc_plan_create(*cfg, *w) : nullptr;
+    int hard = 0;
+    c->tc = (cfg->dtype == BEAGLE_BF16) ? tc_plan_create(*cfg, *w, &hard) : nullptr;
+    if (hard) {
+        delete c;
+        return BEAGLE_ERR_CUDA;     // a GPU is present but the tensor-map encoder is not: never fall back silently
+    }
     *out = c;
     return BEAGLE_OK;
 }
@@ -282,6 +303,18 @@ beagle_status beagle_destroy(beagle_ctx* ctx) {
     release_events(ctx);
     tc_plan_destroy(ctx->tc);
     delete ctx;
+    return BEAGLE_OK;
+}
+
+beagle_status beagle_check_device(beagle_ctx* ctx, void* stream_) {
+    if (ctx == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (cudaStreamSynchronize(stream) != cudaSuccess) return fail(ctx, BEAGLE_ERR_CUDA, "check_device: %s", cudaGetErrorString(cudaGetLastError()));
+    if (!ctx->dev_error_cleared) return BEAGLE_OK;
+    int word = 0;
+    if (cudaMemcpy(&word, ctx->dev_error, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return fail(ctx, BEAGLE_ERR_CUDA, "check_device: %s", cudaGetErrorString(cudaGetLastError()));
+    if (word != 0) return fail(ctx, BEAGLE_ERR_DEVICE, "a kernel gave up on a bounded wait (pipeline barrier never completed)");
     return BEAGLE_OK;
 }
 
@@ -642,6 +675,13 @@ beagle_status beagle_block_forward(beagle_ctx* ctx, int32_t batch, int32_t S, co
                 StageTimer timer_(ctx, ST_BLK_ARGMAX, stream);
                 ctx->launches += launch_row_argmax(0, logits_out_dev, M, c.vocab, keys, ids, stream);
             }
+        } else if (ctx->tc != nullptr) {
+            // arg-max only: the LM-head GEMM emits one packed key per (row, column tile); no logits are written
+            memset(&g, 0, sizeof(g));
+            g.M = M; g.A = H; g.lda = c.hidden; g.K = c.hidden; g.W = ctx->w.w_lm; g.N = c.vocab; g.keys = keys;
+            BEAGLE_GEMM(ST_BLK_LM_HEAD, GEMM_ARGMAX_KEYS, g, "LM head");
+            StageTimer timer_(ctx, ST_BLK_ARGMAX, stream);
+            ctx->launches += tc_keys_to_ids(keys, M, tc_argmax_tiles(c.vocab), ids, stream);
         } else {
             float* chunk = reinterpret_cast<float*>(ws + L.logits);
             for (int r0 = 0; r0 < M; r0 += L.lm_chunk_rows) {

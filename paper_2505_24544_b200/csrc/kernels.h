@@ -69,7 +69,8 @@ enum GemmEpilogue {
     GEMM_RESID = 1,      // C = A W^T + R
     GEMM_SILU_MUL = 2,   // C = SiLU(A W^T) * (A W2^T)
     GEMM_F32 = 3,        // C fp32
-    GEMM_KV_CACHE = 4    // scatter rows into the cache: row r -> (slot, pos) through SeqRows
+    GEMM_KV_CACHE = 4,   // scatter rows into the cache: row r -> (slot, pos) through SeqRows
+    GEMM_ARGMAX_KEYS = 5 // no C: one packed arg-max key per (row, column tile)   (tensor-core path only)
 };
 struct SeqRows {        // packed-row -> (slot, position) map of a prefill call
     int32_t n;
@@ -84,6 +85,8 @@ struct GemmArgs {
     void* C; int ldc;
     const void* R; int ldr;
     void* cache; int Hkv, dh, cap;  // GEMM_KV_CACHE
+    unsigned long long* keys;       // GEMM_ARGMAX_KEYS
+    int* error_word;                // device word set to 1 when a bounded wait ran out
     SeqRows rows;
 };
 int launch_gemm_simt(int dtype, int epi, const GemmArgs& a, cudaStream_t stream);
