@@ -37,7 +37,8 @@ struct beagle_ctx {
     void* kcache = nullptr;
     void* vcache = nullptr;
     // serve-time workspace regions
-    void *x, *xn, *q, *o, *y, *yn, *act, *h, *h_slot, *attn_scratch;
+    void *x, *xn, *q, *o, *y, *yn, *act, *h, *h_slot, *hs, *attn_scratch;
+    float* sk_partial = nullptr;    // fp32 split partials of the tensor-core serve projections
     int32_t *last_token, *ids;
     unsigned long long *lm_partials, *verify_keys;
     int* dev_error = nullptr;       // device word raised by a kernel whose bounded wait ran out
@@ -87,6 +88,8 @@ struct StageTimer {
 namespace {
 
 constexpr size_t kAlign = 256;
+constexpr int kServeTcMinBatch = 8;     // serve-time batches above this use the tensor-core projections
+constexpr int kPrefillSkinnyMaxRows = 512;   // prefill calls up to this many rows use the same kernels in chunks
 size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
 beagle_status fail(beagle_ctx* ctx, beagle_status st, const char* fmt, ...) {
@@ -119,7 +122,7 @@ beagle_status check_config(const beagle_config* c) {
 }
 
 struct ServeLayout {
-    size_t x, xn, q, o, y, yn, act, h, h_slot, attn, last_token, ids, lm_partials, verify_keys, dev_error, total;
+    size_t x, xn, q, o, y, yn, act, h, h_slot, hs, attn, sk_partial, last_token, ids, lm_partials, verify_keys, dev_error, total;
     int lm_blocks;
 };
 ServeLayout serve_layout(const beagle_config& c) {
@@ -134,6 +137,18 @@ ServeLayout serve_layout(const beagle_config& c) {
     L.y = take(B * d * elt); L.yn = take(B * d * elt);
     L.act = take(B * m * elt); L.h = take(B * d * elt);
     L.h_slot = take((size_t)c.max_slots * d * elt);
+    L.hs = take(B * d * elt);
+    {
+        const int kd = c.n_kv_heads * c.head_dim;
+        size_t need = 0;
+        if (c.dtype == BEAGLE_BF16) {
+            const size_t cand[5] = {tc_skinny_partial_bytes((int)qd, (int)d, 1), tc_skinny_partial_bytes(kd, (int)d, 2),
+                                    tc_skinny_partial_bytes((int)d, (int)qd, 1), tc_skinny_partial_bytes((int)m, (int)d, 2),
+                                    tc_skinny_partial_bytes((int)d, (int)m, 1)};
+            for (size_t v : cand) need = v > need ? v : need;
+        }
+        L.sk_partial = take(need);
+    }
     L.attn = take(attn_decode_scratch_bytes((int)B, c.n_q_heads, c.head_dim, c.max_ctx + c.max_draft));
     L.last_token = take((size_t)c.max_slots * sizeof(int32_t));
     L.ids = take(B * 65 * sizeof(int32_t));
@@ -246,7 +261,8 @@ beagle_status beagle_create(const beagle_config* cfg, const beagle_weights* w, v
     const ServeLayout L = serve_layout(*cfg);
     c->x = c->ws + L.x; c->xn = c->ws + L.xn; c->q = c->ws + L.q; c->o = c->ws + L.o;
     c->y = c->ws + L.y; c->yn = c->ws + L.yn; c->act = c->ws + L.act; c->h = c->ws + L.h;
-    c->h_slot = c->ws + L.h_slot; c->attn_scratch = c->ws + L.attn;
+    c->h_slot = c->ws + L.h_slot; c->hs = c->ws + L.hs; c->attn_scratch = c->ws + L.attn;
+    c->sk_partial = reinterpret_cast<float*>(c->ws + L.sk_partial);
     c->last_token = reinterpret_cast<int32_t*>(c->ws + L.last_token);
     c->ids = reinterpret_cast<int32_t*>(c->ws + L.ids);
     c->lm_partials = reinterpret_cast<unsigned long long*>(c->ws + L.lm_partials);
@@ -394,7 +410,8 @@ beagle_status beagle_prefill_kv(beagle_ctx* ctx, int32_t batch, const int32_t* s
         }
         rows.n = n;
         rows.row_start[n] = r;
-        if (total <= 16) {
+        const bool small = ctx->tc != nullptr ? total <= kServeTcMinBatch : total <= 16;
+        if (small) {
             // few rows (the states accepted by one verification): weight-streaming path
             GemvArgs a;
             memset(&a, 0, sizeof(a));
@@ -408,6 +425,28 @@ beagle_status beagle_prefill_kv(beagle_ctx* ctx, int32_t batch, const int32_t* s
                     a.pos.idx[i] = rows.pos_start[s] + (i - rows.row_start[s]);
                 }
             ctx->launches += launch_gemv(c.dtype, GEMV_KV, a, stream);
+        } else if (ctx->tc != nullptr && total <= kPrefillSkinnyMaxRows) {
+            // up to a few hundred rows (one verification of a whole batch): chunks of 64 rows on the
+            // tensor cores with the weights as the wide operand; W_k, W_v stay in L2 between chunks
+            clear_error_word_once(ctx, stream);
+            int s = 0;
+            for (int r0 = 0; r0 < (int)total; r0 += kMaxCallBatch) {
+                const int nb = (int)total - r0 < kMaxCallBatch ? (int)total - r0 : kMaxCallBatch;
+                SkinnyArgs a;
+                memset(&a, 0, sizeof(a));
+                a.W = ctx->w.w_k; a.W2 = ctx->w.w_v; a.N = ctx->kd; a.K = c.hidden;
+                a.X = static_cast<const char*>(hidden_dev) + (size_t)r0 * c.hidden * ctx->elt; a.ldx = c.hidden; a.B = nb;
+                a.kcache = ctx->kcache; a.vcache = ctx->vcache; a.Hkv = c.n_kv_heads; a.dh = c.head_dim; a.cap = ctx->cap;
+                a.partial = ctx->sk_partial; a.error_word = ctx->dev_error;
+                for (int i = 0; i < nb; ++i) {
+                    while (r0 + i >= rows.row_start[s + 1]) ++s;
+                    a.slot.idx[i] = rows.slot[s];
+                    a.pos.idx[i] = rows.pos_start[s] + (r0 + i - rows.row_start[s]);
+                }
+                const int rc = tc_skinny(ctx->tc, SK_KV, a, stream);
+                if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "K/V projection: unsupported shape");
+                ctx->launches += rc;
+            }
         } else {
             GemmArgs g;
             memset(&g, 0, sizeof(g));
@@ -474,90 +513,157 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
         if (meta.kv_len[b] > max_kv) max_kv = meta.kv_len[b];
     }
 
-    // (1) concat: K/V of the previous step's state joins the cache tail (Section 4.1, cache paragraph)
-    if (any_append) {
-        StageTimer timer_(ctx, ST_KV_APPEND, stream);
-        GemvArgs a;
-        memset(&a, 0, sizeof(a));
-        a.W = ctx->w.w_k; a.W2 = ctx->w.w_v; a.N = ctx->kd; a.K = c.hidden;
-        a.X = ctx->h_slot; a.ldx = c.hidden; a.B = batch; a.xrow = slots;
-        a.kcache = ctx->kcache; a.vcache = ctx->vcache; a.Hkv = c.n_kv_heads; a.dh = c.head_dim; a.cap = ctx->cap;
-        a.orow2 = slots; a.pos = app_pos;
-        ctx->launches += launch_gemv(dt, GEMV_KV, a, stream);
-    }
-    // (2) x = E[t], xn = RMSNorm(x)
+    // Batches above 8 rows run their projections on the tensor cores (weights streamed once);
+    // smaller ones on the weight-streaming CUDA-core kernel.
+    const bool use_tc = ctx->tc != nullptr && batch > kServeTcMinBatch;
+    if (use_tc) clear_error_word_once(ctx, stream);
+    int rc = 0;
+#define BEAGLE_SKINNY(MODE, ARGS, WHAT)                                                   \
+    do {                                                                                  \
+        ARGS.partial = ctx->sk_partial;                                                   \
+        ARGS.error_word = ctx->dev_error;                                                 \
+        rc = tc_skinny(ctx->tc, MODE, ARGS, stream);                                      \
+        if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, WHAT ": unsupported shape");      \
+        ctx->launches += rc;                                                              \
+    } while (0)
+
+    // (1) x = E[t], xn = RMSNorm(x); the tensor-core path also gathers the slots' previous states
     {
         StageTimer timer_(ctx, ST_EMBED_NORM, stream);
         ctx->launches += launch_embed_norm(dt, tokens_in_dev, ctx->last_token, &meta, ctx->w.embed, c.vocab, nullptr, ctx->w.g_q,
-                                           c.hidden, c.rms_eps, c.norm_q, ctx->x, ctx->xn, batch, stream);
+                                           c.hidden, c.rms_eps, c.norm_q, ctx->x, ctx->xn, batch,
+                                           (use_tc && any_append) ? ctx->h_slot : nullptr, ctx->hs, stream);
+    }
+    // (2) concat: K/V of the previous step's state joins the cache tail (Section 4.1, cache paragraph)
+    if (any_append) {
+        StageTimer timer_(ctx, ST_KV_APPEND, stream);
+        if (use_tc) {
+            SkinnyArgs a;
+            memset(&a, 0, sizeof(a));
+            a.W = ctx->w.w_k; a.W2 = ctx->w.w_v; a.N = ctx->kd; a.K = c.hidden; a.X = ctx->hs; a.ldx = c.hidden; a.B = batch;
+            a.kcache = ctx->kcache; a.vcache = ctx->vcache; a.Hkv = c.n_kv_heads; a.dh = c.head_dim; a.cap = ctx->cap;
+            a.slot = slots; a.pos = app_pos;
+            BEAGLE_SKINNY(SK_KV, a, "K/V append");
+        } else {
+            GemvArgs a;
+            memset(&a, 0, sizeof(a));
+            a.W = ctx->w.w_k; a.W2 = ctx->w.w_v; a.N = ctx->kd; a.K = c.hidden;
+            a.X = ctx->h_slot; a.ldx = c.hidden; a.B = batch; a.xrow = slots;
+            a.kcache = ctx->kcache; a.vcache = ctx->vcache; a.Hkv = c.n_kv_heads; a.dh = c.head_dim; a.cap = ctx->cap;
+            a.orow2 = slots; a.pos = app_pos;
+            ctx->launches += launch_gemv(dt, GEMV_KV, a, stream);
+        }
     }
     // (3) Q = W_q xn
     {
         StageTimer timer_(ctx, ST_Q_PROJ, stream);
-        GemvArgs a;
-        memset(&a, 0, sizeof(a));
-        a.W = ctx->w.w_q; a.N = ctx->qd; a.K = c.hidden; a.X = ctx->xn; a.ldx = c.hidden; a.B = batch; a.xrow = ident;
-        a.out = ctx->q; a.ldo = ctx->qd;
-        ctx->launches += launch_gemv(dt, GEMV_STORE, a, stream);
+        if (use_tc) {
+            SkinnyArgs a;
+            memset(&a, 0, sizeof(a));
+            a.W = ctx->w.w_q; a.N = ctx->qd; a.K = c.hidden; a.X = ctx->xn; a.ldx = c.hidden; a.B = batch;
+            a.out = ctx->q; a.ldo = ctx->qd;
+            BEAGLE_SKINNY(SK_STORE, a, "Q projection");
+        } else {
+            GemvArgs a;
+            memset(&a, 0, sizeof(a));
+            a.W = ctx->w.w_q; a.N = ctx->qd; a.K = c.hidden; a.X = ctx->xn; a.ldx = c.hidden; a.B = batch; a.xrow = ident;
+            a.out = ctx->q; a.ldo = ctx->qd;
+            ctx->launches += launch_gemv(dt, GEMV_STORE, a, stream);
+        }
     }
     // (4) o = softmax(Q K^T / sqrt(dh)) V over the cache
     {
         StageTimer timer_(ctx, ST_ATTN_DECODE, stream);
-        const int rc = launch_attn_decode(dt, ctx->q, ctx->kcache, ctx->vcache, meta, batch, c.n_q_heads, c.n_kv_heads,
-                                          c.head_dim, ctx->cap, max_kv, ctx->attn_scratch, ctx->o, stream);
+        rc = launch_attn_decode(dt, ctx->q, ctx->kcache, ctx->vcache, meta, batch, c.n_q_heads, c.n_kv_heads,
+                                c.head_dim, ctx->cap, max_kv, ctx->attn_scratch, ctx->o, stream);
         if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "attention: unsupported head shape");
         ctx->launches += rc;
     }
-    // (5) y = W_o o + x
-    {
+    // (5) y = W_o o + x   (6) yn = RMSNorm(y)
+    if (use_tc) {
         StageTimer timer_(ctx, ST_O_PROJ, stream);
-        GemvArgs a;
+        SkinnyArgs a;
         memset(&a, 0, sizeof(a));
-        a.W = ctx->w.w_o; a.N = c.hidden; a.K = ctx->qd; a.X = ctx->o; a.ldx = ctx->qd; a.B = batch; a.xrow = ident;
+        a.W = ctx->w.w_o; a.N = c.hidden; a.K = ctx->qd; a.X = ctx->o; a.ldx = ctx->qd; a.B = batch;
         a.out = ctx->y; a.ldo = c.hidden; a.resid = ctx->x; a.ldr = c.hidden;
-        ctx->launches += launch_gemv(dt, GEMV_RESID, a, stream);
-    }
-    // (6) yn = RMSNorm(y)
-    {
+        a.norm_out = ctx->yn; a.gain = ctx->w.g_mlp; a.eps = c.rms_eps; a.do_norm = c.norm_mlp;   // the finishing kernel normalises
+        BEAGLE_SKINNY(SK_RESID, a, "O projection");
+    } else {
+        {
+            StageTimer timer_(ctx, ST_O_PROJ, stream);
+            GemvArgs a;
+            memset(&a, 0, sizeof(a));
+            a.W = ctx->w.w_o; a.N = c.hidden; a.K = ctx->qd; a.X = ctx->o; a.ldx = ctx->qd; a.B = batch; a.xrow = ident;
+            a.out = ctx->y; a.ldo = c.hidden; a.resid = ctx->x; a.ldr = c.hidden;
+            ctx->launches += launch_gemv(dt, GEMV_RESID, a, stream);
+        }
         StageTimer timer_(ctx, ST_MLP_NORM, stream);
         ctx->launches += launch_embed_norm(dt, nullptr, nullptr, nullptr, nullptr, 0, ctx->y, ctx->w.g_mlp, c.hidden, c.rms_eps,
-                                           c.norm_mlp, nullptr, ctx->yn, batch, stream);
+                                           c.norm_mlp, nullptr, ctx->yn, batch, nullptr, nullptr, stream);
     }
     // (7) act = SiLU(W_gate yn) * (W_up yn)
     {
         StageTimer timer_(ctx, ST_GATE_UP, stream);
-        GemvArgs a;
-        memset(&a, 0, sizeof(a));
-        a.W = ctx->w.w_gate; a.W2 = ctx->w.w_up; a.N = c.mlp_dim; a.K = c.hidden; a.X = ctx->yn; a.ldx = c.hidden;
-        a.B = batch; a.xrow = ident; a.out = ctx->act; a.ldo = c.mlp_dim;
-        ctx->launches += launch_gemv(dt, GEMV_SILU_MUL, a, stream);
+        if (use_tc) {
+            SkinnyArgs a;
+            memset(&a, 0, sizeof(a));
+            a.W = ctx->w.w_gate; a.W2 = ctx->w.w_up; a.N = c.mlp_dim; a.K = c.hidden; a.X = ctx->yn; a.ldx = c.hidden; a.B = batch;
+            a.out = ctx->act; a.ldo = c.mlp_dim;
+            BEAGLE_SKINNY(SK_SILU_MUL, a, "gate/up projection");
+        } else {
+            GemvArgs a;
+            memset(&a, 0, sizeof(a));
+            a.W = ctx->w.w_gate; a.W2 = ctx->w.w_up; a.N = c.mlp_dim; a.K = c.hidden; a.X = ctx->yn; a.ldx = c.hidden;
+            a.B = batch; a.xrow = ident; a.out = ctx->act; a.ldo = c.mlp_dim;
+            ctx->launches += launch_gemv(dt, GEMV_SILU_MUL, a, stream);
+        }
     }
     // (8) h = W_down act + y ; kept per slot for the next step's K/V append
     {
         StageTimer timer_(ctx, ST_DOWN, stream);
-        GemvArgs a;
-        memset(&a, 0, sizeof(a));
-        a.W = ctx->w.w_down; a.N = c.hidden; a.K = c.mlp_dim; a.X = ctx->act; a.ldx = c.mlp_dim; a.B = batch; a.xrow = ident;
-        a.out = ctx->h; a.ldo = c.hidden; a.resid = ctx->y; a.ldr = c.hidden;
-        a.out2 = ctx->h_slot; a.ld2 = c.hidden; a.orow2 = slots;
-        ctx->launches += launch_gemv(dt, GEMV_RESID, a, stream);
+        if (use_tc) {
+            SkinnyArgs a;
+            memset(&a, 0, sizeof(a));
+            a.W = ctx->w.w_down; a.N = c.hidden; a.K = c.mlp_dim; a.X = ctx->act; a.ldx = c.mlp_dim; a.B = batch;
+            a.out = ctx->h; a.ldo = c.hidden; a.resid = ctx->y; a.ldr = c.hidden;
+            a.out2 = ctx->h_slot; a.ld2 = c.hidden; a.orow2 = slots;
+            BEAGLE_SKINNY(SK_RESID, a, "down projection");
+        } else {
+            GemvArgs a;
+            memset(&a, 0, sizeof(a));
+            a.W = ctx->w.w_down; a.N = c.hidden; a.K = c.mlp_dim; a.X = ctx->act; a.ldx = c.mlp_dim; a.B = batch; a.xrow = ident;
+            a.out = ctx->h; a.ldo = c.hidden; a.resid = ctx->y; a.ldr = c.hidden;
+            a.out2 = ctx->h_slot; a.ld2 = c.hidden; a.orow2 = slots;
+            ctx->launches += launch_gemv(dt, GEMV_RESID, a, stream);
+        }
     }
     if (hidden_out_dev != nullptr) {
         cudaMemcpyAsync(hidden_out_dev, ctx->h, (size_t)batch * c.hidden * ctx->elt, cudaMemcpyDeviceToDevice, stream);
     }
     // (9) z = W_lm h, greedy token
     {
-        GemvArgs a;
-        memset(&a, 0, sizeof(a));
-        a.W = ctx->w.w_lm; a.N = c.vocab; a.K = c.hidden; a.X = ctx->h; a.ldx = c.hidden; a.B = batch; a.xrow = ident;
-        a.logits = logits_out_dev; a.partials = ctx->lm_partials;
+        int nblk = ctx->lm_blocks;
         {
             StageTimer timer_(ctx, ST_LM_HEAD, stream);
-            ctx->launches += launch_gemv(dt, GEMV_LOGITS, a, stream);
+            if (use_tc) {
+                SkinnyArgs a;
+                memset(&a, 0, sizeof(a));
+                a.W = ctx->w.w_lm; a.N = c.vocab; a.K = c.hidden; a.X = ctx->h; a.ldx = c.hidden; a.B = batch;
+                a.logits = logits_out_dev; a.keys = ctx->lm_partials;
+                BEAGLE_SKINNY(SK_LOGITS, a, "LM head");
+                nblk = tc_skinny_key_tiles(c.vocab);
+            } else {
+                GemvArgs a;
+                memset(&a, 0, sizeof(a));
+                a.W = ctx->w.w_lm; a.N = c.vocab; a.K = c.hidden; a.X = ctx->h; a.ldx = c.hidden; a.B = batch; a.xrow = ident;
+                a.logits = logits_out_dev; a.partials = ctx->lm_partials;
+                ctx->launches += launch_gemv(dt, GEMV_LOGITS, a, stream);
+            }
         }
         StageTimer timer_(ctx, ST_ARGMAX, stream);
-        ctx->launches += launch_argmax_finalize(ctx->lm_partials, ctx->lm_blocks, meta, batch, tokens_out_dev, tokens_out_stride, ctx->last_token, stream);
+        ctx->launches += launch_argmax_finalize(ctx->lm_partials, nblk, meta, batch, tokens_out_dev, tokens_out_stride, ctx->last_token, stream);
     }
+#undef BEAGLE_SKINNY
     st = cuda_ok(ctx, "draft_step");
     if (st != BEAGLE_OK) return st;
     for (int b = 0; b < batch; ++b) {
@@ -615,7 +721,7 @@ beagle_status beagle_block_forward(beagle_ctx* ctx, int32_t batch, int32_t S, co
     {
         StageTimer timer_(ctx, ST_BLK_EMBED, stream);
         ctx->launches += launch_embed_norm(dt, tokens_dev, nullptr, nullptr, ctx->w.embed, c.vocab, nullptr,
-                                           ctx->w.g_q, c.hidden, c.rms_eps, c.norm_q, X, Xn, M, stream);
+                                           ctx->w.g_q, c.hidden, c.rms_eps, c.norm_q, X, Xn, M, nullptr, nullptr, stream);
     }
     GemmArgs g;
     memset(&g, 0, sizeof(g));
@@ -651,7 +757,7 @@ beagle_status beagle_block_forward(beagle_ctx* ctx, int32_t batch, int32_t S, co
         {
             StageTimer timer_(ctx, ST_BLK_NORM, stream);
             ctx->launches += launch_embed_norm(dt, nullptr, nullptr, nullptr, nullptr, 0, Y, ctx->w.g_mlp, c.hidden, c.rms_eps,
-                                               c.norm_mlp, nullptr, Yn, M, stream);
+                                               c.norm_mlp, nullptr, Yn, M, nullptr, nullptr, stream);
         }
         memset(&g, 0, sizeof(g));
         g.M = M; g.A = Yn; g.lda = c.hidden; g.K = c.hidden; g.W = ctx->w.w_gate; g.W2 = ctx->w.w_up; g.N = c.mlp_dim;

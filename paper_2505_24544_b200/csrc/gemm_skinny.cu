@@ -1,0 +1,366 @@
+// Serve-time projections for 9..64 batch rows on the tensor cores ("swap-AB"): the weight matrix
+// [N, K] supplies the 128 rows of each tcgen05.mma, the batch's activations [B, K] its BN <= 64
+// columns, so every weight byte crosses HBM exactly once per projection whatever the batch.
+//
+// One CTA = one 128-row weight tile x one slice of K.  Warp 0 streams the tile with TMA
+// (128-byte swizzle, a ring of stages), warp 1 issues the MMAs into a TMEM accumulator of BN
+// columns, warps 2..5 read the accumulator (thread = output feature, register j = batch row j)
+// and either write fp32 partial sums [split][matrix][b][n] for the finishing kernel below or, for
+// the LM head, logits and one packed arg-max key per (b, tile).  Shared memory is sized so that
+// two CTAs share an SM: one CTA's prologue and epilogue hide behind the other's stream.
+//
+// Every wait on an mbarrier is bounded; a wait that runs out raises a device error word and the
+// CTA drains its copies and frees its TMEM instead of hanging.
+#include <cstring>
+
+#include "gemm_tc.h"
+#include "tc_plan.h"
+#include "tc_ptx.cuh"
+
+namespace beagle {
+
+namespace {
+
+using namespace tc;
+constexpr int BM = 128;
+constexpr int kSkThreads = 192;
+constexpr int kCtaSlots = 296;          // CTAs the split policy aims at (two per SM on 148 SMs)
+constexpr int kABytes = BM * BK * 2;
+
+template <int BN>
+struct SkSmem {
+    static constexpr int kStageBytes = kABytes + BN * BK * 2;
+    static constexpr int kStages = BN <= 16 ? 6 : (BN <= 32 ? 5 : 4);
+    static constexpr int kKeyBytes = 4 * BN * 8;
+    static constexpr int kBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/ + kKeyBytes;
+};
+
+struct SkArgs {
+    int N, K, B;              // weight rows, reduction length, valid batch rows
+    int nmat;                 // weight matrices (blockIdx.y)
+    int kb_per_split;         // k-blocks of 64 per blockIdx.z slice
+    float* partial;           // [split][nmat][B][N]
+    float* logits;            // [B][N] or null
+    unsigned long long* keys; // [B][gridDim.x]
+    int* error_word;
+};
+
+template <int BN, bool LOGITS>
+__global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_constant__ CUtensorMap tmW,
+                                                               const __grid_constant__ CUtensorMap tmW2,
+                                                               const __grid_constant__ CUtensorMap tmX, const SkArgs args) {
+    using SM = SkSmem<BN>;
+    constexpr int kStages = SM::kStages;
+    constexpr uint32_t kTmemCols = BN < 32 ? 32 : BN;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + kStages * SM::kStageBytes);
+    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * kStages, bar_acc = bar_empty + 8 * kStages;
+    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 1);
+    volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
+    unsigned long long* s_keys = reinterpret_cast<unsigned long long*>(smem_gen + kStages * SM::kStageBytes + 256);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ta = blockIdx.x, mat = blockIdx.y;
+    const int kb_total = (args.K + BK - 1) / BK;
+    const int kb0 = blockIdx.z * args.kb_per_split;
+    const int nkb = max(0, min(args.kb_per_split, kb_total - kb0));
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+        mbar_init(bar_acc, 1);
+        *s_abort = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc<kTmemCols>(smem_u32(s_tmem));
+    fence_before();
+    __syncthreads();
+    fence_after();
+    const uint32_t tmem_base = *s_tmem;
+
+    if (warp == 0) {
+        // ---------------- TMA producer
+        if (lane == 0) {
+            const CUtensorMap* mapW = mat ? &tmW2 : &tmW;
+            const uint64_t stream_once = policy_evict_first(), keep = policy_evict_last();
+            int issued = 0;
+            for (int kb = 0; kb < nkb; ++kb) {
+                const int s = kb % kStages;
+                const uint32_t ph = (kb / kStages) & 1;
+                if (!mbar_wait(bar_empty + 8 * s, ph ^ 1, s_abort)) break;
+                const uint32_t sa = smem_base + s * SM::kStageBytes, sb = sa + kABytes;
+                mbar_expect_tx(bar_full + 8 * s, SM::kStageBytes);
+                const int kc = (kb0 + kb) * BK;
+                tma_load_2d_hint(sa, mapW, bar_full + 8 * s, kc, ta * BM, stream_once);
+                tma_load_2d_hint(sb, &tmX, bar_full + 8 * s, kc, 0, keep);
+                ++issued;
+            }
+            if (*s_abort) {
+                // copies already issued still land in shared memory: wait (bounded) for the last of each stage
+                for (int kb = max(0, issued - kStages); kb < issued; ++kb) {
+                    const int s = kb % kStages;
+                    const uint32_t ph = (kb / kStages) & 1;
+                    for (uint32_t i = 0; i < kSpinLimit; ++i)
+                        if (mbar_try_wait(bar_full + 8 * s, ph)) break;
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(BM, BN);
+            for (int kb = 0; kb < nkb; ++kb) {
+                const int s = kb % kStages;
+                const uint32_t ph = (kb / kStages) & 1;
+                if (!mbar_wait(bar_full + 8 * s, ph, s_abort)) break;
+                fence_after();
+                const uint32_t sa = smem_base + s * SM::kStageBytes, sb = sa + kABytes;
+                const uint64_t da = umma_desc(sa), db = umma_desc(sb);
+#pragma unroll
+                for (int k = 0; k < BK / UMMA_K; ++k) {
+                    const uint64_t koff = static_cast<uint64_t>((k * UMMA_K * 2) >> 4);   // advance inside the swizzle atom
+                    umma_bf16(tmem_base, da + koff, db + koff, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                }
+                umma_commit(bar_empty + 8 * s);       // frees the stage once these MMAs have read it
+            }
+            umma_commit(bar_acc);                     // accumulator complete (or nothing was issued)
+        }
+    } else {
+        // ---------------- epilogue: warp w reads TMEM lanes [32*(w%4), +32)
+        const int q = warp & 3;
+        const int feat = ta * BM + q * 32 + lane;    // output feature owned by this thread
+        bool ok = nkb > 0;
+        if (ok) ok = mbar_wait(bar_acc, 0, s_abort);
+        ok = __all_sync(0xffffffffu, ok);            // the TMEM loads below are warp-collective
+        fence_after();
+        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+        if (ok) {
+#pragma unroll
+            for (int c0 = 0; c0 < BN; c0 += 16) {
+                uint32_t r[16];
+                __syncwarp();
+                tmem_ld16(taddr + c0, r);
+                tmem_ld_wait();
+                if (!LOGITS) {
+                    if (feat < args.N) {
+                        float* dst = args.partial + ((size_t)(blockIdx.z * args.nmat + mat) * args.B) * args.N + feat;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (c0 + j < args.B) dst[(size_t)(c0 + j) * args.N] = __uint_as_float(r[j]);
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int col = c0 + j;
+                        if (col >= args.B) break;                         // uniform across the warp
+                        const float v = __uint_as_float(r[j]);
+                        unsigned long long key = feat < args.N ? argmax_key(v, feat) : 0ull;
+                        if (args.logits != nullptr && feat < args.N) args.logits[(size_t)col * args.N + feat] = v;
+                        key = warp_max_u64(key);
+                        if (lane == 0) s_keys[q * BN + col] = key;
+                    }
+                }
+            }
+        }
+        if (LOGITS) {
+            asm volatile("bar.sync 1, 128;" ::: "memory");                // the four epilogue warps only
+            const int col = threadIdx.x - 64;
+            if (ok && col < args.B) {
+                unsigned long long key = s_keys[col];
+#pragma unroll
+                for (int w = 1; w < 4; ++w) { const unsigned long long o = s_keys[w * BN + col]; key = o > key ? o : key; }
+                args.keys[(size_t)col * gridDim.x + ta] = key;
+            }
+        }
+    }
+
+    fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && *s_abort && args.error_word != nullptr) atomicExch(args.error_word, 1);
+    if (warp == 1) {
+        fence_after();
+        tmem_dealloc<kTmemCols>(tmem_base);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------- finishing kernel
+// Adds the fp32 split partials of one projection in a fixed order and applies its epilogue.
+struct FinishArgs {
+    const float* partial;   // [splits][nmat][B][N]
+    int splits, nmat, B, N;
+    bf16* out; int ldo;
+    const bf16* resid; int ldr;
+    bf16* out2; int ld2; RowMap orow2;     // second copy (per-slot state)
+    bf16* norm_out; const bf16* gain; float eps; int do_norm;   // RMSNorm of the stored result (optional)
+    bf16* kcache; bf16* vcache; int Hkv, dh, cap; RowMap slot; RowMap pos;
+};
+
+constexpr int kFinThreads = 256;
+constexpr int kFinCols = kFinThreads * 4;   // features per CTA and pass
+
+template <int MODE>
+__global__ void __launch_bounds__(kFinThreads) tc_finish_kernel(const FinishArgs a) {
+    const int b = blockIdx.x;
+    const size_t mstride = (size_t)a.B * a.N;
+    const size_t zstride = mstride * a.nmat;
+    const float* p0 = a.partial + (size_t)b * a.N;
+    const float* p1 = p0 + mstride;                 // second matrix (gate/up, K/V)
+    const bool whole_row = (MODE == SK_RESID && a.norm_out != nullptr);
+    const int n_begin = whole_row ? 0 : blockIdx.y * kFinCols;
+    const int n_end = whole_row ? a.N : min(a.N, n_begin + kFinCols);
+    float ss = 0.f;
+    for (int n = n_begin + threadIdx.x * 4; n < n_end; n += kFinThreads * 4) {     // N is a multiple of 4
+        float4 s0 = make_float4(0.f, 0.f, 0.f, 0.f), s1 = s0;
+        for (int z = 0; z < a.splits; ++z) {
+            const float4 t = *reinterpret_cast<const float4*>(p0 + z * zstride + n);
+            s0.x += t.x; s0.y += t.y; s0.z += t.z; s0.w += t.w;
+            if (MODE == SK_SILU_MUL || MODE == SK_KV) {
+                const float4 u = *reinterpret_cast<const float4*>(p1 + z * zstride + n);
+                s1.x += u.x; s1.y += u.y; s1.z += u.z; s1.w += u.w;
+            }
+        }
+        float v[4] = {s0.x, s0.y, s0.z, s0.w};
+        if (MODE == SK_SILU_MUL) {
+            v[0] = silu_f(s0.x) * s1.x; v[1] = silu_f(s0.y) * s1.y; v[2] = silu_f(s0.z) * s1.z; v[3] = silu_f(s0.w) * s1.w;
+        }
+        if (MODE == SK_RESID) {
+            const bf16* r = a.resid + (size_t)b * a.ldr + n;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) v[j] += __bfloat162float(r[j]);
+        }
+        if (MODE == SK_KV) {
+            const int slot = a.slot.idx[b], pos = a.pos.idx[b];
+            if (pos >= 0) {
+                const float v1[4] = {s1.x, s1.y, s1.z, s1.w};
+                const size_t at = (((size_t)slot * a.Hkv + n / a.dh) * a.cap + pos) * a.dh + n % a.dh;   // dh % 4 == 0
+#pragma unroll
+                for (int j = 0; j < 4; ++j) { a.kcache[at + j] = __float2bfloat16_rn(v[j]); a.vcache[at + j] = __float2bfloat16_rn(v1[j]); }
+            }
+        } else {
+            bf16 o[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) { o[j] = __float2bfloat16_rn(v[j]); const float f = __bfloat162float(o[j]); ss += f * f; }
+            bf16* dst = a.out + (size_t)b * a.ldo + n;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) dst[j] = o[j];
+            if (a.out2 != nullptr) {
+                bf16* d2 = a.out2 + (size_t)a.orow2.idx[b] * a.ld2 + n;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) d2[j] = o[j];
+            }
+        }
+    }
+    if (whole_row) {
+        __shared__ float s_part[kFinThreads / 32];
+        __shared__ float s_scale;
+        ss = warp_sum(ss);
+        if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = ss;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            float t = 0.f;
+            for (int w = 0; w < kFinThreads / 32; ++w) t += s_part[w];
+            s_scale = a.do_norm ? rsqrtf(t / (float)a.N + a.eps) : 1.0f;
+        }
+        __syncthreads();
+        const float sc = s_scale;
+        // each thread re-reads the values it wrote itself
+        for (int n = threadIdx.x * 4; n < a.N; n += kFinThreads * 4) {
+            const bf16* src = a.out + (size_t)b * a.ldo + n;
+            bf16* dst = a.norm_out + (size_t)b * a.ldo + n;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const float g = a.do_norm ? __bfloat162float(a.gain[n + j]) : 1.0f;
+                dst[j] = __float2bfloat16_rn(__bfloat162float(src[j]) * sc * g);
+            }
+        }
+    }
+}
+
+struct SplitPlan { int tiles, kb_total, kb_per_split, splits; };
+SplitPlan split_plan(int N, int K, int nmat, bool allow_split) {
+    SplitPlan s;
+    s.tiles = (N + BM - 1) / BM;
+    s.kb_total = (K + BK - 1) / BK;
+    int want = allow_split ? kCtaSlots / (s.tiles * nmat) : 1;
+    if (want < 1) want = 1;
+    s.kb_per_split = (s.kb_total + want - 1) / want;
+    if (s.kb_per_split < 4) s.kb_per_split = s.kb_total < 4 ? s.kb_total : 4;
+    s.splits = (s.kb_total + s.kb_per_split - 1) / s.kb_per_split;
+    return s;
+}
+
+template <int BN, bool LOGITS>
+int launch_sk(const CUtensorMap& w, const CUtensorMap& w2, const CUtensorMap& x, const SkArgs& args, dim3 grid, cudaStream_t stream) {
+    using SM = SkSmem<BN>;
+    static bool attr_done = false;
+    if (!attr_done) {
+        if (cudaFuncSetAttribute(tc_skinny_kernel<BN, LOGITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kBytes) != cudaSuccess) return -1;
+        attr_done = true;
+    }
+    tc_skinny_kernel<BN, LOGITS><<<grid, kSkThreads, SM::kBytes, stream>>>(w, w2, x, args);
+    return 1;
+}
+
+template <bool LOGITS>
+int launch_sk_bn(int bn, const CUtensorMap& w, const CUtensorMap& w2, const CUtensorMap& x, const SkArgs& args, dim3 grid, cudaStream_t stream) {
+    switch (bn) {
+        case 16: return launch_sk<16, LOGITS>(w, w2, x, args, grid, stream);
+        case 32: return launch_sk<32, LOGITS>(w, w2, x, args, grid, stream);
+        default: return launch_sk<64, LOGITS>(w, w2, x, args, grid, stream);
+    }
+}
+
+}  // namespace
+
+size_t tc_skinny_partial_bytes(int N, int K, int nmat) {
+    const SplitPlan s = split_plan(N, K, nmat, true);
+    return (size_t)s.splits * nmat * kMaxCallBatch * N * sizeof(float);
+}
+
+int tc_skinny_key_tiles(int N) { return (N + BM - 1) / BM; }
+
+int tc_skinny(TcPlan* p, int mode, const SkinnyArgs& g, cudaStream_t stream) {
+    if (p == nullptr || g.B <= 0 || g.B > kMaxCallBatch) return -1;
+    if (g.K % 8 || g.ldx % 8) return -1;                        // TMA: 16-byte row pitch
+    if (mode != SK_LOGITS && (g.N % 4)) return -1;              // finishing kernel: float4
+    if (reinterpret_cast<uintptr_t>(g.X) & 15) return -1;
+    if (mode == SK_KV && (g.dh % 4)) return -1;
+    const int nmat = (mode == SK_SILU_MUL || mode == SK_KV) ? 2 : 1;
+    const int bn = g.B <= 16 ? 16 : (g.B <= 32 ? 32 : 64);
+    const CUtensorMap* mapW = tc_weight_map(p, g.W, g.N, g.K, BM);
+    const CUtensorMap* mapW2 = nmat == 2 ? tc_weight_map(p, g.W2, g.N, g.K, BM) : mapW;
+    CUtensorMap mapX;
+    if (mapW == nullptr || mapW2 == nullptr || !tc_encode_map(p, &mapX, g.X, g.B, g.K, g.ldx, bn)) return -1;
+    const bool logits = (mode == SK_LOGITS);
+    const SplitPlan sp = split_plan(g.N, g.K, nmat, !logits);
+    SkArgs a;
+    memset(&a, 0, sizeof(a));
+    a.N = g.N; a.K = g.K; a.B = g.B; a.nmat = nmat; a.kb_per_split = sp.kb_per_split;
+    a.partial = g.partial; a.logits = g.logits; a.keys = g.keys; a.error_word = g.error_word;
+    dim3 grid(sp.tiles, nmat, sp.splits);
+    if (logits) return launch_sk_bn<true>(bn, *mapW, *mapW2, mapX, a, grid, stream);
+    if (launch_sk_bn<false>(bn, *mapW, *mapW2, mapX, a, grid, stream) < 0) return -1;
+
+    FinishArgs f;
+    memset(&f, 0, sizeof(f));
+    f.partial = g.partial; f.splits = sp.splits; f.nmat = nmat; f.B = g.B; f.N = g.N;
+    f.out = static_cast<bf16*>(g.out); f.ldo = g.ldo;
+    f.resid = static_cast<const bf16*>(g.resid); f.ldr = g.ldr;
+    f.out2 = static_cast<bf16*>(g.out2); f.ld2 = g.ld2; f.orow2 = g.orow2;
+    f.norm_out = static_cast<bf16*>(g.norm_out); f.gain = static_cast<const bf16*>(g.gain); f.eps = g.eps; f.do_norm = g.do_norm;
+    f.kcache = static_cast<bf16*>(g.kcache); f.vcache = static_cast<bf16*>(g.vcache); f.Hkv = g.Hkv; f.dh = g.dh; f.cap = g.cap;
+    f.slot = g.slot; f.pos = g.pos;
+    const bool whole_row = (mode == SK_RESID && g.norm_out != nullptr);
+    dim3 fgrid(g.B, whole_row ? 1 : (g.N + kFinCols - 1) / kFinCols);
+    switch (mode) {
+        case SK_STORE: tc_finish_kernel<SK_STORE><<<fgrid, kFinThreads, 0, stream>>>(f); break;
+        case SK_RESID: tc_finish_kernel<SK_RESID><<<fgrid, kFinThreads, 0, stream>>>(f); break;
+        case SK_SILU_MUL: tc_finish_kernel<SK_SILU_MUL><<<fgrid, kFinThreads, 0, stream>>>(f); break;
+        case SK_KV: tc_finish_kernel<SK_KV><<<fgrid, kFinThreads, 0, stream>>>(f); break;
+        default: return -1;
+    }
+    return 2;
+}
+
+}  // namespace beagle

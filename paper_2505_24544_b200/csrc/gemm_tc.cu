@@ -3,14 +3,9 @@
 // issued with tcgen05.mma by one thread.  Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer and
 // TMEM owner, warps 2..5 = epilogue (each reads its own quarter of the 128 TMEM lanes).
 //
-// Two uses of the same main loop:
-//   * dense projections of the block / prefill path: A = activations [M, K], B = weights [N, K];
-//     epilogues: store, +residual, SiLU(g)*u (two accumulators), fp32 logits, packed arg-max keys,
-//     scatter into the K/V cache;
-//   * serve-time projections for 9..64 rows ("swap-AB"): A = weights [N_out, K] so that the long
-//     dimension fills the 128 MMA rows, B = the batch's activations [<=64, K]; K may be split over
-//     blockIdx.z, each split writing fp32 partial sums that a finishing kernel reduces in a fixed
-//     order (deterministic), or, for the LM head, logits and arg-max keys directly.
+// Used by the dense projections of the block / prefill path: A = activations [M, K], B = weights
+// [N, K]; epilogues: store, +residual, SiLU(g)*u (two accumulators), fp32 logits, packed arg-max
+// keys, scatter into the K/V cache.
 //
 // Every wait on an mbarrier is bounded; a wait that runs out sets a device error word and the CTA
 // drains and frees its TMEM instead of hanging.
@@ -18,120 +13,33 @@
 
 #include <cstdio>
 #include <cstring>
-#include <map>
 
 #include "gemm_tc.h"
+#include "tc_plan.h"
+#include "tc_ptx.cuh"
 
 namespace beagle {
 
 namespace {
 
-constexpr int BM = 128, BK = 64, UMMA_K = 16;
-constexpr uint32_t kSpinLimit = 1u << 22;
+using namespace tc;
+constexpr int BM = 128;
 constexpr int kTcThreads = 192;
-
-// ---------------------------------------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok;
-}
-// Bounded wait.  Returns false when it gave up (and raises the CTA's abort flag).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 255u) == 255u && *abort_flag) return false;
-    }
-    *abort_flag = 1;
-    return false;
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1)
-        : "memory");
-}
-__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, uint64_t hint) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
-        ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "l"(hint)
-        : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes (64 elements),
-// 128-byte swizzled, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
-    uint64_t d = 0;
-    d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);   // start address, 16-byte units
-    d |= static_cast<uint64_t>(1024u >> 4) << 32;              // stride between 8-row groups
-    d |= static_cast<uint64_t>(1) << 46;                       // descriptor version of this architecture
-    d |= static_cast<uint64_t>(2) << 61;                       // 128-byte swizzle
-    return d;
-}
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr));
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-__host__ __device__ constexpr uint32_t make_idesc(int bn) {
-    return (1u << 4)            // D: fp32
-           | (1u << 7)          // A: bf16
-           | (1u << 10)         // B: bf16
-           | (static_cast<uint32_t>(bn >> 3) << 17) | (static_cast<uint32_t>(BM >> 4) << 24);   // K-major A and B
-}
 
 // ---------------------------------------------------------------------------------------------- kernel
 enum TcEpilogue {
-    TC_STORE = 0, TC_RESID = 1, TC_SILU_MUL = 2, TC_F32 = 3, TC_KV_CACHE = 4, TC_ARGMAX = 5,   // dense: rows = tile of A
-    TC_SKINNY_PARTIAL = 6,   // swap-AB: fp32 partial sums [z][col][a_rows]
-    TC_SKINNY_LOGITS = 7     // swap-AB LM head: logits[col][a_row] (optional) + arg-max keys [col][tile]
+    TC_STORE = 0, TC_RESID = 1, TC_SILU_MUL = 2, TC_F32 = 3, TC_KV_CACHE = 4, TC_ARGMAX = 5
 };
 
 struct TcArgs {
     int a_rows, b_rows, K;        // A: [a_rows, K]; B: [b_rows, K]
-    int kb_per_split;             // k-blocks of 64 per blockIdx.z slice
-    int group_m;                  // rasterisation: A tiles per group (dense path)
+    int group_m;                  // rasterisation: A tiles per group
     int tiles_a, tiles_b;
     void* C; int ldc;
     const void* R; int ldr;
     void* cache; int Hkv, dh, cap;
     SeqRows rows;
     unsigned long long* keys; int keys_ld;
-    float* partial; int partial_cols;     // skinny: [z][partial_cols][a_rows]
-    float* logits;
-    int valid_cols;                        // skinny: batch rows actually used
-    int a_rows_second;                     // skinny with two weight matrices: rows of each
     int* error_word;
 };
 
@@ -144,14 +52,12 @@ struct TcSmem {
 
 template <int BN, bool DUAL, int EPI>
 __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
-                                                            const __grid_constant__ CUtensorMap tmA2,
                                                             const __grid_constant__ CUtensorMap tmB,
                                                             const __grid_constant__ CUtensorMap tmB2, const TcArgs args) {
     using SM = TcSmem<BN, DUAL>;
     constexpr int kStages = SM::kStages;
     constexpr int kABytes = BM * BK * 2, kBBytes = BN * BK * 2;
     constexpr uint32_t kTmemCols = (DUAL ? 2 * BN : BN) < 32 ? 32 : (DUAL ? 2 * BN : BN);
-    constexpr bool SKINNY = (EPI == TC_SKINNY_PARTIAL || EPI == TC_SKINNY_LOGITS);
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -164,10 +70,7 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
 
     // tile coordinates
     int ta, tb;
-    if (SKINNY) {
-        ta = blockIdx.x;
-        tb = 0;
-    } else {
+    {
         const int pid = blockIdx.x;
         const int per_group = args.group_m * args.tiles_b;
         const int g = pid / per_group;
@@ -176,31 +79,25 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
         ta = first + (pid % per_group) % gsize;
         tb = (pid % per_group) / gsize;
     }
-    const int second = (SKINNY && args.a_rows_second > 0 && blockIdx.y == 1) ? 1 : 0;   // second weight matrix
-    const int kb0 = blockIdx.z * args.kb_per_split;
-    const int kb_total = (args.K + BK - 1) / BK;
-    const int nkb = max(0, min(args.kb_per_split, kb_total - kb0));
+    const int nkb = (args.K + BK - 1) / BK;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
         mbar_init(bar_acc, 1);
         *s_abort = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        fence_barrier_init();
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        tmem_alloc<kTmemCols>(smem_u32(s_tmem));
     }
-    tc_fence_before();
+    fence_before();
     __syncthreads();
-    tc_fence_after();
+    fence_after();
     const uint32_t tmem_base = *s_tmem;
 
     if (warp == 0) {
         // ---------------- TMA producer
         if (lane == 0) {
-            const CUtensorMap* mapA = second ? &tmA2 : &tmA;
             int issued = 0;
             for (int kb = 0; kb < nkb; ++kb) {
                 const int s = kb % kStages;
@@ -208,8 +105,8 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
                 if (!mbar_wait(bar_empty + 8 * s, ph ^ 1, s_abort)) break;
                 const uint32_t sa = smem_base + s * SM::kStageBytes, sb = sa + kABytes;
                 mbar_expect_tx(bar_full + 8 * s, kABytes + kBBytes * (DUAL ? 2 : 1));
-                const int kc = (kb0 + kb) * BK;
-                tma_load_2d(sa, mapA, bar_full + 8 * s, kc, ta * BM);
+                const int kc = kb * BK;
+                tma_load_2d(sa, &tmA, bar_full + 8 * s, kc, ta * BM);
                 tma_load_2d(sb, &tmB, bar_full + 8 * s, kc, tb * BN);
                 if (DUAL) tma_load_2d(sb + kBBytes, &tmB2, bar_full + 8 * s, kc, tb * BN);
                 ++issued;
@@ -227,14 +124,14 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     } else if (warp == 1) {
         // ---------------- MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc(BN);
+            constexpr uint32_t idesc = make_idesc(BM, BN);
             bool ok = true;
             for (int kb = 0; kb < nkb && ok; ++kb) {
                 const int s = kb % kStages;
                 const uint32_t ph = (kb / kStages) & 1;
                 ok = mbar_wait(bar_full + 8 * s, ph, s_abort);
                 if (!ok) break;
-                tc_fence_after();
+                fence_after();
                 const uint32_t sa = smem_base + s * SM::kStageBytes, sb = sa + kABytes;
                 const uint64_t da = umma_desc(sa), db = umma_desc(sb), db2 = umma_desc(sb + kBBytes);
 #pragma unroll
@@ -255,41 +152,11 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
         const int arow = ta * BM + row_in_tile;      // row of A this thread owns
         bool ok = true;
         if (nkb > 0) ok = mbar_wait(bar_acc, 0, s_abort);
-        tc_fence_after();
+        ok = __all_sync(0xffffffffu, ok);            // the TMEM loads below are warp-collective
+        fence_after();
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
         if (ok && nkb > 0) {
-            if (SKINNY) {
-                unsigned long long best = 0ull;
-                const int feat = arow;                                  // output feature
-                const int nrows_a = second ? args.a_rows_second : args.a_rows;
-#pragma unroll
-                for (int c0 = 0; c0 < BN; c0 += 16) {
-                    uint32_t r[16];
-                    __syncwarp();
-                    tmem_ld16(taddr + c0, r);
-                    tmem_ld_wait();
-                    if (EPI == TC_SKINNY_PARTIAL) {
-                        if (feat < nrows_a) {
-                            float* dst = args.partial + ((size_t)(blockIdx.z * 2 + second) * args.partial_cols) * args.a_rows;
-#pragma unroll
-                            for (int j = 0; j < 16; ++j)
-                                if (c0 + j < args.valid_cols) dst[(size_t)(c0 + j) * args.a_rows + feat] = __uint_as_float(r[j]);
-                        }
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const int col = c0 + j;
-                            if (col >= args.valid_cols) continue;           // uniform across the warp
-                            const float v = __uint_as_float(r[j]);
-                            unsigned long long key = feat < args.a_rows ? argmax_key(v, feat) : 0ull;
-                            if (args.logits != nullptr && feat < args.a_rows) args.logits[(size_t)col * args.a_rows + feat] = v;
-                            key = warp_max_u64(key);
-                            if (lane == 0) atomicMax(&args.keys[(size_t)col * args.keys_ld + ta], key);   // 4 warps share one slot
-                        }
-                    }
-                }
-                (void)best;
-            } else {
+            {
                 const int m = arow;
                 int slot = 0, pos = 0;
                 if (EPI == TC_KV_CACHE && m < args.a_rows) {
@@ -375,102 +242,12 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
         }
     }
 
-    tc_fence_before();
+    fence_before();
     __syncthreads();
     if (threadIdx.x == 0 && *s_abort && args.error_word != nullptr) atomicExch(args.error_word, 1);
     if (warp == 1) {
-        tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
-    }
-}
-
-// ---------------------------------------------------------------------------------------------- finishing kernels (serve path)
-// Sums the fp32 split-K partials of one projection in a fixed order and applies its epilogue.
-enum FinishMode { FIN_STORE = 0, FIN_RESID = 1, FIN_SILU_MUL = 2, FIN_KV = 3 };
-
-struct FinishArgs {
-    const float* partial;   // [z][2][cols][N]
-    int splits, cols, N;
-    int B;
-    bf16* out; int ldo;
-    const bf16* resid; int ldr;
-    bf16* out2; int ld2; RowMap orow2;     // second copy (per-slot state)
-    // fused RMSNorm of the result (optional): norm_out = out * rsqrt(mean(out^2)+eps) * gain
-    bf16* norm_out; const bf16* gain; float eps; int do_norm;
-    bf16* kcache; bf16* vcache; int Hkv, dh, cap; RowMap slot; RowMap pos;
-};
-
-template <int MODE>
-__global__ void __launch_bounds__(256) tc_finish_kernel(const FinishArgs a) {
-    const int b = blockIdx.x;
-    const size_t zstride = (size_t)2 * a.cols * a.N;
-    const float* p0 = a.partial + (size_t)b * a.N;                       // matrix 0
-    const float* p1 = a.partial + ((size_t)a.cols + b) * a.N;            // matrix 1 (gate/up, K/V)
-    float ss = 0.f;
-    for (int n = threadIdx.x * 4; n < a.N; n += blockDim.x * 4) {
-        float4 s0 = make_float4(0.f, 0.f, 0.f, 0.f), s1 = s0;
-        for (int z = 0; z < a.splits; ++z) {
-            const float4 t = *reinterpret_cast<const float4*>(p0 + z * zstride + n);
-            s0.x += t.x; s0.y += t.y; s0.z += t.z; s0.w += t.w;
-            if (MODE == FIN_SILU_MUL || MODE == FIN_KV) {
-                const float4 u = *reinterpret_cast<const float4*>(p1 + z * zstride + n);
-                s1.x += u.x; s1.y += u.y; s1.z += u.z; s1.w += u.w;
-            }
-        }
-        float v[4] = {s0.x, s0.y, s0.z, s0.w};
-        if (MODE == FIN_SILU_MUL) {
-            v[0] = silu_f(s0.x) * s1.x; v[1] = silu_f(s0.y) * s1.y; v[2] = silu_f(s0.z) * s1.z; v[3] = silu_f(s0.w) * s1.w;
-        }
-        if (MODE == FIN_RESID) {
-            const bf16* r = a.resid + (size_t)b * a.ldr + n;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) v[j] += __bfloat162float(r[j]);
-        }
-        if (MODE == FIN_KV) {
-            const int slot = a.slot.idx[b], pos = a.pos.idx[b];
-            if (pos >= 0) {
-                const float v1[4] = {s1.x, s1.y, s1.z, s1.w};
-                const size_t at = (((size_t)slot * a.Hkv + n / a.dh) * a.cap + pos) * a.dh + n % a.dh;   // dh % 4 == 0
-#pragma unroll
-                for (int j = 0; j < 4; ++j) { a.kcache[at + j] = __float2bfloat16_rn(v[j]); a.vcache[at + j] = __float2bfloat16_rn(v1[j]); }
-            }
-        } else {
-            bf16 o[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) { o[j] = __float2bfloat16_rn(v[j]); const float f = __bfloat162float(o[j]); ss += f * f; }
-            bf16* dst = a.out + (size_t)b * a.ldo + n;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) dst[j] = o[j];
-            if (a.out2 != nullptr) {
-                bf16* d2 = a.out2 + (size_t)a.orow2.idx[b] * a.ld2 + n;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) d2[j] = o[j];
-            }
-        }
-    }
-    if (MODE == FIN_RESID && a.norm_out != nullptr) {
-        __shared__ float s_part[8];
-        __shared__ float s_scale;
-        ss = warp_sum(ss);
-        if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = ss;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            float t = 0.f;
-            for (int w = 0; w < 8; ++w) t += s_part[w];
-            s_scale = a.do_norm ? rsqrtf(t / (float)a.N + a.eps) : 1.0f;
-        }
-        __syncthreads();
-        const float sc = s_scale;
-        // each thread re-reads the values it wrote itself
-        for (int n = threadIdx.x * 4; n < a.N; n += blockDim.x * 4) {
-            const bf16* src = a.out + (size_t)b * a.ldo + n;
-            bf16* dst = a.norm_out + (size_t)b * a.ldo + n;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const float g = a.do_norm ? __bfloat162float(a.gain[n + j]) : 1.0f;
-                dst[j] = __float2bfloat16_rn(__bfloat162float(src[j]) * sc * g);
-            }
-        }
+        fence_after();
+        tmem_dealloc<kTmemCols>(tmem_base);
     }
 }
 
@@ -484,24 +261,9 @@ __global__ void tc_keys_to_ids_kernel(const unsigned long long* __restrict__ key
     if (lane == 0) ids[warp] = argmax_key_index(k);
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
 }  // namespace
 
-struct TcPlan {
-    EncodeTiledFn encode = nullptr;
-    beagle_config cfg;
-    beagle_weights w;
-    std::map<std::pair<const void*, int>, CUtensorMap> weight_maps;   // (pointer, box rows) -> map
-    bool attr_set = false;
-};
-
-namespace {
-
-// K-major bf16 matrix [rows, K] (row stride ld elements), box = 64 columns x box_rows rows, 128-byte swizzle.
-bool encode_map(TcPlan* p, CUtensorMap* out, const void* base, long long rows, long long K, long long ld, int box_rows) {
+bool tc_encode_map(TcPlan* p, CUtensorMap* out, const void* base, long long rows, long long K, long long ld, int box_rows) {
     cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
     cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
@@ -512,25 +274,26 @@ bool encode_map(TcPlan* p, CUtensorMap* out, const void* base, long long rows, l
     return r == CUDA_SUCCESS;
 }
 
-const CUtensorMap* weight_map(TcPlan* p, const void* W, int rows, int K, int box_rows) {
+const CUtensorMap* tc_weight_map(TcPlan* p, const void* W, int rows, int K, int box_rows) {
     auto key = std::make_pair(W, box_rows);
     auto it = p->weight_maps.find(key);
     if (it != p->weight_maps.end()) return &it->second;
     CUtensorMap m;
-    if (!encode_map(p, &m, W, rows, K, K, box_rows)) return nullptr;
+    if (!tc_encode_map(p, &m, W, rows, K, K, box_rows)) return nullptr;
     return &p->weight_maps.emplace(key, m).first->second;
 }
 
+namespace {
+
 template <int BN, bool DUAL, int EPI>
-int launch_tc(const CUtensorMap& a, const CUtensorMap& a2, const CUtensorMap& b, const CUtensorMap& b2, const TcArgs& args, dim3 grid,
-              cudaStream_t stream) {
+int launch_tc(const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& b2, const TcArgs& args, dim3 grid, cudaStream_t stream) {
     using SM = TcSmem<BN, DUAL>;
     static bool attr_done = false;
     if (!attr_done) {
         if (cudaFuncSetAttribute(tc_gemm_kernel<BN, DUAL, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kBytes) != cudaSuccess) return -1;
         attr_done = true;
     }
-    tc_gemm_kernel<BN, DUAL, EPI><<<grid, kTcThreads, SM::kBytes, stream>>>(a, a2, b, b2, args);
+    tc_gemm_kernel<BN, DUAL, EPI><<<grid, kTcThreads, SM::kBytes, stream>>>(a, b, b2, args);
     return 1;
 }
 
@@ -555,6 +318,9 @@ TcPlan* tc_plan_create(const beagle_config& cfg, const beagle_weights& w, int* h
     p->encode = reinterpret_cast<EncodeTiledFn>(fn);
     p->cfg = cfg;
     p->w = w;
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+        p->sm_count = sms;
     return p;
 }
 
@@ -567,14 +333,13 @@ int tc_gemm(TcPlan* p, int epi, const GemmArgs& g, cudaStream_t stream) {
     const bool dual = (epi == GEMM_SILU_MUL);
     const int BN = dual ? 128 : 256;
     CUtensorMap mapA;
-    if (!encode_map(p, &mapA, g.A, g.M, g.K, g.lda, BM)) return -1;
-    const CUtensorMap* mapB = weight_map(p, g.W, g.N, g.K, BN);
-    const CUtensorMap* mapB2 = dual ? weight_map(p, g.W2, g.N, g.K, BN) : mapB;
+    if (!tc_encode_map(p, &mapA, g.A, g.M, g.K, g.lda, BM)) return -1;
+    const CUtensorMap* mapB = tc_weight_map(p, g.W, g.N, g.K, BN);
+    const CUtensorMap* mapB2 = dual ? tc_weight_map(p, g.W2, g.N, g.K, BN) : mapB;
     if (mapB == nullptr || mapB2 == nullptr) return -1;
     TcArgs a;
     memset(&a, 0, sizeof(a));
     a.a_rows = g.M; a.b_rows = g.N; a.K = g.K;
-    a.kb_per_split = (g.K + BK - 1) / BK;
     a.tiles_a = (g.M + BM - 1) / BM;
     a.tiles_b = (g.N + BN - 1) / BN;
     a.group_m = 16;
@@ -585,12 +350,12 @@ int tc_gemm(TcPlan* p, int epi, const GemmArgs& g, cudaStream_t stream) {
     if (epi == GEMM_KV_CACHE && (g.dh % 16)) return -1;
     dim3 grid(a.tiles_a * a.tiles_b, 1, 1);
     switch (epi) {
-        case GEMM_STORE: return launch_tc<256, false, TC_STORE>(mapA, mapA, *mapB, *mapB, a, grid, stream);
-        case GEMM_RESID: return launch_tc<256, false, TC_RESID>(mapA, mapA, *mapB, *mapB, a, grid, stream);
-        case GEMM_SILU_MUL: return launch_tc<128, true, TC_SILU_MUL>(mapA, mapA, *mapB, *mapB2, a, grid, stream);
-        case GEMM_F32: return launch_tc<256, false, TC_F32>(mapA, mapA, *mapB, *mapB, a, grid, stream);
-        case GEMM_KV_CACHE: return launch_tc<256, false, TC_KV_CACHE>(mapA, mapA, *mapB, *mapB, a, grid, stream);
-        case GEMM_ARGMAX_KEYS: return launch_tc<256, false, TC_ARGMAX>(mapA, mapA, *mapB, *mapB, a, grid, stream);
+        case GEMM_STORE: return launch_tc<256, false, TC_STORE>(mapA, *mapB, *mapB, a, grid, stream);
+        case GEMM_RESID: return launch_tc<256, false, TC_RESID>(mapA, *mapB, *mapB, a, grid, stream);
+        case GEMM_SILU_MUL: return launch_tc<128, true, TC_SILU_MUL>(mapA, *mapB, *mapB2, a, grid, stream);
+        case GEMM_F32: return launch_tc<256, false, TC_F32>(mapA, *mapB, *mapB, a, grid, stream);
+        case GEMM_KV_CACHE: return launch_tc<256, false, TC_KV_CACHE>(mapA, *mapB, *mapB, a, grid, stream);
+        case GEMM_ARGMAX_KEYS: return launch_tc<256, false, TC_ARGMAX>(mapA, *mapB, *mapB, a, grid, stream);
         default: return -1;
     }
 }

@@ -18,4 +18,34 @@ int tc_gemm(TcPlan* plan, int epi, const GemmArgs& a, cudaStream_t stream);
 int tc_argmax_tiles(int N);
 int tc_keys_to_ids(const unsigned long long* keys, int rows, int ntiles, int32_t* ids, cudaStream_t stream);
 
+// ---- serve-time projections for 9..64 rows ("swap-AB") -----------------------------------------
+// The weight matrix supplies the 128 MMA rows and the batch's activations the (<= 64) columns, so
+// the weights are streamed exactly once whatever the batch.  The reduction dimension may be split
+// across CTAs; each split writes fp32 partial sums that a finishing kernel adds in a fixed order
+// and passes through the projection's epilogue.  The LM head writes logits and arg-max keys directly.
+enum SkinnyMode {
+    SK_STORE = 0,      // out[b][n] = W[n,:] . x_b
+    SK_RESID = 1,      // out[b][n] = W[n,:] . x_b + resid[b][n]  (+ copy to out2[orow2[b]], + RMSNorm of the result to norm_out)
+    SK_SILU_MUL = 2,   // out[b][n] = SiLU(W[n,:] . x_b) * (W2[n,:] . x_b)
+    SK_KV = 3,         // W -> key cache, W2 -> value cache at (slot[b], head, pos[b]); pos[b] < 0 skips row b
+    SK_LOGITS = 4      // logits[b][n] fp32 (optional) and one arg-max key per (b, 128-row tile)
+};
+struct SkinnyArgs {
+    const void* W; const void* W2; int N, K;     // weights [N, K] row-major
+    const void* X; int ldx; int B;               // activations [B, K], row stride ldx, B <= 64
+    float* partial;                              // scratch, tc_skinny_partial_bytes() bytes
+    void* out; int ldo;
+    const void* resid; int ldr;
+    void* out2; int ld2; RowMap orow2;
+    void* norm_out; const void* gain; float eps; int do_norm;
+    void* kcache; void* vcache; int Hkv, dh, cap; RowMap slot; RowMap pos;
+    float* logits; unsigned long long* keys;     // keys: [B, tc_skinny_key_tiles(N)]
+    int* error_word;
+};
+// Kernels launched, or -1 when the shape is not covered.
+int tc_skinny(TcPlan* plan, int mode, const SkinnyArgs& a, cudaStream_t stream);
+// Bytes of fp32 partial sums a projection [N, K] with `nmat` weight matrices needs for 64 rows.
+size_t tc_skinny_partial_bytes(int N, int K, int nmat);
+int tc_skinny_key_tiles(int N);
+
 }  // namespace beagle

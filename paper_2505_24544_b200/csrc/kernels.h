@@ -41,9 +41,10 @@ int launch_gemv(int dtype, int mode, const GemvArgs& a, cudaStream_t stream);
 
 // x = E[token] (or rows of src), xn = RMSNorm(x) * g (or x when do_norm == 0).
 // tokens == NULL: row b uses last_token[meta.slot[b]].  src != NULL: no gather, rows of src.
+// gather_src != NULL: row b of gather_dst additionally receives row meta.slot[b] of gather_src.
 int launch_embed_norm(int dtype, const int32_t* tokens, const int32_t* last_token, const BatchMeta* meta,
                       const void* embed, int vocab, const void* src, const void* gain, int d, float eps, int do_norm,
-                      void* x_out, void* xn_out, int rows, cudaStream_t stream);
+                      void* x_out, void* xn_out, int rows, const void* gather_src, void* gather_dst, cudaStream_t stream);
 
 // Split-KV cross-attention decode over the cache + combine.  q, o: [B, Hq*dh] storage type.
 size_t attn_decode_scratch_bytes(int max_batch, int Hq, int dh, int max_kv);

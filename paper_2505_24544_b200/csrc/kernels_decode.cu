@@ -15,8 +15,13 @@ __global__ void __launch_bounds__(256) embed_norm_kernel(const int32_t* __restri
                                                          const T* __restrict__ embed, int vocab,
                                                          const T* __restrict__ src, const T* __restrict__ gain,
                                                          int d, float eps, int do_norm, T* __restrict__ x_out,
-                                                         T* __restrict__ xn_out) {
+                                                         T* __restrict__ xn_out, const T* __restrict__ gather_src,
+                                                         T* __restrict__ gather_dst) {
     const int r = blockIdx.x;
+    if (gather_src != nullptr) {
+        const T* g = gather_src + (size_t)meta.slot[r] * d;
+        for (int i = threadIdx.x; i < d; i += blockDim.x) gather_dst[(size_t)r * d + i] = g[i];
+    }
     const T* row;
     if (src != nullptr) {
         row = src + (size_t)r * d;
@@ -52,18 +57,18 @@ __global__ void __launch_bounds__(256) embed_norm_kernel(const int32_t* __restri
 
 int launch_embed_norm(int dtype, const int32_t* tokens, const int32_t* last_token, const BatchMeta* meta,
                       const void* embed, int vocab, const void* src, const void* gain, int d, float eps, int do_norm,
-                      void* x_out, void* xn_out, int rows, cudaStream_t stream) {
+                      void* x_out, void* xn_out, int rows, const void* gather_src, void* gather_dst, cudaStream_t stream) {
     if (rows <= 0) return 0;
     BatchMeta m;
     if (meta != nullptr) m = *meta; else memset(&m, 0, sizeof(m));
     if (dtype == 0)
         embed_norm_kernel<float><<<rows, 256, 0, stream>>>(tokens, last_token, m, (const float*)embed, vocab,
                                                            (const float*)src, (const float*)gain, d, eps, do_norm,
-                                                           (float*)x_out, (float*)xn_out);
+                                                           (float*)x_out, (float*)xn_out, (const float*)gather_src, (float*)gather_dst);
     else
         embed_norm_kernel<bf16><<<rows, 256, 0, stream>>>(tokens, last_token, m, (const bf16*)embed, vocab,
                                                           (const bf16*)src, (const bf16*)gain, d, eps, do_norm,
-                                                          (bf16*)x_out, (bf16*)xn_out);
+                                                          (bf16*)x_out, (bf16*)xn_out, (const bf16*)gather_src, (bf16*)gather_dst);
     return 1;
 }
 

@@ -1,0 +1,31 @@
+// Host-side state shared by the tensor-core kernels: the driver's tensor-map encoder and a cache
+// of the weight matrices' tensor maps.  Internal to the library.
+#pragma once
+#include <cuda.h>
+
+#include <map>
+#include <utility>
+
+#include "gemm_tc.h"
+
+namespace beagle {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct TcPlan {
+    EncodeTiledFn encode = nullptr;
+    beagle_config cfg;
+    beagle_weights w;
+    std::map<std::pair<const void*, int>, CUtensorMap> weight_maps;   // (pointer, box rows) -> map
+    int sm_count = 148;
+};
+
+// K-major bf16 matrix [rows, K] (row stride ld elements), box = 64 columns x box_rows rows,
+// 128-byte swizzle, out-of-range elements read as zero.
+bool tc_encode_map(TcPlan* p, CUtensorMap* out, const void* base, long long rows, long long K, long long ld, int box_rows);
+// Cached map of a weight matrix [rows, K] (dense, ld = K).
+const CUtensorMap* tc_weight_map(TcPlan* p, const void* W, int rows, int K, int box_rows);
+
+}  // namespace beagle

@@ -85,6 +85,37 @@ def test_small_bf16_ragged_batch_sd_iterations(w):
         first = np.array([out_ref[b, acc_ref[b]] for b in range(w.batch)])
 
 
+@pytest.mark.parametrize("batch", [9, 20, 40, 64])
+def test_batched_serving_tensor_core_projections(batch):
+    """Batches above 8 rows take the tensor-core projections (weights as the wide operand, split
+    reduction + finishing kernel); 9 / 20 / 40 / 64 rows cover the 16-, 32- and 64-column variants."""
+    w = SMALL_GQA.scaled(batch=batch, ctx_min=3, ctx_max=300, gamma=3, seed=2003, mlp_dim=1416)
+    head_gpu, head_cpu, _ = build(w, max_ctx=w.ctx_max + 64)
+    rng = WL.data_rng(w, batch)
+    lengths = WL.make_context_lengths(w, rng)
+    slots = list(rng.permutation(batch))                      # slot ids differ from batch rows
+    slots = [int(s) for s in slots]
+    seqs = prefill_both(head_gpu, head_cpu, w, rng, slots, lengths)          # > 64 rows: chunked / dense prefill
+    first = WL.make_tokens(w, rng, (batch,))
+    for it in range(2):
+        drafted, drafted_ref, _ = run_chain_parity(head_gpu, head_cpu, w, slots, seqs, first, w.gamma)
+        target = WL.make_target_stream(w, rng, drafted_ref)
+        acc, out = head_gpu.verify_greedy(to_dev(drafted_ref.astype(np.int32), w.dtype), target_ids=to_dev(target, w.dtype))
+        acc_ref, out_ref = O.verify_greedy(drafted_ref, target_ids=target)
+        np.testing.assert_array_equal(acc.cpu().numpy(), acc_ref)
+        new_len = (acc_ref + 1).astype(int)
+        hidden = WL.make_hidden(w, rng, int(new_len.sum()))                  # 9..256 rows: tensor-core prefill in chunks
+        head_gpu.prefill_kv(slots, list(map(int, new_len)), to_dev(hidden, w.dtype))
+        r = 0
+        for b, s in enumerate(seqs):
+            O.prefill_kv(head_cpu, s, hidden[r:r + new_len[b]])
+            r += new_len[b]
+            assert head_gpu.slot_lengths(slots[b]) == (s.n_true, 0)
+        first = np.array([out_ref[b, acc_ref[b]] for b in range(batch)])
+    from paper_2505_24544_b200.binding import beagle_check_device
+    beagle_check_device(head_gpu.ctx)
+
+
 def test_empty_cache_concat_off_and_rollback():
     w = SMALL_GQA.scaled(batch=2)
     head_gpu, head_cpu, _ = build(w)
