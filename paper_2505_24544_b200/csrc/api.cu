@@ -279,6 +279,8 @@ beagle_status beagle_create(const beagle_config* cfg, const beagle_weights* w, v
         delete c;
         return BEAGLE_ERR_CUDA;     // a GPU is present but the tensor-map encoder is not: never fall back silently
     }
+    if (c->tc != nullptr)
+        tc_attn_bind_cache(c->tc, c->kcache, c->vcache, (long long)cfg->max_slots * cfg->n_kv_heads * c->cap, cfg->head_dim);
     *out = c;
     return BEAGLE_OK;
 }
@@ -574,8 +576,15 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
     // (4) o = softmax(Q K^T / sqrt(dh)) V over the cache
     {
         StageTimer timer_(ctx, ST_ATTN_DECODE, stream);
-        rc = launch_attn_decode(dt, ctx->q, ctx->kcache, ctx->vcache, meta, batch, c.n_q_heads, c.n_kv_heads,
-                                c.head_dim, ctx->cap, max_kv, ctx->attn_scratch, ctx->o, stream);
+        rc = -1;
+        if (ctx->tc != nullptr) {       // bf16, head_dim 64 / 128: TMA-staged tiles
+            clear_error_word_once(ctx, stream);
+            rc = tc_attn_decode(ctx->tc, ctx->q, meta, batch, c.n_q_heads, c.n_kv_heads, c.head_dim, ctx->cap, max_kv,
+                                ctx->attn_scratch, ctx->o, ctx->dev_error, stream);
+        }
+        if (rc < 0)
+            rc = launch_attn_decode(dt, ctx->q, ctx->kcache, ctx->vcache, meta, batch, c.n_q_heads, c.n_kv_heads,
+                                    c.head_dim, ctx->cap, max_kv, ctx->attn_scratch, ctx->o, stream);
         if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "attention: unsupported head shape");
         ctx->launches += rc;
     }

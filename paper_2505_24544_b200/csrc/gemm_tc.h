@@ -48,4 +48,12 @@ int tc_skinny(TcPlan* plan, int mode, const SkinnyArgs& a, cudaStream_t stream);
 size_t tc_skinny_partial_bytes(int N, int K, int nmat);
 int tc_skinny_key_tiles(int N);
 
+// ---- TMA-staged decode attention over the bf16 cache (head_dim 64 or 128) ----------------------
+// Binds the cache halves ([rows, head_dim] each); false when the shape is not covered.
+bool tc_attn_bind_cache(TcPlan* plan, const void* kcache, const void* vcache, long long rows, int dh);
+// Split-KV partials + combine, as launch_attn_decode; -1 when not covered (caller falls back).
+int tc_attn_decode(TcPlan* plan, const void* q, const BatchMeta& meta, int B, int Hq, int Hkv, int dh, int cap, int max_kv_len,
+                   void* scratch, void* o, int* error_word, cudaStream_t stream);
+int tc_attn_chunk(void);
+
 }  // namespace beagle

@@ -52,6 +52,10 @@ int launch_attn_decode(int dtype, const void* q, const void* kcache, const void*
                        int B, int Hq, int Hkv, int dh, int cap, int max_kv_len, void* scratch, void* o,
                        cudaStream_t stream);
 
+// Merges the split-KV partials (unnormalised o, running max, exp-sum per chunk of `chunk` keys).
+int launch_attn_combine(int dtype, const float* part_o, const float* part_ml, const BatchMeta& meta, int B, int Hq, int dh,
+                        int nchunk_stride, int chunk, void* o, cudaStream_t stream);
+
 // tokens_out[b] (optional) and last_token[slot[b]] from the per-block keys.
 int launch_argmax_finalize(const unsigned long long* partials, int nblk, const BatchMeta& meta, int B,
                            int32_t* tokens_out, int tokens_out_stride, int32_t* last_token, cudaStream_t stream);

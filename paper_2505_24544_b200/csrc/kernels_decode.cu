@@ -223,6 +223,7 @@ int launch_gemv(int dtype, int mode, const GemvArgs& a, cudaStream_t stream) {
 // every key/value row it streams.  LPK lanes cover one cache row with one 16-byte load each.
 // ------------------------------------------------------------------------------------------------
 constexpr int kAttnChunk = 256;
+constexpr int kAttnMinChunk = 128;      // smallest chunk any decode kernel uses (sizes the partial buffers)
 constexpr int kAttnWarps = 4;
 
 template <typename T, int G, int LPK>
@@ -345,10 +346,10 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attn_decode_kernel(
 
 template <typename T>
 __global__ void attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
-                                    const BatchMeta meta, int Hq, int dh, int nchunk_max, T* __restrict__ o) {
+                                    const BatchMeta meta, int Hq, int dh, int nchunk_max, int chunk, T* __restrict__ o) {
     const int h = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
     const int kv_len = meta.kv_len[b];
-    const int nch = (kv_len + kAttnChunk - 1) / kAttnChunk;
+    const int nch = (kv_len + chunk - 1) / chunk;
     const size_t p0 = ((size_t)b * Hq + h) * nchunk_max;
     float M = -INFINITY;
     for (int i = 0; i < nch; ++i) M = fmaxf(M, part_ml[2 * (p0 + i)]);
@@ -361,8 +362,16 @@ __global__ void attn_combine_kernel(const float* __restrict__ part_o, const floa
     o[((size_t)b * Hq + h) * dh + c] = from_float<T>(nch > 0 ? num / den : 0.f);
 }
 
+int launch_attn_combine(int dtype, const float* part_o, const float* part_ml, const BatchMeta& meta, int B, int Hq, int dh,
+                        int nchunk_stride, int chunk, void* o, cudaStream_t stream) {
+    if (B <= 0) return 0;
+    if (dtype == 0) attn_combine_kernel<float><<<dim3(Hq, B), dh, 0, stream>>>(part_o, part_ml, meta, Hq, dh, nchunk_stride, chunk, (float*)o);
+    else attn_combine_kernel<bf16><<<dim3(Hq, B), dh, 0, stream>>>(part_o, part_ml, meta, Hq, dh, nchunk_stride, chunk, (bf16*)o);
+    return 1;
+}
+
 size_t attn_decode_scratch_bytes(int max_batch, int Hq, int dh, int max_kv) {
-    const size_t nch = (size_t)(max_kv + kAttnChunk - 1) / kAttnChunk + 1;
+    const size_t nch = (size_t)(max_kv + kAttnMinChunk - 1) / kAttnMinChunk + 1;
     const size_t rows = (size_t)max_batch * Hq * nch;
     return rows * dh * sizeof(float) + rows * 2 * sizeof(float) + 256;
 }
@@ -409,7 +418,7 @@ static int attn_dispatch(const void* q, const void* kc, const void* vc, const Ba
         if (rc < 0) return rc;
         launched += rc;
     }
-    attn_combine_kernel<T><<<dim3(Hq, B), dh, 0, stream>>>(po, pml, meta, Hq, dh, nch, (T*)o);
+    attn_combine_kernel<T><<<dim3(Hq, B), dh, 0, stream>>>(po, pml, meta, Hq, dh, nch, kAttnChunk, (T*)o);
     return launched + 1;
 }
 int launch_attn_decode(int dtype, const void* q, const void* kcache, const void* vcache, const BatchMeta& meta,

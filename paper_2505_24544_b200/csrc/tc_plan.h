@@ -20,6 +20,8 @@ struct TcPlan {
     beagle_weights w;
     std::map<std::pair<const void*, int>, CUtensorMap> weight_maps;   // (pointer, box rows) -> map
     int sm_count = 148;
+    CUtensorMap cache_k, cache_v;      // the K/V cache as [rows, head_dim] for the staged decode attention
+    bool cache_maps_ok = false;
 };
 
 // K-major bf16 matrix [rows, K] (row stride ld elements), box = 64 columns x box_rows rows,

@@ -131,7 +131,7 @@ def test_empty_cache_concat_off_and_rollback():
     assert head_gpu.slot_lengths(1) == (0, 3)
 
 
-@pytest.mark.parametrize("n", [255, 256, 257, 513])
+@pytest.mark.parametrize("n", [127, 128, 129, 255, 256, 257, 513])
 def test_split_kv_chunk_boundaries(n):
     w = SMALL_MHA.scaled(batch=1)
     head_gpu, head_cpu, _ = build(w, max_ctx=600)
