@@ -755,7 +755,14 @@ beagle_status beagle_block_forward(beagle_ctx* ctx, int32_t batch, int32_t S, co
         }
         {
             StageTimer timer_(ctx, ST_BLK_ATTN, stream);
-            rc = launch_attn_block(dt, Q, Kt, Vt, Kp, Vp, batch, S, c.n_q_heads, c.n_kv_heads, c.head_dim, block, offset, step, O, stream);
+            rc = -1;
+            if (ctx->tc != nullptr) {       // bf16, head_dim 64 / 128: tensor-core tiles
+                clear_error_word_once(ctx, stream);
+                rc = tc_attn_block(ctx->tc, Q, Kt, Vt, Kp, Vp, batch, S, c.n_q_heads, c.n_kv_heads, c.head_dim, block, offset, step, O,
+                                   ctx->dev_error, stream);
+            }
+            if (rc < 0)
+                rc = launch_attn_block(dt, Q, Kt, Vt, Kp, Vp, batch, S, c.n_q_heads, c.n_kv_heads, c.head_dim, block, offset, step, O, stream);
             if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "block attention: unsupported head_dim");
             ctx->launches += rc;
         }

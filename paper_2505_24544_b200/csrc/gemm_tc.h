@@ -56,4 +56,9 @@ int tc_attn_decode(TcPlan* plan, const void* q, const BatchMeta& meta, int B, in
                    void* scratch, void* o, int* error_word, cudaStream_t stream);
 int tc_attn_chunk(void);
 
+// ---- block-masked cross-attention of the multi-token forward (bf16, head_dim 64 or 128) -------
+// Same contract as launch_attn_block; -1 when not covered (caller falls back).
+int tc_attn_block(TcPlan* plan, const void* Q, const void* Kt, const void* Vt, const void* Kp, const void* Vp, int B, int S,
+                  int Hq, int Hkv, int dh, int block, int offset, int step, void* O, int* error_word, cudaStream_t stream);
+
 }  // namespace beagle

@@ -184,6 +184,27 @@ def test_block_forward_small_bf16_equals_oracle_and_sequential(sim_steps):
         assert_close(lg[0].cpu().numpy(), logits[0, n + i - 1].cpu().numpy().astype(np.float64), w.dtype, f"slot {i} block vs sequential")
 
 
+@pytest.mark.parametrize("S,block,offset,sim_steps", [(200, 5, 0, 3), (64, 2, 7, 2), (193, 3, 190, 1)])
+def test_block_forward_bf16_head_dim_128(S, block, offset, sim_steps):
+    """Tensor-core block attention with 128-wide heads: several query/key tiles, a ragged last
+    tile, an offset close to S (almost everything strict-causal) and the predicted-key band."""
+    w = SMALL_MHA
+    head_gpu, head_cpu, _ = build(w, max_slots=1, max_ctx=64)
+    rng = WL.data_rng(w, 1000 + S)
+    B = 2
+    tokens = WL.make_tokens(w, rng, (B, S))
+    hidden = WL.make_hidden(w, rng, B * S).reshape(B, S, w.hidden)
+    logits, argmax, hid = head_gpu.block_forward(to_dev(tokens, w.dtype), to_dev(hidden, w.dtype), block, offset, sim_steps)
+    torch.cuda.synchronize()
+    for b in range(B):
+        ref = O.block_forward(head_cpu, tokens[b], hidden[b], block, offset, sim_steps)
+        assert_close(logits[b].cpu().numpy(), ref["logits"], w.dtype, f"seq {b} logits")
+        assert_close(hid[b].float().cpu().numpy(), ref["hidden"], w.dtype, f"seq {b} hidden")
+        check_tokens(argmax[b].cpu().numpy(), ref["logits"], f"seq {b} argmax")
+    from paper_2505_24544_b200.binding import beagle_check_device
+    beagle_check_device(head_gpu.ctx)
+
+
 def test_verify_greedy_logits_both_dtypes_and_ties():
     w = SMALL_GQA.scaled(batch=5, gamma=6)
     head_gpu, _, _ = build(w)
