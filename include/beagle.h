@@ -196,6 +196,33 @@ beagle_status beagle_profile_read(beagle_ctx* ctx, float* ms_out_host, int32_t* 
 int32_t beagle_profile_stage_count(void);
 const char* beagle_profile_stage_name(int32_t stage);
 
+/* Inspection of the intermediate vectors (no counterpart in the paper; test support).  Every step of
+ * Eq. 1 / Eq. 2 leaves its result in the caller-owned workspace; these calls say where, so that a
+ * checker can compare each kernel's output with the definition applied to that kernel's own inputs.
+ * Rows are the batch rows of the most recent beagle_draft_step (serve) or the batch*S positions of
+ * the most recent beagle_block_forward (block), row-major in the storage type. */
+enum {
+    BEAGLE_BUF_X = 0,      /* e(t)                              [rows, d]      */
+    BEAGLE_BUF_XN = 1,     /* RMSNorm(e(t); g_q)                [rows, d]      */
+    BEAGLE_BUF_Q = 2,      /* W_q xn                            [rows, Hq*dh]  */
+    BEAGLE_BUF_O = 3,      /* attention output                  [rows, Hq*dh]  */
+    BEAGLE_BUF_Y = 4,      /* W_o o + e(t)                      [rows, d]      */
+    BEAGLE_BUF_YN = 5,     /* RMSNorm(y; g_mlp)                 [rows, d]      */
+    BEAGLE_BUF_ACT = 6,    /* SiLU(W_gate yn) * (W_up yn)       [rows, m]      */
+    BEAGLE_BUF_H = 7,      /* W_down act + y                    [rows, d]      */
+    BEAGLE_BUF_KT = 8,     /* block path only: K of the true states       [rows, Hkv*dh] */
+    BEAGLE_BUF_VT = 9,     /* block path only: V of the true states       [rows, Hkv*dh] */
+    BEAGLE_BUF_KP = 10,    /* block path only: K of the predicted states  [rows, Hkv*dh] */
+    BEAGLE_BUF_VP = 11,    /* block path only: V of the predicted states  [rows, Hkv*dh] */
+    BEAGLE_BUF_COUNT = 12
+};
+/* Byte offset and row width (elements) of a serve-time buffer inside the workspace given to beagle_create. */
+beagle_status beagle_workspace_buffer(const beagle_config* cfg, int32_t which, size_t* offset_bytes, int32_t* row_elems);
+/* The same for the workspace of beagle_block_forward(batch, S).  BEAGLE_BUF_H is only meaningful
+ * when hidden_out_dev was NULL (otherwise h went to the caller's buffer). */
+beagle_status beagle_block_workspace_buffer(const beagle_config* cfg, int32_t batch, int32_t S, int32_t which,
+                                            size_t* offset_bytes, int32_t* row_elems);
+
 /* Waits for the stream, then reports BEAGLE_ERR_DEVICE if any kernel of this context abandoned a
  * bounded wait (its outputs are then undefined).  The only call that synchronises. */
 beagle_status beagle_check_device(beagle_ctx* ctx, void* stream);

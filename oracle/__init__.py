@@ -10,11 +10,18 @@ from .beagle_oracle import (  # noqa: F401
     OracleHead,
     OracleSequence,
     rms_norm,
+    round_bf16,
     silu,
     visible_true_count,
     project_kv,
     attention_weights,
     cross_attention,
+    embed_tokens,
+    query_projection,
+    attention_rows,
+    output_projection,
+    mlp_block,
+    lm_head,
     draft_block,
     prefill_kv,
     rollback,

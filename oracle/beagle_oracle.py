@@ -34,6 +34,17 @@ stated in the function that uses them):
   * a query with no visible key gets o = 0;
   * argmax ties go to the lowest index, NaN never wins.
 
+Storage mode.  By default nothing is rounded.  With ``HeadConfig.storage = "bf16"`` the
+values that a bf16 deployment keeps in memory between two operations -- the
+normalised query input, Q, the K/V cache rows, the attention output o, y, the
+normalised MLP input, the MLP hidden vector and the block output h -- are
+rounded to bf16 (round to nearest, ties to even) exactly where they would be
+stored; everything in between stays float64 and the logits are not rounded.
+This is the reading "weights, states and cache in bf16" of the bf16 workloads:
+at the full model sizes the rounding of the cache alone moves logits of
+standard deviation ~2.7 by up to ~5e-2, so a comparison that wants to see
+kernel errors rather than storage noise has to round at the same places.
+
 Pins (tests/test_oracle_*.py, all CPU): hand-worked tiny head, softmax row
 sums, single-key / identical-key special cases, GQA==MHA with repeated heads,
 mask brute force against the literal window rule, block forward == step-by-step
@@ -64,6 +75,7 @@ class HeadConfig:
     rms_eps: float = 1e-5
     norm_q: bool = True
     norm_mlp: bool = True
+    storage: Optional[str] = None   # None: never round; "bf16": round stored intermediates (module docstring)
 
     @property
     def group(self) -> int:
@@ -99,7 +111,38 @@ class OracleHead:
             setattr(self, name, w)
 
 
+    def with_storage(self, storage: Optional[str]) -> "OracleHead":
+        """The same parameters (shared arrays) under another storage mode."""
+        import copy
+        from dataclasses import replace
+        other = copy.copy(self)
+        other.cfg = replace(self.cfg, storage=storage)
+        return other
+
+
 # --------------------------------------------------------------------------- primitives
+
+def round_bf16(a: np.ndarray) -> np.ndarray:
+    """Round float64 values to the nearest bfloat16 (8 significand bits, ties to
+    even), returned as float64.  The 64-bit pattern is rounded directly at the
+    bf16 significand width, so there is no double rounding through float32.
+    For finite inputs inside the bf16 normal range (all values met here)."""
+    a = np.ascontiguousarray(a, dtype=F64)
+    u = a.view(np.uint64)
+    drop = np.uint64(52 - 7)                      # float64 keeps 52 fraction bits, bf16 keeps 7
+    lsb = (u >> drop) & np.uint64(1)
+    r = (u + ((np.uint64(1) << (drop - np.uint64(1))) - np.uint64(1)) + lsb) & ~((np.uint64(1) << drop) - np.uint64(1))
+    return r.view(F64).reshape(a.shape)
+
+
+def _stored(cfg: "HeadConfig", a: np.ndarray) -> np.ndarray:
+    """A value as it is kept in memory under the configuration's storage mode."""
+    if cfg.storage is None:
+        return a
+    if cfg.storage == "bf16":
+        return round_bf16(a)
+    raise ValueError(f"unknown storage mode {cfg.storage!r}")
+
 
 def rms_norm(v: np.ndarray, g: np.ndarray, eps: float) -> np.ndarray:
     """RMSNorm over the last axis: g * v / sqrt(mean(v^2) + eps)."""
@@ -147,8 +190,8 @@ def project_kv(head: OracleHead, states: np.ndarray) -> Tuple[np.ndarray, np.nda
     Returns K, V of shape [n, Hkv, d_h]  (Eq. 2, first line)."""
     c = head.cfg
     s = np.asarray(states, dtype=F64).reshape(-1, c.hidden)
-    k = s @ head.w_k.T
-    v = s @ head.w_v.T
+    k = _stored(c, s @ head.w_k.T)
+    v = _stored(c, s @ head.w_v.T)
     return (k.reshape(-1, c.n_kv_heads, c.head_dim), v.reshape(-1, c.n_kv_heads, c.head_dim))
 
 
@@ -186,6 +229,50 @@ def cross_attention(head: OracleHead, q: np.ndarray, k_vis: np.ndarray,
 
 # --------------------------------------------------------------------------- Eq. 1
 
+def embed_tokens(head: OracleHead, tokens: Sequence[int]) -> np.ndarray:
+    """x = e(t_p): rows of the embedding table."""
+    tok = np.asarray(tokens, dtype=np.int64).reshape(-1)
+    if np.any(tok < 0) or np.any(tok >= head.cfg.vocab):
+        raise ValueError("token id out of range")
+    return head.embed[tok]
+
+
+def query_projection(head: OracleHead, x: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """(xq, Q): xq = RMSNorm(x; g_q) (or x when the flag is off), Q = W_Q^T xq  (Eq. 2, first line)."""
+    c = head.cfg
+    xq = _stored(c, rms_norm(x, head.g_q, c.rms_eps)) if c.norm_q else np.asarray(x, dtype=F64)
+    return xq, _stored(c, xq @ head.w_q.T)
+
+
+def attention_rows(head: OracleHead, q: np.ndarray,
+                   kv_vis: Sequence[Tuple[np.ndarray, np.ndarray]]) -> np.ndarray:
+    """o for independent query rows: row r reads kv_vis[r] = (K, V) of its visible states."""
+    c = head.cfg
+    o = np.zeros((q.shape[0], c.n_q_heads * c.head_dim), dtype=F64)
+    for r in range(q.shape[0]):
+        k_vis, v_vis = kv_vis[r]
+        o[r] = cross_attention(head, q[r].reshape(c.n_q_heads, c.head_dim), k_vis, v_vis)
+    return _stored(c, o)
+
+
+def output_projection(head: OracleHead, o: np.ndarray, x: np.ndarray) -> np.ndarray:
+    """y = W_O^T [o^1..o^H] + e(t_p)  (Eq. 2 last line and the residual of Eq. 1)."""
+    return _stored(head.cfg, o @ head.w_o.T + x)
+
+
+def mlp_block(head: OracleHead, y: np.ndarray) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """(yn, act, h): yn = RMSNorm(y; g_mlp), act = SiLU(W_gate yn) * (W_up yn), h = W_down act + y  (Eq. 1)."""
+    c = head.cfg
+    yn = _stored(c, rms_norm(y, head.g_mlp, c.rms_eps)) if c.norm_mlp else np.asarray(y, dtype=F64)
+    act = _stored(c, silu(yn @ head.w_gate.T) * (yn @ head.w_up.T))
+    return yn, act, _stored(c, act @ head.w_down.T + y)
+
+
+def lm_head(head: OracleHead, h: np.ndarray) -> np.ndarray:
+    """z = e^{-1}(h): the linear map to the vocabulary."""
+    return np.asarray(h, dtype=F64) @ head.w_lm.T
+
+
 def draft_block(head: OracleHead, tokens: Sequence[int],
                 kv_vis: Sequence[Tuple[np.ndarray, np.ndarray]]) -> Dict[str, np.ndarray]:
     """The draft Transformer block (Eq. 1) and the LM head for a set of
@@ -196,23 +283,13 @@ def draft_block(head: OracleHead, tokens: Sequence[int],
     is re-used as key/value input when drafting continues), logits z and the
     greedy token argmax z.
     """
-    c = head.cfg
-    tok = np.asarray(tokens, dtype=np.int64).reshape(-1)
-    if np.any(tok < 0) or np.any(tok >= c.vocab):
-        raise ValueError("token id out of range")
-    x = head.embed[tok]                                         # e(t_p)
-    xq = rms_norm(x, head.g_q, c.rms_eps) if c.norm_q else x
-    q = xq @ head.w_q.T                                         # Q = W_Q^T e(t_p)
-    o = np.zeros((len(tok), c.n_q_heads * c.head_dim), dtype=F64)
-    for r in range(len(tok)):
-        k_vis, v_vis = kv_vis[r]
-        o[r] = cross_attention(head, q[r].reshape(c.n_q_heads, c.head_dim), k_vis, v_vis)
-    y = o @ head.w_o.T + x                                      # y = W_O^T[o] + e(t_p)
-    yn = rms_norm(y, head.g_mlp, c.rms_eps) if c.norm_mlp else y
-    mlp = (silu(yn @ head.w_gate.T) * (yn @ head.w_up.T)) @ head.w_down.T
-    h = mlp + y                                                 # h = MLP(y) + y
-    z = h @ head.w_lm.T                                         # z = e^{-1}(h)
-    return {"x": x, "q": q, "o": o, "y": y, "h": h, "logits": z, "argmax": argmax_lowest(z)}
+    x = embed_tokens(head, tokens)                              # e(t_p)
+    xq, q = query_projection(head, x)                           # Q = W_Q^T e(t_p)
+    o = attention_rows(head, q, kv_vis)
+    y = output_projection(head, o, x)                           # y = W_O^T[o] + e(t_p)
+    yn, act, h = mlp_block(head, y)                             # h = MLP(y) + y
+    z = lm_head(head, h)                                        # z = e^{-1}(h)
+    return {"x": x, "xn": xq, "q": q, "o": o, "y": y, "yn": yn, "act": act, "h": h, "logits": z, "argmax": argmax_lowest(z)}
 
 
 # --------------------------------------------------------------------------- serve-time drafting

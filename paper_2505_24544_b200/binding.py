@@ -27,7 +27,10 @@ EXPORTED_SYMBOLS = (
     "beagle_block_workspace_bytes", "beagle_block_forward", "beagle_verify_greedy", "beagle_last_error",
     "beagle_launch_count", "beagle_profile_enable", "beagle_profile_read", "beagle_profile_stage_count",
     "beagle_profile_stage_name", "beagle_verify_greedy_static", "beagle_check_device",
+    "beagle_workspace_buffer", "beagle_block_workspace_buffer",
 )
+
+BUFFER_IDS = {"x": 0, "xn": 1, "q": 2, "o": 3, "y": 4, "yn": 5, "act": 6, "h": 7, "kt": 8, "vt": 9, "kp": 10, "vp": 11}
 
 
 class BeagleConfig(C.Structure):
@@ -87,6 +90,10 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.beagle_profile_stage_name.restype = C.c_char_p
     lib.beagle_verify_greedy_static.argtypes = [i32, i32, i32, vp, vp, i32, vp, vp, vp, C.c_char_p, C.c_size_t]
     lib.beagle_verify_greedy_static.restype = C.c_int
+    lib.beagle_workspace_buffer.argtypes = [C.POINTER(BeagleConfig), i32, szp, i32p]
+    lib.beagle_workspace_buffer.restype = C.c_int
+    lib.beagle_block_workspace_buffer.argtypes = [C.POINTER(BeagleConfig), i32, i32, i32, szp, i32p]
+    lib.beagle_block_workspace_buffer.restype = C.c_int
     lib.beagle_check_device.argtypes = [vp, vp]
     lib.beagle_check_device.restype = C.c_int
     lib.beagle_launch_count.restype = C.c_int64
@@ -256,6 +263,41 @@ def beagle_verify_greedy_static(draft_tokens: torch.Tensor, target_logits: torch
                                                     _stream(), err, len(err))
     if st != 0:
         raise BeagleError(st, err.value.decode())
+
+
+def beagle_workspace_buffer(ctx: Context, name: str, rows: int) -> torch.Tensor:
+    """View of an intermediate vector of the most recent draft step ([rows, width], storage type)."""
+    off, width = C.c_size_t(), C.c_int32()
+    st = ctx.lib.beagle_workspace_buffer(C.byref(ctx.cfg), BUFFER_IDS[name], C.byref(off), C.byref(width))
+    if st != 0:
+        raise BeagleError(st, f"beagle_workspace_buffer({name})")
+    dt = torch_dtype(ctx.cfg.dtype)
+    n = rows * width.value * dt.itemsize
+    return ctx.ws_buf[off.value:off.value + n].view(dt).view(rows, width.value)
+
+
+def beagle_block_workspace_buffer(ctx: Context, name: str, batch: int, S: int) -> torch.Tensor:
+    """View of an intermediate matrix of the most recent block forward ([batch*S, width], storage type)."""
+    off, width = C.c_size_t(), C.c_int32()
+    st = ctx.lib.beagle_block_workspace_buffer(C.byref(ctx.cfg), batch, S, BUFFER_IDS[name], C.byref(off), C.byref(width))
+    if st != 0:
+        raise BeagleError(st, f"beagle_block_workspace_buffer({name})")
+    dt = torch_dtype(ctx.cfg.dtype)
+    rows = batch * S
+    n = rows * width.value * dt.itemsize
+    return ctx.block_ws[off.value:off.value + n].view(dt).view(rows, width.value)
+
+
+def kv_cache_views(ctx: Context) -> Tuple[torch.Tensor, torch.Tensor]:
+    """The caller-owned cache as ([slot, Hkv, max_ctx + max_draft, dh]) key and value tensors."""
+    c = ctx.cfg
+    dt = torch_dtype(c.dtype)
+    cap = c.max_ctx + c.max_draft
+    half = ctx.kv_buf.numel() // 2
+    n = c.max_slots * c.n_kv_heads * cap * c.head_dim * dt.itemsize
+    k = ctx.kv_buf[:n].view(dt).view(c.max_slots, c.n_kv_heads, cap, c.head_dim)
+    v = ctx.kv_buf[half:half + n].view(dt).view(c.max_slots, c.n_kv_heads, cap, c.head_dim)
+    return k, v
 
 
 def beagle_check_device(ctx: Context) -> None:

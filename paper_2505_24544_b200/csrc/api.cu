@@ -229,6 +229,52 @@ beagle_status beagle_query_sizes(const beagle_config* cfg, size_t* kv_bytes, siz
     return BEAGLE_OK;
 }
 
+beagle_status beagle_workspace_buffer(const beagle_config* cfg, int32_t which, size_t* offset_bytes, int32_t* row_elems) {
+    const beagle_status st = check_config(cfg);
+    if (st != BEAGLE_OK) return st;
+    if (offset_bytes == nullptr || row_elems == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    const ServeLayout L = serve_layout(*cfg);
+    const int d = cfg->hidden, qd = cfg->n_q_heads * cfg->head_dim, m = cfg->mlp_dim;
+    switch (which) {
+        case BEAGLE_BUF_X: *offset_bytes = L.x; *row_elems = d; break;
+        case BEAGLE_BUF_XN: *offset_bytes = L.xn; *row_elems = d; break;
+        case BEAGLE_BUF_Q: *offset_bytes = L.q; *row_elems = qd; break;
+        case BEAGLE_BUF_O: *offset_bytes = L.o; *row_elems = qd; break;
+        case BEAGLE_BUF_Y: *offset_bytes = L.y; *row_elems = d; break;
+        case BEAGLE_BUF_YN: *offset_bytes = L.yn; *row_elems = d; break;
+        case BEAGLE_BUF_ACT: *offset_bytes = L.act; *row_elems = m; break;
+        case BEAGLE_BUF_H: *offset_bytes = L.h; *row_elems = d; break;
+        default: return BEAGLE_ERR_INVALID_ARG;
+    }
+    return BEAGLE_OK;
+}
+
+beagle_status beagle_block_workspace_buffer(const beagle_config* cfg, int32_t batch, int32_t S, int32_t which,
+                                            size_t* offset_bytes, int32_t* row_elems) {
+    const beagle_status st = check_config(cfg);
+    if (st != BEAGLE_OK) return st;
+    if (offset_bytes == nullptr || row_elems == nullptr || batch <= 0 || S <= 0) return BEAGLE_ERR_INVALID_ARG;
+    if ((long long)batch * S > (1ll << 24)) return BEAGLE_ERR_CAPACITY;
+    const BlockLayout L = block_layout(*cfg, batch, S);
+    const int d = cfg->hidden, qd = cfg->n_q_heads * cfg->head_dim, kd = cfg->n_kv_heads * cfg->head_dim, m = cfg->mlp_dim;
+    switch (which) {
+        case BEAGLE_BUF_X: *offset_bytes = L.x; *row_elems = d; break;
+        case BEAGLE_BUF_XN: *offset_bytes = L.xn; *row_elems = d; break;
+        case BEAGLE_BUF_Q: *offset_bytes = L.q; *row_elems = qd; break;
+        case BEAGLE_BUF_O: *offset_bytes = L.o; *row_elems = qd; break;
+        case BEAGLE_BUF_Y: *offset_bytes = L.y; *row_elems = d; break;
+        case BEAGLE_BUF_YN: *offset_bytes = L.yn; *row_elems = d; break;
+        case BEAGLE_BUF_ACT: *offset_bytes = L.act; *row_elems = m; break;
+        case BEAGLE_BUF_H: *offset_bytes = L.h; *row_elems = d; break;
+        case BEAGLE_BUF_KT: *offset_bytes = L.kt; *row_elems = kd; break;
+        case BEAGLE_BUF_VT: *offset_bytes = L.vt; *row_elems = kd; break;
+        case BEAGLE_BUF_KP: *offset_bytes = L.kp; *row_elems = kd; break;
+        case BEAGLE_BUF_VP: *offset_bytes = L.vp; *row_elems = kd; break;
+        default: return BEAGLE_ERR_INVALID_ARG;
+    }
+    return BEAGLE_OK;
+}
+
 beagle_status beagle_create(const beagle_config* cfg, const beagle_weights* w, void* kv_dev, size_t kv_bytes,
                             void* workspace_dev, size_t workspace_bytes, beagle_ctx** out) {
     if (out == nullptr) return BEAGLE_ERR_INVALID_ARG;

@@ -415,6 +415,46 @@ def test_against_torch_library_routines():
     np.testing.assert_array_equal(ours["argmax"], z.argmax(-1).numpy())
 
 
+# ----------------------------------------------------------------------------- storage mode
+
+def test_round_bf16_ties_to_even_and_matches_torch():
+    torch = pytest.importorskip("torch")
+    # exact halves between two bf16 neighbours (spacing 2^-7 in [1, 2)) go to the even one
+    np.testing.assert_array_equal(O.round_bf16(np.array([1 + 2.0 ** -8, 1 + 3 * 2.0 ** -8, -(1 + 2.0 ** -8), 0.0, 1.5])),
+                                  [1.0, 1 + 2.0 ** -6, -1.0, 0.0, 1.5])
+    # a float64 just above a half rounds up although float32 would first round it onto the half
+    np.testing.assert_array_equal(O.round_bf16(np.array([1 + 2.0 ** -8 + 2.0 ** -40])), [1 + 2.0 ** -7])
+    rng = np.random.default_rng(61)
+    a = (rng.normal(size=20000) * 10.0 ** rng.uniform(-5, 5, size=20000)).astype(np.float32).astype(np.float64)
+    t = torch.from_numpy(a.astype(np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+    np.testing.assert_array_equal(O.round_bf16(a), t)
+    np.testing.assert_array_equal(O.round_bf16(t), t)                       # idempotent
+
+
+def test_storage_mode_rounds_only_where_values_are_stored():
+    head, w, rng = small_head(seed=62)
+    c = head.cfg
+    rounded = head.with_storage("bf16")
+    assert rounded.w_q is head.w_q and head.cfg.storage is None            # shared arrays, default untouched
+    states = rng.normal(size=(9, c.hidden))
+    toks = [1, 2, 3]
+    exact = O.draft_block(head, toks, [O.project_kv(head, states)] * 3)
+    stored = O.draft_block(rounded, toks, [O.project_kv(rounded, states)] * 3)
+    for name in ("q", "o", "y", "h"):                                       # stored values are bf16 numbers ...
+        np.testing.assert_array_equal(O.round_bf16(stored[name]), stored[name])
+        assert np.abs(stored[name] - exact[name]).max() > 0                 # ... and differ from the unrounded ones
+        assert np.abs(stored[name] - exact[name]).max() <= 0.05 * (1 + np.abs(exact[name]).max())
+    k, v = O.project_kv(rounded, states)
+    np.testing.assert_array_equal(O.round_bf16(k), k)
+    assert np.abs(O.round_bf16(stored["logits"]) - stored["logits"]).max() > 0      # logits are not rounded
+    # a sequence driven through the cache API sees the same rounded keys
+    seq = O.OracleSequence(rounded)
+    O.prefill_kv(rounded, seq, states)
+    np.testing.assert_array_equal(seq.k_true, k)
+    with pytest.raises(ValueError):
+        O.project_kv(head.with_storage("fp8"), states)
+
+
 # ----------------------------------------------------------------------------- generators
 
 def test_bf16_rounding_of_generator_matches_torch():
