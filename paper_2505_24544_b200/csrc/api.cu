@@ -625,7 +625,9 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
         rc = -1;
         if (ctx->tc != nullptr) {       // bf16, head_dim 64 / 128: TMA-staged tiles
             clear_error_word_once(ctx, stream);
-            rc = tc_attn_decode(ctx->tc, ctx->q, meta, batch, c.n_q_heads, c.n_kv_heads, c.head_dim, ctx->cap, max_kv,
+            int32_t stable[kMaxCallBatch];
+            for (int b = 0; b < batch; ++b) stable[b] = ctx->n_true[seq_slot[b]];
+            rc = tc_attn_decode(ctx->tc, ctx->q, meta, stable, batch, c.n_q_heads, c.n_kv_heads, c.head_dim, ctx->cap, max_kv,
                                 ctx->attn_scratch, ctx->o, ctx->dev_error, stream);
         }
         if (rc < 0)

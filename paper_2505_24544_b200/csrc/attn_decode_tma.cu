@@ -36,6 +36,7 @@ struct AttnWork {                       // by value in the kernel parameters
     int32_t slot[kMaxCallBatch];
     int32_t kv_len[kMaxCallBatch];
     int32_t item_start[kMaxCallBatch + 1];   // prefix sum of chunks per batch row
+    int32_t stable_len[kMaxCallBatch];       // leading rows written before this chain of kernels began (the true states)
 };
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
@@ -92,11 +93,17 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_tma_kernel(const __gr
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, c = lane & 3;
 
+    pdl_launch_dependents();
+    // A chunk that lies entirely inside the true states cannot be touched by the kernels this one
+    // may overlap with (they only append draft states), so its tiles are requested right away;
+    // the last chunks wait for the previous kernels first.
+    const bool stable = start + kChunk <= work.stable_len[b];
     if (threadIdx.x == 0) {
         mbar_init(barK, 1);
         mbar_init(barV, 1);
         s_abort = 0;
         fence_barrier_init();
+        if (!stable) pdl_wait();
         const uint64_t once = policy_evict_first();
         mbar_expect_tx(barK, kTileBytes);
 #pragma unroll
@@ -106,6 +113,7 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_tma_kernel(const __gr
         for (int h = 0; h < kHalves; ++h) tma_load_2d_hint(sV + h * (kChunk * 128), &tmV, barV, h * 64, row0, once);
     }
 
+    pdl_wait();                                                          // Q comes from the previous kernel
     // Q fragments: rows of the A operand are the G query heads of this K/V head (rows >= G are zero)
     uint32_t qa[DH / 16][2];
     {
@@ -242,8 +250,8 @@ int launch_attn(const CUtensorMap& mk, const CUtensorMap& mv, const bf16* q, con
         if (cudaFuncSetAttribute(attn_decode_tma_kernel<DH, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess) return -1;
         attr_done = true;
     }
-    attn_decode_tma_kernel<DH, G><<<dim3(items, Hkv), kWarps * 32, kSmem, stream>>>(mk, mv, q, work, nbatch, Hq, Hkv, cap, nch_stride,
-                                                                                    scale_log2, po, pml, error_word);
+    launch_pdl(attn_decode_tma_kernel<DH, G>, dim3(items, Hkv), dim3(kWarps * 32), (size_t)kSmem, stream, mk, mv, q, work, nbatch, Hq, Hkv,
+               cap, nch_stride, scale_log2, po, pml, error_word);
     return 1;
 }
 
@@ -275,8 +283,8 @@ bool tc_attn_bind_cache(TcPlan* p, const void* kcache, const void* vcache, long 
     return true;
 }
 
-int tc_attn_decode(TcPlan* p, const void* q, const BatchMeta& meta, int B, int Hq, int Hkv, int dh, int cap, int max_kv_len,
-                   void* scratch, void* o, int* error_word, cudaStream_t stream) {
+int tc_attn_decode(TcPlan* p, const void* q, const BatchMeta& meta, const int32_t* stable_len, int B, int Hq, int Hkv, int dh, int cap,
+                   int max_kv_len, void* scratch, void* o, int* error_word, cudaStream_t stream) {
     if (p == nullptr || !p->cache_maps_ok || B <= 0 || B > kMaxCallBatch || Hkv > 65535) return -1;
     if (dh != 64 && dh != 128) return -1;
     const int G = Hq / Hkv;
@@ -286,6 +294,7 @@ int tc_attn_decode(TcPlan* p, const void* q, const BatchMeta& meta, int B, int H
     for (int b = 0; b < B; ++b) {
         work.slot[b] = meta.slot[b];
         work.kv_len[b] = meta.kv_len[b];
+        work.stable_len[b] = stable_len != nullptr ? stable_len[b] : 0;
         work.item_start[b] = items;
         items += (meta.kv_len[b] + kChunk - 1) / kChunk;
     }

@@ -88,4 +88,36 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long k)
 
 __device__ __forceinline__ float silu_f(float u) { return u / (1.0f + __expf(-u)); }
 
+// Programmatic dependent launch.  The serve-time kernels are launched so that a kernel may start
+// while its predecessor in the stream is still draining: everything before pdl_wait() must touch
+// only memory that no kernel of the chain writes (weights, the stable part of the K/V cache) and
+// must write no global memory; pdl_wait() returns once the predecessor has completed and its
+// writes are visible.  Every kernel launched this way calls pdl_wait() on every thread, so that a
+// kernel's completion implies the completion of all kernels before it.  Both are no-ops for a
+// plain launch.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
+// Launch with the programmatic-stream-serialization attribute (falls back to a plain launch if the
+// attribute is refused).
+template <typename... KArgs, typename... Args>
+inline void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...) != cudaSuccess) {
+        cudaGetLastError();
+        cfg.numAttrs = 0;
+        cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+    }
+}
+
 }  // namespace beagle

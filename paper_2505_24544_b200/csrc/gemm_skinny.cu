@@ -67,6 +67,7 @@ __global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_cons
     const int kb0 = blockIdx.z * args.kb_per_split;
     const int nkb = max(0, min(args.kb_per_split, kb_total - kb0));
 
+    pdl_launch_dependents();
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
         mbar_init(bar_acc, 1);
@@ -84,8 +85,18 @@ __global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_cons
         if (lane == 0) {
             const CUtensorMap* mapW = mat ? &tmW2 : &tmW;
             const uint64_t stream_once = policy_evict_first(), keep = policy_evict_last();
-            int issued = 0;
-            for (int kb = 0; kb < nkb; ++kb) {
+            // The weights do not depend on the previous kernel: fill the ring with weight tiles
+            // while that kernel drains, then wait for it and add the activation tiles.
+            const int npre = min(nkb, kStages);
+            for (int kb = 0; kb < npre; ++kb) {
+                mbar_expect_tx(bar_full + 8 * kb, SM::kStageBytes);
+                tma_load_2d_hint(smem_base + kb * SM::kStageBytes, mapW, bar_full + 8 * kb, (kb0 + kb) * BK, ta * BM, stream_once);
+            }
+            pdl_wait();
+            for (int kb = 0; kb < npre; ++kb)
+                tma_load_2d_hint(smem_base + kb * SM::kStageBytes + kABytes, &tmX, bar_full + 8 * kb, (kb0 + kb) * BK, 0, keep);
+            int issued = npre;
+            for (int kb = npre; kb < nkb; ++kb) {
                 const int s = kb % kStages;
                 const uint32_t ph = (kb / kStages) & 1;
                 if (!mbar_wait(bar_empty + 8 * s, ph ^ 1, s_abort)) break;
@@ -130,6 +141,7 @@ __global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_cons
         // ---------------- epilogue: warp w reads TMEM lanes [32*(w%4), +32)
         const int q = warp & 3;
         const int feat = ta * BM + q * 32 + lane;    // output feature owned by this thread
+        pdl_wait();                                  // the buffers written below may still be read by the previous kernel
         bool ok = nkb > 0;
         if (ok) ok = mbar_wait(bar_acc, 0, s_abort);
         ok = __all_sync(0xffffffffu, ok);            // the TMEM loads below are warp-collective
@@ -177,6 +189,7 @@ __global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_cons
 
     fence_before();
     __syncthreads();
+    pdl_wait();                                      // every thread, so that this grid's completion implies its predecessors'
     if (threadIdx.x == 0 && *s_abort && args.error_word != nullptr) atomicExch(args.error_word, 1);
     if (warp == 1) {
         fence_after();
@@ -202,6 +215,8 @@ constexpr int kFinCols = kFinThreads * 4;   // features per CTA and pass
 template <int MODE>
 __global__ void __launch_bounds__(kFinThreads) tc_finish_kernel(const FinishArgs a) {
     const int b = blockIdx.x;
+    pdl_launch_dependents();
+    pdl_wait();
     const size_t mstride = (size_t)a.B * a.N;
     const size_t zstride = mstride * a.nmat;
     const float* p0 = a.partial + (size_t)b * a.N;
@@ -212,12 +227,19 @@ __global__ void __launch_bounds__(kFinThreads) tc_finish_kernel(const FinishArgs
     float ss = 0.f;
     for (int n = n_begin + threadIdx.x * 4; n < n_end; n += kFinThreads * 4) {     // N is a multiple of 4
         float4 s0 = make_float4(0.f, 0.f, 0.f, 0.f), s1 = s0;
-        for (int z = 0; z < a.splits; ++z) {
-            const float4 t = *reinterpret_cast<const float4*>(p0 + z * zstride + n);
-            s0.x += t.x; s0.y += t.y; s0.z += t.z; s0.w += t.w;
-            if (MODE == SK_SILU_MUL || MODE == SK_KV) {
-                const float4 u = *reinterpret_cast<const float4*>(p1 + z * zstride + n);
-                s1.x += u.x; s1.y += u.y; s1.z += u.z; s1.w += u.w;
+        constexpr bool kTwo = (MODE == SK_SILU_MUL || MODE == SK_KV);
+        for (int z0 = 0; z0 < a.splits; z0 += 8) {                 // all loads of a group first, then the adds in split order
+            float4 t[8], u[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const bool in = z0 + j < a.splits;
+                t[j] = in ? *reinterpret_cast<const float4*>(p0 + (size_t)(z0 + j) * zstride + n) : make_float4(0.f, 0.f, 0.f, 0.f);
+                if (kTwo) u[j] = in ? *reinterpret_cast<const float4*>(p1 + (size_t)(z0 + j) * zstride + n) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                s0.x += t[j].x; s0.y += t[j].y; s0.z += t[j].z; s0.w += t[j].w;
+                if (kTwo) { s1.x += u[j].x; s1.y += u[j].y; s1.z += u[j].z; s1.w += u[j].w; }
             }
         }
         float v[4] = {s0.x, s0.y, s0.z, s0.w};
@@ -298,7 +320,7 @@ int launch_sk(const CUtensorMap& w, const CUtensorMap& w2, const CUtensorMap& x,
         if (cudaFuncSetAttribute(tc_skinny_kernel<BN, LOGITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kBytes) != cudaSuccess) return -1;
         attr_done = true;
     }
-    tc_skinny_kernel<BN, LOGITS><<<grid, kSkThreads, SM::kBytes, stream>>>(w, w2, x, args);
+    launch_pdl(tc_skinny_kernel<BN, LOGITS>, grid, dim3(kSkThreads), SM::kBytes, stream, w, w2, x, args);
     return 1;
 }
 
@@ -354,10 +376,10 @@ int tc_skinny(TcPlan* p, int mode, const SkinnyArgs& g, cudaStream_t stream) {
     const bool whole_row = (mode == SK_RESID && g.norm_out != nullptr);
     dim3 fgrid(g.B, whole_row ? 1 : (g.N + kFinCols - 1) / kFinCols);
     switch (mode) {
-        case SK_STORE: tc_finish_kernel<SK_STORE><<<fgrid, kFinThreads, 0, stream>>>(f); break;
-        case SK_RESID: tc_finish_kernel<SK_RESID><<<fgrid, kFinThreads, 0, stream>>>(f); break;
-        case SK_SILU_MUL: tc_finish_kernel<SK_SILU_MUL><<<fgrid, kFinThreads, 0, stream>>>(f); break;
-        case SK_KV: tc_finish_kernel<SK_KV><<<fgrid, kFinThreads, 0, stream>>>(f); break;
+        case SK_STORE: launch_pdl(tc_finish_kernel<SK_STORE>, fgrid, dim3(kFinThreads), 0, stream, f); break;
+        case SK_RESID: launch_pdl(tc_finish_kernel<SK_RESID>, fgrid, dim3(kFinThreads), 0, stream, f); break;
+        case SK_SILU_MUL: launch_pdl(tc_finish_kernel<SK_SILU_MUL>, fgrid, dim3(kFinThreads), 0, stream, f); break;
+        case SK_KV: launch_pdl(tc_finish_kernel<SK_KV>, fgrid, dim3(kFinThreads), 0, stream, f); break;
         default: return -1;
     }
     return 2;

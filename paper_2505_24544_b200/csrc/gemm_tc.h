@@ -52,8 +52,9 @@ int tc_skinny_key_tiles(int N);
 // Binds the cache halves ([rows, head_dim] each); false when the shape is not covered.
 bool tc_attn_bind_cache(TcPlan* plan, const void* kcache, const void* vcache, long long rows, int dh);
 // Split-KV partials + combine, as launch_attn_decode; -1 when not covered (caller falls back).
-int tc_attn_decode(TcPlan* plan, const void* q, const BatchMeta& meta, int B, int Hq, int Hkv, int dh, int cap, int max_kv_len,
-                   void* scratch, void* o, int* error_word, cudaStream_t stream);
+// stable_len[b] (host, nullable): leading cache rows of row b's slot that no kernel still in flight writes.
+int tc_attn_decode(TcPlan* plan, const void* q, const BatchMeta& meta, const int32_t* stable_len, int B, int Hq, int Hkv, int dh,
+                   int cap, int max_kv_len, void* scratch, void* o, int* error_word, cudaStream_t stream);
 int tc_attn_chunk(void);
 
 // ---- block-masked cross-attention of the multi-token forward (bf16, head_dim 64 or 128) -------

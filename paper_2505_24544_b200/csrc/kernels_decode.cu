@@ -17,10 +17,19 @@ __global__ void __launch_bounds__(256) embed_norm_kernel(const int32_t* __restri
                                                          int d, float eps, int do_norm, T* __restrict__ x_out,
                                                          T* __restrict__ xn_out, const T* __restrict__ gather_src,
                                                          T* __restrict__ gather_dst) {
+    constexpr int VEC = VecOf<T>::N;
+    constexpr int kMaxVec = 4;                  // 16-byte pieces a thread keeps in registers (d <= 256 * 4 * VEC)
     const int r = blockIdx.x;
+    const int nvec = d / VEC;                   // d is a multiple of 8
+    // First kernel of a draft step: it waits BEFORE it lets its dependents start, so every kernel
+    // of this step begins after all earlier work in the stream (cache prefill, the previous step)
+    // has completed.  The later kernels' early reads of weights and true-state cache rows rely on it.
+    pdl_wait();
+    pdl_launch_dependents();
     if (gather_src != nullptr) {
-        const T* g = gather_src + (size_t)meta.slot[r] * d;
-        for (int i = threadIdx.x; i < d; i += blockDim.x) gather_dst[(size_t)r * d + i] = g[i];
+        const uint4* g = reinterpret_cast<const uint4*>(gather_src + (size_t)meta.slot[r] * d);
+        uint4* dst = reinterpret_cast<uint4*>(gather_dst + (size_t)r * d);
+        for (int i = threadIdx.x; i < nvec; i += blockDim.x) dst[i] = g[i];
     }
     const T* row;
     if (src != nullptr) {
@@ -30,10 +39,28 @@ __global__ void __launch_bounds__(256) embed_norm_kernel(const int32_t* __restri
         tok = min(max(tok, 0), vocab - 1);      // ids are validated by contract; never read out of range
         row = embed + (size_t)tok * d;
     }
+    const uint4* row4 = reinterpret_cast<const uint4*>(row);
+    const bool in_regs = nvec <= kMaxVec * (int)blockDim.x && (d % VEC) == 0;
+    uint4 keep[kMaxVec];
     float ss = 0.f;
-    for (int i = threadIdx.x; i < d; i += blockDim.x) {
-        float v = to_float<T>(row[i]);
-        ss += v * v;
+    if (in_regs) {
+#pragma unroll
+        for (int j = 0; j < kMaxVec; ++j) {
+            const int i = threadIdx.x + j * blockDim.x;
+            keep[j] = i < nvec ? row4[i] : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int j = 0; j < kMaxVec; ++j) {
+            float f[VEC];
+            unpack16<T>(keep[j], f);
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) ss = fmaf(f[v], f[v], ss);
+        }
+    } else {
+        for (int i = threadIdx.x; i < d; i += blockDim.x) {
+            float v = to_float<T>(row[i]);
+            ss += v * v;
+        }
     }
     __shared__ float s_part[8];
     __shared__ float s_scale;
@@ -47,11 +74,27 @@ __global__ void __launch_bounds__(256) embed_norm_kernel(const int32_t* __restri
     }
     __syncthreads();
     const float sc = s_scale;
-    for (int i = threadIdx.x; i < d; i += blockDim.x) {
-        float v = to_float<T>(row[i]);
-        if (x_out != nullptr) x_out[(size_t)r * d + i] = from_float<T>(v);
-        float g = do_norm ? to_float<T>(gain[i]) : 1.0f;
-        xn_out[(size_t)r * d + i] = from_float<T>(v * sc * g);
+    if (in_regs) {
+#pragma unroll
+        for (int j = 0; j < kMaxVec; ++j) {
+            const int i = threadIdx.x + j * blockDim.x;
+            if (i >= nvec) break;
+            if (x_out != nullptr) reinterpret_cast<uint4*>(x_out + (size_t)r * d)[i] = keep[j];
+            float f[VEC], g[VEC];
+            unpack16<T>(keep[j], f);
+            if (do_norm) unpack16<T>(__ldg(reinterpret_cast<const uint4*>(gain) + i), g);
+            T o[VEC];
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) o[v] = from_float<T>(f[v] * sc * (do_norm ? g[v] : 1.0f));
+            reinterpret_cast<uint4*>(xn_out + (size_t)r * d)[i] = *reinterpret_cast<const uint4*>(o);
+        }
+    } else {
+        for (int i = threadIdx.x; i < d; i += blockDim.x) {
+            float v = to_float<T>(row[i]);
+            if (x_out != nullptr) x_out[(size_t)r * d + i] = from_float<T>(v);
+            float g = do_norm ? to_float<T>(gain[i]) : 1.0f;
+            xn_out[(size_t)r * d + i] = from_float<T>(v * sc * g);
+        }
     }
 }
 
@@ -62,13 +105,13 @@ int launch_embed_norm(int dtype, const int32_t* tokens, const int32_t* last_toke
     BatchMeta m;
     if (meta != nullptr) m = *meta; else memset(&m, 0, sizeof(m));
     if (dtype == 0)
-        embed_norm_kernel<float><<<rows, 256, 0, stream>>>(tokens, last_token, m, (const float*)embed, vocab,
-                                                           (const float*)src, (const float*)gain, d, eps, do_norm,
-                                                           (float*)x_out, (float*)xn_out, (const float*)gather_src, (float*)gather_dst);
+        launch_pdl(embed_norm_kernel<float>, dim3(rows), dim3(256), 0, stream, tokens, last_token, m, (const float*)embed, vocab,
+                   (const float*)src, (const float*)gain, d, eps, do_norm, (float*)x_out, (float*)xn_out,
+                   (const float*)gather_src, (float*)gather_dst);
     else
-        embed_norm_kernel<bf16><<<rows, 256, 0, stream>>>(tokens, last_token, m, (const bf16*)embed, vocab,
-                                                          (const bf16*)src, (const bf16*)gain, d, eps, do_norm,
-                                                          (bf16*)x_out, (bf16*)xn_out, (const bf16*)gather_src, (bf16*)gather_dst);
+        launch_pdl(embed_norm_kernel<bf16>, dim3(rows), dim3(256), 0, stream, tokens, last_token, m, (const bf16*)embed, vocab,
+                   (const bf16*)src, (const bf16*)gain, d, eps, do_norm, (bf16*)x_out, (bf16*)xn_out,
+                   (const bf16*)gather_src, (bf16*)gather_dst);
     return 1;
 }
 
@@ -104,6 +147,15 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvArgs a) {
     }
     const T* X = reinterpret_cast<const T*>(a.X);
     __shared__ unsigned long long s_keys[8][NB];
+
+    // The weights do not depend on the previous kernel: pull the head of this warp's rows towards
+    // L2 while that kernel drains, then wait for the activations.
+    pdl_launch_dependents();
+    if (lane < 16) {                            // the first 2 KB of each row (bf16; 4 KB in fp32, every other line)
+        const int k = lane * 64;
+        if (k < a.K) { prefetch_l2(w0 + k); prefetch_l2(w1 + k); }
+    }
+    pdl_wait();
 
     for (int b0 = 0; b0 < a.B; b0 += NB) {
         const T* xp[NB];
@@ -194,10 +246,10 @@ int gemv_grid_blocks(int mode, int N) {
 
 template <typename T, int MODE>
 static void gemv_dispatch_nb(const GemvArgs& a, dim3 grid, cudaStream_t stream) {
-    if (a.B <= 1) gemv_kernel<T, 1, MODE><<<grid, 256, 0, stream>>>(a);
-    else if (a.B <= 2) gemv_kernel<T, 2, MODE><<<grid, 256, 0, stream>>>(a);
-    else if (a.B <= 4) gemv_kernel<T, 4, MODE><<<grid, 256, 0, stream>>>(a);
-    else gemv_kernel<T, 8, MODE><<<grid, 256, 0, stream>>>(a);
+    if (a.B <= 1) launch_pdl(gemv_kernel<T, 1, MODE>, grid, dim3(256), 0, stream, a);
+    else if (a.B <= 2) launch_pdl(gemv_kernel<T, 2, MODE>, grid, dim3(256), 0, stream, a);
+    else if (a.B <= 4) launch_pdl(gemv_kernel<T, 4, MODE>, grid, dim3(256), 0, stream, a);
+    else launch_pdl(gemv_kernel<T, 8, MODE>, grid, dim3(256), 0, stream, a);
 }
 template <typename T>
 static void gemv_dispatch_mode(int mode, const GemvArgs& a, dim3 grid, cudaStream_t stream) {
@@ -237,6 +289,8 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attn_decode_kernel(
     const int chunk = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
     const int kv_len = meta.kv_len[b];
     const int start = chunk * kAttnChunk;
+    pdl_launch_dependents();
+    pdl_wait();
     if (start >= kv_len) return;
     const int cnt = min(kAttnChunk, kv_len - start);
     const int slot = meta.slot[b];
@@ -344,30 +398,87 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attn_decode_kernel(
     }
 }
 
-template <typename T>
-__global__ void attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
-                                    const BatchMeta meta, int Hq, int dh, int nchunk_max, int chunk, T* __restrict__ o) {
-    const int h = blockIdx.x, b = blockIdx.y, c = threadIdx.x;
+// One warp per (sequence, query head): the lanes first share the chunks' running maxima and
+// exp-sums (each lane a strided subset), then each lane owns dh/32 consecutive output dims and adds
+// the chunks' unnormalised partials with the weights exp(m_i - M), handed around by shuffles.
+template <typename T, int DPL>
+__global__ void __launch_bounds__(256) attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
+                                                          const BatchMeta meta, int nheads_total, int Hq, int dh, int nchunk_max,
+                                                          int chunk, T* __restrict__ o) {
+    const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    pdl_launch_dependents();
+    pdl_wait();
+    if (wid >= nheads_total) return;
+    const int b = wid / Hq;
     const int kv_len = meta.kv_len[b];
     const int nch = (kv_len + chunk - 1) / chunk;
-    const size_t p0 = ((size_t)b * Hq + h) * nchunk_max;
+    const size_t p0 = (size_t)wid * nchunk_max;
+    const int DH = dh;                          // DPL * 32, or 16 with DPL = 1 (upper half-warp idle)
+    const bool act = lane * DPL < DH;
     float M = -INFINITY;
-    for (int i = 0; i < nch; ++i) M = fmaxf(M, part_ml[2 * (p0 + i)]);
-    float num = 0.f, den = 0.f;
-    for (int i = 0; i < nch; ++i) {
-        const float w = __expf(part_ml[2 * (p0 + i)] - M);
-        den = fmaf(w, part_ml[2 * (p0 + i) + 1], den);
-        num = fmaf(w, part_o[(p0 + i) * dh + c], num);
+    for (int i = lane; i < nch; i += 32) M = fmaxf(M, part_ml[2 * (p0 + i)]);
+    M = warp_max(M);
+    float acc[DPL];
+#pragma unroll
+    for (int v = 0; v < DPL; ++v) acc[v] = 0.f;
+    float den = 0.f;
+    for (int i0 = 0; i0 < nch; i0 += 32) {
+        const int i = i0 + lane;
+        float w = 0.f, l = 0.f;
+        if (i < nch) {
+            const float2 ml = *reinterpret_cast<const float2*>(part_ml + 2 * (p0 + i));
+            w = (ml.x == -INFINITY) ? 0.f : __expf(ml.x - M);
+            l = ml.y;
+        }
+        den = fmaf(w, l, den);
+        const int n_here = min(32, nch - i0);
+#pragma unroll 4
+        for (int j = 0; j < n_here; ++j) {
+            const float wj = __shfl_sync(0xffffffffu, w, j);
+            const float* src = part_o + (p0 + i0 + j) * DH + lane * DPL;
+            if (!act) continue;
+            if constexpr (DPL % 4 == 0) {
+#pragma unroll
+                for (int v = 0; v < DPL; v += 4) {
+                    const float4 t = *reinterpret_cast<const float4*>(src + v);
+                    acc[v] = fmaf(wj, t.x, acc[v]); acc[v + 1] = fmaf(wj, t.y, acc[v + 1]);
+                    acc[v + 2] = fmaf(wj, t.z, acc[v + 2]); acc[v + 3] = fmaf(wj, t.w, acc[v + 3]);
+                }
+            } else {
+#pragma unroll
+                for (int v = 0; v < DPL; ++v) acc[v] = fmaf(wj, src[v], acc[v]);
+            }
+        }
     }
-    o[((size_t)b * Hq + h) * dh + c] = from_float<T>(nch > 0 ? num / den : 0.f);
+    den = warp_sum(den);
+    const float inv = (nch > 0 && den > 0.f) ? 1.0f / den : 0.f;
+    T* dst = o + (size_t)wid * DH + lane * DPL;
+    if (act) {
+#pragma unroll
+        for (int v = 0; v < DPL; ++v) dst[v] = from_float<T>(acc[v] * inv);
+    }
+}
+
+template <typename T>
+static int attn_combine_dispatch(const float* part_o, const float* part_ml, const BatchMeta& meta, int B, int Hq, int dh,
+                                 int nchunk_stride, int chunk, T* o, cudaStream_t stream) {
+    const int total = B * Hq;
+    const int grid = (total * 32 + 255) / 256;
+    switch (dh) {
+        case 32: launch_pdl(attn_combine_kernel<T, 1>, dim3(grid), dim3(256), 0, stream, part_o, part_ml, meta, total, Hq, dh, nchunk_stride, chunk, o); return 1;
+        case 64: launch_pdl(attn_combine_kernel<T, 2>, dim3(grid), dim3(256), 0, stream, part_o, part_ml, meta, total, Hq, dh, nchunk_stride, chunk, o); return 1;
+        case 128: launch_pdl(attn_combine_kernel<T, 4>, dim3(grid), dim3(256), 0, stream, part_o, part_ml, meta, total, Hq, dh, nchunk_stride, chunk, o); return 1;
+        case 256: launch_pdl(attn_combine_kernel<T, 8>, dim3(grid), dim3(256), 0, stream, part_o, part_ml, meta, total, Hq, dh, nchunk_stride, chunk, o); return 1;
+        case 16: launch_pdl(attn_combine_kernel<T, 1>, dim3(grid), dim3(256), 0, stream, part_o, part_ml, meta, total, Hq, dh, nchunk_stride, chunk, o); return 1;
+        default: return -1;
+    }
 }
 
 int launch_attn_combine(int dtype, const float* part_o, const float* part_ml, const BatchMeta& meta, int B, int Hq, int dh,
                         int nchunk_stride, int chunk, void* o, cudaStream_t stream) {
     if (B <= 0) return 0;
-    if (dtype == 0) attn_combine_kernel<float><<<dim3(Hq, B), dh, 0, stream>>>(part_o, part_ml, meta, Hq, dh, nchunk_stride, chunk, (float*)o);
-    else attn_combine_kernel<bf16><<<dim3(Hq, B), dh, 0, stream>>>(part_o, part_ml, meta, Hq, dh, nchunk_stride, chunk, (bf16*)o);
-    return 1;
+    return dtype == 0 ? attn_combine_dispatch<float>(part_o, part_ml, meta, B, Hq, dh, nchunk_stride, chunk, (float*)o, stream)
+                      : attn_combine_dispatch<bf16>(part_o, part_ml, meta, B, Hq, dh, nchunk_stride, chunk, (bf16*)o, stream);
 }
 
 size_t attn_decode_scratch_bytes(int max_batch, int Hq, int dh, int max_kv) {
@@ -380,12 +491,12 @@ template <typename T, int G>
 static int attn_dispatch_lpk(int lpk, dim3 grid, cudaStream_t stream, const T* q, const T* kc, const T* vc,
                              const BatchMeta& meta, int Hq, int Hkv, int cap, int nch, float scale, float* po, float* pml) {
     switch (lpk) {
-        case 4: attn_decode_kernel<T, G, 4><<<grid, kAttnWarps * 32, 0, stream>>>(q, kc, vc, meta, Hq, Hkv, cap, nch, scale, po, pml); return 1;
-        case 8: attn_decode_kernel<T, G, 8><<<grid, kAttnWarps * 32, 0, stream>>>(q, kc, vc, meta, Hq, Hkv, cap, nch, scale, po, pml); return 1;
-        case 16: attn_decode_kernel<T, G, 16><<<grid, kAttnWarps * 32, 0, stream>>>(q, kc, vc, meta, Hq, Hkv, cap, nch, scale, po, pml); return 1;
+        case 4: launch_pdl(attn_decode_kernel<T, G, 4>, grid, dim3(kAttnWarps * 32), 0, stream, q, kc, vc, meta, Hq, Hkv, cap, nch, scale, po, pml); return 1;
+        case 8: launch_pdl(attn_decode_kernel<T, G, 8>, grid, dim3(kAttnWarps * 32), 0, stream, q, kc, vc, meta, Hq, Hkv, cap, nch, scale, po, pml); return 1;
+        case 16: launch_pdl(attn_decode_kernel<T, G, 16>, grid, dim3(kAttnWarps * 32), 0, stream, q, kc, vc, meta, Hq, Hkv, cap, nch, scale, po, pml); return 1;
         case 32:
             if constexpr (G * 32 * VecOf<T>::N <= 1024) {   // static shared memory stays under 48 KB
-                attn_decode_kernel<T, G, 32><<<grid, kAttnWarps * 32, 0, stream>>>(q, kc, vc, meta, Hq, Hkv, cap, nch, scale, po, pml);
+                launch_pdl(attn_decode_kernel<T, G, 32>, grid, dim3(kAttnWarps * 32), 0, stream, q, kc, vc, meta, Hq, Hkv, cap, nch, scale, po, pml);
                 return 1;
             } else {
                 return -1;
@@ -418,7 +529,7 @@ static int attn_dispatch(const void* q, const void* kc, const void* vc, const Ba
         if (rc < 0) return rc;
         launched += rc;
     }
-    attn_combine_kernel<T><<<dim3(Hq, B), dh, 0, stream>>>(po, pml, meta, Hq, dh, nch, kAttnChunk, (T*)o);
+    if (attn_combine_dispatch<T>(po, pml, meta, B, Hq, dh, nch, kAttnChunk, (T*)o, stream) < 0) return -1;
     return launched + 1;
 }
 int launch_attn_decode(int dtype, const void* q, const void* kcache, const void* vcache, const BatchMeta& meta,
@@ -436,6 +547,8 @@ __global__ void __launch_bounds__(256) argmax_finalize_kernel(const unsigned lon
                                                               const BatchMeta meta, int32_t* __restrict__ tokens_out,
                                                               int tokens_out_stride, int32_t* __restrict__ last_token) {
     const int b = blockIdx.x;
+    pdl_launch_dependents();
+    pdl_wait();
     unsigned long long key = 0ull;
     for (int i = threadIdx.x; i < nblk; i += blockDim.x) {
         const unsigned long long o = partials[(size_t)b * nblk + i];
@@ -455,7 +568,7 @@ __global__ void __launch_bounds__(256) argmax_finalize_kernel(const unsigned lon
 int launch_argmax_finalize(const unsigned long long* partials, int nblk, const BatchMeta& meta, int B,
                            int32_t* tokens_out, int tokens_out_stride, int32_t* last_token, cudaStream_t stream) {
     if (B <= 0) return 0;
-    argmax_finalize_kernel<<<B, 256, 0, stream>>>(partials, nblk, meta, tokens_out, tokens_out_stride, last_token);
+    launch_pdl(argmax_finalize_kernel, dim3(B), dim3(256), 0, stream, partials, nblk, meta, tokens_out, tokens_out_stride, last_token);
     return 1;
 }
 
