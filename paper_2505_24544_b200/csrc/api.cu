@@ -155,7 +155,7 @@ ServeLayout serve_layout(const beagle_config& c) {
     L.lm_blocks = gemv_grid_blocks(GEMV_LOGITS, c.vocab);
     L.lm_partials = take(B * (size_t)L.lm_blocks * sizeof(unsigned long long));
     L.verify_keys = take(B * 65 * kRowArgmaxSplit * sizeof(unsigned long long));
-    L.dev_error = take(256);
+    L.dev_error = take(256 + B * (size_t)c.n_kv_heads * sizeof(int32_t));     // error word, then the attention completion counters
     L.total = off;
     return L;
 }
@@ -195,7 +195,7 @@ beagle_status cuda_ok(beagle_ctx* ctx, const char* what) {
 // shape (bf16), the CUDA-core kernel otherwise.
 void clear_error_word_once(beagle_ctx* ctx, cudaStream_t stream) {
     if (!ctx->dev_error_cleared) {
-        cudaMemsetAsync(ctx->dev_error, 0, sizeof(int), stream);
+        cudaMemsetAsync(ctx->dev_error, 0, 256 + (size_t)BEAGLE_MAX_CALL_BATCH * ctx->cfg.n_kv_heads * sizeof(int32_t), stream);
         ctx->dev_error_cleared = true;
     }
 }
@@ -628,7 +628,7 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
             int32_t stable[kMaxCallBatch];
             for (int b = 0; b < batch; ++b) stable[b] = ctx->n_true[seq_slot[b]];
             rc = tc_attn_decode(ctx->tc, ctx->q, meta, stable, batch, c.n_q_heads, c.n_kv_heads, c.head_dim, ctx->cap, max_kv,
-                                ctx->attn_scratch, ctx->o, ctx->dev_error, stream);
+                                ctx->attn_scratch, ctx->dev_error + 64, ctx->o, ctx->dev_error, stream);
         }
         if (rc < 0)
             rc = launch_attn_decode(dt, ctx->q, ctx->kcache, ctx->vcache, meta, batch, c.n_q_heads, c.n_kv_heads,

@@ -10,7 +10,9 @@
 // to the unpacking at HBM speed, while the tensor pipe does it in passing.  Each of the four warps
 // owns 32 keys: S = Q K^T (ldmatrix + m16n8k16), a warp-local softmax in registers, O = P V
 // (ldmatrix.trans), then the four partial (m, l, O) triples are merged in shared memory and the
-// chunk's unnormalised partial goes to the split-KV scratch that attn_combine reduces.
+// chunk's unnormalised partial goes to the split-KV scratch.  The CTA that finishes last for its
+// (sequence, K/V head) -- a counter in global memory, reset by that CTA -- merges the chunks of
+// its G heads and writes o, so no second kernel is needed.
 //
 // Rows past the sequence's length inside the last chunk hold whatever the cache held before:
 // their scores are replaced by -inf and their V rows are zeroed in shared memory, so they
@@ -18,6 +20,7 @@
 // device error word and the CTA writes an empty partial instead of hanging.
 #include <cstring>
 
+#include "attn_combine.cuh"
 #include "gemm_tc.h"
 #include "tc_plan.h"
 #include "tc_ptx.cuh"
@@ -67,8 +70,8 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_tma_kernel(const __gr
                                                                      const __grid_constant__ CUtensorMap tmV,
                                                                      const bf16* __restrict__ q, const AttnWork work, int nbatch,
                                                                      int Hq, int Hkv, int cap, int nch_stride, float scale_log2,
-                                                                     float* __restrict__ part_o, float* __restrict__ part_ml,
-                                                                     int* error_word) {
+                                                                     float* part_o, float* part_ml, int* done_count,
+                                                                     bf16* __restrict__ o_out, int* error_word) {
     constexpr int kTileBytes = kChunk * DH * 2;         // one of K / V
     constexpr int kHalves = DH / 64;
     extern __shared__ uint8_t smem_raw[];
@@ -78,7 +81,7 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_tma_kernel(const __gr
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + 2 * kTileBytes);
     const uint32_t barK = smem_u32(bars), barV = barK + 8;
     __shared__ float s_m[kWarps][8], s_l[kWarps][8];
-    __shared__ int s_abort;
+    __shared__ int s_abort, s_last;
 
     // which (sequence, chunk) this CTA owns
     int b = 0;
@@ -233,6 +236,27 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_tma_kernel(const __gr
             part_ml[2 * pi + 1] = good ? L : 0.f;
         }
     }
+    // ---- the last CTA of this (sequence, K/V head) merges all chunks of its G heads
+    // (done_count == NULL: a separate kernel merges, which is faster for large batches)
+    const int nchunks = (kv_len + kChunk - 1) / kChunk;
+    if (done_count != nullptr) {
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const int prev = atomicAdd(&done_count[b * Hkv + kvh], 1);
+            s_last = (prev == nchunks - 1);
+            if (s_last) done_count[b * Hkv + kvh] = 0;                  // ready for the next launch
+        }
+        __syncthreads();
+    }
+    if (done_count != nullptr && s_last) {
+        __threadfence();
+        for (int hg = warp; hg < G; hg += kWarps) {
+            const size_t head = (size_t)b * Hq + kvh * G + hg;
+            attn_combine_warp<bf16, DH / 32, true>(part_o + head * nch_stride * DH, part_ml + 2 * head * nch_stride, nchunks, DH, lane,
+                                             o_out + head * DH);
+        }
+    }
     if (threadIdx.x == 0 && s_abort) {
         if (error_word != nullptr) atomicExch(error_word, 1);
         // the copies may still be in flight: give them a second bounded chance to land before the CTA ends
@@ -243,7 +267,8 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_tma_kernel(const __gr
 
 template <int DH, int G>
 int launch_attn(const CUtensorMap& mk, const CUtensorMap& mv, const bf16* q, const AttnWork& work, int nbatch, int items, int Hq,
-                int Hkv, int cap, int nch_stride, float scale_log2, float* po, float* pml, int* error_word, cudaStream_t stream) {
+                int Hkv, int cap, int nch_stride, float scale_log2, float* po, float* pml, int* done_count, bf16* o, int* error_word,
+                cudaStream_t stream) {
     constexpr int kSmem = 2 * kChunk * DH * 2 + 1024 + 64;
     static bool attr_done = false;
     if (!attr_done) {
@@ -251,19 +276,19 @@ int launch_attn(const CUtensorMap& mk, const CUtensorMap& mv, const bf16* q, con
         attr_done = true;
     }
     launch_pdl(attn_decode_tma_kernel<DH, G>, dim3(items, Hkv), dim3(kWarps * 32), (size_t)kSmem, stream, mk, mv, q, work, nbatch, Hq, Hkv,
-               cap, nch_stride, scale_log2, po, pml, error_word);
+               cap, nch_stride, scale_log2, po, pml, done_count, o, error_word);
     return 1;
 }
 
 template <int DH>
 int launch_attn_g(int G, const CUtensorMap& mk, const CUtensorMap& mv, const bf16* q, const AttnWork& work, int nbatch, int items,
-                  int Hq, int Hkv, int cap, int nch_stride, float scale_log2, float* po, float* pml, int* error_word,
-                  cudaStream_t stream) {
+                  int Hq, int Hkv, int cap, int nch_stride, float scale_log2, float* po, float* pml, int* done_count, bf16* o,
+                  int* error_word, cudaStream_t stream) {
     switch (G) {
-        case 1: return launch_attn<DH, 1>(mk, mv, q, work, nbatch, items, Hq, Hkv, cap, nch_stride, scale_log2, po, pml, error_word, stream);
-        case 2: return launch_attn<DH, 2>(mk, mv, q, work, nbatch, items, Hq, Hkv, cap, nch_stride, scale_log2, po, pml, error_word, stream);
-        case 4: return launch_attn<DH, 4>(mk, mv, q, work, nbatch, items, Hq, Hkv, cap, nch_stride, scale_log2, po, pml, error_word, stream);
-        case 8: return launch_attn<DH, 8>(mk, mv, q, work, nbatch, items, Hq, Hkv, cap, nch_stride, scale_log2, po, pml, error_word, stream);
+        case 1: return launch_attn<DH, 1>(mk, mv, q, work, nbatch, items, Hq, Hkv, cap, nch_stride, scale_log2, po, pml, done_count, o, error_word, stream);
+        case 2: return launch_attn<DH, 2>(mk, mv, q, work, nbatch, items, Hq, Hkv, cap, nch_stride, scale_log2, po, pml, done_count, o, error_word, stream);
+        case 4: return launch_attn<DH, 4>(mk, mv, q, work, nbatch, items, Hq, Hkv, cap, nch_stride, scale_log2, po, pml, done_count, o, error_word, stream);
+        case 8: return launch_attn<DH, 8>(mk, mv, q, work, nbatch, items, Hq, Hkv, cap, nch_stride, scale_log2, po, pml, done_count, o, error_word, stream);
         default: return -1;
     }
 }
@@ -284,7 +309,7 @@ bool tc_attn_bind_cache(TcPlan* p, const void* kcache, const void* vcache, long 
 }
 
 int tc_attn_decode(TcPlan* p, const void* q, const BatchMeta& meta, const int32_t* stable_len, int B, int Hq, int Hkv, int dh, int cap,
-                   int max_kv_len, void* scratch, void* o, int* error_word, cudaStream_t stream) {
+                   int max_kv_len, void* scratch, int* done_count, void* o, int* error_word, cudaStream_t stream) {
     if (p == nullptr || !p->cache_maps_ok || B <= 0 || B > kMaxCallBatch || Hkv > 65535) return -1;
     if (dh != 64 && dh != 128) return -1;
     const int G = Hq / Hkv;
@@ -303,15 +328,24 @@ int tc_attn_decode(TcPlan* p, const void* q, const BatchMeta& meta, const int32_
     float* po = reinterpret_cast<float*>(scratch);
     float* pml = po + (size_t)B * Hq * nch * dh;
     const float scale_log2 = 1.4426950408889634f / sqrtf((float)dh);
+    // Few sequences: the last CTA of each head group merges its chunks (one launch less on a
+    // latency-bound step).  Many sequences: a separate, wider merge kernel is faster than the tails.
+    const bool fuse_merge = B <= 8;
+    if (!fuse_merge) done_count = nullptr;
     int launched = 0;
     if (items > 0) {
         const int rc = dh == 128
-            ? launch_attn_g<128>(G, p->cache_k, p->cache_v, static_cast<const bf16*>(q), work, B, items, Hq, Hkv, cap, nch, scale_log2, po, pml, error_word, stream)
-            : launch_attn_g<64>(G, p->cache_k, p->cache_v, static_cast<const bf16*>(q), work, B, items, Hq, Hkv, cap, nch, scale_log2, po, pml, error_word, stream);
+            ? launch_attn_g<128>(G, p->cache_k, p->cache_v, static_cast<const bf16*>(q), work, B, items, Hq, Hkv, cap, nch, scale_log2, po, pml,
+                                 done_count, static_cast<bf16*>(o), error_word, stream)
+            : launch_attn_g<64>(G, p->cache_k, p->cache_v, static_cast<const bf16*>(q), work, B, items, Hq, Hkv, cap, nch, scale_log2, po, pml,
+                                done_count, static_cast<bf16*>(o), error_word, stream);
         if (rc < 0) return rc;
         launched += rc;
     }
-    launched += launch_attn_combine(1, po, pml, meta, B, Hq, dh, nch, kChunk, o, stream);
+    // rows without any cached state got no CTA: their attention output is zero
+    bool any_empty = !fuse_merge;
+    for (int b = 0; b < B; ++b) any_empty |= (meta.kv_len[b] == 0);
+    if (any_empty) launched += launch_attn_combine(1, po, pml, meta, B, Hq, dh, nch, kChunk, o, stream);
     return launched;
 }
 

@@ -2,6 +2,7 @@
 // projections with fused epilogues, split-KV cross-attention decode over the cache, arg-max and
 // greedy acceptance.  All HBM-bound: 16-byte coalesced loads, fp32 accumulation.
 #include "kernels.h"
+#include "attn_combine.cuh"
 
 namespace beagle {
 
@@ -398,9 +399,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attn_decode_kernel(
     }
 }
 
-// One warp per (sequence, query head): the lanes first share the chunks' running maxima and
-// exp-sums (each lane a strided subset), then each lane owns dh/32 consecutive output dims and adds
-// the chunks' unnormalised partials with the weights exp(m_i - M), handed around by shuffles.
+// One warp per (sequence, query head), see attn_combine_warp.
 template <typename T, int DPL>
 __global__ void __launch_bounds__(256) attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
                                                           const BatchMeta meta, int nheads_total, int Hq, int dh, int nchunk_max,
@@ -409,54 +408,10 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(const float* __restri
     pdl_launch_dependents();
     pdl_wait();
     if (wid >= nheads_total) return;
-    const int b = wid / Hq;
-    const int kv_len = meta.kv_len[b];
+    const int kv_len = meta.kv_len[wid / Hq];
     const int nch = (kv_len + chunk - 1) / chunk;
     const size_t p0 = (size_t)wid * nchunk_max;
-    const int DH = dh;                          // DPL * 32, or 16 with DPL = 1 (upper half-warp idle)
-    const bool act = lane * DPL < DH;
-    float M = -INFINITY;
-    for (int i = lane; i < nch; i += 32) M = fmaxf(M, part_ml[2 * (p0 + i)]);
-    M = warp_max(M);
-    float acc[DPL];
-#pragma unroll
-    for (int v = 0; v < DPL; ++v) acc[v] = 0.f;
-    float den = 0.f;
-    for (int i0 = 0; i0 < nch; i0 += 32) {
-        const int i = i0 + lane;
-        float w = 0.f, l = 0.f;
-        if (i < nch) {
-            const float2 ml = *reinterpret_cast<const float2*>(part_ml + 2 * (p0 + i));
-            w = (ml.x == -INFINITY) ? 0.f : __expf(ml.x - M);
-            l = ml.y;
-        }
-        den = fmaf(w, l, den);
-        const int n_here = min(32, nch - i0);
-#pragma unroll 4
-        for (int j = 0; j < n_here; ++j) {
-            const float wj = __shfl_sync(0xffffffffu, w, j);
-            const float* src = part_o + (p0 + i0 + j) * DH + lane * DPL;
-            if (!act) continue;
-            if constexpr (DPL % 4 == 0) {
-#pragma unroll
-                for (int v = 0; v < DPL; v += 4) {
-                    const float4 t = *reinterpret_cast<const float4*>(src + v);
-                    acc[v] = fmaf(wj, t.x, acc[v]); acc[v + 1] = fmaf(wj, t.y, acc[v + 1]);
-                    acc[v + 2] = fmaf(wj, t.z, acc[v + 2]); acc[v + 3] = fmaf(wj, t.w, acc[v + 3]);
-                }
-            } else {
-#pragma unroll
-                for (int v = 0; v < DPL; ++v) acc[v] = fmaf(wj, src[v], acc[v]);
-            }
-        }
-    }
-    den = warp_sum(den);
-    const float inv = (nch > 0 && den > 0.f) ? 1.0f / den : 0.f;
-    T* dst = o + (size_t)wid * DH + lane * DPL;
-    if (act) {
-#pragma unroll
-        for (int v = 0; v < DPL; ++v) dst[v] = from_float<T>(acc[v] * inv);
-    }
+    attn_combine_warp<T, DPL, false>(part_o + p0 * dh, part_ml + 2 * p0, nch, dh, lane, o + (size_t)wid * dh);
 }
 
 template <typename T>
@@ -543,32 +498,40 @@ int launch_attn_decode(int dtype, const void* q, const void* kcache, const void*
 // ------------------------------------------------------------------------------------------------
 // Arg-max finalisation of the LM head's per-block keys
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) argmax_finalize_kernel(const unsigned long long* __restrict__ partials, int nblk,
-                                                              const BatchMeta meta, int32_t* __restrict__ tokens_out,
-                                                              int tokens_out_stride, int32_t* __restrict__ last_token) {
+__global__ void __launch_bounds__(1024) argmax_finalize_kernel(const unsigned long long* __restrict__ partials, int nblk,
+                                                               const BatchMeta meta, int32_t* __restrict__ tokens_out,
+                                                               int tokens_out_stride, int32_t* __restrict__ last_token) {
     const int b = blockIdx.x;
     pdl_launch_dependents();
     pdl_wait();
+    const unsigned long long* row = partials + (size_t)b * nblk;
     unsigned long long key = 0ull;
-    for (int i = threadIdx.x; i < nblk; i += blockDim.x) {
-        const unsigned long long o = partials[(size_t)b * nblk + i];
-        key = o > key ? o : key;
+    for (int i0 = threadIdx.x; i0 < nblk; i0 += 4 * blockDim.x) {      // four independent loads in flight per thread
+        unsigned long long k[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { const int i = i0 + j * blockDim.x; k[j] = i < nblk ? row[i] : 0ull; }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) key = k[j] > key ? k[j] : key;
     }
     key = warp_max_u64(key);
-    __shared__ unsigned long long s_k[8];
+    __shared__ unsigned long long s_k[32];
     if ((threadIdx.x & 31) == 0) s_k[threadIdx.x >> 5] = key;
     __syncthreads();
-    if (threadIdx.x == 0) {
-        for (int w = 1; w < 8; ++w) key = s_k[w] > key ? s_k[w] : key;
-        const int tok = argmax_key_index(key);
-        if (tokens_out != nullptr) tokens_out[(size_t)b * tokens_out_stride] = tok;
-        last_token[meta.slot[b]] = tok;
+    if (threadIdx.x < 32) {
+        key = threadIdx.x < (blockDim.x >> 5) ? s_k[threadIdx.x] : 0ull;
+        key = warp_max_u64(key);
+        if (threadIdx.x == 0) {
+            const int tok = argmax_key_index(key);
+            if (tokens_out != nullptr) tokens_out[(size_t)b * tokens_out_stride] = tok;
+            last_token[meta.slot[b]] = tok;
+        }
     }
 }
 int launch_argmax_finalize(const unsigned long long* partials, int nblk, const BatchMeta& meta, int B,
                            int32_t* tokens_out, int tokens_out_stride, int32_t* last_token, cudaStream_t stream) {
     if (B <= 0) return 0;
-    launch_pdl(argmax_finalize_kernel, dim3(B), dim3(256), 0, stream, partials, nblk, meta, tokens_out, tokens_out_stride, last_token);
+    const int threads = nblk >= 2048 ? 1024 : 256;
+    launch_pdl(argmax_finalize_kernel, dim3(B), dim3(threads), 0, stream, partials, nblk, meta, tokens_out, tokens_out_stride, last_token);
     return 1;
 }
 
