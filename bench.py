@@ -486,6 +486,8 @@ def main():
     ap.add_argument("--workload", default=HEADLINE, choices=[k for k in WL.WORKLOADS if not k.startswith("c5")])
     ap.add_argument("--only-headline", action="store_true", help="skip the batch-1, block-forward and CPU legs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--only-block", action="store_true", help="diagnostic: time only the block-attention forward (C5 shape)")
+    ap.add_argument("--block-batch", type=int, default=0, help="sequences of the block forward (default: the workload's 8)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -508,6 +510,19 @@ def main():
     peaks = load_peaks()
     traffic = load_ncu_traffic()
     t_wall = time.perf_counter()
+
+    if args.only_block:
+        w5 = WL.WORKLOADS["c5_block_llama2_7b"]
+        if args.block_batch > 0:
+            w5 = w5.scaled(batch=args.block_batch)
+        head5 = BeagleHead.from_workload(w5, WL.make_weights(w5), device=device, max_slots=1, max_ctx=64, max_draft=1)
+        res = bench_block(head5, w5, steps=max(1, args.steps), warmup=args.warmup, peaks=peaks)
+        if rank == 0:
+            print(json.dumps({"metric": "block_positions_per_s", "value": res["positions_per_s"], "unit": "positions/s", "n_gpus": world,
+                              "steps": args.steps, "warmup": args.warmup, "ms_per_step": res["ms_per_forward"], "higher_is_better": True,
+                              "dtype": "bf16", "data": "synthetic", "config": {"workload": w5.name, "batch": w5.batch, "S": w5.ctx_max},
+                              "block_forward": res}), flush=True)
+        return
 
     w = WL.WORKLOADS[args.workload]
     iters = args.steps + args.warmup

@@ -13,26 +13,28 @@ namespace beagle {
 template <bool SAME_KERNEL, typename V>
 __device__ __forceinline__ V ld_partial(const V* p) { return SAME_KERNEL ? __ldcg(p) : *p; }
 
-template <typename T, int DPL, bool SAME_KERNEL>
-__device__ __forceinline__ void attn_combine_warp(const float* part_o, const float* part_ml, int nch, int dh, int lane, T* o) {
+// Merge of chunks [i_begin, i_end): running maximum M, exp-sum den and unnormalised acc (this
+// lane's DPL dims), all relative to M.
+template <int DPL, bool SAME_KERNEL>
+__device__ __forceinline__ void attn_combine_range(const float* part_o, const float* part_ml, int i_begin, int i_end, int dh, int lane,
+                                                   float& M, float& den, float* acc) {
     const bool act = lane * DPL < dh;
-    float M = -INFINITY;
-    for (int i = lane; i < nch; i += 32) M = fmaxf(M, ld_partial<SAME_KERNEL>(part_ml + 2 * i));
+    M = -INFINITY;
+    for (int i = i_begin + lane; i < i_end; i += 32) M = fmaxf(M, ld_partial<SAME_KERNEL>(part_ml + 2 * i));
     M = warp_max(M);
-    float acc[DPL];
 #pragma unroll
     for (int v = 0; v < DPL; ++v) acc[v] = 0.f;
-    float den = 0.f;
-    for (int i0 = 0; i0 < nch; i0 += 32) {
+    den = 0.f;
+    for (int i0 = i_begin; i0 < i_end; i0 += 32) {
         const int i = i0 + lane;
         float w = 0.f, l = 0.f;
-        if (i < nch) {
+        if (i < i_end) {
             const float2 ml = ld_partial<SAME_KERNEL>(reinterpret_cast<const float2*>(part_ml + 2 * i));
             w = (ml.x == -INFINITY) ? 0.f : __expf(ml.x - M);
             l = ml.y;
         }
         den = fmaf(w, l, den);
-        const int n_here = min(32, nch - i0);
+        const int n_here = min(32, i_end - i0);
 #pragma unroll 4
         for (int j = 0; j < n_here; ++j) {
             const float wj = __shfl_sync(0xffffffffu, w, j);
@@ -52,8 +54,14 @@ __device__ __forceinline__ void attn_combine_warp(const float* part_o, const flo
         }
     }
     den = warp_sum(den);
+}
+
+template <typename T, int DPL, bool SAME_KERNEL>
+__device__ __forceinline__ void attn_combine_warp(const float* part_o, const float* part_ml, int nch, int dh, int lane, T* o) {
+    float M, den, acc[DPL];
+    attn_combine_range<DPL, SAME_KERNEL>(part_o, part_ml, 0, nch, dh, lane, M, den, acc);
     const float inv = (nch > 0 && den > 0.f) ? 1.0f / den : 0.f;
-    if (act) {
+    if (lane * DPL < dh) {
 #pragma unroll
         for (int v = 0; v < DPL; ++v) o[lane * DPL + v] = from_float<T>(acc[v] * inv);
     }

@@ -209,8 +209,9 @@ struct FinishArgs {
     bf16* kcache; bf16* vcache; int Hkv, dh, cap; RowMap slot; RowMap pos;
 };
 
-constexpr int kFinThreads = 256;
-constexpr int kFinCols = kFinThreads * 4;   // features per CTA and pass
+constexpr int kFinThreads = 256;             // whole-row mode (fused RMSNorm)
+constexpr int kFinColThreads = 64;           // column mode: many small CTAs, one float4 per thread
+constexpr int kFinCols = kFinColThreads * 4; // features per CTA in column mode
 
 template <int MODE>
 __global__ void __launch_bounds__(kFinThreads) tc_finish_kernel(const FinishArgs a) {
@@ -375,11 +376,12 @@ int tc_skinny(TcPlan* p, int mode, const SkinnyArgs& g, cudaStream_t stream) {
     f.slot = g.slot; f.pos = g.pos;
     const bool whole_row = (mode == SK_RESID && g.norm_out != nullptr);
     dim3 fgrid(g.B, whole_row ? 1 : (g.N + kFinCols - 1) / kFinCols);
+    const dim3 fblock(whole_row ? kFinThreads : kFinColThreads);
     switch (mode) {
-        case SK_STORE: launch_pdl(tc_finish_kernel<SK_STORE>, fgrid, dim3(kFinThreads), 0, stream, f); break;
-        case SK_RESID: launch_pdl(tc_finish_kernel<SK_RESID>, fgrid, dim3(kFinThreads), 0, stream, f); break;
-        case SK_SILU_MUL: launch_pdl(tc_finish_kernel<SK_SILU_MUL>, fgrid, dim3(kFinThreads), 0, stream, f); break;
-        case SK_KV: launch_pdl(tc_finish_kernel<SK_KV>, fgrid, dim3(kFinThreads), 0, stream, f); break;
+        case SK_STORE: launch_pdl(tc_finish_kernel<SK_STORE>, fgrid, fblock, 0, stream, f); break;
+        case SK_RESID: launch_pdl(tc_finish_kernel<SK_RESID>, fgrid, fblock, 0, stream, f); break;
+        case SK_SILU_MUL: launch_pdl(tc_finish_kernel<SK_SILU_MUL>, fgrid, fblock, 0, stream, f); break;
+        case SK_KV: launch_pdl(tc_finish_kernel<SK_KV>, fgrid, fblock, 0, stream, f); break;
         default: return -1;
     }
     return 2;

@@ -399,32 +399,56 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attn_decode_kernel(
     }
 }
 
-// One warp per (sequence, query head), see attn_combine_warp.
+// One CTA of four warps per (sequence, query head): each warp merges a quarter of the chunks
+// (attn_combine_range), warp 0 merges the four results.
 template <typename T, int DPL>
-__global__ void __launch_bounds__(256) attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
-                                                          const BatchMeta meta, int nheads_total, int Hq, int dh, int nchunk_max,
-                                                          int chunk, T* __restrict__ o) {
-    const int wid = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+__global__ void __launch_bounds__(128) attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
+                                                          const BatchMeta meta, int Hq, int dh, int nchunk_max, int chunk,
+                                                          T* __restrict__ o) {
+    const int head = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     pdl_launch_dependents();
     pdl_wait();
-    if (wid >= nheads_total) return;
-    const int kv_len = meta.kv_len[wid / Hq];
+    const int kv_len = meta.kv_len[head / Hq];
     const int nch = (kv_len + chunk - 1) / chunk;
-    const size_t p0 = (size_t)wid * nchunk_max;
-    attn_combine_warp<T, DPL, false>(part_o + p0 * dh, part_ml + 2 * p0, nch, dh, lane, o + (size_t)wid * dh);
+    const size_t p0 = (size_t)head * nchunk_max;
+    const int per = (nch + 3) / 4;
+    float M, den, acc[DPL];
+    attn_combine_range<DPL, false>(part_o + p0 * dh, part_ml + 2 * p0, min(nch, warp * per), min(nch, (warp + 1) * per), dh, lane, M, den, acc);
+    __shared__ float s_M[4], s_den[4], s_acc[4][DPL * 32];
+    if (lane == 0) { s_M[warp] = M; s_den[warp] = den; }
+#pragma unroll
+    for (int v = 0; v < DPL; ++v) s_acc[warp][lane * DPL + v] = acc[v];
+    __syncthreads();
+    if (warp == 0) {
+        const float Mx = fmaxf(fmaxf(s_M[0], s_M[1]), fmaxf(s_M[2], s_M[3]));
+        float d = 0.f, out[DPL];
+#pragma unroll
+        for (int v = 0; v < DPL; ++v) out[v] = 0.f;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            const float wgt = (s_M[w] == -INFINITY) ? 0.f : __expf(s_M[w] - Mx);
+            d = fmaf(wgt, s_den[w], d);
+#pragma unroll
+            for (int v = 0; v < DPL; ++v) out[v] = fmaf(wgt, s_acc[w][lane * DPL + v], out[v]);
+        }
+        const float inv = (nch > 0 && d > 0.f) ? 1.0f / d : 0.f;
+        if (lane * DPL < dh) {
+#pragma unroll
+            for (int v = 0; v < DPL; ++v) o[(size_t)head * dh + lane * DPL + v] = from_float<T>(out[v] * inv);
+        }
+    }
 }
 
 template <typename T>
 static int attn_combine_dispatch(const float* part_o, const float* part_ml, const BatchMeta& meta, int B, int Hq, int dh,
                                  int nchunk_stride, int chunk, T* o, cudaStream_t stream) {
-    const int total = B * Hq;
-    const int grid = (total * 32 + 255) / 256;
+    const int grid = B * Hq;
     switch (dh) {
-        case 32: launch_pdl(attn_combine_kernel<T, 1>, dim3(grid), dim3(256), 0, stream, part_o, part_ml, meta, total, Hq, dh, nchunk_stride, chunk, o); return 1;
-        case 64: launch_pdl(attn_combine_kernel<T, 2>, dim3(grid), dim3(256), 0, stream, part_o, part_ml, meta, total, Hq, dh, nchunk_stride, chunk, o); return 1;
-        case 128: launch_pdl(attn_combine_kernel<T, 4>, dim3(grid), dim3(256), 0, stream, part_o, part_ml, meta, total, Hq, dh, nchunk_stride, chunk, o); return 1;
-        case 256: launch_pdl(attn_combine_kernel<T, 8>, dim3(grid), dim3(256), 0, stream, part_o, part_ml, meta, total, Hq, dh, nchunk_stride, chunk, o); return 1;
-        case 16: launch_pdl(attn_combine_kernel<T, 1>, dim3(grid), dim3(256), 0, stream, part_o, part_ml, meta, total, Hq, dh, nchunk_stride, chunk, o); return 1;
+        case 32: launch_pdl(attn_combine_kernel<T, 1>, dim3(grid), dim3(128), 0, stream, part_o, part_ml, meta, Hq, dh, nchunk_stride, chunk, o); return 1;
+        case 64: launch_pdl(attn_combine_kernel<T, 2>, dim3(grid), dim3(128), 0, stream, part_o, part_ml, meta, Hq, dh, nchunk_stride, chunk, o); return 1;
+        case 128: launch_pdl(attn_combine_kernel<T, 4>, dim3(grid), dim3(128), 0, stream, part_o, part_ml, meta, Hq, dh, nchunk_stride, chunk, o); return 1;
+        case 256: launch_pdl(attn_combine_kernel<T, 8>, dim3(grid), dim3(128), 0, stream, part_o, part_ml, meta, Hq, dh, nchunk_stride, chunk, o); return 1;
+        case 16: launch_pdl(attn_combine_kernel<T, 1>, dim3(grid), dim3(128), 0, stream, part_o, part_ml, meta, Hq, dh, nchunk_stride, chunk, o); return 1;
         default: return -1;
     }
 }
