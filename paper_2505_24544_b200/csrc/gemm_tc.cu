@@ -7,6 +7,10 @@
 // [N, K]; epilogues: store, +residual, SiLU(g)*u (two accumulators), fp32 logits, packed arg-max
 // keys, scatter into the K/V cache.
 //
+// The kernel is persistent: one CTA per SM walks over its tiles with the TMA ring running ahead
+// across tile boundaries and two accumulator buffers in TMEM (512 columns), so the epilogue of
+// a tile overlaps the MMAs of the next.
+//
 // Every wait on an mbarrier is bounded; a wait that runs out sets a device error word and the CTA
 // drains and frees its TMEM instead of hanging.
 #include <cuda.h>
@@ -57,33 +61,36 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     using SM = TcSmem<BN, DUAL>;
     constexpr int kStages = SM::kStages;
     constexpr int kABytes = BM * BK * 2, kBBytes = BN * BK * 2;
-    constexpr uint32_t kTmemCols = (DUAL ? 2 * BN : BN) < 32 ? 32 : (DUAL ? 2 * BN : BN);
+    constexpr uint32_t kAccCols = DUAL ? 2 * BN : BN;       // TMEM columns of one tile's accumulator(s)
+    constexpr uint32_t kTmemCols = 2 * kAccCols;            // two tiles in flight: the epilogue of one overlaps the MMAs of the next
+    static_assert(kTmemCols == 512 || kTmemCols == 256 || kTmemCols == 128 || kTmemCols == 64, "TMEM allocation must be a power of two");
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + kStages * SM::kStageBytes);
-    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * kStages, bar_acc = bar_empty + 8 * kStages;
-    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 1);
+    const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * kStages;
+    const uint32_t bar_acc_full = bar_empty + 8 * kStages, bar_acc_empty = bar_acc_full + 16;     // two accumulator buffers
+    uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
     volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    // tile coordinates
-    int ta, tb;
-    {
-        const int pid = blockIdx.x;
+    // Persistent CTA: tiles blockIdx.x, blockIdx.x + gridDim.x, ...  Consecutive tile ids walk down a
+    // group of `group_m` row tiles before moving to the next column tile (L2 reuse of both operands).
+    const int ntiles = args.tiles_a * args.tiles_b;
+    auto tile_coords = [&](int pid, int& ta, int& tb) {
         const int per_group = args.group_m * args.tiles_b;
         const int g = pid / per_group;
         const int first = g * args.group_m;
         const int gsize = min(args.tiles_a - first, args.group_m);
         ta = first + (pid % per_group) % gsize;
         tb = (pid % per_group) / gsize;
-    }
+    };
     const int nkb = (args.K + BK - 1) / BK;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-        mbar_init(bar_acc, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(bar_acc_full + 8 * b, 1); mbar_init(bar_acc_empty + 8 * b, 4); }
         *s_abort = 0;
         fence_barrier_init();
     }
@@ -98,18 +105,24 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     if (warp == 0) {
         // ---------------- TMA producer
         if (lane == 0) {
-            int issued = 0;
-            for (int kb = 0; kb < nkb; ++kb) {
-                const int s = kb % kStages;
-                const uint32_t ph = (kb / kStages) & 1;
-                if (!mbar_wait(bar_empty + 8 * s, ph ^ 1, s_abort)) break;
-                const uint32_t sa = smem_base + s * SM::kStageBytes, sb = sa + kABytes;
-                mbar_expect_tx(bar_full + 8 * s, kABytes + kBBytes * (DUAL ? 2 : 1));
-                const int kc = kb * BK;
-                tma_load_2d(sa, &tmA, bar_full + 8 * s, kc, ta * BM);
-                tma_load_2d(sb, &tmB, bar_full + 8 * s, kc, tb * BN);
-                if (DUAL) tma_load_2d(sb + kBBytes, &tmB2, bar_full + 8 * s, kc, tb * BN);
-                ++issued;
+            int issued = 0;                           // k-blocks requested so far, over all tiles
+            bool ok = true;
+            for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x) {
+                int ta, tb;
+                tile_coords(t, ta, tb);
+                for (int kb = 0; kb < nkb; ++kb) {
+                    const int s = issued % kStages;
+                    const uint32_t ph = (issued / kStages) & 1;
+                    ok = mbar_wait(bar_empty + 8 * s, ph ^ 1, s_abort);
+                    if (!ok) break;
+                    const uint32_t sa = smem_base + s * SM::kStageBytes, sb = sa + kABytes;
+                    mbar_expect_tx(bar_full + 8 * s, kABytes + kBBytes * (DUAL ? 2 : 1));
+                    const int kc = kb * BK;
+                    tma_load_2d(sa, &tmA, bar_full + 8 * s, kc, ta * BM);
+                    tma_load_2d(sb, &tmB, bar_full + 8 * s, kc, tb * BN);
+                    if (DUAL) tma_load_2d(sb + kBBytes, &tmB2, bar_full + 8 * s, kc, tb * BN);
+                    ++issued;
+                }
             }
             if (*s_abort) {
                 // drain: copies already issued still land in shared memory; wait (bounded) for the last of each stage
@@ -126,36 +139,50 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc(BM, BN);
             bool ok = true;
-            for (int kb = 0; kb < nkb && ok; ++kb) {
-                const int s = kb % kStages;
-                const uint32_t ph = (kb / kStages) & 1;
-                ok = mbar_wait(bar_full + 8 * s, ph, s_abort);
+            int consumed = 0, it = 0;
+            for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++it) {
+                const int buf = it & 1;
+                // the epilogue must have drained this accumulator buffer (two tiles ago)
+                ok = mbar_wait(bar_acc_empty + 8 * buf, ((it >> 1) & 1) ^ 1, s_abort);
                 if (!ok) break;
                 fence_after();
-                const uint32_t sa = smem_base + s * SM::kStageBytes, sb = sa + kABytes;
-                const uint64_t da = umma_desc(sa), db = umma_desc(sb), db2 = umma_desc(sb + kBBytes);
+                const uint32_t tacc = tmem_base + buf * kAccCols;
+                for (int kb = 0; kb < nkb; ++kb) {
+                    const int s = consumed % kStages;
+                    const uint32_t ph = (consumed / kStages) & 1;
+                    ok = mbar_wait(bar_full + 8 * s, ph, s_abort);
+                    if (!ok) break;
+                    fence_after();
+                    const uint32_t sa = smem_base + s * SM::kStageBytes, sb = sa + kABytes;
+                    const uint64_t da = umma_desc(sa), db = umma_desc(sb), db2 = umma_desc(sb + kBBytes);
 #pragma unroll
-                for (int k = 0; k < BK / UMMA_K; ++k) {
-                    const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
-                    const uint64_t koff = static_cast<uint64_t>((k * UMMA_K * 2) >> 4);   // advance inside the swizzle atom
-                    umma_bf16(tmem_base, da + koff, db + koff, idesc, acc);
-                    if (DUAL) umma_bf16(tmem_base + BN, da + koff, db2 + koff, idesc, acc);
+                    for (int k = 0; k < BK / UMMA_K; ++k) {
+                        const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
+                        const uint64_t koff = static_cast<uint64_t>((k * UMMA_K * 2) >> 4);   // advance inside the swizzle atom
+                        umma_bf16(tacc, da + koff, db + koff, idesc, acc);
+                        if (DUAL) umma_bf16(tacc + BN, da + koff, db2 + koff, idesc, acc);
+                    }
+                    umma_commit(bar_empty + 8 * s);   // frees the stage once these MMAs have read it
+                    ++consumed;
                 }
-                umma_commit(bar_empty + 8 * s);       // frees the stage once these MMAs have read it
+                umma_commit(bar_acc_full + 8 * buf);  // this tile's accumulators are complete (or the tile was abandoned)
             }
-            umma_commit(bar_acc);                     // accumulators complete (or nothing was issued)
         }
     } else {
         // ---------------- epilogue: warp w reads TMEM lanes [32*(w%4), +32)
         const int q = warp & 3;
         const int row_in_tile = q * 32 + lane;
-        const int arow = ta * BM + row_in_tile;      // row of A this thread owns
-        bool ok = true;
-        if (nkb > 0) ok = mbar_wait(bar_acc, 0, s_abort);
-        ok = __all_sync(0xffffffffu, ok);            // the TMEM loads below are warp-collective
-        fence_after();
-        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
-        if (ok && nkb > 0) {
+        int it = 0;
+        for (int t = blockIdx.x; t < ntiles; t += gridDim.x, ++it) {
+            int ta, tb;
+            tile_coords(t, ta, tb);
+            const int buf = it & 1;
+            const int arow = ta * BM + row_in_tile;  // row of A this thread owns
+            bool ok = mbar_wait(bar_acc_full + 8 * buf, (it >> 1) & 1, s_abort);
+            ok = __all_sync(0xffffffffu, ok);        // the TMEM loads below are warp-collective
+            if (!ok) break;
+            fence_after();
+            const uint32_t taddr = tmem_base + buf * kAccCols + (static_cast<uint32_t>(q * 32) << 16);
             {
                 const int m = arow;
                 int slot = 0, pos = 0;
@@ -239,6 +266,10 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
                 }
                 if (EPI == TC_ARGMAX && m < args.a_rows) args.keys[(size_t)m * args.keys_ld + tb] = best;
             }
+            // this warp has read its quarter of the buffer: hand it back to the MMA issuer
+            fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
         }
     }
 
@@ -348,7 +379,8 @@ int tc_gemm(TcPlan* p, int epi, const GemmArgs& g, cudaStream_t stream) {
     a.keys = g.keys; a.keys_ld = a.tiles_b;
     a.error_word = g.error_word;
     if (epi == GEMM_KV_CACHE && (g.dh % 16)) return -1;
-    dim3 grid(a.tiles_a * a.tiles_b, 1, 1);
+    const int ntiles = a.tiles_a * a.tiles_b;
+    dim3 grid(ntiles < p->sm_count ? ntiles : p->sm_count, 1, 1);        // persistent: one CTA per SM
     switch (epi) {
         case GEMM_STORE: return launch_tc<256, false, TC_STORE>(mapA, *mapB, *mapB, a, grid, stream);
         case GEMM_RESID: return launch_tc<256, false, TC_RESID>(mapA, *mapB, *mapB, a, grid, stream);
