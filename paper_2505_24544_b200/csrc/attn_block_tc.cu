@@ -7,7 +7,8 @@
 // processed unmasked, the one or two tiles on the diagonal compare j with n(p) per element, and
 // the predicted keys are a second pass over those diagonal tiles with the band mask.
 //
-// K and V tiles of 64 keys arrive by TMA (128-byte swizzle) in a two-stage ring; each of the four
+// K and V tiles of 64 keys arrive by TMA (128-byte swizzle) in a two-stage ring (64 KB per CTA,
+// three CTAs per SM); each of the four
 // warps owns 16 queries: S = Q K^T (ldmatrix + mma.sync m16n8k16), online softmax in registers,
 // O += P V (ldmatrix.trans).  Attention is about 2.5 % of the block path's flop; the projections
 // around it run on tcgen05.
@@ -54,7 +55,7 @@ struct BlkArgs {
 };
 
 template <int DH>
-__global__ void __launch_bounds__(kWarps * 32) attn_block_tc_kernel(const __grid_constant__ CUtensorMap tmQ,
+__global__ void __launch_bounds__(kWarps * 32, 3) attn_block_tc_kernel(const __grid_constant__ CUtensorMap tmQ,
                                                                    const __grid_constant__ CUtensorMap tmKt,
                                                                    const __grid_constant__ CUtensorMap tmVt,
                                                                    const __grid_constant__ CUtensorMap tmKp,
@@ -64,9 +65,9 @@ __global__ void __launch_bounds__(kWarps * 32) attn_block_tc_kernel(const __grid
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-    const uint32_t sQ = smem_base;
-    const uint32_t sKV = smem_base + kTile;     // stage s: K at sKV + s*2*kTile, V right after it
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + 5 * kTile);
+    const uint32_t sKV = smem_base;             // stage s: K at sKV + s*2*kTile, V right after it
+    const uint32_t sQ = sKV + 2 * kTile;        // the Q tile borrows stage 1's K slot until its fragments are in registers
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + 4 * kTile);
     const uint32_t barQ = smem_u32(bars), barF = barQ + 8;      // barF[2]: tile landed
     __shared__ int s_abort;
 
@@ -133,6 +134,7 @@ __global__ void __launch_bounds__(kWarps * 32) attn_block_tc_kernel(const __grid
 #pragma unroll
     for (int ks = 0; ks < DH / 16; ++ks)
         ldsm_x4(sQ + toff(warp * 16 + (lane & 7) + 8 * ((lane >> 3) & 1), 2 * ks + (lane >> 4)), qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3]);
+    __syncthreads();                                                // stage 1 may now receive K/V tiles
 
     float o[DH / 8][4];
 #pragma unroll
@@ -215,7 +217,7 @@ __global__ void __launch_bounds__(kWarps * 32) attn_block_tc_kernel(const __grid
         __syncthreads();                                            // everyone is done with stage st
     }
 
-    // ---- normalise (the row sums were reduced over the 4 lanes of a row only now) and store through the Q tile's memory
+    // ---- normalise (the row sums were reduced over the 4 lanes of a row only now) and store through stage 0's memory
 #pragma unroll
     for (int r = 0; r < 2; ++r) {
         l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
@@ -223,7 +225,6 @@ __global__ void __launch_bounds__(kWarps * 32) attn_block_tc_kernel(const __grid
     }
     const float inv0 = (ok && l_run[0] > 0.f) ? 1.f / l_run[0] : 0.f;
     const float inv1 = (ok && l_run[1] > 0.f) ? 1.f / l_run[1] : 0.f;
-    __syncthreads();                                                // all warps have read their Q fragments
 #pragma unroll
     for (int nt = 0; nt < DH / 8; ++nt) {
         const int r0 = warp * 16 + g;
@@ -245,7 +246,7 @@ __global__ void __launch_bounds__(kWarps * 32) attn_block_tc_kernel(const __grid
 
 template <int DH>
 int launch_blk(const CUtensorMap* maps, const BlkArgs& a, dim3 grid, cudaStream_t stream) {
-    constexpr int kSmem = 5 * 64 * DH * 2 + 1024 + 64;
+    constexpr int kSmem = 4 * 64 * DH * 2 + 1024 + 64;
     static bool attr_done = false;
     if (!attr_done) {
         if (cudaFuncSetAttribute(attn_block_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess) return -1;
