@@ -29,4 +29,8 @@ from .beagle_oracle import (  # noqa: F401
     block_forward,
     argmax_lowest,
     verify_greedy,
+    softmax_rows,
+    residual_distribution,
+    inverse_cdf,
+    verify_sample,
 )

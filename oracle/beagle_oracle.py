@@ -45,6 +45,9 @@ at the full model sizes the rounding of the cache alone moves logits of
 standard deviation ~2.7 by up to ~5e-2, so a comparison that wants to see
 kernel errors rather than storage noise has to round at the same places.
 
+Speculative-sampling verification (verify_sample) follows Section 3 literally;
+the random numbers it needs are inputs.
+
 Pins (tests/test_oracle_*.py, all CPU): hand-worked tiny head, softmax row
 sums, single-key / identical-key special cases, GQA==MHA with repeated heads,
 mask brute force against the literal window rule, block forward == step-by-step
@@ -475,3 +478,87 @@ def verify_greedy(draft_tokens: np.ndarray, target_logits: Optional[np.ndarray] 
         accept[b] = a
         out[b, : a + 1] = g[b, : a + 1]
     return accept, out
+
+
+# --------------------------------------------------------------------------- speculative-sampling verification
+
+def softmax_rows(logits: np.ndarray, temperature: float = 1.0) -> np.ndarray:
+    """softmax(z / temperature) over the last axis, with max-subtraction."""
+    z = np.asarray(logits, dtype=F64) / F64(temperature)
+    z = z - np.max(z, axis=-1, keepdims=True)
+    e = np.exp(z)
+    return e / np.sum(e, axis=-1, keepdims=True)
+
+
+def residual_distribution(p: np.ndarray, q: Optional[np.ndarray]) -> np.ndarray:
+    """The distribution the extra token is drawn from (Section 3): normalised
+    max(0, p - q) at a rejection; p itself after gamma acceptances, where no
+    draft distribution exists.  If p == q everywhere (no mass left, a case that
+    cannot follow a rejection) it falls back to p."""
+    p = np.asarray(p, dtype=F64)
+    if q is None:
+        return p / np.sum(p)
+    w = np.maximum(0.0, p - np.asarray(q, dtype=F64))
+    s = np.sum(w)
+    return w / s if s > 0.0 else p / np.sum(p)
+
+
+def inverse_cdf(dist: np.ndarray, r: float) -> Tuple[int, float]:
+    """Token drawn from ``dist`` with the uniform r in [0, 1): the smallest v
+    whose cumulative mass exceeds r.  Also returns how far r lies from the
+    nearest cumulative boundary (the decision margin of this draw)."""
+    c = np.cumsum(np.asarray(dist, dtype=F64))
+    c[-1] = max(c[-1], 1.0)
+    v = int(np.searchsorted(c, r, side="right"))
+    v = min(v, len(c) - 1)
+    lo = c[v - 1] if v > 0 else 0.0
+    return v, float(min(r - lo, c[v] - r))
+
+
+def verify_sample(draft_tokens: np.ndarray, draft_logits: np.ndarray, target_logits: np.ndarray,
+                  u_accept: np.ndarray, u_resample: np.ndarray,
+                  temperature: float = 1.0) -> Dict[str, np.ndarray]:
+    """Lossless draft/verify acceptance under sampling (Section 3).
+
+    For one SD iteration of B sequences: drafts t_1..t_gamma [B, gamma], the
+    draft's logits at those positions [gamma, B, V] (one block per draft step),
+    the target's logits at positions 1..gamma+1 [B, gamma+1, V], and the random
+    numbers the method draws, passed in: u_accept [B, gamma] and u_resample [B],
+    uniform in [0, 1).  With p_i = softmax(target_i / T), q_i = softmax(draft_i / T):
+    draft i is accepted iff u_accept[i] < min(1, p_i(t_i) / q_i(t_i)); at the first
+    rejection j (or j = gamma + 1) one token is drawn by inverse CDF with
+    u_resample from the normalised max(0, p_j - q_j) (from p_{gamma+1} when
+    nothing was rejected).
+
+    Returns accept_len [B]; out_tokens [B, gamma+1] = the accepted drafts, the
+    extra token, then -1; and the decision margins accept_margin [B] (smallest
+    |u - ratio| over the tests made) and resample_margin [B] (distance of
+    u_resample to the nearest CDF boundary), which tell a checker where another
+    floating-point precision may legitimately decide otherwise.
+    """
+    draft = np.asarray(draft_tokens, dtype=np.int64)
+    B, gamma = draft.shape
+    ql = np.asarray(draft_logits, dtype=F64).reshape(gamma, B, -1)
+    pl = np.asarray(target_logits, dtype=F64).reshape(B, gamma + 1, -1)
+    ua = np.asarray(u_accept, dtype=F64).reshape(B, gamma)
+    ur = np.asarray(u_resample, dtype=F64).reshape(B)
+    accept = np.zeros(B, dtype=np.int64)
+    out = np.full((B, gamma + 1), -1, dtype=np.int64)
+    am = np.full(B, np.inf)
+    rm = np.zeros(B)
+    for b in range(B):
+        p = softmax_rows(pl[b], temperature)                         # [gamma+1, V]
+        q = softmax_rows(ql[:, b, :], temperature) if gamma else np.zeros((0, p.shape[1]))
+        a = 0
+        while a < gamma:
+            t = int(draft[b, a])
+            ratio = min(1.0, p[a, t] / q[a, t]) if q[a, t] > 0.0 else 1.0
+            am[b] = min(am[b], abs(ua[b, a] - ratio) if ratio < 1.0 else np.inf)
+            if not (ua[b, a] < ratio):
+                break
+            a += 1
+        accept[b] = a
+        out[b, :a] = draft[b, :a]
+        dist = residual_distribution(p[a], q[a] if a < gamma else None)
+        out[b, a], rm[b] = inverse_cdf(dist, ur[b])
+    return {"accept_len": accept, "out_tokens": out, "accept_margin": am, "resample_margin": rm}

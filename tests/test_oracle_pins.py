@@ -415,6 +415,80 @@ def test_against_torch_library_routines():
     np.testing.assert_array_equal(ours["argmax"], z.argmax(-1).numpy())
 
 
+# ----------------------------------------------------------------------------- speculative-sampling verification
+
+def _logits_of(dist):
+    return np.log(np.asarray(dist, dtype=float))
+
+
+def test_verify_sample_first_token_follows_the_target_distribution():
+    """Losslessness (Section 3): whatever q is, the first emitted token is distributed as p_1.
+    Integrated over a midpoint grid of the three uniforms (draft draw, acceptance test, resample);
+    p and q are dyadic so that every threshold falls on a grid line and the integral is exact."""
+    p = np.array([3, 1, 1, 3]) / 8.0
+    q = np.array([1, 4, 2, 1]) / 8.0            # ratios min(1, p/q) = 1, 1/4, 1/2, 1; residual (1/2, 0, 0, 1/2)
+    n = 16
+    mid = (np.arange(n) + 0.5) / n
+    cq = np.cumsum(q)
+    hist = np.zeros(4)
+    ua, ur = np.meshgrid(mid, mid, indexing="ij")
+    B = ua.size
+    for ud in mid:                                               # the draft token itself is drawn from q
+        t = int(np.searchsorted(cq, ud, side="right"))
+        res = O.verify_sample(np.full((B, 1), t), np.broadcast_to(_logits_of(q), (1, B, 4)),
+                              np.broadcast_to(_logits_of(np.stack([p, p])), (B, 2, 4)), ua.reshape(B, 1), ur.reshape(B))
+        hist += np.bincount(res["out_tokens"][:, 0], minlength=4)
+        assert np.all(res["accept_len"] <= 1) and np.all(res["out_tokens"][res["accept_len"] == 1, 0] == t)
+    np.testing.assert_allclose(hist / hist.sum(), p, atol=1e-12)
+
+
+def test_verify_sample_special_cases():
+    V = 5
+    rng = np.random.default_rng(71)
+    z = rng.normal(size=(3, V))
+    draft = np.array([[1, 4]])
+    u = rng.random((1, 2))
+    # q == p: every draft is accepted, the extra token comes from p_{gamma+1} by inverse CDF
+    r = O.verify_sample(draft, z[:2][:, None, :], z[None], u, np.array([0.999999]))
+    assert r["accept_len"][0] == 2 and r["out_tokens"][0].tolist() == [1, 4, V - 1]
+    r = O.verify_sample(draft, z[:2][:, None, :], z[None], u, np.array([0.0]))
+    assert r["out_tokens"][0].tolist() == [1, 4, 0]
+    # the target gives the first draft (almost) no mass: rejected at once, and the residual never returns it
+    zt = z.copy(); zt[0, 1] = -80.0
+    for ur in (0.0, 0.3, 0.7, 0.999):
+        r = O.verify_sample(draft, z[:2][:, None, :], zt[None], np.array([[1e-9, 0.5]]), np.array([ur]))
+        assert r["accept_len"][0] == 0 and r["out_tokens"][0, 0] != 1 and r["out_tokens"][0, 1:].tolist() == [-1, -1]
+    # residual distribution by hand: p = (.5,.5,0), q = (.75,.25,0) -> max(0,p-q) = (0,.25,0) -> token 1 always
+    np.testing.assert_allclose(O.residual_distribution([0.5, 0.5, 0.0], [0.75, 0.25, 0.0]), [0, 1, 0])
+    np.testing.assert_allclose(O.residual_distribution([0.2, 0.8], None), [0.2, 0.8])
+    assert O.inverse_cdf(np.array([0.25, 0.5, 0.25]), 0.25)[0] == 1 and O.inverse_cdf(np.array([0.25, 0.5, 0.25]), 0.2499)[0] == 0
+    # temperature: T -> small makes both sides one-hot, so the rule reduces to greedy matching
+    zq = np.array([[0.0, 3.0, 1.0]]); zp = np.array([[0.0, 1.0, 3.0], [2.0, 0.0, 0.0]])
+    r = O.verify_sample(np.array([[1]]), zq[:, None, :], zp[None], np.array([[0.5]]), np.array([0.5]), temperature=0.01)
+    assert r["accept_len"][0] == 0 and r["out_tokens"][0, 0] == 2            # target's top-1 replaces the rejected draft
+    np.testing.assert_allclose(O.softmax_rows(np.array([[0.0, np.log(3.0)]])), [[0.25, 0.75]])
+    np.testing.assert_allclose(O.softmax_rows(np.array([[0.0, np.log(3.0)]]), temperature=0.5), [[0.1, 0.9]])
+
+
+def test_verify_sample_acceptance_rate_matches_closed_form():
+    """With drafts drawn from q, a position is accepted with probability sum_v min(p(v), q(v))."""
+    rng = np.random.default_rng(72)
+    V, gamma, B = 6, 3, 60000
+    zp, zq = rng.normal(size=(gamma + 1, V)), rng.normal(size=(gamma, V))
+    p, q = O.softmax_rows(zp), O.softmax_rows(zq)
+    draft = np.stack([rng.choice(V, size=B, p=q[i]) for i in range(gamma)], axis=1)
+    r = O.verify_sample(draft, np.broadcast_to(zq[:, None, :], (gamma, B, V)), np.broadcast_to(zp[None], (B, gamma + 1, V)),
+                        rng.random((B, gamma)), rng.random(B))
+    alpha = np.minimum(p[:gamma], q).sum(axis=1)
+    expect = alpha[0] + alpha[0] * alpha[1] + alpha[0] * alpha[1] * alpha[2]      # E[accept_len], tail-sum
+    assert abs(r["accept_len"].mean() - expect) < 4 * np.sqrt(gamma) / np.sqrt(B) + 1e-3
+    assert np.all((r["out_tokens"] >= 0).sum(axis=1) == r["accept_len"] + 1)
+    # the extra token after full acceptance follows p_{gamma+1}
+    full = r["accept_len"] == gamma
+    h = np.bincount(r["out_tokens"][full, gamma], minlength=V) / full.sum()
+    np.testing.assert_allclose(h, p[gamma], atol=4 / np.sqrt(full.sum()))
+
+
 # ----------------------------------------------------------------------------- storage mode
 
 def test_round_bf16_ties_to_even_and_matches_torch():
