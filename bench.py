@@ -465,6 +465,37 @@ def bench_block(head, w: WL.Workload, steps: int, warmup: int, peaks):
     }
 
 
+def bench_verify_sample(head, w: WL.Workload, steps: int, warmup: int, peaks):
+    """Acceptance under sampling on the workload's shape: batch x (gamma+1) bf16 target rows and
+    gamma x batch fp32 draft rows of V logits; HBM-bound (every logit is read once, two rows per
+    sequence a second time)."""
+    import torch
+    dev = head.device
+    g = torch.Generator(device=dev)
+    g.manual_seed(w.seed + 1)
+    B, gamma, V = w.batch, w.gamma, w.vocab
+    zq = torch.randn(gamma, B, V, generator=g, device=dev, dtype=torch.float32) * 2
+    zp = (zq.transpose(0, 1) * 0.7 + torch.randn(B, gamma, V, generator=g, device=dev) * 1.4)
+    zp = torch.cat([zp, torch.randn(B, 1, V, generator=g, device=dev) * 2], dim=1).to(torch.bfloat16).contiguous()
+    draft = torch.distributions.Categorical(logits=zq).sample().transpose(0, 1).to(torch.int32).contiguous()
+    ua = torch.rand(B, gamma, generator=g, device=dev)
+    ur = torch.rand(B, generator=g, device=dev)
+    for _ in range(warmup):
+        acc, _ = head.verify_sample(draft, zq, zp, ua, ur)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        acc, _ = head.verify_sample(draft, zq, zp, ua, ur)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    by = B * (gamma + 1) * V * 2 + gamma * B * V * 4 + 2 * B * V * (2 + 4)
+    return {"us_per_call": 1e3 * ms, "algorithmic_mb": by / 1e6, "gbs": by / (ms * 1e-3) / 1e9,
+            "frac_of_hbm_peak": by / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "mean_accept_len": float(acc.float().mean()),
+            "note": "156 MB of logits is close to L2 size: repeated calls partly hit L2"}
+
+
 def WL_vis(p: int, block: int, offset: int = 0) -> int:
     """Visible true keys of position p under the inverse block mask (flop accounting only)."""
     return p - 1 if p <= offset else offset + block * ((p - 1 - offset) // block)
@@ -580,6 +611,7 @@ def main():
     if not args.only_headline and world == 1:
         # batch-1 serving on the same head (Llama-3-8B shape) and on the Llama-2-7B shaped head
         others = {}
+        line["verify_sample"] = bench_verify_sample(head, w, steps=max(3, min(20, args.steps)), warmup=3, peaks=peaks)
         if w.name == HEADLINE:
             w3 = WL.WORKLOADS["c3_llama3_8b_b1"]
             scn3 = ServeScenario(head, w3, iters, device)

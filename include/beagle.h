@@ -157,6 +157,21 @@ beagle_status beagle_verify_greedy(beagle_ctx* ctx, int32_t batch, int32_t gamma
                                    int32_t logits_dtype, const int32_t* target_ids_dev,
                                    int32_t* accept_len_dev, int32_t* out_tokens_dev, void* stream);
 
+/* Acceptance under sampling (Section 3: each draft is accepted with probability min(1, p(t)/q(t)); at the
+ * first rejection j, or at j = gamma+1 when nothing was rejected, one token is drawn from the
+ * normalised max(0, p_j - q_j), from p_{gamma+1} in the latter case).  p = softmax(target / temperature),
+ * q = softmax(draft / temperature).  The random numbers are the caller's: u_accept_dev fp32 [batch, gamma]
+ * and u_resample_dev fp32 [batch], uniform in [0, 1); the extra token is the smallest id whose
+ * cumulative residual mass exceeds u_resample times the total.  draft_logits_dev: fp32
+ * [gamma, batch, V], one [batch, V] block per draft step as beagle_draft_step writes it;
+ * target_logits_dev: [batch, gamma+1, V], logits_dtype BEAGLE_FP32 or BEAGLE_BF16; logits are finite.
+ * accept_len_dev[b] = a; out_tokens_dev[b] = the a accepted drafts, the extra token, then -1
+ * ([batch, gamma+1]).  gamma <= 64, temperature > 0. */
+beagle_status beagle_verify_sample(beagle_ctx* ctx, int32_t batch, int32_t gamma, const int32_t* draft_tokens_dev,
+                                   const float* draft_logits_dev, const void* target_logits_dev, int32_t logits_dtype,
+                                   float temperature, const float* u_accept_dev, const float* u_resample_dev,
+                                   int32_t* accept_len_dev, int32_t* out_tokens_dev, void* stream);
+
 /* Greedy acceptance from target logits with NO memory handed over by the caller beyond the inputs
  * and outputs.  (The paper has no counterpart: this is a packaging variant of beagle_verify_greedy.)
  *

@@ -538,8 +538,8 @@ def verify_sample(draft_tokens: np.ndarray, draft_logits: np.ndarray, target_log
     """
     draft = np.asarray(draft_tokens, dtype=np.int64)
     B, gamma = draft.shape
-    ql = np.asarray(draft_logits, dtype=F64).reshape(gamma, B, -1)
     pl = np.asarray(target_logits, dtype=F64).reshape(B, gamma + 1, -1)
+    ql = np.asarray(draft_logits, dtype=F64).reshape(gamma, B, pl.shape[-1])
     ua = np.asarray(u_accept, dtype=F64).reshape(B, gamma)
     ur = np.asarray(u_resample, dtype=F64).reshape(B)
     accept = np.zeros(B, dtype=np.int64)

@@ -27,7 +27,7 @@ EXPORTED_SYMBOLS = (
     "beagle_block_workspace_bytes", "beagle_block_forward", "beagle_verify_greedy", "beagle_last_error",
     "beagle_launch_count", "beagle_profile_enable", "beagle_profile_read", "beagle_profile_stage_count",
     "beagle_profile_stage_name", "beagle_verify_greedy_static", "beagle_check_device",
-    "beagle_workspace_buffer", "beagle_block_workspace_buffer",
+    "beagle_workspace_buffer", "beagle_block_workspace_buffer", "beagle_verify_sample",
 )
 
 BUFFER_IDS = {"x": 0, "xn": 1, "q": 2, "o": 3, "y": 4, "yn": 5, "act": 6, "h": 7, "kt": 8, "vt": 9, "kp": 10, "vp": 11}
@@ -94,6 +94,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.beagle_workspace_buffer.restype = C.c_int
     lib.beagle_block_workspace_buffer.argtypes = [C.POINTER(BeagleConfig), i32, i32, i32, szp, i32p]
     lib.beagle_block_workspace_buffer.restype = C.c_int
+    lib.beagle_verify_sample.argtypes = [vp, i32, i32, vp, vp, vp, i32, C.c_float, vp, vp, vp, vp, vp]
+    lib.beagle_verify_sample.restype = C.c_int
     lib.beagle_check_device.argtypes = [vp, vp]
     lib.beagle_check_device.restype = C.c_int
     lib.beagle_launch_count.restype = C.c_int64
@@ -246,6 +248,24 @@ def beagle_verify_greedy(ctx: Context, draft_tokens: torch.Tensor, target_logits
                                            _ptr(target_ids), _ptr(accept_len), _ptr(out_tokens), _stream()))
 
 
+def beagle_verify_sample(ctx: Context, draft_tokens: torch.Tensor, draft_logits: torch.Tensor, target_logits: torch.Tensor,
+                         u_accept: torch.Tensor, u_resample: torch.Tensor, accept_len: torch.Tensor, out_tokens: torch.Tensor,
+                         temperature: float = 1.0) -> None:
+    """draft_logits: fp32 [gamma, batch, V]; target_logits: [batch, gamma+1, V] fp32 or bf16; uniforms fp32."""
+    batch, gamma = draft_tokens.shape
+    if draft_logits.dtype != torch.float32 or u_accept.dtype != torch.float32 or u_resample.dtype != torch.float32:
+        raise ValueError("draft_logits and the uniforms must be float32")
+    if target_logits.dtype == torch.bfloat16:
+        code = BEAGLE_BF16
+    elif target_logits.dtype == torch.float32:
+        code = BEAGLE_FP32
+    else:
+        raise ValueError("target_logits must be float32 or bfloat16")
+    ctx.check(ctx.lib.beagle_verify_sample(ctx.handle, batch, gamma, _ptr(draft_tokens), _ptr(draft_logits), _ptr(target_logits), code,
+                                           float(temperature), _ptr(u_accept), _ptr(u_resample), _ptr(accept_len), _ptr(out_tokens),
+                                           _stream()))
+
+
 def beagle_verify_greedy_static(draft_tokens: torch.Tensor, target_logits: torch.Tensor, accept_len: torch.Tensor,
                                 out_tokens: torch.Tensor) -> None:
     """Greedy acceptance for callers that may not allocate: no context, no workspace -- the
@@ -369,6 +389,13 @@ class BeagleHead:
         accept = torch.empty(B, dtype=torch.int32, device=self.device)
         out = torch.empty(B, gamma + 1, dtype=torch.int32, device=self.device)
         beagle_verify_greedy(self.ctx, draft_tokens, target_logits, target_ids, accept, out)
+        return accept, out
+
+    def verify_sample(self, draft_tokens, draft_logits, target_logits, u_accept, u_resample, temperature=1.0):
+        B, gamma = draft_tokens.shape
+        accept = torch.empty(B, dtype=torch.int32, device=self.device)
+        out = torch.empty(B, gamma + 1, dtype=torch.int32, device=self.device)
+        beagle_verify_sample(self.ctx, draft_tokens, draft_logits, target_logits, u_accept, u_resample, accept, out, temperature)
         return accept, out
 
     def slot_lengths(self, slot):

@@ -41,6 +41,7 @@ struct beagle_ctx {
     float* sk_partial = nullptr;    // fp32 split partials of the tensor-core serve projections
     int32_t *last_token, *ids;
     unsigned long long *lm_partials, *verify_keys;
+    void* vs_scratch = nullptr;     // log-sum-exp partials and chunk masses of beagle_verify_sample
     int* dev_error = nullptr;       // device word raised by a kernel whose bounded wait ran out
     bool dev_error_cleared = false;
     int lm_blocks = 0;
@@ -122,7 +123,7 @@ beagle_status check_config(const beagle_config* c) {
 }
 
 struct ServeLayout {
-    size_t x, xn, q, o, y, yn, act, h, h_slot, hs, attn, sk_partial, last_token, ids, lm_partials, verify_keys, dev_error, total;
+    size_t x, xn, q, o, y, yn, act, h, h_slot, hs, attn, sk_partial, last_token, ids, lm_partials, verify_keys, vs_scratch, dev_error, total;
     int lm_blocks;
 };
 ServeLayout serve_layout(const beagle_config& c) {
@@ -155,6 +156,7 @@ ServeLayout serve_layout(const beagle_config& c) {
     L.lm_blocks = gemv_grid_blocks(GEMV_LOGITS, c.vocab);
     L.lm_partials = take(B * (size_t)L.lm_blocks * sizeof(unsigned long long));
     L.verify_keys = take(B * 65 * kRowArgmaxSplit * sizeof(unsigned long long));
+    L.vs_scratch = take(verify_sample_scratch_bytes((int)B, 64));
     L.dev_error = take(256 + B * (size_t)c.n_kv_heads * sizeof(int32_t));     // error word, then the attention completion counters
     L.total = off;
     return L;
@@ -313,6 +315,7 @@ beagle_status beagle_create(const beagle_config* cfg, const beagle_weights* w, v
     c->ids = reinterpret_cast<int32_t*>(c->ws + L.ids);
     c->lm_partials = reinterpret_cast<unsigned long long*>(c->ws + L.lm_partials);
     c->verify_keys = reinterpret_cast<unsigned long long*>(c->ws + L.verify_keys);
+    c->vs_scratch = c->ws + L.vs_scratch;
     c->dev_error = reinterpret_cast<int*>(c->ws + L.dev_error);
     c->lm_blocks = L.lm_blocks;
     c->n_true.assign(cfg->max_slots, 0);
@@ -892,6 +895,26 @@ beagle_status beagle_verify_greedy(beagle_ctx* ctx, int32_t batch, int32_t gamma
     }
     ctx->launches += launch_accept(draft_tokens_dev, ids, batch, gamma, accept_len_dev, out_tokens_dev, stream);
     return cuda_ok(ctx, "verify_greedy");
+}
+
+beagle_status beagle_verify_sample(beagle_ctx* ctx, int32_t batch, int32_t gamma, const int32_t* draft_tokens_dev,
+                                   const float* draft_logits_dev, const void* target_logits_dev, int32_t logits_dtype,
+                                   float temperature, const float* u_accept_dev, const float* u_resample_dev,
+                                   int32_t* accept_len_dev, int32_t* out_tokens_dev, void* stream_) {
+    if (ctx == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    if (batch < 0 || batch > BEAGLE_MAX_CALL_BATCH) return fail(ctx, BEAGLE_ERR_CAPACITY, "batch %d outside [0, %d]", batch, BEAGLE_MAX_CALL_BATCH);
+    if (gamma < 0 || gamma > 64) return fail(ctx, BEAGLE_ERR_CAPACITY, "gamma %d outside [0, 64]", gamma);
+    if (!(temperature > 0.f)) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "verify_sample: temperature must be > 0");
+    if (batch == 0) return BEAGLE_OK;
+    if (target_logits_dev == nullptr || u_resample_dev == nullptr || accept_len_dev == nullptr || out_tokens_dev == nullptr ||
+        (gamma > 0 && (draft_tokens_dev == nullptr || draft_logits_dev == nullptr || u_accept_dev == nullptr)))
+        return fail(ctx, BEAGLE_ERR_INVALID_ARG, "verify_sample: NULL argument");
+    if (logits_dtype != BEAGLE_FP32 && logits_dtype != BEAGLE_BF16) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "verify_sample: unknown logits_dtype");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    StageTimer timer_(ctx, ST_VERIFY, stream);
+    ctx->launches += launch_verify_sample(logits_dtype, draft_tokens_dev, draft_logits_dev, target_logits_dev, batch, gamma, ctx->cfg.vocab,
+                                          temperature, u_accept_dev, u_resample_dev, ctx->vs_scratch, accept_len_dev, out_tokens_dev, stream);
+    return cuda_ok(ctx, "verify_sample");
 }
 
 }  // extern "C"

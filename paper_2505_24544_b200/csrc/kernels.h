@@ -68,6 +68,14 @@ int launch_row_argmax(int logits_dtype, const void* logits, int rows, int V, uns
 int launch_accept(const int32_t* draft, const int32_t* target_ids, int B, int gamma, int32_t* accept_len,
                   int32_t* out_tokens, cudaStream_t stream);
 
+// Acceptance under sampling (Section 3): min(1, p/q) tests with the uniforms u_accept [B, gamma], then one
+// token by inverse CDF (u_resample [B]) from the normalised max(0, p_j - q_j).  draft_logits fp32
+// [gamma, B, V]; target_logits [B, gamma+1, V] fp32 or bf16.
+size_t verify_sample_scratch_bytes(int max_batch, int max_gamma);
+int launch_verify_sample(int logits_dtype, const int32_t* draft, const float* draft_logits, const void* target_logits, int B, int gamma, int V,
+                         float temperature, const float* u_accept, const float* u_resample, void* scratch, int32_t* accept_len,
+                         int32_t* out_tokens, cudaStream_t stream);
+
 // ---- block path ------------------------------------------------------------------------------
 enum GemmEpilogue {
     GEMM_STORE = 0,      // C = A W^T                     (storage type)

@@ -190,6 +190,9 @@ def test_c3_c4_llama3_8b_full(llama3_heads):
     tok, logits, _ = gpu.draft_step(slots, tokens_in=to_dev(first.astype(np.int32), w.dtype), want_logits=True)
     greedy_tokens_are_argmax_of_logits(tok, logits)
     beagle_check_device(gpu.ctx)
+    # acceptance under sampling at the full vocabulary (32 x 7 x 128256 target logits)
+    from test_parity_gpu import check_verify_sample
+    check_verify_sample(gpu, w, WL.data_rng(w, 41), w.batch, w.gamma, "bf16", 1.0)
 
     # C3: batch 1, 4096 states, depth 8, on slot 0
     w3 = WL.WORKLOADS["c3_llama3_8b_b1"]

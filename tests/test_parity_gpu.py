@@ -224,6 +224,66 @@ def test_verify_greedy_logits_both_dtypes_and_ties():
     assert out_ref[4, 0] == 0 or acc_ref[4] >= 0
 
 
+def check_verify_sample(head_gpu, w, rng, batch, gamma, dt, temperature, logit_scale=2.0):
+    """beagle_verify_sample against the oracle.  Integer outputs are bit-exact wherever the oracle's
+    decision margins (|u - ratio| of the acceptance tests, distance of u_resample to a CDF
+    boundary) exceed what fp32 sums over the vocabulary can move; those are all but a few rows."""
+    V = w.vocab
+    zq = (rng.standard_normal((gamma, batch, V)) * logit_scale).astype(np.float32)
+    zp = WL.round_to_storage((zq.transpose(1, 0, 2)[:, :, :] * 0.7 + rng.standard_normal((batch, gamma, V)) * logit_scale * 0.7).reshape(-1), dt)
+    zp = np.concatenate([zp.reshape(batch, gamma, V), WL.round_to_storage((rng.standard_normal((batch, 1, V)) * logit_scale).reshape(-1), dt).reshape(batch, 1, V)], axis=1)
+    q = O.softmax_rows(zq, temperature)
+    draft = np.array([[rng.choice(V, p=q[i, b]) for i in range(gamma)] for b in range(batch)], dtype=np.int32).reshape(batch, gamma)
+    ua = rng.random((batch, gamma), dtype=np.float32)
+    ur = rng.random(batch, dtype=np.float32)
+    ref = O.verify_sample(draft, zq, zp, ua, ur, temperature)
+    acc, out = head_gpu.verify_sample(to_dev(draft, w.dtype), to_dev(zq, "fp32"), to_dev(zp, dt), to_dev(ua, "fp32"), to_dev(ur, "fp32"), temperature)
+    acc, out = acc.cpu().numpy(), out.cpu().numpy()
+    # acceptance tests: exact wherever u is not within 1e-4 of the ratio (fp32 log-sum-exp over V moves it by ~1e-6)
+    sure = ref["accept_margin"] > 1e-4
+    assert sure.mean() >= 0.9
+    np.testing.assert_array_equal(acc[sure], ref["accept_len"][sure])
+    p_all = O.softmax_rows(zp, temperature)
+    exact = 0
+    for b in range(batch):
+        a = int(acc[b])
+        # every row: a valid result shape (accepted drafts, one extra token, padding)
+        assert 0 <= a <= gamma and np.array_equal(out[b, :a], draft[b, :a]) and 0 <= out[b, a] < V and np.all(out[b, a + 1:] == -1)
+        if a != ref["accept_len"][b]:
+            continue
+        # the extra token: u_resample must fall into the token's interval of the oracle's fp64 CDF, up to the 2e-5 that
+        # an fp32 running sum over the vocabulary can be off (at V = 128256 the intervals themselves are ~1e-5 wide,
+        # so only this statement, not equality, is meaningful there); equal to the oracle's token when r is clear of a boundary
+        cdf = np.cumsum(O.residual_distribution(p_all[b, a], q[a, b] if a < gamma else None))
+        v = int(out[b, a])
+        lo = cdf[v - 1] if v > 0 else 0.0
+        assert lo - 2e-5 <= ur[b] <= cdf[v] + 2e-5, (b, v, lo, float(ur[b]), cdf[v])
+        if ref["resample_margin"][b] > 2e-5:
+            assert v == ref["out_tokens"][b, a]
+        exact += int(v == ref["out_tokens"][b, a])
+    assert exact >= 0.5 * batch
+    return ref
+
+
+@pytest.mark.parametrize("dt,temperature", [("fp32", 1.0), ("bf16", 0.7)])
+def test_verify_sample_small(dt, temperature):
+    w = SMALL_GQA.scaled(batch=24, gamma=5)
+    head_gpu, _, _ = build(w)
+    rng = WL.data_rng(w, 31)
+    ref = check_verify_sample(head_gpu, w, rng, 24, 5, dt, temperature)
+    assert 0 < ref["accept_len"].mean() < 5                      # both rejections and acceptances occur
+    check_verify_sample(head_gpu, w, rng, 3, 0, dt, temperature)  # gamma = 0: only the extra token, drawn from p_1
+    # p == q: everything is accepted and the extra token comes from p_{gamma+1}
+    z = rng.standard_normal((2, 4, w.vocab)).astype(np.float32)
+    draft = rng.integers(0, w.vocab, (4, 2)).astype(np.int32)
+    zp = np.concatenate([z.transpose(1, 0, 2), rng.standard_normal((4, 1, w.vocab)).astype(np.float32)], axis=1)
+    ua, ur = rng.random((4, 2), dtype=np.float32), rng.random(4, dtype=np.float32)
+    acc, out = head_gpu.verify_sample(to_dev(draft, w.dtype), to_dev(z, "fp32"), to_dev(zp, "fp32"), to_dev(ua, "fp32"), to_dev(ur, "fp32"))
+    ref = O.verify_sample(draft, z, zp, ua, ur)
+    assert acc.cpu().numpy().tolist() == [2, 2, 2, 2] == ref["accept_len"].tolist()
+    np.testing.assert_array_equal(out.cpu().numpy(), ref["out_tokens"])
+
+
 def test_status_codes_for_capacity_and_state():
     from paper_2505_24544_b200.binding import BeagleError
     w = SMALL_GQA.scaled(batch=1, gamma=2)
