@@ -33,4 +33,7 @@ from .beagle_oracle import (  # noqa: F401
     residual_distribution,
     inverse_cdf,
     verify_sample,
+    cross_entropy_rows,
+    loss_weights,
+    block_loss,
 )

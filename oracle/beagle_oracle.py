@@ -562,3 +562,66 @@ def verify_sample(draft_tokens: np.ndarray, draft_logits: np.ndarray, target_log
         dist = residual_distribution(p[a], q[a] if a < gamma else None)
         out[b, a], rm[b] = inverse_cdf(dist, ur[b])
     return {"accept_len": accept, "out_tokens": out, "accept_margin": am, "resample_margin": rm}
+
+
+# --------------------------------------------------------------------------- block-attention training losses (forward)
+
+def cross_entropy_rows(draft_logits: np.ndarray, target_logits: Optional[np.ndarray] = None,
+                       target_ids: Optional[np.ndarray] = None) -> np.ndarray:
+    """-E_{t ~ p}[log q(t)] per row, q = softmax(draft_logits); p = softmax(target_logits),
+    or the point mass at target_ids (exactly one of the two is given)."""
+    z = np.asarray(draft_logits, dtype=F64)
+    m = np.max(z, axis=-1, keepdims=True)
+    logq = z - (m + np.log(np.sum(np.exp(z - m), axis=-1, keepdims=True)))
+    if (target_logits is None) == (target_ids is None):
+        raise ValueError("give exactly one of target_logits / target_ids")
+    if target_ids is not None:
+        ids = np.asarray(target_ids, dtype=np.int64).reshape(-1)
+        return -logq[np.arange(logq.shape[0]), ids]
+    return -np.sum(softmax_rows(target_logits) * logq, axis=-1)
+
+
+def loss_weights(S: int, block: int, offset: int, sim_steps: int, stage: str) -> Tuple[np.ndarray, int]:
+    """Weight of every (1-based) position's loss term and the number of windows N.
+
+    Positions p <= offset lie in no window and carry no term.  In a window starting at n the
+    query at p = n + i is the i-step-ahead prediction.  'early' (Eq. 4): every window position
+    counts once.  'late' (Eq. 7 with l = i and beta*_{i,i} = k - i + 1): the slot-i prediction made
+    at simulation step i counts k - i + 1 times for i <= sim_steps and not at all beyond.
+    """
+    if stage not in ("early", "late"):
+        raise ValueError(stage)
+    w = np.zeros(S, dtype=F64)
+    for p in range(offset + 1, S + 1):
+        i = p - visible_true_count(p, block, offset)
+        if stage == "early":
+            w[p - 1] = 1.0
+        elif i <= sim_steps:
+            w[p - 1] = block - i + 1
+    n_windows = -(-(S - offset) // block)
+    return w, n_windows
+
+
+def block_loss(head: OracleHead, tokens: np.ndarray, hidden: np.ndarray, block: int, offset: int, stage: str,
+               sim_steps: int = 1, target_logits: Optional[np.ndarray] = None,
+               target_ids: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
+    """Early-stage (Eq. 4) or late-stage (Eq. 7) loss of a batch of sequences, forward only.
+
+    tokens [B, S], hidden [B, S, d]; the target model's distribution at position p (it predicts
+    token p+1, like the draft state at p, Eq. 1) is softmax(target_logits[b, p-1]) or the point
+    mass at target_ids[b, p-1].  Early stage: sim_steps must be 1.  Returns 'ce' [B, S] (every
+    position's cross-entropy from the block forward), 'weights' [S], 'n_windows' and
+    'loss' = sum_b sum_p weights[p] ce[b, p] / (B * n_windows).
+    """
+    tok = np.asarray(tokens, dtype=np.int64)
+    B, S = tok.shape
+    if stage == "early" and sim_steps != 1:
+        raise ValueError("the early-stage loss uses the plain inverse block mask (sim_steps = 1)")
+    w, n_windows = loss_weights(S, block, offset, sim_steps, stage)
+    ce = np.zeros((B, S), dtype=F64)
+    for b in range(B):
+        out = block_forward(head, tok[b], np.asarray(hidden)[b], block, offset, sim_steps)
+        ce[b] = cross_entropy_rows(out["logits"],
+                                   None if target_logits is None else np.asarray(target_logits)[b],
+                                   None if target_ids is None else np.asarray(target_ids)[b])
+    return {"ce": ce, "weights": w, "n_windows": n_windows, "loss": float(np.sum(ce * w[None, :]) / (B * n_windows))}

@@ -489,6 +489,60 @@ def test_verify_sample_acceptance_rate_matches_closed_form():
     np.testing.assert_allclose(h, p[gamma], atol=4 / np.sqrt(full.sum()))
 
 
+# ----------------------------------------------------------------------------- training losses (forward)
+
+def test_cross_entropy_closed_forms():
+    V = 7
+    # uniform draft: CE = log V whatever the target; equal distributions: CE = entropy
+    np.testing.assert_allclose(O.cross_entropy_rows(np.zeros((2, V)), target_ids=[3, 0]), np.log(V))
+    p = np.array([0.5, 0.25, 0.125, 0.125])
+    np.testing.assert_allclose(O.cross_entropy_rows(np.log(p)[None], target_logits=np.log(p)[None] + 5.0), [1.75 * np.log(2)])
+    # hand case: q = (1/4, 3/4), p = (1/2, 1/2): -(log 1/4 + log 3/4) / 2
+    np.testing.assert_allclose(O.cross_entropy_rows(np.array([[0.0, np.log(3.0)]]), target_logits=np.zeros((1, 2))),
+                               [-(np.log(0.25) + np.log(0.75)) / 2])
+    # a (nearly) one-hot soft target equals the hard label
+    z = np.random.default_rng(80).normal(size=(3, V))
+    hot = np.full((3, V), -60.0); hot[[0, 1, 2], [4, 0, 6]] = 60.0
+    np.testing.assert_allclose(O.cross_entropy_rows(z, target_logits=hot), O.cross_entropy_rows(z, target_ids=[4, 0, 6]), rtol=1e-12)
+    # Gibbs: CE(p, q) >= entropy(p)
+    t = np.random.default_rng(81).normal(size=(3, V))
+    pt = O.softmax_rows(t)
+    assert np.all(O.cross_entropy_rows(z, target_logits=t) >= -np.sum(pt * np.log(pt), axis=-1) - 1e-12)
+
+
+def test_loss_weights_follow_eq4_and_eq7():
+    # S = 11, k = 4, offset 2: windows start at 2, 6, 10 -> N = 3; slots of positions 3..11: 1 2 3 4 1 2 3 4 1
+    w, n = O.loss_weights(11, 4, 2, 1, "early")
+    assert n == 3 and w.tolist() == [0, 0] + [1] * 9
+    w, n = O.loss_weights(11, 4, 2, 4, "late")            # beta* = k - i + 1
+    assert w.tolist() == [0, 0, 4, 3, 2, 1, 4, 3, 2, 1, 4]
+    w, n = O.loss_weights(11, 4, 2, 2, "late")            # only two simulated steps: slots 3, 4 carry no term
+    assert w.tolist() == [0, 0, 4, 3, 0, 0, 4, 3, 0, 0, 4]
+    assert O.loss_weights(8, 4, 0, 1, "early")[1] == 2 and O.loss_weights(9, 4, 0, 1, "early")[1] == 3
+
+
+def test_block_loss_is_the_weighted_mean_of_block_forward_cross_entropies():
+    head, w, rng = small_head(seed=82)
+    B, S, k, off = 2, 13, 3, 1
+    tokens = rng.integers(0, head.cfg.vocab, (B, S))
+    hidden = rng.normal(size=(B, S, head.cfg.hidden))
+    tl = rng.normal(size=(B, S, head.cfg.vocab)) * 2
+    out = O.block_loss(head, tokens, hidden, k, off, "late", sim_steps=3, target_logits=tl)
+    ref = 0.0
+    for b in range(B):
+        lg = O.block_forward(head, tokens[b], hidden[b], k, off, 3)["logits"]
+        q = O.softmax_rows(lg); p = O.softmax_rows(tl[b])
+        for pos in range(off + 1, S + 1):
+            i = pos - O.visible_true_count(pos, k, off)
+            ref += (k - i + 1) * -(p[pos - 1] * np.log(q[pos - 1])).sum()
+    assert out["n_windows"] == 4
+    np.testing.assert_allclose(out["loss"], ref / (B * 4), rtol=1e-12)
+    early = O.block_loss(head, tokens, hidden, k, off, "early", target_ids=tokens)
+    assert early["ce"].shape == (B, S) and early["loss"] > 0
+    with pytest.raises(ValueError):
+        O.block_loss(head, tokens, hidden, k, off, "early", sim_steps=2, target_ids=tokens)
+
+
 # ----------------------------------------------------------------------------- storage mode
 
 def test_round_bf16_ties_to_even_and_matches_torch():
