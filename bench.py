@@ -456,7 +456,20 @@ def bench_block(head, w: WL.Workload, steps: int, warmup: int, peaks):
     st = {k: {"ms": v[0], "tflops": (flops[k] / (v[0] * 1e-3) / 1e12) if k in flops and v[0] > 0 else None} for k, v in stages.items()}
     lm = st.get("blk_lm_head", {})
     peak = peaks["bf16_tflops_sustained"]
+    # loss forward (Eq. 4, hard labels): the same forward with the cross-entropy epilogue instead of the arg-max one
+    labels = torch.randint(0, w.vocab, (w.batch, S), generator=g, device=dev, dtype=torch.int32)
+    loss = torch.empty(1, dtype=torch.float32, device=dev)
+    for _ in range(2):
+        B.beagle_block_loss(head.ctx, tokens, hidden, w.block, 0, 1, "early", None, labels, loss, None)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(steps):
+        B.beagle_block_loss(head.ctx, tokens, hidden, w.block, 0, 1, "early", None, labels, loss, None)
+    e1.record()
+    torch.cuda.synchronize()
+    loss_ms = e0.elapsed_time(e1) / steps
     return {
+        "loss_forward": {"ms": loss_ms, "tflops": total / (loss_ms * 1e-3) / 1e12, "loss": float(loss.item()), "stage": "early, hard labels"},
         "workload": w.name, "positions_per_s": M / (ms * 1e-3), "ms_per_forward": ms, "tflop_per_forward": total / 1e12,
         "tflops": total / (ms * 1e-3) / 1e12, "gpu_launches": launches, "stages": st,
         "roofline": {"bound": "tensor", "kernel": "blk_lm_head", "achieved": lm.get("tflops"), "peak": peak, "unit": "TFLOP/s",

@@ -146,6 +146,22 @@ beagle_status beagle_block_forward(beagle_ctx* ctx, int32_t batch, int32_t S, co
                                    float* logits_out_dev, int32_t* argmax_out_dev, void* hidden_out_dev,
                                    void* ws_dev, size_t ws_bytes, void* stream);
 
+/* Forward of the block-attention training losses (Section 4.2): the block forward above, followed by the
+ * cross-entropy -E_{t ~ p}[log q(t)] of every position, q = softmax of the draft logits at that position, p the
+ * target model's distribution there (it predicts the next token, like the draft state of Eq. 1): the softmax of
+ * target_logits_dev [batch, S, V] (logits_dtype BEAGLE_FP32 | BEAGLE_BF16) or the point mass at target_ids_dev
+ * int32 [batch, S]; exactly one of the two is non-NULL.  stage 0 = early loss (Eq. 4; sim_steps must be 1): every
+ * position inside a window counts once.  stage 1 = late loss (Eq. 7 with l = i and beta*_{i,i} = k - i + 1): the
+ * window-slot-i prediction counts block - i + 1 times for i <= sim_steps and not at all beyond.  Positions
+ * p <= offset lie in no window.  loss_out_dev fp32 [1] = sum of the weighted terms / (batch * windows), windows =
+ * ceil((S - offset) / block), summed in a fixed order; ce_out_dev fp32 [batch, S] (nullable) = every position's
+ * unweighted cross-entropy.  The logits are never materialised (bf16 configurations).  Workspace as for
+ * beagle_block_forward.  No gradients are computed. */
+beagle_status beagle_block_loss(beagle_ctx* ctx, int32_t batch, int32_t S, const int32_t* tokens_dev, const void* hidden_dev,
+                                int32_t block, int32_t offset, int32_t sim_steps, int32_t stage, const void* target_logits_dev,
+                                int32_t logits_dtype, const int32_t* target_ids_dev, float* loss_out_dev, float* ce_out_dev,
+                                void* ws_dev, size_t ws_bytes, void* stream);
+
 /* Greedy acceptance (Section 3: in greedy decoding the draft's and the target's top-1 tokens are
  * matched and only a contiguous prefix is accepted, plus one extra target token).  Exactly one of
  * target_logits_dev ([batch, gamma+1, V], logits_dtype BEAGLE_FP32 or BEAGLE_BF16) and

@@ -27,7 +27,7 @@ EXPORTED_SYMBOLS = (
     "beagle_block_workspace_bytes", "beagle_block_forward", "beagle_verify_greedy", "beagle_last_error",
     "beagle_launch_count", "beagle_profile_enable", "beagle_profile_read", "beagle_profile_stage_count",
     "beagle_profile_stage_name", "beagle_verify_greedy_static", "beagle_check_device",
-    "beagle_workspace_buffer", "beagle_block_workspace_buffer", "beagle_verify_sample",
+    "beagle_workspace_buffer", "beagle_block_workspace_buffer", "beagle_verify_sample", "beagle_block_loss",
 )
 
 BUFFER_IDS = {"x": 0, "xn": 1, "q": 2, "o": 3, "y": 4, "yn": 5, "act": 6, "h": 7, "kt": 8, "vt": 9, "kp": 10, "vp": 11}
@@ -94,6 +94,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.beagle_workspace_buffer.restype = C.c_int
     lib.beagle_block_workspace_buffer.argtypes = [C.POINTER(BeagleConfig), i32, i32, i32, szp, i32p]
     lib.beagle_block_workspace_buffer.restype = C.c_int
+    lib.beagle_block_loss.argtypes = [vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, i32, vp, vp, vp, vp, C.c_size_t, vp]
+    lib.beagle_block_loss.restype = C.c_int
     lib.beagle_verify_sample.argtypes = [vp, i32, i32, vp, vp, vp, i32, C.c_float, vp, vp, vp, vp, vp]
     lib.beagle_verify_sample.restype = C.c_int
     lib.beagle_check_device.argtypes = [vp, vp]
@@ -233,6 +235,26 @@ def beagle_block_forward(ctx: Context, tokens: torch.Tensor, hidden: torch.Tenso
     ctx.check(ctx.lib.beagle_block_forward(ctx.handle, batch, S, _ptr(tokens), _ptr(hidden), block, offset, sim_steps,
                                            _ptr(logits_out), _ptr(argmax_out), _ptr(hidden_out),
                                            ctx.block_ws.data_ptr(), ctx.block_ws.numel(), _stream()))
+
+
+def beagle_block_loss(ctx: Context, tokens: torch.Tensor, hidden: torch.Tensor, block: int, offset: int, sim_steps: int, stage: str,
+                      target_logits: Optional[torch.Tensor], target_ids: Optional[torch.Tensor], loss_out: torch.Tensor,
+                      ce_out: Optional[torch.Tensor]) -> None:
+    """stage: "early" (Eq. 4) or "late" (Eq. 7); loss_out fp32 [1]; ce_out fp32 [batch, S] or None."""
+    batch, S = tokens.shape
+    need = beagle_block_workspace_bytes(ctx, batch, S)
+    if ctx.block_ws is None or ctx.block_ws.numel() < need:
+        ctx.block_ws = None
+        ctx.block_ws = torch.empty(need, dtype=torch.uint8, device=tokens.device)
+    code = BEAGLE_FP32
+    if target_logits is not None:
+        if target_logits.dtype == torch.bfloat16:
+            code = BEAGLE_BF16
+        elif target_logits.dtype != torch.float32:
+            raise ValueError("target_logits must be float32 or bfloat16")
+    ctx.check(ctx.lib.beagle_block_loss(ctx.handle, batch, S, _ptr(tokens), _ptr(hidden), block, offset, sim_steps,
+                                        {"early": 0, "late": 1}[stage], _ptr(target_logits), code, _ptr(target_ids), _ptr(loss_out),
+                                        _ptr(ce_out), ctx.block_ws.data_ptr(), ctx.block_ws.numel(), _stream()))
 
 
 def beagle_verify_greedy(ctx: Context, draft_tokens: torch.Tensor, target_logits: Optional[torch.Tensor],
@@ -383,6 +405,13 @@ class BeagleHead:
         hid = torch.empty(B, S, self.cfg.hidden, dtype=self.dtype, device=self.device) if want_hidden else None
         beagle_block_forward(self.ctx, tokens, hidden, block, offset, sim_steps, logits, argmax, hid)
         return logits, argmax, hid
+
+    def block_loss(self, tokens, hidden, block, offset, stage, sim_steps=1, target_logits=None, target_ids=None):
+        B, S = tokens.shape
+        loss = torch.empty(1, dtype=torch.float32, device=self.device)
+        ce = torch.empty(B, S, dtype=torch.float32, device=self.device)
+        beagle_block_loss(self.ctx, tokens, hidden, block, offset, sim_steps, stage, target_logits, target_ids, loss, ce)
+        return loss, ce
 
     def verify_greedy(self, draft_tokens, target_logits=None, target_ids=None):
         B, gamma = draft_tokens.shape

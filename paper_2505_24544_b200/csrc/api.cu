@@ -163,7 +163,7 @@ ServeLayout serve_layout(const beagle_config& c) {
 }
 
 struct BlockLayout {
-    size_t x, xn, q, kt, vt, kp, vp, o, y, yn, act, h, logits, keys, ids, total;
+    size_t x, xn, q, kt, vt, kp, vp, o, y, yn, act, h, logits, keys, ids, ce_part, ce_rows, wce, total;
     int lm_chunk_rows;
 };
 constexpr int kLmChunkRows = 2048;
@@ -183,6 +183,9 @@ BlockLayout block_layout(const beagle_config& c, int batch, int S) {
     const size_t key_cols = (size_t)(tc_argmax_tiles(c.vocab) > kRowArgmaxSplit ? tc_argmax_tiles(c.vocab) : kRowArgmaxSplit);
     L.keys = take(M * key_cols * sizeof(unsigned long long));
     L.ids = take(M * sizeof(int32_t));
+    L.ce_part = take(M * (size_t)tc_argmax_tiles(c.vocab) * kCeFields * sizeof(float));     // loss forward: per (row, column tile)
+    L.ce_rows = take(M * sizeof(float));
+    L.wce = take(M * sizeof(float));
     L.total = off;
     return L;
 }
@@ -210,7 +213,7 @@ int dense_gemm(beagle_ctx* ctx, int epi, const GemmArgs& a, cudaStream_t stream)
         const int rc = tc_gemm(ctx->tc, epi, t, stream);
         if (rc >= 0) return rc;
     }
-    if (epi == GEMM_ARGMAX_KEYS) return -1;
+    if (epi == GEMM_ARGMAX_KEYS || epi == GEMM_CE) return -1;
     return launch_gemm_simt(ctx->cfg.dtype, epi, a, stream);
 }
 
@@ -744,10 +747,17 @@ beagle_status beagle_block_workspace_bytes(const beagle_config* cfg, int32_t bat
     return BEAGLE_OK;
 }
 
-beagle_status beagle_block_forward(beagle_ctx* ctx, int32_t batch, int32_t S, const int32_t* tokens_dev,
-                                   const void* hidden_dev, int32_t block, int32_t offset, int32_t sim_steps,
-                                   float* logits_out_dev, int32_t* argmax_out_dev, void* hidden_out_dev,
-                                   void* ws_dev, size_t ws_bytes, void* stream_) {
+struct LossSpec {                  // beagle_block_loss: what replaces the LM head's outputs
+    int stage;                     // 0 early (Eq. 4), 1 late (Eq. 7)
+    const void* tgt; int tgt_dtype;
+    const int32_t* labels;
+    float* loss_out; float* ce_out;
+};
+
+static beagle_status block_forward_impl(beagle_ctx* ctx, int32_t batch, int32_t S, const int32_t* tokens_dev,
+                                        const void* hidden_dev, int32_t block, int32_t offset, int32_t sim_steps,
+                                        float* logits_out_dev, int32_t* argmax_out_dev, void* hidden_out_dev,
+                                        void* ws_dev, size_t ws_bytes, void* stream_, const LossSpec* loss) {
     if (ctx == nullptr) return BEAGLE_ERR_INVALID_ARG;
     if (batch <= 0 || S <= 0 || tokens_dev == nullptr || hidden_dev == nullptr || ws_dev == nullptr)
         return fail(ctx, BEAGLE_ERR_INVALID_ARG, "block_forward: NULL or empty argument");
@@ -836,8 +846,38 @@ beagle_status beagle_block_forward(beagle_ctx* ctx, int32_t batch, int32_t S, co
         BEAGLE_GEMM(ST_BLK_DOWN, GEMM_RESID, g, "down projection");
     }
 
+    // loss forward: cross-entropy partials straight from the LM-head GEMM, merged, weighted and reduced
+    if (loss != nullptr) {
+        float* part = reinterpret_cast<float*>(ws + L.ce_part);
+        int ntiles = 1;
+        if (ctx->tc != nullptr) {
+            memset(&g, 0, sizeof(g));
+            g.M = M; g.A = H; g.lda = c.hidden; g.K = c.hidden; g.W = ctx->w.w_lm; g.N = c.vocab;
+            g.tgt = loss->tgt; g.tgt_dtype = loss->tgt_dtype; g.ldt = c.vocab; g.labels = loss->labels; g.ce_part = part;
+            BEAGLE_GEMM(ST_BLK_LM_HEAD, GEMM_CE, g, "LM head (loss)");
+            ntiles = tc_argmax_tiles(c.vocab);
+        } else {
+            float* chunk = reinterpret_cast<float*>(ws + L.logits);
+            const size_t trow = (size_t)c.vocab * (loss->tgt_dtype == BEAGLE_BF16 ? 2 : 4);
+            for (int r0 = 0; r0 < M; r0 += L.lm_chunk_rows) {
+                const int rows = M - r0 < L.lm_chunk_rows ? M - r0 : L.lm_chunk_rows;
+                memset(&g, 0, sizeof(g));
+                g.M = rows; g.A = static_cast<const char*>(H) + (size_t)r0 * c.hidden * ctx->elt; g.lda = c.hidden; g.K = c.hidden;
+                g.W = ctx->w.w_lm; g.N = c.vocab; g.C = chunk; g.ldc = c.vocab;
+                BEAGLE_GEMM(ST_BLK_LM_HEAD, GEMM_F32, g, "LM head");
+                ctx->launches += launch_row_ce(chunk, rows, c.vocab,
+                                               loss->tgt != nullptr ? static_cast<const char*>(loss->tgt) + (size_t)r0 * trow : nullptr,
+                                               loss->tgt_dtype, loss->labels != nullptr ? loss->labels + r0 : nullptr,
+                                               part + (size_t)r0 * kCeFields, stream);
+            }
+        }
+        StageTimer timer_(ctx, ST_BLK_ARGMAX, stream);
+        ctx->launches += launch_ce_finalize(part, ntiles, batch, S, block, offset, sim_steps, loss->stage,
+                                            reinterpret_cast<float*>(ws + L.ce_rows), reinterpret_cast<float*>(ws + L.wce), loss->ce_out,
+                                            loss->loss_out, stream);
+    }
     // LM head at every position
-    if (logits_out_dev != nullptr || argmax_out_dev != nullptr) {
+    if (loss == nullptr && (logits_out_dev != nullptr || argmax_out_dev != nullptr)) {
         unsigned long long* keys = reinterpret_cast<unsigned long long*>(ws + L.keys);
         int32_t* ids = argmax_out_dev != nullptr ? argmax_out_dev : reinterpret_cast<int32_t*>(ws + L.ids);
         if (logits_out_dev != nullptr) {
@@ -870,6 +910,33 @@ beagle_status beagle_block_forward(beagle_ctx* ctx, int32_t batch, int32_t S, co
     }
 #undef BEAGLE_GEMM
     return cuda_ok(ctx, "block_forward");
+}
+
+beagle_status beagle_block_forward(beagle_ctx* ctx, int32_t batch, int32_t S, const int32_t* tokens_dev,
+                                   const void* hidden_dev, int32_t block, int32_t offset, int32_t sim_steps,
+                                   float* logits_out_dev, int32_t* argmax_out_dev, void* hidden_out_dev,
+                                   void* ws_dev, size_t ws_bytes, void* stream_) {
+    return block_forward_impl(ctx, batch, S, tokens_dev, hidden_dev, block, offset, sim_steps, logits_out_dev, argmax_out_dev,
+                              hidden_out_dev, ws_dev, ws_bytes, stream_, nullptr);
+}
+
+beagle_status beagle_block_loss(beagle_ctx* ctx, int32_t batch, int32_t S, const int32_t* tokens_dev, const void* hidden_dev,
+                                int32_t block, int32_t offset, int32_t sim_steps, int32_t stage, const void* target_logits_dev,
+                                int32_t logits_dtype, const int32_t* target_ids_dev, float* loss_out_dev, float* ce_out_dev,
+                                void* ws_dev, size_t ws_bytes, void* stream_) {
+    if (ctx == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    if (stage != 0 && stage != 1) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "block_loss: stage must be 0 (early) or 1 (late)");
+    if (stage == 0 && sim_steps != 1) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "block_loss: the early-stage loss uses sim_steps = 1");
+    if ((target_logits_dev == nullptr) == (target_ids_dev == nullptr))
+        return fail(ctx, BEAGLE_ERR_INVALID_ARG, "block_loss: give exactly one of target_logits / target_ids");
+    if (target_logits_dev != nullptr && logits_dtype != BEAGLE_FP32 && logits_dtype != BEAGLE_BF16)
+        return fail(ctx, BEAGLE_ERR_INVALID_ARG, "block_loss: unknown logits_dtype");
+    if (loss_out_dev == nullptr) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "block_loss: loss_out is NULL");
+    LossSpec spec;
+    spec.stage = stage; spec.tgt = target_logits_dev; spec.tgt_dtype = target_logits_dev != nullptr ? logits_dtype : 0;
+    spec.labels = target_ids_dev; spec.loss_out = loss_out_dev; spec.ce_out = ce_out_dev;
+    return block_forward_impl(ctx, batch, S, tokens_dev, hidden_dev, block, offset, sim_steps, nullptr, nullptr, nullptr, ws_dev,
+                              ws_bytes, stream_, &spec);
 }
 
 beagle_status beagle_verify_greedy(beagle_ctx* ctx, int32_t batch, int32_t gamma, const int32_t* draft_tokens_dev,

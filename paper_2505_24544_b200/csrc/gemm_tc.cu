@@ -32,7 +32,7 @@ constexpr int kTcThreads = 192;
 
 // ---------------------------------------------------------------------------------------------- kernel
 enum TcEpilogue {
-    TC_STORE = 0, TC_RESID = 1, TC_SILU_MUL = 2, TC_F32 = 3, TC_KV_CACHE = 4, TC_ARGMAX = 5
+    TC_STORE = 0, TC_RESID = 1, TC_SILU_MUL = 2, TC_F32 = 3, TC_KV_CACHE = 4, TC_ARGMAX = 5, TC_CE = 6
 };
 
 struct TcArgs {
@@ -44,6 +44,7 @@ struct TcArgs {
     void* cache; int Hkv, dh, cap;
     SeqRows rows;
     unsigned long long* keys; int keys_ld;
+    const void* tgt; int tgt_dtype; int ldt; const int32_t* labels; float* ce_part;   // TC_CE
     int* error_word;
 };
 
@@ -193,6 +194,9 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
                     pos = args.rows.pos_start[b] + (m - args.rows.row_start[b]);
                 }
                 unsigned long long best = 0ull;
+                float ce_mq = -INFINITY, ce_sq = 0.f, ce_mt = -INFINITY, ce_st = 0.f, ce_dot = 0.f;   // TC_CE running partial
+                const int label = (EPI == TC_CE && args.tgt == nullptr && m < args.a_rows) ? args.labels[m] : -1;
+                if (EPI == TC_CE && args.tgt == nullptr) ce_mt = 0.f;
 #pragma unroll 1
                 for (int c0 = 0; c0 < BN; c0 += 16) {
                     uint32_t r[16], r2[16];
@@ -207,6 +211,41 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
 #pragma unroll
                         for (int j = 0; j < 16; ++j)
                             if (n0 + j < args.b_rows) { const unsigned long long k = argmax_key(__uint_as_float(r[j]), n0 + j); best = k > best ? k : best; }
+                    } else if (EPI == TC_CE) {
+                        const int nv = min(16, args.b_rows - n0);
+                        float cm = -INFINITY;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) if (j < nv) cm = fmaxf(cm, __uint_as_float(r[j]));
+                        if (cm > ce_mq) { ce_sq *= __expf(ce_mq - cm); ce_mq = cm; }
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) if (j < nv) ce_sq += __expf(__uint_as_float(r[j]) - ce_mq);
+                        if (args.tgt != nullptr) {
+                            float t[16];
+                            if (args.tgt_dtype == 0) {
+                                const float* tp = reinterpret_cast<const float*>(args.tgt) + (size_t)m * args.ldt + n0;
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) t[j] = j < nv ? tp[j] : -INFINITY;
+                            } else {
+                                const bf16* tp = reinterpret_cast<const bf16*>(args.tgt) + (size_t)m * args.ldt + n0;
+                                if (full && ((reinterpret_cast<uintptr_t>(tp) & 15) == 0)) {
+                                    unpack16<bf16>(*reinterpret_cast<const uint4*>(tp), t);
+                                    unpack16<bf16>(*reinterpret_cast<const uint4*>(tp + 8), t + 8);
+                                } else {
+#pragma unroll
+                                    for (int j = 0; j < 16; ++j) t[j] = j < nv ? __bfloat162float(tp[j]) : -INFINITY;
+                                }
+                            }
+                            float tm = -INFINITY;
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) if (j < nv) tm = fmaxf(tm, t[j]);
+                            if (tm > ce_mt) { const float f = __expf(ce_mt - tm); ce_st *= f; ce_dot *= f; ce_mt = tm; }
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                if (j < nv) { const float e = __expf(t[j] - ce_mt); ce_st += e; ce_dot = fmaf(e, __uint_as_float(r[j]), ce_dot); }
+                        } else if (label >= n0 && label < n0 + nv) {
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) if (n0 + j == label) { ce_dot = __uint_as_float(r[j]); ce_st = 1.f; }
+                        }
                     } else if (EPI == TC_F32) {
                         float* dst = reinterpret_cast<float*>(args.C) + (size_t)m * args.ldc + n0;
                         if (full && ((reinterpret_cast<uintptr_t>(dst) & 15) == 0)) {
@@ -265,6 +304,10 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
                     }
                 }
                 if (EPI == TC_ARGMAX && m < args.a_rows) args.keys[(size_t)m * args.keys_ld + tb] = best;
+                if (EPI == TC_CE && m < args.a_rows) {
+                    float* dst = args.ce_part + ((size_t)m * args.tiles_b + tb) * kCeFields;
+                    dst[0] = ce_mq; dst[1] = ce_sq; dst[2] = ce_mt; dst[3] = ce_st; dst[4] = ce_dot;
+                }
             }
             // this warp has read its quarter of the buffer: hand it back to the MMA issuer
             fence_before();
@@ -377,6 +420,7 @@ int tc_gemm(TcPlan* p, int epi, const GemmArgs& g, cudaStream_t stream) {
     a.C = g.C; a.ldc = g.ldc; a.R = g.R; a.ldr = g.ldr;
     a.cache = g.cache; a.Hkv = g.Hkv; a.dh = g.dh; a.cap = g.cap; a.rows = g.rows;
     a.keys = g.keys; a.keys_ld = a.tiles_b;
+    a.tgt = g.tgt; a.tgt_dtype = g.tgt_dtype; a.ldt = g.ldt; a.labels = g.labels; a.ce_part = g.ce_part;
     a.error_word = g.error_word;
     if (epi == GEMM_KV_CACHE && (g.dh % 16)) return -1;
     const int ntiles = a.tiles_a * a.tiles_b;
@@ -388,6 +432,7 @@ int tc_gemm(TcPlan* p, int epi, const GemmArgs& g, cudaStream_t stream) {
         case GEMM_F32: return launch_tc<256, false, TC_F32>(mapA, *mapB, *mapB, a, grid, stream);
         case GEMM_KV_CACHE: return launch_tc<256, false, TC_KV_CACHE>(mapA, *mapB, *mapB, a, grid, stream);
         case GEMM_ARGMAX_KEYS: return launch_tc<256, false, TC_ARGMAX>(mapA, *mapB, *mapB, a, grid, stream);
+        case GEMM_CE: return launch_tc<256, false, TC_CE>(mapA, *mapB, *mapB, a, grid, stream);
         default: return -1;
     }
 }

@@ -83,8 +83,13 @@ enum GemmEpilogue {
     GEMM_SILU_MUL = 2,   // C = SiLU(A W^T) * (A W2^T)
     GEMM_F32 = 3,        // C fp32
     GEMM_KV_CACHE = 4,   // scatter rows into the cache: row r -> (slot, pos) through SeqRows
-    GEMM_ARGMAX_KEYS = 5 // no C: one packed arg-max key per (row, column tile)   (tensor-core path only)
+    GEMM_ARGMAX_KEYS = 5,// no C: one packed arg-max key per (row, column tile)   (tensor-core path only)
+    GEMM_CE = 6          // no C: cross-entropy partials per (row, column tile)       (tensor-core path only)
 };
+// Cross-entropy partial of one (row, column range): running max / exp-sum of the draft logits z,
+// running max / exp-sum of the target logits t and sum exp(t - tmax) * z (soft targets); with hard
+// labels tmax = 0, tsum = 1 if the label lies in the range (else 0) and dot = z[label] (else 0).
+constexpr int kCeFields = 5;
 struct SeqRows {        // packed-row -> (slot, position) map of a prefill call
     int32_t n;
     int32_t slot[kMaxCallBatch];
@@ -99,10 +104,22 @@ struct GemmArgs {
     const void* R; int ldr;
     void* cache; int Hkv, dh, cap;  // GEMM_KV_CACHE
     unsigned long long* keys;       // GEMM_ARGMAX_KEYS
+    const void* tgt; int tgt_dtype; int ldt;   // GEMM_CE, soft targets: target logits [M, ldt] (0 fp32, 1 bf16)
+    const int32_t* labels;          // GEMM_CE, hard targets: [M] (used when tgt == NULL)
+    float* ce_part;                 // GEMM_CE: [M][column tiles][kCeFields]
     int* error_word;                // device word set to 1 when a bounded wait ran out
     SeqRows rows;
 };
 int launch_gemm_simt(int dtype, int epi, const GemmArgs& a, cudaStream_t stream);
+
+// ---- block-path losses (Eq. 4 / Eq. 7, forward) -------------------------------------------------
+// Cross-entropy partials (one column range = the whole row) from materialised fp32 draft logits.
+int launch_row_ce(const float* logits, int rows, int V, const void* tgt, int tgt_dtype, const int32_t* labels, float* ce_part,
+                  cudaStream_t stream);
+// ce[row] from the partials of `ntiles` column ranges, wce[row] = weight(position) * ce[row], then
+// loss = sum(wce) / (batch * windows), summed in a fixed order.  stage: 0 early, 1 late.
+int launch_ce_finalize(const float* ce_part, int ntiles, int batch, int S, int block, int offset, int sim_steps, int stage,
+                       float* ce_rows, float* wce, float* ce_out, float* loss_out, cudaStream_t stream);
 
 // Block-masked cross-attention: query row (b, p) reads true keys [0, n(p)) of Kt/Vt and, when
 // step > 1, predicted keys n(p) .. n(p)+min(slot, step)-2 of Kp/Vp.  All [B*S, H*dh] row-major.

@@ -251,4 +251,20 @@ def test_c5_block_forward_full_sampled_positions(llama2_heads, sim_steps):
     torch.cuda.synchronize()
     greedy_tokens_are_argmax_of_logits(argmax[0], logits[0])
     block_stage_parity(gpu, cpu, w, tokens[:1], hidden[:1], w.block, 0, sim_steps, 0, positions[:12], argmax_gpu=argmax, logits_gpu=logits)
+    # loss forward at full size (hard labels; the fused epilogue never writes the 2 GB of logits): per-position
+    # cross-entropy against the oracle's, computed from the library's own h of the same call, on sampled positions
+    from paper_2505_24544_b200.binding import beagle_block_workspace_buffer
+    labels = WL.make_tokens(w, rng, (B, S))
+    stage = "early" if sim_steps == 1 else "late"
+    loss, ce = gpu.block_loss(tok_dev, hid_dev, w.block, 0, stage, sim_steps=sim_steps, target_ids=to_dev(labels, w.dtype))
+    torch.cuda.synchronize()
+    h_all = beagle_block_workspace_buffer(gpu.ctx, "h", B, S)
+    rows = np.array([b * S + p - 1 for b in (0, B - 1) for p in positions])
+    z_ref = O.lm_head(cpu, h_all[torch.from_numpy(rows).cuda()].float().cpu().numpy().astype(np.float64))
+    ce_ref = O.cross_entropy_rows(z_ref, target_ids=labels.reshape(-1)[rows])
+    ce_np = ce.cpu().numpy().astype(np.float64)
+    np.testing.assert_allclose(ce_np.reshape(-1)[rows], ce_ref, rtol=1e-4, atol=1e-3)
+    wts, n_win = O.loss_weights(S, w.block, 0, sim_steps, stage)
+    own = float(np.sum(ce_np * wts[None, :]) / (B * n_win))
+    assert abs(float(loss.item()) - own) <= 1e-5 * abs(own)
     beagle_check_device(gpu.ctx)

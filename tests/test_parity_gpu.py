@@ -205,6 +205,38 @@ def test_block_forward_bf16_head_dim_128(S, block, offset, sim_steps):
     beagle_check_device(head_gpu.ctx)
 
 
+@pytest.mark.parametrize("name,stage,sim_steps,soft", [("c1", "early", 1, True), ("c1", "late", 3, False), ("gqa", "early", 1, False),
+                                                        ("gqa", "late", 4, True), ("mha", "late", 2, True)])
+def test_block_loss_forward(name, stage, sim_steps, soft):
+    """Early (Eq. 4) and late (Eq. 7) losses: every position's cross-entropy and the weighted mean
+    against the oracle.  c1 = fp32 (materialised logits), gqa / mha = bf16 (fused GEMM epilogue;
+    V = 4099 / 5000 leave a ragged last column tile)."""
+    w = {"c1": WL.WORKLOADS["c1_tiny_fp32"], "gqa": SMALL_GQA, "mha": SMALL_MHA}[name]
+    head_gpu, head_cpu, _ = build(w, max_slots=1, max_ctx=64)
+    rng = WL.data_rng(w, 500 + sim_steps)
+    B, S, block, offset = 2, 75, 4, 2
+    tokens = WL.make_tokens(w, rng, (B, S))
+    hidden = WL.make_hidden(w, rng, B * S).reshape(B, S, w.hidden)
+    tl = WL.round_to_storage((rng.standard_normal((B, S, w.vocab)) * 2).astype(np.float32).reshape(-1), w.dtype).reshape(B, S, w.vocab)
+    ids = WL.make_tokens(w, rng, (B, S))
+    kw = dict(target_logits=to_dev(tl, w.dtype)) if soft else dict(target_ids=to_dev(ids, w.dtype))
+    loss, ce = head_gpu.block_loss(to_dev(tokens, w.dtype), to_dev(hidden, w.dtype), block, offset, stage, sim_steps=sim_steps, **kw)
+    torch.cuda.synchronize()
+    ref = O.block_loss(head_cpu, tokens, hidden, block, offset, stage, sim_steps=sim_steps,
+                       **(dict(target_logits=tl) if soft else dict(target_ids=ids)))
+    ce = ce.cpu().numpy().astype(np.float64)
+    atol, rtol = (1e-4, 1e-4) if w.dtype == "fp32" else (3e-2, 1e-2)      # a cross-entropy moves by at most the largest logit error
+    err = np.abs(ce - ref["ce"])
+    assert np.all(err <= atol + rtol * np.abs(ref["ce"])), f"cross-entropy: max abs err {err.max():.3e}"
+    # the scalar is the weighted mean of the library's own per-position values (fixed-order fp32 sum) ...
+    own = float(np.sum(ce * ref["weights"][None, :]) / (B * ref["n_windows"]))
+    assert abs(float(loss.item()) - own) <= 1e-5 * abs(own)
+    # ... and agrees with the oracle's
+    assert abs(float(loss.item()) - ref["loss"]) <= (1e-4 if w.dtype == "fp32" else 1e-2) * abs(ref["loss"])
+    from paper_2505_24544_b200.binding import beagle_check_device
+    beagle_check_device(head_gpu.ctx)
+
+
 def test_verify_greedy_logits_both_dtypes_and_ties():
     w = SMALL_GQA.scaled(batch=5, gamma=6)
     head_gpu, _, _ = build(w)
