@@ -36,4 +36,8 @@ from .beagle_oracle import (  # noqa: F401
     cross_entropy_rows,
     loss_weights,
     block_loss,
+    log_softmax_rows,
+    top_k_lowest,
+    draft_tree,
+    verify_tree_greedy,
 )

@@ -625,3 +625,115 @@ def block_loss(head: OracleHead, tokens: np.ndarray, hidden: np.ndarray, block: 
                                    None if target_logits is None else np.asarray(target_logits)[b],
                                    None if target_ids is None else np.asarray(target_ids)[b])
     return {"ce": ce, "weights": w, "n_windows": n_windows, "loss": float(np.sum(ce * w[None, :]) / (B * n_windows))}
+
+
+# --------------------------------------------------------------------------- dynamic draft tree (EAGLE-2's method, which the paper adopts)
+
+def log_softmax_rows(logits: np.ndarray) -> np.ndarray:
+    z = np.asarray(logits, dtype=F64)
+    m = np.max(z, axis=-1, keepdims=True)
+    return z - (m + np.log(np.sum(np.exp(z - m), axis=-1, keepdims=True)))
+
+
+def top_k_lowest(values: np.ndarray, k: int) -> np.ndarray:
+    """Indices of the k largest values, largest first; equal values in index order."""
+    v = np.asarray(values, dtype=F64)
+    order = np.lexsort((np.arange(v.shape[0]), -v))
+    return order[:k]
+
+
+def draft_tree(head: OracleHead, seq: OracleSequence, root_token: int, depth: int, topk: int,
+               n_candidates: int) -> Dict[str, np.ndarray]:
+    """Dynamic draft tree over the true states cached in ``seq`` (the experimental setup's
+    "dynamic draft attention tree": depth = 1 + ``depth`` forwards, ``topk`` children per node,
+    ``n_candidates`` nodes handed to verification).
+
+    The root token is forwarded first; its ``topk`` most likely next tokens become the first
+    frontier, each scored by its log-probability.  ``depth`` times: every frontier node is forwarded
+    -- its query is its token's embedding, and it reads the true states plus the draft states of
+    the root and of its own ancestors (concatenation of newly generated states, Section 4.1) --
+    and proposes its ``topk`` children with score = own score + log-probability; the ``topk`` best
+    of all children form the next frontier.  Finally the ``n_candidates`` best nodes overall are
+    kept (a parent never scores below its child, so they form a tree).  Ties go to the smaller
+    token id / the earlier node.
+
+    Returns tokens [N], parents [N] (index into the returned arrays, -1 = child of the root),
+    scores [N], depths [N] (1 = child of the root), in creation order, and for every frontier
+    forward the rows it ran: 'forward_nodes' (list of arrays of node ids, in all-node numbering)
+    with 'all_tokens', 'all_parents', 'all_scores' of every node ever created.
+    """
+    c = head.cfg
+    k_true, v_true = seq.k_true, seq.v_true
+
+    def forward(tokens, state_lists):
+        kv = []
+        for states in state_lists:
+            if states:
+                k, v = project_kv(head, np.stack(states))
+                kv.append((np.concatenate([k_true, k]), np.concatenate([v_true, v])))
+            else:
+                kv.append((k_true, v_true))
+        return draft_block(head, tokens, kv)
+
+    out = forward([int(root_token)], [[]])
+    h_root = out["h"][0]
+    logq = log_softmax_rows(out["logits"][0])
+    first = top_k_lowest(logq, topk)
+    tok = [int(t) for t in first]
+    par = [-1] * topk
+    sc = [float(logq[t]) for t in first]
+    dep = [1] * topk
+    state_of: Dict[int, np.ndarray] = {}            # node id -> its draft state h (only forwarded nodes)
+    frontier = list(range(topk))
+    forwards = []
+    for _ in range(depth):
+        lists = []
+        for f in frontier:
+            chain = []
+            a = par[f]
+            while a >= 0:
+                chain.append(state_of[a])
+                a = par[a]
+            lists.append([h_root] + chain[::-1])
+        out = forward([tok[f] for f in frontier], lists)
+        forwards.append(np.asarray(frontier))
+        lq = log_softmax_rows(out["logits"])
+        base = len(tok)
+        for r, f in enumerate(frontier):
+            state_of[f] = out["h"][r]
+            for t in top_k_lowest(lq[r], topk):
+                tok.append(int(t)); par.append(f); sc.append(sc[f] + float(lq[r, t])); dep.append(dep[f] + 1)
+        new = np.arange(base, len(tok))
+        frontier = [int(new[i]) for i in top_k_lowest(np.asarray(sc)[new], topk)]
+    keep = np.sort(top_k_lowest(np.asarray(sc), min(n_candidates, len(tok))))
+    remap = {int(n): i for i, n in enumerate(keep)}
+    return {
+        "tokens": np.asarray([tok[n] for n in keep], dtype=np.int64),
+        "parents": np.asarray([remap[par[n]] if par[n] >= 0 else -1 for n in keep], dtype=np.int64),
+        "scores": np.asarray([sc[n] for n in keep], dtype=F64),
+        "depths": np.asarray([dep[n] for n in keep], dtype=np.int64),
+        "all_tokens": np.asarray(tok, dtype=np.int64), "all_parents": np.asarray(par, dtype=np.int64),
+        "all_scores": np.asarray(sc, dtype=F64), "forward_nodes": forwards, "kept_nodes": keep,
+    }
+
+
+def verify_tree_greedy(tokens: np.ndarray, parents: np.ndarray, target_root_id: int,
+                       target_ids: np.ndarray) -> Tuple[int, np.ndarray, np.ndarray]:
+    """Greedy acceptance on a draft tree (Section 3 applied along the tree's paths): starting at
+    the root, follow the child whose token equals the target's top-1 token at the current node
+    (``target_root_id`` at the root, ``target_ids[n]`` after node n); stop when no child matches
+    and emit the target's token there.  Returns (accept_len, emitted tokens, accepted node ids)."""
+    tokens = np.asarray(tokens, dtype=np.int64)
+    parents = np.asarray(parents, dtype=np.int64)
+    cur, want = -1, int(target_root_id)
+    path, out = [], []
+    while True:
+        nxt = [n for n in range(len(tokens)) if parents[n] == cur and tokens[n] == want]
+        if not nxt:
+            break
+        cur = nxt[0]
+        path.append(cur)
+        out.append(want)
+        want = int(np.asarray(target_ids)[cur])
+    out.append(want)
+    return len(path), np.asarray(out, dtype=np.int64), np.asarray(path, dtype=np.int64)

@@ -543,6 +543,84 @@ def test_block_loss_is_the_weighted_mean_of_block_forward_cross_entropies():
         O.block_loss(head, tokens, hidden, k, off, "early", sim_steps=2, target_ids=tokens)
 
 
+# ----------------------------------------------------------------------------- dynamic draft tree
+
+def _tree_fixture(seed=90, n=9):
+    head, w, rng = small_head(seed=seed)
+    seq = O.OracleSequence(head)
+    O.prefill_kv(head, seq, rng.normal(size=(n, head.cfg.hidden)))
+    return head, seq, rng
+
+
+def test_tree_with_one_child_per_node_is_chain_drafting():
+    """topk = 1: the tree is a path, and it is exactly the greedy chain of draft_step with concat."""
+    head, seq, rng = _tree_fixture()
+    tree = O.draft_tree(head, seq, root_token=7, depth=4, topk=1, n_candidates=10)
+    chain, lp = [], []
+    tok = [7]
+    for s in range(5):
+        out = O.draft_step(head, [seq], tokens_in=tok if s == 0 else None, concat=True)
+        chain.append(int(out["argmax"][0]))
+        lp.append(O.log_softmax_rows(out["logits"][0])[chain[-1]])
+    O.rollback(seq)
+    assert tree["tokens"].tolist() == chain and tree["parents"].tolist() == [-1, 0, 1, 2, 3]
+    np.testing.assert_allclose(tree["scores"], np.cumsum(lp), rtol=1e-12)
+
+
+def test_tree_scores_are_path_log_probabilities_and_selection_is_closed():
+    head, seq, rng = _tree_fixture(seed=91)
+    K, D, N = 3, 3, 14
+    tree = O.draft_tree(head, seq, root_token=11, depth=D, topk=K, n_candidates=N)
+    tok, par, sc = tree["tokens"], tree["parents"], tree["scores"]
+    assert len(tok) == N and len(tree["all_tokens"]) == K + D * K * K
+    assert np.all(par < np.arange(N)) and np.all(par[tree["depths"] == 1] == -1)
+    # every kept node's score is the sum of log q along its path, recomputed by forced chain drafting
+    for n in range(N):
+        path = []
+        a = n
+        while a >= 0:
+            path.append(int(tok[a])); a = int(par[a])
+        path = path[::-1]
+        total, feed = 0.0, 11
+        for t in path:
+            out = O.draft_step(head, [seq], tokens_in=[feed], concat=True)
+            total += O.log_softmax_rows(out["logits"][0])[t]
+            feed = t
+        O.rollback(seq)
+        np.testing.assert_allclose(sc[n], total, rtol=1e-10, atol=1e-10)
+        if par[n] >= 0:
+            assert sc[par[n]] >= sc[n]
+    # the kept set is the top-N of everything that was created, and siblings are distinct tokens
+    assert np.sort(tree["all_scores"])[::-1][N - 1] <= sc.min() + 1e-15
+    for p_ in set(par.tolist()):
+        sib = tok[par == p_]
+        assert len(set(sib.tolist())) == len(sib)
+    # each expansion level forwards the topk best children of the level before
+    a_sc, a_par = tree["all_scores"], tree["all_parents"]
+    level = np.arange(K, K + K * K)
+    np.testing.assert_array_equal(np.sort(tree["forward_nodes"][1]), np.sort(level[O.top_k_lowest(a_sc[level], K)]))
+
+
+def test_top_k_lowest_and_tree_verification_by_hand():
+    assert O.top_k_lowest(np.array([1.0, 3.0, 3.0, 2.0, 3.0]), 3).tolist() == [1, 2, 4]
+    np.testing.assert_allclose(np.exp(O.log_softmax_rows(np.array([[0.0, np.log(3.0)]]))), [[0.25, 0.75]])
+    #        root -> 0:'a'(5) -> 2:'c'(7) -> 4:'e'(9)
+    #             -> 1:'b'(6) -> 3:'d'(8)
+    tokens, parents = np.array([5, 6, 7, 8, 9]), np.array([-1, -1, 0, 1, 2])
+    # target wants 6 at the root, then 8 after node 1, then 4 after node 3: path (1, 3), three tokens emitted
+    a, out, path = O.verify_tree_greedy(tokens, parents, 6, np.array([0, 8, 0, 4, 0]))
+    assert a == 2 and out.tolist() == [6, 8, 4] and path.tolist() == [1, 3]
+    # nothing matches at the root: only the target's own token
+    a, out, path = O.verify_tree_greedy(tokens, parents, 1, np.array([0, 8, 0, 4, 0]))
+    assert a == 0 and out.tolist() == [1] and path.tolist() == []
+    # a match that is not a child of the current node does not count (7 is a child of node 0, not of the root)
+    a, out, _ = O.verify_tree_greedy(tokens, parents, 7, np.zeros(5, dtype=int))
+    assert a == 0 and out.tolist() == [7]
+    # lossless: the emitted tokens are exactly the target's greedy tokens along the accepted path
+    a, out, path = O.verify_tree_greedy(tokens, parents, 5, np.array([7, 0, 9, 0, 2]))
+    assert a == 3 and out.tolist() == [5, 7, 9, 2] and path.tolist() == [0, 2, 4]
+
+
 # ----------------------------------------------------------------------------- storage mode
 
 def test_round_bf16_ties_to_even_and_matches_torch():
