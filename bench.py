@@ -509,6 +509,36 @@ def bench_verify_sample(head, w: WL.Workload, steps: int, warmup: int, peaks):
             "note": "156 MB of logits is close to L2 size: repeated calls partly hit L2"}
 
 
+def bench_draft_tree(head, w: WL.Workload, scn, steps: int, warmup: int, peaks):
+    """Dynamic draft tree at the paper's setting (depth 1 + 6, top-10, 60 candidates) on one sequence
+    of the batch-1 workload: 7 forwards of 1 / 10 rows, each streaming the head's weights once."""
+    import torch
+    from paper_2505_24544_b200 import binding as B
+    depth, topk, n_cand = 6, 10, 60
+    scn.reset()
+    root = scn.first_tokens[0, :1].contiguous()
+    tok = torch.empty(n_cand, dtype=torch.int32, device=head.device)
+    par = torch.empty_like(tok)
+    sc = torch.empty(n_cand, dtype=torch.float32, device=head.device)
+    for _ in range(warmup):
+        B.beagle_draft_tree(head.ctx, 0, root, depth, topk, n_cand, tok, par, sc)
+    torch.cuda.synchronize()
+    l0 = head.launch_count
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        B.beagle_draft_tree(head.ctx, 0, root, depth, topk, n_cand, tok, par, sc)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    e, d, qd, kd, m, V = elt(w), w.hidden, w.n_q_heads * w.head_dim, w.n_kv_heads * w.head_dim, w.mlp_dim, w.vocab
+    weights = e * (2 * d * qd + 2 * d * kd + 3 * d * m + V * d)
+    gb = (depth + 1) * weights / 1e9
+    return {"ms_per_tree": ms, "candidates_per_s": n_cand / (ms * 1e-3), "depth": depth, "topk": topk, "candidates": n_cand,
+            "algorithmic_gb_per_tree": gb, "achieved_gbs": gb / (ms * 1e-3), "frac_of_hbm_peak": gb / (ms * 1e-3) / peaks["hbm_gbs"],
+            "gpu_launches": (head.launch_count - l0) // steps}
+
+
 def WL_vis(p: int, block: int, offset: int = 0) -> int:
     """Visible true keys of position p under the inverse block mask (flop accounting only)."""
     return p - 1 if p <= offset else offset + block * ((p - 1 - offset) // block)
@@ -571,7 +601,7 @@ def main():
     w = WL.WORKLOADS[args.workload]
     iters = args.steps + args.warmup
     extra = iters * (w.gamma + 1) + 64
-    max_draft = max(x.gamma for x in WL.WORKLOADS.values())
+    max_draft = 64          # chain depth <= 8; the draft tree (depth 6, top-10) keeps 51 draft states
     weights = WL.make_weights(w)
     head = BeagleHead.from_workload(w, weights, device=device, max_slots=w.batch, max_ctx=w.ctx_max + extra, max_draft=max_draft)
     del weights
@@ -632,6 +662,7 @@ def main():
             ms3, l3 = time_serve(scn3, args.steps, args.warmup, 1)
             st3 = profile_serve(scn3, args.steps, args.warmup)
             others[w3.name] = summarize_b1(w3, scn3, ms3, l3, st3, args, peaks)
+            line["draft_tree"] = bench_draft_tree(head, w3, scn3, steps=max(3, min(20, args.steps)), warmup=3, peaks=peaks)
             del scn3
         del scn
         head.ctx.close()

@@ -188,6 +188,32 @@ beagle_status beagle_verify_sample(beagle_ctx* ctx, int32_t batch, int32_t gamma
                                    float temperature, const float* u_accept_dev, const float* u_resample_dev,
                                    int32_t* accept_len_dev, int32_t* out_tokens_dev, void* stream);
 
+/* Dynamic draft tree for one sequence (the "dynamic draft attention tree" of the experimental setup, i.e. the
+ * method of EAGLE-2 with depth = 1 + `depth`, `topk` children per node and `n_candidates` nodes kept; the paper's
+ * runs use 6, 10 and 60).  The root token *root_token_dev (the target's last token) is forwarded over the slot's true
+ * states; its topk most likely next tokens become the first frontier, each scored by its log-probability.  `depth`
+ * times every frontier node is forwarded -- it reads the true states plus the draft states of the root and of its own
+ * ancestors, which are projected into the cache tail as in beagle_draft_step with concat -- and proposes its topk
+ * children with score = own score + log-probability; the topk best of all children form the next frontier.  Finally
+ * the n_candidates best nodes overall are written in creation order: tree_tokens_dev int32 [n_candidates],
+ * tree_parents_dev int32 (index into the same arrays, -1 = child of the root), tree_scores_dev fp32.  Equal values
+ * are ordered by the smaller token id / the earlier node.  The whole tree is drafted without a host synchronisation.
+ * Limits: topk <= 16, depth <= 8, n_candidates <= 64 and <= topk + depth*topk^2; 1 + (depth-1)*topk <= max_draft;
+ * bf16 configurations with head_dim 64 or 128.  Any chain-draft tail of the slot is dropped first; afterwards the
+ * slot holds true states only (call beagle_prefill_kv with the accepted states as usual). */
+beagle_status beagle_draft_tree(beagle_ctx* ctx, int32_t slot, const int32_t* root_token_dev, int32_t depth, int32_t topk,
+                                int32_t n_candidates, int32_t* tree_tokens_dev, int32_t* tree_parents_dev, float* tree_scores_dev,
+                                void* stream);
+
+/* Greedy acceptance on a draft tree (Section 3 applied along the tree's paths): target_ids_dev int32 [n_nodes + 1]
+ * holds the target's top-1 token at the root ([0]) and after every node n ([1 + n]).  Starting at the root the child
+ * whose token equals the target's token at the current node is followed; where none matches the walk stops and the
+ * target's token there is emitted.  accept_len_dev[0] = nodes accepted; out_tokens_dev int32 [out_cap] = the emitted
+ * tokens then -1 (out_cap >= depth + 2 holds every case); path_dev int32 [out_cap] (nullable) = the accepted nodes. */
+beagle_status beagle_verify_tree_greedy(beagle_ctx* ctx, int32_t n_nodes, const int32_t* tree_tokens_dev, const int32_t* tree_parents_dev,
+                                        const int32_t* target_ids_dev, int32_t out_cap, int32_t* accept_len_dev, int32_t* out_tokens_dev,
+                                        int32_t* path_dev, void* stream);
+
 /* Greedy acceptance from target logits with NO memory handed over by the caller beyond the inputs
  * and outputs.  (The paper has no counterpart: this is a packaging variant of beagle_verify_greedy.)
  *

@@ -660,10 +660,18 @@ def draft_tree(head: OracleHead, seq: OracleSequence, root_token: int, depth: in
     Returns tokens [N], parents [N] (index into the returned arrays, -1 = child of the root),
     scores [N], depths [N] (1 = child of the root), in creation order, and for every frontier
     forward the rows it ran: 'forward_nodes' (list of arrays of node ids, in all-node numbering)
-    with 'all_tokens', 'all_parents', 'all_scores' of every node ever created.
+    with 'all_tokens', 'all_parents', 'all_scores' of every node ever created.  'cut_margin' is the
+    smallest score gap across any of the selections made (k-th against (k+1)-th child, frontier,
+    final n-th against (n+1)-th): below it another floating-point precision may select otherwise.
     """
     c = head.cfg
     k_true, v_true = seq.k_true, seq.v_true
+    margin = [np.inf]
+
+    def cut(values, k):
+        v = np.sort(np.asarray(values, dtype=F64))[::-1]
+        if k < len(v):
+            margin[0] = min(margin[0], float(v[k - 1] - v[k]))
 
     def forward(tokens, state_lists):
         kv = []
@@ -678,6 +686,7 @@ def draft_tree(head: OracleHead, seq: OracleSequence, root_token: int, depth: in
     out = forward([int(root_token)], [[]])
     h_root = out["h"][0]
     logq = log_softmax_rows(out["logits"][0])
+    cut(logq, topk)
     first = top_k_lowest(logq, topk)
     tok = [int(t) for t in first]
     par = [-1] * topk
@@ -701,10 +710,13 @@ def draft_tree(head: OracleHead, seq: OracleSequence, root_token: int, depth: in
         base = len(tok)
         for r, f in enumerate(frontier):
             state_of[f] = out["h"][r]
+            cut(lq[r], topk)
             for t in top_k_lowest(lq[r], topk):
                 tok.append(int(t)); par.append(f); sc.append(sc[f] + float(lq[r, t])); dep.append(dep[f] + 1)
         new = np.arange(base, len(tok))
+        cut(np.asarray(sc)[new], topk)
         frontier = [int(new[i]) for i in top_k_lowest(np.asarray(sc)[new], topk)]
+    cut(sc, min(n_candidates, len(tok)))
     keep = np.sort(top_k_lowest(np.asarray(sc), min(n_candidates, len(tok))))
     remap = {int(n): i for i, n in enumerate(keep)}
     return {
@@ -713,7 +725,7 @@ def draft_tree(head: OracleHead, seq: OracleSequence, root_token: int, depth: in
         "scores": np.asarray([sc[n] for n in keep], dtype=F64),
         "depths": np.asarray([dep[n] for n in keep], dtype=np.int64),
         "all_tokens": np.asarray(tok, dtype=np.int64), "all_parents": np.asarray(par, dtype=np.int64),
-        "all_scores": np.asarray(sc, dtype=F64), "forward_nodes": forwards, "kept_nodes": keep,
+        "all_scores": np.asarray(sc, dtype=F64), "forward_nodes": forwards, "kept_nodes": keep, "cut_margin": margin[0],
     }
 
 

@@ -27,7 +27,7 @@ EXPORTED_SYMBOLS = (
     "beagle_block_workspace_bytes", "beagle_block_forward", "beagle_verify_greedy", "beagle_last_error",
     "beagle_launch_count", "beagle_profile_enable", "beagle_profile_read", "beagle_profile_stage_count",
     "beagle_profile_stage_name", "beagle_verify_greedy_static", "beagle_check_device",
-    "beagle_workspace_buffer", "beagle_block_workspace_buffer", "beagle_verify_sample", "beagle_block_loss",
+    "beagle_workspace_buffer", "beagle_block_workspace_buffer", "beagle_verify_sample", "beagle_block_loss", "beagle_draft_tree", "beagle_verify_tree_greedy",
 )
 
 BUFFER_IDS = {"x": 0, "xn": 1, "q": 2, "o": 3, "y": 4, "yn": 5, "act": 6, "h": 7, "kt": 8, "vt": 9, "kp": 10, "vp": 11}
@@ -96,6 +96,10 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.beagle_block_workspace_buffer.restype = C.c_int
     lib.beagle_block_loss.argtypes = [vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, i32, vp, vp, vp, vp, C.c_size_t, vp]
     lib.beagle_block_loss.restype = C.c_int
+    lib.beagle_draft_tree.argtypes = [vp, i32, vp, i32, i32, i32, vp, vp, vp, vp]
+    lib.beagle_draft_tree.restype = C.c_int
+    lib.beagle_verify_tree_greedy.argtypes = [vp, i32, vp, vp, vp, i32, vp, vp, vp, vp]
+    lib.beagle_verify_tree_greedy.restype = C.c_int
     lib.beagle_verify_sample.argtypes = [vp, i32, i32, vp, vp, vp, i32, C.c_float, vp, vp, vp, vp, vp]
     lib.beagle_verify_sample.restype = C.c_int
     lib.beagle_check_device.argtypes = [vp, vp]
@@ -288,6 +292,18 @@ def beagle_verify_sample(ctx: Context, draft_tokens: torch.Tensor, draft_logits:
                                            _stream()))
 
 
+def beagle_draft_tree(ctx: Context, slot: int, root_token: torch.Tensor, depth: int, topk: int, n_candidates: int,
+                      tree_tokens: torch.Tensor, tree_parents: torch.Tensor, tree_scores: torch.Tensor) -> None:
+    ctx.check(ctx.lib.beagle_draft_tree(ctx.handle, int(slot), _ptr(root_token), depth, topk, n_candidates, _ptr(tree_tokens),
+                                        _ptr(tree_parents), _ptr(tree_scores), _stream()))
+
+
+def beagle_verify_tree_greedy(ctx: Context, tree_tokens: torch.Tensor, tree_parents: torch.Tensor, target_ids: torch.Tensor,
+                              accept_len: torch.Tensor, out_tokens: torch.Tensor, path: Optional[torch.Tensor] = None) -> None:
+    ctx.check(ctx.lib.beagle_verify_tree_greedy(ctx.handle, tree_tokens.numel(), _ptr(tree_tokens), _ptr(tree_parents), _ptr(target_ids),
+                                                out_tokens.numel(), _ptr(accept_len), _ptr(out_tokens), _ptr(path), _stream()))
+
+
 def beagle_verify_greedy_static(draft_tokens: torch.Tensor, target_logits: torch.Tensor, accept_len: torch.Tensor,
                                 out_tokens: torch.Tensor) -> None:
     """Greedy acceptance for callers that may not allocate: no context, no workspace -- the
@@ -426,6 +442,20 @@ class BeagleHead:
         out = torch.empty(B, gamma + 1, dtype=torch.int32, device=self.device)
         beagle_verify_sample(self.ctx, draft_tokens, draft_logits, target_logits, u_accept, u_resample, accept, out, temperature)
         return accept, out
+
+    def draft_tree(self, slot, root_token, depth, topk, n_candidates):
+        tok = torch.empty(n_candidates, dtype=torch.int32, device=self.device)
+        par = torch.empty(n_candidates, dtype=torch.int32, device=self.device)
+        sc = torch.empty(n_candidates, dtype=torch.float32, device=self.device)
+        beagle_draft_tree(self.ctx, slot, root_token, depth, topk, n_candidates, tok, par, sc)
+        return tok, par, sc
+
+    def verify_tree_greedy(self, tree_tokens, tree_parents, target_ids, out_cap):
+        acc = torch.empty(1, dtype=torch.int32, device=self.device)
+        out = torch.empty(out_cap, dtype=torch.int32, device=self.device)
+        path = torch.empty(out_cap, dtype=torch.int32, device=self.device)
+        beagle_verify_tree_greedy(self.ctx, tree_tokens, tree_parents, target_ids, acc, out, path)
+        return acc, out, path
 
     def slot_lengths(self, slot):
         return beagle_slot_lengths(self.ctx, slot)

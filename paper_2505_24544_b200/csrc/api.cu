@@ -42,6 +42,8 @@ struct beagle_ctx {
     int32_t *last_token, *ids;
     unsigned long long *lm_partials, *verify_keys;
     void* vs_scratch = nullptr;     // log-sum-exp partials and chunk masses of beagle_verify_sample
+    void* tree_mem = nullptr;       // node / frontier arrays of beagle_draft_tree
+    float* tree_logits = nullptr;   // [kTreeMaxTopk, V] logits of the frontier rows
     int* dev_error = nullptr;       // device word raised by a kernel whose bounded wait ran out
     bool dev_error_cleared = false;
     int lm_blocks = 0;
@@ -123,7 +125,7 @@ beagle_status check_config(const beagle_config* c) {
 }
 
 struct ServeLayout {
-    size_t x, xn, q, o, y, yn, act, h, h_slot, hs, attn, sk_partial, last_token, ids, lm_partials, verify_keys, vs_scratch, dev_error, total;
+    size_t x, xn, q, o, y, yn, act, h, h_slot, hs, attn, sk_partial, last_token, ids, lm_partials, verify_keys, vs_scratch, tree_mem, tree_logits, dev_error, total;
     int lm_blocks;
 };
 ServeLayout serve_layout(const beagle_config& c) {
@@ -157,6 +159,8 @@ ServeLayout serve_layout(const beagle_config& c) {
     L.lm_partials = take(B * (size_t)L.lm_blocks * sizeof(unsigned long long));
     L.verify_keys = take(B * 65 * kRowArgmaxSplit * sizeof(unsigned long long));
     L.vs_scratch = take(verify_sample_scratch_bytes((int)B, 64));
+    L.tree_mem = take(tree_arrays_bytes(c.vocab));
+    L.tree_logits = take(c.dtype == BEAGLE_BF16 ? (size_t)kTreeMaxTopk * c.vocab * sizeof(float) : 0);
     L.dev_error = take(256 + B * (size_t)c.n_kv_heads * sizeof(int32_t));     // error word, then the attention completion counters
     L.total = off;
     return L;
@@ -319,6 +323,8 @@ beagle_status beagle_create(const beagle_config* cfg, const beagle_weights* w, v
     c->lm_partials = reinterpret_cast<unsigned long long*>(c->ws + L.lm_partials);
     c->verify_keys = reinterpret_cast<unsigned long long*>(c->ws + L.verify_keys);
     c->vs_scratch = c->ws + L.vs_scratch;
+    c->tree_mem = c->ws + L.tree_mem;
+    c->tree_logits = reinterpret_cast<float*>(c->ws + L.tree_logits);
     c->dev_error = reinterpret_cast<int*>(c->ws + L.dev_error);
     c->lm_blocks = L.lm_blocks;
     c->n_true.assign(cfg->max_slots, 0);
@@ -982,6 +988,139 @@ beagle_status beagle_verify_sample(beagle_ctx* ctx, int32_t batch, int32_t gamma
     ctx->launches += launch_verify_sample(logits_dtype, draft_tokens_dev, draft_logits_dev, target_logits_dev, batch, gamma, ctx->cfg.vocab,
                                           temperature, u_accept_dev, u_resample_dev, ctx->vs_scratch, accept_len_dev, out_tokens_dev, stream);
     return cuda_ok(ctx, "verify_sample");
+}
+
+beagle_status beagle_draft_tree(beagle_ctx* ctx, int32_t slot, const int32_t* root_token_dev, int32_t depth, int32_t topk,
+                                int32_t n_candidates, int32_t* tree_tokens_dev, int32_t* tree_parents_dev, float* tree_scores_dev,
+                                void* stream_) {
+    if (ctx == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    const beagle_config& c = ctx->cfg;
+    if (slot < 0 || slot >= c.max_slots) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "slot %d out of range", slot);
+    if (root_token_dev == nullptr || tree_tokens_dev == nullptr || tree_parents_dev == nullptr || tree_scores_dev == nullptr)
+        return fail(ctx, BEAGLE_ERR_INVALID_ARG, "draft_tree: NULL argument");
+    if (depth < 0 || depth > kTreeMaxDepth || topk < 1 || topk > kTreeMaxTopk || topk > c.vocab)
+        return fail(ctx, BEAGLE_ERR_CAPACITY, "draft_tree: need 0 <= depth <= %d and 1 <= topk <= %d", kTreeMaxDepth, kTreeMaxTopk);
+    const int total = topk + depth * topk * topk;
+    if (n_candidates < 1 || n_candidates > kTreeMaxCandidates || n_candidates > total)
+        return fail(ctx, BEAGLE_ERR_CAPACITY, "draft_tree: n_candidates must be in [1, min(%d, %d)]", kTreeMaxCandidates, total);
+    if (ctx->tc == nullptr || (c.head_dim != 64 && c.head_dim != 128))
+        return fail(ctx, BEAGLE_ERR_UNSUPPORTED, "draft_tree: needs the bf16 tensor-core path with head_dim 64 or 128");
+    const int tail = depth > 0 ? 1 + (depth - 1) * topk : 0;          // draft states that enter the cache
+    if (tail > c.max_draft) return fail(ctx, BEAGLE_ERR_CAPACITY, "draft_tree: %d draft states exceed max_draft %d", tail, c.max_draft);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    clear_error_word_once(ctx, stream);
+    const TreeArrays T = tree_arrays_carve(ctx->tree_mem, c.vocab);
+    const int n_true = ctx->n_true[slot];
+    // the tree starts from the true states: whatever chain-draft tail the slot had is dropped
+    ctx->n_draft[slot] = 0; ctx->pending[slot] = 0; ctx->has_token[slot] = 0;
+    const int dt = c.dtype;
+    int rc = 0;
+#define BEAGLE_TREE_SKINNY(MODE, ARGS, WHAT)                                              \
+    do {                                                                                  \
+        ARGS.partial = ctx->sk_partial;                                                   \
+        ARGS.error_word = ctx->dev_error;                                                 \
+        rc = tc_skinny(ctx->tc, MODE, ARGS, stream);                                      \
+        if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, WHAT ": unsupported shape");      \
+        ctx->launches += rc;                                                              \
+    } while (0)
+
+    for (int e = 0; e <= depth; ++e) {
+        const int rows = e == 0 ? 1 : topk;                           // forward 0: the root; forward e: the frontier of level e
+        const int nanc = e;                                           // ancestor states a row reads: the root's + e - 1 of its own line
+        BatchMeta meta;
+        memset(&meta, 0, sizeof(meta));
+        RowMap slots, pos;
+        for (int b = 0; b < kMaxCallBatch; ++b) { slots.idx[b] = slot; pos.idx[b] = -1; meta.slot[b] = slot; meta.kv_len[b] = n_true; }
+        // x = E[token], xn = RMSNorm(x)
+        ctx->launches += launch_embed_norm(dt, e == 0 ? root_token_dev : T.frontier_tok, nullptr, &meta, ctx->w.embed, c.vocab, nullptr, ctx->w.g_q,
+                                           c.hidden, c.rms_eps, c.norm_q, ctx->x, ctx->xn, rows, nullptr, nullptr, stream);
+        // the states produced by the previous forward join the cache tail (concatenation, Section 4.1)
+        if (e >= 1) {
+            const int nprev = e == 1 ? 1 : topk;
+            for (int r = 0; r < nprev; ++r) pos.idx[r] = n_true + (e == 1 ? 0 : 1 + (e - 2) * topk + r);
+            SkinnyArgs a;
+            memset(&a, 0, sizeof(a));
+            a.W = ctx->w.w_k; a.W2 = ctx->w.w_v; a.N = ctx->kd; a.K = c.hidden; a.X = ctx->h; a.ldx = c.hidden; a.B = nprev;
+            a.kcache = ctx->kcache; a.vcache = ctx->vcache; a.Hkv = c.n_kv_heads; a.dh = c.head_dim; a.cap = ctx->cap;
+            a.slot = slots; a.pos = pos;
+            BEAGLE_TREE_SKINNY(SK_KV, a, "K/V append");
+        }
+        {
+            SkinnyArgs a;
+            memset(&a, 0, sizeof(a));
+            a.W = ctx->w.w_q; a.N = ctx->qd; a.K = c.hidden; a.X = ctx->xn; a.ldx = c.hidden; a.B = rows;
+            a.out = ctx->q; a.ldo = ctx->qd;
+            BEAGLE_TREE_SKINNY(SK_STORE, a, "Q projection");
+        }
+        // attention: the true states (shared by the rows) in chunks, the ancestors' states as one extra chunk
+        {
+            int32_t stable[kMaxCallBatch];
+            for (int b = 0; b < rows; ++b) stable[b] = n_true;
+            float *po = nullptr, *pml = nullptr;
+            int nch = 0;
+            rc = tc_attn_decode(ctx->tc, ctx->q, meta, stable, rows, c.n_q_heads, c.n_kv_heads, c.head_dim, ctx->cap, n_true,
+                                ctx->attn_scratch, nullptr, ctx->o, ctx->dev_error, stream, 1, &po, &pml, &nch);
+            if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "attention: unsupported head shape");
+            ctx->launches += rc;
+            if (nanc > 0) {
+                rc = launch_attn_tail(ctx->q, ctx->kcache, ctx->vcache, T.frontier_anc, nanc, rows, slot, n_true, c.n_q_heads, c.n_kv_heads,
+                                      c.head_dim, ctx->cap, nch, (n_true + tc_attn_chunk() - 1) / tc_attn_chunk(), po, pml, stream);
+                if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "tree attention: unsupported head_dim");
+                ctx->launches += rc;
+            }
+            ctx->launches += launch_attn_combine(1, po, pml, meta, rows, c.n_q_heads, c.head_dim, nch, tc_attn_chunk(), ctx->o, stream,
+                                                 nanc > 0 ? 1 : 0);
+        }
+        {
+            SkinnyArgs a;
+            memset(&a, 0, sizeof(a));
+            a.W = ctx->w.w_o; a.N = c.hidden; a.K = ctx->qd; a.X = ctx->o; a.ldx = ctx->qd; a.B = rows;
+            a.out = ctx->y; a.ldo = c.hidden; a.resid = ctx->x; a.ldr = c.hidden;
+            a.norm_out = ctx->yn; a.gain = ctx->w.g_mlp; a.eps = c.rms_eps; a.do_norm = c.norm_mlp;
+            BEAGLE_TREE_SKINNY(SK_RESID, a, "O projection");
+        }
+        {
+            SkinnyArgs a;
+            memset(&a, 0, sizeof(a));
+            a.W = ctx->w.w_gate; a.W2 = ctx->w.w_up; a.N = c.mlp_dim; a.K = c.hidden; a.X = ctx->yn; a.ldx = c.hidden; a.B = rows;
+            a.out = ctx->act; a.ldo = c.mlp_dim;
+            BEAGLE_TREE_SKINNY(SK_SILU_MUL, a, "gate/up projection");
+        }
+        {
+            SkinnyArgs a;
+            memset(&a, 0, sizeof(a));
+            a.W = ctx->w.w_down; a.N = c.hidden; a.K = c.mlp_dim; a.X = ctx->act; a.ldx = c.mlp_dim; a.B = rows;
+            a.out = ctx->h; a.ldo = c.hidden; a.resid = ctx->y; a.ldr = c.hidden;
+            BEAGLE_TREE_SKINNY(SK_RESID, a, "down projection");
+        }
+        {
+            SkinnyArgs a;
+            memset(&a, 0, sizeof(a));
+            a.W = ctx->w.w_lm; a.N = c.vocab; a.K = c.hidden; a.X = ctx->h; a.ldx = c.hidden; a.B = rows;
+            a.logits = ctx->tree_logits; a.keys = ctx->lm_partials;
+            BEAGLE_TREE_SKINNY(SK_LOGITS, a, "LM head");
+        }
+        ctx->launches += launch_topk_logprob(ctx->tree_logits, rows, c.vocab, topk, T, stream);
+        ctx->launches += launch_tree_expand(T, topk, e, e == 0 ? 0 : topk + (e - 1) * topk * topk, stream);
+    }
+#undef BEAGLE_TREE_SKINNY
+    ctx->launches += launch_tree_rerank(T, total, n_candidates, tree_tokens_dev, tree_parents_dev, tree_scores_dev, stream);
+    return cuda_ok(ctx, "draft_tree");
+}
+
+beagle_status beagle_verify_tree_greedy(beagle_ctx* ctx, int32_t n_nodes, const int32_t* tree_tokens_dev, const int32_t* tree_parents_dev,
+                                        const int32_t* target_ids_dev, int32_t out_cap, int32_t* accept_len_dev, int32_t* out_tokens_dev,
+                                        int32_t* path_dev, void* stream_) {
+    if (ctx == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    if (n_nodes < 0 || n_nodes > 4096) return fail(ctx, BEAGLE_ERR_CAPACITY, "verify_tree: n_nodes %d outside [0, 4096]", n_nodes);
+    if (out_cap < 1) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "verify_tree: out_cap must be >= 1");
+    if (target_ids_dev == nullptr || accept_len_dev == nullptr || out_tokens_dev == nullptr ||
+        (n_nodes > 0 && (tree_tokens_dev == nullptr || tree_parents_dev == nullptr)))
+        return fail(ctx, BEAGLE_ERR_INVALID_ARG, "verify_tree: NULL argument");
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    ctx->launches += launch_tree_verify(tree_tokens_dev, tree_parents_dev, n_nodes, target_ids_dev, out_cap, accept_len_dev, out_tokens_dev,
+                                        path_dev, stream);
+    return cuda_ok(ctx, "verify_tree_greedy");
 }
 
 }  // extern "C"

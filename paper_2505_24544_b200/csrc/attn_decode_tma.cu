@@ -309,7 +309,8 @@ bool tc_attn_bind_cache(TcPlan* p, const void* kcache, const void* vcache, long 
 }
 
 int tc_attn_decode(TcPlan* p, const void* q, const BatchMeta& meta, const int32_t* stable_len, int B, int Hq, int Hkv, int dh, int cap,
-                   int max_kv_len, void* scratch, int* done_count, void* o, int* error_word, cudaStream_t stream) {
+                   int max_kv_len, void* scratch, int* done_count, void* o, int* error_word, cudaStream_t stream, int defer_merge,
+                   float** part_o_out, float** part_ml_out, int* nch_stride_out) {
     if (p == nullptr || !p->cache_maps_ok || B <= 0 || B > kMaxCallBatch || Hkv > 65535) return -1;
     if (dh != 64 && dh != 128) return -1;
     const int G = Hq / Hkv;
@@ -330,7 +331,8 @@ int tc_attn_decode(TcPlan* p, const void* q, const BatchMeta& meta, const int32_
     const float scale_log2 = 1.4426950408889634f / sqrtf((float)dh);
     // Few sequences: the last CTA of each head group merges its chunks (one launch less on a
     // latency-bound step).  Many sequences: a separate, wider merge kernel is faster than the tails.
-    const bool fuse_merge = B <= 8;
+    const bool fuse_merge = B <= 8 && !defer_merge;
+    if (part_o_out != nullptr) { *part_o_out = po; *part_ml_out = pml; *nch_stride_out = nch; }
     if (!fuse_merge) done_count = nullptr;
     int launched = 0;
     if (items > 0) {
@@ -345,7 +347,7 @@ int tc_attn_decode(TcPlan* p, const void* q, const BatchMeta& meta, const int32_
     // rows without any cached state got no CTA: their attention output is zero
     bool any_empty = !fuse_merge;
     for (int b = 0; b < B; ++b) any_empty |= (meta.kv_len[b] == 0);
-    if (any_empty) launched += launch_attn_combine(1, po, pml, meta, B, Hq, dh, nch, kChunk, o, stream);
+    if (any_empty && !defer_merge) launched += launch_attn_combine(1, po, pml, meta, B, Hq, dh, nch, kChunk, o, stream);
     return launched;
 }
 

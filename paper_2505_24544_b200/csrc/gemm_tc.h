@@ -54,7 +54,9 @@ bool tc_attn_bind_cache(TcPlan* plan, const void* kcache, const void* vcache, lo
 // Split-KV partials + combine, as launch_attn_decode; -1 when not covered (caller falls back).
 // stable_len[b] (host, nullable): leading cache rows of row b's slot that no kernel still in flight writes.
 int tc_attn_decode(TcPlan* plan, const void* q, const BatchMeta& meta, const int32_t* stable_len, int B, int Hq, int Hkv, int dh,
-                   int cap, int max_kv_len, void* scratch, int* done_count, void* o, int* error_word, cudaStream_t stream);
+                   int cap, int max_kv_len, void* scratch, int* done_count, void* o, int* error_word, cudaStream_t stream,
+                   int defer_merge = 0, float** part_o_out = nullptr, float** part_ml_out = nullptr, int* nch_stride_out = nullptr);
+// defer_merge: only the chunk partials are written; the caller adds its own chunks and merges (tree drafting).
 // done_count: B*Hkv device ints, zero before the first launch (the kernel leaves them zero).
 int tc_attn_chunk(void);
 

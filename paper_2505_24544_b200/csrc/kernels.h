@@ -53,8 +53,9 @@ int launch_attn_decode(int dtype, const void* q, const void* kcache, const void*
                        cudaStream_t stream);
 
 // Merges the split-KV partials (unnormalised o, running max, exp-sum per chunk of `chunk` keys).
+// extra_chunks: partials stored right after a row's regular chunks (the tree's ancestor states) to merge as well.
 int launch_attn_combine(int dtype, const float* part_o, const float* part_ml, const BatchMeta& meta, int B, int Hq, int dh,
-                        int nchunk_stride, int chunk, void* o, cudaStream_t stream);
+                        int nchunk_stride, int chunk, void* o, cudaStream_t stream, int extra_chunks = 0);
 
 // tokens_out[b] (optional) and last_token[slot[b]] from the per-block keys.
 int launch_argmax_finalize(const unsigned long long* partials, int nblk, const BatchMeta& meta, int B,
@@ -75,6 +76,28 @@ size_t verify_sample_scratch_bytes(int max_batch, int max_gamma);
 int launch_verify_sample(int logits_dtype, const int32_t* draft, const float* draft_logits, const void* target_logits, int B, int gamma, int V,
                          float temperature, const float* u_accept, const float* u_resample, void* scratch, int32_t* accept_len,
                          int32_t* out_tokens, cudaStream_t stream);
+
+// ---- dynamic-tree drafting: device-side bookkeeping -------------------------------------------
+constexpr int kTreeMaxTopk = 16, kTreeMaxDepth = 8, kTreeMaxCandidates = 64;
+constexpr int kTreeMaxNodes = kTreeMaxTopk + kTreeMaxDepth * kTreeMaxTopk * kTreeMaxTopk;
+struct TreeArrays {
+    int32_t* node_tok; int32_t* node_par; float* node_score;       // every node created, in creation order
+    int32_t* child_tok; float* child_lq;                           // [rows][k] of the last forward: k best children, log-probabilities
+    int32_t* frontier_node; int32_t* frontier_tok;                 // [k] nodes to forward next and their tokens
+    int32_t* frontier_anc;                                         // [k][kTreeMaxDepth + 1] tail positions of their ancestors' states
+    float2* topk_lse; unsigned long long* topk_keys;               // per (row, vocabulary slice): (max, exp-sum) and the slice's k best keys
+};
+size_t tree_arrays_bytes(int vocab);
+TreeArrays tree_arrays_carve(void* mem, int vocab);
+int launch_topk_logprob(const float* logits, int rows, int V, int k, const TreeArrays& t, cudaStream_t stream);
+int launch_tree_expand(const TreeArrays& t, int k, int level, int base, cudaStream_t stream);
+int launch_tree_rerank(const TreeArrays& t, int total, int n, int32_t* out_tok, int32_t* out_par, float* out_score, cudaStream_t stream);
+// Attention partial over each row's ancestor draft states, stored as split-KV chunk `chunk_idx` (bf16, dh 64 / 128).
+int launch_attn_tail(const void* q, const void* kcache, const void* vcache, const int32_t* anc, int nanc, int rows, int slot, int n_true, int Hq,
+                     int Hkv, int dh, int cap, int nch_stride, int chunk_idx, float* part_o, float* part_ml, cudaStream_t stream);
+// Greedy walk: target_ids[0] is the target's token at the root, target_ids[1 + n] after node n.
+int launch_tree_verify(const int32_t* tok, const int32_t* par, int n, const int32_t* target_ids, int out_cap, int32_t* accept_len,
+                       int32_t* out_tokens, int32_t* path, cudaStream_t stream);
 
 // ---- block path ------------------------------------------------------------------------------
 enum GemmEpilogue {

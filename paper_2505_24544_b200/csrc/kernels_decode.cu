@@ -404,12 +404,12 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attn_decode_kernel(
 template <typename T, int DPL>
 __global__ void __launch_bounds__(128) attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
                                                           const BatchMeta meta, int Hq, int dh, int nchunk_max, int chunk,
-                                                          T* __restrict__ o) {
+                                                          int extra_chunks, T* __restrict__ o) {
     const int head = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     pdl_launch_dependents();
     pdl_wait();
     const int kv_len = meta.kv_len[head / Hq];
-    const int nch = (kv_len + chunk - 1) / chunk;
+    const int nch = (kv_len + chunk - 1) / chunk + extra_chunks;
     const size_t p0 = (size_t)head * nchunk_max;
     const int per = (nch + 3) / 4;
     float M, den, acc[DPL];
@@ -441,23 +441,23 @@ __global__ void __launch_bounds__(128) attn_combine_kernel(const float* __restri
 
 template <typename T>
 static int attn_combine_dispatch(const float* part_o, const float* part_ml, const BatchMeta& meta, int B, int Hq, int dh,
-                                 int nchunk_stride, int chunk, T* o, cudaStream_t stream) {
+                                 int nchunk_stride, int chunk, T* o, cudaStream_t stream, int extra = 0) {
     const int grid = B * Hq;
     switch (dh) {
-        case 32: launch_pdl(attn_combine_kernel<T, 1>, dim3(grid), dim3(128), 0, stream, part_o, part_ml, meta, Hq, dh, nchunk_stride, chunk, o); return 1;
-        case 64: launch_pdl(attn_combine_kernel<T, 2>, dim3(grid), dim3(128), 0, stream, part_o, part_ml, meta, Hq, dh, nchunk_stride, chunk, o); return 1;
-        case 128: launch_pdl(attn_combine_kernel<T, 4>, dim3(grid), dim3(128), 0, stream, part_o, part_ml, meta, Hq, dh, nchunk_stride, chunk, o); return 1;
-        case 256: launch_pdl(attn_combine_kernel<T, 8>, dim3(grid), dim3(128), 0, stream, part_o, part_ml, meta, Hq, dh, nchunk_stride, chunk, o); return 1;
-        case 16: launch_pdl(attn_combine_kernel<T, 1>, dim3(grid), dim3(128), 0, stream, part_o, part_ml, meta, Hq, dh, nchunk_stride, chunk, o); return 1;
+        case 32: launch_pdl(attn_combine_kernel<T, 1>, dim3(grid), dim3(128), 0, stream, part_o, part_ml, meta, Hq, dh, nchunk_stride, chunk, extra, o); return 1;
+        case 64: launch_pdl(attn_combine_kernel<T, 2>, dim3(grid), dim3(128), 0, stream, part_o, part_ml, meta, Hq, dh, nchunk_stride, chunk, extra, o); return 1;
+        case 128: launch_pdl(attn_combine_kernel<T, 4>, dim3(grid), dim3(128), 0, stream, part_o, part_ml, meta, Hq, dh, nchunk_stride, chunk, extra, o); return 1;
+        case 256: launch_pdl(attn_combine_kernel<T, 8>, dim3(grid), dim3(128), 0, stream, part_o, part_ml, meta, Hq, dh, nchunk_stride, chunk, extra, o); return 1;
+        case 16: launch_pdl(attn_combine_kernel<T, 1>, dim3(grid), dim3(128), 0, stream, part_o, part_ml, meta, Hq, dh, nchunk_stride, chunk, extra, o); return 1;
         default: return -1;
     }
 }
 
 int launch_attn_combine(int dtype, const float* part_o, const float* part_ml, const BatchMeta& meta, int B, int Hq, int dh,
-                        int nchunk_stride, int chunk, void* o, cudaStream_t stream) {
+                        int nchunk_stride, int chunk, void* o, cudaStream_t stream, int extra_chunks) {
     if (B <= 0) return 0;
-    return dtype == 0 ? attn_combine_dispatch<float>(part_o, part_ml, meta, B, Hq, dh, nchunk_stride, chunk, (float*)o, stream)
-                      : attn_combine_dispatch<bf16>(part_o, part_ml, meta, B, Hq, dh, nchunk_stride, chunk, (bf16*)o, stream);
+    return dtype == 0 ? attn_combine_dispatch<float>(part_o, part_ml, meta, B, Hq, dh, nchunk_stride, chunk, (float*)o, stream, extra_chunks)
+                      : attn_combine_dispatch<bf16>(part_o, part_ml, meta, B, Hq, dh, nchunk_stride, chunk, (bf16*)o, stream, extra_chunks);
 }
 
 size_t attn_decode_scratch_bytes(int max_batch, int Hq, int dh, int max_kv) {

@@ -316,6 +316,88 @@ def test_verify_sample_small(dt, temperature):
     np.testing.assert_array_equal(out.cpu().numpy(), ref["out_tokens"])
 
 
+def tree_paths(tokens, parents, scores):
+    """{token path from the root: score} of a tree given as parallel arrays."""
+    out = {}
+    for n in range(len(tokens)):
+        path, a = [], n
+        while a >= 0:
+            path.append(int(tokens[a])); a = int(parents[a])
+        out[tuple(path[::-1])] = float(scores[n])
+    return out
+
+
+@pytest.mark.parametrize("name,n_ctx,depth,topk,n_cand,seed", [("gqa", 300, 3, 4, 20, 908), ("mha", 130, 6, 10, 60, 904), ("gqa", 0, 2, 3, 9, 903),
+                                                                ("gqa", 77, 0, 5, 5, 900)])
+def test_draft_tree_and_tree_verification(name, n_ctx, depth, topk, n_cand, seed):
+    """Dynamic draft tree against the oracle.  Which node wins a selection is a floating-point decision
+    (dozens of top-k cuts with gaps down to 1e-3), so: what is unique is compared -- every kept path's
+    score against the oracle's replay of that path, the kept set itself wherever the oracle's smallest
+    selection gap is clear -- and the rest is checked to be valid: every kept child lies in the oracle's
+    top-k of its parent up to the tolerance, and the sets overlap.  Then greedy acceptance along the tree."""
+    w = {"gqa": SMALL_GQA, "mha": SMALL_MHA}[name].scaled(batch=1)
+    from paper_2505_24544_b200.binding import BeagleHead
+    weights = WL.make_weights(w)
+    weights["w_lm"] = weights["w_lm"] * 32.0          # peaked next-token distributions (still exact in bf16)
+    head_gpu, head_cpu = BeagleHead.from_workload(w, weights, max_slots=2, max_ctx=n_ctx + 8, max_draft=64), oracle_head(w, weights)
+    rng = WL.data_rng(w, seed)
+    seqs = prefill_both(head_gpu, head_cpu, w, rng, [1], [n_ctx])
+    root = WL.make_tokens(w, rng, (1,))
+    ref = O.draft_tree(head_cpu, seqs[0], int(root[0]), depth, topk, n_cand)
+    tok, par, sc = head_gpu.draft_tree(1, to_dev(root, w.dtype), depth, topk, n_cand)
+    torch.cuda.synchronize()
+    tok, par, sc = tok.cpu().numpy(), par.cpu().numpy(), sc.cpu().numpy()
+    assert head_gpu.slot_lengths(1) == (n_ctx, 0)
+    assert np.all(par < np.arange(n_cand)) and np.all(par >= -1)
+    got, want = tree_paths(tok, par, sc), tree_paths(ref["tokens"], ref["parents"], ref["scores"])
+    assert len(got) == n_cand                                     # siblings are distinct tokens
+    step_tol = 3e-2                                               # one log-probability of bf16 logits (2e-2 + 1e-2 |z|, |z| ~ 1)
+    # (1) every kept path replayed by the oracle (forced chain drafting with concatenation): same score;
+    #     every kept child within the oracle's top-k of its parent
+    for path, score in got.items():
+        total, feed = 0.0, int(root[0])
+        for t in path:
+            out = O.draft_step(head_cpu, seqs, tokens_in=[feed], concat=True)
+            lq = O.log_softmax_rows(out["logits"][0])
+            kth = np.sort(lq)[-topk]
+            assert lq[t] >= kth - 2 * step_tol, (path, t, float(lq[t]), float(kth))
+            total += lq[t]
+            feed = t
+        O.rollback(seqs[0])
+        assert abs(score - total) <= len(path) * step_tol, (path, score, total)
+    # (2) the kept set: identical where every selection gap of the oracle is clear, overlapping otherwise
+    if ref["cut_margin"] > 2 * (depth + 1) * step_tol:
+        assert set(got) == set(want), "the selected token paths differ although every selection margin is clear"
+    assert len(set(got) & set(want)) >= 0.7 * n_cand
+    worst_kept = min(want.values())
+    assert min(got.values()) >= worst_kept - 2 * (depth + 1) * step_tol
+    # greedy acceptance along the tree, on the library's own tree: follow one of its leaves, then deviate
+    n = n_cand
+    leaf = int(np.argmax([len(k) for k in tree_paths(tok, par, sc)]))          # a deepest node
+    chain, a = [], leaf
+    while a >= 0:
+        chain.append(a); a = int(par[a])
+    chain = chain[::-1]
+    target = WL.make_tokens(w, rng, (n + 1,)).astype(np.int32)
+    target[0] = tok[chain[0]]
+    for i in range(len(chain) - 1):
+        target[1 + chain[i]] = tok[chain[i + 1]]
+    for cut_at in (len(chain), 1, 0):
+        tgt = target.copy()
+        if cut_at < len(chain):                                                   # break the path after cut_at nodes
+            idx = 0 if cut_at == 0 else 1 + chain[cut_at - 1]
+            tgt[idx] = (int(tgt[idx]) + 1) % w.vocab
+            while any(par[j] == (chain[cut_at - 1] if cut_at else -1) and tok[j] == tgt[idx] for j in range(n)):
+                tgt[idx] = (int(tgt[idx]) + 1) % w.vocab
+        acc, out, path = head_gpu.verify_tree_greedy(to_dev(tok, w.dtype), to_dev(par, w.dtype), to_dev(tgt, w.dtype), depth + 2)
+        a_ref, out_ref, path_ref = O.verify_tree_greedy(tok, par, int(tgt[0]), tgt[1:])
+        assert int(acc.item()) == a_ref == cut_at
+        assert out.cpu().numpy()[:a_ref + 1].tolist() == out_ref.tolist() and np.all(out.cpu().numpy()[a_ref + 1:] == -1)
+        assert path.cpu().numpy()[:a_ref].tolist() == path_ref.tolist()
+    from paper_2505_24544_b200.binding import beagle_check_device
+    beagle_check_device(head_gpu.ctx)
+
+
 def test_status_codes_for_capacity_and_state():
     from paper_2505_24544_b200.binding import BeagleError
     w = SMALL_GQA.scaled(batch=1, gamma=2)
