@@ -398,6 +398,34 @@ def test_draft_tree_and_tree_verification(name, n_ctx, depth, topk, n_cand, seed
     beagle_check_device(head_gpu.ctx)
 
 
+def test_argmax_rules_nan_negative_zero_and_largest_call():
+    """Arg-max conventions on the GPU (lowest index on ties, NaN never wins, -0 equals +0) and the
+    largest verification call the ABI admits (64 sequences x gamma 64)."""
+    w = SMALL_GQA.scaled(batch=64, gamma=64)
+    head_gpu, _, _ = build(w, max_slots=1, max_ctx=16)
+    rng = WL.data_rng(w, 64)
+    V = w.vocab
+    logits = rng.standard_normal((64, 65, V)).astype(np.float32)
+    logits[0, 0, :] = np.nan                                   # an all-NaN row: id 0
+    logits[0, 1, 5] = np.nan; logits[0, 1, 6] = 9.0            # NaN next to the maximum
+    logits[0, 2, :] = -0.0; logits[0, 2, 17] = 0.0             # -0 == +0: lowest index wins, not the +0
+    logits[0, 3, :] = -np.inf; logits[0, 3, 4098] = -1e30      # the last id of a row whose length is not a multiple of 8
+    draft = rng.integers(0, V, (64, 64)).astype(np.int32)
+    ref_ids = O.argmax_lowest(logits)
+    draft[1, :] = ref_ids[1, :64]                              # one sequence accepts everything
+    draft[2, :10] = ref_ids[2, :10]
+    acc, out = head_gpu.verify_greedy(to_dev(draft, w.dtype), target_logits=to_dev(logits, "fp32"))
+    acc_ref, out_ref = O.verify_greedy(draft, target_logits=logits)
+    np.testing.assert_array_equal(acc.cpu().numpy(), acc_ref)
+    np.testing.assert_array_equal(out.cpu().numpy(), out_ref)
+    assert ref_ids[0, 0] == 0 and ref_ids[0, 1] == 6 and ref_ids[0, 2] == 0 and ref_ids[0, 3] == 4098
+    assert acc_ref[1] == 64 and acc_ref[2] >= 10
+    from paper_2505_24544_b200.binding import BeagleError
+    with pytest.raises(BeagleError) as e:                      # one more sequence than a call admits
+        head_gpu.verify_greedy(torch.zeros(65, 4, dtype=torch.int32, device="cuda"), target_ids=torch.zeros(65, 5, dtype=torch.int32, device="cuda"))
+    assert e.value.status == 3
+
+
 def test_status_codes_for_capacity_and_state():
     from paper_2505_24544_b200.binding import BeagleError
     w = SMALL_GQA.scaled(batch=1, gamma=2)
