@@ -687,7 +687,7 @@ def main():
     line["clocks"] = sampler.stop()
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.only_headline:
-        n_seq, n_it = min(8, w.batch), 4                 # about 10 s of numpy on the machine's cores
+        n_seq, n_it = min(8, w.batch), 10                # about 10 s of numpy on the machine's cores
         val, sec, threads = oracle_sample(w, n_seq, n_it)
         line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": sec,
                                 "sample": f"{n_seq} of {w.batch} sequences x {n_it} SD iterations of {w.gamma} draft tokens, context prefill untimed"}

@@ -426,6 +426,48 @@ def test_argmax_rules_nan_negative_zero_and_largest_call():
     assert e.value.status == 3
 
 
+@pytest.mark.parametrize("batch", [2, 12])
+def test_draft_chain_replays_from_a_cuda_graph(batch):
+    """The draft chain enqueues kernels only (no host synchronisation, tokens fed device to device), so it
+    can be captured once and replayed: the replay reproduces the eager tokens bit for bit."""
+    w = SMALL_GQA.scaled(batch=batch, gamma=4)
+    head_gpu, _, _ = build(w, max_ctx=400)
+    rng = WL.data_rng(w, 123)
+    lengths = WL.make_context_lengths(w.scaled(ctx_min=100, ctx_max=300), rng)
+    slots = list(range(batch))
+    hidden = to_dev(WL.make_hidden(w, rng, int(lengths.sum())), w.dtype)
+    first = to_dev(WL.make_tokens(w, rng, (batch,)), w.dtype)
+    target = to_dev(WL.make_tokens(w, rng, (batch, w.gamma + 1)), w.dtype)
+    from paper_2505_24544_b200 import binding as B
+
+    def chain(draft, acc, out):
+        for s in range(w.gamma):
+            B.beagle_draft_step(head_gpu.ctx, slots, first if s == 0 else None, True, draft[:, s])
+        B.beagle_verify_greedy(head_gpu.ctx, draft, None, target, acc, out)
+
+    def fresh():
+        return (torch.zeros(batch, w.gamma, dtype=torch.int32, device="cuda"), torch.zeros(batch, dtype=torch.int32, device="cuda"),
+                torch.zeros(batch, w.gamma + 1, dtype=torch.int32, device="cuda"))
+
+    head_gpu.prefill_kv(slots, [int(n) for n in lengths], hidden)
+    eager = fresh()
+    chain(*eager)                                    # also the first call on this device: one-time set-up happens here
+    torch.cuda.synchronize()
+    head_gpu.rollback(slots)
+    captured = fresh()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        chain(*captured)
+    for _ in range(2):
+        for t in captured:
+            t.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        for a, b in zip(eager, captured):
+            assert torch.equal(a, b)
+    assert int(eager[0].abs().sum()) > 0
+
+
 def test_status_codes_for_capacity_and_state():
     from paper_2505_24544_b200.binding import BeagleError
     w = SMALL_GQA.scaled(batch=1, gamma=2)
