@@ -30,7 +30,7 @@ constexpr int kABytes = BM * BK * 2;
 template <int BN>
 struct SkSmem {
     static constexpr int kStageBytes = kABytes + BN * BK * 2;
-    static constexpr int kStages = BN <= 16 ? 6 : (BN <= 32 ? 5 : 4);
+    static constexpr int kStages = 3;            // 54-72 KB per CTA: three CTAs per SM, so a dependent launch finds a free slot to prefetch in
     static constexpr int kKeyBytes = 4 * BN * 8;
     static constexpr int kBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/ + kKeyBytes;
 };
@@ -45,10 +45,42 @@ struct SkArgs {
     int* error_word;
 };
 
-template <int BN, bool LOGITS>
+// Arguments of a projection's epilogue: adds the fp32 split partials in a fixed order, then store /
+// +residual / SiLU*mul / K,V cache scatter (and, in the finishing kernel, RMSNorm of the result).
+struct FinishArgs {
+    const float* partial;   // [splits][nmat][B][N]
+    int splits, nmat, B, N;
+    bf16* out; int ldo;
+    const bf16* resid; int ldr;
+    bf16* out2; int ld2; RowMap orow2;     // second copy (per-slot state)
+    bf16* norm_out; const bf16* gain; float eps; int do_norm;   // RMSNorm of the stored result (optional)
+    bf16* kcache; bf16* vcache; int Hkv, dh, cap; RowMap slot; RowMap pos;
+};
+
+// Cluster helpers (the fused variant runs the K splits of one tile as one thread-block cluster).
+__device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ld_cluster_f32(uint32_t local_addr, uint32_t rank) {
+    uint32_t ra;
+    float v;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(local_addr), "r"(rank));
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(ra) : "memory");
+    return v;
+}
+
+// VAR 0: fp32 split partials to global memory (a finishing kernel follows).  VAR 1: LM head (logits + keys).
+// VAR 2: the CTAs that share a tile form a cluster (its K splits, or gate and up); each leaves its accumulator
+// in its own shared memory and, after a cluster barrier, reduces one slice of the tile's rows over all CTAs'
+// shared memory (distributed shared memory, fixed order) and applies the epilogue: no partials, no second kernel.
+template <int BN, int VAR>
 __global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_constant__ CUtensorMap tmW,
                                                                const __grid_constant__ CUtensorMap tmW2,
-                                                               const __grid_constant__ CUtensorMap tmX, const SkArgs args) {
+                                                               const __grid_constant__ CUtensorMap tmX, const SkArgs args,
+                                                               const FinishArgs fin, const int mode) {
+    constexpr bool LOGITS = (VAR == 1), FUSED = (VAR == 2);
     using SM = SkSmem<BN>;
     constexpr int kStages = SM::kStages;
     constexpr uint32_t kTmemCols = BN < 32 ? 32 : BN;
@@ -154,7 +186,11 @@ __global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_cons
                 __syncwarp();
                 tmem_ld16(taddr + c0, r);
                 tmem_ld_wait();
-                if (!LOGITS) {
+                if (FUSED) {
+                    float* red = reinterpret_cast<float*>(smem_gen);     // [BN][128]: the ring is idle once the accumulator is complete
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) red[(c0 + j) * BM + q * 32 + lane] = __uint_as_float(r[j]);
+                } else if (!LOGITS) {
                     if (feat < args.N) {
                         float* dst = args.partial + ((size_t)(blockIdx.z * args.nmat + mat) * args.B) * args.N + feat;
 #pragma unroll
@@ -175,6 +211,10 @@ __global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_cons
                 }
             }
         }
+        if (FUSED && !ok) {                                               // an empty K slice (or an abandoned wait) adds nothing
+            float* red = reinterpret_cast<float*>(smem_gen);
+            for (int c = 0; c < BN; ++c) red[c * BM + q * 32 + lane] = 0.f;
+        }
         if (LOGITS) {
             asm volatile("bar.sync 1, 128;" ::: "memory");                // the four epilogue warps only
             const int col = threadIdx.x - 64;
@@ -187,6 +227,42 @@ __global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_cons
         }
     }
 
+    if (FUSED) {
+        // every CTA of the cluster has its [BN][128] accumulator in shared memory; CTA r reduces rows [r*rows, +rows)
+        __syncthreads();
+        pdl_wait();
+        cluster_sync_all();
+        const bool pair = (mode == SK_SILU_MUL);                     // cluster = (gate, up); otherwise = the K splits
+        const int csize = pair ? 2 : (int)gridDim.z;
+        const int rank = (int)cluster_rank();
+        const int rows = BM / csize;
+        const uint32_t red0 = smem_base;
+        const int me = pair ? 0 : mat;                               // K/V: this cluster's matrix
+        for (int idx = threadIdx.x; idx < rows * args.B; idx += kSkThreads) {
+            const int rl = idx % rows, col = idx / rows;
+            const int row = rank * rows + rl, n = ta * BM + row;
+            if (n >= args.N) continue;
+            const uint32_t la = red0 + (uint32_t)(col * BM + row) * 4u;
+            float v = 0.f, v1 = 0.f;
+            if (pair) { v = ld_cluster_f32(la, 0); v1 = ld_cluster_f32(la, 1); }
+            else { for (int z = 0; z < csize; ++z) v += ld_cluster_f32(la, (uint32_t)z); }
+            if (mode == SK_SILU_MUL) {
+                fin.out[(size_t)col * fin.ldo + n] = __float2bfloat16_rn(silu_f(v) * v1);
+            } else if (mode == SK_KV) {
+                const int pos = fin.pos.idx[col];
+                if (pos >= 0) {
+                    bf16* cache = me ? fin.vcache : fin.kcache;
+                    cache[(((size_t)fin.slot.idx[col] * fin.Hkv + n / fin.dh) * fin.cap + pos) * fin.dh + n % fin.dh] = __float2bfloat16_rn(v);
+                }
+            } else {
+                if (mode == SK_RESID) v += __bfloat162float(fin.resid[(size_t)col * fin.ldr + n]);
+                const bf16 o = __float2bfloat16_rn(v);
+                fin.out[(size_t)col * fin.ldo + n] = o;
+                if (fin.out2 != nullptr) fin.out2[(size_t)fin.orow2.idx[col] * fin.ld2 + n] = o;
+            }
+        }
+        cluster_sync_all();                                          // nobody leaves while its shared memory is being read
+    }
     fence_before();
     __syncthreads();
     pdl_wait();                                      // every thread, so that this grid's completion implies its predecessors'
@@ -199,15 +275,6 @@ __global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_cons
 
 // ---------------------------------------------------------------------------------------------- finishing kernel
 // Adds the fp32 split partials of one projection in a fixed order and applies its epilogue.
-struct FinishArgs {
-    const float* partial;   // [splits][nmat][B][N]
-    int splits, nmat, B, N;
-    bf16* out; int ldo;
-    const bf16* resid; int ldr;
-    bf16* out2; int ld2; RowMap orow2;     // second copy (per-slot state)
-    bf16* norm_out; const bf16* gain; float eps; int do_norm;   // RMSNorm of the stored result (optional)
-    bf16* kcache; bf16* vcache; int Hkv, dh, cap; RowMap slot; RowMap pos;
-};
 
 constexpr int kFinThreads = 256;             // whole-row mode (fused RMSNorm)
 constexpr int kFinColThreads = 64;           // column mode: many small CTAs, one float4 per thread
@@ -313,24 +380,41 @@ SplitPlan split_plan(int N, int K, int nmat, bool allow_split) {
     return s;
 }
 
-template <int BN, bool LOGITS>
-int launch_sk(const CUtensorMap& w, const CUtensorMap& w2, const CUtensorMap& x, const SkArgs& args, dim3 grid, cudaStream_t stream) {
+template <int BN, int VAR>
+int launch_sk(const CUtensorMap& w, const CUtensorMap& w2, const CUtensorMap& x, const SkArgs& args, const FinishArgs& fin, int mode,
+              dim3 grid, dim3 cluster, cudaStream_t stream) {
     using SM = SkSmem<BN>;
     static bool attr_done = false;
     if (!attr_done) {
-        if (cudaFuncSetAttribute(tc_skinny_kernel<BN, LOGITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kBytes) != cudaSuccess) return -1;
+        if (cudaFuncSetAttribute(tc_skinny_kernel<BN, VAR>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kBytes) != cudaSuccess) return -1;
         attr_done = true;
     }
-    launch_pdl(tc_skinny_kernel<BN, LOGITS>, grid, dim3(kSkThreads), SM::kBytes, stream, w, w2, x, args);
+    if (VAR != 2) {
+        launch_pdl(tc_skinny_kernel<BN, VAR>, grid, dim3(kSkThreads), SM::kBytes, stream, w, w2, x, args, fin, mode);
+        return 1;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = dim3(kSkThreads); cfg.dynamicSmemBytes = SM::kBytes; cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cluster.x; attr[0].val.clusterDim.y = cluster.y; attr[0].val.clusterDim.z = cluster.z;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 2;
+    if (cudaLaunchKernelEx(&cfg, tc_skinny_kernel<BN, VAR>, w, w2, x, args, fin, mode) != cudaSuccess) {
+        cudaGetLastError();
+        return -1;                                   // the caller falls back to partials + finishing kernel
+    }
     return 1;
 }
 
-template <bool LOGITS>
-int launch_sk_bn(int bn, const CUtensorMap& w, const CUtensorMap& w2, const CUtensorMap& x, const SkArgs& args, dim3 grid, cudaStream_t stream) {
+template <int VAR>
+int launch_sk_bn(int bn, const CUtensorMap& w, const CUtensorMap& w2, const CUtensorMap& x, const SkArgs& args, const FinishArgs& fin, int mode,
+                 dim3 grid, dim3 cluster, cudaStream_t stream) {
     switch (bn) {
-        case 16: return launch_sk<16, LOGITS>(w, w2, x, args, grid, stream);
-        case 32: return launch_sk<32, LOGITS>(w, w2, x, args, grid, stream);
-        default: return launch_sk<64, LOGITS>(w, w2, x, args, grid, stream);
+        case 16: return launch_sk<16, VAR>(w, w2, x, args, fin, mode, grid, cluster, stream);
+        case 32: return launch_sk<32, VAR>(w, w2, x, args, fin, mode, grid, cluster, stream);
+        default: return launch_sk<64, VAR>(w, w2, x, args, fin, mode, grid, cluster, stream);
     }
 }
 
@@ -362,11 +446,9 @@ int tc_skinny(TcPlan* p, int mode, const SkinnyArgs& g, cudaStream_t stream) {
     a.N = g.N; a.K = g.K; a.B = g.B; a.nmat = nmat; a.kb_per_split = sp.kb_per_split;
     a.partial = g.partial; a.logits = g.logits; a.keys = g.keys; a.error_word = g.error_word;
     dim3 grid(sp.tiles, nmat, sp.splits);
-    if (logits) return launch_sk_bn<true>(bn, *mapW, *mapW2, mapX, a, grid, stream);
-    if (launch_sk_bn<false>(bn, *mapW, *mapW2, mapX, a, grid, stream) < 0) return -1;
-
     FinishArgs f;
     memset(&f, 0, sizeof(f));
+    if (logits) return launch_sk_bn<1>(bn, *mapW, *mapW2, mapX, a, f, mode, grid, dim3(1, 1, 1), stream);
     f.partial = g.partial; f.splits = sp.splits; f.nmat = nmat; f.B = g.B; f.N = g.N;
     f.out = static_cast<bf16*>(g.out); f.ldo = g.ldo;
     f.resid = static_cast<const bf16*>(g.resid); f.ldr = g.ldr;
@@ -375,6 +457,18 @@ int tc_skinny(TcPlan* p, int mode, const SkinnyArgs& g, cudaStream_t stream) {
     f.kcache = static_cast<bf16*>(g.kcache); f.vcache = static_cast<bf16*>(g.vcache); f.Hkv = g.Hkv; f.dh = g.dh; f.cap = g.cap;
     f.slot = g.slot; f.pos = g.pos;
     const bool whole_row = (mode == SK_RESID && g.norm_out != nullptr);
+    // Preferred: the CTAs of a tile reduce among themselves (cluster of the K splits, or of gate and up).  The fused
+    // RMSNorm needs whole rows, so that projection keeps the finishing kernel.
+    if (!whole_row) {
+        int cs = 1;                                   // power-of-two number of K splits, at most 8 (portable cluster size)
+        while (cs * 2 <= sp.splits && cs * 2 <= 8) cs *= 2;
+        if (mode == SK_SILU_MUL) cs = 1;
+        SkArgs af = a;
+        af.kb_per_split = (sp.kb_total + cs - 1) / cs;
+        const dim3 fgrid_c(sp.tiles, nmat, cs), cluster(1, mode == SK_SILU_MUL ? 2 : 1, cs);
+        if (launch_sk_bn<2>(bn, *mapW, *mapW2, mapX, af, f, mode, fgrid_c, cluster, stream) > 0) return 1;
+    }
+    if (launch_sk_bn<0>(bn, *mapW, *mapW2, mapX, a, f, mode, grid, dim3(1, 1, 1), stream) < 0) return -1;
     dim3 fgrid(g.B, whole_row ? 1 : (g.N + kFinCols - 1) / kFinCols);
     const dim3 fblock(whole_row ? kFinThreads : kFinColThreads);
     switch (mode) {
