@@ -138,7 +138,9 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     } else if (warp == 1) {
         // ---------------- MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc(BM, BN);
+            // gate and up tiles sit back to back in the stage (256 rows of 128 bytes), so one MMA of N = 2*BN
+            // fills both accumulators and reads the A tile once
+            constexpr uint32_t idesc = make_idesc(BM, DUAL ? 2 * BN : BN);
             bool ok = true;
             int consumed = 0, it = 0;
             for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++it) {
@@ -155,13 +157,12 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
                     if (!ok) break;
                     fence_after();
                     const uint32_t sa = smem_base + s * SM::kStageBytes, sb = sa + kABytes;
-                    const uint64_t da = umma_desc(sa), db = umma_desc(sb), db2 = umma_desc(sb + kBBytes);
+                    const uint64_t da = umma_desc(sa), db = umma_desc(sb);
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; ++k) {
                         const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
                         const uint64_t koff = static_cast<uint64_t>((k * UMMA_K * 2) >> 4);   // advance inside the swizzle atom
                         umma_bf16(tacc, da + koff, db + koff, idesc, acc);
-                        if (DUAL) umma_bf16(tacc + BN, da + koff, db2 + koff, idesc, acc);
                     }
                     umma_commit(bar_empty + 8 * s);   // frees the stage once these MMAs have read it
                     ++consumed;
@@ -197,15 +198,10 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
                 float ce_mq = -INFINITY, ce_sq = 0.f, ce_mt = -INFINITY, ce_st = 0.f, ce_dot = 0.f;   // TC_CE running partial
                 const int label = (EPI == TC_CE && args.tgt == nullptr && m < args.a_rows) ? args.labels[m] : -1;
                 if (EPI == TC_CE && args.tgt == nullptr) ce_mt = 0.f;
-#pragma unroll 1
-                for (int c0 = 0; c0 < BN; c0 += 16) {
-                    uint32_t r[16], r2[16];
-                    __syncwarp();
-                    tmem_ld16(taddr + c0, r);
-                    if (DUAL) tmem_ld16(taddr + BN + c0, r2);
-                    tmem_ld_wait();
+                // 16 accumulator columns of this thread's row (r, and r2 = the second matrix of a gated pair)
+                auto consume = [&](const int c0, const uint32_t* r, const uint32_t* r2) {
                     const int n0 = tb * BN + c0;
-                    if (m >= args.a_rows || n0 >= args.b_rows) continue;
+                    if (m >= args.a_rows || n0 >= args.b_rows) return;
                     const bool full = (n0 + 16 <= args.b_rows);
                     if (EPI == TC_ARGMAX) {
 #pragma unroll
@@ -302,6 +298,18 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
                             }
                         }
                     }
+                };
+                // two TMEM loads in flight per wait
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    uint32_t ra[16], rb[16], ra2[16], rb2[16];
+                    __syncwarp();
+                    tmem_ld16(taddr + c0, ra);
+                    tmem_ld16(taddr + c0 + 16, rb);
+                    if (DUAL) { tmem_ld16(taddr + BN + c0, ra2); tmem_ld16(taddr + BN + c0 + 16, rb2); }
+                    tmem_ld_wait();
+                    consume(c0, ra, ra2);
+                    consume(c0 + 16, rb, rb2);
                 }
                 if (EPI == TC_ARGMAX && m < args.a_rows) args.keys[(size_t)m * args.keys_ld + tb] = best;
                 if (EPI == TC_CE && m < args.a_rows) {
