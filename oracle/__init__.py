@@ -36,6 +36,9 @@ from .beagle_oracle import (  # noqa: F401
     cross_entropy_rows,
     loss_weights,
     block_loss,
+    smooth_l1,
+    rms_norm_backward,
+    block_loss_grad,
     log_softmax_rows,
     top_k_lowest,
     draft_tree,

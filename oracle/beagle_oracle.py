@@ -48,6 +48,14 @@ kernel errors rather than storage noise has to round at the same places.
 Speculative-sampling verification (verify_sample) follows Section 3 literally;
 the random numbers it needs are inputs.
 
+Training step (block_loss_grad): the losses of Section 4.2 (Eq. 4, Eq. 7), the
+hidden-state regression term of Appendix B (smooth-L1, as in the EAGLE papers
+it cites) and their gradient in every parameter, by the chain rule written out
+operation by operation.  Under simulation the predicted states are constants of
+the differentiation (the function's docstring states this reading).  Pinned by
+central differences of block_loss and by automatic differentiation of a torch
+restatement.
+
 Pins (tests/test_oracle_*.py, all CPU): hand-worked tiny head, softmax row
 sums, single-key / identical-key special cases, GQA==MHA with repeated heads,
 mask brute force against the literal window rule, block forward == step-by-step
@@ -625,6 +633,155 @@ def block_loss(head: OracleHead, tokens: np.ndarray, hidden: np.ndarray, block: 
                                    None if target_logits is None else np.asarray(target_logits)[b],
                                    None if target_ids is None else np.asarray(target_ids)[b])
     return {"ce": ce, "weights": w, "n_windows": n_windows, "loss": float(np.sum(ce * w[None, :]) / (B * n_windows))}
+
+
+# --------------------------------------------------------------------------- block-attention training step: loss and gradients
+
+def smooth_l1(r: np.ndarray) -> np.ndarray:
+    """Smooth-L1 (Huber, threshold 1) element-wise: r^2 / 2 for |r| < 1, |r| - 1/2 otherwise.  The
+    hidden-state regression term that Appendix B adds to both training stages is the one of the
+    EAGLE papers, which is this function averaged over elements."""
+    r = np.asarray(r, dtype=F64)
+    a = np.abs(r)
+    return np.where(a < 1.0, 0.5 * r * r, a - 0.5)
+
+
+def rms_norm_backward(v: np.ndarray, g: np.ndarray, eps: float, dn: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """(dv, dg) of n = g * v * r, r = (mean(v^2) + eps)^(-1/2), row by row."""
+    v = np.asarray(v, dtype=F64)
+    r = 1.0 / np.sqrt(np.mean(v * v, axis=-1, keepdims=True) + eps)
+    gd = g * dn
+    dv = r * gd - v * (r ** 3) * np.mean(v * gd, axis=-1, keepdims=True)
+    return dv, np.sum(dn * v * r, axis=0)
+
+
+def block_loss_grad(head: OracleHead, tokens: np.ndarray, hidden: np.ndarray, block: int, offset: int, stage: str,
+                    sim_steps: int = 1, target_logits: Optional[np.ndarray] = None,
+                    target_ids: Optional[np.ndarray] = None, vloss_coef: float = 0.0) -> Dict[str, object]:
+    """One training step's loss and its gradient with respect to every parameter of the head.
+
+    total = L + vloss_coef * vloss, L the early (Eq. 4) or late (Eq. 7) loss of ``block_loss``;
+    vloss = mean over the positions that carry a loss term (weight > 0) and over the d components of
+    smooth_l1(h_hat_p - h_p): the draft state at p regresses on the target's true state at p, whose
+    place it takes as a key/value input when drafting continues (Section 4.1).
+
+    Gradient flow under simulation (the paper does not spell it out): the states predicted at
+    earlier simulation steps enter the final step as key/value INPUTS, exactly as the true states
+    they replace do, and are constants of the differentiation; W_K and W_V receive the gradient of
+    projecting them.  With sim_steps = 1 there is no predicted state and nothing is cut.
+
+    Returns 'loss' (the L term), 'vloss', 'total', and 'grads': name -> array shaped like the
+    parameter (embed, g_q, w_q, w_k, w_v, w_o, g_mlp, w_gate, w_up, w_down, w_lm).
+    """
+    c = head.cfg
+    tok = np.asarray(tokens, dtype=np.int64)
+    B, S = tok.shape
+    hid_all = np.asarray(hidden, dtype=F64).reshape(B, S, c.hidden)
+    if stage == "early" and sim_steps != 1:
+        raise ValueError("the early-stage loss uses the plain inverse block mask (sim_steps = 1)")
+    w, n_windows = loss_weights(S, block, offset, sim_steps, stage)
+    n_reg = B * int(np.count_nonzero(w))
+    grads = {name: np.zeros(shape_of(c), dtype=F64) for name, shape_of in _WEIGHT_SHAPES.items()}
+    loss = 0.0
+    vloss = 0.0
+    inv_sqrt = 1.0 / np.sqrt(F64(c.head_dim))
+    G = c.group
+    for b in range(B):
+        hid = hid_all[b]
+        # the states that earlier simulation steps wrote in place: constants of this step
+        h_pred = block_forward(head, tok[b], hid, block, offset, sim_steps)["hidden"] if sim_steps > 1 else None
+        k_true, v_true = project_kv(head, hid)
+        if h_pred is not None:
+            k_pred, v_pred = project_kv(head, h_pred)
+        kv, src = [], []                                    # per position: visible (K, V) and where each row came from
+        for p in range(1, S + 1):
+            n = visible_true_count(p, block, offset)
+            extra = list(range(n, n + min(p - n, sim_steps) - 1))        # 0-based rows of predicted states
+            if extra:
+                kv.append((np.concatenate([k_true[:n], k_pred[extra]]), np.concatenate([v_true[:n], v_pred[extra]])))
+            else:
+                kv.append((k_true[:n], v_true[:n]))
+            src.append((n, extra))
+        f = draft_block(head, tok[b], kv)
+        x, xn, q, o, y, yn, h, z = f["x"], f["xn"], f["q"], f["o"], f["y"], f["yn"], f["h"], f["logits"]
+        gate, up = yn @ head.w_gate.T, yn @ head.w_up.T
+        sig = 1.0 / (1.0 + np.exp(-gate))
+        act = gate * sig * up
+        # loss terms
+        qd = softmax_rows(z)
+        if target_ids is not None:
+            pd = np.zeros_like(qd)
+            pd[np.arange(S), np.asarray(target_ids, dtype=np.int64)[b]] = 1.0
+        else:
+            pd = softmax_rows(np.asarray(target_logits, dtype=F64)[b])
+        ce = cross_entropy_rows(z, None if target_logits is None else np.asarray(target_logits)[b],
+                                None if target_ids is None else np.asarray(target_ids)[b])
+        coef = w / (B * n_windows)
+        loss += float(np.sum(coef * ce))
+        dz = coef[:, None] * (qd - pd)
+        reg = (w > 0).astype(F64)[:, None]
+        resid = h - hid
+        dh = dz @ head.w_lm
+        if n_reg > 0:
+            vloss += float(np.sum(reg * smooth_l1(resid)) / (n_reg * c.hidden))
+            dh = dh + vloss_coef * reg * np.clip(resid, -1.0, 1.0) / (n_reg * c.hidden)
+        grads["w_lm"] += dz.T @ h
+        # h = y + W_down act
+        grads["w_down"] += dh.T @ act
+        dact = dh @ head.w_down
+        dgate = dact * up * (sig * (1.0 + gate * (1.0 - sig)))
+        dup = dact * gate * sig
+        grads["w_gate"] += dgate.T @ yn
+        grads["w_up"] += dup.T @ yn
+        dyn = dgate @ head.w_gate + dup @ head.w_up
+        if c.norm_mlp:
+            dy_n, dg = rms_norm_backward(y, head.g_mlp, c.rms_eps, dyn)
+            grads["g_mlp"] += dg
+        else:
+            dy_n = dyn
+        dy = dh + dy_n
+        # y = W_O o + x
+        grads["w_o"] += dy.T @ o
+        do = (dy @ head.w_o).reshape(S, c.n_q_heads, c.head_dim)
+        dq = np.zeros((S, c.n_q_heads, c.head_dim), dtype=F64)
+        dk_true = np.zeros_like(k_true); dv_true = np.zeros_like(v_true)
+        dk_pred = np.zeros_like(k_true); dv_pred = np.zeros_like(v_true)
+        qh = q.reshape(S, c.n_q_heads, c.head_dim)
+        for r in range(S):
+            k_vis, v_vis = kv[r]
+            nv = k_vis.shape[0]
+            if nv == 0:
+                continue
+            wts = attention_weights(head, qh[r], k_vis)                  # [Hq, nv]
+            dk_vis = np.zeros_like(k_vis); dv_vis = np.zeros_like(v_vis)
+            for hh in range(c.n_q_heads):
+                kh = hh // G
+                dp = v_vis[:, kh, :] @ do[r, hh]
+                ds = wts[hh] * (dp - np.dot(wts[hh], dp))
+                dq[r, hh] = (ds @ k_vis[:, kh, :]) * inv_sqrt
+                dk_vis[:, kh, :] += np.outer(ds, qh[r, hh]) * inv_sqrt
+                dv_vis[:, kh, :] += np.outer(wts[hh], do[r, hh])
+            n, extra = src[r]
+            dk_true[:n] += dk_vis[:n]; dv_true[:n] += dv_vis[:n]
+            for t, row in enumerate(extra):
+                dk_pred[row] += dk_vis[n + t]; dv_pred[row] += dv_vis[n + t]
+        kd = c.n_kv_heads * c.head_dim
+        grads["w_k"] += dk_true.reshape(S, kd).T @ hid
+        grads["w_v"] += dv_true.reshape(S, kd).T @ hid
+        if h_pred is not None:
+            grads["w_k"] += dk_pred.reshape(S, kd).T @ h_pred
+            grads["w_v"] += dv_pred.reshape(S, kd).T @ h_pred
+        dq2 = dq.reshape(S, -1)
+        grads["w_q"] += dq2.T @ xn
+        dxn = dq2 @ head.w_q
+        if c.norm_q:
+            dx_n, dg = rms_norm_backward(x, head.g_q, c.rms_eps, dxn)
+            grads["g_q"] += dg
+        else:
+            dx_n = dxn
+        dx = dy + dx_n
+        np.add.at(grads["embed"], tok[b], dx)
+    return {"loss": loss, "vloss": vloss, "total": loss + vloss_coef * vloss, "grads": grads}
 
 
 # --------------------------------------------------------------------------- dynamic draft tree (EAGLE-2's method, which the paper adopts)

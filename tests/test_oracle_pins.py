@@ -545,6 +545,139 @@ def test_block_loss_is_the_weighted_mean_of_block_forward_cross_entropies():
 
 # ----------------------------------------------------------------------------- dynamic draft tree
 
+# ----------------------------------------------------------------------------- gradients of the training losses
+
+def _grad_fixture(seed, B=2, S=9, **kw):
+    head, w, rng = small_head(seed=seed, d=16, hq=4, hkv=2, dh=4, m=24, V=19, std=0.4, **kw)
+    tokens = rng.integers(0, 19, (B, S))
+    hidden = rng.normal(0, 1.0, (B, S, 16))
+    tgt = rng.normal(0, 2.0, (B, S, 19))
+    return head, w, tokens, hidden, tgt
+
+
+def test_smooth_l1_and_rmsnorm_backward_by_differences():
+    r = np.array([-3.0, -1.0, -0.5, 0.0, 0.25, 1.0, 2.0])
+    assert np.allclose(O.smooth_l1(r), [2.5, 0.5, 0.125, 0.0, 0.03125, 0.5, 1.5])
+    rng = np.random.default_rng(5)
+    v, g, dn = rng.normal(size=(3, 7)), 1 + rng.normal(0, 0.2, 7), rng.normal(size=(3, 7))
+    dv, dg = O.rms_norm_backward(v, g, 1e-5, dn)
+    f = lambda vv, gg: float(np.sum(O.rms_norm(vv, gg, 1e-5) * dn))
+    e = 1e-6
+    for idx in [(0, 0), (1, 3), (2, 6)]:
+        vp, vm = v.copy(), v.copy(); vp[idx] += e; vm[idx] -= e
+        assert abs((f(vp, g) - f(vm, g)) / (2 * e) - dv[idx]) < 1e-7
+    for i in (0, 4):
+        gp, gm = g.copy(), g.copy(); gp[i] += e; gm[i] -= e
+        assert abs((f(v, gp) - f(v, gm)) / (2 * e) - dg[i]) < 1e-7
+
+
+@pytest.mark.parametrize("block,offset,labels,norms", [(3, 0, False, True), (4, 2, True, True), (2, 1, False, False)])
+def test_early_stage_gradient_is_the_derivative_of_block_loss(block, offset, labels, norms):
+    """Eq. 4: central differences of block_loss (a separate function) in every parameter tensor,
+    at the entries of largest gradient magnitude and at random ones."""
+    head, w, tokens, hidden, tgt = _grad_fixture(31 + block, norm_q=norms, norm_mlp=norms)
+    ids = np.argmax(tgt, axis=-1)
+    kw = dict(target_ids=ids) if labels else dict(target_logits=tgt)
+    out = O.block_loss_grad(head, tokens, hidden, block, offset, "early", **kw)
+    base = O.block_loss(head, tokens, hidden, block, offset, "early", **kw)["loss"]
+    assert abs(out["loss"] - base) < 1e-12 and out["vloss"] >= 0 and out["total"] == out["loss"]
+    rng = np.random.default_rng(7)
+    e = 1e-5
+    for name, g in out["grads"].items():
+        if not norms and name in ("g_q", "g_mlp"):
+            assert not g.any()
+            continue
+        flat = np.abs(g).reshape(-1)
+        picks = list(np.argsort(flat)[-2:]) + list(rng.integers(0, flat.size, 2))
+        for k in picks:
+            idx = np.unravel_index(int(k), g.shape)
+            vals = []
+            for sgn in (1, -1):
+                w2 = {n: a.copy() for n, a in w.items()}
+                w2[name][idx] += sgn * e
+                vals.append(O.block_loss(O.OracleHead(head.cfg, w2), tokens, hidden, block, offset, "early", **kw)["loss"])
+            fd = (vals[0] - vals[1]) / (2 * e)
+            assert abs(fd - g[idx]) < 1e-7 + 1e-5 * abs(fd), (name, idx, fd, g[idx])
+
+
+def _torch_training_loss(torch, c, T, tokens, hidden, tgt, block, offset, stage, sim_steps, vcoef, pred_states):
+    """An independent restatement with torch (float64, autograd): the final simulation step with the
+    predicted states given as constants."""
+    Fn = torch.nn.functional
+    B, S = tokens.shape
+    w, n_windows = O.loss_weights(S, block, offset, sim_steps, stage)
+    n_reg = B * int(np.count_nonzero(w))
+    rms = lambda v, g: v * torch.rsqrt(v.pow(2).mean(-1, keepdim=True) + c.rms_eps) * g
+    total_l, total_v = 0.0, 0.0
+    for b in range(B):
+        x = T["embed"][torch.tensor(tokens[b])]
+        xn = rms(x, T["g_q"]) if c.norm_q else x
+        q = Fn.linear(xn, T["w_q"]).view(S, c.n_q_heads, c.head_dim)
+        hs = torch.tensor(hidden[b])
+        rows = []
+        for p in range(1, S + 1):
+            n = O.visible_true_count(p, block, offset)
+            extra = list(range(n, n + min(p - n, sim_steps) - 1))
+            src = torch.cat([hs[:n], torch.tensor(pred_states[b][extra]).view(-1, c.hidden)]) if extra else hs[:n]
+            if src.shape[0] == 0:
+                rows.append(torch.zeros(c.n_q_heads * c.head_dim, dtype=torch.float64))
+                continue
+            k = Fn.linear(src, T["w_k"]).view(-1, c.n_kv_heads, c.head_dim).repeat_interleave(c.group, dim=1)
+            v = Fn.linear(src, T["w_v"]).view(-1, c.n_kv_heads, c.head_dim).repeat_interleave(c.group, dim=1)
+            a = torch.einsum("hd,jhd->hj", q[p - 1], k) / math.sqrt(c.head_dim)
+            rows.append(torch.einsum("hj,jhd->hd", torch.softmax(a, dim=-1), v).reshape(-1))
+        o = torch.stack(rows)
+        y = Fn.linear(o, T["w_o"]) + x
+        yn = rms(y, T["g_mlp"]) if c.norm_mlp else y
+        h = Fn.linear(Fn.silu(Fn.linear(yn, T["w_gate"])) * Fn.linear(yn, T["w_up"]), T["w_down"]) + y
+        logq = torch.log_softmax(Fn.linear(h, T["w_lm"]), dim=-1)
+        ce = -(torch.softmax(torch.tensor(tgt[b]), dim=-1) * logq).sum(-1)
+        wt = torch.tensor(w)
+        total_l = total_l + (wt * ce).sum() / (B * n_windows)
+        reg = (wt > 0).to(torch.float64)[:, None]
+        total_v = total_v + (reg * Fn.smooth_l1_loss(h, hs, reduction="none", beta=1.0)).sum() / (n_reg * c.hidden)
+    return total_l, total_v, total_l + vcoef * total_v
+
+
+@pytest.mark.parametrize("stage,block,offset,sim_steps,vcoef", [("early", 3, 1, 1, 10.0), ("late", 4, 0, 3, 10.0), ("late", 3, 2, 3, 0.0)])
+def test_training_gradients_against_torch_autograd(stage, block, offset, sim_steps, vcoef):
+    """Eq. 4 / Eq. 7 plus the regression term of Appendix B: every parameter's gradient against
+    automatic differentiation of an independent restatement; under simulation the predicted states
+    are constants there as well (they come from the oracle's own forward)."""
+    torch = pytest.importorskip("torch")
+    head, w, tokens, hidden, tgt = _grad_fixture(50 + block)
+    c = head.cfg
+    out = O.block_loss_grad(head, tokens, hidden, block, offset, stage, sim_steps, target_logits=tgt, vloss_coef=vcoef)
+    pred = [O.block_forward(head, tokens[b], hidden[b], block, offset, sim_steps)["hidden"] for b in range(tokens.shape[0])]
+    T = {n: torch.tensor(np.asarray(v), dtype=torch.float64, requires_grad=True) for n, v in w.items()}
+    l, v, total = _torch_training_loss(torch, c, T, tokens, hidden, tgt, block, offset, stage, sim_steps, vcoef, pred)
+    total.backward()
+    assert abs(float(l.detach()) - out["loss"]) < 1e-10 and abs(float(v.detach()) - out["vloss"]) < 1e-10
+    assert abs(out["loss"] - O.block_loss(head, tokens, hidden, block, offset, stage, sim_steps, target_logits=tgt)["loss"]) < 1e-12
+    for name, g in out["grads"].items():
+        ref = T[name].grad.numpy()
+        assert np.max(np.abs(ref - g)) < 1e-10 * (1 + np.max(np.abs(ref))), name
+        assert np.max(np.abs(ref)) > 0, name
+
+
+def test_regression_term_alone_has_the_closed_form_gradient_in_w_down():
+    """With the loss coefficient on the cross-entropy's side removed (labels that the draft already
+    predicts with certainty are not needed: take vloss alone through total - loss), d vloss / d W_down
+    = (clip(h - h_true, -1, 1) / (rows d))^T act."""
+    head, w, tokens, hidden, tgt = _grad_fixture(77, B=1, S=6)
+    a = O.block_loss_grad(head, tokens, hidden, 3, 0, "early", target_logits=tgt, vloss_coef=0.0)
+    b = O.block_loss_grad(head, tokens, hidden, 3, 0, "early", target_logits=tgt, vloss_coef=4.0)
+    kv_rows = []
+    k_true, v_true = O.project_kv(head, hidden[0])
+    for p in range(1, 7):
+        n = O.visible_true_count(p, 3, 0)
+        kv_rows.append((k_true[:n], v_true[:n]))
+    f = O.draft_block(head, tokens[0], kv_rows)
+    expect = (np.clip(f["h"] - hidden[0], -1, 1) / (6 * 16)).T @ f["act"]
+    assert np.allclose((b["grads"]["w_down"] - a["grads"]["w_down"]) / 4.0, expect, atol=1e-12)
+    assert abs(b["total"] - (a["loss"] + 4.0 * a["vloss"])) < 1e-12
+
+
 def _tree_fixture(seed=90, n=9):
     head, w, rng = small_head(seed=seed)
     seq = O.OracleSequence(head)
