@@ -162,6 +162,48 @@ beagle_status beagle_block_loss(beagle_ctx* ctx, int32_t batch, int32_t S, const
                                 int32_t logits_dtype, const int32_t* target_ids_dev, float* loss_out_dev, float* ce_out_dev,
                                 void* ws_dev, size_t ws_bytes, void* stream);
 
+/* Gradient buffers of beagle_block_grad: fp32 DEVICE pointers shaped like the parameters of beagle_weights
+ * (row-major [out, in]); a NULL entry means that gradient is not wanted and its products are skipped.  Every
+ * non-NULL buffer is overwritten (not accumulated into).  Owned by the caller. */
+typedef struct beagle_grads {
+    float* embed;    /* [V, d]: scatter-add of the query-side input gradients by token id (fp32 atomics: the
+                        order of the additions, hence the last bits, may differ between runs) */
+    float* g_q;      /* [d]        */
+    float* w_q;      /* [Hq*dh, d] */
+    float* w_k;      /* [Hkv*dh, d]*/
+    float* w_v;      /* [Hkv*dh, d]*/
+    float* w_o;      /* [d, Hq*dh] */
+    float* g_mlp;    /* [d]        */
+    float* w_gate;   /* [m, d]     */
+    float* w_up;     /* [m, d]     */
+    float* w_down;   /* [d, m]     */
+    float* w_lm;     /* [V, d]     */
+} beagle_grads;
+
+/* Workspace bytes of beagle_block_grad for `batch` sequences of S positions. */
+beagle_status beagle_block_grad_workspace_bytes(const beagle_config* cfg, int32_t batch, int32_t S, size_t* bytes);
+
+/* One training step of the block path (Section 4.2; Appendix B for the regression term): the forward of
+ * beagle_block_loss, then the gradient of
+ *     total = L + vloss_coef * vloss
+ * in every parameter whose entry of `grads` is non-NULL.  L is the early (Eq. 4, stage 0) or late (Eq. 7, stage 1)
+ * loss exactly as beagle_block_loss defines it.  vloss is the hidden-state regression of Appendix B (the one of the
+ * EAGLE papers): the mean, over the positions that carry a loss term (weight > 0) and over the d components, of
+ * smooth_l1(h_hat_p - h_p), smooth_l1(r) = r^2/2 for |r| < 1 and |r| - 1/2 otherwise, h_hat_p the draft state at
+ * position p (row p of the block forward's hidden output) and h_p = hidden_dev[b, p], the target's true state at
+ * the same position.
+ * Simulation (sim_steps > 1): the states predicted at earlier simulation steps enter the final step as key/value
+ * inputs, like the true states they replace; they are constants of the differentiation, and W_k / W_v receive the
+ * gradient of projecting them.  With sim_steps = 1 nothing is cut.
+ * Arguments as for beagle_block_loss; vloss_coef >= 0 (the paper trains with 10).  loss_out_dev fp32 [3] =
+ * {L, vloss, total}.  Intermediate gradients are kept in the storage type (bf16 or fp32), accumulated in fp32 inside
+ * every product; parameter gradients are fp32 and, except `embed`, summed in a fixed order.  hidden, mlp_dim and
+ * head_dim must be multiples of 8 (SHAPE otherwise).  ws_dev: 256-byte aligned, beagle_block_grad_workspace_bytes. */
+beagle_status beagle_block_grad(beagle_ctx* ctx, int32_t batch, int32_t S, const int32_t* tokens_dev, const void* hidden_dev,
+                                int32_t block, int32_t offset, int32_t sim_steps, int32_t stage, const void* target_logits_dev,
+                                int32_t logits_dtype, const int32_t* target_ids_dev, float vloss_coef, const beagle_grads* grads,
+                                float* loss_out_dev, void* ws_dev, size_t ws_bytes, void* stream);
+
 /* Greedy acceptance (Section 3: in greedy decoding the draft's and the target's top-1 tokens are
  * matched and only a contiguous prefix is accepted, plus one extra target token).  Exactly one of
  * target_logits_dev ([batch, gamma+1, V], logits_dtype BEAGLE_FP32 or BEAGLE_BF16) and

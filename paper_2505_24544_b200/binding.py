@@ -28,6 +28,7 @@ EXPORTED_SYMBOLS = (
     "beagle_launch_count", "beagle_profile_enable", "beagle_profile_read", "beagle_profile_stage_count",
     "beagle_profile_stage_name", "beagle_verify_greedy_static", "beagle_check_device",
     "beagle_workspace_buffer", "beagle_block_workspace_buffer", "beagle_verify_sample", "beagle_block_loss", "beagle_draft_tree", "beagle_verify_tree_greedy",
+    "beagle_block_grad_workspace_bytes", "beagle_block_grad",
 )
 
 BUFFER_IDS = {"x": 0, "xn": 1, "q": 2, "o": 3, "y": 4, "yn": 5, "act": 6, "h": 7, "kt": 8, "vt": 9, "kp": 10, "vp": 11}
@@ -43,6 +44,10 @@ class BeagleConfig(C.Structure):
 
 
 class BeagleWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in WEIGHT_NAMES]
+
+
+class BeagleGrads(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in WEIGHT_NAMES]
 
 
@@ -96,6 +101,11 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.beagle_block_workspace_buffer.restype = C.c_int
     lib.beagle_block_loss.argtypes = [vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, i32, vp, vp, vp, vp, C.c_size_t, vp]
     lib.beagle_block_loss.restype = C.c_int
+    lib.beagle_block_grad_workspace_bytes.argtypes = [C.POINTER(BeagleConfig), i32, i32, szp]
+    lib.beagle_block_grad_workspace_bytes.restype = C.c_int
+    lib.beagle_block_grad.argtypes = [vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, i32, vp, C.c_float, C.POINTER(BeagleGrads), vp, vp,
+                                      C.c_size_t, vp]
+    lib.beagle_block_grad.restype = C.c_int
     lib.beagle_draft_tree.argtypes = [vp, i32, vp, i32, i32, i32, vp, vp, vp, vp]
     lib.beagle_draft_tree.restype = C.c_int
     lib.beagle_verify_tree_greedy.argtypes = [vp, i32, vp, vp, vp, i32, vp, vp, vp, vp]
@@ -261,6 +271,40 @@ def beagle_block_loss(ctx: Context, tokens: torch.Tensor, hidden: torch.Tensor, 
                                         _ptr(ce_out), ctx.block_ws.data_ptr(), ctx.block_ws.numel(), _stream()))
 
 
+def beagle_block_grad_workspace_bytes(ctx: Context, batch: int, S: int) -> int:
+    n = C.c_size_t()
+    st = ctx.lib.beagle_block_grad_workspace_bytes(C.byref(ctx.cfg), batch, S, C.byref(n))
+    if st != 0:
+        raise BeagleError(st, "beagle_block_grad_workspace_bytes")
+    return n.value
+
+
+def beagle_block_grad(ctx: Context, tokens: torch.Tensor, hidden: torch.Tensor, block: int, offset: int, sim_steps: int, stage: str,
+                      target_logits: Optional[torch.Tensor], target_ids: Optional[torch.Tensor], vloss_coef: float,
+                      grads: Dict[str, Optional[torch.Tensor]], loss_out: torch.Tensor) -> None:
+    """grads: parameter name -> fp32 tensor shaped like the parameter (missing / None: not computed); loss_out fp32 [3]."""
+    batch, S = tokens.shape
+    need = beagle_block_grad_workspace_bytes(ctx, batch, S)
+    if ctx.block_ws is None or ctx.block_ws.numel() < need:
+        ctx.block_ws = None
+        ctx.block_ws = torch.empty(need, dtype=torch.uint8, device=tokens.device)
+    code = BEAGLE_FP32
+    if target_logits is not None:
+        if target_logits.dtype == torch.bfloat16:
+            code = BEAGLE_BF16
+        elif target_logits.dtype != torch.float32:
+            raise ValueError("target_logits must be float32 or bfloat16")
+    g = BeagleGrads()
+    for name in WEIGHT_NAMES:
+        t = grads.get(name)
+        if t is not None and t.dtype != torch.float32:
+            raise ValueError("gradient buffers must be float32")
+        setattr(g, name, _ptr(t))
+    ctx.check(ctx.lib.beagle_block_grad(ctx.handle, batch, S, _ptr(tokens), _ptr(hidden), block, offset, sim_steps,
+                                        {"early": 0, "late": 1}[stage], _ptr(target_logits), code, _ptr(target_ids), float(vloss_coef),
+                                        C.byref(g), _ptr(loss_out), ctx.block_ws.data_ptr(), ctx.block_ws.numel(), _stream()))
+
+
 def beagle_verify_greedy(ctx: Context, draft_tokens: torch.Tensor, target_logits: Optional[torch.Tensor],
                          target_ids: Optional[torch.Tensor], accept_len: torch.Tensor, out_tokens: torch.Tensor) -> None:
     batch, gamma = draft_tokens.shape
@@ -387,6 +431,7 @@ class BeagleHead:
         self.cfg = BeagleConfig(hidden, n_q_heads, n_kv_heads, head_dim, mlp_dim, vocab, code, rms_eps, int(norm_q),
                                 int(norm_mlp), max_slots, max_ctx, max_draft)
         self.ctx = Context(self.cfg, weights)
+        self.weight_shapes = {n: tuple(weights[n].shape) for n in WEIGHT_NAMES}
         self.device = self.ctx.kv_buf.device
         self.dtype = torch_dtype(code)
 
@@ -428,6 +473,14 @@ class BeagleHead:
         ce = torch.empty(B, S, dtype=torch.float32, device=self.device)
         beagle_block_loss(self.ctx, tokens, hidden, block, offset, sim_steps, stage, target_logits, target_ids, loss, ce)
         return loss, ce
+
+    def block_grad(self, tokens, hidden, block, offset, stage, sim_steps=1, target_logits=None, target_ids=None, vloss_coef=0.0,
+                   params=WEIGHT_NAMES):
+        """One training step: returns (losses fp32 [3] = L, vloss, total; dict of fp32 gradients for `params`)."""
+        grads = {n: torch.empty(tuple(getattr(self, "weight_shapes")[n]), dtype=torch.float32, device=self.device) for n in params}
+        losses = torch.empty(3, dtype=torch.float32, device=self.device)
+        beagle_block_grad(self.ctx, tokens, hidden, block, offset, sim_steps, stage, target_logits, target_ids, vloss_coef, grads, losses)
+        return losses, grads
 
     def verify_greedy(self, draft_tokens, target_logits=None, target_ids=None):
         B, gamma = draft_tokens.shape

@@ -15,12 +15,14 @@ using namespace beagle;
 enum Stage {
     ST_KV_APPEND = 0, ST_EMBED_NORM, ST_Q_PROJ, ST_ATTN_DECODE, ST_O_PROJ, ST_MLP_NORM, ST_GATE_UP, ST_DOWN, ST_LM_HEAD,
     ST_ARGMAX, ST_PREFILL, ST_VERIFY, ST_BLK_EMBED, ST_BLK_QKV, ST_BLK_PRED_KV, ST_BLK_ATTN, ST_BLK_O, ST_BLK_NORM,
-    ST_BLK_GATE_UP, ST_BLK_DOWN, ST_BLK_LM_HEAD, ST_BLK_ARGMAX, ST_COUNT
+    ST_BLK_GATE_UP, ST_BLK_DOWN, ST_BLK_LM_HEAD, ST_BLK_ARGMAX, ST_BWD_DLOGITS, ST_BWD_DX, ST_BWD_DW, ST_BWD_ATTN,
+    ST_BWD_TRANSPOSE, ST_BWD_ELEMENTWISE, ST_COUNT
 };
 static const char* const kStageNames[ST_COUNT] = {
     "kv_append", "embed_norm", "q_proj", "attn_decode", "o_proj", "mlp_norm", "gate_up", "down_proj", "lm_head",
     "argmax_finalize", "prefill_kv", "verify", "blk_embed", "blk_qkv", "blk_pred_kv", "blk_attn", "blk_o_proj", "blk_norm",
-    "blk_gate_up", "blk_down", "blk_lm_head", "blk_argmax"};
+    "blk_gate_up", "blk_down", "blk_lm_head", "blk_argmax", "bwd_dlogits", "bwd_dx_gemm", "bwd_dw_gemm", "bwd_attn",
+    "bwd_transpose", "bwd_elementwise"};
 
 struct StageRecord { int stage; cudaEvent_t start, stop; };
 
@@ -190,6 +192,42 @@ BlockLayout block_layout(const beagle_config& c, int batch, int S) {
     L.ce_part = take(M * (size_t)tc_argmax_tiles(c.vocab) * kCeFields * sizeof(float));     // loss forward: per (row, column tile)
     L.ce_rows = take(M * sizeof(float));
     L.wce = take(M * sizeof(float));
+    L.total = off;
+    return L;
+}
+
+// Workspace of one training step: the forward's regions, then what the backward adds.
+struct GradLayout {
+    BlockLayout fwd;
+    size_t gate, up, dact, dz, dh0, dh, dyn, dy, d_o, dq, dkt, dvt, dkp, dvp, dxn, ta, tb, wt, lse, delta, stats, vrow, dgpart, total;
+    int Mp, Vp;        // rows and vocabulary padded to a multiple of 8 (contraction lengths of the transposed products)
+};
+GradLayout grad_layout(const beagle_config& c, int batch, int S) {
+    GradLayout L;
+    L.fwd = block_layout(c, batch, S);
+    const size_t elt = c.dtype == BEAGLE_BF16 ? 2 : 4;
+    const size_t M = (size_t)batch * S;
+    const size_t d = c.hidden, qd = (size_t)c.n_q_heads * c.head_dim, kd = (size_t)c.n_kv_heads * c.head_dim, m = c.mlp_dim, V = c.vocab;
+    L.Mp = (int)((M + 7) / 8 * 8);
+    L.Vp = (int)((V + 7) / 8 * 8);
+    size_t off = L.fwd.total;
+    auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + bytes); return at; };
+    auto max2 = [](size_t a, size_t b) { return a > b ? a : b; };
+    L.gate = take(M * m * elt); L.up = take(M * m * elt); L.dact = take(M * m * elt);
+    L.dz = take(M * (size_t)L.Vp * elt);
+    L.dh0 = take(M * d * elt); L.dh = take(M * d * elt); L.dyn = take(M * d * elt); L.dy = take(M * d * elt);
+    L.d_o = take(M * qd * elt); L.dq = take(M * qd * elt);
+    L.dkt = take(M * kd * elt); L.dvt = take(M * kd * elt); L.dkp = take(M * kd * elt); L.dvp = take(M * kd * elt);
+    L.dxn = take(M * d * elt);
+    // transposed operands: TA holds d(out)^T [features, rows], TB the layer input^T; K/V use two row blocks side by side
+    const size_t widest = max2(max2(V, m), max2(qd, d));
+    L.ta = take(max2(widest * (size_t)L.Mp, kd * 2 * (size_t)L.Mp) * elt);
+    L.tb = take(max2(max2(m, qd) * (size_t)L.Mp, d * 2 * (size_t)L.Mp) * elt);
+    // one transposed weight at a time: [in, out] (hidden, mlp_dim and head_dim are multiples of 8; the vocabulary is padded)
+    L.wt = take(max2(d * (size_t)L.Vp, max2(m, qd) * d) * elt);
+    L.lse = take(M * c.n_q_heads * sizeof(float)); L.delta = take(M * c.n_q_heads * sizeof(float));
+    L.stats = take(M * 4 * sizeof(float)); L.vrow = take(M * sizeof(float));
+    L.dgpart = take((size_t)rmsnorm_bwd_parts((int)M) * d * sizeof(float));
     L.total = off;
     return L;
 }
@@ -758,12 +796,16 @@ struct LossSpec {                  // beagle_block_loss: what replaces the LM he
     const void* tgt; int tgt_dtype;
     const int32_t* labels;
     float* loss_out; float* ce_out;
+    void* gate; void* up;          // training step: the final pass keeps W_gate n and W_up n (NULL: fused SiLU-mul GEMM)
+    float* row_stats;              // training step: every row's merged softmax statistics (4 floats), or NULL
+    float* lse2;                   // training step: the attention rows' base-2 log-sum-exp (tensor-core attention only), or NULL
+    bool lse2_written;             // set when the last pass ran the tensor-core attention and filled lse2
 };
 
 static beagle_status block_forward_impl(beagle_ctx* ctx, int32_t batch, int32_t S, const int32_t* tokens_dev,
                                         const void* hidden_dev, int32_t block, int32_t offset, int32_t sim_steps,
                                         float* logits_out_dev, int32_t* argmax_out_dev, void* hidden_out_dev,
-                                        void* ws_dev, size_t ws_bytes, void* stream_, const LossSpec* loss) {
+                                        void* ws_dev, size_t ws_bytes, void* stream_, LossSpec* loss) {
     if (ctx == nullptr) return BEAGLE_ERR_INVALID_ARG;
     if (batch <= 0 || S <= 0 || tokens_dev == nullptr || hidden_dev == nullptr || ws_dev == nullptr)
         return fail(ctx, BEAGLE_ERR_INVALID_ARG, "block_forward: NULL or empty argument");
@@ -825,8 +867,10 @@ static beagle_status block_forward_impl(beagle_ctx* ctx, int32_t batch, int32_t 
             rc = -1;
             if (ctx->tc != nullptr) {       // bf16, head_dim 64 / 128: tensor-core tiles
                 clear_error_word_once(ctx, stream);
+                float* lse2 = (loss != nullptr && step == sim_steps) ? loss->lse2 : nullptr;
                 rc = tc_attn_block(ctx->tc, Q, Kt, Vt, Kp, Vp, batch, S, c.n_q_heads, c.n_kv_heads, c.head_dim, block, offset, step, O,
-                                   ctx->dev_error, stream);
+                                   ctx->dev_error, stream, lse2);
+                if (rc >= 0 && lse2 != nullptr) loss->lse2_written = true;
             }
             if (rc < 0)
                 rc = launch_attn_block(dt, Q, Kt, Vt, Kp, Vp, batch, S, c.n_q_heads, c.n_kv_heads, c.head_dim, block, offset, step, O, stream);
@@ -845,7 +889,15 @@ static beagle_status block_forward_impl(beagle_ctx* ctx, int32_t batch, int32_t 
         memset(&g, 0, sizeof(g));
         g.M = M; g.A = Yn; g.lda = c.hidden; g.K = c.hidden; g.W = ctx->w.w_gate; g.W2 = ctx->w.w_up; g.N = c.mlp_dim;
         g.C = ACT; g.ldc = c.mlp_dim;
-        BEAGLE_GEMM(ST_BLK_GATE_UP, GEMM_SILU_MUL, g, "gate/up projection");
+        if (loss != nullptr && loss->gate != nullptr && step == sim_steps) {
+            g.W2 = nullptr; g.C = loss->gate;
+            BEAGLE_GEMM(ST_BLK_GATE_UP, GEMM_STORE, g, "gate projection");
+            g.W = ctx->w.w_up; g.C = loss->up;
+            BEAGLE_GEMM(ST_BLK_GATE_UP, GEMM_STORE, g, "up projection");
+            ctx->launches += launch_silu_mul(dt, loss->gate, loss->up, ACT, (size_t)M * c.mlp_dim, stream);
+        } else {
+            BEAGLE_GEMM(ST_BLK_GATE_UP, GEMM_SILU_MUL, g, "gate/up projection");
+        }
         memset(&g, 0, sizeof(g));
         g.M = M; g.A = ACT; g.lda = c.mlp_dim; g.K = c.mlp_dim; g.W = ctx->w.w_down; g.N = c.hidden; g.C = H; g.ldc = c.hidden;
         g.R = Y; g.ldr = c.hidden;
@@ -880,7 +932,7 @@ static beagle_status block_forward_impl(beagle_ctx* ctx, int32_t batch, int32_t 
         StageTimer timer_(ctx, ST_BLK_ARGMAX, stream);
         ctx->launches += launch_ce_finalize(part, ntiles, batch, S, block, offset, sim_steps, loss->stage,
                                             reinterpret_cast<float*>(ws + L.ce_rows), reinterpret_cast<float*>(ws + L.wce), loss->ce_out,
-                                            loss->loss_out, stream);
+                                            loss->loss_out, stream, loss->row_stats);
     }
     // LM head at every position
     if (loss == nullptr && (logits_out_dev != nullptr || argmax_out_dev != nullptr)) {
@@ -941,8 +993,221 @@ beagle_status beagle_block_loss(beagle_ctx* ctx, int32_t batch, int32_t S, const
     LossSpec spec;
     spec.stage = stage; spec.tgt = target_logits_dev; spec.tgt_dtype = target_logits_dev != nullptr ? logits_dtype : 0;
     spec.labels = target_ids_dev; spec.loss_out = loss_out_dev; spec.ce_out = ce_out_dev;
+    spec.gate = nullptr; spec.up = nullptr; spec.row_stats = nullptr; spec.lse2 = nullptr; spec.lse2_written = false;
     return block_forward_impl(ctx, batch, S, tokens_dev, hidden_dev, block, offset, sim_steps, nullptr, nullptr, nullptr, ws_dev,
                               ws_bytes, stream_, &spec);
+}
+
+beagle_status beagle_block_grad_workspace_bytes(const beagle_config* cfg, int32_t batch, int32_t S, size_t* bytes) {
+    const beagle_status st = check_config(cfg);
+    if (st != BEAGLE_OK) return st;
+    if (bytes == nullptr || batch <= 0 || S <= 0) return BEAGLE_ERR_INVALID_ARG;
+    if ((long long)batch * S > (1ll << 24)) return BEAGLE_ERR_CAPACITY;
+    *bytes = grad_layout(*cfg, batch, S).total;
+    return BEAGLE_OK;
+}
+
+beagle_status beagle_block_grad(beagle_ctx* ctx, int32_t batch, int32_t S, const int32_t* tokens_dev, const void* hidden_dev,
+                                int32_t block, int32_t offset, int32_t sim_steps, int32_t stage, const void* target_logits_dev,
+                                int32_t logits_dtype, const int32_t* target_ids_dev, float vloss_coef, const beagle_grads* grads,
+                                float* loss_out_dev, void* ws_dev, size_t ws_bytes, void* stream_) {
+    if (ctx == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    if (grads == nullptr || loss_out_dev == nullptr) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "block_grad: grads / loss_out is NULL");
+    if (batch <= 0 || S <= 0) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "block_grad: empty batch");
+    if ((long long)batch * S > (1ll << 24)) return fail(ctx, BEAGLE_ERR_CAPACITY, "block_grad: too many positions");
+    if (stage != 0 && stage != 1) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "block_grad: stage must be 0 (early) or 1 (late)");
+    if (stage == 0 && sim_steps != 1) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "block_grad: the early-stage loss uses sim_steps = 1");
+    if ((target_logits_dev == nullptr) == (target_ids_dev == nullptr))
+        return fail(ctx, BEAGLE_ERR_INVALID_ARG, "block_grad: give exactly one of target_logits / target_ids");
+    if (target_logits_dev != nullptr && logits_dtype != BEAGLE_FP32 && logits_dtype != BEAGLE_BF16)
+        return fail(ctx, BEAGLE_ERR_INVALID_ARG, "block_grad: unknown logits_dtype");
+    if (!(vloss_coef >= 0.f)) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "block_grad: vloss_coef must be >= 0");
+    const beagle_config& c = ctx->cfg;
+    if (c.hidden % 8 || c.mlp_dim % 8 || c.head_dim % 8) return fail(ctx, BEAGLE_ERR_SHAPE, "block_grad: hidden, mlp_dim and head_dim must be multiples of 8");
+    const GradLayout L = grad_layout(c, batch, S);
+    if (ws_dev == nullptr || ws_bytes < L.total) return fail(ctx, BEAGLE_ERR_CAPACITY, "block_grad: workspace %zu < %zu bytes", ws_bytes, L.total);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    char* ws = static_cast<char*>(ws_dev);
+    const int dt = c.dtype;
+    const int M = batch * S, Mp = L.Mp, Vp = L.Vp;
+    const int d = c.hidden, qd = ctx->qd, kd = ctx->kd, m = c.mlp_dim, V = c.vocab;
+
+    // ---- forward of the training step: keeps every activation, W_gate n and W_up n, and the rows' softmax statistics
+    LossSpec spec;
+    spec.stage = stage; spec.tgt = target_logits_dev; spec.tgt_dtype = target_logits_dev != nullptr ? logits_dtype : 0;
+    spec.labels = target_ids_dev; spec.loss_out = loss_out_dev; spec.ce_out = nullptr;
+    spec.gate = ws + L.gate; spec.up = ws + L.up; spec.row_stats = reinterpret_cast<float*>(ws + L.stats);
+    spec.lse2 = reinterpret_cast<float*>(ws + L.lse); spec.lse2_written = false;
+    beagle_status st = block_forward_impl(ctx, batch, S, tokens_dev, hidden_dev, block, offset, sim_steps, nullptr, nullptr, nullptr, ws_dev,
+                                          ws_bytes, stream_, &spec);
+    if (st != BEAGLE_OK) return st;
+
+    const BlockLayout& F = L.fwd;
+    void *X = ws + F.x, *Xn = ws + F.xn, *Q = ws + F.q, *Kt = ws + F.kt, *Vt = ws + F.vt, *Kp = ws + F.kp, *Vp_ = ws + F.vp;
+    void *O = ws + F.o, *Y = ws + F.y, *Yn = ws + F.yn, *ACT = ws + F.act, *H = ws + F.h;
+    void *G = ws + L.gate, *U = ws + L.up, *DACT = ws + L.dact, *DZ = ws + L.dz, *DH0 = ws + L.dh0, *DH = ws + L.dh, *DYN = ws + L.dyn;
+    void *DY = ws + L.dy, *DO = ws + L.d_o, *DQ = ws + L.dq, *DKT = ws + L.dkt, *DVT = ws + L.dvt, *DKP = ws + L.dkp, *DVP = ws + L.dvp;
+    void *DXN = ws + L.dxn, *TA = ws + L.ta, *TB = ws + L.tb, *WT = ws + L.wt;
+    float* dgpart = reinterpret_cast<float*>(ws + L.dgpart);
+    int rc;
+    GemmArgs g;
+#define BEAGLE_BWD_GEMM(STAGE, EPI, WHAT)                                              \
+    do {                                                                               \
+        StageTimer timer_(ctx, STAGE, stream);                                         \
+        rc = dense_gemm(ctx, EPI, g, stream);                                          \
+        if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, WHAT ": unsupported shape");   \
+        ctx->launches += rc;                                                           \
+    } while (0)
+    auto transpose = [&](const void* in, int rows, int cols, int ld_in, void* out, int ld_out, int col0, int rows_pad) {
+        StageTimer timer_(ctx, ST_BWD_TRANSPOSE, stream);
+        ctx->launches += launch_transpose_pad(dt, in, rows, cols, ld_in, out, ld_out, col0, rows_pad, stream);
+    };
+    // dX = dY W: A = dY [M, n_out_pad], "weight" = W^T [n_in, n_out_pad] (transposed here, padded columns zero)
+    auto dx_gemm = [&](int epi, const void* dYm, int ldy, const void* W, int n_out, int n_in, void* out, const void* resid) -> int {
+        const int np = (n_out + 7) / 8 * 8;
+        transpose(W, n_out, n_in, n_in, WT, np, 0, np);
+        memset(&g, 0, sizeof(g));
+        g.M = M; g.A = dYm; g.lda = ldy; g.K = np; g.W = WT; g.N = n_in; g.C = out; g.ldc = n_in; g.R = resid; g.ldr = n_in;
+        g.w_transient = 1;
+        StageTimer timer_(ctx, ST_BWD_DX, stream);
+        const int r = dense_gemm(ctx, epi, g, stream);
+        if (r > 0) ctx->launches += r;
+        return r;
+    };
+    // dW = dY^T X: A = dY^T [n_out, K], "weight" = X^T [n_in, K], K = Mp (or 2 Mp with two row blocks side by side), fp32 out
+    auto dw_gemm = [&](int n_out, int n_in, int Kc, float* out) -> int {
+        memset(&g, 0, sizeof(g));
+        g.M = n_out; g.A = TA; g.lda = Kc; g.K = Kc; g.W = TB; g.N = n_in; g.C = out; g.ldc = n_in; g.w_transient = 1;
+        StageTimer timer_(ctx, ST_BWD_DW, stream);
+        const int r = dense_gemm(ctx, GEMM_F32, g, stream);
+        if (r > 0) ctx->launches += r;
+        return r;
+    };
+#define BEAGLE_NEED(EXPR, WHAT) do { if ((EXPR) < 0) return fail(ctx, BEAGLE_ERR_SHAPE, WHAT ": unsupported shape"); } while (0)
+
+    // ---- d z = weight * (softmax(z) - p) / (batch * windows), from re-materialised logits, chunk by chunk
+    const int windows = (S - offset + block - 1) / block;
+    const float ce_scale = 1.0f / ((float)batch * (float)windows);
+    {
+        float* chunk = reinterpret_cast<float*>(ws + F.logits);
+        for (int r0 = 0; r0 < M; r0 += F.lm_chunk_rows) {
+            const int rows = M - r0 < F.lm_chunk_rows ? M - r0 : F.lm_chunk_rows;
+            memset(&g, 0, sizeof(g));
+            g.M = rows; g.A = static_cast<const char*>(H) + (size_t)r0 * d * ctx->elt; g.lda = d; g.K = d;
+            g.W = ctx->w.w_lm; g.N = V; g.C = chunk; g.ldc = V;
+            BEAGLE_BWD_GEMM(ST_BWD_DLOGITS, GEMM_F32, "LM head (backward)");
+            StageTimer timer_(ctx, ST_BWD_DLOGITS, stream);
+            ctx->launches += launch_dlogits(dt, chunk, rows, V, target_logits_dev, spec.tgt_dtype, target_ids_dev,
+                                            reinterpret_cast<const float*>(ws + L.stats), r0, S, block, offset, sim_steps, stage, ce_scale, DZ, Vp,
+                                            stream);
+        }
+    }
+    // ---- regression term (Appendix B): value and its gradient in h
+    {
+        int reg_rows = 0;      // positions with a loss term, per sequence
+        for (int p = offset + 1; p <= S; ++p) {
+            const int slot = p - (offset + block * ((p - 1 - offset) / block));
+            if (stage == 0 || slot <= sim_steps) ++reg_rows;
+        }
+        const float n_reg = (float)batch * (float)reg_rows * (float)d;
+        const float vscale = reg_rows > 0 ? 1.0f / n_reg : 0.f;
+        StageTimer timer_(ctx, ST_BWD_ELEMENTWISE, stream);
+        ctx->launches += launch_vloss(dt, H, hidden_dev, M, d, S, block, offset, sim_steps, stage, vloss_coef * vscale, vscale, vloss_coef, DH0,
+                                      reinterpret_cast<float*>(ws + L.vrow), loss_out_dev, stream);
+    }
+    // ---- LM head: dh = dz W_lm + dh0;  dW_lm = dz^T h
+    BEAGLE_NEED(dx_gemm(GEMM_RESID, DZ, Vp, ctx->w.w_lm, V, d, DH, DH0), "dh");
+    if (grads->w_lm != nullptr) {
+        transpose(DZ, M, V, Vp, TA, Mp, 0, Mp);
+        transpose(H, M, d, d, TB, Mp, 0, Mp);
+        BEAGLE_NEED(dw_gemm(V, d, Mp, grads->w_lm), "dW_lm");
+    }
+    // ---- MLP: h = y + W_down act
+    BEAGLE_NEED(dx_gemm(GEMM_STORE, DH, d, ctx->w.w_down, d, m, DACT, nullptr), "dact");
+    if (grads->w_down != nullptr) {
+        transpose(DH, M, d, d, TA, Mp, 0, Mp);
+        transpose(ACT, M, m, m, TB, Mp, 0, Mp);
+        BEAGLE_NEED(dw_gemm(d, m, Mp, grads->w_down), "dW_down");
+    }
+    {
+        StageTimer timer_(ctx, ST_BWD_ELEMENTWISE, stream);
+        ctx->launches += launch_silu_mul_bwd(dt, G, U, DACT, (size_t)M * m, stream);     // G <- d gate, U <- d up
+    }
+    BEAGLE_NEED(dx_gemm(GEMM_STORE, G, m, ctx->w.w_gate, m, d, DYN, nullptr), "dyn (gate)");
+    BEAGLE_NEED(dx_gemm(GEMM_RESID, U, m, ctx->w.w_up, m, d, DYN, DYN), "dyn (up)");
+    if (grads->w_gate != nullptr || grads->w_up != nullptr) {
+        transpose(Yn, M, d, d, TB, Mp, 0, Mp);
+        if (grads->w_gate != nullptr) {
+            transpose(G, M, m, m, TA, Mp, 0, Mp);
+            BEAGLE_NEED(dw_gemm(m, d, Mp, grads->w_gate), "dW_gate");
+        }
+        if (grads->w_up != nullptr) {
+            transpose(U, M, m, m, TA, Mp, 0, Mp);
+            BEAGLE_NEED(dw_gemm(m, d, Mp, grads->w_up), "dW_up");
+        }
+    }
+    {   // dy = dh + RMSNorm backward of dyn
+        StageTimer timer_(ctx, ST_BWD_ELEMENTWISE, stream);
+        rc = launch_rmsnorm_bwd(dt, Y, ctx->w.g_mlp, DYN, DH, M, d, c.rms_eps, c.norm_mlp, DY, dgpart, grads->g_mlp, stream);
+        if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "block_grad: hidden too large for the RMSNorm backward");
+        ctx->launches += rc;
+    }
+    // ---- output projection: y = W_O o + x
+    BEAGLE_NEED(dx_gemm(GEMM_STORE, DY, d, ctx->w.w_o, d, qd, DO, nullptr), "do");
+    if (grads->w_o != nullptr) {
+        transpose(DY, M, d, d, TA, Mp, 0, Mp);
+        transpose(O, M, qd, qd, TB, Mp, 0, Mp);
+        BEAGLE_NEED(dw_gemm(d, qd, Mp, grads->w_o), "dW_o");
+    }
+    // ---- attention
+    {
+        StageTimer timer_(ctx, ST_BWD_ATTN, stream);
+        rc = -1;
+        if (spec.lse2_written)       // bf16, head_dim 64 / 128: tensor-core tiles, from the forward's log-sum-exp
+            rc = tc_attn_block_bwd(ctx->tc, Q, Kt, Vt, Kp, Vp_, O, DO, spec.lse2, batch, S, c.n_q_heads, c.n_kv_heads, c.head_dim, block, offset,
+                                   sim_steps, reinterpret_cast<float*>(ws + L.delta), DQ, DKT, DVT, DKP, DVP, ctx->dev_error, stream);
+        if (rc < 0)
+            rc = launch_attn_block_bwd(dt, Q, Kt, Vt, Kp, Vp_, DO, batch, S, c.n_q_heads, c.n_kv_heads, c.head_dim, block, offset, sim_steps, DQ,
+                                       DKT, DVT, DKP, DVP, reinterpret_cast<float*>(ws + L.lse), reinterpret_cast<float*>(ws + L.delta), stream);
+        if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "block_grad: unsupported head_dim");
+        ctx->launches += rc;
+    }
+    // ---- projections: dW_q = dq^T xn;  dW_k = dk_true^T h_true + dk_pred^T h_hat (same for V)
+    if (grads->w_q != nullptr) {
+        transpose(DQ, M, qd, qd, TA, Mp, 0, Mp);
+        transpose(Xn, M, d, d, TB, Mp, 0, Mp);
+        BEAGLE_NEED(dw_gemm(qd, d, Mp, grads->w_q), "dW_q");
+    }
+    if (grads->w_k != nullptr || grads->w_v != nullptr) {
+        const int Kc = sim_steps > 1 ? 2 * Mp : Mp;
+        transpose(hidden_dev, M, d, d, TB, Kc, 0, Mp);
+        if (sim_steps > 1) transpose(H, M, d, d, TB, Kc, Mp, Mp);
+        if (grads->w_k != nullptr) {
+            transpose(DKT, M, kd, kd, TA, Kc, 0, Mp);
+            if (sim_steps > 1) transpose(DKP, M, kd, kd, TA, Kc, Mp, Mp);
+            BEAGLE_NEED(dw_gemm(kd, d, Kc, grads->w_k), "dW_k");
+        }
+        if (grads->w_v != nullptr) {
+            transpose(DVT, M, kd, kd, TA, Kc, 0, Mp);
+            if (sim_steps > 1) transpose(DVP, M, kd, kd, TA, Kc, Mp, Mp);
+            BEAGLE_NEED(dw_gemm(kd, d, Kc, grads->w_v), "dW_v");
+        }
+    }
+    // ---- query side down to the embedding: dxn = dq W_q, dx = dy + RMSNorm backward
+    if (grads->g_q != nullptr || grads->embed != nullptr) {
+        BEAGLE_NEED(dx_gemm(GEMM_STORE, DQ, qd, ctx->w.w_q, qd, d, DXN, nullptr), "dxn");
+        StageTimer timer_(ctx, ST_BWD_ELEMENTWISE, stream);
+        rc = launch_rmsnorm_bwd(dt, X, ctx->w.g_q, DXN, DY, M, d, c.rms_eps, c.norm_q, DYN, dgpart, grads->g_q, stream);   // DYN <- dx
+        if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "block_grad: hidden too large for the RMSNorm backward");
+        ctx->launches += rc;
+        if (grads->embed != nullptr) {
+            cudaMemsetAsync(grads->embed, 0, (size_t)V * d * sizeof(float), stream);
+            ctx->launches += launch_embed_grad(dt, tokens_dev, DYN, M, d, grads->embed, stream);
+        }
+    }
+#undef BEAGLE_BWD_GEMM
+#undef BEAGLE_NEED
+    return cuda_ok(ctx, "block_grad");
 }
 
 beagle_status beagle_verify_greedy(beagle_ctx* ctx, int32_t batch, int32_t gamma, const int32_t* draft_tokens_dev,

@@ -16,6 +16,7 @@
 
 #include "gemm_tc.h"
 #include "tc_plan.h"
+#include "mma_tiles.cuh"
 #include "tc_ptx.cuh"
 
 namespace beagle {
@@ -23,34 +24,15 @@ namespace beagle {
 namespace {
 
 using namespace tc;
+using namespace mma_tiles;
 
 constexpr int kBQ = 64, kBKey = 64, kWarps = 4;
-
-__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
-}
-__device__ __forceinline__ void mma16816(float* d, const uint32_t* a, uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
-    __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&t);
-}
-// 16-byte chunk `chunk` of row `row` in a [64 rows x 64 cols] bf16 tile written with the 128-byte
-// swizzle; wider rows use consecutive tiles.
-__device__ __forceinline__ uint32_t toff(int row, int chunk) {
-    return static_cast<uint32_t>((chunk >> 3) * (64 * 128) + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
-}
 
 struct BlkArgs {
     int S, Hq, Hkv, block, offset, step;
     float scale_log2;
     bf16* O;            // [B*S, Hq*DH]
+    float* lse2;        // optional [B*S, Hq]: base-2 log-sum-exp of the scaled scores of every row (0 for a row without keys)
     int* error_word;
 };
 
@@ -223,6 +205,13 @@ __global__ void __launch_bounds__(kWarps * 32, 3) attn_block_tc_kernel(const __g
         l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 1);
         l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
     }
+    if (a.lse2 != nullptr && c == 0) {
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            const int row = q0 + warp * 16 + g + 8 * r;
+            if (row < a.S) a.lse2[((size_t)(row_base + row)) * a.Hq + h] = l_run[r] > 0.f ? m_run[r] + log2f(l_run[r]) : 0.f;
+        }
+    }
     const float inv0 = (ok && l_run[0] > 0.f) ? 1.f / l_run[0] : 0.f;
     const float inv1 = (ok && l_run[1] > 0.f) ? 1.f / l_run[1] : 0.f;
 #pragma unroll
@@ -259,7 +248,7 @@ int launch_blk(const CUtensorMap* maps, const BlkArgs& a, dim3 grid, cudaStream_
 }  // namespace
 
 int tc_attn_block(TcPlan* p, const void* Q, const void* Kt, const void* Vt, const void* Kp, const void* Vp, int B, int S, int Hq,
-                  int Hkv, int dh, int block, int offset, int step, void* O, int* error_word, cudaStream_t stream) {
+                  int Hkv, int dh, int block, int offset, int step, void* O, int* error_word, cudaStream_t stream, float* lse2) {
     if (p == nullptr || (dh != 64 && dh != 128) || B <= 0 || S <= 0 || B > 65535 || Hq > 65535) return -1;
     const long long rows = (long long)B * S;
     CUtensorMap maps[5];
@@ -271,6 +260,7 @@ int tc_attn_block(TcPlan* p, const void* Q, const void* Kt, const void* Vt, cons
     a.S = S; a.Hq = Hq; a.Hkv = Hkv; a.block = block; a.offset = offset; a.step = step;
     a.scale_log2 = 1.4426950408889634f / sqrtf((float)dh);
     a.O = static_cast<bf16*>(O);
+    a.lse2 = lse2;
     a.error_word = error_word;
     dim3 grid((S + kBQ - 1) / kBQ, Hq, B);
     return dh == 128 ? launch_blk<128>(maps, a, grid, stream) : launch_blk<64>(maps, a, grid, stream);

@@ -64,7 +64,7 @@ __global__ void __launch_bounds__(256) row_ce_kernel(const float* __restrict__ l
 // One warp per row: merge the column tiles' partials, ce = lse(z) - E_p[z], weight by the position.
 __global__ void __launch_bounds__(256) ce_finalize_kernel(const float* __restrict__ ce_part, int ntiles, int rows, int S, int block, int offset,
                                                          int sim_steps, int stage, float* __restrict__ ce_rows, float* __restrict__ wce,
-                                                         float* __restrict__ ce_out) {
+                                                         float* __restrict__ ce_out, float4* __restrict__ row_stats) {
     const int row = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (row >= rows) return;
     CePart acc = {-INFINITY, 0.f, -INFINITY, 0.f, 0.f};
@@ -87,6 +87,7 @@ __global__ void __launch_bounds__(256) ce_finalize_kernel(const float* __restric
         ce_rows[row] = ce;
         wce[row] = w * ce;
         if (ce_out != nullptr) ce_out[row] = ce;
+        if (row_stats != nullptr) row_stats[row] = make_float4(acc.mq, acc.sq, acc.mt, acc.st);
     }
 }
 
@@ -115,10 +116,11 @@ int launch_row_ce(const float* logits, int rows, int V, const void* tgt, int tgt
 }
 
 int launch_ce_finalize(const float* ce_part, int ntiles, int batch, int S, int block, int offset, int sim_steps, int stage,
-                       float* ce_rows, float* wce, float* ce_out, float* loss_out, cudaStream_t stream) {
+                       float* ce_rows, float* wce, float* ce_out, float* loss_out, cudaStream_t stream, float* row_stats) {
     const int rows = batch * S;
     if (rows <= 0) return 0;
-    ce_finalize_kernel<<<(rows * 32 + 255) / 256, 256, 0, stream>>>(ce_part, ntiles, rows, S, block, offset, sim_steps, stage, ce_rows, wce, ce_out);
+    ce_finalize_kernel<<<(rows * 32 + 255) / 256, 256, 0, stream>>>(ce_part, ntiles, rows, S, block, offset, sim_steps, stage, ce_rows, wce, ce_out,
+                                                                     reinterpret_cast<float4*>(row_stats));
     const int windows = (S - offset + block - 1) / block;
     ce_reduce_kernel<<<1, 1024, 0, stream>>>(wce, rows, 1.0f / ((float)batch * (float)windows), loss_out);
     return 2;

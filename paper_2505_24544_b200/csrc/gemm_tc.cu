@@ -416,7 +416,14 @@ int tc_gemm(TcPlan* p, int epi, const GemmArgs& g, cudaStream_t stream) {
     const int BN = dual ? 128 : 256;
     CUtensorMap mapA;
     if (!tc_encode_map(p, &mapA, g.A, g.M, g.K, g.lda, BM)) return -1;
-    const CUtensorMap* mapB = tc_weight_map(p, g.W, g.N, g.K, BN);
+    CUtensorMap transient;
+    const CUtensorMap* mapB;
+    if (g.w_transient) {
+        if (dual || (reinterpret_cast<uintptr_t>(g.W) & 15) || !tc_encode_map(p, &transient, g.W, g.N, g.K, g.K, BN)) return -1;
+        mapB = &transient;
+    } else {
+        mapB = tc_weight_map(p, g.W, g.N, g.K, BN);
+    }
     const CUtensorMap* mapB2 = dual ? tc_weight_map(p, g.W2, g.N, g.K, BN) : mapB;
     if (mapB == nullptr || mapB2 == nullptr) return -1;
     TcArgs a;

@@ -63,6 +63,12 @@ int tc_attn_chunk(void);
 // ---- block-masked cross-attention of the multi-token forward (bf16, head_dim 64 or 128) -------
 // Same contract as launch_attn_block; -1 when not covered (caller falls back).
 int tc_attn_block(TcPlan* plan, const void* Q, const void* Kt, const void* Vt, const void* Kp, const void* Vp, int B, int S,
-                  int Hq, int Hkv, int dh, int block, int offset, int step, void* O, int* error_word, cudaStream_t stream);
+                  int Hq, int Hkv, int dh, int block, int offset, int step, void* O, int* error_word, cudaStream_t stream,
+                  float* lse2 = nullptr);
+// lse2 (optional, fp32 [B*S, Hq]): base-2 log-sum-exp of every row's scaled scores, for the backward below.
+// Backward (same contract as launch_attn_block_bwd, bf16, head_dim 64 / 128); delta: fp32 [B*S, Hq] scratch.
+int tc_attn_block_bwd(TcPlan* plan, const void* Q, const void* Kt, const void* Vt, const void* Kp, const void* Vp, const void* O, const void* dO,
+                      const float* lse2, int B, int S, int Hq, int Hkv, int dh, int block, int offset, int step, float* delta, void* dQ,
+                      void* dKt, void* dVt, void* dKp, void* dVp, int* error_word, cudaStream_t stream);
 
 }  // namespace beagle

@@ -131,6 +131,7 @@ struct GemmArgs {
     const int32_t* labels;          // GEMM_CE, hard targets: [M] (used when tgt == NULL)
     float* ce_part;                 // GEMM_CE: [M][column tiles][kCeFields]
     int* error_word;                // device word set to 1 when a bounded wait ran out
+    int w_transient;                // W is a workspace buffer (its tensor map is not cached by pointer)
     SeqRows rows;
 };
 int launch_gemm_simt(int dtype, int epi, const GemmArgs& a, cudaStream_t stream);
@@ -141,8 +142,33 @@ int launch_row_ce(const float* logits, int rows, int V, const void* tgt, int tgt
                   cudaStream_t stream);
 // ce[row] from the partials of `ntiles` column ranges, wce[row] = weight(position) * ce[row], then
 // loss = sum(wce) / (batch * windows), summed in a fixed order.  stage: 0 early, 1 late.
+// row_stats (optional, 4 floats per row): the row's merged max / exp-sum of z and of the target logits.
 int launch_ce_finalize(const float* ce_part, int ntiles, int batch, int S, int block, int offset, int sim_steps, int stage,
-                       float* ce_rows, float* wce, float* ce_out, float* loss_out, cudaStream_t stream);
+                       float* ce_rows, float* wce, float* ce_out, float* loss_out, cudaStream_t stream, float* row_stats = nullptr);
+
+// ---- block-path training step: backward (Eq. 4 / Eq. 7 and the state regression of Appendix B) ----
+// out[c][col0 + r] = in[r][c]; columns col0 + rows .. col0 + rows_pad - 1 of every output row are zeroed.
+int launch_transpose_pad(int dtype, const void* in, int rows, int cols, int ld_in, void* out, int ld_out, int col0, int rows_pad,
+                         cudaStream_t stream);
+int launch_silu_mul(int dtype, const void* gate, const void* up, void* act, size_t n, cudaStream_t stream);
+// In place: gate <- d gate, up <- d up.
+int launch_silu_mul_bwd(int dtype, void* gate, void* up, const void* dact, size_t n, cudaStream_t stream);
+// d z [row0 .. row0 + rows) = weight(position) * scale * (softmax(z) - p) from a chunk of fp32 logits; columns V..ldz-1 zeroed.
+int launch_dlogits(int dtype, const float* logits, int rows, int V, const void* tgt, int tgt_dtype, const int32_t* labels, const float* stats,
+                   int row0, int S, int block, int offset, int sim_steps, int stage, float scale, void* dz, int ldz, cudaStream_t stream);
+// dh0 = grad_coef * reg * clip(h - h_true, -1, 1); loss3[1] = vscale * sum smooth_l1, loss3[2] = loss3[0] + vcoef * loss3[1].
+int launch_vloss(int dtype, const void* h, const void* h_true, int rows, int d, int S, int block, int offset, int sim_steps, int stage,
+                 float grad_coef, float vscale, float vcoef, void* dh0, float* row_sum, float* loss3, cudaStream_t stream);
+int rmsnorm_bwd_parts(int rows);     // rows of the dg_part scratch ([parts][d] fp32)
+// out = add + d v of n = RMSNorm(v; gain) given d n (do_norm == 0: out = add + dn); dg_out (optional) = d gain.
+int launch_rmsnorm_bwd(int dtype, const void* v, const void* gain, const void* dn, const void* add, int rows, int d, float eps, int do_norm,
+                       void* out, float* dg_part, float* dg_out, cudaStream_t stream);
+int launch_embed_grad(int dtype, const int32_t* tokens, const void* dx, int rows, int d, float* dembed, cudaStream_t stream);
+// Attention backward of the block-masked cross-attention (same visibility rule as launch_attn_block).
+// lse, delta: fp32 [B*S, Hq] scratch.  dKp / dVp are written only when step > 1.
+int launch_attn_block_bwd(int dtype, const void* Q, const void* Kt, const void* Vt, const void* Kp, const void* Vp, const void* dO, int B, int S,
+                          int Hq, int Hkv, int dh, int block, int offset, int step, void* dQ, void* dKt, void* dVt, void* dKp, void* dVp,
+                          float* lse, float* delta, cudaStream_t stream);
 
 // Block-masked cross-attention: query row (b, p) reads true keys [0, n(p)) of Kt/Vt and, when
 // step > 1, predicted keys n(p) .. n(p)+min(slot, step)-2 of Kp/Vp.  All [B*S, H*dh] row-major.

@@ -237,6 +237,71 @@ def test_block_loss_forward(name, stage, sim_steps, soft):
     beagle_check_device(head_gpu.ctx)
 
 
+GRAD_TOL = {"fp32": (2e-4, 1e-5), "bf16": (4e-2, 2e-2)}     # (max error / max |ref|, Frobenius error / Frobenius norm)
+
+
+@pytest.mark.parametrize("name,stage,sim_steps,soft,vcoef", [("c1", "early", 1, True, 10.0), ("c1", "late", 3, False, 0.0),
+                                                              ("gqa", "early", 1, False, 10.0), ("gqa", "late", 4, True, 10.0),
+                                                              ("mha", "late", 2, True, 0.0)])
+def test_block_grad(name, stage, sim_steps, soft, vcoef):
+    """One training step (Eq. 4 / Eq. 7 plus the state regression of Appendix B): the three loss values and the
+    gradient in every parameter against the oracle.  fp32: tight.  bf16: the intermediate gradients are stored
+    in bf16 (relative 2^-9 each, a handful of stages deep) and each parameter gradient sums B*S of them, so the
+    error is measured against the tensor's largest entry and in Frobenius norm."""
+    w = {"c1": WL.WORKLOADS["c1_tiny_fp32"], "gqa": SMALL_GQA, "mha": SMALL_MHA}[name]
+    head_gpu, head_cpu, _ = build(w, max_slots=1, max_ctx=64)
+    rng = WL.data_rng(w, 700 + sim_steps)
+    B, S, block, offset = 2, 75, 4, 2
+    tokens = WL.make_tokens(w, rng, (B, S))
+    tokens[1, 5] = tokens[0, 7]                                            # a repeated token: its embedding rows add up
+    hidden = WL.make_hidden(w, rng, B * S).reshape(B, S, w.hidden)
+    tl = WL.round_to_storage((rng.standard_normal((B, S, w.vocab)) * 2).astype(np.float32).reshape(-1), w.dtype).reshape(B, S, w.vocab)
+    ids = WL.make_tokens(w, rng, (B, S))
+    kw = dict(target_logits=to_dev(tl, w.dtype)) if soft else dict(target_ids=to_dev(ids, w.dtype))
+    losses, grads = head_gpu.block_grad(to_dev(tokens, w.dtype), to_dev(hidden, w.dtype), block, offset, stage, sim_steps=sim_steps,
+                                        vloss_coef=vcoef, **kw)
+    torch.cuda.synchronize()
+    ref = O.block_loss_grad(head_cpu, tokens, hidden, block, offset, stage, sim_steps=sim_steps, vloss_coef=vcoef,
+                            **(dict(target_logits=tl) if soft else dict(target_ids=ids)))
+    got = losses.cpu().numpy().astype(np.float64)
+    rel = 1e-4 if w.dtype == "fp32" else 1e-2
+    assert abs(got[0] - ref["loss"]) <= rel * abs(ref["loss"])
+    assert abs(got[1] - ref["vloss"]) <= rel * abs(ref["vloss"]) + 1e-7
+    assert abs(got[2] - (got[0] + vcoef * got[1])) <= 1e-5 * abs(got[2])
+    tol_max, tol_fro = GRAD_TOL[w.dtype]
+    report = {}
+    for pname, g_ref in ref["grads"].items():
+        g = grads[pname].cpu().numpy().astype(np.float64)
+        assert g.shape == g_ref.shape and np.all(np.isfinite(g)), pname
+        scale = np.max(np.abs(g_ref))
+        assert scale > 0, pname
+        report[pname] = (np.max(np.abs(g - g_ref)) / scale, np.linalg.norm(g - g_ref) / np.linalg.norm(g_ref))
+    bad = {k: v for k, v in report.items() if v[0] > tol_max or v[1] > tol_fro}
+    assert not bad, f"gradient errors (max/max, fro/fro): {report}"
+    from paper_2505_24544_b200.binding import beagle_check_device
+    beagle_check_device(head_gpu.ctx)
+
+
+def test_block_grad_subset_and_repeatability():
+    """Only the requested gradients are written; two runs give the same bits for every fixed-order gradient."""
+    w = SMALL_GQA
+    head_gpu, _, _ = build(w, max_slots=1, max_ctx=64)
+    rng = WL.data_rng(w, 733)
+    B, S = 1, 41
+    tokens = to_dev(WL.make_tokens(w, rng, (B, S)), w.dtype)
+    hidden = to_dev(WL.make_hidden(w, rng, B * S).reshape(B, S, w.hidden), w.dtype)
+    ids = to_dev(WL.make_tokens(w, rng, (B, S)), w.dtype)
+    names = ("w_q", "w_k", "w_down", "g_mlp")
+    l1, g1 = head_gpu.block_grad(tokens, hidden, 3, 0, "late", sim_steps=2, target_ids=ids, vloss_coef=10.0, params=names)
+    l2, g2 = head_gpu.block_grad(tokens, hidden, 3, 0, "late", sim_steps=2, target_ids=ids, vloss_coef=10.0,
+                                 params=("w_q", "w_k", "w_v", "w_o", "g_q", "g_mlp", "w_gate", "w_up", "w_down", "w_lm"))
+    torch.cuda.synchronize()
+    assert set(g1) == set(names)
+    assert torch.equal(l1, l2)
+    for n in names:
+        assert torch.equal(g1[n], g2[n]), n
+
+
 def test_verify_greedy_logits_both_dtypes_and_ties():
     w = SMALL_GQA.scaled(batch=5, gamma=6)
     head_gpu, _, _ = build(w)
