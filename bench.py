@@ -468,8 +468,39 @@ def bench_block(head, w: WL.Workload, steps: int, warmup: int, peaks):
     e1.record()
     torch.cuda.synchronize()
     loss_ms = e0.elapsed_time(e1) / steps
+    # one training step (forward + backward, Eq. 4 with hard labels plus the state regression, coefficient 10):
+    # gradients of the head's own parameters (the embedding and the LM head belong to the target model)
+    own = ("g_q", "w_q", "w_k", "w_v", "w_o", "g_mlp", "w_gate", "w_up", "w_down")
+    grads = {n: torch.empty(head.weight_shapes[n], dtype=torch.float32, device=dev) for n in own}
+    losses = torch.empty(3, dtype=torch.float32, device=dev)
+
+    def train_step():
+        B.beagle_block_grad(head.ctx, tokens, hidden, w.block, 0, 1, "early", None, labels, 10.0, grads, losses)
+
+    for _ in range(2):
+        train_step()
+    torch.cuda.synchronize()
+    l0 = head.launch_count
+    e0.record()
+    for _ in range(steps):
+        train_step()
+    e1.record()
+    torch.cuda.synchronize()
+    train_ms = e0.elapsed_time(e1) / steps
+    train_launches = (head.launch_count - l0) // steps
+    B.beagle_profile_enable(head.ctx, True)
+    train_step()
+    torch.cuda.synchronize()
+    tstages = {k: {"ms": v[0], "n": v[1]} for k, v in B.beagle_profile_read(head.ctx).items()}
+    B.beagle_profile_enable(head.ctx, False)
+    # forward once, re-materialised logits once, then two products per linear layer (dX and dW; no dX for K/V inputs, no dW for the LM head)
+    train_flop = total + flops["blk_lm_head"] + flops["blk_lm_head"] + 2 * (flops["blk_gate_up"] + flops["blk_down"] + flops["blk_o_proj"]) \
+        + 2.0 * M * d * (qd + 2 * kd) + 2.0 * M * d * qd + 2.5 * flops["blk_attn"]
     return {
         "loss_forward": {"ms": loss_ms, "tflops": total / (loss_ms * 1e-3) / 1e12, "loss": float(loss.item()), "stage": "early, hard labels"},
+        "train_step": {"ms": train_ms, "tflop": train_flop / 1e12, "tflops": train_flop / (train_ms * 1e-3) / 1e12, "gpu_launches": train_launches,
+                       "positions_per_s": M / (train_ms * 1e-3), "losses": [float(x) for x in losses.tolist()], "stages": tstages,
+                       "what": "forward + backward, early stage, hard labels, vloss 10, gradients of the head's own parameters"},
         "workload": w.name, "positions_per_s": M / (ms * 1e-3), "ms_per_forward": ms, "tflop_per_forward": total / 1e12,
         "tflops": total / (ms * 1e-3) / 1e12, "gpu_launches": launches, "stages": st,
         "roofline": {"bound": "tensor", "kernel": "blk_lm_head", "achieved": lm.get("tflops"), "peak": peak, "unit": "TFLOP/s",

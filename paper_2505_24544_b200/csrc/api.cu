@@ -199,7 +199,7 @@ BlockLayout block_layout(const beagle_config& c, int batch, int S) {
 // Workspace of one training step: the forward's regions, then what the backward adds.
 struct GradLayout {
     BlockLayout fwd;
-    size_t gate, up, dact, dz, dh0, dh, dyn, dy, d_o, dq, dkt, dvt, dkp, dvp, dxn, ta, tb, wt, lse, delta, stats, vrow, dgpart, total;
+    size_t gate, up, dact, dz, dh0, dh, dyn, dy, d_o, dq, dkt, dvt, dkp, dvp, dxn, ta, tb, wt, lse, delta, stats, coef, vrow, dgpart, total;
     int Mp, Vp;        // rows and vocabulary padded to a multiple of 8 (contraction lengths of the transposed products)
 };
 GradLayout grad_layout(const beagle_config& c, int batch, int S) {
@@ -226,7 +226,7 @@ GradLayout grad_layout(const beagle_config& c, int batch, int S) {
     // one transposed weight at a time: [in, out] (hidden, mlp_dim and head_dim are multiples of 8; the vocabulary is padded)
     L.wt = take(max2(d * (size_t)L.Vp, max2(m, qd) * d) * elt);
     L.lse = take(M * c.n_q_heads * sizeof(float)); L.delta = take(M * c.n_q_heads * sizeof(float));
-    L.stats = take(M * 4 * sizeof(float)); L.vrow = take(M * sizeof(float));
+    L.stats = take(M * 4 * sizeof(float)); L.coef = take(M * sizeof(float)); L.vrow = take(M * sizeof(float));
     L.dgpart = take((size_t)rmsnorm_bwd_parts((int)M) * d * sizeof(float));
     L.total = off;
     return L;
@@ -255,7 +255,7 @@ int dense_gemm(beagle_ctx* ctx, int epi, const GemmArgs& a, cudaStream_t stream)
         const int rc = tc_gemm(ctx->tc, epi, t, stream);
         if (rc >= 0) return rc;
     }
-    if (epi == GEMM_ARGMAX_KEYS || epi == GEMM_CE) return -1;
+    if (epi == GEMM_ARGMAX_KEYS || epi == GEMM_CE || epi == GEMM_DLOGITS) return -1;
     return launch_gemm_simt(ctx->cfg.dtype, epi, a, stream);
 }
 
@@ -1088,7 +1088,19 @@ beagle_status beagle_block_grad(beagle_ctx* ctx, int32_t batch, int32_t S, const
     // ---- d z = weight * (softmax(z) - p) / (batch * windows), from re-materialised logits, chunk by chunk
     const int windows = (S - offset + block - 1) / block;
     const float ce_scale = 1.0f / ((float)batch * (float)windows);
-    {
+    bool dz_done = false;
+    if (ctx->tc != nullptr) {      // fused: the LM-head GEMM is run again and its epilogue turns the logits into d z
+        float* coef = reinterpret_cast<float*>(ws + L.coef);
+        StageTimer timer_(ctx, ST_BWD_DLOGITS, stream);
+        ctx->launches += launch_loss_coef(M, S, block, offset, sim_steps, stage, ce_scale, coef, stream);
+        memset(&g, 0, sizeof(g));
+        g.M = M; g.A = H; g.lda = d; g.K = d; g.W = ctx->w.w_lm; g.N = V; g.C = DZ; g.ldc = Vp;
+        g.tgt = target_logits_dev; g.tgt_dtype = spec.tgt_dtype; g.ldt = V; g.labels = target_ids_dev;
+        g.row_stats = reinterpret_cast<const float*>(ws + L.stats); g.row_coef = coef;
+        rc = dense_gemm(ctx, GEMM_DLOGITS, g, stream);
+        if (rc > 0) { ctx->launches += rc; dz_done = true; }
+    }
+    if (!dz_done) {
         float* chunk = reinterpret_cast<float*>(ws + F.logits);
         for (int r0 = 0; r0 < M; r0 += F.lm_chunk_rows) {
             const int rows = M - r0 < F.lm_chunk_rows ? M - r0 : F.lm_chunk_rows;

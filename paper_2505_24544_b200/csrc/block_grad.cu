@@ -37,6 +37,37 @@ __global__ void __launch_bounds__(256) transpose_pad_kernel(const T* __restrict_
     }
 }
 
+// bf16, 64 x 64 tiles, 4-byte global accesses on both sides.  ld_in, ld_out and col0 even; in / out 4-byte aligned.
+__global__ void __launch_bounds__(256) transpose_pad_bf16_kernel(const bf16* __restrict__ in, int rows, int cols, int ld_in, bf16* __restrict__ out,
+                                                                int ld_out, int col0, int rows_pad) {
+    __shared__ __align__(4) bf16 tile[64][66];
+    const int r0 = blockIdx.x * 64, c0 = blockIdx.y * 64;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const bf16 zero = __float2bfloat16_rn(0.f);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = r0 + ty + i * 8, c = c0 + 2 * tx;
+        __nv_bfloat162 v;
+        v.x = zero; v.y = zero;
+        if (r < rows) {
+            if (c + 1 < cols) v = *reinterpret_cast<const __nv_bfloat162*>(in + (size_t)r * ld_in + c);
+            else if (c < cols) v.x = in[(size_t)r * ld_in + c];
+        }
+        *reinterpret_cast<__nv_bfloat162*>(&tile[ty + i * 8][2 * tx]) = v;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int c = c0 + ty + i * 8, r = r0 + 2 * tx;
+        if (c < cols && r < rows_pad) {            // rows_pad is even: r + 1 < rows_pad as well
+            __nv_bfloat162 v;
+            v.x = tile[2 * tx][ty + i * 8];
+            v.y = tile[2 * tx + 1][ty + i * 8];
+            *reinterpret_cast<__nv_bfloat162*>(out + (size_t)c * ld_out + col0 + r) = v;
+        }
+    }
+}
+
 // act = SiLU(gate) * up, element-wise (the training forward keeps gate and up for the backward).
 template <typename T>
 __global__ void __launch_bounds__(256) silu_mul_kernel(const T* __restrict__ gate, const T* __restrict__ up, T* __restrict__ act, size_t n) {
@@ -88,6 +119,12 @@ __global__ void __launch_bounds__(256) dlogits_kernel(const float* __restrict__ 
     }
 }
 
+__global__ void __launch_bounds__(256) loss_coef_kernel(int rows, int S, int block, int offset, int sim_steps, int stage, float scale,
+                                                       float* __restrict__ coef) {
+    const int row = blockIdx.x * blockDim.x + threadIdx.x;
+    if (row < rows) coef[row] = loss_weight(row, S, block, offset, sim_steps, stage) * scale;
+}
+
 // Regression term: dh0[row] = coef * reg(row) * clip(h - h_true, -1, 1), and the row's sum of
 // smooth_l1(h - h_true) (reg(row) = 1 where the position carries a loss term).
 template <typename T>
@@ -134,51 +171,83 @@ __global__ void __launch_bounds__(1024) loss_total_kernel(const float* __restric
 // ------------------------------------------------------------------------------------------------
 // RMSNorm backward.  n = g * v * r, r = (mean(v^2) + eps)^(-1/2):
 //   dv = r * (g * dn) - v * r^3 * mean(v * g * dn);   dg = sum_rows dn * v * r.
-// out = add + dv (add may be NULL).  One warp per row; a CTA of 8 warps walks rows blockIdx.x*8+w,
-// += gridDim.x*8, keeps its dg contribution in shared memory (fixed order within the CTA) and writes
-// one partial row per CTA; colsum_kernel adds the partials in a fixed order.
-// do_norm == 0: out = add + dn, no dg.
+// out = add + dv (add may be NULL).  One CTA of 256 threads per row at a time (rows blockIdx.x,
+// += gridDim.x); a thread owns the 16-byte pieces tid, tid + 256, ... of the row (at most kRmsVec of
+// them), keeps its columns' dg sums in registers and writes them as one partial row per CTA;
+// colsum_kernel adds the partials in a fixed order.  do_norm == 0: out = add + dn, no dg.
 // ------------------------------------------------------------------------------------------------
+constexpr int kRmsVec = 4;
 template <typename T>
 __global__ void __launch_bounds__(256) rmsnorm_bwd_kernel(const T* __restrict__ v, const T* __restrict__ gain, const T* __restrict__ dn,
                                                          const T* __restrict__ add, int rows, int d, float eps, int do_norm,
                                                          T* __restrict__ out, float* __restrict__ dg_part) {
-    extern __shared__ float s_dg[];                 // [8][d]
+    constexpr int VN = VecOf<T>::N;
+    const int nvec = d / VN;
+    __shared__ float s_red[2][2][8];                // [parity][sum v^2 | sum v g dn][warp]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    float* my = s_dg + (size_t)warp * d;
-    if (do_norm && dg_part != nullptr)
-        for (int i = lane; i < d; i += 32) my[i] = 0.f;
-    for (int row = blockIdx.x * 8 + warp; row < rows; row += gridDim.x * 8) {
-        const T* vr = v + (size_t)row * d;
-        const T* dr = dn + (size_t)row * d;
-        if (!do_norm) {
-            for (int i = lane; i < d; i += 32)
-                out[(size_t)row * d + i] = from_float<T>(to_float<T>(dr[i]) + (add != nullptr ? to_float<T>(add[(size_t)row * d + i]) : 0.f));
-            continue;
-        }
+    float dg[kRmsVec][VN];
+#pragma unroll
+    for (int k = 0; k < kRmsVec; ++k)
+#pragma unroll
+        for (int i = 0; i < VN; ++i) dg[k][i] = 0.f;
+    int par = 0;
+    for (int row = blockIdx.x; row < rows; row += gridDim.x, par ^= 1) {
+        const size_t base = (size_t)row * d;
+        float x[kRmsVec][VN], gd[kRmsVec][VN], dnx[kRmsVec][VN];
         float ss = 0.f, dot = 0.f;
-        for (int i = lane; i < d; i += 32) {
-            const float x = to_float<T>(vr[i]);
-            ss = fmaf(x, x, ss);
-            dot = fmaf(x, to_float<T>(gain[i]) * to_float<T>(dr[i]), dot);
+#pragma unroll
+        for (int k = 0; k < kRmsVec; ++k) {
+            const int ch = threadIdx.x + k * 256;
+            if (ch < nvec) {
+                float dd[VN], gg[VN];
+                unpack16<T>(ld_cached16(v + base + ch * VN), x[k]);
+                unpack16<T>(ld_cached16(dn + base + ch * VN), dd);
+                if (do_norm) unpack16<T>(ld_cached16(gain + ch * VN), gg);
+#pragma unroll
+                for (int i = 0; i < VN; ++i) {
+                    gd[k][i] = do_norm ? gg[i] * dd[i] : dd[i];
+                    dnx[k][i] = dd[i] * x[k][i];
+                    ss = fmaf(x[k][i], x[k][i], ss);
+                    dot = fmaf(x[k][i], gd[k][i], dot);
+                }
+            }
         }
-        ss = warp_sum(ss); dot = warp_sum(dot);
-        const float r = rsqrtf(ss / (float)d + eps);
-        const float k = r * r * r * dot / (float)d;
-        for (int i = lane; i < d; i += 32) {
-            const float x = to_float<T>(vr[i]), g = to_float<T>(gain[i]), dd = to_float<T>(dr[i]);
-            const float dv = r * g * dd - x * k;
-            out[(size_t)row * d + i] = from_float<T>(dv + (add != nullptr ? to_float<T>(add[(size_t)row * d + i]) : 0.f));
-            if (dg_part != nullptr) my[i] += dd * x * r;
+        float r = 1.f, kfac = 0.f;
+        if (do_norm) {
+            ss = warp_sum(ss); dot = warp_sum(dot);
+            if (lane == 0) { s_red[par][0][warp] = ss; s_red[par][1][warp] = dot; }
+            __syncthreads();                        // the other parity's slots are rewritten only after the next barrier
+            float tss = 0.f, tdot = 0.f;
+#pragma unroll
+            for (int w8 = 0; w8 < 8; ++w8) { tss += s_red[par][0][w8]; tdot += s_red[par][1][w8]; }
+            r = rsqrtf(tss / (float)d + eps);
+            kfac = r * r * r * tdot / (float)d;
+        }
+#pragma unroll
+        for (int k = 0; k < kRmsVec; ++k) {
+            const int ch = threadIdx.x + k * 256;
+            if (ch < nvec) {
+                float av[VN];
+                if (add != nullptr) unpack16<T>(ld_cached16(add + base + ch * VN), av);
+                T o8[VN];
+#pragma unroll
+                for (int i = 0; i < VN; ++i) {
+                    const float dv = do_norm ? r * gd[k][i] - x[k][i] * kfac : gd[k][i];
+                    o8[i] = from_float<T>(dv + (add != nullptr ? av[i] : 0.f));
+                    dg[k][i] = fmaf(dnx[k][i], r, dg[k][i]);
+                }
+                *reinterpret_cast<uint4*>(out + base + ch * VN) = *reinterpret_cast<const uint4*>(o8);
+            }
         }
     }
     if (!do_norm || dg_part == nullptr) return;
-    __syncthreads();
-    for (int i = threadIdx.x; i < d; i += blockDim.x) {
-        float t = 0.f;
 #pragma unroll
-        for (int w = 0; w < 8; ++w) t += s_dg[(size_t)w * d + i];
-        dg_part[(size_t)blockIdx.x * d + i] = t;
+    for (int k = 0; k < kRmsVec; ++k) {
+        const int ch = threadIdx.x + k * 256;
+        if (ch < nvec) {
+#pragma unroll
+            for (int i = 0; i < VN; ++i) dg_part[(size_t)blockIdx.x * d + ch * VN + i] = dg[k][i];
+        }
     }
 }
 
@@ -348,6 +417,12 @@ inline int ew_blocks(size_t n) {
 int launch_transpose_pad(int dtype, const void* in, int rows, int cols, int ld_in, void* out, int ld_out, int col0, int rows_pad,
                          cudaStream_t stream) {
     if (rows_pad <= 0 || cols <= 0) return 0;
+    if (dtype != 0 && !(ld_in & 1) && !(ld_out & 1) && !(col0 & 1) && !(rows_pad & 1) && !(reinterpret_cast<uintptr_t>(in) & 3) &&
+        !(reinterpret_cast<uintptr_t>(out) & 3)) {
+        dim3 grid64((rows_pad + 63) / 64, (cols + 63) / 64);
+        transpose_pad_bf16_kernel<<<grid64, 256, 0, stream>>>((const bf16*)in, rows, cols, ld_in, (bf16*)out, ld_out, col0, rows_pad);
+        return 1;
+    }
     dim3 grid((rows_pad + 31) / 32, (cols + 31) / 32);
     if (dtype == 0) transpose_pad_kernel<float><<<grid, 256, 0, stream>>>((const float*)in, rows, cols, ld_in, (float*)out, ld_out, col0, rows_pad);
     else transpose_pad_kernel<bf16><<<grid, 256, 0, stream>>>((const bf16*)in, rows, cols, ld_in, (bf16*)out, ld_out, col0, rows_pad);
@@ -381,6 +456,12 @@ int launch_dlogits(int dtype, const float* logits, int rows, int V, const void* 
     return 1;
 }
 
+int launch_loss_coef(int rows, int S, int block, int offset, int sim_steps, int stage, float scale, float* coef, cudaStream_t stream) {
+    if (rows <= 0) return 0;
+    loss_coef_kernel<<<(rows + 255) / 256, 256, 0, stream>>>(rows, S, block, offset, sim_steps, stage, scale, coef);
+    return 1;
+}
+
 int launch_vloss(int dtype, const void* h, const void* h_true, int rows, int d, int S, int block, int offset, int sim_steps, int stage,
                  float grad_coef, float vscale, float vcoef, void* dh0, float* row_sum, float* loss3, cudaStream_t stream) {
     if (rows <= 0) return 0;
@@ -394,31 +475,25 @@ int launch_vloss(int dtype, const void* h, const void* h_true, int rows, int d, 
     return 2;
 }
 
-int rmsnorm_bwd_parts(int rows) { return rows < 8 * 148 ? (rows + 7) / 8 : 148; }
+int rmsnorm_bwd_parts(int rows) { return rows < 148 * 8 ? rows : 148 * 8; }
 
 int launch_rmsnorm_bwd(int dtype, const void* v, const void* gain, const void* dn, const void* add, int rows, int d, float eps, int do_norm,
                        void* out, float* dg_part, float* dg_out, cudaStream_t stream) {
     if (rows <= 0) return 0;
+    const int vn = dtype == 0 ? 4 : 8;
+    if (d % vn || d / vn > kRmsVec * 256) return -1;
     const int parts = rmsnorm_bwd_parts(rows);
-    const size_t smem = (size_t)8 * d * sizeof(float);
-    if (smem > 200 * 1024) return -1;
     float* part = (do_norm && dg_out != nullptr) ? dg_part : nullptr;
-    if (dtype == 0) {
-        static bool attr = false;
-        if (!attr) { cudaFuncSetAttribute(rmsnorm_bwd_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); attr = true; }
-        rmsnorm_bwd_kernel<float><<<parts, 256, smem, stream>>>((const float*)v, (const float*)gain, (const float*)dn, (const float*)add, rows, d,
-                                                                eps, do_norm, (float*)out, part);
-    } else {
-        static bool attr = false;
-        if (!attr) { cudaFuncSetAttribute(rmsnorm_bwd_kernel<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); attr = true; }
-        rmsnorm_bwd_kernel<bf16><<<parts, 256, smem, stream>>>((const bf16*)v, (const bf16*)gain, (const bf16*)dn, (const bf16*)add, rows, d, eps,
-                                                               do_norm, (bf16*)out, part);
-    }
+    if (dtype == 0)
+        rmsnorm_bwd_kernel<float><<<parts, 256, 0, stream>>>((const float*)v, (const float*)gain, (const float*)dn, (const float*)add, rows, d, eps,
+                                                             do_norm, (float*)out, part);
+    else
+        rmsnorm_bwd_kernel<bf16><<<parts, 256, 0, stream>>>((const bf16*)v, (const bf16*)gain, (const bf16*)dn, (const bf16*)add, rows, d, eps,
+                                                            do_norm, (bf16*)out, part);
     int n = 1;
     if (dg_out != nullptr) {
-        if (do_norm) colsum_kernel<<<(d + 255) / 256, 256, 0, stream>>>(dg_part, parts, d, dg_out);
+        if (do_norm) { colsum_kernel<<<(d + 255) / 256, 256, 0, stream>>>(dg_part, parts, d, dg_out); ++n; }
         else cudaMemsetAsync(dg_out, 0, (size_t)d * sizeof(float), stream);
-        n += do_norm ? 1 : 0;
     }
     return n;
 }

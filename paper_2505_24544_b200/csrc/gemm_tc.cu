@@ -32,7 +32,7 @@ constexpr int kTcThreads = 192;
 
 // ---------------------------------------------------------------------------------------------- kernel
 enum TcEpilogue {
-    TC_STORE = 0, TC_RESID = 1, TC_SILU_MUL = 2, TC_F32 = 3, TC_KV_CACHE = 4, TC_ARGMAX = 5, TC_CE = 6
+    TC_STORE = 0, TC_RESID = 1, TC_SILU_MUL = 2, TC_F32 = 3, TC_KV_CACHE = 4, TC_ARGMAX = 5, TC_CE = 6, TC_DLOGITS = 7
 };
 
 struct TcArgs {
@@ -44,7 +44,8 @@ struct TcArgs {
     void* cache; int Hkv, dh, cap;
     SeqRows rows;
     unsigned long long* keys; int keys_ld;
-    const void* tgt; int tgt_dtype; int ldt; const int32_t* labels; float* ce_part;   // TC_CE
+    const void* tgt; int tgt_dtype; int ldt; const int32_t* labels; float* ce_part;   // TC_CE, TC_DLOGITS
+    const float* row_stats; const float* row_coef;                                    // TC_DLOGITS
     int* error_word;
 };
 
@@ -196,8 +197,15 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
                 }
                 unsigned long long best = 0ull;
                 float ce_mq = -INFINITY, ce_sq = 0.f, ce_mt = -INFINITY, ce_st = 0.f, ce_dot = 0.f;   // TC_CE running partial
-                const int label = (EPI == TC_CE && args.tgt == nullptr && m < args.a_rows) ? args.labels[m] : -1;
+                const int label = ((EPI == TC_CE || EPI == TC_DLOGITS) && args.tgt == nullptr && m < args.a_rows) ? args.labels[m] : -1;
                 if (EPI == TC_CE && args.tgt == nullptr) ce_mt = 0.f;
+                // TC_DLOGITS: the row's softmax statistics (max z, 1 / exp-sum z, max t, 1 / exp-sum t) and loss coefficient
+                float dl_mq = 0.f, dl_iq = 0.f, dl_mt = 0.f, dl_it = 0.f, dl_coef = 0.f;
+                if (EPI == TC_DLOGITS && m < args.a_rows) {
+                    const float4 st = reinterpret_cast<const float4*>(args.row_stats)[m];
+                    dl_mq = st.x; dl_iq = 1.0f / st.y; dl_mt = st.z; dl_it = args.tgt != nullptr ? 1.0f / st.w : 0.f;
+                    dl_coef = args.row_coef[m];
+                }
                 // 16 accumulator columns of this thread's row (r, and r2 = the second matrix of a gated pair)
                 auto consume = [&](const int c0, const uint32_t* r, const uint32_t* r2) {
                     const int n0 = tb * BN + c0;
@@ -259,6 +267,32 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
 #pragma unroll
                             for (int j = 0; j < 16; ++j) v[j] = silu_f(v[j]) * __uint_as_float(r2[j]);
                         }
+                        if (EPI == TC_DLOGITS) {        // d z = coef * (softmax(z) - p)
+                            const int nv = min(16, args.b_rows - n0);
+                            float t[16];
+                            if (args.tgt != nullptr) {
+                                if (args.tgt_dtype == 0) {
+                                    const float* tp = reinterpret_cast<const float*>(args.tgt) + (size_t)m * args.ldt + n0;
+#pragma unroll
+                                    for (int j = 0; j < 16; ++j) t[j] = j < nv ? tp[j] : -INFINITY;
+                                } else {
+                                    const bf16* tp = reinterpret_cast<const bf16*>(args.tgt) + (size_t)m * args.ldt + n0;
+                                    if (full && ((reinterpret_cast<uintptr_t>(tp) & 15) == 0)) {
+                                        unpack16<bf16>(*reinterpret_cast<const uint4*>(tp), t);
+                                        unpack16<bf16>(*reinterpret_cast<const uint4*>(tp + 8), t + 8);
+                                    } else {
+#pragma unroll
+                                        for (int j = 0; j < 16; ++j) t[j] = j < nv ? __bfloat162float(tp[j]) : -INFINITY;
+                                    }
+                                }
+                            }
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                const float q = __expf(v[j] - dl_mq) * dl_iq;
+                                const float pt = args.tgt != nullptr ? __expf(t[j] - dl_mt) * dl_it : (n0 + j == label ? 1.f : 0.f);
+                                v[j] = dl_coef != 0.f ? dl_coef * (q - pt) : 0.f;
+                            }
+                        }
                         if (EPI == TC_RESID) {
                             const bf16* rp = reinterpret_cast<const bf16*>(args.R) + (size_t)m * args.ldr + n0;
                             if (full && ((reinterpret_cast<uintptr_t>(rp) & 15) == 0)) {
@@ -296,6 +330,9 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
                                     dst[j] = __float2bfloat16_rn(v[j]);
                                 }
                             }
+                            if (EPI == TC_DLOGITS)      // the padded columns of the row (b_rows .. ldc - 1) read as zero
+                                for (int j = 0; j < 16; ++j)
+                                    if (n0 + j >= args.b_rows && n0 + j < args.ldc) dst[j] = __float2bfloat16_rn(0.f);
                         }
                     }
                 };
@@ -436,6 +473,7 @@ int tc_gemm(TcPlan* p, int epi, const GemmArgs& g, cudaStream_t stream) {
     a.cache = g.cache; a.Hkv = g.Hkv; a.dh = g.dh; a.cap = g.cap; a.rows = g.rows;
     a.keys = g.keys; a.keys_ld = a.tiles_b;
     a.tgt = g.tgt; a.tgt_dtype = g.tgt_dtype; a.ldt = g.ldt; a.labels = g.labels; a.ce_part = g.ce_part;
+    a.row_stats = g.row_stats; a.row_coef = g.row_coef;
     a.error_word = g.error_word;
     if (epi == GEMM_KV_CACHE && (g.dh % 16)) return -1;
     const int ntiles = a.tiles_a * a.tiles_b;
@@ -448,6 +486,7 @@ int tc_gemm(TcPlan* p, int epi, const GemmArgs& g, cudaStream_t stream) {
         case GEMM_KV_CACHE: return launch_tc<256, false, TC_KV_CACHE>(mapA, *mapB, *mapB, a, grid, stream);
         case GEMM_ARGMAX_KEYS: return launch_tc<256, false, TC_ARGMAX>(mapA, *mapB, *mapB, a, grid, stream);
         case GEMM_CE: return launch_tc<256, false, TC_CE>(mapA, *mapB, *mapB, a, grid, stream);
+        case GEMM_DLOGITS: return launch_tc<256, false, TC_DLOGITS>(mapA, *mapB, *mapB, a, grid, stream);
         default: return -1;
     }
 }

@@ -107,7 +107,8 @@ enum GemmEpilogue {
     GEMM_F32 = 3,        // C fp32
     GEMM_KV_CACHE = 4,   // scatter rows into the cache: row r -> (slot, pos) through SeqRows
     GEMM_ARGMAX_KEYS = 5,// no C: one packed arg-max key per (row, column tile)   (tensor-core path only)
-    GEMM_CE = 6          // no C: cross-entropy partials per (row, column tile)       (tensor-core path only)
+    GEMM_CE = 6,         // no C: cross-entropy partials per (row, column tile)       (tensor-core path only)
+    GEMM_DLOGITS = 7     // C = row_coef * (softmax(A W^T) - p), storage type, from the rows' softmax statistics (tensor-core path only)
 };
 // Cross-entropy partial of one (row, column range): running max / exp-sum of the draft logits z,
 // running max / exp-sum of the target logits t and sum exp(t - tmax) * z (soft targets); with hard
@@ -130,6 +131,8 @@ struct GemmArgs {
     const void* tgt; int tgt_dtype; int ldt;   // GEMM_CE, soft targets: target logits [M, ldt] (0 fp32, 1 bf16)
     const int32_t* labels;          // GEMM_CE, hard targets: [M] (used when tgt == NULL)
     float* ce_part;                 // GEMM_CE: [M][column tiles][kCeFields]
+    const float* row_stats;         // GEMM_DLOGITS: [M][4] = max z, exp-sum z, max t, exp-sum t of every row
+    const float* row_coef;          // GEMM_DLOGITS: [M] loss weight of the row times the loss scale
     int* error_word;                // device word set to 1 when a bounded wait ran out
     int w_transient;                // W is a workspace buffer (its tensor map is not cached by pointer)
     SeqRows rows;
@@ -157,6 +160,8 @@ int launch_silu_mul_bwd(int dtype, void* gate, void* up, const void* dact, size_
 int launch_dlogits(int dtype, const float* logits, int rows, int V, const void* tgt, int tgt_dtype, const int32_t* labels, const float* stats,
                    int row0, int S, int block, int offset, int sim_steps, int stage, float scale, void* dz, int ldz, cudaStream_t stream);
 // dh0 = grad_coef * reg * clip(h - h_true, -1, 1); loss3[1] = vscale * sum smooth_l1, loss3[2] = loss3[0] + vcoef * loss3[1].
+// coef[row] = loss weight of the row's position (Eq. 4 / Eq. 7) * scale.
+int launch_loss_coef(int rows, int S, int block, int offset, int sim_steps, int stage, float scale, float* coef, cudaStream_t stream);
 int launch_vloss(int dtype, const void* h, const void* h_true, int rows, int d, int S, int block, int offset, int sim_steps, int stage,
                  float grad_coef, float vscale, float vcoef, void* dh0, float* row_sum, float* loss3, cudaStream_t stream);
 int rmsnorm_bwd_parts(int rows);     // rows of the dg_part scratch ([parts][d] fp32)

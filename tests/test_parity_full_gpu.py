@@ -290,3 +290,39 @@ def test_c5_block_forward_full_sampled_positions(llama2_heads, sim_steps):
     own = float(np.sum(ce_np * wts[None, :]) / (B * n_win))
     assert abs(float(loss.item()) - own) <= 1e-5 * abs(own)
     beagle_check_device(gpu.ctx)
+
+
+def test_c5_block_grad_full_model_dims(llama2_heads):
+    """One training step at the Llama-2-7B head's dimensions (d 4096, 32 heads x 128, m 11008, V 32000) on one
+    sequence of 1000 positions (15 query tiles and a ragged tail; window 4, offset 3; early-stage loss with soft
+    bf16 targets, state regression 10): every parameter gradient against the storage-mode oracle.  All tensor-core
+    paths run in the shapes of the benchmark (fused d-logits epilogue, transposed products, attention backward).
+    Tolerance: the forward's logits already differ from the oracle's by about 2e-2 + 1e-2 |z| at this size (bf16
+    storage), so softmax(z) - p, and with it every gradient, carries a relative error of a few percent; the gradients
+    are compared in Frobenius norm and against the tensor's largest entry."""
+    _, gpu, cpu = llama2_heads
+    from paper_2505_24544_b200.binding import beagle_check_device
+    w = WL.WORKLOADS["c5_block_llama2_7b"]
+    rng = WL.data_rng(w, 77)
+    B, S, block, offset = 1, 1000, 4, 3
+    tokens = WL.make_tokens(w, rng, (B, S))
+    hidden = WL.make_hidden(w, rng, B * S).reshape(B, S, w.hidden)
+    tl = WL.round_to_storage((rng.standard_normal((B, S, w.vocab)) * 2).astype(np.float32).reshape(-1), "bf16").reshape(B, S, w.vocab)
+    names = ("g_q", "w_q", "w_k", "w_v", "w_o", "g_mlp", "w_gate", "w_up", "w_down", "w_lm")
+    losses, grads = gpu.block_grad(to_dev(tokens, w.dtype), to_dev(hidden, w.dtype), block, offset, "early", sim_steps=1,
+                                   target_logits=to_dev(tl, "bf16"), vloss_coef=10.0, params=names)
+    torch.cuda.synchronize()
+    ref = O.block_loss_grad(cpu, tokens, hidden, block, offset, "early", sim_steps=1, target_logits=tl, vloss_coef=10.0)
+    got = losses.cpu().numpy().astype(np.float64)
+    assert abs(got[0] - ref["loss"]) <= 1e-2 * abs(ref["loss"])
+    assert abs(got[1] - ref["vloss"]) <= 1e-2 * abs(ref["vloss"])
+    report = {}
+    for n in names:
+        g = grads[n].cpu().numpy().astype(np.float64)
+        r = ref["grads"][n]
+        assert np.all(np.isfinite(g)), n
+        report[n] = (float(np.max(np.abs(g - r)) / np.max(np.abs(r))), float(np.linalg.norm(g - r) / np.linalg.norm(r)))
+    print("block_grad full dims (max/max, fro/fro):", {k: (round(a, 4), round(b, 4)) for k, (a, b) in report.items()})
+    bad = {k: v for k, v in report.items() if v[0] > 4e-2 or v[1] > 3e-2}
+    assert not bad, f"gradient errors: {report}"
+    beagle_check_device(gpu.ctx)
