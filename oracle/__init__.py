@@ -36,6 +36,7 @@ from .beagle_oracle import (  # noqa: F401
     cross_entropy_rows,
     loss_weights,
     block_loss,
+    rope_rotate,
     smooth_l1,
     rms_norm_backward,
     block_loss_grad,

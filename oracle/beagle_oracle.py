@@ -34,6 +34,14 @@ stated in the function that uses them):
   * a query with no visible key gets o = 0;
   * argmax ties go to the lowest index, NaN never wins.
 
+Positional option.  Eq. 2 has no positional term and the five workloads use
+none.  With ``HeadConfig.rope_theta > 0`` the queries and keys carry a rotary
+position embedding in the LLaMA convention ("rotate half"): within every head,
+components i and i + d_h/2 are rotated by the angle pos * theta^(-2i/d_h),
+pos = position - 1 (the query at position p uses p - 1; the key made from the
+state at position j uses j - 1, true or predicted), so a score depends on
+p - j only.  Values are not rotated.
+
 Storage mode.  By default nothing is rounded.  With ``HeadConfig.storage = "bf16"`` the
 values that a bf16 deployment keeps in memory between two operations -- the
 normalised query input, Q, the K/V cache rows, the attention output o, y, the
@@ -87,6 +95,7 @@ class HeadConfig:
     norm_q: bool = True
     norm_mlp: bool = True
     storage: Optional[str] = None   # None: never round; "bf16": round stored intermediates (module docstring)
+    rope_theta: float = 0.0         # 0: no positional term (Eq. 2 as printed); > 0: rotary embedding base (module docstring)
 
     @property
     def group(self) -> int:
@@ -168,6 +177,21 @@ def silu(u: np.ndarray) -> np.ndarray:
     return u / (1.0 + np.exp(-u))
 
 
+def rope_rotate(x: np.ndarray, pos: np.ndarray, theta: float, inverse: bool = False) -> np.ndarray:
+    """Rotary position embedding, "rotate half": x [rows, H, d_h], pos [rows] (0-based); component i < d_h/2
+    of every head pairs with component i + d_h/2 and the pair is rotated by pos * theta^(-2i/d_h)
+    (by the opposite angle when ``inverse``: the transpose of the rotation)."""
+    x = np.asarray(x, dtype=F64)
+    half = x.shape[-1] // 2
+    freq = F64(theta) ** (-2.0 * np.arange(half, dtype=F64) / x.shape[-1])
+    ang = np.asarray(pos, dtype=F64)[:, None] * freq[None, :]
+    if inverse:
+        ang = -ang
+    cs, sn = np.cos(ang)[:, None, :], np.sin(ang)[:, None, :]
+    x1, x2 = x[..., :half], x[..., half:]
+    return np.concatenate([x1 * cs - x2 * sn, x2 * cs + x1 * sn], axis=-1)
+
+
 def argmax_lowest(z: np.ndarray) -> np.ndarray:
     """Arg-max over the last axis; ties go to the lowest index, NaN never wins
     (a row of NaNs gives 0)."""
@@ -196,14 +220,19 @@ def visible_true_count(p: int, block: int, offset: int) -> int:
 
 # --------------------------------------------------------------------------- Eq. 2
 
-def project_kv(head: OracleHead, states: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+def project_kv(head: OracleHead, states: np.ndarray, pos: Optional[np.ndarray] = None) -> Tuple[np.ndarray, np.ndarray]:
     """K_j = W_K^T h_j, V_j = W_V^T h_j for every row of ``states`` [n, d].
-    Returns K, V of shape [n, Hkv, d_h]  (Eq. 2, first line)."""
+    Returns K, V of shape [n, Hkv, d_h]  (Eq. 2, first line).  ``pos`` [n]: 0-based positions of the
+    states, needed (and used) only with the rotary option: K is rotated, V is not."""
     c = head.cfg
     s = np.asarray(states, dtype=F64).reshape(-1, c.hidden)
-    k = _stored(c, s @ head.w_k.T)
-    v = _stored(c, s @ head.w_v.T)
-    return (k.reshape(-1, c.n_kv_heads, c.head_dim), v.reshape(-1, c.n_kv_heads, c.head_dim))
+    k = _stored(c, s @ head.w_k.T).reshape(-1, c.n_kv_heads, c.head_dim)
+    v = _stored(c, s @ head.w_v.T).reshape(-1, c.n_kv_heads, c.head_dim)
+    if c.rope_theta > 0:
+        if pos is None:
+            raise ValueError("the rotary option needs the states' positions")
+        k = _stored(c, rope_rotate(k, pos, c.rope_theta))
+    return k, v
 
 
 def attention_weights(head: OracleHead, q: np.ndarray, k_vis: np.ndarray) -> np.ndarray:
@@ -248,11 +277,17 @@ def embed_tokens(head: OracleHead, tokens: Sequence[int]) -> np.ndarray:
     return head.embed[tok]
 
 
-def query_projection(head: OracleHead, x: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
-    """(xq, Q): xq = RMSNorm(x; g_q) (or x when the flag is off), Q = W_Q^T xq  (Eq. 2, first line)."""
+def query_projection(head: OracleHead, x: np.ndarray, pos: Optional[np.ndarray] = None) -> Tuple[np.ndarray, np.ndarray]:
+    """(xq, Q): xq = RMSNorm(x; g_q) (or x when the flag is off), Q = W_Q^T xq  (Eq. 2, first line);
+    with the rotary option Q is rotated by the queries' 0-based positions ``pos``."""
     c = head.cfg
     xq = _stored(c, rms_norm(x, head.g_q, c.rms_eps)) if c.norm_q else np.asarray(x, dtype=F64)
-    return xq, _stored(c, xq @ head.w_q.T)
+    q = _stored(c, xq @ head.w_q.T)
+    if c.rope_theta > 0:
+        if pos is None:
+            raise ValueError("the rotary option needs the queries' positions")
+        q = _stored(c, rope_rotate(q.reshape(-1, c.n_q_heads, c.head_dim), pos, c.rope_theta).reshape(q.shape))
+    return xq, q
 
 
 def attention_rows(head: OracleHead, q: np.ndarray,
@@ -285,7 +320,7 @@ def lm_head(head: OracleHead, h: np.ndarray) -> np.ndarray:
 
 
 def draft_block(head: OracleHead, tokens: Sequence[int],
-                kv_vis: Sequence[Tuple[np.ndarray, np.ndarray]]) -> Dict[str, np.ndarray]:
+                kv_vis: Sequence[Tuple[np.ndarray, np.ndarray]], pos: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
     """The draft Transformer block (Eq. 1) and the LM head for a set of
     independent query rows.  Row r has token ``tokens[r]`` and reads the
     visible keys/values ``kv_vis[r] = (K [nv,Hkv,d_h], V [nv,Hkv,d_h])``.
@@ -295,7 +330,7 @@ def draft_block(head: OracleHead, tokens: Sequence[int],
     greedy token argmax z.
     """
     x = embed_tokens(head, tokens)                              # e(t_p)
-    xq, q = query_projection(head, x)                           # Q = W_Q^T e(t_p)
+    xq, q = query_projection(head, x, pos)                      # Q = W_Q^T e(t_p)   (pos: rotary option only)
     o = attention_rows(head, q, kv_vis)
     y = output_projection(head, o, x)                           # y = W_O^T[o] + e(t_p)
     yn, act, h = mlp_block(head, y)                             # h = MLP(y) + y
@@ -319,6 +354,7 @@ class OracleSequence:
         self.v_draft: List[np.ndarray] = []
         self.pending_h: Optional[np.ndarray] = None   # previous step's h, not yet appended
         self.pending_token: Optional[int] = None      # previous step's greedy token
+        self.steps = 0                                # draft steps since the cache was last reset to true states
 
     @property
     def n_true(self) -> int:
@@ -333,6 +369,7 @@ def rollback(seq: OracleSequence) -> None:
     """Reset the cache to true states only."""
     seq.k_draft, seq.v_draft = [], []
     seq.pending_h, seq.pending_token = None, None
+    seq.steps = 0
 
 
 def prefill_kv(head: OracleHead, seq: OracleSequence, hidden_rows: np.ndarray) -> None:
@@ -341,7 +378,7 @@ def prefill_kv(head: OracleHead, seq: OracleSequence, hidden_rows: np.ndarray) -
     rows = np.asarray(hidden_rows, dtype=F64).reshape(-1, head.cfg.hidden)
     if rows.shape[0] == 0:
         return
-    k, v = project_kv(head, rows)
+    k, v = project_kv(head, rows, np.arange(seq.n_true, seq.n_true + rows.shape[0]))
     seq.k_true = np.concatenate([seq.k_true, k], axis=0)
     seq.v_true = np.concatenate([seq.v_true, v], axis=0)
 
@@ -357,6 +394,7 @@ def draft_step(head: OracleHead, seqs: Sequence[OracleSequence],
     """
     toks: List[int] = []
     kv: List[Tuple[np.ndarray, np.ndarray]] = []
+    qpos: List[int] = []
     for b, seq in enumerate(seqs):
         if tokens_in is None:
             if seq.pending_token is None:
@@ -364,18 +402,21 @@ def draft_step(head: OracleHead, seqs: Sequence[OracleSequence],
             toks.append(int(seq.pending_token))
         else:
             toks.append(int(tokens_in[b]))
+        # the s-th step since the reset queries position n + s (0-based n + s - 1); the previous step's state sits one before it
         if seq.pending_h is not None and concat:
-            k, v = project_kv(head, seq.pending_h[None, :])
+            k, v = project_kv(head, seq.pending_h[None, :], np.array([seq.n_true + seq.steps - 1]))
             seq.k_draft.append(k[0])
             seq.v_draft.append(v[0])
         seq.pending_h = None
+        qpos.append(seq.n_true + seq.steps)
+        seq.steps += 1
         if seq.k_draft:
             k_vis = np.concatenate([seq.k_true, np.stack(seq.k_draft)], axis=0)
             v_vis = np.concatenate([seq.v_true, np.stack(seq.v_draft)], axis=0)
         else:
             k_vis, v_vis = seq.k_true, seq.v_true
         kv.append((k_vis, v_vis))
-    out = draft_block(head, toks, kv)
+    out = draft_block(head, toks, kv, np.asarray(qpos))
     for b, seq in enumerate(seqs):
         seq.pending_h = out["h"][b].copy()
         seq.pending_token = int(out["argmax"][b])
@@ -428,7 +469,7 @@ def block_forward(head: OracleHead, tokens: Sequence[int], hidden: np.ndarray, b
         need.add(p)
     active = sorted(need)
 
-    k_true, v_true = project_kv(head, hid)                       # K_j, V_j of every true state
+    k_true, v_true = project_kv(head, hid, np.arange(S))         # K_j, V_j of every true state
     k_pred: Dict[int, np.ndarray] = {}                           # position -> [Hkv, d_h]
     v_pred: Dict[int, np.ndarray] = {}
     result: Dict[int, Tuple[np.ndarray, np.ndarray, int]] = {}
@@ -443,11 +484,11 @@ def block_forward(head: OracleHead, tokens: Sequence[int], hidden: np.ndarray, b
             ks = [k_true[:n]] + [k_pred[n + r][None] for r in range(1, step)]
             vs = [v_true[:n]] + [v_pred[n + r][None] for r in range(1, step)]
             kv.append((np.concatenate(ks, axis=0), np.concatenate(vs, axis=0)))
-        out = draft_block(head, tok[[p - 1 for p in rows]], kv)
+        out = draft_block(head, tok[[p - 1 for p in rows]], kv, np.asarray([p - 1 for p in rows]))
         for r, p in enumerate(rows):
             result[p] = (out["h"][r], out["logits"][r], int(out["argmax"][r]))
             if slot_of(p) == step and step < sim_steps:
-                k, v = project_kv(head, out["h"][r][None, :])    # saved predicted state
+                k, v = project_kv(head, out["h"][r][None, :], np.array([p - 1]))    # saved predicted state
                 k_pred[p], v_pred[p] = k[0], v[0]
 
     pos = np.asarray(want, dtype=np.int64)
@@ -690,9 +731,9 @@ def block_loss_grad(head: OracleHead, tokens: np.ndarray, hidden: np.ndarray, bl
         hid = hid_all[b]
         # the states that earlier simulation steps wrote in place: constants of this step
         h_pred = block_forward(head, tok[b], hid, block, offset, sim_steps)["hidden"] if sim_steps > 1 else None
-        k_true, v_true = project_kv(head, hid)
+        k_true, v_true = project_kv(head, hid, np.arange(S))
         if h_pred is not None:
-            k_pred, v_pred = project_kv(head, h_pred)
+            k_pred, v_pred = project_kv(head, h_pred, np.arange(S))
         kv, src = [], []                                    # per position: visible (K, V) and where each row came from
         for p in range(1, S + 1):
             n = visible_true_count(p, block, offset)
@@ -702,7 +743,7 @@ def block_loss_grad(head: OracleHead, tokens: np.ndarray, hidden: np.ndarray, bl
             else:
                 kv.append((k_true[:n], v_true[:n]))
             src.append((n, extra))
-        f = draft_block(head, tok[b], kv)
+        f = draft_block(head, tok[b], kv, np.arange(S))
         x, xn, q, o, y, yn, h, z = f["x"], f["xn"], f["q"], f["o"], f["y"], f["yn"], f["h"], f["logits"]
         gate, up = yn @ head.w_gate.T, yn @ head.w_up.T
         sig = 1.0 / (1.0 + np.exp(-gate))
@@ -765,6 +806,10 @@ def block_loss_grad(head: OracleHead, tokens: np.ndarray, hidden: np.ndarray, bl
             dk_true[:n] += dk_vis[:n]; dv_true[:n] += dv_vis[:n]
             for t, row in enumerate(extra):
                 dk_pred[row] += dk_vis[n + t]; dv_pred[row] += dv_vis[n + t]
+        if c.rope_theta > 0:        # back through the rotations (orthogonal: the transpose is the opposite angle)
+            dq = rope_rotate(dq, np.arange(S), c.rope_theta, inverse=True)
+            dk_true = rope_rotate(dk_true, np.arange(S), c.rope_theta, inverse=True)
+            dk_pred = rope_rotate(dk_pred, np.arange(S), c.rope_theta, inverse=True)
         kd = c.n_kv_heads * c.head_dim
         grads["w_k"] += dk_true.reshape(S, kd).T @ hid
         grads["w_v"] += dv_true.reshape(S, kd).T @ hid
@@ -830,15 +875,18 @@ def draft_tree(head: OracleHead, seq: OracleSequence, root_token: int, depth: in
         if k < len(v):
             margin[0] = min(margin[0], float(v[k - 1] - v[k]))
 
+    n_true = k_true.shape[0]
+
     def forward(tokens, state_lists):
+        # a row that reads a draft states after the true ones is the token at 0-based position n_true + a
         kv = []
         for states in state_lists:
             if states:
-                k, v = project_kv(head, np.stack(states))
+                k, v = project_kv(head, np.stack(states), n_true + np.arange(len(states)))
                 kv.append((np.concatenate([k_true, k]), np.concatenate([v_true, v])))
             else:
                 kv.append((k_true, v_true))
-        return draft_block(head, tokens, kv)
+        return draft_block(head, tokens, kv, np.asarray([n_true + len(st) for st in state_lists]))
 
     out = forward([int(root_token)], [[]])
     h_root = out["h"][0]

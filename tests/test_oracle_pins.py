@@ -545,6 +545,56 @@ def test_block_loss_is_the_weighted_mean_of_block_forward_cross_entropies():
 
 # ----------------------------------------------------------------------------- dynamic draft tree
 
+# ----------------------------------------------------------------------------- rotary option
+
+def test_rope_rotation_by_hand_and_orthogonality():
+    # d_h = 2: one pair, frequency 1: position pi/2 turns (1, 0) into (0, 1)
+    x = np.array([[[1.0, 0.0]]])
+    np.testing.assert_allclose(O.rope_rotate(x, np.array([np.pi / 2]), 10000.0), [[[0.0, 1.0]]], atol=1e-15)
+    # d_h = 4, theta = 10000: pair (0, 2) turns by pos, pair (1, 3) by pos / 100
+    x = np.array([[[1.0, 2.0, 3.0, 4.0]]])
+    pos = 7.0
+    a, b = pos, pos / 100.0
+    want = [1 * np.cos(a) - 3 * np.sin(a), 2 * np.cos(b) - 4 * np.sin(b), 3 * np.cos(a) + 1 * np.sin(a), 4 * np.cos(b) + 2 * np.sin(b)]
+    np.testing.assert_allclose(O.rope_rotate(x, np.array([pos]), 10000.0)[0, 0], want, atol=1e-14)
+    rng = np.random.default_rng(3)
+    y = rng.normal(size=(5, 3, 8))
+    p5 = np.array([0, 1, 17, 400, 8191])
+    r = O.rope_rotate(y, p5, 500000.0)
+    np.testing.assert_allclose(r[0], y[0], atol=0)                                       # position 0: identity
+    np.testing.assert_allclose(np.linalg.norm(r, axis=-1), np.linalg.norm(y, axis=-1), rtol=1e-13)
+    np.testing.assert_allclose(O.rope_rotate(r, p5, 500000.0, inverse=True), y, atol=1e-12)
+
+
+def test_rope_scores_depend_on_relative_position_only():
+    rng = np.random.default_rng(4)
+    q, k = rng.normal(size=(1, 2, 16)), rng.normal(size=(1, 2, 16))
+    def score(p, j):
+        return np.sum(O.rope_rotate(q, np.array([p]), 10000.0) * O.rope_rotate(k, np.array([j]), 10000.0), axis=-1)
+    np.testing.assert_allclose(score(9, 4), score(109, 104), atol=1e-12)
+    np.testing.assert_allclose(score(9, 4), score(5, 0), atol=1e-12)
+    assert np.max(np.abs(score(9, 4) - score(9, 5))) > 1e-3
+
+
+@pytest.mark.parametrize("block,offset,sim_steps", [(4, 0, 4), (4, 3, 1), (3, 2, 2)])
+def test_rope_block_forward_equals_sequential_drafting(block, offset, sim_steps):
+    """With the rotary option both paths must place every query and every key (true or predicted) at the same
+    position; and the option must change the result (key order now matters)."""
+    head, w, rng = small_head(20 + block, rope_theta=10000.0)
+    S = 17
+    tokens = rng.integers(0, head.cfg.vocab, S)
+    hidden = rng.normal(size=(S, head.cfg.hidden))
+    out = O.block_forward(head, tokens, hidden, block, offset, sim_steps)
+    ref_h, ref_z = sequential_reference(head, tokens, hidden, block, offset, sim_steps)
+    np.testing.assert_allclose(out["hidden"], ref_h, atol=1e-10)
+    np.testing.assert_allclose(out["logits"], ref_z, atol=1e-10)
+    plain = O.block_forward(O.OracleHead(O.HeadConfig(*[getattr(head.cfg, f) for f in ("hidden", "n_q_heads", "n_kv_heads", "head_dim", "mlp_dim", "vocab")]), w),
+                            tokens, hidden, block, offset, sim_steps)
+    assert np.max(np.abs(plain["logits"][-1] - out["logits"][-1])) > 1e-3
+    # position 1 of a sequence has no key and position 2 one key: rotations cannot change a one-key softmax
+    np.testing.assert_allclose(plain["logits"][:2], out["logits"][:2], atol=1e-10)
+
+
 # ----------------------------------------------------------------------------- gradients of the training losses
 
 def _grad_fixture(seed, B=2, S=9, **kw):
@@ -571,11 +621,12 @@ def test_smooth_l1_and_rmsnorm_backward_by_differences():
         assert abs((f(v, gp) - f(v, gm)) / (2 * e) - dg[i]) < 1e-7
 
 
-@pytest.mark.parametrize("block,offset,labels,norms", [(3, 0, False, True), (4, 2, True, True), (2, 1, False, False)])
-def test_early_stage_gradient_is_the_derivative_of_block_loss(block, offset, labels, norms):
+@pytest.mark.parametrize("block,offset,labels,norms,theta", [(3, 0, False, True, 0.0), (4, 2, True, True, 0.0), (2, 1, False, False, 0.0),
+                                                             (3, 1, False, True, 10000.0)])
+def test_early_stage_gradient_is_the_derivative_of_block_loss(block, offset, labels, norms, theta):
     """Eq. 4: central differences of block_loss (a separate function) in every parameter tensor,
     at the entries of largest gradient magnitude and at random ones."""
-    head, w, tokens, hidden, tgt = _grad_fixture(31 + block, norm_q=norms, norm_mlp=norms)
+    head, w, tokens, hidden, tgt = _grad_fixture(31 + block, norm_q=norms, norm_mlp=norms, rope_theta=theta)
     ids = np.argmax(tgt, axis=-1)
     kw = dict(target_ids=ids) if labels else dict(target_logits=tgt)
     out = O.block_loss_grad(head, tokens, hidden, block, offset, "early", **kw)
@@ -602,8 +653,20 @@ def test_early_stage_gradient_is_the_derivative_of_block_loss(block, offset, lab
 
 def _torch_training_loss(torch, c, T, tokens, hidden, tgt, block, offset, stage, sim_steps, vcoef, pred_states):
     """An independent restatement with torch (float64, autograd): the final simulation step with the
-    predicted states given as constants."""
+    predicted states given as constants.  Rotary option in the usual rotate-half form
+    x * cos + rotate_half(x) * sin with the angles repeated over the two halves."""
     Fn = torch.nn.functional
+
+    def rope(x, pos):              # x [rows, H, d_h]
+        if c.rope_theta <= 0:
+            return x
+        half = c.head_dim // 2
+        inv = c.rope_theta ** (-torch.arange(0, half, dtype=torch.float64) * 2 / c.head_dim)
+        ang = torch.as_tensor(pos, dtype=torch.float64)[:, None] * inv[None, :]
+        emb = torch.cat([ang, ang], dim=-1)[:, None, :]
+        rot = torch.cat([-x[..., half:], x[..., :half]], dim=-1)
+        return x * emb.cos() + rot * emb.sin()
+
     B, S = tokens.shape
     w, n_windows = O.loss_weights(S, block, offset, sim_steps, stage)
     n_reg = B * int(np.count_nonzero(w))
@@ -612,7 +675,7 @@ def _torch_training_loss(torch, c, T, tokens, hidden, tgt, block, offset, stage,
     for b in range(B):
         x = T["embed"][torch.tensor(tokens[b])]
         xn = rms(x, T["g_q"]) if c.norm_q else x
-        q = Fn.linear(xn, T["w_q"]).view(S, c.n_q_heads, c.head_dim)
+        q = rope(Fn.linear(xn, T["w_q"]).view(S, c.n_q_heads, c.head_dim), np.arange(S))
         hs = torch.tensor(hidden[b])
         rows = []
         for p in range(1, S + 1):
@@ -622,7 +685,7 @@ def _torch_training_loss(torch, c, T, tokens, hidden, tgt, block, offset, stage,
             if src.shape[0] == 0:
                 rows.append(torch.zeros(c.n_q_heads * c.head_dim, dtype=torch.float64))
                 continue
-            k = Fn.linear(src, T["w_k"]).view(-1, c.n_kv_heads, c.head_dim).repeat_interleave(c.group, dim=1)
+            k = rope(Fn.linear(src, T["w_k"]).view(-1, c.n_kv_heads, c.head_dim), np.array(list(range(n)) + extra)).repeat_interleave(c.group, dim=1)
             v = Fn.linear(src, T["w_v"]).view(-1, c.n_kv_heads, c.head_dim).repeat_interleave(c.group, dim=1)
             a = torch.einsum("hd,jhd->hj", q[p - 1], k) / math.sqrt(c.head_dim)
             rows.append(torch.einsum("hj,jhd->hd", torch.softmax(a, dim=-1), v).reshape(-1))
@@ -639,13 +702,15 @@ def _torch_training_loss(torch, c, T, tokens, hidden, tgt, block, offset, stage,
     return total_l, total_v, total_l + vcoef * total_v
 
 
-@pytest.mark.parametrize("stage,block,offset,sim_steps,vcoef", [("early", 3, 1, 1, 10.0), ("late", 4, 0, 3, 10.0), ("late", 3, 2, 3, 0.0)])
-def test_training_gradients_against_torch_autograd(stage, block, offset, sim_steps, vcoef):
+@pytest.mark.parametrize("stage,block,offset,sim_steps,vcoef,theta", [("early", 3, 1, 1, 10.0, 0.0), ("late", 4, 0, 3, 10.0, 0.0),
+                                                                      ("late", 3, 2, 3, 0.0, 0.0), ("early", 4, 2, 1, 10.0, 10000.0),
+                                                                      ("late", 4, 1, 3, 0.0, 500000.0)])
+def test_training_gradients_against_torch_autograd(stage, block, offset, sim_steps, vcoef, theta):
     """Eq. 4 / Eq. 7 plus the regression term of Appendix B: every parameter's gradient against
     automatic differentiation of an independent restatement; under simulation the predicted states
     are constants there as well (they come from the oracle's own forward)."""
     torch = pytest.importorskip("torch")
-    head, w, tokens, hidden, tgt = _grad_fixture(50 + block)
+    head, w, tokens, hidden, tgt = _grad_fixture(50 + block, rope_theta=theta)
     c = head.cfg
     out = O.block_loss_grad(head, tokens, hidden, block, offset, stage, sim_steps, target_logits=tgt, vloss_coef=vcoef)
     pred = [O.block_forward(head, tokens[b], hidden[b], block, offset, sim_steps)["hidden"] for b in range(tokens.shape[0])]
