@@ -69,6 +69,12 @@ typedef struct beagle_config {
     int32_t max_slots;    /* sequences the cache holds                                             */
     int32_t max_ctx;      /* true states per sequence                                              */
     int32_t max_draft;    /* draft states appended per sequence between two resets                 */
+    float   rope_theta;   /* 0: no positional term (Eq. 2 as printed).  > 0: rotary position embedding with this base,
+                             LLaMA "rotate half" convention: inside each head, components i and i + dh/2 of Q and K are
+                             rotated by pos * theta^(-2i/dh), pos = position - 1 (0-based): the query of position p by
+                             p - 1, the key made from the state at position j (true, draft or predicted) by j - 1.  Values
+                             are not rotated.  In serve-time drafting a slot with n true states queries position
+                             n + s at the s-th beagle_draft_step since its last prefill / rollback / reset.          */
 } beagle_config;
 
 /* Device pointers, row-major [out, in], BORROWED: they must outlive the context. */

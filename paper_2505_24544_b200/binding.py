@@ -39,7 +39,7 @@ class BeagleConfig(C.Structure):
         ("hidden", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
         ("mlp_dim", C.c_int32), ("vocab", C.c_int32), ("dtype", C.c_int32), ("rms_eps", C.c_float),
         ("norm_q", C.c_int32), ("norm_mlp", C.c_int32), ("max_slots", C.c_int32), ("max_ctx", C.c_int32),
-        ("max_draft", C.c_int32),
+        ("max_draft", C.c_int32), ("rope_theta", C.c_float),
     ]
 
 
@@ -426,24 +426,24 @@ class BeagleHead:
 
     def __init__(self, *, hidden: int, n_q_heads: int, n_kv_heads: int, head_dim: int, mlp_dim: int, vocab: int,
                  dtype: str, weights: Dict[str, torch.Tensor], max_slots: int, max_ctx: int, max_draft: int,
-                 rms_eps: float = 1e-5, norm_q: bool = True, norm_mlp: bool = True):
+                 rms_eps: float = 1e-5, norm_q: bool = True, norm_mlp: bool = True, rope_theta: float = 0.0):
         code = {"fp32": BEAGLE_FP32, "bf16": BEAGLE_BF16}[dtype]
         self.cfg = BeagleConfig(hidden, n_q_heads, n_kv_heads, head_dim, mlp_dim, vocab, code, rms_eps, int(norm_q),
-                                int(norm_mlp), max_slots, max_ctx, max_draft)
+                                int(norm_mlp), max_slots, max_ctx, max_draft, float(rope_theta))
         self.ctx = Context(self.cfg, weights)
         self.weight_shapes = {n: tuple(weights[n].shape) for n in WEIGHT_NAMES}
         self.device = self.ctx.kv_buf.device
         self.dtype = torch_dtype(code)
 
     @classmethod
-    def from_workload(cls, w, weights_np, device="cuda", max_slots=None, max_ctx=None, max_draft=None) -> "BeagleHead":
+    def from_workload(cls, w, weights_np, device="cuda", max_slots=None, max_ctx=None, max_draft=None, rope_theta=0.0) -> "BeagleHead":
         """Uploads numpy float32 weights (already rounded to the storage type) and builds the head."""
         dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
         weights = {k: torch.from_numpy(v).to(device=device, dtype=dt).contiguous() for k, v in weights_np.items()}
         return cls(hidden=w.hidden, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads, head_dim=w.head_dim,
                    mlp_dim=w.mlp_dim, vocab=w.vocab, dtype=w.dtype, weights=weights,
                    max_slots=max_slots or w.batch, max_ctx=max_ctx or (w.ctx_max + 64),
-                   max_draft=max_draft or max(w.gamma, 1), rms_eps=w.rms_eps)
+                   max_draft=max_draft or max(w.gamma, 1), rms_eps=w.rms_eps, rope_theta=rope_theta)
 
     def prefill_kv(self, seq_slot, new_len, hidden):
         beagle_prefill_kv(self.ctx, seq_slot, new_len, hidden)

@@ -46,6 +46,10 @@ struct beagle_ctx {
     void* vs_scratch = nullptr;     // log-sum-exp partials and chunk masses of beagle_verify_sample
     void* tree_mem = nullptr;       // node / frontier arrays of beagle_draft_tree
     float* tree_logits = nullptr;   // [kTreeMaxTopk, V] logits of the frontier rows
+    float* rope_table = nullptr;    // (cos, sin) per (position, i < dh/2); rotary option only
+    bool rope_ready = false;
+    int rope_rows = 0;              // positions the table covers
+    std::vector<int32_t> steps;     // draft steps of a slot since its cache was last reset to true states
     int* dev_error = nullptr;       // device word raised by a kernel whose bounded wait ran out
     bool dev_error_cleared = false;
     int lm_blocks = 0;
@@ -116,6 +120,7 @@ beagle_status check_config(const beagle_config* c) {
         c->vocab <= 0 || c->max_slots <= 0 || c->max_ctx <= 0 || c->max_draft < 0)
         return BEAGLE_ERR_INVALID_ARG;
     if (!(c->rms_eps >= 0.f)) return BEAGLE_ERR_INVALID_ARG;
+    if (!(c->rope_theta >= 0.f) || (c->rope_theta > 0.f && c->rope_theta < 1.f)) return BEAGLE_ERR_INVALID_ARG;
     if (c->hidden % 8 || c->mlp_dim % 8) return BEAGLE_ERR_SHAPE;
     if (c->n_q_heads % c->n_kv_heads) return BEAGLE_ERR_SHAPE;
     const int g = c->n_q_heads / c->n_kv_heads;
@@ -127,7 +132,7 @@ beagle_status check_config(const beagle_config* c) {
 }
 
 struct ServeLayout {
-    size_t x, xn, q, o, y, yn, act, h, h_slot, hs, attn, sk_partial, last_token, ids, lm_partials, verify_keys, vs_scratch, tree_mem, tree_logits, dev_error, total;
+    size_t x, xn, q, o, y, yn, act, h, h_slot, hs, attn, sk_partial, last_token, ids, lm_partials, verify_keys, vs_scratch, tree_mem, tree_logits, rope, dev_error, total;
     int lm_blocks;
 };
 ServeLayout serve_layout(const beagle_config& c) {
@@ -163,13 +168,14 @@ ServeLayout serve_layout(const beagle_config& c) {
     L.vs_scratch = take(verify_sample_scratch_bytes((int)B, 64));
     L.tree_mem = take(tree_arrays_bytes(c.vocab));
     L.tree_logits = take(c.dtype == BEAGLE_BF16 ? (size_t)kTreeMaxTopk * c.vocab * sizeof(float) : 0);
+    L.rope = take(c.rope_theta > 0.f ? ((size_t)c.max_ctx + c.max_draft + 1) * (c.head_dim / 2) * 2 * sizeof(float) : 0);
     L.dev_error = take(256 + B * (size_t)c.n_kv_heads * sizeof(int32_t));     // error word, then the attention completion counters
     L.total = off;
     return L;
 }
 
 struct BlockLayout {
-    size_t x, xn, q, kt, vt, kp, vp, o, y, yn, act, h, logits, keys, ids, ce_part, ce_rows, wce, total;
+    size_t x, xn, q, kt, vt, kp, vp, o, y, yn, act, h, logits, keys, ids, ce_part, ce_rows, wce, rope, total;
     int lm_chunk_rows;
 };
 constexpr int kLmChunkRows = 2048;
@@ -192,6 +198,7 @@ BlockLayout block_layout(const beagle_config& c, int batch, int S) {
     L.ce_part = take(M * (size_t)tc_argmax_tiles(c.vocab) * kCeFields * sizeof(float));     // loss forward: per (row, column tile)
     L.ce_rows = take(M * sizeof(float));
     L.wce = take(M * sizeof(float));
+    L.rope = take(c.rope_theta > 0.f ? (size_t)S * (c.head_dim / 2) * 2 * sizeof(float) : 0);
     L.total = off;
     return L;
 }
@@ -244,6 +251,14 @@ void clear_error_word_once(beagle_ctx* ctx, cudaStream_t stream) {
     if (!ctx->dev_error_cleared) {
         cudaMemsetAsync(ctx->dev_error, 0, 256 + (size_t)BEAGLE_MAX_CALL_BATCH * ctx->cfg.n_kv_heads * sizeof(int32_t), stream);
         ctx->dev_error_cleared = true;
+    }
+}
+
+// Rotary option: the serve-time table is built by the first call that needs it, on that call's stream.
+void rope_table_once(beagle_ctx* ctx, cudaStream_t stream) {
+    if (ctx->cfg.rope_theta > 0.f && !ctx->rope_ready) {
+        ctx->launches += launch_rope_table(ctx->cfg.rope_theta, ctx->cfg.head_dim, ctx->rope_rows, ctx->rope_table, stream);
+        ctx->rope_ready = true;
     }
 }
 
@@ -363,11 +378,14 @@ beagle_status beagle_create(const beagle_config* cfg, const beagle_weights* w, v
     c->vs_scratch = c->ws + L.vs_scratch;
     c->tree_mem = c->ws + L.tree_mem;
     c->tree_logits = reinterpret_cast<float*>(c->ws + L.tree_logits);
+    c->rope_table = reinterpret_cast<float*>(c->ws + L.rope);
+    c->rope_rows = cfg->max_ctx + cfg->max_draft + 1;
     c->dev_error = reinterpret_cast<int*>(c->ws + L.dev_error);
     c->lm_blocks = L.lm_blocks;
     c->n_true.assign(cfg->max_slots, 0);
     c->n_draft.assign(cfg->max_slots, 0);
     c->pending.assign(cfg->max_slots, 0);
+    c->steps.assign(cfg->max_slots, 0);
     c->has_token.assign(cfg->max_slots, 0);
     int hard = 0;
     c->tc = (cfg->dtype == BEAGLE_BF16) ? tc_plan_create(*cfg, *w, &hard) : nullptr;
@@ -454,6 +472,7 @@ beagle_status beagle_rollback(beagle_ctx* ctx, int32_t batch, const int32_t* seq
         ctx->n_draft[seq_slot[b]] = 0;
         ctx->pending[seq_slot[b]] = 0;
         ctx->has_token[seq_slot[b]] = 0;
+        ctx->steps[seq_slot[b]] = 0;
     }
     return BEAGLE_OK;
 }
@@ -463,6 +482,7 @@ beagle_status beagle_reset_slot(beagle_ctx* ctx, int32_t slot) {
     if (slot < 0 || slot >= ctx->cfg.max_slots) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "slot %d out of range", slot);
     ctx->n_true[slot] = ctx->n_draft[slot] = 0;
     ctx->pending[slot] = ctx->has_token[slot] = 0;
+    ctx->steps[slot] = 0;
     return BEAGLE_OK;
 }
 
@@ -559,6 +579,10 @@ beagle_status beagle_prefill_kv(beagle_ctx* ctx, int32_t batch, const int32_t* s
             if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "V projection: unsupported shape");
             ctx->launches += rc;
         }
+        if (c.rope_theta > 0.f) {       // rotary option: the new key rows are rotated in place by their positions
+            rope_table_once(ctx, stream);
+            ctx->launches += launch_rope_cache_rows(c.dtype, ctx->kcache, total, c.n_kv_heads, c.head_dim, ctx->cap, rows, ctx->rope_table, stream);
+        }
         st = cuda_ok(ctx, "prefill_kv");
         if (st != BEAGLE_OK) return st;
     }
@@ -568,6 +592,7 @@ beagle_status beagle_prefill_kv(beagle_ctx* ctx, int32_t batch, const int32_t* s
         ctx->n_draft[s] = 0;
         ctx->pending[s] = 0;
         ctx->has_token[s] = 0;
+        ctx->steps[s] = 0;
     }
     return BEAGLE_OK;
 }
@@ -592,6 +617,11 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
             any_append = true;
         }
     }
+    if (c.rope_theta > 0.f)
+        for (int b = 0; b < batch; ++b)
+            if (ctx->n_true[seq_slot[b]] + ctx->steps[seq_slot[b]] >= ctx->rope_rows)
+                return fail(ctx, BEAGLE_ERR_CAPACITY, "slot %d: position %d exceeds max_ctx + max_draft", seq_slot[b],
+                            ctx->n_true[seq_slot[b]] + ctx->steps[seq_slot[b]] + 1);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const int dt = c.dtype;
 
@@ -668,6 +698,19 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
             a.out = ctx->q; a.ldo = ctx->qd;
             ctx->launches += launch_gemv(dt, GEMV_STORE, a, stream);
         }
+    }
+    // (3') rotary option: the s-th step since the reset queries position n + s; the state appended now sits one before it
+    if (c.rope_theta > 0.f) {
+        StageTimer timer_(ctx, ST_Q_PROJ, stream);
+        rope_table_once(ctx, stream);
+        RowMap qpos, kpos;
+        memset(&qpos, 0, sizeof(qpos)); memset(&kpos, 0, sizeof(kpos));
+        for (int b = 0; b < batch; ++b) {
+            qpos.idx[b] = ctx->n_true[seq_slot[b]] + ctx->steps[seq_slot[b]];
+            kpos.idx[b] = qpos.idx[b] > 0 ? qpos.idx[b] - 1 : 0;
+        }
+        ctx->launches += launch_rope_serve(dt, ctx->q, batch, c.n_q_heads, ctx->kcache, any_append ? batch : 0, c.n_kv_heads, c.head_dim, ctx->cap,
+                                           slots, app_pos, qpos, kpos, ctx->rope_table, stream);
     }
     // (4) o = softmax(Q K^T / sqrt(dh)) V over the cache
     {
@@ -778,6 +821,7 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
         if (concat && ctx->pending[s]) ctx->n_draft[s] += 1;
         ctx->pending[s] = 1;
         ctx->has_token[s] = 1;
+        ctx->steps[s] += 1;
     }
     return BEAGLE_OK;
 }
@@ -851,6 +895,14 @@ static beagle_status block_forward_impl(beagle_ctx* ctx, int32_t batch, int32_t 
     BEAGLE_GEMM(ST_BLK_QKV, GEMM_STORE, g, "K projection");
     g.W = ctx->w.w_v; g.C = Vt;
     BEAGLE_GEMM(ST_BLK_QKV, GEMM_STORE, g, "V projection");
+    // rotary option: position p - 1 for the query of position p and for the key of the state at position p
+    float* rope = reinterpret_cast<float*>(ws + L.rope);
+    if (c.rope_theta > 0.f) {
+        StageTimer timer_(ctx, ST_BLK_QKV, stream);
+        ctx->launches += launch_rope_table(c.rope_theta, c.head_dim, S, rope, stream);
+        ctx->launches += launch_rope_rows(dt, Q, M, c.n_q_heads, c.head_dim, S, 0, 0, rope, stream);
+        ctx->launches += launch_rope_rows(dt, Kt, M, c.n_kv_heads, c.head_dim, S, 0, 0, rope, stream);
+    }
 
     for (int step = 1; step <= sim_steps; ++step) {
         if (step > 1) {
@@ -861,6 +913,7 @@ static beagle_status block_forward_impl(beagle_ctx* ctx, int32_t batch, int32_t 
             BEAGLE_GEMM(ST_BLK_PRED_KV, GEMM_STORE, g, "predicted K projection");
             g.W = ctx->w.w_v; g.C = Vp;
             BEAGLE_GEMM(ST_BLK_PRED_KV, GEMM_STORE, g, "predicted V projection");
+            if (c.rope_theta > 0.f) ctx->launches += launch_rope_rows(dt, Kp, M, c.n_kv_heads, c.head_dim, S, 0, 0, rope, stream);
         }
         {
             StageTimer timer_(ctx, ST_BLK_ATTN, stream);
@@ -1184,6 +1237,13 @@ beagle_status beagle_block_grad(beagle_ctx* ctx, int32_t batch, int32_t S, const
         if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "block_grad: unsupported head_dim");
         ctx->launches += rc;
     }
+    if (c.rope_theta > 0.f) {      // back through the rotations: the transpose of a rotation is the opposite angle
+        StageTimer timer_(ctx, ST_BWD_ELEMENTWISE, stream);
+        const float* rope = reinterpret_cast<const float*>(ws + F.rope);
+        ctx->launches += launch_rope_rows(dt, DQ, M, c.n_q_heads, c.head_dim, S, 0, 1, rope, stream);
+        ctx->launches += launch_rope_rows(dt, DKT, M, c.n_kv_heads, c.head_dim, S, 0, 1, rope, stream);
+        if (sim_steps > 1) ctx->launches += launch_rope_rows(dt, DKP, M, c.n_kv_heads, c.head_dim, S, 0, 1, rope, stream);
+    }
     // ---- projections: dW_q = dq^T xn;  dW_k = dk_true^T h_true + dk_pred^T h_hat (same for V)
     if (grads->w_q != nullptr) {
         transpose(DQ, M, qd, qd, TA, Mp, 0, Mp);
@@ -1289,7 +1349,10 @@ beagle_status beagle_draft_tree(beagle_ctx* ctx, int32_t slot, const int32_t* ro
     const TreeArrays T = tree_arrays_carve(ctx->tree_mem, c.vocab);
     const int n_true = ctx->n_true[slot];
     // the tree starts from the true states: whatever chain-draft tail the slot had is dropped
-    ctx->n_draft[slot] = 0; ctx->pending[slot] = 0; ctx->has_token[slot] = 0;
+    ctx->n_draft[slot] = 0; ctx->pending[slot] = 0; ctx->has_token[slot] = 0; ctx->steps[slot] = 0;
+    if (c.rope_theta > 0.f && n_true + depth >= ctx->rope_rows)
+        return fail(ctx, BEAGLE_ERR_CAPACITY, "draft_tree: positions up to %d exceed max_ctx + max_draft", n_true + depth + 1);
+    rope_table_once(ctx, stream);
     const int dt = c.dtype;
     int rc = 0;
 #define BEAGLE_TREE_SKINNY(MODE, ARGS, WHAT)                                              \
@@ -1328,6 +1391,12 @@ beagle_status beagle_draft_tree(beagle_ctx* ctx, int32_t slot, const int32_t* ro
             a.W = ctx->w.w_q; a.N = ctx->qd; a.K = c.hidden; a.X = ctx->xn; a.ldx = c.hidden; a.B = rows;
             a.out = ctx->q; a.ldo = ctx->qd;
             BEAGLE_TREE_SKINNY(SK_STORE, a, "Q projection");
+        }
+        if (c.rope_theta > 0.f) {      // rotary option: the rows of forward e are tokens at position n_true + e + 1; the states appended now sit one before
+            RowMap qpos, kpos;
+            for (int b = 0; b < kMaxCallBatch; ++b) { qpos.idx[b] = n_true + e; kpos.idx[b] = n_true + (e > 0 ? e - 1 : 0); }
+            ctx->launches += launch_rope_serve(dt, ctx->q, rows, c.n_q_heads, ctx->kcache, e >= 1 ? (e == 1 ? 1 : topk) : 0, c.n_kv_heads, c.head_dim,
+                                               ctx->cap, slots, pos, qpos, kpos, ctx->rope_table, stream);
         }
         // attention: the true states (shared by the rows) in chunks, the ancestors' states as one extra chunk
         {

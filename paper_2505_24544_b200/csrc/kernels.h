@@ -99,6 +99,15 @@ int launch_attn_tail(const void* q, const void* kcache, const void* vcache, cons
 int launch_tree_verify(const int32_t* tok, const int32_t* par, int n, const int32_t* target_ids, int out_cap, int32_t* accept_len,
                        int32_t* out_tokens, int32_t* path, cudaStream_t stream);
 
+// ---- optional rotary position embedding (rotate-half; table of (cos, sin) per (position, i < dh/2)) ----
+int launch_rope_table(float theta, int dh, int npos, float* table, cudaStream_t stream);
+// Rows of a dense [rows, H*dh] matrix in place; row r sits at position pos_base + r % S; inverse: opposite angle.
+int launch_rope_rows(int dtype, void* x, long long rows, int H, int dh, int S, int pos_base, int inverse, const float* table,
+                     cudaStream_t stream);
+// One draft step: query rows b < nq at positions qpos[b]; the key rows appended for b < nk at cache row app[b] (< 0: none), position kpos[b].
+int launch_rope_serve(int dtype, void* q, int nq, int Hq, void* kcache, int nk, int Hkv, int dh, int cap, const RowMap& slot, const RowMap& app,
+                      const RowMap& qpos, const RowMap& kpos, const float* table, cudaStream_t stream);
+
 // ---- block path ------------------------------------------------------------------------------
 enum GemmEpilogue {
     GEMM_STORE = 0,      // C = A W^T                     (storage type)
@@ -138,6 +147,9 @@ struct GemmArgs {
     SeqRows rows;
 };
 int launch_gemm_simt(int dtype, int epi, const GemmArgs& a, cudaStream_t stream);
+// Key rows a prefill appended (cache row = position), rotated in place.
+int launch_rope_cache_rows(int dtype, void* kcache, long long total_rows, int Hkv, int dh, int cap, const SeqRows& rows, const float* table,
+                           cudaStream_t stream);
 
 // ---- block-path losses (Eq. 4 / Eq. 7, forward) -------------------------------------------------
 // Cross-entropy partials (one column range = the whole row) from materialised fp32 draft logits.

@@ -31,8 +31,9 @@ def tolerances(dtype: str):
     return (2e-2, 1e-2) if dtype == "bf16" else (1e-5, 1e-5)
 
 
-def oracle_head(w: WL.Workload, weights_np, storage=None) -> O.OracleHead:
-    cfg = O.HeadConfig(w.hidden, w.n_q_heads, w.n_kv_heads, w.head_dim, w.mlp_dim, w.vocab, rms_eps=w.rms_eps, storage=storage)
+def oracle_head(w: WL.Workload, weights_np, storage=None, rope_theta=0.0) -> O.OracleHead:
+    cfg = O.HeadConfig(w.hidden, w.n_q_heads, w.n_kv_heads, w.head_dim, w.mlp_dim, w.vocab, rms_eps=w.rms_eps, storage=storage,
+                       rope_theta=rope_theta)
     return O.OracleHead(cfg, weights_np)
 
 

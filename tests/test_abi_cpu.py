@@ -35,7 +35,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_config_struct_matches_header():
     from paper_2505_24544_b200.binding import BeagleConfig, BeagleWeights
-    assert C.sizeof(BeagleConfig) == 13 * 4
+    assert C.sizeof(BeagleConfig) == 14 * 4                  # 12 int32 and 2 floats, no padding
     assert C.sizeof(BeagleWeights) == 11 * C.sizeof(C.c_void_p)
 
 
@@ -58,6 +58,13 @@ def test_query_sizes_and_shape_validation(lib):
     assert lib.beagle_query_sizes(C.byref(bad), C.byref(kv), C.byref(ws)) == 2
     bad = good_config(); bad.dtype = 7
     assert lib.beagle_query_sizes(C.byref(bad), C.byref(kv), C.byref(ws)) == 1
+    # rotary option: a base below 1 (or negative) is rejected; a valid one adds the (cos, sin) table to the workspace
+    bad = good_config(); bad.rope_theta = -1.0
+    assert lib.beagle_query_sizes(C.byref(bad), C.byref(kv), C.byref(ws)) == 1
+    rope = good_config(); rope.rope_theta = 500000.0
+    ws2 = C.c_size_t()
+    assert lib.beagle_query_sizes(C.byref(rope), C.byref(kv), C.byref(ws2)) == 0
+    assert ws2.value - ws.value == (8192 + 8 + 1) * 64 * 8 + (-(8192 + 8 + 1) * 64 * 8) % 256
     bad = good_config(); bad.vocab = 0
     assert lib.beagle_query_sizes(C.byref(bad), C.byref(kv), C.byref(ws)) == 1
     n = C.c_size_t()

@@ -15,7 +15,7 @@ pytestmark = pytest.mark.gpu
 def build(w: WL.Workload, **kw):
     from paper_2505_24544_b200.binding import BeagleHead
     weights = WL.make_weights(w)
-    return BeagleHead.from_workload(w, weights, **kw), oracle_head(w, weights), weights
+    return BeagleHead.from_workload(w, weights, **kw), oracle_head(w, weights, rope_theta=kw.get("rope_theta", 0.0)), weights
 
 
 SMALL_GQA = WL.WORKLOADS["c3_llama3_8b_b1"].scaled(name="small_gqa", hidden=512, n_q_heads=8, n_kv_heads=2, head_dim=64,
@@ -57,10 +57,12 @@ def test_c1_tiny_fp32_chain_then_verify():
         assert int(acc_ref[0]) >= planted_len
 
 
+@pytest.mark.parametrize("rope", [0.0, 10000.0])
 @pytest.mark.parametrize("w", [SMALL_GQA, SMALL_MHA], ids=lambda w: w.name)
-def test_small_bf16_ragged_batch_sd_iterations(w):
-    """Several speculative-decoding iterations: draft chain, verify, append the accepted true states."""
-    head_gpu, head_cpu, _ = build(w, max_ctx=w.ctx_max + 64)
+def test_small_bf16_ragged_batch_sd_iterations(w, rope):
+    """Several speculative-decoding iterations: draft chain, verify, append the accepted true states
+    (also with the rotary option: positions continue across prefill, draft tail and reset)."""
+    head_gpu, head_cpu, _ = build(w, max_ctx=w.ctx_max + 64, rope_theta=rope)
     rng = WL.data_rng(w)
     lengths = WL.make_context_lengths(w, rng)
     lengths[0] = w.ctx_min                           # the shortest cache (1 key for the GQA case)
@@ -85,12 +87,12 @@ def test_small_bf16_ragged_batch_sd_iterations(w):
         first = np.array([out_ref[b, acc_ref[b]] for b in range(w.batch)])
 
 
-@pytest.mark.parametrize("batch", [9, 20, 40, 64])
-def test_batched_serving_tensor_core_projections(batch):
+@pytest.mark.parametrize("batch,rope", [(9, 0.0), (20, 0.0), (20, 500000.0), (40, 0.0), (64, 0.0)])
+def test_batched_serving_tensor_core_projections(batch, rope):
     """Batches above 8 rows take the tensor-core projections (weights as the wide operand, split
     reduction + finishing kernel); 9 / 20 / 40 / 64 rows cover the 16-, 32- and 64-column variants."""
     w = SMALL_GQA.scaled(batch=batch, ctx_min=3, ctx_max=300, gamma=3, seed=2003, mlp_dim=1416)
-    head_gpu, head_cpu, _ = build(w, max_ctx=w.ctx_max + 64)
+    head_gpu, head_cpu, _ = build(w, max_ctx=w.ctx_max + 64, rope_theta=rope)
     rng = WL.data_rng(w, batch)
     lengths = WL.make_context_lengths(w, rng)
     slots = list(rng.permutation(batch))                      # slot ids differ from batch rows
@@ -116,9 +118,10 @@ def test_batched_serving_tensor_core_projections(batch):
     beagle_check_device(head_gpu.ctx)
 
 
-def test_empty_cache_concat_off_and_rollback():
+@pytest.mark.parametrize("rope", [0.0, 10000.0])
+def test_empty_cache_concat_off_and_rollback(rope):
     w = SMALL_GQA.scaled(batch=2)
-    head_gpu, head_cpu, _ = build(w)
+    head_gpu, head_cpu, _ = build(w, rope_theta=rope)
     rng = WL.data_rng(w, 2)
     seqs = prefill_both(head_gpu, head_cpu, w, rng, [1, 0], [0, 300])      # slot 1 has no key at all
     first = WL.make_tokens(w, rng, (2,))
@@ -140,10 +143,11 @@ def test_split_kv_chunk_boundaries(n):
     run_chain_parity(head_gpu, head_cpu, w, [0], seqs, WL.make_tokens(w, rng, (1,)), 2)
 
 
-@pytest.mark.parametrize("block,offset,sim_steps", [(4, 0, 1), (4, 3, 1), (4, 0, 4), (4, 3, 4), (3, 1, 2), (1, 0, 1)])
-def test_block_forward_c1_fp32(block, offset, sim_steps):
+@pytest.mark.parametrize("block,offset,sim_steps,rope", [(4, 0, 1, 0.0), (4, 3, 1, 0.0), (4, 0, 4, 0.0), (4, 3, 4, 0.0), (3, 1, 2, 0.0), (1, 0, 1, 0.0),
+                                                         (4, 3, 4, 10000.0), (5, 0, 4, 0.0)])
+def test_block_forward_c1_fp32(block, offset, sim_steps, rope):
     w = WL.WORKLOADS["c1_tiny_fp32"]
-    head_gpu, head_cpu, _ = build(w)
+    head_gpu, head_cpu, _ = build(w, rope_theta=rope)
     rng = WL.data_rng(w, 10 * block + offset)
     B, S = 2, 70
     tokens = WL.make_tokens(w, rng, (B, S))
@@ -157,11 +161,12 @@ def test_block_forward_c1_fp32(block, offset, sim_steps):
         check_tokens(argmax[b].cpu().numpy(), ref["logits"], f"seq {b} argmax")
 
 
-@pytest.mark.parametrize("sim_steps", [1, 4])
-def test_block_forward_small_bf16_equals_oracle_and_sequential(sim_steps):
-    """Block forward against the oracle, and against the library's own step-by-step drafting."""
+@pytest.mark.parametrize("sim_steps,rope", [(1, 0.0), (4, 0.0), (4, 10000.0)])
+def test_block_forward_small_bf16_equals_oracle_and_sequential(sim_steps, rope):
+    """Block forward against the oracle, and against the library's own step-by-step drafting
+    (with the rotary option the two paths must also agree on every position)."""
     w = SMALL_GQA
-    head_gpu, head_cpu, _ = build(w, max_slots=1, max_ctx=256)
+    head_gpu, head_cpu, _ = build(w, max_slots=1, max_ctx=256, rope_theta=rope)
     rng = WL.data_rng(w, 77 + sim_steps)
     B, S, block, offset = 2, 131, 4, 2
     tokens = WL.make_tokens(w, rng, (B, S))
@@ -184,7 +189,7 @@ def test_block_forward_small_bf16_equals_oracle_and_sequential(sim_steps):
         assert_close(lg[0].cpu().numpy(), logits[0, n + i - 1].cpu().numpy().astype(np.float64), w.dtype, f"slot {i} block vs sequential")
 
 
-@pytest.mark.parametrize("S,block,offset,sim_steps", [(200, 5, 0, 3), (64, 2, 7, 2), (193, 3, 190, 1)])
+@pytest.mark.parametrize("S,block,offset,sim_steps", [(200, 5, 0, 3), (64, 2, 7, 2), (193, 3, 190, 1), (130, 5, 2, 4)])
 def test_block_forward_bf16_head_dim_128(S, block, offset, sim_steps):
     """Tensor-core block attention with 128-wide heads: several query/key tiles, a ragged last
     tile, an offset close to S (almost everything strict-causal) and the predicted-key band."""
@@ -240,16 +245,17 @@ def test_block_loss_forward(name, stage, sim_steps, soft):
 GRAD_TOL = {"fp32": (2e-4, 1e-5), "bf16": (4e-2, 2e-2)}     # (max error / max |ref|, Frobenius error / Frobenius norm)
 
 
-@pytest.mark.parametrize("name,stage,sim_steps,soft,vcoef", [("c1", "early", 1, True, 10.0), ("c1", "late", 3, False, 0.0),
-                                                              ("gqa", "early", 1, False, 10.0), ("gqa", "late", 4, True, 10.0),
-                                                              ("mha", "late", 2, True, 0.0)])
-def test_block_grad(name, stage, sim_steps, soft, vcoef):
+@pytest.mark.parametrize("name,stage,sim_steps,soft,vcoef,rope", [("c1", "early", 1, True, 10.0, 0.0), ("c1", "late", 3, False, 0.0, 0.0),
+                                                                   ("gqa", "early", 1, False, 10.0, 0.0), ("gqa", "late", 4, True, 10.0, 0.0),
+                                                                   ("mha", "late", 2, True, 0.0, 0.0), ("c1", "late", 2, True, 10.0, 10000.0),
+                                                                   ("mha", "late", 3, False, 10.0, 500000.0)])
+def test_block_grad(name, stage, sim_steps, soft, vcoef, rope):
     """One training step (Eq. 4 / Eq. 7 plus the state regression of Appendix B): the three loss values and the
     gradient in every parameter against the oracle.  fp32: tight.  bf16: the intermediate gradients are stored
     in bf16 (relative 2^-9 each, a handful of stages deep) and each parameter gradient sums B*S of them, so the
     error is measured against the tensor's largest entry and in Frobenius norm."""
     w = {"c1": WL.WORKLOADS["c1_tiny_fp32"], "gqa": SMALL_GQA, "mha": SMALL_MHA}[name]
-    head_gpu, head_cpu, _ = build(w, max_slots=1, max_ctx=64)
+    head_gpu, head_cpu, _ = build(w, max_slots=1, max_ctx=64, rope_theta=rope)
     rng = WL.data_rng(w, 700 + sim_steps)
     B, S, block, offset = 2, 75, 4, 2
     tokens = WL.make_tokens(w, rng, (B, S))
@@ -392,9 +398,10 @@ def tree_paths(tokens, parents, scores):
     return out
 
 
-@pytest.mark.parametrize("name,n_ctx,depth,topk,n_cand,seed", [("gqa", 300, 3, 4, 20, 908), ("mha", 130, 6, 10, 60, 904), ("gqa", 0, 2, 3, 9, 903),
-                                                                ("gqa", 77, 0, 5, 5, 900)])
-def test_draft_tree_and_tree_verification(name, n_ctx, depth, topk, n_cand, seed):
+@pytest.mark.parametrize("name,n_ctx,depth,topk,n_cand,seed,rope", [("gqa", 300, 3, 4, 20, 908, 0.0), ("mha", 130, 6, 10, 60, 904, 0.0),
+                                                                     ("gqa", 0, 2, 3, 9, 903, 0.0), ("gqa", 77, 0, 5, 5, 900, 0.0),
+                                                                     ("gqa", 300, 3, 4, 20, 908, 10000.0)])
+def test_draft_tree_and_tree_verification(name, n_ctx, depth, topk, n_cand, seed, rope):
     """Dynamic draft tree against the oracle.  Which node wins a selection is a floating-point decision
     (dozens of top-k cuts with gaps down to 1e-3), so: what is unique is compared -- every kept path's
     score against the oracle's replay of that path, the kept set itself wherever the oracle's smallest
@@ -404,7 +411,8 @@ def test_draft_tree_and_tree_verification(name, n_ctx, depth, topk, n_cand, seed
     from paper_2505_24544_b200.binding import BeagleHead
     weights = WL.make_weights(w)
     weights["w_lm"] = weights["w_lm"] * 32.0          # peaked next-token distributions (still exact in bf16)
-    head_gpu, head_cpu = BeagleHead.from_workload(w, weights, max_slots=2, max_ctx=n_ctx + 8, max_draft=64), oracle_head(w, weights)
+    head_gpu = BeagleHead.from_workload(w, weights, max_slots=2, max_ctx=n_ctx + 8, max_draft=64, rope_theta=rope)
+    head_cpu = oracle_head(w, weights, rope_theta=rope)
     rng = WL.data_rng(w, seed)
     seqs = prefill_both(head_gpu, head_cpu, w, rng, [1], [n_ctx])
     root = WL.make_tokens(w, rng, (1,))
