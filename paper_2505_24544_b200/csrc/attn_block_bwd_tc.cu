@@ -251,6 +251,7 @@ __global__ void __launch_bounds__(kWarps * 32, 2) attn_bwd_kv_tc_kernel(const __
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + 6 * kTile);
     const uint32_t barKV = smem_u32(bars), barF = barKV + 8;
     __shared__ int s_abort;
+    __shared__ float s_ls[2][kBQ], s_dl[2][kBQ];     // the query tile's log-sum-exp and delta, per stage
 
     const int kt = blockIdx.x, kvh = blockIdx.y;
     const int b = blockIdx.z / nz, pred = blockIdx.z % nz;
@@ -314,10 +315,16 @@ __global__ void __launch_bounds__(kWarps * 32, 2) attn_bwd_kv_tc_kernel(const __
     for (int it = 0; it < n_iter; ++it) {
         const int st = it & 1;
         if (threadIdx.x == 0 && it + 1 < n_iter) issue(it + 1);
-        if (ok) ok = mbar_wait(barF + 8 * st, (it >> 1) & 1, &s_abort);
-        ok = __all_sync(0xffffffffu, ok);
         const int qt = qt_lo + it / G, h = kvh * G + it % G;
         const int qb = qt * kBQ;
+        {   // this tile's row statistics (stage st was last read two iterations ago, before that iteration's closing barrier)
+            const int qi = qb + (threadIdx.x & 63);
+            const float val = qi < a.S ? (threadIdx.x < 64 ? a.lse2 : a.delta)[(size_t)(row_base + qi) * a.Hq + h] : 0.f;
+            (threadIdx.x < 64 ? s_ls : s_dl)[st][threadIdx.x & 63] = val;
+        }
+        if (ok) ok = mbar_wait(barF + 8 * st, (it >> 1) & 1, &s_abort);
+        ok = __all_sync(0xffffffffu, ok);
+        __syncthreads();
         const uint32_t sQ = sQd + st * 2 * kTile, sdO = sQ + kTile;
         if (ok) {
             float s[8][4], dp[8][4];
@@ -356,8 +363,7 @@ __global__ void __launch_bounds__(kWarps * 32, 2) attn_bwd_kv_tc_kernel(const __
                 for (int u = 0; u < 2; ++u) {
                     const int qi = qb + nt * 8 + 2 * c + u;                 // 0-based query position
                     const bool valid = qi < a.S;
-                    const size_t at = (size_t)(row_base + (valid ? qi : 0)) * a.Hq + h;
-                    const float ls = a.lse2[at], dl = a.delta[at];
+                    const float ls = s_ls[st][nt * 8 + 2 * c + u], dl = s_dl[st][nt * 8 + 2 * c + u];
                     int n = 0, hi = 0;
                     if (!full && valid) {
                         n = visible_true(qi + 1, a.block, a.offset);

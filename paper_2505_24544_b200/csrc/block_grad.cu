@@ -37,52 +37,83 @@ __global__ void __launch_bounds__(256) transpose_pad_kernel(const T* __restrict_
     }
 }
 
-// bf16, 64 x 64 tiles, 4-byte global accesses on both sides.  ld_in, ld_out and col0 even; in / out 4-byte aligned.
+// bf16, 64 x 64 tiles, 16-byte global accesses on both sides.  The tile lives in shared memory as 64 rows of eight
+// 16-byte chunks; chunk cc of row r is stored at chunk position cc ^ ((r >> 3) & 7), so that the eight rows
+// r = 8 rc + j (rc = 0..7) which one output chunk gathers from lie in different banks.
+// Needs ld_in, ld_out, col0, rows_pad multiples of 8 and 16-byte aligned bases.
 __global__ void __launch_bounds__(256) transpose_pad_bf16_kernel(const bf16* __restrict__ in, int rows, int cols, int ld_in, bf16* __restrict__ out,
                                                                 int ld_out, int col0, int rows_pad) {
-    __shared__ __align__(4) bf16 tile[64][66];
+    __shared__ __align__(16) bf16 tile[64 * 64];
     const int r0 = blockIdx.x * 64, c0 = blockIdx.y * 64;
-    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-    const bf16 zero = __float2bfloat16_rn(0.f);
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const int r = r0 + ty + i * 8, c = c0 + 2 * tx;
-        __nv_bfloat162 v;
-        v.x = zero; v.y = zero;
-        if (r < rows) {
-            if (c + 1 < cols) v = *reinterpret_cast<const __nv_bfloat162*>(in + (size_t)r * ld_in + c);
-            else if (c < cols) v.x = in[(size_t)r * ld_in + c];
+    for (int k = 0; k < 2; ++k) {
+        const int id = threadIdx.x + 256 * k;
+        const int r = id >> 3, cc = id & 7;
+        const int gr = r0 + r, gc = c0 + cc * 8;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (gr < rows) {
+            if (gc + 8 <= cols) {
+                v = *reinterpret_cast<const uint4*>(in + (size_t)gr * ld_in + gc);
+            } else if (gc < cols) {
+                bf16 e[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) e[i] = gc + i < cols ? in[(size_t)gr * ld_in + gc + i] : __float2bfloat16_rn(0.f);
+                v = *reinterpret_cast<const uint4*>(e);
+            }
         }
-        *reinterpret_cast<__nv_bfloat162*>(&tile[ty + i * 8][2 * tx]) = v;
+        *reinterpret_cast<uint4*>(tile + r * 64 + ((cc ^ ((r >> 3) & 7)) << 3)) = v;
     }
     __syncthreads();
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const int c = c0 + ty + i * 8, r = r0 + 2 * tx;
-        if (c < cols && r < rows_pad) {            // rows_pad is even: r + 1 < rows_pad as well
-            __nv_bfloat162 v;
-            v.x = tile[2 * tx][ty + i * 8];
-            v.y = tile[2 * tx + 1][ty + i * 8];
-            *reinterpret_cast<__nv_bfloat162*>(out + (size_t)c * ld_out + col0 + r) = v;
+    for (int k = 0; k < 2; ++k) {
+        const int id = threadIdx.x + 256 * k;
+        const int rc = id & 7, c = id >> 3;                 // output row c0 + c, elements r0 + 8 rc .. + 7
+        if (c0 + c < cols && r0 + rc * 8 < rows_pad) {
+            bf16 e[8];
+            const int pc = (((c >> 3) ^ rc) << 3) + (c & 7);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) e[j] = tile[(rc * 8 + j) * 64 + pc];
+            *reinterpret_cast<uint4*>(out + (size_t)(c0 + c) * ld_out + col0 + r0 + rc * 8) = *reinterpret_cast<const uint4*>(e);
         }
     }
 }
 
-// act = SiLU(gate) * up, element-wise (the training forward keeps gate and up for the backward).
+// act = SiLU(gate) * up, element-wise (the training forward keeps gate and up for the backward).  16-byte pieces; n is a
+// multiple of the vector width (mlp_dim is a multiple of 8).
 template <typename T>
 __global__ void __launch_bounds__(256) silu_mul_kernel(const T* __restrict__ gate, const T* __restrict__ up, T* __restrict__ act, size_t n) {
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
-        act[i] = from_float<T>(silu_f(to_float<T>(gate[i])) * to_float<T>(up[i]));
+    constexpr int VN = VecOf<T>::N;
+    const size_t nv = n / VN;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nv; i += (size_t)gridDim.x * blockDim.x) {
+        float g[VN], u[VN];
+        unpack16<T>(reinterpret_cast<const uint4*>(gate)[i], g);
+        unpack16<T>(reinterpret_cast<const uint4*>(up)[i], u);
+        T o[VN];
+#pragma unroll
+        for (int k = 0; k < VN; ++k) o[k] = from_float<T>(silu_f(g[k]) * u[k]);
+        reinterpret_cast<uint4*>(act)[i] = *reinterpret_cast<const uint4*>(o);
+    }
 }
 
 // In place: gate <- d gate = dact * up * sigma(gate) (1 + gate (1 - sigma(gate))), up <- d up = dact * SiLU(gate).
 template <typename T>
 __global__ void __launch_bounds__(256) silu_mul_bwd_kernel(T* __restrict__ gate, T* __restrict__ up, const T* __restrict__ dact, size_t n) {
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-        const float g = to_float<T>(gate[i]), u = to_float<T>(up[i]), da = to_float<T>(dact[i]);
-        const float sg = 1.0f / (1.0f + __expf(-g));
-        gate[i] = from_float<T>(da * u * sg * (1.0f + g * (1.0f - sg)));
-        up[i] = from_float<T>(da * g * sg);
+    constexpr int VN = VecOf<T>::N;
+    const size_t nv = n / VN;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nv; i += (size_t)gridDim.x * blockDim.x) {
+        float g[VN], u[VN], da[VN];
+        unpack16<T>(reinterpret_cast<const uint4*>(gate)[i], g);
+        unpack16<T>(reinterpret_cast<const uint4*>(up)[i], u);
+        unpack16<T>(reinterpret_cast<const uint4*>(dact)[i], da);
+        T og[VN], ou[VN];
+#pragma unroll
+        for (int k = 0; k < VN; ++k) {
+            const float sg = 1.0f / (1.0f + __expf(-g[k]));
+            og[k] = from_float<T>(da[k] * u[k] * sg * (1.0f + g[k] * (1.0f - sg)));
+            ou[k] = from_float<T>(da[k] * g[k] * sg);
+        }
+        reinterpret_cast<uint4*>(gate)[i] = *reinterpret_cast<const uint4*>(og);
+        reinterpret_cast<uint4*>(up)[i] = *reinterpret_cast<const uint4*>(ou);
     }
 }
 
@@ -177,7 +208,7 @@ __global__ void __launch_bounds__(1024) loss_total_kernel(const float* __restric
 // colsum_kernel adds the partials in a fixed order.  do_norm == 0: out = add + dn, no dg.
 // ------------------------------------------------------------------------------------------------
 constexpr int kRmsVec = 4;
-template <typename T>
+template <typename T, int NV>      // NV: 16-byte pieces per thread (d <= NV * 256 * pieces' width)
 __global__ void __launch_bounds__(256) rmsnorm_bwd_kernel(const T* __restrict__ v, const T* __restrict__ gain, const T* __restrict__ dn,
                                                          const T* __restrict__ add, int rows, int d, float eps, int do_norm,
                                                          T* __restrict__ out, float* __restrict__ dg_part) {
@@ -185,30 +216,28 @@ __global__ void __launch_bounds__(256) rmsnorm_bwd_kernel(const T* __restrict__ 
     const int nvec = d / VN;
     __shared__ float s_red[2][2][8];                // [parity][sum v^2 | sum v g dn][warp]
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    float dg[kRmsVec][VN];
+    float dg[NV][VN];
 #pragma unroll
-    for (int k = 0; k < kRmsVec; ++k)
+    for (int k = 0; k < NV; ++k)
 #pragma unroll
         for (int i = 0; i < VN; ++i) dg[k][i] = 0.f;
     int par = 0;
     for (int row = blockIdx.x; row < rows; row += gridDim.x, par ^= 1) {
         const size_t base = (size_t)row * d;
-        float x[kRmsVec][VN], gd[kRmsVec][VN], dnx[kRmsVec][VN];
+        float x[NV][VN], dd[NV][VN];
         float ss = 0.f, dot = 0.f;
 #pragma unroll
-        for (int k = 0; k < kRmsVec; ++k) {
+        for (int k = 0; k < NV; ++k) {
             const int ch = threadIdx.x + k * 256;
             if (ch < nvec) {
-                float dd[VN], gg[VN];
+                float gg[VN];
                 unpack16<T>(ld_cached16(v + base + ch * VN), x[k]);
-                unpack16<T>(ld_cached16(dn + base + ch * VN), dd);
+                unpack16<T>(ld_cached16(dn + base + ch * VN), dd[k]);
                 if (do_norm) unpack16<T>(ld_cached16(gain + ch * VN), gg);
 #pragma unroll
                 for (int i = 0; i < VN; ++i) {
-                    gd[k][i] = do_norm ? gg[i] * dd[i] : dd[i];
-                    dnx[k][i] = dd[i] * x[k][i];
                     ss = fmaf(x[k][i], x[k][i], ss);
-                    dot = fmaf(x[k][i], gd[k][i], dot);
+                    dot = fmaf(x[k][i], do_norm ? gg[i] * dd[k][i] : dd[k][i], dot);
                 }
             }
         }
@@ -224,17 +253,18 @@ __global__ void __launch_bounds__(256) rmsnorm_bwd_kernel(const T* __restrict__ 
             kfac = r * r * r * tdot / (float)d;
         }
 #pragma unroll
-        for (int k = 0; k < kRmsVec; ++k) {
+        for (int k = 0; k < NV; ++k) {
             const int ch = threadIdx.x + k * 256;
             if (ch < nvec) {
-                float av[VN];
+                float av[VN], gg[VN];
                 if (add != nullptr) unpack16<T>(ld_cached16(add + base + ch * VN), av);
+                if (do_norm) unpack16<T>(ld_cached16(gain + ch * VN), gg);
                 T o8[VN];
 #pragma unroll
                 for (int i = 0; i < VN; ++i) {
-                    const float dv = do_norm ? r * gd[k][i] - x[k][i] * kfac : gd[k][i];
+                    const float dv = do_norm ? r * gg[i] * dd[k][i] - x[k][i] * kfac : dd[k][i];
                     o8[i] = from_float<T>(dv + (add != nullptr ? av[i] : 0.f));
-                    dg[k][i] = fmaf(dnx[k][i], r, dg[k][i]);
+                    dg[k][i] = fmaf(dd[k][i] * x[k][i], r, dg[k][i]);
                 }
                 *reinterpret_cast<uint4*>(out + base + ch * VN) = *reinterpret_cast<const uint4*>(o8);
             }
@@ -242,7 +272,7 @@ __global__ void __launch_bounds__(256) rmsnorm_bwd_kernel(const T* __restrict__ 
     }
     if (!do_norm || dg_part == nullptr) return;
 #pragma unroll
-    for (int k = 0; k < kRmsVec; ++k) {
+    for (int k = 0; k < NV; ++k) {
         const int ch = threadIdx.x + k * 256;
         if (ch < nvec) {
 #pragma unroll
@@ -407,8 +437,8 @@ __global__ void __launch_bounds__(128) attn_block_bwd_kv_kernel(const T* __restr
     }
 }
 
-inline int ew_blocks(size_t n) {
-    const size_t b = (n + 255) / 256;
+inline int ew_blocks(size_t n) {      // n elements, eight (four) per thread
+    const size_t b = (n / 4 + 255) / 256 + 1;
     return (int)(b < 148 * 16 ? b : 148 * 16);
 }
 
@@ -417,8 +447,8 @@ inline int ew_blocks(size_t n) {
 int launch_transpose_pad(int dtype, const void* in, int rows, int cols, int ld_in, void* out, int ld_out, int col0, int rows_pad,
                          cudaStream_t stream) {
     if (rows_pad <= 0 || cols <= 0) return 0;
-    if (dtype != 0 && !(ld_in & 1) && !(ld_out & 1) && !(col0 & 1) && !(rows_pad & 1) && !(reinterpret_cast<uintptr_t>(in) & 3) &&
-        !(reinterpret_cast<uintptr_t>(out) & 3)) {
+    if (dtype != 0 && !(ld_in & 7) && !(ld_out & 7) && !(col0 & 7) && !(rows_pad & 7) && !(reinterpret_cast<uintptr_t>(in) & 15) &&
+        !(reinterpret_cast<uintptr_t>(out) & 15)) {
         dim3 grid64((rows_pad + 63) / 64, (cols + 63) / 64);
         transpose_pad_bf16_kernel<<<grid64, 256, 0, stream>>>((const bf16*)in, rows, cols, ld_in, (bf16*)out, ld_out, col0, rows_pad);
         return 1;
@@ -482,14 +512,15 @@ int launch_rmsnorm_bwd(int dtype, const void* v, const void* gain, const void* d
     if (rows <= 0) return 0;
     const int vn = dtype == 0 ? 4 : 8;
     if (d % vn || d / vn > kRmsVec * 256) return -1;
+    const int nv = (d / vn + 255) / 256;            // 16-byte pieces per thread
     const int parts = rmsnorm_bwd_parts(rows);
     float* part = (do_norm && dg_out != nullptr) ? dg_part : nullptr;
-    if (dtype == 0)
-        rmsnorm_bwd_kernel<float><<<parts, 256, 0, stream>>>((const float*)v, (const float*)gain, (const float*)dn, (const float*)add, rows, d, eps,
-                                                             do_norm, (float*)out, part);
-    else
-        rmsnorm_bwd_kernel<bf16><<<parts, 256, 0, stream>>>((const bf16*)v, (const bf16*)gain, (const bf16*)dn, (const bf16*)add, rows, d, eps,
-                                                            do_norm, (bf16*)out, part);
+#define BEAGLE_RMS(T, NV)                                                                                                              \
+    rmsnorm_bwd_kernel<T, NV><<<parts, 256, 0, stream>>>((const T*)v, (const T*)gain, (const T*)dn, (const T*)add, rows, d, eps, do_norm, \
+                                                         (T*)out, part)
+    if (dtype == 0) { if (nv <= 1) BEAGLE_RMS(float, 1); else if (nv == 2) BEAGLE_RMS(float, 2); else BEAGLE_RMS(float, 4); }
+    else { if (nv <= 1) BEAGLE_RMS(bf16, 1); else if (nv == 2) BEAGLE_RMS(bf16, 2); else BEAGLE_RMS(bf16, 4); }
+#undef BEAGLE_RMS
     int n = 1;
     if (dg_out != nullptr) {
         if (do_norm) { colsum_kernel<<<(d + 255) / 256, 256, 0, stream>>>(dg_part, parts, d, dg_out); ++n; }
