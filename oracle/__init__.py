@@ -21,6 +21,7 @@ from .beagle_oracle import (  # noqa: F401
     attention_rows,
     output_projection,
     mlp_block,
+    down_projection,
     lm_head,
     draft_block,
     prefill_kv,

@@ -306,12 +306,17 @@ def output_projection(head: OracleHead, o: np.ndarray, x: np.ndarray) -> np.ndar
     return _stored(head.cfg, o @ head.w_o.T + x)
 
 
+def down_projection(head: OracleHead, act: np.ndarray, y: np.ndarray) -> np.ndarray:
+    """h = W_down act + y: the MLP's last matrix and the residual of Eq. 1."""
+    return _stored(head.cfg, np.asarray(act, dtype=F64) @ head.w_down.T + y)
+
+
 def mlp_block(head: OracleHead, y: np.ndarray) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
     """(yn, act, h): yn = RMSNorm(y; g_mlp), act = SiLU(W_gate yn) * (W_up yn), h = W_down act + y  (Eq. 1)."""
     c = head.cfg
     yn = _stored(c, rms_norm(y, head.g_mlp, c.rms_eps)) if c.norm_mlp else np.asarray(y, dtype=F64)
     act = _stored(c, silu(yn @ head.w_gate.T) * (yn @ head.w_up.T))
-    return yn, act, _stored(c, act @ head.w_down.T + y)
+    return yn, act, down_projection(head, act, y)
 
 
 def lm_head(head: OracleHead, h: np.ndarray) -> np.ndarray:

@@ -157,7 +157,8 @@ def serve_stage_parity(head_gpu, head_cpu: O.OracleHead, w: WL.Workload, slots, 
     yn_ref, act_ref, h_ref = O.mlp_block(head_cpu, buf["y"])
     assert_close(buf["yn"], yn_ref, dt, "stage yn")
     assert_close(buf["act"], act_ref, dt, "stage act")
-    assert_close(buf["h"], h_ref, dt, "stage h")
+    assert_close(buf["h"], h_ref, dt, "stage h (gate/up + down from the library's y)")
+    assert_close(buf["h"], O.down_projection(head_cpu, buf["act"], buf["y"]), dt, "stage h (down projection of the library's act)")
     z_ref = O.lm_head(head_cpu, buf["h"])
     if logits_gpu is not None:
         err = np.abs(_np(logits_gpu) - z_ref)
