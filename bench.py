@@ -277,15 +277,17 @@ def time_serve_e2e(scn: ServeScenario, steps: int, warmup: int, world: int):
     scn.reset()
     new_len = [1] * w.batch
     h2d = d2h = 0
+    seq_row0 = np.arange(w.batch, dtype=np.int64) * (w.gamma + 1)      # first row of every sequence in host_hidden[it]
 
     def one(it, count):
         nonlocal new_len, h2d, d2h
         if it > 0:
-            r = 0
-            for b in range(w.batch):                       # pack the accepted rows of every sequence
-                n = new_len[b]
-                stage_h[r:r + n].copy_(host_hidden[it, b * (w.gamma + 1): b * (w.gamma + 1) + n])
-                r += n
+            # pack the accepted rows of every sequence into the pinned staging buffer with one gather
+            counts = np.asarray(new_len, dtype=np.int64)
+            r = int(counts.sum())
+            first_row = np.cumsum(counts) - counts
+            idx = np.repeat(seq_row0 - first_row, counts) + np.arange(r)
+            torch.index_select(host_hidden[it], 0, torch.from_numpy(idx), out=stage_h[:r])
             dev_h[:r].copy_(stage_h[:r], non_blocking=True)
             if count:
                 h2d += r * w.hidden * stage_h.element_size()
