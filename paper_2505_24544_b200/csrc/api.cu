@@ -175,7 +175,8 @@ ServeLayout serve_layout(const beagle_config& c) {
 }
 
 struct BlockLayout {
-    size_t x, xn, q, kt, vt, kp, vp, o, y, yn, act, h, logits, keys, ids, ce_part, ce_rows, wce, rope, total;
+    size_t x, xn, q, kt, vt, kp, vp, vtT, vpT, o, y, yn, act, h, logits, keys, ids, ce_part, ce_rows, wce, rope, total;
+    int Sp;             // positions per sequence padded to a multiple of 8 (columns of a sequence in the transposed values)
     int lm_chunk_rows;
 };
 constexpr int kLmChunkRows = 2048;
@@ -188,6 +189,9 @@ BlockLayout block_layout(const beagle_config& c, int batch, int S) {
     auto take = [&](size_t bytes) { size_t at = off; off = align_up(off + bytes); return at; };
     L.x = take(M * d * elt); L.xn = take(M * d * elt); L.q = take(M * qd * elt);
     L.kt = take(M * kd * elt); L.vt = take(M * kd * elt); L.kp = take(M * kd * elt); L.vp = take(M * kd * elt);
+    L.Sp = (S + 7) / 8 * 8;
+    const size_t vT = c.dtype == BEAGLE_BF16 ? kd * (size_t)batch * L.Sp * elt : 0;       // V^T for the tcgen05 attention
+    L.vtT = take(vT); L.vpT = take(vT);
     L.o = take(M * qd * elt); L.y = take(M * d * elt); L.yn = take(M * d * elt);
     L.act = take(M * m * elt); L.h = take(M * d * elt);
     L.lm_chunk_rows = (int)(M < (size_t)kLmChunkRows ? M : (size_t)kLmChunkRows);
@@ -921,8 +925,22 @@ static beagle_status block_forward_impl(beagle_ctx* ctx, int32_t batch, int32_t 
             if (ctx->tc != nullptr) {       // bf16, head_dim 64 / 128: tensor-core tiles
                 clear_error_word_once(ctx, stream);
                 float* lse2 = (loss != nullptr && step == sim_steps) ? loss->lse2 : nullptr;
-                rc = tc_attn_block(ctx->tc, Q, Kt, Vt, Kp, Vp, batch, S, c.n_q_heads, c.n_kv_heads, c.head_dim, block, offset, step, O,
-                                   ctx->dev_error, stream, lse2);
+                if (c.head_dim == 64 || c.head_dim == 128) {
+                    // tcgen05 path: it consumes the values transposed (keys contiguous), one padded column block per sequence
+                    void *VtT = ws + L.vtT, *VpT = ws + L.vpT;
+                    const int ldT = batch * L.Sp;
+                    int nt = 0;
+                    if (step == 1)
+                        nt += launch_transpose_pad_batched(dt, Vt, S, ctx->kd, ctx->kd, (size_t)S * ctx->kd, VtT, ldT, 0, L.Sp, L.Sp, batch, stream);
+                    if (step > 1)
+                        nt += launch_transpose_pad_batched(dt, Vp, S, ctx->kd, ctx->kd, (size_t)S * ctx->kd, VpT, ldT, 0, L.Sp, L.Sp, batch, stream);
+                    rc = tc_attn_block_umma(ctx->tc, Q, Kt, VtT, Kp, step > 1 ? VpT : VtT, batch, S, L.Sp, c.n_q_heads, c.n_kv_heads, c.head_dim,
+                                            block, offset, step, O, ctx->dev_error, stream, lse2);
+                    if (rc >= 0) rc += nt; else ctx->launches += nt;
+                }
+                if (rc < 0)
+                    rc = tc_attn_block(ctx->tc, Q, Kt, Vt, Kp, Vp, batch, S, c.n_q_heads, c.n_kv_heads, c.head_dim, block, offset, step, O,
+                                       ctx->dev_error, stream, lse2);
                 if (rc >= 0 && lse2 != nullptr) loss->lse2_written = true;
             }
             if (rc < 0)

@@ -18,10 +18,13 @@ namespace {
 // every output row are zero-filled (the contraction length is padded to a multiple of 8).
 // 32 x 32 tiles through shared memory.
 // ------------------------------------------------------------------------------------------------
+// blockIdx.z = batch: the input advances by in_bs elements and the output column offset by col_bs per batch.
 template <typename T>
 __global__ void __launch_bounds__(256) transpose_pad_kernel(const T* __restrict__ in, int rows, int cols, int ld_in, T* __restrict__ out,
-                                                           int ld_out, int col0, int rows_pad) {
+                                                           int ld_out, int col0, int rows_pad, size_t in_bs, int col_bs) {
     __shared__ T tile[32][33];
+    in += (size_t)blockIdx.z * in_bs;
+    col0 += (int)blockIdx.z * col_bs;
     const int r0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;     // 8 rows of 32 threads
 #pragma unroll
@@ -42,8 +45,10 @@ __global__ void __launch_bounds__(256) transpose_pad_kernel(const T* __restrict_
 // r = 8 rc + j (rc = 0..7) which one output chunk gathers from lie in different banks.
 // Needs ld_in, ld_out, col0, rows_pad multiples of 8 and 16-byte aligned bases.
 __global__ void __launch_bounds__(256) transpose_pad_bf16_kernel(const bf16* __restrict__ in, int rows, int cols, int ld_in, bf16* __restrict__ out,
-                                                                int ld_out, int col0, int rows_pad) {
+                                                                int ld_out, int col0, int rows_pad, size_t in_bs, int col_bs) {
     __shared__ __align__(16) bf16 tile[64 * 64];
+    in += (size_t)blockIdx.z * in_bs;
+    col0 += (int)blockIdx.z * col_bs;
     const int r0 = blockIdx.x * 64, c0 = blockIdx.y * 64;
 #pragma unroll
     for (int k = 0; k < 2; ++k) {
@@ -444,19 +449,29 @@ inline int ew_blocks(size_t n) {      // n elements, eight (four) per thread
 
 }  // namespace
 
-int launch_transpose_pad(int dtype, const void* in, int rows, int cols, int ld_in, void* out, int ld_out, int col0, int rows_pad,
-                         cudaStream_t stream) {
-    if (rows_pad <= 0 || cols <= 0) return 0;
-    if (dtype != 0 && !(ld_in & 7) && !(ld_out & 7) && !(col0 & 7) && !(rows_pad & 7) && !(reinterpret_cast<uintptr_t>(in) & 15) &&
-        !(reinterpret_cast<uintptr_t>(out) & 15)) {
-        dim3 grid64((rows_pad + 63) / 64, (cols + 63) / 64);
-        transpose_pad_bf16_kernel<<<grid64, 256, 0, stream>>>((const bf16*)in, rows, cols, ld_in, (bf16*)out, ld_out, col0, rows_pad);
+int launch_transpose_pad_batched(int dtype, const void* in, int rows, int cols, int ld_in, size_t in_batch_stride, void* out, int ld_out, int col0,
+                                 int col_batch_stride, int rows_pad, int nbatch, cudaStream_t stream) {
+    if (rows_pad <= 0 || cols <= 0 || nbatch <= 0) return 0;
+    if (dtype != 0 && !(ld_in & 7) && !(ld_out & 7) && !(col0 & 7) && !(rows_pad & 7) && !(in_batch_stride & 7) && !(col_batch_stride & 7) &&
+        !(reinterpret_cast<uintptr_t>(in) & 15) && !(reinterpret_cast<uintptr_t>(out) & 15)) {
+        dim3 grid64((rows_pad + 63) / 64, (cols + 63) / 64, nbatch);
+        transpose_pad_bf16_kernel<<<grid64, 256, 0, stream>>>((const bf16*)in, rows, cols, ld_in, (bf16*)out, ld_out, col0, rows_pad, in_batch_stride,
+                                                              col_batch_stride);
         return 1;
     }
-    dim3 grid((rows_pad + 31) / 32, (cols + 31) / 32);
-    if (dtype == 0) transpose_pad_kernel<float><<<grid, 256, 0, stream>>>((const float*)in, rows, cols, ld_in, (float*)out, ld_out, col0, rows_pad);
-    else transpose_pad_kernel<bf16><<<grid, 256, 0, stream>>>((const bf16*)in, rows, cols, ld_in, (bf16*)out, ld_out, col0, rows_pad);
+    dim3 grid((rows_pad + 31) / 32, (cols + 31) / 32, nbatch);
+    if (dtype == 0)
+        transpose_pad_kernel<float><<<grid, 256, 0, stream>>>((const float*)in, rows, cols, ld_in, (float*)out, ld_out, col0, rows_pad, in_batch_stride,
+                                                              col_batch_stride);
+    else
+        transpose_pad_kernel<bf16><<<grid, 256, 0, stream>>>((const bf16*)in, rows, cols, ld_in, (bf16*)out, ld_out, col0, rows_pad, in_batch_stride,
+                                                             col_batch_stride);
     return 1;
+}
+
+int launch_transpose_pad(int dtype, const void* in, int rows, int cols, int ld_in, void* out, int ld_out, int col0, int rows_pad,
+                         cudaStream_t stream) {
+    return launch_transpose_pad_batched(dtype, in, rows, cols, ld_in, 0, out, ld_out, col0, 0, rows_pad, 1, stream);
 }
 
 int launch_silu_mul(int dtype, const void* gate, const void* up, void* act, size_t n, cudaStream_t stream) {

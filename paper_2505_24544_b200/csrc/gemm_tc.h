@@ -66,6 +66,10 @@ int tc_attn_block(TcPlan* plan, const void* Q, const void* Kt, const void* Vt, c
                   int Hq, int Hkv, int dh, int block, int offset, int step, void* O, int* error_word, cudaStream_t stream,
                   float* lse2 = nullptr);
 // lse2 (optional, fp32 [B*S, Hq]): base-2 log-sum-exp of every row's scaled scores, for the backward below.
+// The same on tcgen05 (both products as tcgen05.mma, accumulators in tensor memory).  VtT / VpT: the values TRANSPOSED,
+// [Hkv*dh, B*Sp] with sequence b's position j at column b*Sp + j, Sp >= S a multiple of 8 (padding columns finite).
+int tc_attn_block_umma(TcPlan* plan, const void* Q, const void* Kt, const void* VtT, const void* Kp, const void* VpT, int B, int S, int Sp, int Hq,
+                       int Hkv, int dh, int block, int offset, int step, void* O, int* error_word, cudaStream_t stream, float* lse2 = nullptr);
 // Backward (same contract as launch_attn_block_bwd, bf16, head_dim 64 / 128); delta: fp32 [B*S, Hq] scratch.
 int tc_attn_block_bwd(TcPlan* plan, const void* Q, const void* Kt, const void* Vt, const void* Kp, const void* Vp, const void* O, const void* dO,
                       const float* lse2, int B, int S, int Hq, int Hkv, int dh, int block, int offset, int step, float* delta, void* dQ,

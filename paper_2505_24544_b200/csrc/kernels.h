@@ -165,6 +165,9 @@ int launch_ce_finalize(const float* ce_part, int ntiles, int batch, int S, int b
 // out[c][col0 + r] = in[r][c]; columns col0 + rows .. col0 + rows_pad - 1 of every output row are zeroed.
 int launch_transpose_pad(int dtype, const void* in, int rows, int cols, int ld_in, void* out, int ld_out, int col0, int rows_pad,
                          cudaStream_t stream);
+// The same for `nbatch` matrices: matrix z starts at in + z * in_batch_stride and lands at column col0 + z * col_batch_stride.
+int launch_transpose_pad_batched(int dtype, const void* in, int rows, int cols, int ld_in, size_t in_batch_stride, void* out, int ld_out, int col0,
+                                 int col_batch_stride, int rows_pad, int nbatch, cudaStream_t stream);
 int launch_silu_mul(int dtype, const void* gate, const void* up, void* act, size_t n, cudaStream_t stream);
 // In place: gate <- d gate, up <- d up.
 int launch_silu_mul_bwd(int dtype, void* gate, void* up, const void* dact, size_t n, cudaStream_t stream);
