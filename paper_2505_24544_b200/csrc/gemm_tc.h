@@ -75,4 +75,11 @@ int tc_attn_block_bwd(TcPlan* plan, const void* Q, const void* Kt, const void* V
                       const float* lse2, int B, int S, int Hq, int Hkv, int dh, int block, int offset, int step, float* delta, void* dQ,
                       void* dKt, void* dVt, void* dKp, void* dVp, int* error_word, cudaStream_t stream);
 
+// Attention backward on tcgen05.  QT / dOT: [Hq*dh, B*Sp], KtT / KpT: [Hkv*dh, B*Sp] transposed copies (sequence b's position j at
+// column b*Sp + j, Sp a multiple of 8); everything else as tc_attn_block_bwd.
+int tc_attn_block_bwd_umma(TcPlan* plan, const void* Q, const void* Kt, const void* Vt, const void* Kp, const void* Vp, const void* O,
+                           const void* dO, const float* lse2, const void* QT, const void* dOT, const void* KtT, const void* KpT, int B, int S,
+                           int Sp, int Hq, int Hkv, int dh, int block, int offset, int step, float* delta, void* dQ, void* dKt, void* dVt,
+                           void* dKp, void* dVp, int* error_word, cudaStream_t stream);
+
 }  // namespace beagle
