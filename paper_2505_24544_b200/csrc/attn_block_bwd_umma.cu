@@ -297,35 +297,35 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kv_umma_kernel(const 
             const bool full = !pred && qb + kBS <= a.S && nvis(qb + 1, a.block, a.offset) >= kt0 + kBM;
             uint32_t pk_p[16], pk_ds[16];
             const uint32_t ts = tmem_base + st * 128 + lane_off + 32 * half;
+            uint32_t rs[2][16], rd[2][16];
+#pragma unroll
+            for (int c = 0; c < 2; ++c) { tmem_ld16(ts + 16 * c, rs[c]); tmem_ld16(ts + kBS + 16 * c, rd[c]); }
+            tmem_ld_wait();
+            fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(s_empty + 8 * st);        // this warp's part of the buffer is in registers
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
-                uint32_t rs[16], rd[16];
-                tmem_ld16(ts + 16 * c, rs);
-                tmem_ld16(ts + kBS + 16 * c, rd);
-                tmem_ld_wait();
 #pragma unroll
                 for (int i = 0; i < 16; i += 2) {
                     float pv[2], dv[2];
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
                         const int col = 32 * half + 16 * c + i + u;
-                        float p = exp2f(fmaf(__uint_as_float(rs[i + u]), a.scale_log2, -s_ls[st][col]));
+                        float p = exp2f(fmaf(__uint_as_float(rs[c][i + u]), a.scale_log2, -s_ls[st][col]));
                         if (!full) {
                             const int n = s_n[st][col], hi = s_hi[st][col];
                             const bool vis = pred ? (key >= n && key < hi) : (key < n);
                             p = vis ? p : 0.f;
                         }
                         pv[u] = p;
-                        dv[u] = p * (__uint_as_float(rd[i + u]) - s_dl[st][col]);
+                        dv[u] = p * (__uint_as_float(rd[c][i + u]) - s_dl[st][col]);
                     }
                     const __nv_bfloat162 tp = __floats2bfloat162_rn(pv[0], pv[1]), td = __floats2bfloat162_rn(dv[0], dv[1]);
                     pk_p[(16 * c + i) >> 1] = *reinterpret_cast<const uint32_t*>(&tp);
                     pk_ds[(16 * c + i) >> 1] = *reinterpret_cast<const uint32_t*>(&td);
                 }
             }
-            fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(s_empty + 8 * st);        // this warp's quarter of the buffer has been read
             if (ok) ok = mbar_wait(p_empty, (j & 1) ^ 1, s_abort);   // the previous tile's products have read the operand tiles
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) continue;
@@ -547,29 +547,29 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_q_umma_kernel(const _
             const int lo = pred ? n_row : 0, hi = pred ? hi_row : n_row;
             uint32_t pk[16];
             const uint32_t ts = tmem_base + st * 128 + lane_off + 32 * half;
+            uint32_t rs[2][16], rd[2][16];
+#pragma unroll
+            for (int c = 0; c < 2; ++c) { tmem_ld16(ts + 16 * c, rs[c]); tmem_ld16(ts + kBS + 16 * c, rd[c]); }
+            tmem_ld_wait();
+            fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(s_empty + 8 * st);        // this warp's part of the buffer is in registers
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
-                uint32_t rs[16], rd[16];
-                tmem_ld16(ts + 16 * c, rs);
-                tmem_ld16(ts + kBS + 16 * c, rd);
-                tmem_ld_wait();
 #pragma unroll
                 for (int i = 0; i < 16; i += 2) {
                     float dv[2];
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
                         const int key = kt0 + 32 * half + 16 * c + i + u;
-                        float p = exp2f(fmaf(__uint_as_float(rs[i + u]), a.scale_log2, -ls));
+                        float p = exp2f(fmaf(__uint_as_float(rs[c][i + u]), a.scale_log2, -ls));
                         if (!full) p = (key >= lo && key < hi) ? p : 0.f;
-                        dv[u] = p * (__uint_as_float(rd[i + u]) - dl);
+                        dv[u] = p * (__uint_as_float(rd[c][i + u]) - dl);
                     }
                     const __nv_bfloat162 td = __floats2bfloat162_rn(dv[0], dv[1]);
                     pk[(16 * c + i) >> 1] = *reinterpret_cast<const uint32_t*>(&td);
                 }
             }
-            fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(s_empty + 8 * st);
             if (ok) ok = mbar_wait(p_empty, (j & 1) ^ 1, s_abort);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
