@@ -286,12 +286,23 @@ __global__ void __launch_bounds__(256) rmsnorm_bwd_kernel(const T* __restrict__ 
     }
 }
 
+// out[i] = sum over the partial rows, in a fixed order: a CTA owns 32 columns, its 8 warps take the partial rows
+// w, w + 8, ... (lane = column), and the 8 warp sums are added in warp order.
 __global__ void __launch_bounds__(256) colsum_kernel(const float* __restrict__ part, int nparts, int d, float* __restrict__ out) {
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= d) return;
+    __shared__ float s[8][32];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int i = blockIdx.x * 32 + lane;
     float t = 0.f;
-    for (int p = 0; p < nparts; ++p) t += part[(size_t)p * d + i];
-    out[i] = t;
+    if (i < d)
+        for (int p = warp; p < nparts; p += 8) t += part[(size_t)p * d + i];
+    s[warp][lane] = t;
+    __syncthreads();
+    if (warp == 0 && i < d) {
+        float r = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) r += s[w][lane];
+        out[i] = r;
+    }
 }
 
 // d embed[token[row]] += dx[row]   (fp32 atomics: the order of the additions is not fixed)
@@ -538,7 +549,7 @@ int launch_rmsnorm_bwd(int dtype, const void* v, const void* gain, const void* d
 #undef BEAGLE_RMS
     int n = 1;
     if (dg_out != nullptr) {
-        if (do_norm) { colsum_kernel<<<(d + 255) / 256, 256, 0, stream>>>(dg_part, parts, d, dg_out); ++n; }
+        if (do_norm) { colsum_kernel<<<(d + 31) / 32, 256, 0, stream>>>(dg_part, parts, d, dg_out); ++n; }
         else cudaMemsetAsync(dg_out, 0, (size_t)d * sizeof(float), stream);
     }
     return n;
