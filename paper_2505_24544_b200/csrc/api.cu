@@ -941,9 +941,6 @@ static beagle_status block_forward_impl(beagle_ctx* ctx, int32_t batch, int32_t 
                                             block, offset, step, O, ctx->dev_error, stream, lse2);
                     if (rc >= 0) rc += nt; else ctx->launches += nt;
                 }
-                if (rc < 0)
-                    rc = tc_attn_block(ctx->tc, Q, Kt, Vt, Kp, Vp, batch, S, c.n_q_heads, c.n_kv_heads, c.head_dim, block, offset, step, O,
-                                       ctx->dev_error, stream, lse2);
                 if (rc >= 0 && lse2 != nullptr) loss->lse2_written = true;
             }
             if (rc < 0)
@@ -1262,9 +1259,6 @@ beagle_status beagle_block_grad(beagle_ctx* ctx, int32_t batch, int32_t S, const
                                         c.n_q_heads, c.n_kv_heads, c.head_dim, block, offset, sim_steps, reinterpret_cast<float*>(ws + L.delta), DQ,
                                         DKT, DVT, DKP, DVP, ctx->dev_error, stream);
         }
-        if (rc < 0 && spec.lse2_written)
-            rc = tc_attn_block_bwd(ctx->tc, Q, Kt, Vt, Kp, Vp_, O, DO, spec.lse2, batch, S, c.n_q_heads, c.n_kv_heads, c.head_dim, block, offset,
-                                   sim_steps, reinterpret_cast<float*>(ws + L.delta), DQ, DKT, DVT, DKP, DVP, ctx->dev_error, stream);
         if (rc < 0)
             rc = launch_attn_block_bwd(dt, Q, Kt, Vt, Kp, Vp_, DO, batch, S, c.n_q_heads, c.n_kv_heads, c.head_dim, block, offset, sim_steps, DQ,
                                        DKT, DVT, DKP, DVP, reinterpret_cast<float*>(ws + L.lse), reinterpret_cast<float*>(ws + L.delta), stream);
