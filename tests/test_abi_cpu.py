@@ -70,6 +70,11 @@ def test_query_sizes_and_shape_validation(lib):
     n = C.c_size_t()
     assert lib.beagle_block_workspace_bytes(C.byref(cfg), 8, 2048, C.byref(n)) == 0 and n.value > 0
     assert lib.beagle_block_workspace_bytes(C.byref(cfg), 0, 2048, C.byref(n)) == 1
+    # the training step's workspace contains the forward's
+    g = C.c_size_t()
+    assert lib.beagle_block_grad_workspace_bytes(C.byref(cfg), 8, 2048, C.byref(g)) == 0 and g.value > n.value and g.value % 256 == 0
+    assert lib.beagle_block_grad_workspace_bytes(C.byref(cfg), 8, 0, C.byref(g)) == 1
+    assert lib.beagle_block_grad_workspace_bytes(C.byref(cfg), 1 << 13, 1 << 13, C.byref(g)) == 3       # more than 2^24 positions
 
 
 def test_null_context_is_rejected(lib):
@@ -77,6 +82,10 @@ def test_null_context_is_rejected(lib):
     assert lib.beagle_draft_step(None, 0, None, None, 1, None, 1, None, None, None) == 1
     assert lib.beagle_verify_greedy(None, 0, 0, None, None, 0, None, None, None, None) == 1
     assert lib.beagle_block_forward(None, 1, 1, None, None, 1, 0, 1, None, None, None, None, 0, None) == 1
+    assert lib.beagle_block_loss(None, 1, 1, None, None, 1, 0, 1, 0, None, 0, None, None, None, None, 0, None) == 1
+    assert lib.beagle_block_grad(None, 1, 1, None, None, 1, 0, 1, 0, None, 0, None, 0.0, None, None, None, 0, None) == 1
+    assert lib.beagle_verify_sample(None, 0, 0, None, None, None, 0, 1.0, None, None, None, None, None) == 1
+    assert lib.beagle_draft_tree(None, 0, None, 1, 1, 1, None, None, None, None) == 1
     assert lib.beagle_destroy(None) == 1
     assert lib.beagle_version().decode().startswith("beagle")
 

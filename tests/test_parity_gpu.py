@@ -563,3 +563,30 @@ def test_status_codes_for_capacity_and_state():
         head_gpu.draft_step([0, 0], tokens_in=torch.zeros(2, dtype=torch.int32, device="cuda"))
     assert e.value.status == 1
     torch.cuda.synchronize()
+
+
+def test_status_codes_of_the_training_entry_points():
+    """Argument errors of beagle_block_loss / beagle_block_grad are reported before any launch."""
+    from paper_2505_24544_b200.binding import BeagleError
+    w = SMALL_GQA
+    head_gpu, _, _ = build(w, max_slots=1, max_ctx=16)
+    rng = WL.data_rng(w, 11)
+    tokens = to_dev(WL.make_tokens(w, rng, (1, 12)), w.dtype)
+    hidden = to_dev(WL.make_hidden(w, rng, 12).reshape(1, 12, w.hidden), w.dtype)
+    ids = to_dev(WL.make_tokens(w, rng, (1, 12)), w.dtype)
+    tl = torch.zeros(1, 12, w.vocab, dtype=torch.float32, device="cuda")
+    for kw in (dict(stage="early", sim_steps=2, target_ids=ids),                 # the early stage has no simulation
+               dict(stage="late", sim_steps=5, target_ids=ids),                  # sim_steps > block
+               dict(stage="late", sim_steps=2),                                  # no target at all
+               dict(stage="late", sim_steps=2, target_ids=ids, target_logits=tl),   # both targets
+               dict(stage="late", sim_steps=2, target_ids=ids, vloss_coef=-1.0)):
+        with pytest.raises(BeagleError) as e:
+            head_gpu.block_grad(tokens, hidden, 4, 0, **kw)
+        assert e.value.status == 1, kw
+    with pytest.raises(BeagleError) as e:
+        head_gpu.block_loss(tokens, hidden, 4, 12, "early", target_ids=ids)      # offset must lie inside the sequence
+    assert e.value.status == 1
+    # and a valid call still works afterwards
+    losses, grads = head_gpu.block_grad(tokens, hidden, 4, 0, "late", sim_steps=2, target_ids=ids, vloss_coef=10.0, params=("w_o",))
+    torch.cuda.synchronize()
+    assert torch.isfinite(losses).all() and torch.isfinite(grads["w_o"]).all()
