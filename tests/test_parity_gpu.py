@@ -590,3 +590,40 @@ def test_status_codes_of_the_training_entry_points():
     losses, grads = head_gpu.block_grad(tokens, hidden, 4, 0, "late", sim_steps=2, target_ids=ids, vloss_coef=10.0, params=("w_o",))
     torch.cuda.synchronize()
     assert torch.isfinite(losses).all() and torch.isfinite(grads["w_o"]).all()
+
+
+@pytest.mark.parametrize("name,S,block,offset,sim_steps", [("gqa", 1, 1, 0, 1), ("gqa", 2, 4, 0, 2), ("mha", 127, 4, 0, 4), ("mha", 128, 3, 1, 3),
+                                                           ("gqa", 129, 5, 128, 2), ("gqa", 257, 4, 3, 4)])
+def test_block_forward_and_grad_tile_edges(name, S, block, offset, sim_steps):
+    """Sequence lengths around the 128-query / 64-key tiles of the tensor-core attention kernels (and the degenerate
+    S = 1, where no query sees a key): forward logits and one training step against the oracle."""
+    w = {"gqa": SMALL_GQA, "mha": SMALL_MHA}[name]
+    head_gpu, head_cpu, _ = build(w, max_slots=1, max_ctx=64)
+    rng = WL.data_rng(w, 900 + S)
+    B = 2
+    tokens = WL.make_tokens(w, rng, (B, S))
+    hidden = WL.make_hidden(w, rng, B * S).reshape(B, S, w.hidden)
+    ids = WL.make_tokens(w, rng, (B, S))
+    tok_dev, hid_dev = to_dev(tokens, w.dtype), to_dev(hidden, w.dtype)
+    logits, argmax, hid = head_gpu.block_forward(tok_dev, hid_dev, block, offset, sim_steps)
+    torch.cuda.synchronize()
+    for b in range(B):
+        ref = O.block_forward(head_cpu, tokens[b], hidden[b], block, offset, sim_steps)
+        assert_close(logits[b].cpu().numpy(), ref["logits"], w.dtype, f"seq {b} logits")
+        check_tokens(argmax[b].cpu().numpy(), ref["logits"], f"seq {b} argmax")
+    losses, grads = head_gpu.block_grad(tok_dev, hid_dev, block, offset, "late", sim_steps=sim_steps, target_ids=to_dev(ids, w.dtype),
+                                        vloss_coef=10.0)
+    torch.cuda.synchronize()
+    ref = O.block_loss_grad(head_cpu, tokens, hidden, block, offset, "late", sim_steps=sim_steps, target_ids=ids, vloss_coef=10.0)
+    assert abs(float(losses[0]) - ref["loss"]) <= 1e-2 * abs(ref["loss"]) + 1e-6
+    tol_max, tol_fro = GRAD_TOL[w.dtype]
+    for pname, g_ref in ref["grads"].items():
+        g = grads[pname].cpu().numpy().astype(np.float64)
+        scale = np.max(np.abs(g_ref))
+        if scale == 0:       # no key, or a single key (softmax of one score is constant): no gradient reaches the query side
+            assert np.max(np.abs(g)) <= 1e-8, pname      # the GPU's is rounding residue of delta = dO . bf16(O) against dO . V
+            continue
+        assert np.max(np.abs(g - g_ref)) <= tol_max * scale, (pname, np.max(np.abs(g - g_ref)) / scale)
+        assert np.linalg.norm(g - g_ref) <= tol_fro * np.linalg.norm(g_ref), pname
+    from paper_2505_24544_b200.binding import beagle_check_device
+    beagle_check_device(head_gpu.ctx)
