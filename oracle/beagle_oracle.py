@@ -53,6 +53,9 @@ at the full model sizes the rounding of the cache alone moves logits of
 standard deviation ~2.7 by up to ~5e-2, so a comparison that wants to see
 kernel errors rather than storage noise has to round at the same places.
 
+FP8 option (not in the paper): lm_head_fp8 is the LM head with weights and incoming
+states quantised row-wise to FP8 E4M3; round_e4m3 follows the published format.
+
 Speculative-sampling verification (verify_sample) follows Section 3 literally;
 the random numbers it needs are inputs.
 
@@ -153,6 +156,40 @@ def round_bf16(a: np.ndarray) -> np.ndarray:
     lsb = (u >> drop) & np.uint64(1)
     r = (u + ((np.uint64(1) << (drop - np.uint64(1))) - np.uint64(1)) + lsb) & ~((np.uint64(1) << drop) - np.uint64(1))
     return r.view(F64).reshape(a.shape)
+
+
+def round_e4m3(a: np.ndarray) -> np.ndarray:
+    """Round to the nearest FP8 E4M3 value (the OCP 8-bit format "e4m3fn": 4 exponent bits with bias 7, 3 fraction
+    bits, no infinities, largest magnitude 448, subnormal step 2^-9), ties to even, magnitudes above 448 saturate
+    to 448.  Returned as float64 (every E4M3 value is exactly representable)."""
+    a = np.asarray(a, dtype=F64)
+    mag = np.abs(a)
+    with np.errstate(divide="ignore"):
+        e = np.floor(np.log2(np.where(mag > 0, mag, 1.0)))
+    e = np.maximum(e, -6.0)                               # below 2^-6 the spacing stays that of the subnormals
+    step = np.exp2(e - 3.0)                               # 3 fraction bits
+    q = np.rint(mag / step) * step                        # numpy rounds halves to even
+    return np.sign(a) * np.minimum(q, 448.0)
+
+
+def quantize_rows_e4m3(x: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
+    """Row-wise FP8 quantisation as the optional FP8 LM head uses it: scale_r = max|x_r| / 448 (1 for a zero row),
+    q_r = round_e4m3(x_r / scale_r), so that x_r ~ scale_r * q_r.  The scale and the quotient are formed in
+    float32 -- the quantised code is an integer decision, taken in the precision the kernel takes it in.
+    Returns (q as float64 values, scale as float64)."""
+    x32 = np.asarray(x, dtype=np.float32)
+    amax = np.max(np.abs(x32), axis=-1, keepdims=True)
+    scale = np.where(amax > 0, amax / np.float32(448.0), np.float32(1.0)).astype(np.float32)
+    q = round_e4m3((x32 / scale).astype(np.float32).astype(F64))
+    return q, scale[..., 0].astype(F64)
+
+
+def lm_head_fp8(head: "OracleHead", h: np.ndarray) -> np.ndarray:
+    """Logits with the LM head's weights and the incoming states both quantised row-wise to FP8 E4M3:
+    z[b, v] = scale_h[b] * scale_w[v] * sum_i q_h[b, i] q_w[v, i]."""
+    qh, sh = quantize_rows_e4m3(np.asarray(h, dtype=F64))
+    qw, sw = quantize_rows_e4m3(head.w_lm)
+    return (qh @ qw.T) * sh[:, None] * sw[None, :]
 
 
 def _stored(cfg: "HeadConfig", a: np.ndarray) -> np.ndarray:

@@ -881,3 +881,40 @@ def test_workload_shapes_and_determinism():
     w4 = WL.WORKLOADS["c4_llama3_8b_b32"]
     n = WL.make_context_lengths(w4, WL.data_rng(w4))
     assert n.shape == (32,) and n.min() >= 512 and n.max() <= 8192
+
+
+# ----------------------------------------------------------------------------- FP8 option
+
+def test_round_e4m3_hand_values_and_torch():
+    """E4M3 by its definition: spacing 2^(e-3) in [2^e, 2^(e+1)), subnormal step 2^-9, largest value 448, ties to even."""
+    x = np.array([0.0, 1.0, 1.0625, 1.1875, 1.3125, 17.0, 18.0, 19.0, 448.0, 1000.0, -460.0, 2.0 ** -9, 2.0 ** -10, 1.5 * 2.0 ** -9, 0.0179])
+    want = np.array([0.0, 1.0, 1.0, 1.25, 1.25, 16.0, 18.0, 20.0, 448.0, 448.0, -448.0, 2.0 ** -9, 0.0, 2.0 ** -8, 0.017578125])
+    np.testing.assert_array_equal(O.round_e4m3(x), want)
+    torch = pytest.importorskip("torch")
+    if not hasattr(torch, "float8_e4m3fn"):
+        pytest.skip("this torch has no float8_e4m3fn")
+    rng = np.random.default_rng(8)
+    v = np.concatenate([rng.normal(0, 100, 4000), rng.normal(0, 1, 4000), rng.normal(0, 0.01, 4000), rng.uniform(-448, 448, 4000)])
+    v = v[np.abs(v) <= 448].astype(np.float32)
+    t = torch.from_numpy(v).to(torch.float8_e4m3fn).to(torch.float64).numpy()
+    np.testing.assert_array_equal(O.round_e4m3(v.astype(np.float64)), t)
+    # every one of the 2 x 127 finite codes is a fixed point
+    codes = torch.arange(0, 256, dtype=torch.uint8).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    codes = codes[np.isfinite(codes)]
+    np.testing.assert_array_equal(O.round_e4m3(codes), codes)
+
+
+def test_fp8_lm_head_is_the_quantised_product_and_close_to_the_exact_one():
+    head, w, rng = small_head(61, d=64, V=40)
+    h = rng.normal(0, 1.5, (5, 64))
+    z8 = O.lm_head_fp8(head, h)
+    qh, sh = O.quantize_rows_e4m3(h)
+    qw, sw = O.quantize_rows_e4m3(w["w_lm"])
+    assert np.max(np.abs(qh)) == 448 and np.all(np.max(np.abs(qw), axis=1) == 448)          # the row maximum maps to the largest code
+    for b in (0, 4):
+        for v in (0, 39):
+            assert abs(z8[b, v] - sh[b] * sw[v] * float(np.dot(qh[b], qw[v]))) < 1e-12
+    z = O.lm_head(head, h)
+    assert np.max(np.abs(z8 - z)) < 0.08 * np.max(np.abs(z))        # 3 fraction bits on both operands, averaged over 64 terms
+    assert np.max(np.abs(z8 - z)) > 1e-4                            # and it is not the unquantised product
+    np.testing.assert_array_equal(O.quantize_rows_e4m3(np.zeros((1, 8)))[0], np.zeros((1, 8)))
