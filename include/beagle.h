@@ -90,6 +90,13 @@ typedef struct beagle_weights {
     const void* w_up;     /* [m, d]            */
     const void* w_down;   /* [d, m]            */
     const void* w_lm;     /* [V, d]            */
+    /* Optional FP8 copy of the LM head (NULL, NULL = none; not part of the paper).  w_lm_fp8: [V, d] bytes, FP8 E4M3;
+     * w_lm_scale: fp32 [V]; row v of w_lm ~ w_lm_scale[v] * w_lm_fp8[v, :], as beagle_quantize_rows_e4m3 makes them.
+     * When given, beagle_draft_step with more than 8 rows (bf16 configurations) streams these bytes instead of w_lm:
+     * the step's states h are quantised the same way per row and z = scale_h * scale_w * (q_h . q_w), accumulated
+     * in fp32.  Every other entry point (and smaller batches) keeps using w_lm, which must still be valid. */
+    const void* w_lm_fp8;
+    const float* w_lm_scale;
 } beagle_weights;
 
 /* Bytes of the key/value cache ([2][max_slots][Hkv][max_ctx+max_draft][dh] in the storage type)
@@ -134,6 +141,14 @@ beagle_status beagle_rollback(beagle_ctx* ctx, int32_t batch, const int32_t* seq
 beagle_status beagle_reset_slot(beagle_ctx* ctx, int32_t slot);
 /* Current number of true / draft states of a slot (host bookkeeping). */
 beagle_status beagle_slot_lengths(const beagle_ctx* ctx, int32_t slot, int32_t* n_true, int32_t* n_draft);
+
+/* Row-wise FP8 quantisation (for beagle_weights.w_lm_fp8 / w_lm_scale): for each of `rows` rows of `cols` elements
+ * (cols a multiple of 8) of src_dev (dtype BEAGLE_FP32 | BEAGLE_BF16, dense, 16-byte aligned):
+ * scale[r] = max|x[r, :]| / 448 (1 for an all-zero row), q[r, c] = E4M3(x[r, c] / scale[r]) with round to nearest
+ * even and saturation; both divisions are IEEE single precision.  q_out_dev: rows * cols bytes; scale_out_dev: fp32
+ * [rows].  Needs no context. */
+beagle_status beagle_quantize_rows_e4m3(const void* src_dev, int32_t dtype, int64_t rows, int32_t cols, void* q_out_dev,
+                                        float* scale_out_dev, void* stream);
 
 /* Workspace bytes of beagle_block_forward for `batch` sequences of S positions. */
 beagle_status beagle_block_workspace_bytes(const beagle_config* cfg, int32_t batch, int32_t S, size_t* bytes);

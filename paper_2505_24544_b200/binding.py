@@ -28,7 +28,7 @@ EXPORTED_SYMBOLS = (
     "beagle_launch_count", "beagle_profile_enable", "beagle_profile_read", "beagle_profile_stage_count",
     "beagle_profile_stage_name", "beagle_verify_greedy_static", "beagle_check_device",
     "beagle_workspace_buffer", "beagle_block_workspace_buffer", "beagle_verify_sample", "beagle_block_loss", "beagle_draft_tree", "beagle_verify_tree_greedy",
-    "beagle_block_grad_workspace_bytes", "beagle_block_grad",
+    "beagle_block_grad_workspace_bytes", "beagle_block_grad", "beagle_quantize_rows_e4m3",
 )
 
 BUFFER_IDS = {"x": 0, "xn": 1, "q": 2, "o": 3, "y": 4, "yn": 5, "act": 6, "h": 7, "kt": 8, "vt": 9, "kp": 10, "vp": 11}
@@ -44,7 +44,7 @@ class BeagleConfig(C.Structure):
 
 
 class BeagleWeights(C.Structure):
-    _fields_ = [(n, C.c_void_p) for n in WEIGHT_NAMES]
+    _fields_ = [(n, C.c_void_p) for n in WEIGHT_NAMES] + [("w_lm_fp8", C.c_void_p), ("w_lm_scale", C.c_void_p)]
 
 
 class BeagleGrads(C.Structure):
@@ -106,6 +106,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.beagle_block_grad.argtypes = [vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, i32, vp, C.c_float, C.POINTER(BeagleGrads), vp, vp,
                                       C.c_size_t, vp]
     lib.beagle_block_grad.restype = C.c_int
+    lib.beagle_quantize_rows_e4m3.argtypes = [vp, i32, C.c_int64, i32, vp, vp, vp]
+    lib.beagle_quantize_rows_e4m3.restype = C.c_int
     lib.beagle_draft_tree.argtypes = [vp, i32, vp, i32, i32, i32, vp, vp, vp, vp]
     lib.beagle_draft_tree.restype = C.c_int
     lib.beagle_verify_tree_greedy.argtypes = [vp, i32, vp, vp, vp, i32, vp, vp, vp, vp]
@@ -161,6 +163,13 @@ class Context:
                 raise ValueError(f"weight {n}: expected contiguous {dt} CUDA tensor")
             self.weights[n] = t
             setattr(w, n, t.data_ptr())
+        for n, want in (("w_lm_fp8", torch.uint8), ("w_lm_scale", torch.float32)):      # optional FP8 copy of the LM head
+            t = weights.get(n)
+            if t is not None:
+                if t.dtype != want or not t.is_cuda or not t.is_contiguous():
+                    raise ValueError(f"weight {n}: expected contiguous {want} CUDA tensor")
+                self.weights[n] = t
+                setattr(w, n, t.data_ptr())
         kv, ws = C.c_size_t(), C.c_size_t()
         st = self.lib.beagle_query_sizes(C.byref(cfg), C.byref(kv), C.byref(ws))
         if st != 0:
@@ -269,6 +278,20 @@ def beagle_block_loss(ctx: Context, tokens: torch.Tensor, hidden: torch.Tensor, 
     ctx.check(ctx.lib.beagle_block_loss(ctx.handle, batch, S, _ptr(tokens), _ptr(hidden), block, offset, sim_steps,
                                         {"early": 0, "late": 1}[stage], _ptr(target_logits), code, _ptr(target_ids), _ptr(loss_out),
                                         _ptr(ce_out), ctx.block_ws.data_ptr(), ctx.block_ws.numel(), _stream()))
+
+
+def beagle_quantize_rows_e4m3(x: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Row-wise FP8 E4M3 quantisation of a [rows, cols] fp32 / bf16 CUDA tensor: (uint8 codes [rows, cols], fp32 scales [rows])."""
+    if x.dim() != 2 or not x.is_cuda or not x.is_contiguous() or x.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError("need a contiguous 2-D float32 / bfloat16 CUDA tensor")
+    rows, cols = x.shape
+    q = torch.empty(rows, cols, dtype=torch.uint8, device=x.device)
+    scale = torch.empty(rows, dtype=torch.float32, device=x.device)
+    st = load_library().beagle_quantize_rows_e4m3(x.data_ptr(), BEAGLE_BF16 if x.dtype == torch.bfloat16 else BEAGLE_FP32, rows, cols,
+                                                  q.data_ptr(), scale.data_ptr(), _stream())
+    if st != 0:
+        raise BeagleError(st, "beagle_quantize_rows_e4m3")
+    return q, scale
 
 
 def beagle_block_grad_workspace_bytes(ctx: Context, batch: int, S: int) -> int:
@@ -436,10 +459,14 @@ class BeagleHead:
         self.dtype = torch_dtype(code)
 
     @classmethod
-    def from_workload(cls, w, weights_np, device="cuda", max_slots=None, max_ctx=None, max_draft=None, rope_theta=0.0) -> "BeagleHead":
-        """Uploads numpy float32 weights (already rounded to the storage type) and builds the head."""
+    def from_workload(cls, w, weights_np, device="cuda", max_slots=None, max_ctx=None, max_draft=None, rope_theta=0.0,
+                      fp8_lm_head=False) -> "BeagleHead":
+        """Uploads numpy float32 weights (already rounded to the storage type) and builds the head.
+        fp8_lm_head: also make the FP8 copy of the LM head (used by draft steps of more than 8 rows)."""
         dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
         weights = {k: torch.from_numpy(v).to(device=device, dtype=dt).contiguous() for k, v in weights_np.items()}
+        if fp8_lm_head:
+            weights["w_lm_fp8"], weights["w_lm_scale"] = beagle_quantize_rows_e4m3(weights["w_lm"])
         return cls(hidden=w.hidden, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads, head_dim=w.head_dim,
                    mlp_dim=w.mlp_dim, vocab=w.vocab, dtype=w.dtype, weights=weights,
                    max_slots=max_slots or w.batch, max_ctx=max_ctx or (w.ctx_max + 64),

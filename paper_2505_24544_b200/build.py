@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB_DIR = os.path.join(HERE, "lib")
 LIB_PATH = os.path.join(LIB_DIR, "libbeagle.so")
-SOURCES = ["api.cu", "kernels_decode.cu", "kernels_block.cu", "gemm_tc.cu", "gemm_skinny.cu", "attn_decode_tma.cu", "attn_block_umma.cu", "attn_block_bwd_umma.cu", "verify_sample.cu", "block_loss.cu", "block_grad.cu", "rope.cu", "tree.cu", "noalloc.cu"]
+SOURCES = ["api.cu", "kernels_decode.cu", "kernels_block.cu", "gemm_tc.cu", "gemm_skinny.cu", "attn_decode_tma.cu", "attn_block_umma.cu", "attn_block_bwd_umma.cu", "verify_sample.cu", "block_loss.cu", "block_grad.cu", "rope.cu", "quant_fp8.cu", "tree.cu", "noalloc.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
     "-Xcompiler", "-fPIC", "--use_fast_math", "-Xptxas", "-v",

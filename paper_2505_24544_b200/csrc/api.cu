@@ -46,6 +46,8 @@ struct beagle_ctx {
     void* vs_scratch = nullptr;     // log-sum-exp partials and chunk masses of beagle_verify_sample
     void* tree_mem = nullptr;       // node / frontier arrays of beagle_draft_tree
     float* tree_logits = nullptr;   // [kTreeMaxTopk, V] logits of the frontier rows
+    void* hq = nullptr;             // FP8 LM head: quantised states of the step and their row scales
+    float* hscale = nullptr;
     float* rope_table = nullptr;    // (cos, sin) per (position, i < dh/2); rotary option only
     bool rope_ready = false;
     int rope_rows = 0;              // positions the table covers
@@ -132,7 +134,7 @@ beagle_status check_config(const beagle_config* c) {
 }
 
 struct ServeLayout {
-    size_t x, xn, q, o, y, yn, act, h, h_slot, hs, attn, sk_partial, last_token, ids, lm_partials, verify_keys, vs_scratch, tree_mem, tree_logits, rope, dev_error, total;
+    size_t x, xn, q, o, y, yn, act, h, h_slot, hs, attn, sk_partial, last_token, ids, lm_partials, verify_keys, vs_scratch, tree_mem, tree_logits, rope, hq, hscale, dev_error, total;
     int lm_blocks;
 };
 ServeLayout serve_layout(const beagle_config& c) {
@@ -169,6 +171,7 @@ ServeLayout serve_layout(const beagle_config& c) {
     L.tree_mem = take(tree_arrays_bytes(c.vocab));
     L.tree_logits = take(c.dtype == BEAGLE_BF16 ? (size_t)kTreeMaxTopk * c.vocab * sizeof(float) : 0);
     L.rope = take(c.rope_theta > 0.f ? ((size_t)c.max_ctx + c.max_draft + 1) * (c.head_dim / 2) * 2 * sizeof(float) : 0);
+    L.hq = take(B * d); L.hscale = take(B * sizeof(float));                    // FP8 LM head: the step's states as E4M3 bytes + row scales
     L.dev_error = take(256 + B * (size_t)c.n_kv_heads * sizeof(int32_t));     // error word, then the attention completion counters
     L.total = off;
     return L;
@@ -352,8 +355,10 @@ beagle_status beagle_create(const beagle_config* cfg, const beagle_weights* w, v
     if (st != BEAGLE_OK) return st;
     if (w == nullptr || kv_dev == nullptr || workspace_dev == nullptr) return BEAGLE_ERR_INVALID_ARG;
     const void* const* wp = reinterpret_cast<const void* const*>(w);
-    for (size_t i = 0; i < sizeof(beagle_weights) / sizeof(void*); ++i)
+    for (size_t i = 0; i < 11; ++i)                              // the eleven parameters; the FP8 copy of the LM head is optional
         if (wp[i] == nullptr || (reinterpret_cast<uintptr_t>(wp[i]) & 15)) return BEAGLE_ERR_INVALID_ARG;
+    if ((w->w_lm_fp8 == nullptr) != (w->w_lm_scale == nullptr)) return BEAGLE_ERR_INVALID_ARG;
+    if (w->w_lm_fp8 != nullptr && ((reinterpret_cast<uintptr_t>(w->w_lm_fp8) & 15) || cfg->hidden % 16)) return BEAGLE_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(kv_dev) & (kAlign - 1)) || (reinterpret_cast<uintptr_t>(workspace_dev) & (kAlign - 1)))
         return BEAGLE_ERR_INVALID_ARG;
     size_t need_kv, need_ws;
@@ -385,6 +390,8 @@ beagle_status beagle_create(const beagle_config* cfg, const beagle_weights* w, v
     c->vs_scratch = c->ws + L.vs_scratch;
     c->tree_mem = c->ws + L.tree_mem;
     c->tree_logits = reinterpret_cast<float*>(c->ws + L.tree_logits);
+    c->hq = c->ws + L.hq;
+    c->hscale = reinterpret_cast<float*>(c->ws + L.hscale);
     c->rope_table = reinterpret_cast<float*>(c->ws + L.rope);
     c->rope_rows = cfg->max_ctx + cfg->max_draft + 1;
     c->dev_error = reinterpret_cast<int*>(c->ws + L.dev_error);
@@ -807,6 +814,12 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
                 memset(&a, 0, sizeof(a));
                 a.W = ctx->w.w_lm; a.N = c.vocab; a.K = c.hidden; a.X = ctx->h; a.ldx = c.hidden; a.B = batch;
                 a.logits = logits_out_dev; a.keys = ctx->lm_partials;
+                if (ctx->w.w_lm_fp8 != nullptr) {       // optional FP8 LM head: quantise this step's states, stream the byte weights
+                    rc = launch_quantize_rows_e4m3(dt, ctx->h, batch, c.hidden, ctx->hq, ctx->hscale, stream);
+                    if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "FP8 LM head: hidden must be a multiple of 8");
+                    ctx->launches += rc;
+                    a.W8 = ctx->w.w_lm_fp8; a.w_scale = ctx->w.w_lm_scale; a.X8 = ctx->hq; a.x_scale = ctx->hscale;
+                }
                 BEAGLE_SKINNY(SK_LOGITS, a, "LM head");
                 nblk = tc_skinny_key_tiles(c.vocab);
             } else {
@@ -831,6 +844,16 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
         ctx->steps[s] += 1;
     }
     return BEAGLE_OK;
+}
+
+beagle_status beagle_quantize_rows_e4m3(const void* src_dev, int32_t dtype, int64_t rows, int32_t cols, void* q_out_dev,
+                                        float* scale_out_dev, void* stream_) {
+    if (src_dev == nullptr || q_out_dev == nullptr || scale_out_dev == nullptr || rows < 0 || cols <= 0) return BEAGLE_ERR_INVALID_ARG;
+    if (dtype != BEAGLE_FP32 && dtype != BEAGLE_BF16) return BEAGLE_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(src_dev) & 15) || (reinterpret_cast<uintptr_t>(q_out_dev) & 7)) return BEAGLE_ERR_INVALID_ARG;
+    if (launch_quantize_rows_e4m3(dtype, src_dev, rows, cols, q_out_dev, scale_out_dev, static_cast<cudaStream_t>(stream_)) < 0)
+        return BEAGLE_ERR_SHAPE;
+    return cudaGetLastError() == cudaSuccess ? BEAGLE_OK : BEAGLE_ERR_CUDA;
 }
 
 beagle_status beagle_block_workspace_bytes(const beagle_config* cfg, int32_t batch, int32_t S, size_t* bytes) {

@@ -42,6 +42,8 @@ struct SkArgs {
     float* partial;           // [split][nmat][B][N]
     float* logits;            // [B][N] or null
     unsigned long long* keys; // [B][gridDim.x]
+    const float* w_scale;     // FP8 LM head: per weight row
+    const float* x_scale;     // FP8 LM head: per batch row
     int* error_word;
 };
 
@@ -75,7 +77,10 @@ __device__ __forceinline__ float ld_cluster_f32(uint32_t local_addr, uint32_t ra
 // VAR 2: the CTAs that share a tile form a cluster (its K splits, or gate and up); each leaves its accumulator
 // in its own shared memory and, after a cluster barrier, reduces one slice of the tile's rows over all CTAs'
 // shared memory (distributed shared memory, fixed order) and applies the epilogue: no partials, no second kernel.
-template <int BN, int VAR>
+// FP8 (LM head only): both operands are FP8 E4M3 bytes with a scale per row; a 128-byte swizzle row then holds 128
+// elements and one MMA reads 32 of them, the same bytes as in the bf16 case, so only the element coordinates of the
+// copies, the MMA kind and the epilogue's scaling differ.
+template <int BN, int VAR, bool FP8>
 __global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_constant__ CUtensorMap tmW,
                                                                const __grid_constant__ CUtensorMap tmW2,
                                                                const __grid_constant__ CUtensorMap tmX, const SkArgs args,
@@ -95,7 +100,8 @@ __global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_cons
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ta = blockIdx.x, mat = blockIdx.y;
-    const int kb_total = (args.K + BK - 1) / BK;
+    constexpr int BKE = FP8 ? 2 * BK : BK;        // elements per 128-byte row of a tile
+    const int kb_total = (args.K + BKE - 1) / BKE;
     const int kb0 = blockIdx.z * args.kb_per_split;
     const int nkb = max(0, min(args.kb_per_split, kb_total - kb0));
 
@@ -122,11 +128,11 @@ __global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_cons
             const int npre = min(nkb, kStages);
             for (int kb = 0; kb < npre; ++kb) {
                 mbar_expect_tx(bar_full + 8 * kb, SM::kStageBytes);
-                tma_load_2d_hint(smem_base + kb * SM::kStageBytes, mapW, bar_full + 8 * kb, (kb0 + kb) * BK, ta * BM, stream_once);
+                tma_load_2d_hint(smem_base + kb * SM::kStageBytes, mapW, bar_full + 8 * kb, (kb0 + kb) * BKE, ta * BM, stream_once);
             }
             pdl_wait();
             for (int kb = 0; kb < npre; ++kb)
-                tma_load_2d_hint(smem_base + kb * SM::kStageBytes + kABytes, &tmX, bar_full + 8 * kb, (kb0 + kb) * BK, 0, keep);
+                tma_load_2d_hint(smem_base + kb * SM::kStageBytes + kABytes, &tmX, bar_full + 8 * kb, (kb0 + kb) * BKE, 0, keep);
             int issued = npre;
             for (int kb = npre; kb < nkb; ++kb) {
                 const int s = kb % kStages;
@@ -134,7 +140,7 @@ __global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_cons
                 if (!mbar_wait(bar_empty + 8 * s, ph ^ 1, s_abort)) break;
                 const uint32_t sa = smem_base + s * SM::kStageBytes, sb = sa + kABytes;
                 mbar_expect_tx(bar_full + 8 * s, SM::kStageBytes);
-                const int kc = (kb0 + kb) * BK;
+                const int kc = (kb0 + kb) * BKE;
                 tma_load_2d_hint(sa, mapW, bar_full + 8 * s, kc, ta * BM, stream_once);
                 tma_load_2d_hint(sb, &tmX, bar_full + 8 * s, kc, 0, keep);
                 ++issued;
@@ -152,7 +158,7 @@ __global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_cons
     } else if (warp == 1) {
         // ---------------- MMA issuer
         if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc(BM, BN);
+            constexpr uint32_t idesc = FP8 ? make_idesc_e4m3(BM, BN) : make_idesc(BM, BN);
             for (int kb = 0; kb < nkb; ++kb) {
                 const int s = kb % kStages;
                 const uint32_t ph = (kb / kStages) & 1;
@@ -163,7 +169,8 @@ __global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_cons
 #pragma unroll
                 for (int k = 0; k < BK / UMMA_K; ++k) {
                     const uint64_t koff = static_cast<uint64_t>((k * UMMA_K * 2) >> 4);   // advance inside the swizzle atom
-                    umma_bf16(tmem_base, da + koff, db + koff, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                    if (FP8) umma_e4m3(tmem_base, da + koff, db + koff, idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                    else umma_bf16(tmem_base, da + koff, db + koff, idesc, (kb > 0 || k > 0) ? 1u : 0u);
                 }
                 umma_commit(bar_empty + 8 * s);       // frees the stage once these MMAs have read it
             }
@@ -202,7 +209,8 @@ __global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_cons
                     for (int j = 0; j < 16; ++j) {
                         const int col = c0 + j;
                         if (col >= args.B) break;                         // uniform across the warp
-                        const float v = __uint_as_float(r[j]);
+                        float v = __uint_as_float(r[j]);
+                        if (FP8) v *= (feat < args.N ? args.w_scale[feat] : 0.f) * args.x_scale[col];
                         unsigned long long key = feat < args.N ? argmax_key(v, feat) : 0ull;
                         if (args.logits != nullptr && feat < args.N) args.logits[(size_t)col * args.N + feat] = v;
                         key = warp_max_u64(key);
@@ -380,17 +388,17 @@ SplitPlan split_plan(int N, int K, int nmat, bool allow_split) {
     return s;
 }
 
-template <int BN, int VAR>
+template <int BN, int VAR, bool FP8 = false>
 int launch_sk(const CUtensorMap& w, const CUtensorMap& w2, const CUtensorMap& x, const SkArgs& args, const FinishArgs& fin, int mode,
               dim3 grid, dim3 cluster, cudaStream_t stream) {
     using SM = SkSmem<BN>;
     static bool attr_done = false;
     if (!attr_done) {
-        if (cudaFuncSetAttribute(tc_skinny_kernel<BN, VAR>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kBytes) != cudaSuccess) return -1;
+        if (cudaFuncSetAttribute(tc_skinny_kernel<BN, VAR, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kBytes) != cudaSuccess) return -1;
         attr_done = true;
     }
     if (VAR != 2) {
-        launch_pdl(tc_skinny_kernel<BN, VAR>, grid, dim3(kSkThreads), SM::kBytes, stream, w, w2, x, args, fin, mode);
+        launch_pdl(tc_skinny_kernel<BN, VAR, FP8>, grid, dim3(kSkThreads), SM::kBytes, stream, w, w2, x, args, fin, mode);
         return 1;
     }
     cudaLaunchConfig_t cfg = {};
@@ -401,7 +409,7 @@ int launch_sk(const CUtensorMap& w, const CUtensorMap& w2, const CUtensorMap& x,
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr; cfg.numAttrs = 2;
-    if (cudaLaunchKernelEx(&cfg, tc_skinny_kernel<BN, VAR>, w, w2, x, args, fin, mode) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, tc_skinny_kernel<BN, VAR, FP8>, w, w2, x, args, fin, mode) != cudaSuccess) {
         cudaGetLastError();
         return -1;                                   // the caller falls back to partials + finishing kernel
     }
@@ -440,6 +448,25 @@ int tc_skinny(TcPlan* p, int mode, const SkinnyArgs& g, cudaStream_t stream) {
     CUtensorMap mapX;
     if (mapW == nullptr || mapW2 == nullptr || !tc_encode_map(p, &mapX, g.X, g.B, g.K, g.ldx, bn)) return -1;
     const bool logits = (mode == SK_LOGITS);
+    if (logits && g.W8 != nullptr) {
+        // FP8 LM head: byte tensor maps (128 elements per swizzle row), scales applied in the epilogue
+        if (g.K % 16 || g.X8 == nullptr || g.w_scale == nullptr || g.x_scale == nullptr || (reinterpret_cast<uintptr_t>(g.X8) & 15)) return -1;
+        const CUtensorMap* mapW8 = tc_weight_map_u8(p, g.W8, g.N, g.K, BM);
+        CUtensorMap mapX8;
+        if (mapW8 == nullptr || !tc_encode_map_u8(p, &mapX8, g.X8, g.B, g.K, g.K, bn)) return -1;
+        SkArgs a8;
+        memset(&a8, 0, sizeof(a8));
+        a8.N = g.N; a8.K = g.K; a8.B = g.B; a8.nmat = 1; a8.kb_per_split = (g.K + 2 * BK - 1) / (2 * BK);
+        a8.logits = g.logits; a8.keys = g.keys; a8.w_scale = g.w_scale; a8.x_scale = g.x_scale; a8.error_word = g.error_word;
+        FinishArgs f8;
+        memset(&f8, 0, sizeof(f8));
+        const dim3 grid8((g.N + BM - 1) / BM, 1, 1);
+        switch (bn) {
+            case 16: return launch_sk<16, 1, true>(*mapW8, *mapW8, mapX8, a8, f8, mode, grid8, dim3(1, 1, 1), stream);
+            case 32: return launch_sk<32, 1, true>(*mapW8, *mapW8, mapX8, a8, f8, mode, grid8, dim3(1, 1, 1), stream);
+            default: return launch_sk<64, 1, true>(*mapW8, *mapW8, mapX8, a8, f8, mode, grid8, dim3(1, 1, 1), stream);
+        }
+    }
     const SplitPlan sp = split_plan(g.N, g.K, nmat, !logits);
     SkArgs a;
     memset(&a, 0, sizeof(a));

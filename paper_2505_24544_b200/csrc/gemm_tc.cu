@@ -393,6 +393,26 @@ bool tc_encode_map(TcPlan* p, CUtensorMap* out, const void* base, long long rows
     return r == CUDA_SUCCESS;
 }
 
+bool tc_encode_map_u8(TcPlan* p, CUtensorMap* out, const void* base, long long rows, long long K, long long ld, int box_rows) {
+    cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld};
+    cuuint32_t box[2] = {128u, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    const CUresult r = p->encode(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+const CUtensorMap* tc_weight_map_u8(TcPlan* p, const void* W, int rows, int K, int box_rows) {
+    auto key = std::make_pair(W, box_rows);
+    auto it = p->weight_maps.find(key);
+    if (it != p->weight_maps.end()) return &it->second;
+    CUtensorMap m;
+    if (!tc_encode_map_u8(p, &m, W, rows, K, K, box_rows)) return nullptr;
+    return &p->weight_maps.emplace(key, m).first->second;
+}
+
 const CUtensorMap* tc_weight_map(TcPlan* p, const void* W, int rows, int K, int box_rows) {
     auto key = std::make_pair(W, box_rows);
     auto it = p->weight_maps.find(key);

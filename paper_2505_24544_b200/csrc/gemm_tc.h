@@ -40,6 +40,9 @@ struct SkinnyArgs {
     void* norm_out; const void* gain; float eps; int do_norm;
     void* kcache; void* vcache; int Hkv, dh, cap; RowMap slot; RowMap pos;
     float* logits; unsigned long long* keys;     // keys: [B, tc_skinny_key_tiles(N)]
+    // SK_LOGITS with FP8 operands (optional): W8 [N, K] and X8 [B, K] (dense) hold E4M3 bytes, w_scale [N] / x_scale [B] the
+    // rows' scales; logits = w_scale[n] * x_scale[b] * sum_k W8[n, k] X8[b, k].  W / X are then unused.
+    const void* W8; const float* w_scale; const void* X8; const float* x_scale;
     int* error_word;
 };
 // Kernels launched, or -1 when the shape is not covered.

@@ -99,6 +99,9 @@ int launch_attn_tail(const void* q, const void* kcache, const void* vcache, cons
 int launch_tree_verify(const int32_t* tok, const int32_t* par, int n, const int32_t* target_ids, int out_cap, int32_t* accept_len,
                        int32_t* out_tokens, int32_t* path, cudaStream_t stream);
 
+// ---- optional FP8 LM head: q[r, :] = e4m3(x[r, :] / scale[r]), scale[r] = max|x[r, :]| / 448; cols a multiple of 8 ----
+int launch_quantize_rows_e4m3(int dtype, const void* x, long long rows, int cols, void* q, float* scale, cudaStream_t stream);
+
 // ---- optional rotary position embedding (rotate-half; table of (cos, sin) per (position, i < dh/2)) ----
 int launch_rope_table(float theta, int dh, int npos, float* table, cudaStream_t stream);
 // Rows of a dense [rows, H*dh] matrix in place; row r sits at position pos_base + r % S; inverse: opposite angle.

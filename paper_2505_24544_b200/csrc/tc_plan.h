@@ -27,6 +27,9 @@ struct TcPlan {
 // K-major bf16 matrix [rows, K] (row stride ld elements), box = 64 columns x box_rows rows,
 // 128-byte swizzle, out-of-range elements read as zero.
 bool tc_encode_map(TcPlan* p, CUtensorMap* out, const void* base, long long rows, long long K, long long ld, int box_rows);
+// The same for a K-major matrix of bytes (FP8): box = 128 columns x box_rows rows.
+bool tc_encode_map_u8(TcPlan* p, CUtensorMap* out, const void* base, long long rows, long long K, long long ld, int box_rows);
+const CUtensorMap* tc_weight_map_u8(TcPlan* p, const void* W, int rows, int K, int box_rows);
 // Cached map of a weight matrix [rows, K] (dense, ld = K).
 const CUtensorMap* tc_weight_map(TcPlan* p, const void* W, int rows, int K, int box_rows);
 

@@ -36,7 +36,7 @@ def test_every_declared_symbol_is_exported(lib):
 def test_config_struct_matches_header():
     from paper_2505_24544_b200.binding import BeagleConfig, BeagleWeights
     assert C.sizeof(BeagleConfig) == 14 * 4                  # 12 int32 and 2 floats, no padding
-    assert C.sizeof(BeagleWeights) == 11 * C.sizeof(C.c_void_p)
+    assert C.sizeof(BeagleWeights) == 13 * C.sizeof(C.c_void_p)      # eleven parameters + the optional FP8 LM head (codes, scales)
 
 
 def good_config():
@@ -86,6 +86,7 @@ def test_null_context_is_rejected(lib):
     assert lib.beagle_block_grad(None, 1, 1, None, None, 1, 0, 1, 0, None, 0, None, 0.0, None, None, None, 0, None) == 1
     assert lib.beagle_verify_sample(None, 0, 0, None, None, None, 0, 1.0, None, None, None, None, None) == 1
     assert lib.beagle_draft_tree(None, 0, None, 1, 1, 1, None, None, None, None) == 1
+    assert lib.beagle_quantize_rows_e4m3(None, 1, 4, 64, None, None, None) == 1
     assert lib.beagle_destroy(None) == 1
     assert lib.beagle_version().decode().startswith("beagle")
 

@@ -627,3 +627,50 @@ def test_block_forward_and_grad_tile_edges(name, S, block, offset, sim_steps):
         assert np.linalg.norm(g - g_ref) <= tol_fro * np.linalg.norm(g_ref), pname
     from paper_2505_24544_b200.binding import beagle_check_device
     beagle_check_device(head_gpu.ctx)
+
+
+@pytest.mark.parametrize("dt", ["bf16", "fp32"])
+def test_quantize_rows_e4m3_codes_are_bit_exact(dt):
+    """The FP8 codes are an integer decision: the oracle takes it in the kernel's precision (float32 scale and quotient,
+    round to nearest even, saturating), so codes and scales must agree exactly."""
+    from paper_2505_24544_b200.binding import beagle_quantize_rows_e4m3
+    rng = np.random.default_rng(77)
+    x = (rng.standard_normal((37, 520)) * np.exp(rng.normal(0, 2, (37, 1)))).astype(np.float32)
+    x[5] = 0.0                                                     # an all-zero row: scale 1, codes 0
+    x[6, 3] = 3.0e4                                                # one dominant entry: the rest falls into the subnormals
+    x = WL.round_to_storage(x.reshape(-1), dt).reshape(x.shape)
+    q, scale = beagle_quantize_rows_e4m3(to_dev(x, dt))
+    torch.cuda.synchronize()
+    q_ref, s_ref = O.quantize_rows_e4m3(x)
+    np.testing.assert_array_equal(scale.cpu().numpy().astype(np.float64), s_ref)
+    got = q.view(torch.float8_e4m3fn).to(torch.float32).cpu().numpy().astype(np.float64)
+    np.testing.assert_array_equal(got, q_ref)
+
+
+@pytest.mark.parametrize("batch", [9, 33, 64])
+def test_fp8_lm_head_batched_draft_steps(batch):
+    """Optional FP8 LM head (draft steps of more than 8 rows): logits against the oracle's quantised product of the
+    library's own states of that step, then the greedy tokens; the rest of the step is the ordinary bf16 path."""
+    from paper_2505_24544_b200.binding import BeagleHead, beagle_workspace_buffer, beagle_check_device
+    w = SMALL_GQA.scaled(batch=batch, ctx_min=3, ctx_max=200, gamma=3, seed=2005, vocab=4099)
+    weights = WL.make_weights(w)
+    head_gpu = BeagleHead.from_workload(w, weights, max_ctx=w.ctx_max + 64, fp8_lm_head=True)
+    head_cpu = oracle_head(w, weights)
+    rng = WL.data_rng(w, batch)
+    lengths = WL.make_context_lengths(w, rng)
+    slots = list(range(batch))
+    prefill_both(head_gpu, head_cpu, w, rng, slots, lengths)
+    first = to_dev(WL.make_tokens(w, rng, (batch,)), w.dtype)
+    for step in range(3):
+        tok, logits, _ = head_gpu.draft_step(slots, tokens_in=first if step == 0 else None, want_logits=True)
+        torch.cuda.synchronize()
+        h = beagle_workspace_buffer(head_gpu.ctx, "h", batch).float().cpu().numpy().astype(np.float64)
+        z_ref = O.lm_head_fp8(head_cpu, h)
+        z = logits.cpu().numpy().astype(np.float64)
+        err = np.abs(z - z_ref)
+        assert np.all(err <= 1e-3 + 1e-3 * np.abs(z_ref)), f"step {step}: max abs err {err.max():.3e}"   # fp32 sums of exact FP8 products
+        check_tokens(tok.cpu().numpy(), z_ref, f"step {step} greedy token")
+        # and the quantised head is a usable stand-in for the bf16 one (3 fraction bits, averaged over 512 terms)
+        z_bf16 = O.lm_head(head_cpu, h)
+        assert np.max(np.abs(z_ref - z_bf16)) < 0.1 * np.max(np.abs(z_bf16))
+    beagle_check_device(head_gpu.ctx)
