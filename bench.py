@@ -697,6 +697,26 @@ def main():
             others[w3.name] = summarize_b1(w3, scn3, ms3, l3, st3, args, peaks)
             line["draft_tree"] = bench_draft_tree(head, w3, scn3, steps=max(3, min(20, args.steps)), warmup=3, peaks=peaks)
             del scn3
+            # the same batch-32 scenario with the optional FP8 (E4M3) copy of the LM head (NOT the headline: another arithmetic type
+            # for the largest weight stream; greedy verification stays lossless, only the acceptance rate could change)
+            w8 = dict(head.ctx.weights)
+            w8["w_lm_fp8"], w8["w_lm_scale"] = B.beagle_quantize_rows_e4m3(w8["w_lm"])
+            head8 = BeagleHead(hidden=w.hidden, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads, head_dim=w.head_dim, mlp_dim=w.mlp_dim,
+                               vocab=w.vocab, dtype=w.dtype, weights=w8, max_slots=w.batch, max_ctx=w.ctx_max + extra, max_draft=max_draft,
+                               rms_eps=w.rms_eps)
+            scn8 = ServeScenario(head8, w, iters, device)
+            scn8.rehearse()
+            ms8, l8 = time_serve(scn8, args.steps, args.warmup, 1)
+            st8 = profile_serve(scn8, args.steps, args.warmup)
+            lm8 = st8.get("lm_head")
+            line["fp8_lm_head"] = {"value": serve_result(scn8, w, ms8, args.steps, 1), "unit": UNIT, "ms_per_step": ms8 / args.steps,
+                                   "gpu_launches": l8, "dtype": "bf16, LM head weights and its input states in FP8 E4M3 with row scales",
+                                   "lm_head_us": (1e3 * lm8[0] / lm8[1]) if lm8 else None,
+                                   "lm_head_gbs": ((w.vocab * w.hidden + w.batch * w.hidden) / (lm8[0] / lm8[1] * 1e-3) / 1e9) if lm8 else None,
+                                   "speedup_over_bf16": (ms / args.steps) / (ms8 / args.steps)}
+            del scn8
+            head8.ctx.close()
+            del head8, w8
         del scn
         head.ctx.close()
         del head
