@@ -240,6 +240,55 @@ def time_serve(scn: ServeScenario, steps: int, warmup: int, world: int):
     return e0.elapsed_time(e1), scn.head.launch_count - l0
 
 
+def bench_draft_chain(scn: ServeScenario, reps: int = 30, warmup: int = 3):
+    """The gamma chained draft steps alone (token fed device to device, concatenation on), captured once as a CUDA graph and
+    replayed: median device time over `reps` replays, each bracketed by its own event pair, and the same chain enqueued call
+    by call for comparison.  Every replay repeats the same work (same cache rows read and rewritten).  Weights exceed L2; the
+    K/V cache of a batch-1 workload (17 MB) stays L2-resident between replays, as it does between the steps of a real chain."""
+    import torch
+    from paper_2505_24544_b200 import binding as B
+    w, head = scn.w, scn.head
+    scn.reset()
+    draft = torch.zeros(w.batch, w.gamma, dtype=torch.int32, device=scn.device)
+
+    def chain():
+        for s in range(w.gamma):
+            B.beagle_draft_step(head.ctx, scn.slots, scn.first_tokens[0] if s == 0 else None, True, draft[:, s])
+
+    def timed(fn):
+        ts = []
+        for i in range(warmup + reps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            if i >= warmup:
+                ts.append(e0.elapsed_time(e1))
+        return float(np.median(ts)), float(np.min(ts))
+
+    def eager():
+        chain()
+        head.rollback(scn.slots)
+
+    eager_ms, _ = timed(eager)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        chain()
+    head.rollback(scn.slots)
+    graph_ms, graph_min = timed(g.replay)
+    del g
+    toks = w.batch * w.gamma
+    mean_ctx = float(np.mean(scn.lengths)) + (w.gamma - 1) / 2.0
+    # step 1 has no draft state to append, so it does not stream W_k / W_v
+    gb = (sum(step_bytes(w, float(np.mean(scn.lengths)) + s) for s in range(w.gamma))
+          - elt(w) * 2 * w.hidden * w.n_kv_heads * w.head_dim) / 1e9
+    return {"value": toks / (graph_ms * 1e-3), "unit": UNIT, "ms_per_chain": graph_ms, "min_ms": graph_min, "reps": reps,
+            "timing": "median over CUDA-graph replays of gamma draft steps (argmax and draft-state append included), one event pair each",
+            "enqueued_call_by_call": {"value": toks / (eager_ms * 1e-3), "ms_per_chain": eager_ms},
+            "algorithmic_gb_per_chain": gb, "achieved_gbs": gb / (graph_ms * 1e-3), "mean_ctx": mean_ctx}
+
+
 def profile_serve(scn: ServeScenario, steps: int, warmup: int):
     """Same iterations with every stage bracketed by CUDA events inside the library."""
     import torch
@@ -688,6 +737,7 @@ def main():
         # batch-1 serving on the same head (Llama-3-8B shape) and on the Llama-2-7B shaped head
         others = {}
         line["verify_sample"] = bench_verify_sample(head, w, steps=max(3, min(20, args.steps)), warmup=3, peaks=peaks)
+        chains = {w.name: bench_draft_chain(scn)}
         if w.name == HEADLINE:
             w3 = WL.WORKLOADS["c3_llama3_8b_b1"]
             scn3 = ServeScenario(head, w3, iters, device)
@@ -695,6 +745,7 @@ def main():
             ms3, l3 = time_serve(scn3, args.steps, args.warmup, 1)
             st3 = profile_serve(scn3, args.steps, args.warmup)
             others[w3.name] = summarize_b1(w3, scn3, ms3, l3, st3, args, peaks)
+            chains[w3.name] = bench_draft_chain(scn3)
             line["draft_tree"] = bench_draft_tree(head, w3, scn3, steps=max(3, min(20, args.steps)), warmup=3, peaks=peaks)
             del scn3
             # the same batch-32 scenario with the optional FP8 (E4M3) copy of the LM head (NOT the headline: another arithmetic type
@@ -731,7 +782,11 @@ def main():
         ms2, l2 = time_serve(scn2, args.steps, args.warmup, 1)
         st2 = profile_serve(scn2, args.steps, args.warmup)
         others[w2.name] = summarize_b1(w2, scn2, ms2, l2, st2, args, peaks)
+        chains[w2.name] = bench_draft_chain(scn2)
+        for c in chains.values():
+            c["frac_of_hbm_peak"] = c["achieved_gbs"] / peaks["hbm_gbs"]
         line["batch1"] = others
+        line["draft_chain"] = chains
         del scn2
         line["block_forward"] = bench_block(head2, w5, steps=max(2, min(5, args.steps)), warmup=3, peaks=peaks)
         head2.ctx.close()
