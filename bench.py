@@ -642,6 +642,7 @@ def main():
     ap.add_argument("--workload", default=HEADLINE, choices=[k for k in WL.WORKLOADS if not k.startswith("c5")])
     ap.add_argument("--only-headline", action="store_true", help="skip the batch-1, block-forward and CPU legs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--fp8-lm-head", action="store_true", help="diagnostic: the serve scenario with the optional FP8 LM head (not the headline arithmetic)")
     ap.add_argument("--only-block", action="store_true", help="diagnostic: time only the block-attention forward (C5 shape)")
     ap.add_argument("--block-batch", type=int, default=0, help="sequences of the block forward (default: the workload's 8)")
     args = ap.parse_args()
@@ -685,7 +686,8 @@ def main():
     extra = iters * (w.gamma + 1) + 64
     max_draft = 64          # chain depth <= 8; the draft tree (depth 6, top-10) keeps 51 draft states
     weights = WL.make_weights(w)
-    head = BeagleHead.from_workload(w, weights, device=device, max_slots=w.batch, max_ctx=w.ctx_max + extra, max_draft=max_draft)
+    head = BeagleHead.from_workload(w, weights, device=device, max_slots=w.batch, max_ctx=w.ctx_max + extra, max_draft=max_draft,
+                                    fp8_lm_head=args.fp8_lm_head)
     del weights
 
     sampler = ClockSampler(physical_gpu_index(local))
@@ -705,6 +707,8 @@ def main():
     for name, (sms, cnt) in stages.items():
         per = sms / cnt
         by = stage_bytes(w, name, mean_ctx)
+        if args.fp8_lm_head and name == "lm_head":
+            by = w.vocab * w.hidden + w.batch * w.hidden          # one byte per element
         stage_out[name] = {"us_per_launch": 1e3 * per, "launches": cnt, "share": sms / max(1e-9, sum(v[0] for v in stages.values())),
                            "gbs": (by / (per * 1e-3) / 1e9) if by else None}
     dom = max((k for k in stage_out if stage_out[k]["gbs"]), key=lambda k: stage_out[k]["share"])
@@ -714,12 +718,16 @@ def main():
                 "algorithmic_bytes_per_launch": stage_bytes(w, dom, mean_ctx), "peak_source": peaks["source"],
                 "attn_decode_gbs": stage_out.get("attn_decode", {}).get("gbs"),
                 "attn_decode_frac": (stage_out["attn_decode"]["gbs"] / peaks["hbm_gbs"]) if stage_out.get("attn_decode", {}).get("gbs") else None}
-    step_gb = step_bytes(w, mean_ctx) * w.gamma / 1e9
+    if args.fp8_lm_head:
+        roofline["traffic"] = None
+        roofline["algorithmic_bytes_per_launch"] = (w.vocab * w.hidden + w.batch * w.hidden) if dom == "lm_head" else roofline["algorithmic_bytes_per_launch"]
+    step_gb = (step_bytes(w, mean_ctx) - (w.vocab * w.hidden if args.fp8_lm_head else 0)) * w.gamma / 1e9
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+        "dtype": ("bf16" if w.dtype == "bf16" else "f32") + ("+e4m3 LM head (diagnostic run, not the headline)" if args.fp8_lm_head else ""),
+        "data": "synthetic",
         "config": {"workload": w.name, "batch": w.batch, "gamma": w.gamma, "ctx": [w.ctx_min, w.ctx_max],
                    "hidden": w.hidden, "heads": [w.n_q_heads, w.n_kv_heads, w.head_dim], "mlp": w.mlp_dim, "vocab": w.vocab,
                    "step": "one SD iteration: prefill_kv(accepted states) + gamma x draft_step(concat) + verify_greedy",

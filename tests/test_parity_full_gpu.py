@@ -236,6 +236,49 @@ def test_c3_c4_llama3_8b_full(llama3_heads):
     beagle_check_device(gpu.ctx)
 
 
+def test_c4_fp8_lm_head_full_vocabulary(llama3_heads):
+    """The optional FP8 LM head at the Llama-3-8B head's size (128256 x 4096 byte weights, 32 rows), in the launch
+    configuration the benchmark times: codes and scales of sampled weight rows and of the step's states bit for bit,
+    logits of sampled vocabulary columns (both ends, tile boundaries, a random draw) against the oracle's quantised
+    product, and on ALL columns the fused greedy token is the arg-max of the returned logits."""
+    w, gpu, cpu = llama3_heads
+    from paper_2505_24544_b200.binding import (BeagleHead, beagle_check_device, beagle_quantize_rows_e4m3,
+                                               beagle_workspace_buffer)
+    w8 = dict(gpu.ctx.weights)
+    w8["w_lm_fp8"], w8["w_lm_scale"] = beagle_quantize_rows_e4m3(w8["w_lm"])
+    gpu8 = BeagleHead(hidden=w.hidden, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads, head_dim=w.head_dim, mlp_dim=w.mlp_dim,
+                      vocab=w.vocab, dtype=w.dtype, weights=w8, max_slots=w.batch, max_ctx=640, max_draft=8, rms_eps=w.rms_eps)
+    try:
+        rng = WL.data_rng(w, 58)
+        cols = np.unique(np.concatenate([np.arange(0, 130), np.arange(w.vocab - 130, w.vocab), np.arange(64000 - 4, 64000 + 4),
+                                         rng.integers(0, w.vocab, 1500)]))
+        qw_ref, sw_ref = O.quantize_rows_e4m3(cpu.w_lm[cols])
+        idx = torch.from_numpy(cols).cuda()
+        qw = w8["w_lm_fp8"][idx].view(torch.float8_e4m3fn).float().cpu().numpy().astype(np.float64)
+        np.testing.assert_array_equal(qw, qw_ref)
+        np.testing.assert_array_equal(w8["w_lm_scale"][idx].cpu().numpy().astype(np.float64), sw_ref)
+
+        slots = list(range(w.batch))
+        lengths = rng.integers(300, 600, w.batch)
+        gpu8.prefill_kv(slots, [int(n) for n in lengths], to_dev(WL.make_hidden(w, rng, int(lengths.sum())), w.dtype))
+        first = to_dev(WL.make_tokens(w, rng, (w.batch,)), w.dtype)
+        for step in range(2):
+            tok, logits, _ = gpu8.draft_step(slots, tokens_in=first if step == 0 else None, want_logits=True)
+            torch.cuda.synchronize()
+            h = beagle_workspace_buffer(gpu8.ctx, "h", w.batch).float().cpu().numpy().astype(np.float64)
+            qh, sh = O.quantize_rows_e4m3(h)
+            z_ref = (qh @ qw_ref.T) * sh[:, None] * sw_ref[None, :]
+            z = logits[:, idx].cpu().numpy().astype(np.float64)
+            err = np.abs(z - z_ref)
+            assert np.all(err <= 1e-3 + 1e-3 * np.abs(z_ref)), f"step {step}: max abs err {err.max():.3e}"
+            greedy_tokens_are_argmax_of_logits(tok, logits)
+        beagle_check_device(gpu8.ctx)
+    finally:
+        gpu8.ctx.close()
+        del gpu8, w8
+        torch.cuda.empty_cache()
+
+
 @pytest.mark.parametrize("sim_steps", [1, 4])
 def test_c5_block_forward_full_sampled_positions(llama2_heads, sim_steps):
     """8 x 2048 positions, window 4: the GPU computes everything (arg-max-only LM head, as the
