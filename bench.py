@@ -391,6 +391,7 @@ def stage_bytes(w: WL.Workload, stage: str, mean_ctx: float):
         "q_proj": e * (qd * d + B * d + B * qd),
         "o_proj": e * (d * qd + B * qd + 2 * B * d),
         "kv_append": e * (2 * kd * d + B * d + 2 * B * kd),
+        "qkv_proj": e * (qd * d + B * d + B * qd + 2 * kd * d + B * d + 2 * B * kd),
         "attn_decode": e * (B * 2 * kd * mean_ctx + 2 * B * qd),
     }.get(stage)
 

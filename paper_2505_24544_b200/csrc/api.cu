@@ -16,13 +16,13 @@ enum Stage {
     ST_KV_APPEND = 0, ST_EMBED_NORM, ST_Q_PROJ, ST_ATTN_DECODE, ST_O_PROJ, ST_MLP_NORM, ST_GATE_UP, ST_DOWN, ST_LM_HEAD,
     ST_ARGMAX, ST_PREFILL, ST_VERIFY, ST_BLK_EMBED, ST_BLK_QKV, ST_BLK_PRED_KV, ST_BLK_ATTN, ST_BLK_O, ST_BLK_NORM,
     ST_BLK_GATE_UP, ST_BLK_DOWN, ST_BLK_LM_HEAD, ST_BLK_ARGMAX, ST_BWD_DLOGITS, ST_BWD_DX, ST_BWD_DW, ST_BWD_ATTN,
-    ST_BWD_TRANSPOSE, ST_BWD_ELEMENTWISE, ST_COUNT
+    ST_BWD_TRANSPOSE, ST_BWD_ELEMENTWISE, ST_QKV_PROJ, ST_COUNT
 };
 static const char* const kStageNames[ST_COUNT] = {
     "kv_append", "embed_norm", "q_proj", "attn_decode", "o_proj", "mlp_norm", "gate_up", "down_proj", "lm_head",
     "argmax_finalize", "prefill_kv", "verify", "blk_embed", "blk_qkv", "blk_pred_kv", "blk_attn", "blk_o_proj", "blk_norm",
     "blk_gate_up", "blk_down", "blk_lm_head", "blk_argmax", "bwd_dlogits", "bwd_dx_gemm", "bwd_dw_gemm", "bwd_attn",
-    "bwd_transpose", "bwd_elementwise"};
+    "bwd_transpose", "bwd_elementwise", "qkv_proj"};
 
 struct StageRecord { int stage; cudaEvent_t start, stop; };
 
@@ -676,8 +676,23 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
                                            c.hidden, c.rms_eps, c.norm_q, ctx->x, ctx->xn, batch,
                                            (use_tc && any_append) ? ctx->h_slot : nullptr, ctx->hs, stream);
     }
+    // (2) + (3) on the tensor-core path: the K/V append and the query projection read different inputs and write different
+    // outputs, so they share one launch
+    bool merged_qkv = false;
+    if (use_tc && any_append) {
+        StageTimer timer_(ctx, ST_QKV_PROJ, stream);
+        SkinnyArgs q, kv;
+        memset(&q, 0, sizeof(q)); memset(&kv, 0, sizeof(kv));
+        q.W = ctx->w.w_q; q.N = ctx->qd; q.K = c.hidden; q.X = ctx->xn; q.ldx = c.hidden; q.B = batch;
+        q.out = ctx->q; q.ldo = ctx->qd; q.error_word = ctx->dev_error;
+        kv.W = ctx->w.w_k; kv.W2 = ctx->w.w_v; kv.N = ctx->kd; kv.K = c.hidden; kv.X = ctx->hs; kv.ldx = c.hidden; kv.B = batch;
+        kv.kcache = ctx->kcache; kv.vcache = ctx->vcache; kv.Hkv = c.n_kv_heads; kv.dh = c.head_dim; kv.cap = ctx->cap;
+        kv.slot = slots; kv.pos = app_pos;
+        rc = tc_skinny_qkv(ctx->tc, q, kv, stream);
+        if (rc > 0) { ctx->launches += rc; merged_qkv = true; }
+    }
     // (2) concat: K/V of the previous step's state joins the cache tail (Section 4.1, cache paragraph)
-    if (any_append) {
+    if (any_append && !merged_qkv) {
         StageTimer timer_(ctx, ST_KV_APPEND, stream);
         if (use_tc) {
             SkinnyArgs a;
@@ -697,7 +712,7 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
         }
     }
     // (3) Q = W_q xn
-    {
+    if (!merged_qkv) {
         StageTimer timer_(ctx, ST_Q_PROJ, stream);
         if (use_tc) {
             SkinnyArgs a;

@@ -25,6 +25,7 @@ using namespace tc;
 constexpr int BM = 128;
 constexpr int kSkThreads = 192;
 constexpr int kCtaSlots = 296;          // CTAs the split policy aims at (two per SM on 148 SMs)
+constexpr int kQkvCtaSlots = 444;       // the merged Q + K/V launch: three CTAs per SM fit, its clusters must all be resident at once
 constexpr int kABytes = BM * BK * 2;
 
 template <int BN>
@@ -80,11 +81,10 @@ __device__ __forceinline__ float ld_cluster_f32(uint32_t local_addr, uint32_t ra
 // FP8 (LM head only): both operands are FP8 E4M3 bytes with a scale per row; a 128-byte swizzle row then holds 128
 // elements and one MMA reads 32 of them, the same bytes as in the bf16 case, so only the element coordinates of the
 // copies, the MMA kind and the epilogue's scaling differ.
+// The body takes this CTA's weight map, activation map, tile index `ta` and matrix index `mat` from its entry point.
 template <int BN, int VAR, bool FP8>
-__global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_constant__ CUtensorMap tmW,
-                                                               const __grid_constant__ CUtensorMap tmW2,
-                                                               const __grid_constant__ CUtensorMap tmX, const SkArgs args,
-                                                               const FinishArgs fin, const int mode) {
+__device__ __forceinline__ void sk_body(const CUtensorMap* mapW, const CUtensorMap* mapX, const SkArgs& args, const FinishArgs& fin,
+                                        const int mode, const int ta, const int mat) {
     constexpr bool LOGITS = (VAR == 1), FUSED = (VAR == 2);
     using SM = SkSmem<BN>;
     constexpr int kStages = SM::kStages;
@@ -99,7 +99,6 @@ __global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_cons
     unsigned long long* s_keys = reinterpret_cast<unsigned long long*>(smem_gen + kStages * SM::kStageBytes + 256);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int ta = blockIdx.x, mat = blockIdx.y;
     constexpr int BKE = FP8 ? 2 * BK : BK;        // elements per 128-byte row of a tile
     const int kb_total = (args.K + BKE - 1) / BKE;
     const int kb0 = blockIdx.z * args.kb_per_split;
@@ -121,7 +120,6 @@ __global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_cons
     if (warp == 0) {
         // ---------------- TMA producer
         if (lane == 0) {
-            const CUtensorMap* mapW = mat ? &tmW2 : &tmW;
             const uint64_t stream_once = policy_evict_first(), keep = policy_evict_last();
             // The weights do not depend on the previous kernel: fill the ring with weight tiles
             // while that kernel drains, then wait for it and add the activation tiles.
@@ -132,7 +130,7 @@ __global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_cons
             }
             pdl_wait();
             for (int kb = 0; kb < npre; ++kb)
-                tma_load_2d_hint(smem_base + kb * SM::kStageBytes + kABytes, &tmX, bar_full + 8 * kb, (kb0 + kb) * BKE, 0, keep);
+                tma_load_2d_hint(smem_base + kb * SM::kStageBytes + kABytes, mapX, bar_full + 8 * kb, (kb0 + kb) * BKE, 0, keep);
             int issued = npre;
             for (int kb = npre; kb < nkb; ++kb) {
                 const int s = kb % kStages;
@@ -142,7 +140,7 @@ __global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_cons
                 mbar_expect_tx(bar_full + 8 * s, SM::kStageBytes);
                 const int kc = (kb0 + kb) * BKE;
                 tma_load_2d_hint(sa, mapW, bar_full + 8 * s, kc, ta * BM, stream_once);
-                tma_load_2d_hint(sb, &tmX, bar_full + 8 * s, kc, 0, keep);
+                tma_load_2d_hint(sb, mapX, bar_full + 8 * s, kc, 0, keep);
                 ++issued;
             }
             if (*s_abort) {
@@ -279,6 +277,34 @@ __global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_cons
         fence_after();
         tmem_dealloc<kTmemCols>(tmem_base);
     }
+}
+
+template <int BN, int VAR, bool FP8>
+__global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_constant__ CUtensorMap tmW,
+                                                               const __grid_constant__ CUtensorMap tmW2,
+                                                               const __grid_constant__ CUtensorMap tmX, const SkArgs args,
+                                                               const FinishArgs fin, const int mode) {
+    sk_body<BN, VAR, FP8>(blockIdx.y ? &tmW2 : &tmW, &tmX, args, fin, mode, blockIdx.x, blockIdx.y);
+}
+
+// Two projections of one draft step in ONE launch (cluster variant): tiles [0, q_tiles) of blockIdx.x are the query projection
+// (W_q on the normalised embeddings, stored), the next kv_tiles the key and the last kv_tiles the value projection of the
+// previous step's states (written to the cache).  Same reduction length, same K slices, one kernel boundary fewer.
+template <int BN>
+__global__ void __launch_bounds__(kSkThreads) tc_skinny_qkv_kernel(const __grid_constant__ CUtensorMap tmWq,
+                                                                   const __grid_constant__ CUtensorMap tmWk,
+                                                                   const __grid_constant__ CUtensorMap tmWv,
+                                                                   const __grid_constant__ CUtensorMap tmXq,
+                                                                   const __grid_constant__ CUtensorMap tmXkv, const SkArgs args,
+                                                                   const FinishArgs fin, const int q_tiles, const int kv_tiles,
+                                                                   const int kv_N) {
+    const int x = blockIdx.x;
+    const bool kv = x >= q_tiles;
+    const int mat = kv ? (x - q_tiles) / kv_tiles : 0;
+    const int ta = kv ? (x - q_tiles) % kv_tiles : x;
+    SkArgs a = args;
+    if (kv) a.N = kv_N;
+    sk_body<BN, 2, false>(kv ? (mat ? &tmWv : &tmWk) : &tmWq, kv ? &tmXkv : &tmXq, a, fin, kv ? (int)SK_KV : (int)SK_STORE, ta, mat);
 }
 
 // ---------------------------------------------------------------------------------------------- finishing kernel
@@ -426,7 +452,63 @@ int launch_sk_bn(int bn, const CUtensorMap& w, const CUtensorMap& w2, const CUte
     }
 }
 
+template <int BN>
+int launch_sk_qkv(const CUtensorMap& wq, const CUtensorMap& wk, const CUtensorMap& wv, const CUtensorMap& xq, const CUtensorMap& xkv,
+                  const SkArgs& args, const FinishArgs& fin, int q_tiles, int kv_tiles, int kv_N, int cs, cudaStream_t stream) {
+    using SM = SkSmem<BN>;
+    static bool attr_done = false;
+    if (!attr_done) {
+        if (cudaFuncSetAttribute(tc_skinny_qkv_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kBytes) != cudaSuccess) return -1;
+        attr_done = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(q_tiles + 2 * kv_tiles, 1, cs); cfg.blockDim = dim3(kSkThreads); cfg.dynamicSmemBytes = SM::kBytes; cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = cs;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 2;
+    if (cudaLaunchKernelEx(&cfg, tc_skinny_qkv_kernel<BN>, wq, wk, wv, xq, xkv, args, fin, q_tiles, kv_tiles, kv_N) != cudaSuccess) {
+        cudaGetLastError();
+        return -1;
+    }
+    return 1;
+}
+
 }  // namespace
+
+int tc_skinny_qkv(TcPlan* p, const SkinnyArgs& q, const SkinnyArgs& kv, cudaStream_t stream) {
+    if (p == nullptr || q.B <= 0 || q.B > kMaxCallBatch || kv.B != q.B || kv.K != q.K) return -1;
+    if (q.K % 8 || q.ldx % 8 || kv.ldx % 8 || (q.N % 4) || (kv.N % 4) || (kv.dh % 4)) return -1;
+    if ((reinterpret_cast<uintptr_t>(q.X) & 15) || (reinterpret_cast<uintptr_t>(kv.X) & 15)) return -1;
+    const int bn = q.B <= 16 ? 16 : (q.B <= 32 ? 32 : 64);
+    const CUtensorMap* mapWq = tc_weight_map(p, q.W, q.N, q.K, BM);
+    const CUtensorMap* mapWk = tc_weight_map(p, kv.W, kv.N, kv.K, BM);
+    const CUtensorMap* mapWv = tc_weight_map(p, kv.W2, kv.N, kv.K, BM);
+    CUtensorMap mapXq, mapXkv;
+    if (mapWq == nullptr || mapWk == nullptr || mapWv == nullptr || !tc_encode_map(p, &mapXq, q.X, q.B, q.K, q.ldx, bn) ||
+        !tc_encode_map(p, &mapXkv, kv.X, kv.B, kv.K, kv.ldx, bn))
+        return -1;
+    const int q_tiles = (q.N + BM - 1) / BM, kv_tiles = (kv.N + BM - 1) / BM;
+    const int kb_total = (q.K + BK - 1) / BK;
+    int cs = 1;                                       // K splits = cluster size: a power of two, at most 8, slices of at least 4 k-blocks
+    while (cs * 2 <= 8 && (q_tiles + 2 * kv_tiles) * cs * 2 <= kQkvCtaSlots && kb_total / (cs * 2) >= 4) cs *= 2;
+    SkArgs a;
+    memset(&a, 0, sizeof(a));
+    a.N = q.N; a.K = q.K; a.B = q.B; a.nmat = 1; a.kb_per_split = (kb_total + cs - 1) / cs; a.error_word = q.error_word;
+    FinishArgs f;
+    memset(&f, 0, sizeof(f));
+    f.splits = cs; f.nmat = 1; f.B = q.B; f.N = q.N;
+    f.out = static_cast<bf16*>(q.out); f.ldo = q.ldo;
+    f.kcache = static_cast<bf16*>(kv.kcache); f.vcache = static_cast<bf16*>(kv.vcache); f.Hkv = kv.Hkv; f.dh = kv.dh; f.cap = kv.cap;
+    f.slot = kv.slot; f.pos = kv.pos;
+    switch (bn) {
+        case 16: return launch_sk_qkv<16>(*mapWq, *mapWk, *mapWv, mapXq, mapXkv, a, f, q_tiles, kv_tiles, kv.N, cs, stream);
+        case 32: return launch_sk_qkv<32>(*mapWq, *mapWk, *mapWv, mapXq, mapXkv, a, f, q_tiles, kv_tiles, kv.N, cs, stream);
+        default: return launch_sk_qkv<64>(*mapWq, *mapWk, *mapWv, mapXq, mapXkv, a, f, q_tiles, kv_tiles, kv.N, cs, stream);
+    }
+}
 
 size_t tc_skinny_partial_bytes(int N, int K, int nmat) {
     const SplitPlan s = split_plan(N, K, nmat, true);

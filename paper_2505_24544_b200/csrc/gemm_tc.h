@@ -47,6 +47,9 @@ struct SkinnyArgs {
 };
 // Kernels launched, or -1 when the shape is not covered.
 int tc_skinny(TcPlan* plan, int mode, const SkinnyArgs& a, cudaStream_t stream);
+// The query projection (SK_STORE arguments `q`) and the K/V append (SK_KV arguments `kv`) of one draft step as ONE launch;
+// same reduction length and batch.  1, or -1 when not covered (the caller then launches the two separately).
+int tc_skinny_qkv(TcPlan* plan, const SkinnyArgs& q, const SkinnyArgs& kv, cudaStream_t stream);
 // Bytes of fp32 partial sums a projection [N, K] with `nmat` weight matrices needs for 64 rows.
 size_t tc_skinny_partial_bytes(int N, int K, int nmat);
 int tc_skinny_key_tiles(int N);
