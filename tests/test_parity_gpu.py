@@ -118,6 +118,43 @@ def test_batched_serving_tensor_core_projections(batch, rope):
     beagle_check_device(head_gpu.ctx)
 
 
+@pytest.mark.parametrize("batch", [4, 12])
+def test_chain_continues_with_another_batch_composition(batch):
+    """A step that continues from the device-resident greedy tokens may name fewer sequences, or another order, than the step
+    before it (every sequence carries its own token, state and draft depth; batches of 8 rows or fewer and larger ones take different kernels)."""
+    w = SMALL_GQA.scaled(batch=batch, ctx_min=5, ctx_max=200, gamma=4, seed=2011)
+    head_gpu, head_cpu, _ = build(w, max_ctx=w.ctx_max + 64, max_draft=8)
+    rng = WL.data_rng(w, batch)
+    lengths = WL.make_context_lengths(w, rng)
+    slots = [int(s) for s in rng.permutation(batch)]
+    seqs = prefill_both(head_gpu, head_cpu, w, rng, slots, lengths)
+    first = WL.make_tokens(w, rng, (batch,))
+    drafted, _, _ = run_chain_parity(head_gpu, head_cpu, w, slots, seqs, first, 2)
+
+    def step(rows, what):
+        t, logits, hidden = head_gpu.draft_step([slots[r] for r in rows], tokens_in=None, want_logits=True, want_hidden=True)
+        torch.cuda.synchronize()
+        out = O.draft_step(head_cpu, [seqs[r] for r in rows], tokens_in=None)
+        assert_close(logits.float().cpu().numpy(), out["logits"], w.dtype, what + " logits")
+        assert_close(hidden.float().cpu().numpy(), out["h"], w.dtype, what + " hidden")
+        gt = t.cpu().numpy()
+        check_tokens(gt, out["logits"], what + " tokens")
+        for r, tok in zip(rows, gt):
+            seqs[r].pending_token = int(tok)              # near a tie either id is right: both sides go on from the library's
+
+    for r in range(batch):
+        seqs[r].pending_token = int(drafted[r, -1])
+    sub = [batch - 1, 0, 2] + list(range(3, batch - 1, 2))
+    step(sub, "permuted subset")
+    step(sub, "same subset again")
+    step(list(range(batch)), "all sequences, unequal depths")
+    step(list(range(batch)), "all sequences again")
+    from paper_2505_24544_b200.binding import beagle_check_device
+    beagle_check_device(head_gpu.ctx)
+    for r in range(batch):
+        assert head_gpu.slot_lengths(slots[r]) == (int(lengths[r]), 5 if r in sub else 3)
+
+
 @pytest.mark.parametrize("rope", [0.0, 10000.0])
 def test_empty_cache_concat_off_and_rollback(rope):
     w = SMALL_GQA.scaled(batch=2)
