@@ -760,13 +760,18 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
     }
     // (5) y = W_o o + x   (6) yn = RMSNorm(y)
     if (use_tc) {
-        StageTimer timer_(ctx, ST_O_PROJ, stream);
-        SkinnyArgs a;
-        memset(&a, 0, sizeof(a));
-        a.W = ctx->w.w_o; a.N = c.hidden; a.K = ctx->qd; a.X = ctx->o; a.ldx = ctx->qd; a.B = batch;
-        a.out = ctx->y; a.ldo = c.hidden; a.resid = ctx->x; a.ldr = c.hidden;
-        a.norm_out = ctx->yn; a.gain = ctx->w.g_mlp; a.eps = c.rms_eps; a.do_norm = c.norm_mlp;   // the finishing kernel normalises
-        BEAGLE_SKINNY(SK_RESID, a, "O projection");
+        {
+            StageTimer timer_(ctx, ST_O_PROJ, stream);
+            SkinnyArgs a;
+            memset(&a, 0, sizeof(a));
+            a.W = ctx->w.w_o; a.N = c.hidden; a.K = ctx->qd; a.X = ctx->o; a.ldx = ctx->qd; a.B = batch;
+            a.out = ctx->y; a.ldo = c.hidden; a.resid = ctx->x; a.ldr = c.hidden;      // cluster variant: residual added in the reduction
+            BEAGLE_SKINNY(SK_RESID, a, "O projection");
+        }
+        // a row kernel over the 32 x d result is cheaper than a finishing kernel that re-reads all fp32 split partials
+        StageTimer timer_(ctx, ST_MLP_NORM, stream);
+        ctx->launches += launch_embed_norm(dt, nullptr, nullptr, nullptr, nullptr, 0, ctx->y, ctx->w.g_mlp, c.hidden, c.rms_eps,
+                                           c.norm_mlp, nullptr, ctx->yn, batch, nullptr, nullptr, stream);
     } else {
         {
             StageTimer timer_(ctx, ST_O_PROJ, stream);
