@@ -1446,6 +1446,7 @@ beagle_status beagle_draft_tree(beagle_ctx* ctx, int32_t slot, const int32_t* ro
         ctx->launches += launch_embed_norm(dt, e == 0 ? root_token_dev : T.frontier_tok, nullptr, &meta, ctx->w.embed, c.vocab, nullptr, ctx->w.g_q,
                                            c.hidden, c.rms_eps, c.norm_q, ctx->x, ctx->xn, rows, nullptr, nullptr, stream);
         // the states produced by the previous forward join the cache tail (concatenation, Section 4.1)
+        bool merged_qkv = false;
         if (e >= 1) {
             const int nprev = e == 1 ? 1 : topk;
             for (int r = 0; r < nprev; ++r) pos.idx[r] = n_true + (e == 1 ? 0 : 1 + (e - 2) * topk + r);
@@ -1454,9 +1455,18 @@ beagle_status beagle_draft_tree(beagle_ctx* ctx, int32_t slot, const int32_t* ro
             a.W = ctx->w.w_k; a.W2 = ctx->w.w_v; a.N = ctx->kd; a.K = c.hidden; a.X = ctx->h; a.ldx = c.hidden; a.B = nprev;
             a.kcache = ctx->kcache; a.vcache = ctx->vcache; a.Hkv = c.n_kv_heads; a.dh = c.head_dim; a.cap = ctx->cap;
             a.slot = slots; a.pos = pos;
-            BEAGLE_TREE_SKINNY(SK_KV, a, "K/V append");
+            // one launch with the query projection when possible (rows beyond nprev have pos = -1 and are skipped)
+            SkinnyArgs q;
+            memset(&q, 0, sizeof(q));
+            q.W = ctx->w.w_q; q.N = ctx->qd; q.K = c.hidden; q.X = ctx->xn; q.ldx = c.hidden; q.B = rows;
+            q.out = ctx->q; q.ldo = ctx->qd; q.error_word = ctx->dev_error;
+            SkinnyArgs kv = a;
+            kv.B = rows;
+            rc = tc_skinny_qkv(ctx->tc, q, kv, stream);
+            if (rc > 0) { ctx->launches += rc; merged_qkv = true; }
+            else BEAGLE_TREE_SKINNY(SK_KV, a, "K/V append");
         }
-        {
+        if (!merged_qkv) {
             SkinnyArgs a;
             memset(&a, 0, sizeof(a));
             a.W = ctx->w.w_q; a.N = ctx->qd; a.K = c.hidden; a.X = ctx->xn; a.ldx = c.hidden; a.B = rows;
@@ -1493,9 +1503,10 @@ beagle_status beagle_draft_tree(beagle_ctx* ctx, int32_t slot, const int32_t* ro
             memset(&a, 0, sizeof(a));
             a.W = ctx->w.w_o; a.N = c.hidden; a.K = ctx->qd; a.X = ctx->o; a.ldx = ctx->qd; a.B = rows;
             a.out = ctx->y; a.ldo = c.hidden; a.resid = ctx->x; a.ldr = c.hidden;
-            a.norm_out = ctx->yn; a.gain = ctx->w.g_mlp; a.eps = c.rms_eps; a.do_norm = c.norm_mlp;
             BEAGLE_TREE_SKINNY(SK_RESID, a, "O projection");
         }
+        ctx->launches += launch_embed_norm(dt, nullptr, nullptr, nullptr, nullptr, 0, ctx->y, ctx->w.g_mlp, c.hidden, c.rms_eps, c.norm_mlp,
+                                           nullptr, ctx->yn, rows, nullptr, nullptr, stream);
         {
             SkinnyArgs a;
             memset(&a, 0, sizeof(a));
