@@ -528,7 +528,8 @@ __global__ void __launch_bounds__(1024) argmax_finalize_kernel(const unsigned lo
                                                                const BatchMeta meta, int32_t* __restrict__ tokens_out,
                                                                int tokens_out_stride, int32_t* __restrict__ last_token) {
     const int b = blockIdx.x;
-    pdl_launch_dependents();
+    const bool release_early = gridDim.x > 8;      // as in the decode attention: early for large batches, at the end for small ones (measured)
+    if (release_early) pdl_launch_dependents();
     pdl_wait();
     const unsigned long long* row = partials + (size_t)b * nblk;
     unsigned long long key = 0ull;
@@ -552,6 +553,7 @@ __global__ void __launch_bounds__(1024) argmax_finalize_kernel(const unsigned lo
             last_token[meta.slot[b]] = tok;
         }
     }
+    if (!release_early) pdl_launch_dependents();
 }
 int launch_argmax_finalize(const unsigned long long* partials, int nblk, const BatchMeta& meta, int B,
                            int32_t* tokens_out, int tokens_out_stride, int32_t* last_token, cudaStream_t stream) {
