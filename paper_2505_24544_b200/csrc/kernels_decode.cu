@@ -26,7 +26,8 @@ __global__ void __launch_bounds__(256) embed_norm_kernel(const int32_t* __restri
     // of this step begins after all earlier work in the stream (cache prefill, the previous step)
     // has completed.  The later kernels' early reads of weights and true-state cache rows rely on it.
     pdl_wait();
-    pdl_launch_dependents();
+    const bool release_early = gridDim.x > 8;      // small batches: at the end (measured, as in the projection kernel below)
+    if (release_early) pdl_launch_dependents();
     if (gather_src != nullptr) {
         const uint4* g = reinterpret_cast<const uint4*>(gather_src + (size_t)meta.slot[r] * d);
         uint4* dst = reinterpret_cast<uint4*>(gather_dst + (size_t)r * d);
@@ -97,6 +98,7 @@ __global__ void __launch_bounds__(256) embed_norm_kernel(const int32_t* __restri
             xn_out[(size_t)r * d + i] = from_float<T>(v * sc * g);
         }
     }
+    if (!release_early) pdl_launch_dependents();
 }
 
 int launch_embed_norm(int dtype, const int32_t* tokens, const int32_t* last_token, const BatchMeta* meta,
