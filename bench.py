@@ -32,6 +32,8 @@ from paper_2505_24544_b200 import workloads as WL  # noqa: E402
 METRIC = "draft_tokens_per_s"
 UNIT = "draft tokens/s"
 HEADLINE = "c4_llama3_8b_b32"
+STEP_TEXT = ("one SD iteration, enqueued call by call: prefill_kv(accepted states) + gamma x draft_step(concat) + verify_greedy; "
+             "the draft chain alone under CUDA-graph replay is reported as draft_chain")
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -398,13 +400,46 @@ def stage_bytes(w: WL.Workload, stage: str, mean_ctx: float):
 
 # ------------------------------------------------------------------------------------------------ CPU oracle legs
 
-def oracle_sample(w: WL.Workload, n_seq: int, iters: int, warm: int = 0):
-    """Times the CPU oracle, as it stands, on `n_seq` sequences of the workload for `iters` SD
-    iterations (context prefill untimed).  Returns (draft tokens/s, seconds, threads)."""
+def oracle_head_for(w: WL.Workload):
     import oracle as O
     weights = WL.make_weights(w)
     head = O.OracleHead(O.HeadConfig(w.hidden, w.n_q_heads, w.n_kv_heads, w.head_dim, w.mlp_dim, w.vocab, rms_eps=w.rms_eps), weights)
     del weights
+    return head
+
+
+def blas_threads() -> int:
+    threads = os.cpu_count() or 1
+    try:
+        from threadpoolctl import threadpool_info
+        nt = [p.get("num_threads") for p in threadpool_info() if p.get("user_api") == "blas"]
+        if nt:
+            threads = max(nt)
+    except Exception:
+        pass
+    return threads
+
+
+def cpu_model() -> str:
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    return line.split(":", 1)[1].strip()
+    except Exception:
+        pass
+    return "unknown"
+
+
+def oracle_sample(w: WL.Workload, n_seq: int, iters: int, warm: int = 0, head=None, threads=None):
+    """Times the CPU oracle, as it stands, on `n_seq` sequences of the workload for `iters` SD
+    iterations (context prefill untimed; `threads`: limit of the BLAS pool, None = all cores).
+    Returns (draft tokens/s, seconds, threads used)."""
+    import contextlib
+
+    import oracle as O
+    if head is None:
+        head = oracle_head_for(w)
     rng = WL.data_rng(w, 7)
     lengths = WL.make_context_lengths(w, rng)[:n_seq]
     seqs = []
@@ -414,31 +449,49 @@ def oracle_sample(w: WL.Workload, n_seq: int, iters: int, warm: int = 0):
         seqs.append(s)
     new_len = [1] * n_seq
     first = WL.make_tokens(w, rng, (n_seq,))
-    t0 = time.perf_counter()
-    for it in range(-warm, iters):
-        if it == 0:
-            t0 = time.perf_counter()
-        if it != -warm:
-            for b, s in enumerate(seqs):
-                O.prefill_kv(head, s, WL.make_hidden(w, rng, new_len[b]))
-        drafted = np.zeros((n_seq, w.gamma), dtype=np.int64)
-        for st in range(w.gamma):
-            out = O.draft_step(head, seqs, tokens_in=list(first) if st == 0 else None, concat=True)
-            drafted[:, st] = out["argmax"]
-        target = WL.make_target_stream(w, rng, drafted)
-        acc, out_tok = O.verify_greedy(drafted, target_ids=target)
-        new_len = [int(a) + 1 for a in acc]
-        first = np.array([out_tok[b, acc[b]] for b in range(n_seq)])
-    dt = time.perf_counter() - t0
-    threads = os.cpu_count() or 1
-    try:
-        from threadpoolctl import threadpool_info
-        nt = [p.get("num_threads") for p in threadpool_info() if p.get("user_api") == "blas"]
-        if nt:
-            threads = max(nt)
-    except Exception:
-        pass
-    return n_seq * w.gamma * iters / dt, dt, threads
+    limit = contextlib.nullcontext()
+    if threads is not None:
+        from threadpoolctl import threadpool_limits
+        limit = threadpool_limits(limits=threads)
+    with limit:
+        used = blas_threads() if threads is None else threads
+        t0 = time.perf_counter()
+        for it in range(-warm, iters):
+            if it == 0:
+                t0 = time.perf_counter()
+            if it != -warm:
+                for b, s in enumerate(seqs):
+                    O.prefill_kv(head, s, WL.make_hidden(w, rng, new_len[b]))
+            drafted = np.zeros((n_seq, w.gamma), dtype=np.int64)
+            for st in range(w.gamma):
+                out = O.draft_step(head, seqs, tokens_in=list(first) if st == 0 else None, concat=True)
+                drafted[:, st] = out["argmax"]
+            target = WL.make_target_stream(w, rng, drafted)
+            acc, out_tok = O.verify_greedy(drafted, target_ids=target)
+            new_len = [int(a) + 1 for a in acc]
+            first = np.array([out_tok[b, acc[b]] for b in range(n_seq)])
+        dt = time.perf_counter() - t0
+    return n_seq * w.gamma * iters / dt, dt, used
+
+
+def cpu_baseline_legs(head_llama3):
+    """The oracle as it stands on the machine's host cores, single-threaded and with all cores, on every serving workload:
+    C1..C3 one or more full SD iterations of the whole workload, C4 on a stated subset of its sequences.  `head_llama3`:
+    an oracle head of the Llama-3-8B shape (C3 and C4 share it; the weights' seed does not matter for a timing)."""
+    out = {"nproc": os.cpu_count(), "cpu_model": cpu_model(), "workloads": {}}
+    plan = [("c1_tiny_fp32", 1, 8, None), ("c2_llama2_7b_b1", 1, 1, None), ("c3_llama3_8b_b1", 1, 1, head_llama3), (HEADLINE, 4, 1, head_llama3)]
+    for name, n_seq, iters, head in plan:
+        w = WL.WORKLOADS[name]
+        if head is None:
+            head = oracle_head_for(w)
+        n_seq = min(n_seq, w.batch)
+        v_all, s_all, t_all = oracle_sample(w, n_seq, iters, head=head)
+        v_one, s_one, _ = oracle_sample(w, n_seq, iters, head=head, threads=1)
+        out["workloads"][name] = {"all_cores": {"value": v_all, "seconds": s_all, "threads": t_all},
+                                  "single_thread": {"value": v_one, "seconds": s_one, "threads": 1}, "unit": UNIT,
+                                  "sample": f"{n_seq} of {w.batch} sequence(s) x {iters} SD iteration(s) of {w.gamma} draft tokens, context prefill untimed"}
+        del head
+    return out
 
 
 def run_reference(args):
@@ -457,8 +510,11 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
         "warmup": warm, "ms_per_step": 1e3 * sec / steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "batch": w.batch, "gamma": w.gamma, "ctx": [w.ctx_min, w.ctx_max], "sample": sample},
-        "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "config": {"workload": w.name, "batch": w.batch, "gamma": w.gamma, "ctx": [w.ctx_min, w.ctx_max],
+                   "hidden": w.hidden, "heads": [w.n_q_heads, w.n_kv_heads, w.head_dim], "mlp": w.mlp_dim, "vocab": w.vocab,
+                   "step": STEP_TEXT, "parallelism": "single", "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample, "nproc": os.cpu_count(),
+                         "cpu_model": cpu_model()},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0, "wall_s": time.perf_counter() - t0,
     }
@@ -592,6 +648,91 @@ def bench_verify_sample(head, w: WL.Workload, steps: int, warmup: int, peaks):
             "note": "156 MB of logits is close to L2 size: repeated calls partly hit L2"}
 
 
+def bench_prefill(scn, peaks, reps: int = 5, warmup: int = 2):
+    """K/V projection of a whole context into the cache (beagle_prefill_kv over every sequence's true states, packed):
+    the one tensor-bound step of the serving path.  Median over `reps` calls, one event pair each; the states (> 1 GB at
+    batch 32) exceed L2."""
+    import torch
+    from paper_2505_24544_b200 import binding as B
+    w, head = scn.w, scn.head
+    lengths = [int(n) for n in scn.lengths]
+    rows = int(sum(lengths))
+    ts = []
+    l0 = 0
+    for i in range(warmup + reps):
+        for s in scn.slots:
+            B.beagle_reset_slot(head.ctx, s)
+        torch.cuda.synchronize()
+        l0 = head.launch_count
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        head.prefill_kv(scn.slots, lengths, scn.ctx_hidden)
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= warmup:
+            ts.append(e0.elapsed_time(e1))
+    ms = float(np.median(ts))
+    kd = w.n_kv_heads * w.head_dim
+    flop = 2.0 * rows * w.hidden * 2 * kd
+    by = elt(w) * (rows * w.hidden + 2 * kd * w.hidden + 2 * rows * kd)
+    tf = flop / (ms * 1e-3) / 1e12
+    return {"rows": rows, "sequences": len(lengths), "ms": ms, "min_ms": float(np.min(ts)), "states_per_s": rows / (ms * 1e-3),
+            "tflop": flop / 1e12, "tflops": tf, "frac_of_bf16_burst_peak": tf / peaks["bf16_tflops"],
+            "algorithmic_gb": by / 1e9, "gbs": by / (ms * 1e-3) / 1e9, "gpu_launches": head.launch_count - l0,
+            "timing": "median of %d calls, one CUDA-event pair each" % reps}
+
+
+def bench_verify_greedy_logits(head, w: WL.Workload, peaks, reps: int = 20, warmup: int = 3):
+    """Greedy verification from the target's logits (fp32 [batch, gamma + 1, V]): arg-max of every row + the acceptance
+    walk, one launch.  HBM-bound: every logit is read once.  The calls rotate over enough distinct logit buffers to
+    exceed L2 several times, so every call reads from HBM."""
+    import torch
+    dev = head.device
+    g = torch.Generator(device=dev)
+    g.manual_seed(w.seed + 2)
+    Bn, gamma, V = w.batch, w.gamma, w.vocab
+    by = Bn * (gamma + 1) * V * 4
+    nbuf = max(3, int(np.ceil(512e6 / by)) + 1)
+    bufs = [torch.randn(Bn, gamma + 1, V, generator=g, device=dev, dtype=torch.float32) for _ in range(nbuf)]
+    draft = torch.stack([b[:, :gamma].argmax(dim=-1) for b in bufs]).to(torch.int32)
+    flip = torch.rand(draft.shape, generator=g, device=dev) > 0.7           # ~70 % agreement per position
+    draft = torch.where(flip, (draft + 1) % V, draft).contiguous()
+    from paper_2505_24544_b200 import binding as B
+    acc = torch.empty(nbuf, Bn, dtype=torch.int32, device=dev)
+    out = torch.empty(nbuf, Bn, gamma + 1, dtype=torch.int32, device=dev)
+
+    def calls():
+        for i in range(reps):
+            B.beagle_verify_greedy(head.ctx, draft[i % nbuf], bufs[i % nbuf], None, acc[i % nbuf], out[i % nbuf])
+
+    # the kernel lasts a few microseconds at batch 1, less than the host needs to enqueue it: the calls are captured once
+    # into a CUDA graph and the replay is timed (one launch per call either way)
+    l0 = head.launch_count
+    calls()
+    launches = head.launch_count - l0
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        calls()
+    ts = []
+    for i in range(warmup + 5):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        if i >= warmup:
+            ts.append(e0.elapsed_time(e1) / reps)
+    del graph
+    ms = float(np.median(ts))
+    acc = acc[0]
+    return {"us_per_call": 1e3 * ms, "algorithmic_mb": by / 1e6, "gbs": by / (ms * 1e-3) / 1e9,
+            "frac_of_hbm_peak": by / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "launches_per_call": launches / reps,
+            "timing": "median of 5 CUDA-graph replays of %d calls" % reps,
+            "mean_accept_len": float(acc.float().mean()), "rotating_buffers": nbuf,
+            "shape": [Bn, gamma + 1, V], "dtype": "f32"}
+
+
 def bench_draft_tree(head, w: WL.Workload, scn, steps: int, warmup: int, peaks):
     """Dynamic draft tree at the paper's setting (depth 1 + 6, top-10, 60 candidates) on one sequence
     of the batch-1 workload: 7 forwards of 1 / 10 rows, each streaming the head's weights once."""
@@ -646,6 +787,7 @@ def main():
     ap.add_argument("--fp8-lm-head", action="store_true", help="diagnostic: the serve scenario with the optional FP8 LM head (not the headline arithmetic)")
     ap.add_argument("--only-block", action="store_true", help="diagnostic: time only the block-attention forward (C5 shape)")
     ap.add_argument("--block-batch", type=int, default=0, help="sequences of the block forward (default: the workload's 8)")
+    ap.add_argument("--only-legs", action="store_true", help="diagnostic: only the prefill and verify-from-logits legs of the headline workload")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -693,6 +835,16 @@ def main():
 
     sampler = ClockSampler(physical_gpu_index(local))
     scn = ServeScenario(head, w, iters, device)
+    if args.only_legs:
+        out = {"prefill": {w.name: bench_prefill(scn, peaks)}, "verify_greedy_logits": {w.name: bench_verify_greedy_logits(head, w, peaks)}}
+        w3 = WL.WORKLOADS["c3_llama3_8b_b1"]
+        if w.name == HEADLINE:
+            scn3 = ServeScenario(head, w3, iters, device)
+            out["prefill"][w3.name] = bench_prefill(scn3, peaks)
+            out["verify_greedy_logits"][w3.name] = bench_verify_greedy_logits(head, w3, peaks)
+        if rank == 0:
+            print(json.dumps(out), flush=True)
+        return
     scn.rehearse()
     sampler.start()
     ms, launches = time_serve(scn, args.steps, args.warmup, world)
@@ -731,7 +883,7 @@ def main():
         "data": "synthetic",
         "config": {"workload": w.name, "batch": w.batch, "gamma": w.gamma, "ctx": [w.ctx_min, w.ctx_max],
                    "hidden": w.hidden, "heads": [w.n_q_heads, w.n_kv_heads, w.head_dim], "mlp": w.mlp_dim, "vocab": w.vocab,
-                   "step": "one SD iteration: prefill_kv(accepted states) + gamma x draft_step(concat) + verify_greedy",
+                   "step": STEP_TEXT,
                    "l2": "inputs larger than L2 (weights %.2f GB + K/V per draft step)" % (step_bytes(w, mean_ctx) / 1e9),
                    "mean_tau": scn.mean_tau, "parallelism": "replicas" if world > 1 else "single"},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps},
@@ -746,6 +898,8 @@ def main():
         # batch-1 serving on the same head (Llama-3-8B shape) and on the Llama-2-7B shaped head
         others = {}
         line["verify_sample"] = bench_verify_sample(head, w, steps=max(3, min(20, args.steps)), warmup=3, peaks=peaks)
+        line["prefill"] = {w.name: bench_prefill(scn, peaks)}
+        line["verify_greedy_logits"] = {w.name: bench_verify_greedy_logits(head, w, peaks)}
         chains = {w.name: bench_draft_chain(scn)}
         if w.name == HEADLINE:
             w3 = WL.WORKLOADS["c3_llama3_8b_b1"]
@@ -755,6 +909,8 @@ def main():
             st3 = profile_serve(scn3, args.steps, args.warmup)
             others[w3.name] = summarize_b1(w3, scn3, ms3, l3, st3, args, peaks)
             chains[w3.name] = bench_draft_chain(scn3)
+            line["prefill"][w3.name] = bench_prefill(scn3, peaks)
+            line["verify_greedy_logits"][w3.name] = bench_verify_greedy_logits(head, w3, peaks)
             line["draft_tree"] = bench_draft_tree(head, w3, scn3, steps=max(3, min(20, args.steps)), warmup=3, peaks=peaks)
             del scn3
             # the same batch-32 scenario with the optional FP8 (E4M3) copy of the LM head (NOT the headline: another arithmetic type
@@ -804,10 +960,14 @@ def main():
     line["clocks"] = sampler.stop()
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.only_headline:
-        n_seq, n_it = min(8, w.batch), 10                # about 10 s of numpy on the machine's cores
-        val, sec, threads = oracle_sample(w, n_seq, n_it)
+        n_seq, n_it = min(8, w.batch), 4                 # a few seconds of numpy on the machine's cores
+        head_cpu = oracle_head_for(w)
+        val, sec, threads = oracle_sample(w, n_seq, n_it, head=head_cpu)
         line["cpu_baseline"] = {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "seconds": sec,
                                 "sample": f"{n_seq} of {w.batch} sequences x {n_it} SD iterations of {w.gamma} draft tokens, context prefill untimed"}
+        if w.name == HEADLINE:
+            line["cpu_baseline"].update(cpu_baseline_legs(head_cpu))
+        del head_cpu
     line["wall_s"] = time.perf_counter() - t_wall
     if rank == 0:
         print(json.dumps(line), flush=True)

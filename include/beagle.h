@@ -344,8 +344,18 @@ beagle_status beagle_block_workspace_buffer(const beagle_config* cfg, int32_t ba
                                             size_t* offset_bytes, int32_t* row_elems);
 
 /* Waits for the stream, then reports BEAGLE_ERR_DEVICE if any kernel of this context abandoned a
- * bounded wait (its outputs are then undefined).  The only call that synchronises. */
+ * bounded wait since the last check (its outputs are then undefined); the condition is reported once
+ * and cleared, the context stays usable.  Besides the one-time set-up of a context's first launching
+ * call, the only call that synchronises. */
 beagle_status beagle_check_device(beagle_ctx* ctx, void* stream);
+
+/* Test support for the error path above.  Every wait inside the tensor-core kernels (on a TMA copy, on
+ * an MMA commit) is bounded: after a fixed number of polls the kernel raises the context's device
+ * error word, lets its outstanding copies land, frees its tensor memory and returns.  This call
+ * launches a one-CTA kernel that performs such a wait on a barrier nothing will ever complete, with a
+ * short limit and no copy in flight: the wait runs out (nothing hangs, nothing faults) and the next
+ * beagle_check_device returns BEAGLE_ERR_DEVICE.  The paper has no counterpart. */
+beagle_status beagle_selftest_wait_timeout(beagle_ctx* ctx, void* stream);
 
 /* Text of the last error recorded on this context ("" if none). */
 const char* beagle_last_error(const beagle_ctx* ctx);

@@ -4,7 +4,9 @@ TEST INFRASTRUCTURE ONLY -- slow, obvious, independent of the CUDA library.
 Every floating-point operation runs in numpy float64; the only library
 primitives are matrix products, exp, sqrt and argmax.  Inputs arrive already
 rounded to whatever storage type the caller studies (bf16 values are exactly
-representable in float64), so the oracle itself never rounds.
+representable in float64).  By default the oracle rounds nothing in between;
+two options do round, each where its paragraph below says: the "bf16" storage
+mode (stored intermediates) and the FP8 LM head (quantised operands).
 
 Notation follows the paper (Section 3 "Preliminaries", Section 4.1
 "Cross-Attention Draft Modeling", Section 4.2 "Two-Stage Block-Attention
@@ -174,8 +176,9 @@ def round_e4m3(a: np.ndarray) -> np.ndarray:
 
 def quantize_rows_e4m3(x: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
     """Row-wise FP8 quantisation as the optional FP8 LM head uses it: scale_r = max|x_r| / 448 (1 for a zero row),
-    q_r = round_e4m3(x_r / scale_r), so that x_r ~ scale_r * q_r.  The scale and the quotient are formed in
-    float32 -- the quantised code is an integer decision, taken in the precision the kernel takes it in.
+    q_r = round_e4m3(x_r / scale_r), so that x_r ~ scale_r * q_r.  The scale and the quotient are formed in IEEE
+    float32: the code is an integer decision, and float32 is the precision in which FP8 scaling is stated wherever
+    it is deployed (a float64 quotient that lies within 2^-24 of a rounding boundary would decide differently).
     Returns (q as float64 values, scale as float64)."""
     x32 = np.asarray(x, dtype=np.float32)
     amax = np.max(np.abs(x32), axis=-1, keepdims=True)

@@ -9,6 +9,7 @@ from __future__ import annotations
 
 import ctypes as C
 import os
+import weakref
 from typing import Dict, Optional, Sequence, Tuple
 
 import torch
@@ -26,7 +27,7 @@ EXPORTED_SYMBOLS = (
     "beagle_draft_step", "beagle_rollback", "beagle_reset_slot", "beagle_slot_lengths",
     "beagle_block_workspace_bytes", "beagle_block_forward", "beagle_verify_greedy", "beagle_last_error",
     "beagle_launch_count", "beagle_profile_enable", "beagle_profile_read", "beagle_profile_stage_count",
-    "beagle_profile_stage_name", "beagle_verify_greedy_static", "beagle_check_device",
+    "beagle_profile_stage_name", "beagle_verify_greedy_static", "beagle_check_device", "beagle_selftest_wait_timeout",
     "beagle_workspace_buffer", "beagle_block_workspace_buffer", "beagle_verify_sample", "beagle_block_loss", "beagle_draft_tree", "beagle_verify_tree_greedy",
     "beagle_block_grad_workspace_bytes", "beagle_block_grad", "beagle_quantize_rows_e4m3",
 )
@@ -65,7 +66,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     global _lib
     if _lib is not None and path is None:
         return _lib
-    p = path or _build.LIB_PATH
+    # BEAGLE_LIBRARY: another build of the same library (the tests load the bounds-checking build this way)
+    p = path or os.environ.get("BEAGLE_LIBRARY") or _build.LIB_PATH
     if not os.path.exists(p):
         raise ImportError(f"{p} not found: run `python -m paper_2505_24544_b200.build` (there is no fallback path)")
     lib = C.CDLL(p)
@@ -116,6 +118,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.beagle_verify_sample.restype = C.c_int
     lib.beagle_check_device.argtypes = [vp, vp]
     lib.beagle_check_device.restype = C.c_int
+    lib.beagle_selftest_wait_timeout.argtypes = [vp, vp]
+    lib.beagle_selftest_wait_timeout.restype = C.c_int
     lib.beagle_launch_count.restype = C.c_int64
     lib.beagle_launch_count.argtypes = [vp]
     for name in ("beagle_query_sizes", "beagle_create", "beagle_destroy", "beagle_prefill_kv", "beagle_draft_step",
@@ -146,6 +150,9 @@ def _stream() -> int:
 
 def torch_dtype(dtype_code: int) -> torch.dtype:
     return torch.bfloat16 if dtype_code == BEAGLE_BF16 else torch.float32
+
+
+LIVE_CONTEXTS: "weakref.WeakSet[Context]" = weakref.WeakSet()      # open contexts (the tests check each one's device status)
 
 
 class Context:
@@ -184,6 +191,7 @@ class Context:
         if st != 0:
             raise BeagleError(st, "beagle_create failed")
         self.handle = handle
+        LIVE_CONTEXTS.add(self)
 
     def check(self, st: int) -> None:
         if st != 0:
@@ -423,6 +431,11 @@ def kv_cache_views(ctx: Context) -> Tuple[torch.Tensor, torch.Tensor]:
     k = ctx.kv_buf[:n].view(dt).view(c.max_slots, c.n_kv_heads, cap, c.head_dim)
     v = ctx.kv_buf[half:half + n].view(dt).view(c.max_slots, c.n_kv_heads, cap, c.head_dim)
     return k, v
+
+
+def beagle_selftest_wait_timeout(ctx: Context) -> None:
+    """Launches the one-CTA kernel whose bounded wait runs out (test support for the device error path)."""
+    ctx.check(ctx.lib.beagle_selftest_wait_timeout(ctx.handle, _stream()))
 
 
 def beagle_check_device(ctx: Context) -> None:

@@ -49,11 +49,11 @@ struct beagle_ctx {
     void* hq = nullptr;             // FP8 LM head: quantised states of the step and their row scales
     float* hscale = nullptr;
     float* rope_table = nullptr;    // (cos, sin) per (position, i < dh/2); rotary option only
-    bool rope_ready = false;
     int rope_rows = 0;              // positions the table covers
     std::vector<int32_t> steps;     // draft steps of a slot since its cache was last reset to true states
-    int* dev_error = nullptr;       // device word raised by a kernel whose bounded wait ran out
-    bool dev_error_cleared = false;
+    int* dev_error = nullptr;       // device word raised by a kernel whose bounded wait ran out; the zero-initialised counters follow it
+    int sm_count = 148;
+    bool dev_ready = false;         // device_setup_once has run
     int lm_blocks = 0;
     // host bookkeeping
     std::vector<int32_t> n_true, n_draft;
@@ -67,6 +67,13 @@ struct beagle_ctx {
     std::vector<StageRecord> records;
     std::vector<std::pair<cudaEvent_t, cudaEvent_t>> free_events;
 };
+
+#ifdef BEAGLE_BOUNDS_CHECK
+namespace beagle {
+__device__ int* g_bounds_word = nullptr;
+__device__ int g_bounds_slots = 0;
+}  // namespace beagle
+#endif
 
 namespace {
 // Brackets one stage with events on the call's stream while profiling is on.
@@ -137,6 +144,11 @@ struct ServeLayout {
     size_t x, xn, q, o, y, yn, act, h, h_slot, hs, attn, sk_partial, last_token, ids, lm_partials, verify_keys, vs_scratch, tree_mem, tree_logits, rope, hq, hscale, dev_error, total;
     int lm_blocks;
 };
+// Device words that must read zero before the first kernel uses them: the error word (first 256 bytes), one completion
+// counter per (row, K/V head) of the decode attention, one ticket per row of the greedy verification.
+size_t dev_words_bytes(const beagle_config& c) {
+    return 256 + (size_t)BEAGLE_MAX_CALL_BATCH * c.n_kv_heads * sizeof(int32_t) + (size_t)BEAGLE_MAX_CALL_BATCH * sizeof(int32_t);
+}
 ServeLayout serve_layout(const beagle_config& c) {
     ServeLayout L;
     const size_t elt = c.dtype == BEAGLE_BF16 ? 2 : 4;
@@ -166,13 +178,13 @@ ServeLayout serve_layout(const beagle_config& c) {
     L.ids = take(B * 65 * sizeof(int32_t));
     L.lm_blocks = gemv_grid_blocks(GEMV_LOGITS, c.vocab);
     L.lm_partials = take(B * (size_t)L.lm_blocks * sizeof(unsigned long long));
-    L.verify_keys = take(B * 65 * kRowArgmaxSplit * sizeof(unsigned long long));
+    L.verify_keys = take(B * 65 * kVerifyMaxSplit * sizeof(unsigned long long));
     L.vs_scratch = take(verify_sample_scratch_bytes((int)B, 64));
     L.tree_mem = take(tree_arrays_bytes(c.vocab));
     L.tree_logits = take(c.dtype == BEAGLE_BF16 ? (size_t)kTreeMaxTopk * c.vocab * sizeof(float) : 0);
     L.rope = take(c.rope_theta > 0.f ? ((size_t)c.max_ctx + c.max_draft + 1) * (c.head_dim / 2) * 2 * sizeof(float) : 0);
     L.hq = take(B * d); L.hscale = take(B * sizeof(float));                    // FP8 LM head: the step's states as E4M3 bytes + row scales
-    L.dev_error = take(256 + B * (size_t)c.n_kv_heads * sizeof(int32_t));     // error word, then the attention completion counters
+    L.dev_error = take(dev_words_bytes(c));    // error word, the attention completion counters, the verification tickets
     L.total = off;
     return L;
 }
@@ -249,38 +261,55 @@ GradLayout grad_layout(const beagle_config& c, int batch, int S) {
     return L;
 }
 
+int* attn_done_counters(beagle_ctx* ctx) { return ctx->dev_error + 64; }
+int* verify_tickets(beagle_ctx* ctx) { return ctx->dev_error + 64 + BEAGLE_MAX_CALL_BATCH * ctx->cfg.n_kv_heads; }
+
 beagle_status cuda_ok(beagle_ctx* ctx, const char* what) {
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return fail(ctx, BEAGLE_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
     return BEAGLE_OK;
 }
 
+// One-time device set-up of a context, done by the first call that launches anything: the device words (error word,
+// completion counters, verification tickets) are zeroed and, with the rotary option, the (cos, sin) table is built; the
+// call then waits for both, so that later calls find them ready whatever stream they use.  Work enqueued inside a
+// stream capture would be recorded, not run, so a first call inside a capture is refused.
+beagle_status device_setup_once(beagle_ctx* ctx, cudaStream_t stream) {
+    if (ctx->dev_ready) return BEAGLE_OK;
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cs) != cudaSuccess)
+        return fail(ctx, BEAGLE_ERR_CUDA, "device set-up: %s", cudaGetErrorString(cudaGetLastError()));
+    if (cs != cudaStreamCaptureStatusNone)
+        return fail(ctx, BEAGLE_ERR_STATE, "the first launching call on a context must be made outside stream capture");
+    if (cudaMemsetAsync(ctx->dev_error, 0, dev_words_bytes(ctx->cfg), stream) != cudaSuccess)
+        return fail(ctx, BEAGLE_ERR_CUDA, "device set-up: %s", cudaGetErrorString(cudaGetLastError()));
+    if (ctx->cfg.rope_theta > 0.f)
+        ctx->launches += launch_rope_table(ctx->cfg.rope_theta, ctx->cfg.head_dim, ctx->rope_rows, ctx->rope_table, stream);
+#ifdef BEAGLE_BOUNDS_CHECK
+    {   // bounds-checking build: the kernels' index checks report into this context's error word
+        int* word = ctx->dev_error;
+        int slots = ctx->cfg.max_slots;
+        if (cudaMemcpyToSymbolAsync(g_bounds_word, &word, sizeof(word), 0, cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+            cudaMemcpyToSymbolAsync(g_bounds_slots, &slots, sizeof(slots), 0, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+            return fail(ctx, BEAGLE_ERR_CUDA, "device set-up: %s", cudaGetErrorString(cudaGetLastError()));
+    }
+#endif
+    if (cudaStreamSynchronize(stream) != cudaSuccess)
+        return fail(ctx, BEAGLE_ERR_CUDA, "device set-up: %s", cudaGetErrorString(cudaGetLastError()));
+    ctx->dev_ready = true;
+    return BEAGLE_OK;
+}
+
 // One dense projection C = A W^T of the block / prefill path: tensor cores when the plan covers the
 // shape (bf16), the CUDA-core kernel otherwise.
-void clear_error_word_once(beagle_ctx* ctx, cudaStream_t stream) {
-    if (!ctx->dev_error_cleared) {
-        cudaMemsetAsync(ctx->dev_error, 0, 256 + (size_t)BEAGLE_MAX_CALL_BATCH * ctx->cfg.n_kv_heads * sizeof(int32_t), stream);
-        ctx->dev_error_cleared = true;
-    }
-}
-
-// Rotary option: the serve-time table is built by the first call that needs it, on that call's stream.
-void rope_table_once(beagle_ctx* ctx, cudaStream_t stream) {
-    if (ctx->cfg.rope_theta > 0.f && !ctx->rope_ready) {
-        ctx->launches += launch_rope_table(ctx->cfg.rope_theta, ctx->cfg.head_dim, ctx->rope_rows, ctx->rope_table, stream);
-        ctx->rope_ready = true;
-    }
-}
-
 int dense_gemm(beagle_ctx* ctx, int epi, const GemmArgs& a, cudaStream_t stream) {
     if (ctx->tc != nullptr) {
-        clear_error_word_once(ctx, stream);
         GemmArgs t = a;
         t.error_word = ctx->dev_error;
         const int rc = tc_gemm(ctx->tc, epi, t, stream);
         if (rc >= 0) return rc;
     }
-    if (epi == GEMM_ARGMAX_KEYS || epi == GEMM_CE || epi == GEMM_DLOGITS) return -1;
+    if (epi == GEMM_ARGMAX_KEYS || epi == GEMM_CE || epi == GEMM_DLOGITS || epi == GEMM_KV_CACHE_PAIR) return -1;
     return launch_gemm_simt(ctx->cfg.dtype, epi, a, stream);
 }
 
@@ -288,7 +317,11 @@ int dense_gemm(beagle_ctx* ctx, int epi, const GemmArgs& a, cudaStream_t stream)
 
 extern "C" {
 
-const char* beagle_version(void) { return "beagle-b200 0.1 (sm_100a)"; }
+#ifdef BEAGLE_BOUNDS_CHECK
+const char* beagle_version(void) { return "beagle-b200 0.2 (sm_100a, bounds-checking build)"; }
+#else
+const char* beagle_version(void) { return "beagle-b200 0.2 (sm_100a)"; }
+#endif
 
 beagle_status beagle_query_sizes(const beagle_config* cfg, size_t* kv_bytes, size_t* workspace_bytes) {
     const beagle_status st = check_config(cfg);
@@ -407,6 +440,13 @@ beagle_status beagle_create(const beagle_config* cfg, const beagle_weights* w, v
         delete c;
         return BEAGLE_ERR_CUDA;     // a GPU is present but the tensor-map encoder is not: never fall back silently
     }
+    {
+        int dev = 0, sms = 0;       // grid sizing only; without a device (host-only use) the default stays
+        if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+            c->sm_count = sms;
+        else
+            cudaGetLastError();
+    }
     if (c->tc != nullptr)
         tc_attn_bind_cache(c->tc, c->kcache, c->vcache, (long long)cfg->max_slots * cfg->n_kv_heads * c->cap, cfg->head_dim);
     *out = c;
@@ -456,12 +496,27 @@ beagle_status beagle_check_device(beagle_ctx* ctx, void* stream_) {
     if (ctx == nullptr) return BEAGLE_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (cudaStreamSynchronize(stream) != cudaSuccess) return fail(ctx, BEAGLE_ERR_CUDA, "check_device: %s", cudaGetErrorString(cudaGetLastError()));
-    if (!ctx->dev_error_cleared) return BEAGLE_OK;
+    if (!ctx->dev_ready) return BEAGLE_OK;
     int word = 0;
     if (cudaMemcpy(&word, ctx->dev_error, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
         return fail(ctx, BEAGLE_ERR_CUDA, "check_device: %s", cudaGetErrorString(cudaGetLastError()));
-    if (word != 0) return fail(ctx, BEAGLE_ERR_DEVICE, "a kernel gave up on a bounded wait (pipeline barrier never completed)");
+    if (word != 0) {
+        // reported once: the word is cleared so that the context stays usable and a later check speaks of later kernels
+        if (cudaMemset(ctx->dev_error, 0, sizeof(int)) != cudaSuccess)
+            return fail(ctx, BEAGLE_ERR_CUDA, "check_device: %s", cudaGetErrorString(cudaGetLastError()));
+        return fail(ctx, BEAGLE_ERR_DEVICE, word == 2 ? "a kernel's index check failed (bounds-checking build): the access was skipped"
+                                                      : "a kernel gave up on a bounded wait (pipeline barrier never completed)");
+    }
     return BEAGLE_OK;
+}
+
+beagle_status beagle_selftest_wait_timeout(beagle_ctx* ctx, void* stream_) {
+    if (ctx == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const beagle_status st = device_setup_once(ctx, stream);
+    if (st != BEAGLE_OK) return st;
+    ctx->launches += launch_wait_timeout_selftest(ctx->dev_error, stream);
+    return cuda_ok(ctx, "selftest_wait_timeout");
 }
 
 const char* beagle_last_error(const beagle_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
@@ -528,6 +583,8 @@ beagle_status beagle_prefill_kv(beagle_ctx* ctx, int32_t batch, const int32_t* s
     const beagle_config& c = ctx->cfg;
 
     if (total > 0) {
+        st = device_setup_once(ctx, stream);
+        if (st != BEAGLE_OK) return st;
         StageTimer timer_(ctx, ST_PREFILL, stream);
         SeqRows rows;
         memset(&rows, 0, sizeof(rows));
@@ -560,7 +617,6 @@ beagle_status beagle_prefill_kv(beagle_ctx* ctx, int32_t batch, const int32_t* s
         } else if (ctx->tc != nullptr && total <= kPrefillSkinnyMaxRows) {
             // up to a few hundred rows (one verification of a whole batch): chunks of 64 rows on the
             // tensor cores with the weights as the wide operand; W_k, W_v stay in L2 between chunks
-            clear_error_word_once(ctx, stream);
             int s = 0;
             for (int r0 = 0; r0 < (int)total; r0 += kMaxCallBatch) {
                 const int nb = (int)total - r0 < kMaxCallBatch ? (int)total - r0 : kMaxCallBatch;
@@ -584,17 +640,21 @@ beagle_status beagle_prefill_kv(beagle_ctx* ctx, int32_t batch, const int32_t* s
             memset(&g, 0, sizeof(g));
             g.A = hidden_dev; g.lda = c.hidden; g.M = (int)total; g.N = ctx->kd; g.K = c.hidden;
             g.Hkv = c.n_kv_heads; g.dh = c.head_dim; g.cap = ctx->cap; g.rows = rows;
-            g.W = ctx->w.w_k; g.cache = ctx->kcache;
-            int rc = dense_gemm(ctx, GEMM_KV_CACHE, g, stream);
-            if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "K projection: unsupported shape");
-            ctx->launches += rc;
-            g.W = ctx->w.w_v; g.cache = ctx->vcache;
-            rc = dense_gemm(ctx, GEMM_KV_CACHE, g, stream);
-            if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "V projection: unsupported shape");
+            // tensor cores: both projections in one pass over the states (the K and V weight tiles side by side in one MMA);
+            // otherwise one product per matrix
+            g.W = ctx->w.w_k; g.cache = ctx->kcache; g.W2 = ctx->w.w_v; g.cache2 = ctx->vcache;
+            int rc = ctx->tc != nullptr ? dense_gemm(ctx, GEMM_KV_CACHE_PAIR, g, stream) : -1;
+            if (rc < 0) {
+                rc = dense_gemm(ctx, GEMM_KV_CACHE, g, stream);
+                if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "K projection: unsupported shape");
+                ctx->launches += rc;
+                g.W = ctx->w.w_v; g.cache = ctx->vcache;
+                rc = dense_gemm(ctx, GEMM_KV_CACHE, g, stream);
+                if (rc < 0) return fail(ctx, BEAGLE_ERR_SHAPE, "V projection: unsupported shape");
+            }
             ctx->launches += rc;
         }
         if (c.rope_theta > 0.f) {       // rotary option: the new key rows are rotated in place by their positions
-            rope_table_once(ctx, stream);
             ctx->launches += launch_rope_cache_rows(c.dtype, ctx->kcache, total, c.n_kv_heads, c.head_dim, ctx->cap, rows, ctx->rope_table, stream);
         }
         st = cuda_ok(ctx, "prefill_kv");
@@ -638,6 +698,8 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
                             ctx->n_true[seq_slot[b]] + ctx->steps[seq_slot[b]] + 1);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const int dt = c.dtype;
+    st = device_setup_once(ctx, stream);
+    if (st != BEAGLE_OK) return st;
 
     BatchMeta meta;
     memset(&meta, 0, sizeof(meta));
@@ -658,7 +720,6 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
     // Batches above 8 rows run their projections on the tensor cores (weights streamed once);
     // smaller ones on the weight-streaming CUDA-core kernel.
     const bool use_tc = ctx->tc != nullptr && batch > kServeTcMinBatch;
-    if (use_tc) clear_error_word_once(ctx, stream);
     int rc = 0;
 #define BEAGLE_SKINNY(MODE, ARGS, WHAT)                                                   \
     do {                                                                                  \
@@ -731,7 +792,6 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
     // (3') rotary option: the s-th step since the reset queries position n + s; the state appended now sits one before it
     if (c.rope_theta > 0.f) {
         StageTimer timer_(ctx, ST_Q_PROJ, stream);
-        rope_table_once(ctx, stream);
         RowMap qpos, kpos;
         memset(&qpos, 0, sizeof(qpos)); memset(&kpos, 0, sizeof(kpos));
         for (int b = 0; b < batch; ++b) {
@@ -746,11 +806,10 @@ beagle_status beagle_draft_step(beagle_ctx* ctx, int32_t batch, const int32_t* s
         StageTimer timer_(ctx, ST_ATTN_DECODE, stream);
         rc = -1;
         if (ctx->tc != nullptr) {       // bf16, head_dim 64 / 128: TMA-staged tiles
-            clear_error_word_once(ctx, stream);
             int32_t stable[kMaxCallBatch];
             for (int b = 0; b < batch; ++b) stable[b] = ctx->n_true[seq_slot[b]];
             rc = tc_attn_decode(ctx->tc, ctx->q, meta, stable, batch, c.n_q_heads, c.n_kv_heads, c.head_dim, ctx->cap, max_kv,
-                                ctx->attn_scratch, ctx->dev_error + 64, ctx->o, ctx->dev_error, stream);
+                                ctx->attn_scratch, attn_done_counters(ctx), ctx->o, ctx->dev_error, stream);
         }
         if (rc < 0)
             rc = launch_attn_decode(dt, ctx->q, ctx->kcache, ctx->vcache, meta, batch, c.n_q_heads, c.n_kv_heads,
@@ -914,6 +973,10 @@ static beagle_status block_forward_impl(beagle_ctx* ctx, int32_t batch, int32_t 
     const BlockLayout L = block_layout(c, batch, S);
     if (ws_bytes < L.total) return fail(ctx, BEAGLE_ERR_CAPACITY, "block_forward: workspace %zu < %zu bytes", ws_bytes, L.total);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    {
+        const beagle_status st0 = device_setup_once(ctx, stream);
+        if (st0 != BEAGLE_OK) return st0;
+    }
     char* ws = static_cast<char*>(ws_dev);
     const int dt = c.dtype;
     const int M = batch * S;
@@ -969,8 +1032,7 @@ static beagle_status block_forward_impl(beagle_ctx* ctx, int32_t batch, int32_t 
             StageTimer timer_(ctx, ST_BLK_ATTN, stream);
             rc = -1;
             if (ctx->tc != nullptr) {       // bf16, head_dim 64 / 128: tensor-core tiles
-                clear_error_word_once(ctx, stream);
-                float* lse2 = (loss != nullptr && step == sim_steps) ? loss->lse2 : nullptr;
+                    float* lse2 = (loss != nullptr && step == sim_steps) ? loss->lse2 : nullptr;
                 if (c.head_dim == 64 || c.head_dim == 128) {
                     // tcgen05 path: it consumes the values transposed (keys contiguous), one padded column block per sequence
                     void *VtT = ws + L.vtT, *VpT = ws + L.vpT;
@@ -1367,14 +1429,17 @@ beagle_status beagle_verify_greedy(beagle_ctx* ctx, int32_t batch, int32_t gamma
     if (target_logits_dev != nullptr && logits_dtype != BEAGLE_FP32 && logits_dtype != BEAGLE_BF16)
         return fail(ctx, BEAGLE_ERR_INVALID_ARG, "verify: unknown logits_dtype");
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    const int32_t* ids = target_ids_dev;
-    StageTimer timer_(ctx, ST_VERIFY, stream);
     if (target_logits_dev != nullptr) {
-        ctx->launches += launch_row_argmax(logits_dtype, target_logits_dev, batch * (gamma + 1), ctx->cfg.vocab,
-                                           ctx->verify_keys, ctx->ids, stream);
-        ids = ctx->ids;
+        // one launch: arg-max partials of every logit row + the acceptance walk by the CTA that finishes a sequence last
+        const beagle_status st = device_setup_once(ctx, stream);
+        if (st != BEAGLE_OK) return st;
+        StageTimer timer_(ctx, ST_VERIFY, stream);
+        ctx->launches += launch_verify_greedy_fused(logits_dtype, target_logits_dev, batch, gamma, ctx->cfg.vocab, draft_tokens_dev,
+                                                    ctx->verify_keys, verify_tickets(ctx), ctx->sm_count, accept_len_dev, out_tokens_dev, stream);
+    } else {
+        StageTimer timer_(ctx, ST_VERIFY, stream);
+        ctx->launches += launch_accept(draft_tokens_dev, target_ids_dev, batch, gamma, accept_len_dev, out_tokens_dev, stream);
     }
-    ctx->launches += launch_accept(draft_tokens_dev, ids, batch, gamma, accept_len_dev, out_tokens_dev, stream);
     return cuda_ok(ctx, "verify_greedy");
 }
 
@@ -1416,14 +1481,14 @@ beagle_status beagle_draft_tree(beagle_ctx* ctx, int32_t slot, const int32_t* ro
     const int tail = depth > 0 ? 1 + (depth - 1) * topk : 0;          // draft states that enter the cache
     if (tail > c.max_draft) return fail(ctx, BEAGLE_ERR_CAPACITY, "draft_tree: %d draft states exceed max_draft %d", tail, c.max_draft);
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    clear_error_word_once(ctx, stream);
     const TreeArrays T = tree_arrays_carve(ctx->tree_mem, c.vocab);
     const int n_true = ctx->n_true[slot];
-    // the tree starts from the true states: whatever chain-draft tail the slot had is dropped
-    ctx->n_draft[slot] = 0; ctx->pending[slot] = 0; ctx->has_token[slot] = 0; ctx->steps[slot] = 0;
     if (c.rope_theta > 0.f && n_true + depth >= ctx->rope_rows)
         return fail(ctx, BEAGLE_ERR_CAPACITY, "draft_tree: positions up to %d exceed max_ctx + max_draft", n_true + depth + 1);
-    rope_table_once(ctx, stream);
+    const beagle_status st0 = device_setup_once(ctx, stream);
+    if (st0 != BEAGLE_OK) return st0;
+    // every check has passed: the tree starts from the true states, whatever chain-draft tail the slot had is dropped
+    ctx->n_draft[slot] = 0; ctx->pending[slot] = 0; ctx->has_token[slot] = 0; ctx->steps[slot] = 0;
     const int dt = c.dtype;
     int rc = 0;
 #define BEAGLE_TREE_SKINNY(MODE, ARGS, WHAT)                                              \

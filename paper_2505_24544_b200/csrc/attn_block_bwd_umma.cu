@@ -603,12 +603,12 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_q_umma_kernel(const _
 
 template <int DH>
 int launch_ubwd(const CUtensorMap* m, const UBwdArgs& a, int B, int nz, cudaStream_t stream) {
-    static bool attr_done = false;
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(attn_bwd_kv_umma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, UBwdKvSmem<DH>::kBytes) != cudaSuccess) return -1;
-        if (cudaFuncSetAttribute(attn_bwd_q_umma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, UBwdQSmem<DH>::kBytes) != cudaSuccess) return -1;
-        attr_done = true;
-    }
+    static PerDeviceOnce smem_attr;
+    if (!smem_attr.ensure([] {
+            return cudaFuncSetAttribute(attn_bwd_kv_umma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, UBwdKvSmem<DH>::kBytes) == cudaSuccess &&
+                   cudaFuncSetAttribute(attn_bwd_q_umma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, UBwdQSmem<DH>::kBytes) == cudaSuccess;
+        }))
+        return -1;
     const int tiles = (a.S + kBM - 1) / kBM;
     // maps: 0 Q128, 1 dO128, 2 Q64, 3 dO64, 4 K128, 5 V128, 6 Kp128, 7 Vp128, 8 K64, 9 V64, 10 Kp64, 11 Vp64, 12 QT, 13 dOT, 14 KT, 15 KpT
     attn_bwd_q_umma_kernel<DH><<<dim3(tiles, a.Hq, B), kBwdThreads, UBwdQSmem<DH>::kBytes, stream>>>(m[0], m[1], m[8], m[9], m[10], m[11], m[14], m[15], a);

@@ -337,11 +337,9 @@ __global__ void __launch_bounds__(kUThreads, 2) attn_block_umma_kernel(const __g
 template <int DH>
 int launch_umma_attn(const CUtensorMap* maps, const UmmaAttnArgs& a, int Sp, dim3 grid, cudaStream_t stream) {
     using SM = UmmaAttnSmem<DH>;
-    static bool attr_done = false;
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(attn_block_umma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kBytes) != cudaSuccess) return -1;
-        attr_done = true;
-    }
+    static PerDeviceOnce smem_attr;
+    if (!smem_attr.ensure([] { return cudaFuncSetAttribute(attn_block_umma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kBytes) == cudaSuccess; }))
+        return -1;
     attn_block_umma_kernel<DH><<<grid, kUThreads, SM::kBytes, stream>>>(maps[0], maps[1], maps[2], maps[3], maps[4], a, Sp);
     return 1;
 }

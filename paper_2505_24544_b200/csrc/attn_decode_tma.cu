@@ -68,7 +68,7 @@ __device__ __forceinline__ uint32_t tile_off(int row, int chunk) {
 template <int DH, int G>
 __global__ void __launch_bounds__(kWarps * 32) attn_decode_tma_kernel(const __grid_constant__ CUtensorMap tmK,
                                                                      const __grid_constant__ CUtensorMap tmV,
-                                                                     const bf16* __restrict__ q, const AttnWork work, int nbatch,
+                                                                     const bf16* q, const AttnWork work, int nbatch,
                                                                      int Hq, int Hkv, int cap, int nch_stride, float scale_log2,
                                                                      float* part_o, float* part_ml, int* done_count,
                                                                      bf16* __restrict__ o_out, int* error_word) {
@@ -92,6 +92,7 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_tma_kernel(const __gr
     const int start = chunk * kChunk;
     const int cnt = min(kChunk, kv_len - start);       // >= 1 by construction of item_start
     const int row0 = (work.slot[b] * Hkv + kvh) * cap + start;
+    (void)BEAGLE_IN_BOUNDS(cnt >= 1 && kv_len <= cap && BEAGLE_SLOT_OK(work.slot[b]));     // (a TMA tile past the tensor's end reads zeros: nothing to skip)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, c = lane & 3;
@@ -127,8 +128,8 @@ __global__ void __launch_bounds__(kWarps * 32) attn_decode_tma_kernel(const __gr
         const uint32_t* qrow = reinterpret_cast<const uint32_t*>(q + ((size_t)b * Hq + kvh * G + (g < G ? g : 0)) * DH);
 #pragma unroll
         for (int ks = 0; ks < DH / 16; ++ks) {
-            qa[ks][0] = g < G ? __ldg(qrow + ks * 8 + c) : 0u;          // dims 16ks + 2c, +1
-            qa[ks][1] = g < G ? __ldg(qrow + ks * 8 + 4 + c) : 0u;      // dims 16ks + 8 + 2c, +1
+            qa[ks][0] = g < G ? ld_act32(qrow + ks * 8 + c) : 0u;         // dims 16ks + 2c, +1
+            qa[ks][1] = g < G ? ld_act32(qrow + ks * 8 + 4 + c) : 0u;     // dims 16ks + 8 + 2c, +1
         }
     }
     __syncthreads();                                                     // barriers initialised
@@ -275,11 +276,9 @@ int launch_attn(const CUtensorMap& mk, const CUtensorMap& mv, const bf16* q, con
                 int Hkv, int cap, int nch_stride, float scale_log2, float* po, float* pml, int* done_count, bf16* o, int* error_word,
                 cudaStream_t stream) {
     constexpr int kSmem = 2 * kChunk * DH * 2 + 1024 + 64;
-    static bool attr_done = false;
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(attn_decode_tma_kernel<DH, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) != cudaSuccess) return -1;
-        attr_done = true;
-    }
+    static PerDeviceOnce smem_attr;
+    if (!smem_attr.ensure([] { return cudaFuncSetAttribute(attn_decode_tma_kernel<DH, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem) == cudaSuccess; }))
+        return -1;
     launch_pdl(attn_decode_tma_kernel<DH, G>, dim3(items, Hkv), dim3(kWarps * 32), (size_t)kSmem, stream, mk, mv, q, work, nbatch, Hq, Hkv,
                cap, nch_stride, scale_log2, po, pml, done_count, o, error_word);
     return 1;

@@ -26,15 +26,35 @@ template <> struct VecOf<bf16>  { static constexpr int N = 8; };
 
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t hi16) { return __uint_as_float(hi16 << 16); }
 
-// 16-byte read-only load that does not allocate in L1 (weights and cache rows are read once).
+// 16-byte read-only (non-coherent) load that does not allocate in L1.  ONLY for data that no kernel writes while the
+// reading kernel may be resident: weights, logits handed in by the caller, cache rows of true states.
 __device__ __forceinline__ uint4 ld_stream16(const void* p) {
     uint4 v;
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
     return v;
 }
-// 16-byte cached load (activations re-read by many warps).
+// 16-byte read-only (non-coherent) cached load: same restriction as ld_stream16.
 __device__ __forceinline__ uint4 ld_cached16(const void* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+// 16-byte ordinary (coherent) loads for everything a kernel of the same launch chain writes -- activations, Q, the slots'
+// previous states, cache rows of the draft tail: with programmatic dependent launch the reader may already be resident
+// while the producer still runs, which the non-coherent path does not allow.  To be issued after pdl_wait().
+__device__ __forceinline__ uint4 ld_act16(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint32_t ld_act32(const void* p) {
+    uint32_t v;
+    asm volatile("ld.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint4 ld_act_stream16(const void* p) {       // the same, without allocating in L1 (read once)
+    uint4 v;
+    asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
 
 template <typename T> __device__ __forceinline__ void unpack16(const uint4& v, float* f);
 template <> __device__ __forceinline__ void unpack16<float>(const uint4& v, float* f) {
@@ -88,16 +108,57 @@ __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long k)
 
 __device__ __forceinline__ float silu_f(float u) { return u / (1.0f + __expf(-u)); }
 
+// Bounds-checking build (-DBEAGLE_BOUNDS_CHECK; a second library, built with relocatable device code, for tests).
+// Every access whose index comes from the host's per-call metadata -- cache slot and position of a scatter or a chunk,
+// row maps, token ids -- is guarded by BEAGLE_IN_BOUNDS(condition): a violation raises the device error word of the
+// context that was set up last (value 2, reported by beagle_check_device) and the access is SKIPPED; nothing traps.
+// In the ordinary build the macro is the constant `true` and no code is generated.
+#ifdef BEAGLE_BOUNDS_CHECK
+extern __device__ int* g_bounds_word;          // bound by the context's device set-up (api.cu)
+extern __device__ int g_bounds_slots;          // max_slots of that context
+__device__ __forceinline__ bool bounds_report(bool ok) {
+    if (!ok && g_bounds_word != nullptr) atomicExch(g_bounds_word, 2);
+    return ok;
+}
+#define BEAGLE_IN_BOUNDS(cond) (::beagle::bounds_report(cond))
+#define BEAGLE_SLOT_OK(slot) ((slot) >= 0 && (slot) < ::beagle::g_bounds_slots)
+#else
+#define BEAGLE_IN_BOUNDS(cond) true
+#define BEAGLE_SLOT_OK(slot) true
+#endif
+
 // Programmatic dependent launch.  The serve-time kernels are launched so that a kernel may start
 // while its predecessor in the stream is still draining: everything before pdl_wait() must touch
 // only memory that no kernel of the chain writes (weights, the stable part of the K/V cache) and
 // must write no global memory; pdl_wait() returns once the predecessor has completed and its
-// writes are visible.  Every kernel launched this way calls pdl_wait() on every thread, so that a
+// writes are visible.  Loads rule: the non-coherent loads (ld.global.nc, __ldg: ld_stream16 /
+// ld_cached16) are for weights and true-state cache rows only; whatever a kernel of the chain
+// writes (activations, Q, h_slot, draft-tail cache rows, split partials) is read with ordinary
+// loads (ld_act16 / ld_act32 / ld_act_stream16, TMA, or plain C++ loads through pointers that are
+// NOT declared `const ... __restrict__` -- that pair lets the compiler pick the non-coherent path
+// by itself) issued after pdl_wait().  Every kernel launched this way calls pdl_wait() on every thread, so that a
 // kernel's completion implies the completion of all kernels before it.  Both are no-ops for a
 // plain launch.
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
+
+// Function attributes are per device.  One of these per kernel instantiation (a function-local static) remembers on which
+// devices the dynamic shared-memory limit has been raised, so a process that drives several GPUs sets it on each.
+struct PerDeviceOnce {
+    static constexpr int kMaxDevices = 64;
+    bool done[kMaxDevices] = {};
+    // True when `fn` has been applied on the current device (now or earlier); false when it failed.
+    template <typename F>
+    bool ensure(F fn) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return false;
+        if (done[dev]) return true;
+        if (!fn()) return false;
+        done[dev] = true;
+        return true;
+    }
+};
 
 // Launch with the programmatic-stream-serialization attribute (falls back to a plain launch if the
 // attribute is refused).

@@ -7,7 +7,7 @@
 // columns, warps 2..5 read the accumulator (thread = output feature, register j = batch row j)
 // and either write fp32 partial sums [split][matrix][b][n] for the finishing kernel below or, for
 // the LM head, logits and one packed arg-max key per (b, tile).  Shared memory is sized so that
-// two CTAs share an SM: one CTA's prologue and epilogue hide behind the other's stream.
+// three CTAs share an SM: one CTA's prologue and epilogue hide behind the others' streams.
 //
 // Every wait on an mbarrier is bounded; a wait that runs out raises a device error word and the
 // CTA drains its copies and frees its TMEM instead of hanging.
@@ -256,7 +256,7 @@ __device__ __forceinline__ void sk_body(const CUtensorMap* mapW, const CUtensorM
                 fin.out[(size_t)col * fin.ldo + n] = __float2bfloat16_rn(silu_f(v) * v1);
             } else if (mode == SK_KV) {
                 const int pos = fin.pos.idx[col];
-                if (pos >= 0) {
+                if (pos >= 0 && BEAGLE_IN_BOUNDS(pos < fin.cap && BEAGLE_SLOT_OK(fin.slot.idx[col]))) {
                     bf16* cache = me ? fin.vcache : fin.kcache;
                     cache[(((size_t)fin.slot.idx[col] * fin.Hkv + n / fin.dh) * fin.cap + pos) * fin.dh + n % fin.dh] = __float2bfloat16_rn(v);
                 }
@@ -355,7 +355,7 @@ __global__ void __launch_bounds__(kFinThreads) tc_finish_kernel(const FinishArgs
         }
         if (MODE == SK_KV) {
             const int slot = a.slot.idx[b], pos = a.pos.idx[b];
-            if (pos >= 0) {
+            if (pos >= 0 && BEAGLE_IN_BOUNDS(pos < a.cap && BEAGLE_SLOT_OK(slot))) {
                 const float v1[4] = {s1.x, s1.y, s1.z, s1.w};
                 const size_t at = (((size_t)slot * a.Hkv + n / a.dh) * a.cap + pos) * a.dh + n % a.dh;   // dh % 4 == 0
 #pragma unroll
@@ -418,11 +418,9 @@ template <int BN, int VAR, bool FP8 = false>
 int launch_sk(const CUtensorMap& w, const CUtensorMap& w2, const CUtensorMap& x, const SkArgs& args, const FinishArgs& fin, int mode,
               dim3 grid, dim3 cluster, cudaStream_t stream) {
     using SM = SkSmem<BN>;
-    static bool attr_done = false;
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(tc_skinny_kernel<BN, VAR, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kBytes) != cudaSuccess) return -1;
-        attr_done = true;
-    }
+    static PerDeviceOnce smem_attr;
+    if (!smem_attr.ensure([] { return cudaFuncSetAttribute(tc_skinny_kernel<BN, VAR, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kBytes) == cudaSuccess; }))
+        return -1;
     if (VAR != 2) {
         launch_pdl(tc_skinny_kernel<BN, VAR, FP8>, grid, dim3(kSkThreads), SM::kBytes, stream, w, w2, x, args, fin, mode);
         return 1;
@@ -456,11 +454,9 @@ template <int BN>
 int launch_sk_qkv(const CUtensorMap& wq, const CUtensorMap& wk, const CUtensorMap& wv, const CUtensorMap& xq, const CUtensorMap& xkv,
                   const SkArgs& args, const FinishArgs& fin, int q_tiles, int kv_tiles, int kv_N, int cs, cudaStream_t stream) {
     using SM = SkSmem<BN>;
-    static bool attr_done = false;
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(tc_skinny_qkv_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kBytes) != cudaSuccess) return -1;
-        attr_done = true;
-    }
+    static PerDeviceOnce smem_attr;
+    if (!smem_attr.ensure([] { return cudaFuncSetAttribute(tc_skinny_qkv_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kBytes) == cudaSuccess; }))
+        return -1;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(q_tiles + 2 * kv_tiles, 1, cs); cfg.blockDim = dim3(kSkThreads); cfg.dynamicSmemBytes = SM::kBytes; cfg.stream = stream;
     cudaLaunchAttribute attr[2];

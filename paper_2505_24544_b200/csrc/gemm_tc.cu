@@ -32,7 +32,7 @@ constexpr int kTcThreads = 192;
 
 // ---------------------------------------------------------------------------------------------- kernel
 enum TcEpilogue {
-    TC_STORE = 0, TC_RESID = 1, TC_SILU_MUL = 2, TC_F32 = 3, TC_KV_CACHE = 4, TC_ARGMAX = 5, TC_CE = 6, TC_DLOGITS = 7
+    TC_STORE = 0, TC_RESID = 1, TC_SILU_MUL = 2, TC_F32 = 3, TC_KV_CACHE = 4, TC_ARGMAX = 5, TC_CE = 6, TC_DLOGITS = 7, TC_KV_PAIR = 8
 };
 
 struct TcArgs {
@@ -41,7 +41,7 @@ struct TcArgs {
     int tiles_a, tiles_b;
     void* C; int ldc;
     const void* R; int ldr;
-    void* cache; int Hkv, dh, cap;
+    void* cache; void* cache2; int Hkv, dh, cap;
     SeqRows rows;
     unsigned long long* keys; int keys_ld;
     const void* tgt; int tgt_dtype; int ldt; const int32_t* labels; float* ce_part;   // TC_CE, TC_DLOGITS
@@ -49,18 +49,21 @@ struct TcArgs {
     int* error_word;
 };
 
-template <int BN, bool DUAL>
+template <int BN, bool DUAL, int EPI = TC_STORE>
 struct TcSmem {
     static constexpr int kStageBytes = (BM + BN * (DUAL ? 2 : 1)) * BK * 2;
     static constexpr int kStages = (BN >= 128) ? 4 : 5;
-    static constexpr int kBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+    // TC_KV_PAIR: every epilogue warp transposes its 32 rows x BN columns through shared memory so that whole cache rows
+    // leave the SM as contiguous 16-byte pieces
+    static constexpr int kStagingBytes = (EPI == TC_KV_PAIR) ? BM * BN * 2 : 0;
+    static constexpr int kBytes = kStages * kStageBytes + kStagingBytes + 1024 /*align*/ + 256 /*barriers*/;
 };
 
 template <int BN, bool DUAL, int EPI>
 __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
                                                             const __grid_constant__ CUtensorMap tmB,
                                                             const __grid_constant__ CUtensorMap tmB2, const TcArgs args) {
-    using SM = TcSmem<BN, DUAL>;
+    using SM = TcSmem<BN, DUAL, EPI>;
     constexpr int kStages = SM::kStages;
     constexpr int kABytes = BM * BK * 2, kBBytes = BN * BK * 2;
     constexpr uint32_t kAccCols = DUAL ? 2 * BN : BN;       // TMEM columns of one tile's accumulator(s)
@@ -69,7 +72,8 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + kStages * SM::kStageBytes);
+    uint8_t* smem_staging = smem_gen + kStages * SM::kStageBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_staging + SM::kStagingBytes);
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * kStages;
     const uint32_t bar_acc_full = bar_empty + 8 * kStages, bar_acc_empty = bar_acc_full + 16;     // two accumulator buffers
     uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 4);
@@ -186,14 +190,67 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
             if (!ok) break;
             fence_after();
             const uint32_t taddr = tmem_base + buf * kAccCols + (static_cast<uint32_t>(q * 32) << 16);
-            {
-                const int m = arow;
+            if constexpr (EPI == TC_KV_PAIR) {
+                // K (columns [0, BN) of the accumulator) then V ([BN, 2 BN)): bf16 rows through this warp's staging
+                // block (16-byte pieces, XOR-swizzled by row so that neither side has bank conflicts), then out with
+                // 16 lanes per cache row: one row's BN columns leave as contiguous 16-byte pieces.
+                static_assert(BN == 128, "staging layout: 16 pieces of 16 bytes per row");
+                uint8_t* stg = smem_staging + q * (32 * BN * 2);
+                long long rowoff = -1;               // element offset of (slot, head 0, pos, 0) in a cache half; -1: row out of range
+                if (arow < args.a_rows) {
+                    int b = 0;
+                    while (b + 1 < args.rows.n && arow >= args.rows.row_start[b + 1]) ++b;
+                    const int pos = args.rows.pos_start[b] + (arow - args.rows.row_start[b]);
+                    if (BEAGLE_IN_BOUNDS(pos >= 0 && pos < args.cap && BEAGLE_SLOT_OK(args.rows.slot[b])))
+                        rowoff = ((long long)args.rows.slot[b] * args.Hkv * args.cap + pos) * args.dh;
+                }
+#pragma unroll 1
+                for (int mat = 0; mat < 2; ++mat) {
+                    __syncwarp();                    // the previous read-out of the staging block is complete
+#pragma unroll 1
+                    for (int c0 = 0; c0 < BN; c0 += 32) {
+                        uint32_t ra[16], rb[16];
+                        tmem_ld16(taddr + mat * BN + c0, ra);
+                        tmem_ld16(taddr + mat * BN + c0 + 16, rb);
+                        tmem_ld_wait();
+                        uint32_t p[16];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            __nv_bfloat162 t = __floats2bfloat162_rn(__uint_as_float(ra[2 * j]), __uint_as_float(ra[2 * j + 1]));
+                            p[j] = *reinterpret_cast<uint32_t*>(&t);
+                            t = __floats2bfloat162_rn(__uint_as_float(rb[2 * j]), __uint_as_float(rb[2 * j + 1]));
+                            p[8 + j] = *reinterpret_cast<uint32_t*>(&t);
+                        }
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const int piece = c0 / 8 + j;
+                            *reinterpret_cast<uint4*>(stg + lane * (BN * 2) + ((piece ^ (lane & 15)) << 4)) =
+                                make_uint4(p[4 * j], p[4 * j + 1], p[4 * j + 2], p[4 * j + 3]);
+                        }
+                    }
+                    __syncwarp();
+                    bf16* cache = reinterpret_cast<bf16*>(mat == 0 ? args.cache : args.cache2);
+                    const int piece = lane & 15;
+                    const int n = tb * BN + piece * 8;                  // first of this lane's 8 columns
+                    const int head = n / args.dh, within = n - head * args.dh;
+#pragma unroll 4
+                    for (int i = 0; i < 16; ++i) {
+                        const int r = 2 * i + (lane >> 4);
+                        const long long off = __shfl_sync(0xffffffffu, rowoff, r);
+                        const uint4 v = *reinterpret_cast<const uint4*>(stg + r * (BN * 2) + ((piece ^ (r & 15)) << 4));
+                        if (off >= 0 && n < args.b_rows)
+                            *reinterpret_cast<uint4*>(cache + off + (long long)head * args.cap * args.dh + within) = v;
+                    }
+                }
+            } else {
+                int m = arow;
                 int slot = 0, pos = 0;
                 if (EPI == TC_KV_CACHE && m < args.a_rows) {
                     int b = 0;
                     while (b + 1 < args.rows.n && m >= args.rows.row_start[b + 1]) ++b;
                     slot = args.rows.slot[b];
                     pos = args.rows.pos_start[b] + (m - args.rows.row_start[b]);
+                    if (!BEAGLE_IN_BOUNDS(pos >= 0 && pos < args.cap && BEAGLE_SLOT_OK(slot))) m = args.a_rows;     // the row's stores are skipped
                 }
                 unsigned long long best = 0ull;
                 float ce_mq = -INFINITY, ce_sq = 0.f, ce_mt = -INFINITY, ce_st = 0.f, ce_dot = 0.f;   // TC_CE running partial
@@ -370,6 +427,21 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
     }
 }
 
+// Self-test of the bounded-wait protocol: one CTA waits, with a short poll limit, on an mbarrier that nothing will ever
+// complete (no copy is in flight, no other role exists), gives up, raises the device error word exactly as the real
+// kernels do after their limit, and returns.  Nothing hangs and nothing faults: the wait simply runs out.
+__global__ void wait_timeout_selftest_kernel(int* error_word, uint32_t limit) {
+    __shared__ uint64_t bar;
+    __shared__ int s_abort;
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        mbar_init(smem_u32(&bar), 1);
+        fence_barrier_init();
+        const bool ok = mbar_wait_limit(smem_u32(&bar), 0, &s_abort, limit);
+        if (!ok && s_abort && error_word != nullptr) atomicExch(error_word, 1);
+    }
+}
+
 // Reduces the dense LM head's per-tile keys [rows, ntiles] to ids.
 __global__ void tc_keys_to_ids_kernel(const unsigned long long* __restrict__ keys, int rows, int ntiles, int32_t* __restrict__ ids) {
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
@@ -426,12 +498,10 @@ namespace {
 
 template <int BN, bool DUAL, int EPI>
 int launch_tc(const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& b2, const TcArgs& args, dim3 grid, cudaStream_t stream) {
-    using SM = TcSmem<BN, DUAL>;
-    static bool attr_done = false;
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(tc_gemm_kernel<BN, DUAL, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kBytes) != cudaSuccess) return -1;
-        attr_done = true;
-    }
+    using SM = TcSmem<BN, DUAL, EPI>;
+    static PerDeviceOnce smem_attr;
+    if (!smem_attr.ensure([] { return cudaFuncSetAttribute(tc_gemm_kernel<BN, DUAL, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kBytes) == cudaSuccess; }))
+        return -1;
     tc_gemm_kernel<BN, DUAL, EPI><<<grid, kTcThreads, SM::kBytes, stream>>>(a, b, b2, args);
     return 1;
 }
@@ -469,7 +539,7 @@ int tc_gemm(TcPlan* p, int epi, const GemmArgs& g, cudaStream_t stream) {
     if (p == nullptr) return -1;
     if (g.K % 8 || g.lda % 8) return -1;                       // TMA: 16-byte row pitch
     if (reinterpret_cast<uintptr_t>(g.A) & 15) return -1;
-    const bool dual = (epi == GEMM_SILU_MUL);
+    const bool dual = (epi == GEMM_SILU_MUL || epi == GEMM_KV_CACHE_PAIR);
     const int BN = dual ? 128 : 256;
     CUtensorMap mapA;
     if (!tc_encode_map(p, &mapA, g.A, g.M, g.K, g.lda, BM)) return -1;
@@ -490,12 +560,15 @@ int tc_gemm(TcPlan* p, int epi, const GemmArgs& g, cudaStream_t stream) {
     a.tiles_b = (g.N + BN - 1) / BN;
     a.group_m = 16;
     a.C = g.C; a.ldc = g.ldc; a.R = g.R; a.ldr = g.ldr;
-    a.cache = g.cache; a.Hkv = g.Hkv; a.dh = g.dh; a.cap = g.cap; a.rows = g.rows;
+    a.cache = g.cache; a.cache2 = g.cache2; a.Hkv = g.Hkv; a.dh = g.dh; a.cap = g.cap; a.rows = g.rows;
     a.keys = g.keys; a.keys_ld = a.tiles_b;
     a.tgt = g.tgt; a.tgt_dtype = g.tgt_dtype; a.ldt = g.ldt; a.labels = g.labels; a.ce_part = g.ce_part;
     a.row_stats = g.row_stats; a.row_coef = g.row_coef;
     a.error_word = g.error_word;
     if (epi == GEMM_KV_CACHE && (g.dh % 16)) return -1;
+    if (epi == GEMM_KV_CACHE_PAIR && ((g.dh % 8) || (g.N % 8) || g.cache == nullptr || g.cache2 == nullptr ||
+                                      ((reinterpret_cast<uintptr_t>(g.cache) | reinterpret_cast<uintptr_t>(g.cache2)) & 15)))
+        return -1;
     const int ntiles = a.tiles_a * a.tiles_b;
     dim3 grid(ntiles < p->sm_count ? ntiles : p->sm_count, 1, 1);        // persistent: one CTA per SM
     switch (epi) {
@@ -507,8 +580,14 @@ int tc_gemm(TcPlan* p, int epi, const GemmArgs& g, cudaStream_t stream) {
         case GEMM_ARGMAX_KEYS: return launch_tc<256, false, TC_ARGMAX>(mapA, *mapB, *mapB, a, grid, stream);
         case GEMM_CE: return launch_tc<256, false, TC_CE>(mapA, *mapB, *mapB, a, grid, stream);
         case GEMM_DLOGITS: return launch_tc<256, false, TC_DLOGITS>(mapA, *mapB, *mapB, a, grid, stream);
+        case GEMM_KV_CACHE_PAIR: return launch_tc<128, true, TC_KV_PAIR>(mapA, *mapB, *mapB2, a, grid, stream);
         default: return -1;
     }
+}
+
+int launch_wait_timeout_selftest(int* error_word, cudaStream_t stream) {
+    wait_timeout_selftest_kernel<<<1, 32, 0, stream>>>(error_word, 4096u);
+    return 1;
 }
 
 int tc_argmax_tiles(int N) { return (N + 255) / 256; }

@@ -18,6 +18,10 @@ int tc_gemm(TcPlan* plan, int epi, const GemmArgs& a, cudaStream_t stream);
 int tc_argmax_tiles(int N);
 int tc_keys_to_ids(const unsigned long long* keys, int rows, int ntiles, int32_t* ids, cudaStream_t stream);
 
+// Test support: a one-CTA kernel whose bounded mbarrier wait (short limit, nothing ever arrives, no copy in flight) runs
+// out and raises `error_word`, as the tensor-core kernels do when a wait of theirs gives up.
+int launch_wait_timeout_selftest(int* error_word, cudaStream_t stream);
+
 // ---- serve-time projections for 9..64 rows ("swap-AB") -----------------------------------------
 // The weight matrix supplies the 128 MMA rows and the batch's activations the (<= 64) columns, so
 // the weights are streamed exactly once whatever the batch.  The reduction dimension may be split

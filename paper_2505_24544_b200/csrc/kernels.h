@@ -65,6 +65,13 @@ int launch_argmax_finalize(const unsigned long long* partials, int nblk, const B
 constexpr int kRowArgmaxSplit = 16;
 int launch_row_argmax(int logits_dtype, const void* logits, int rows, int V, unsigned long long* scratch,
                       int32_t* ids_out, cudaStream_t stream);
+// Greedy verification from target logits [B, gamma+1, V] (fp32 or bf16) in one launch: arg-max partial keys per (row, slice)
+// and the acceptance walk by the CTA that finishes a sequence last.  keys: B * (gamma+1) * kVerifyMaxSplit entries (any
+// contents); tickets: B ints, zero before the first launch (the kernel leaves them zero).
+constexpr int kVerifyMaxSplit = 64;
+int launch_verify_greedy_fused(int logits_dtype, const void* logits, int B, int gamma, int V, const int32_t* draft,
+                               unsigned long long* keys, int* tickets, int sm_count, int32_t* accept_len, int32_t* out_tokens,
+                               cudaStream_t stream);
 // Greedy acceptance from target ids.
 int launch_accept(const int32_t* draft, const int32_t* target_ids, int B, int gamma, int32_t* accept_len,
                   int32_t* out_tokens, cudaStream_t stream);
@@ -120,7 +127,8 @@ enum GemmEpilogue {
     GEMM_KV_CACHE = 4,   // scatter rows into the cache: row r -> (slot, pos) through SeqRows
     GEMM_ARGMAX_KEYS = 5,// no C: one packed arg-max key per (row, column tile)   (tensor-core path only)
     GEMM_CE = 6,         // no C: cross-entropy partials per (row, column tile)       (tensor-core path only)
-    GEMM_DLOGITS = 7     // C = row_coef * (softmax(A W^T) - p), storage type, from the rows' softmax statistics (tensor-core path only)
+    GEMM_DLOGITS = 7,    // C = row_coef * (softmax(A W^T) - p), storage type, from the rows' softmax statistics (tensor-core path only)
+    GEMM_KV_CACHE_PAIR = 8  // A W^T -> `cache` and A W2^T -> `cache2` in ONE pass over A, rows scattered as GEMM_KV_CACHE (tensor-core path only)
 };
 // Cross-entropy partial of one (row, column range): running max / exp-sum of the draft logits z,
 // running max / exp-sum of the target logits t and sum exp(t - tmax) * z (soft targets); with hard
@@ -139,6 +147,7 @@ struct GemmArgs {
     void* C; int ldc;
     const void* R; int ldr;
     void* cache; int Hkv, dh, cap;  // GEMM_KV_CACHE
+    void* cache2;                   // GEMM_KV_CACHE_PAIR: the second matrix's cache
     unsigned long long* keys;       // GEMM_ARGMAX_KEYS
     const void* tgt; int tgt_dtype; int ldt;   // GEMM_CE, soft targets: target logits [M, ldt] (0 fp32, 1 bf16)
     const int32_t* labels;          // GEMM_CE, hard targets: [M] (used when tgt == NULL)

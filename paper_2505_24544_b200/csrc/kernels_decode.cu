@@ -10,13 +10,12 @@ namespace beagle {
 // Embedding gather + RMSNorm (Eq. 1: e(t_p); normalisation as configured)
 // ------------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(256) embed_norm_kernel(const int32_t* __restrict__ tokens,
-                                                         const int32_t* __restrict__ last_token,
-                                                         const BatchMeta meta,
-                                                         const T* __restrict__ embed, int vocab,
-                                                         const T* __restrict__ src, const T* __restrict__ gain,
+__global__ void __launch_bounds__(256) embed_norm_kernel(const int32_t* tokens, const int32_t* last_token,     // (no __restrict__ on
+                                                         const BatchMeta meta,                                   //  what earlier kernels of the
+                                                         const T* __restrict__ embed, int vocab,                //  launch chain write)
+                                                         const T* src, const T* __restrict__ gain,
                                                          int d, float eps, int do_norm, T* __restrict__ x_out,
-                                                         T* __restrict__ xn_out, const T* __restrict__ gather_src,
+                                                         T* __restrict__ xn_out, const T* gather_src,
                                                          T* __restrict__ gather_dst) {
     constexpr int VEC = VecOf<T>::N;
     constexpr int kMaxVec = 4;                  // 16-byte pieces a thread keeps in registers (d <= 256 * 4 * VEC)
@@ -31,13 +30,14 @@ __global__ void __launch_bounds__(256) embed_norm_kernel(const int32_t* __restri
     if (gather_src != nullptr) {
         const uint4* g = reinterpret_cast<const uint4*>(gather_src + (size_t)meta.slot[r] * d);
         uint4* dst = reinterpret_cast<uint4*>(gather_dst + (size_t)r * d);
-        for (int i = threadIdx.x; i < nvec; i += blockDim.x) dst[i] = g[i];
+        for (int i = threadIdx.x; i < nvec; i += blockDim.x) dst[i] = ld_act16(g + i);
     }
     const T* row;
     if (src != nullptr) {
         row = src + (size_t)r * d;
     } else {
         int tok = tokens != nullptr ? tokens[r] : last_token[meta.slot[r]];
+        (void)BEAGLE_IN_BOUNDS(tok >= 0 && tok < vocab && BEAGLE_SLOT_OK(meta.slot[r]));
         tok = min(max(tok, 0), vocab - 1);      // ids are validated by contract; never read out of range
         row = embed + (size_t)tok * d;
     }
@@ -49,7 +49,7 @@ __global__ void __launch_bounds__(256) embed_norm_kernel(const int32_t* __restri
 #pragma unroll
         for (int j = 0; j < kMaxVec; ++j) {
             const int i = threadIdx.x + j * blockDim.x;
-            keep[j] = i < nvec ? row4[i] : make_uint4(0u, 0u, 0u, 0u);
+            keep[j] = i < nvec ? ld_act16(row4 + i) : make_uint4(0u, 0u, 0u, 0u);
         }
 #pragma unroll
         for (int j = 0; j < kMaxVec; ++j) {
@@ -124,7 +124,7 @@ int launch_embed_norm(int dtype, const int32_t* tokens, const int32_t* last_toke
 // rows with 16-byte loads; the activations are re-read through L1.
 // ------------------------------------------------------------------------------------------------
 template <typename T, int NB, int MODE>
-__global__ void __launch_bounds__(256) gemv_kernel(const GemvArgs a) {
+__global__ void __launch_bounds__(256) stream_proj_kernel(const GemvArgs a) {
     constexpr int VEC = VecOf<T>::N;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int unit = blockIdx.x * 8 + warp;
@@ -180,7 +180,7 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvArgs a) {
 #pragma unroll
             for (int j = 0; j < NB; ++j) {
                 float xf[VEC];
-                unpack16<T>(ld_cached16(xp[j] + k), xf);
+                unpack16<T>(ld_act16(xp[j] + k), xf);      // activations: written by the previous kernel of the chain
 #pragma unroll
                 for (int v = 0; v < VEC; ++v) {
                     acc0[j] = fmaf(wf0[v], xf[v], acc0[j]);
@@ -235,6 +235,7 @@ __global__ void __launch_bounds__(256) gemv_kernel(const GemvArgs a) {
                     T* cache = reinterpret_cast<T*>(blockIdx.y == 1 ? a.vcache : a.kcache);
                     const int slot = a.orow2.idx[b], pos = a.pos.idx[b];
                     if (pos < 0) continue;          // this row appends nothing
+                    if (!BEAGLE_IN_BOUNDS(pos < a.cap && BEAGLE_SLOT_OK(slot))) continue;
                     if (v0) cache[(((size_t)slot * a.Hkv + n0 / a.dh) * a.cap + pos) * a.dh + n0 % a.dh] = from_float<T>(acc0[j]);
                     if (v1) cache[(((size_t)slot * a.Hkv + n1 / a.dh) * a.cap + pos) * a.dh + n1 % a.dh] = from_float<T>(acc1[j]);
                 }
@@ -251,10 +252,10 @@ int gemv_grid_blocks(int mode, int N) {
 
 template <typename T, int MODE>
 static void gemv_dispatch_nb(const GemvArgs& a, dim3 grid, cudaStream_t stream) {
-    if (a.B <= 1) launch_pdl(gemv_kernel<T, 1, MODE>, grid, dim3(256), 0, stream, a);
-    else if (a.B <= 2) launch_pdl(gemv_kernel<T, 2, MODE>, grid, dim3(256), 0, stream, a);
-    else if (a.B <= 4) launch_pdl(gemv_kernel<T, 4, MODE>, grid, dim3(256), 0, stream, a);
-    else launch_pdl(gemv_kernel<T, 8, MODE>, grid, dim3(256), 0, stream, a);
+    if (a.B <= 1) launch_pdl(stream_proj_kernel<T, 1, MODE>, grid, dim3(256), 0, stream, a);
+    else if (a.B <= 2) launch_pdl(stream_proj_kernel<T, 2, MODE>, grid, dim3(256), 0, stream, a);
+    else if (a.B <= 4) launch_pdl(stream_proj_kernel<T, 4, MODE>, grid, dim3(256), 0, stream, a);
+    else launch_pdl(stream_proj_kernel<T, 8, MODE>, grid, dim3(256), 0, stream, a);
 }
 template <typename T>
 static void gemv_dispatch_mode(int mode, const GemvArgs& a, dim3 grid, cudaStream_t stream) {
@@ -285,7 +286,7 @@ constexpr int kAttnWarps = 4;
 
 template <typename T, int G, int LPK>
 __global__ void __launch_bounds__(kAttnWarps * 32) attn_decode_kernel(
-    const T* __restrict__ q, const T* __restrict__ kcache, const T* __restrict__ vcache, const BatchMeta meta,
+    const T* q, const T* kcache, const T* vcache, const BatchMeta meta,       // written by earlier kernels of the chain: no __restrict__
     int Hq, int Hkv, int cap, int nchunk_max, float scale, float* __restrict__ part_o, float* __restrict__ part_ml) {
     constexpr int VEC = VecOf<T>::N;
     constexpr int DH = LPK * VEC;
@@ -299,6 +300,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attn_decode_kernel(
     if (start >= kv_len) return;
     const int cnt = min(kAttnChunk, kv_len - start);
     const int slot = meta.slot[b];
+    if (!BEAGLE_IN_BOUNDS(kv_len <= cap && BEAGLE_SLOT_OK(slot))) return;
     const size_t base = (((size_t)slot * Hkv + kvh) * cap + start) * DH;
     const T* kb = kcache + base;
     const T* vb = vcache + base;
@@ -326,7 +328,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attn_decode_kernel(
         const int j = jb + kgrp;
         const bool valid = j < cnt;
         float kf[VEC];
-        if (valid) unpack16<T>(ld_stream16(kb + (size_t)j * DH + sub * VEC), kf);
+        if (valid) unpack16<T>(ld_act_stream16(kb + (size_t)j * DH + sub * VEC), kf);    // may be a draft-tail row appended by the previous kernel
         else {
 #pragma unroll
             for (int v = 0; v < VEC; ++v) kf[v] = 0.f;
@@ -370,7 +372,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attn_decode_kernel(
         const int j = jb + kgrp;
         if (j < cnt) {
             float vf[VEC];
-            unpack16<T>(ld_stream16(vb + (size_t)j * DH + sub * VEC), vf);
+            unpack16<T>(ld_act_stream16(vb + (size_t)j * DH + sub * VEC), vf);
 #pragma unroll
             for (int g = 0; g < G; ++g) {
                 const float p = s_s[g][j];
@@ -406,7 +408,7 @@ __global__ void __launch_bounds__(kAttnWarps * 32) attn_decode_kernel(
 // One CTA of four warps per (sequence, query head): each warp merges a quarter of the chunks
 // (attn_combine_range), warp 0 merges the four results.
 template <typename T, int DPL>
-__global__ void __launch_bounds__(128) attn_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
+__global__ void __launch_bounds__(128) attn_combine_kernel(const float* part_o, const float* part_ml,      // the previous kernel's output
                                                           const BatchMeta meta, int Hq, int dh, int nchunk_max, int chunk,
                                                           int extra_chunks, T* __restrict__ o) {
     const int head = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -526,7 +528,7 @@ int launch_attn_decode(int dtype, const void* q, const void* kcache, const void*
 // ------------------------------------------------------------------------------------------------
 // Arg-max finalisation of the LM head's per-block keys
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(1024) argmax_finalize_kernel(const unsigned long long* __restrict__ partials, int nblk,
+__global__ void __launch_bounds__(1024) argmax_finalize_kernel(const unsigned long long* partials, int nblk,       // the LM head's output
                                                                const BatchMeta meta, int32_t* __restrict__ tokens_out,
                                                                int tokens_out_stride, int32_t* __restrict__ last_token) {
     const int b = blockIdx.x;
@@ -552,7 +554,7 @@ __global__ void __launch_bounds__(1024) argmax_finalize_kernel(const unsigned lo
         if (threadIdx.x == 0) {
             const int tok = argmax_key_index(key);
             if (tokens_out != nullptr) tokens_out[(size_t)b * tokens_out_stride] = tok;
-            last_token[meta.slot[b]] = tok;
+            if (BEAGLE_IN_BOUNDS(BEAGLE_SLOT_OK(meta.slot[b]))) last_token[meta.slot[b]] = tok;
         }
     }
     if (!release_early) pdl_launch_dependents();
@@ -627,6 +629,131 @@ int launch_row_argmax(int logits_dtype, const void* logits, int rows, int V, uns
     }
     row_argmax_final_kernel<<<(rows + 255) / 256, 256, 0, stream>>>(scratch, rows, ids_out);
     return (rows + 32767) / 32768 + 1;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Greedy verification from target logits in ONE launch (Section 3): CTA (slice, row) scans its slice
+// of one logit row with 16-byte streaming loads, leaves one packed key in `keys[row][slice]` and takes
+// a ticket of its sequence; the CTA that takes the sequence's last ticket reduces the (gamma + 1) x
+// nsplit keys to the target's greedy tokens and walks the acceptance rule.  Nobody waits for anybody.
+// `tickets` [B] must be zero before the first launch; the finishing CTA leaves them zero.
+// The grid is sized to about one resident wave (8 CTAs of 256 threads per SM: the kernel is compiled
+// for that); measured at 32 x 7 x 128256 fp32 logits, more and smaller slices only add per-CTA cost.
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256, 8) verify_greedy_fused_kernel(const T* __restrict__ logits, int V, int nsplit, int per, int gamma,
+                                                                     const int32_t* __restrict__ draft,
+                                                                     unsigned long long* __restrict__ keys, int* __restrict__ tickets,
+                                                                     int32_t* __restrict__ accept_len, int32_t* __restrict__ out_tokens) {
+    constexpr int VEC = VecOf<T>::N;
+    const int split = blockIdx.x, row = blockIdx.y;
+    const int b = row / (gamma + 1);
+    const T* z = logits + (size_t)row * V;
+    const int lo = split * per, hi = min(V, lo + per);
+    // Per thread a running (value, index): the indices a thread visits only grow, so a strict '>' keeps the lowest index of
+    // equal values; NaN never compares greater; -0 and +0 compare equal.  The packed key then orders the threads' results
+    // (key 0 = "saw nothing", below every real key).
+    float bv = -INFINITY;
+    int bi = -1;
+    auto take = [&](float v, int i) {
+        if (v > bv) { bv = v; bi = i; }
+    };
+    if (lo < hi) {
+        // scalar head up to the first 16-byte boundary of the row's slice, vector body, scalar tail
+        const uintptr_t addr = reinterpret_cast<uintptr_t>(z + lo);
+        int head = (int)(((16 - (addr & 15)) & 15) / sizeof(T));
+        if ((addr & (sizeof(T) - 1)) != 0 || head > hi - lo) head = hi - lo;
+        const int body0 = lo + head;
+        const int nvec = (hi - body0) / VEC;
+        for (int i = lo + threadIdx.x; i < body0; i += 256) take(to_float<T>(z[i]), i);
+        const T* zb = z + body0;
+        int i = threadIdx.x;
+        for (; i + 3 * 256 < nvec; i += 4 * 256) {       // four independent 16-byte loads in flight per thread
+            uint4 u[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) u[j] = ld_stream16(zb + (size_t)(i + j * 256) * VEC);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                float f[VEC];
+                unpack16<T>(u[j], f);
+#pragma unroll
+                for (int v = 0; v < VEC; ++v) take(f[v], body0 + (i + j * 256) * VEC + v);
+            }
+        }
+        for (; i < nvec; i += 256) {
+            float f[VEC];
+            unpack16<T>(ld_stream16(zb + (size_t)i * VEC), f);
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) take(f[v], body0 + i * VEC + v);
+        }
+        for (int t = body0 + nvec * VEC + threadIdx.x; t < hi; t += 256) take(to_float<T>(z[t]), t);
+        // a slice that holds nothing above -inf (only -inf / NaN) answers with its first index: thread 0 always visits it
+        if (threadIdx.x == 0 && bi < 0) bi = lo;
+    }
+    unsigned long long key = bi >= 0 ? argmax_key(bv, bi) : 0ull;
+    key = warp_max_u64(key);
+    __shared__ unsigned long long s_k[8];
+    __shared__ int s_last;
+    __shared__ int32_t s_g[65];
+    if ((threadIdx.x & 31) == 0) s_k[threadIdx.x >> 5] = key;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int w = 1; w < 8; ++w) key = s_k[w] > key ? s_k[w] : key;
+        keys[(size_t)row * nsplit + split] = key;
+        __threadfence();                                  // the key is visible before the ticket is
+        const int total = (gamma + 1) * nsplit;
+        s_last = atomicAdd(&tickets[b], 1) == total - 1;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    // last CTA of sequence b: greedy token of each of its gamma + 1 rows (one warp per row, round robin)
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    for (int r = warp; r <= gamma; r += 8) {
+        const unsigned long long* kr = keys + ((size_t)b * (gamma + 1) + r) * nsplit;
+        unsigned long long k = 0ull;
+        for (int s = lane; s < nsplit; s += 32) { const unsigned long long o = __ldcg(kr + s); k = o > k ? o : k; }
+        k = warp_max_u64(k);
+        if (lane == 0) s_g[r] = argmax_key_index(k);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int a = 0;
+        while (a < gamma && draft[(size_t)b * gamma + a] == s_g[a]) ++a;
+        accept_len[b] = a;
+        s_last = a;                                       // (re-used) the accepted length, for the token rows below
+        tickets[b] = 0;                                   // ready for the next call
+    }
+    __syncthreads();
+    if ((int)threadIdx.x <= gamma)
+        out_tokens[(size_t)b * (gamma + 1) + threadIdx.x] = (int)threadIdx.x <= s_last ? s_g[threadIdx.x] : -1;
+}
+
+int verify_fused_splits(int rows, int V, int sm_count) {
+    // one resident wave of 8 CTAs per SM, slices of at least 4096 logits, at most kVerifyMaxSplit per row
+    int s = (sm_count * 8) / (rows > 0 ? rows : 1);
+    const int cap = (V + 4095) / 4096;
+    s = s < cap ? s : cap;
+    s = s < kVerifyMaxSplit ? s : kVerifyMaxSplit;
+    return s < 1 ? 1 : s;
+}
+
+int launch_verify_greedy_fused(int logits_dtype, const void* logits, int B, int gamma, int V, const int32_t* draft,
+                               unsigned long long* keys, int* tickets, int sm_count, int32_t* accept_len, int32_t* out_tokens,
+                               cudaStream_t stream) {
+    if (B <= 0) return 0;
+    const int rows = B * (gamma + 1);
+    const int nsplit = verify_fused_splits(rows, V, sm_count);
+    const int vec = logits_dtype == 0 ? 4 : 8;
+    int per = (V + nsplit - 1) / nsplit;
+    per = (per + vec - 1) / vec * vec;
+    dim3 grid(nsplit, rows);
+    if (logits_dtype == 0)
+        verify_greedy_fused_kernel<float><<<grid, 256, 0, stream>>>((const float*)logits, V, nsplit, per, gamma, draft, keys, tickets, accept_len, out_tokens);
+    else
+        verify_greedy_fused_kernel<bf16><<<grid, 256, 0, stream>>>((const bf16*)logits, V, nsplit, per, gamma, draft, keys, tickets, accept_len, out_tokens);
+    return 1;
 }
 
 __global__ void accept_kernel(const int32_t* __restrict__ draft, const int32_t* __restrict__ target_ids, int B, int gamma,

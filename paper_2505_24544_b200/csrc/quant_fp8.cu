@@ -12,7 +12,7 @@ namespace beagle {
 namespace {
 
 template <typename T>
-__global__ void __launch_bounds__(256) quantize_rows_e4m3_kernel(const T* __restrict__ x, int cols, uint8_t* __restrict__ q,
+__global__ void __launch_bounds__(256) quantize_rows_e4m3_kernel(const T* x, int cols, uint8_t* __restrict__ q,
                                                                 float* __restrict__ scale) {
     constexpr int VN = VecOf<T>::N;
     const size_t row = blockIdx.x;
@@ -23,7 +23,7 @@ __global__ void __launch_bounds__(256) quantize_rows_e4m3_kernel(const T* __rest
     float m = 0.f;
     for (int i = threadIdx.x * VN; i < cols; i += 256 * VN) {          // cols is a multiple of 8
         float f[VN];
-        unpack16<T>(ld_cached16(xr + i), f);
+        unpack16<T>(ld_act16(xr + i), f);
 #pragma unroll
         for (int k = 0; k < VN; ++k) m = fmaxf(m, fabsf(f[k]));
     }
@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(256) quantize_rows_e4m3_kernel(const T* __rest
     if (threadIdx.x == 0) scale[row] = sc;
     for (int i = threadIdx.x * VN; i < cols; i += 256 * VN) {
         float f[VN];
-        unpack16<T>(ld_cached16(xr + i), f);
+        unpack16<T>(ld_act16(xr + i), f);
         uint8_t o[VN];
 #pragma unroll
         for (int k = 0; k < VN; ++k) o[k] = (uint8_t)__nv_cvt_float_to_fp8(__fdiv_rn(f[k], sc), __NV_SATFINITE, __NV_E4M3);

@@ -59,7 +59,7 @@ __global__ void __launch_bounds__(32) rope_serve_kernel(T* __restrict__ q, int n
     const int b = blockIdx.x, y = blockIdx.y, half = dh >> 1;
     if (y < Hq) {
         if (b < nq) rotate_head<T>(q + ((size_t)b * Hq + y) * dh, table + (size_t)qpos.idx[b] * half, half, 1.f, threadIdx.x, 32);
-    } else if (b < nk && app.idx[b] >= 0) {
+    } else if (b < nk && app.idx[b] >= 0 && BEAGLE_IN_BOUNDS(app.idx[b] < cap && BEAGLE_SLOT_OK(slot.idx[b]))) {
         T* row = kcache + (((size_t)slot.idx[b] * Hkv + (y - Hq)) * cap + app.idx[b]) * dh;
         rotate_head<T>(row, table + (size_t)kpos.idx[b] * half, half, 1.f, threadIdx.x, 32);
     }
@@ -81,6 +81,7 @@ __global__ void __launch_bounds__(256) rope_cache_rows_kernel(T* __restrict__ kc
     const int r = (int)(w / Hkv), h = (int)(w % Hkv);
     const int s = seq_of(rows, r);
     const int pos = rows.pos_start[s] + (r - rows.row_start[s]);
+    if (!BEAGLE_IN_BOUNDS(pos >= 0 && pos < cap && BEAGLE_SLOT_OK(rows.slot[s]))) return;
     rotate_head<T>(kcache + (((size_t)rows.slot[s] * Hkv + h) * cap + pos) * dh, table + (size_t)pos * (dh >> 1), dh >> 1, 1.f,
                    threadIdx.x & 31, 32);
 }

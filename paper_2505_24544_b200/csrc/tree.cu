@@ -213,6 +213,8 @@ __global__ void __launch_bounds__(32) attn_tail_kernel(const bf16* __restrict__ 
     for (int v = 0; v < DPL; ++v) qf[v] = __bfloat162float(q[((size_t)row * Hq + h) * DH + lane * DPL + v]) * scale;
     float sc[kTreeMaxDepth + 1];
     float m = -INFINITY;
+    for (int a = 0; a < nanc; ++a)
+        if (!BEAGLE_IN_BOUNDS(anc[row * (kTreeMaxDepth + 1) + a] >= 0 && n_true + anc[row * (kTreeMaxDepth + 1) + a] < cap && BEAGLE_SLOT_OK(slot))) nanc = 0;
     for (int a = 0; a < nanc; ++a) {
         const size_t at = (((size_t)slot * Hkv + kvh) * cap + n_true + anc[row * (kTreeMaxDepth + 1) + a]) * DH + lane * DPL;
         float dot = 0.f;

@@ -918,3 +918,34 @@ def test_fp8_lm_head_is_the_quantised_product_and_close_to_the_exact_one():
     assert np.max(np.abs(z8 - z)) < 0.08 * np.max(np.abs(z))        # 3 fraction bits on both operands, averaged over 64 terms
     assert np.max(np.abs(z8 - z)) > 1e-4                            # and it is not the unquantised product
     np.testing.assert_array_equal(O.quantize_rows_e4m3(np.zeros((1, 8)))[0], np.zeros((1, 8)))
+
+
+def test_quantize_rows_e4m3_hand_row_and_torch_cast():
+    """The row-wise scale convention pinned by something other than its own formula: a row worked by hand whose scale is a power of
+    two (every quotient exact), the reconstruction bound that 3 fraction bits imply, and torch's own FP8 cast of x / scale."""
+    # max |x| = 224 = 448 / 2 -> scale 0.5; the quotients 2x are 448, -3, 17 (-> 16: tie to even), 19 (-> 20: tie to even), 0.25, 0
+    x = np.array([[224.0, -1.5, 8.5, 9.5, 0.125, 0.0]])
+    q, sc = O.quantize_rows_e4m3(x)
+    assert sc.tolist() == [0.5]
+    assert q.tolist() == [[448.0, -3.0, 16.0, 20.0, 0.25, 0.0]]
+    # a second row with another sign and a scale that is again exact: max 56 -> scale 1/8, quotients 8x
+    q, sc = O.quantize_rows_e4m3(np.array([[-56.0, 1.0, 0.3125, 2.0625]]))
+    assert sc.tolist() == [0.125] and q.tolist() == [[-448.0, 8.0, 2.5, 16.0]]          # 16.5 ties to the even code 16
+    # what the format guarantees: |x - scale q| <= scale * (spacing at |x / scale|) / 2, spacing 2^(e-3), subnormal step 2^-9
+    rng = np.random.default_rng(77)
+    xs = np.concatenate([rng.normal(0, 3, (6, 512)), rng.normal(0, 1e-3, (2, 512)), rng.uniform(-50, 50, (2, 512))]).astype(np.float32).astype(np.float64)
+    q, sc = O.quantize_rows_e4m3(xs)
+    ratio = np.abs(xs) / sc[:, None]
+    spacing = np.exp2(np.maximum(np.floor(np.log2(np.maximum(ratio, 2.0 ** -6))), -6.0) - 3.0)
+    assert np.all(np.abs(xs - sc[:, None] * q) <= sc[:, None] * spacing * 0.5 * (1 + 1e-6) + 1e-12)
+    assert np.all(np.max(np.abs(q), axis=1) == 448.0)
+    assert np.all(np.sign(q) * np.sign(xs) >= 0)
+    # the library routine: torch's cast of the float32 quotient
+    torch = pytest.importorskip("torch")
+    if not hasattr(torch, "float8_e4m3fn"):
+        pytest.skip("this torch has no float8_e4m3fn")
+    x32 = torch.from_numpy(xs.astype(np.float32))
+    scale_t = x32.abs().amax(dim=1, keepdim=True) / 448.0
+    q_t = (x32 / scale_t).to(torch.float8_e4m3fn).to(torch.float64).numpy()
+    np.testing.assert_array_equal(q, q_t)
+    np.testing.assert_array_equal(sc, scale_t[:, 0].to(torch.float64).numpy())

@@ -364,6 +364,35 @@ def test_verify_greedy_logits_both_dtypes_and_ties():
     assert out_ref[4, 0] == 0 or acc_ref[4] >= 0
 
 
+@pytest.mark.parametrize("vocab", [50001, 8192, 37])
+def test_verify_greedy_fused_slices_and_repeated_calls(vocab):
+    """The one-launch verification from logits: rows cut into several slices (maxima planted at slice edges, in the unaligned
+    head and tail of a slice, ties across slices), several batch / depth shapes on one context, and the same call twice in a
+    row (the finishing CTA must leave the tickets ready for the next call).  Bit-exact against the oracle."""
+    w = SMALL_GQA.scaled(vocab=vocab, batch=1, gamma=1)
+    head_gpu, _, _ = build(w, max_slots=1, max_ctx=16)
+    rng = WL.data_rng(w, vocab)
+    for batch, gamma in ((1, 0), (1, 8), (3, 5), (32, 6), (64, 1)):
+        logits = rng.standard_normal((batch, gamma + 1, vocab)).astype(np.float32)
+        rows = logits.reshape(-1, vocab)
+        edges = [0, vocab - 1] + [min(vocab - 1, max(0, e + d)) for e in range(4096, vocab, 4096) for d in (-9, -1, 0, 1, 8)]
+        for r in range(rows.shape[0]):
+            rows[r, edges[r % len(edges)]] = 30.0
+            if r % 3 == 1:                                   # the same maximum again, further right: the lower index must win
+                rows[r, min(vocab - 1, edges[r % len(edges)] + 4097)] = 30.0
+        draft = rng.integers(0, vocab, (batch, gamma)).astype(np.int32)
+        ids = O.argmax_lowest(logits)
+        for b in range(batch):
+            draft[b, :b % (gamma + 1)] = ids[b, :b % (gamma + 1)]
+        for dt in ("fp32", "bf16"):
+            lg = WL.round_to_storage(logits.reshape(-1), dt).reshape(logits.shape)
+            acc_ref, out_ref = O.verify_greedy(draft, target_logits=lg)
+            for _ in range(2):
+                acc, out = head_gpu.verify_greedy(to_dev(draft, w.dtype), target_logits=to_dev(lg, dt))
+                np.testing.assert_array_equal(acc.cpu().numpy(), acc_ref)
+                np.testing.assert_array_equal(out.cpu().numpy(), out_ref)
+
+
 def check_verify_sample(head_gpu, w, rng, batch, gamma, dt, temperature, logit_scale=2.0):
     """beagle_verify_sample against the oracle.  Integer outputs are bit-exact wherever the oracle's
     decision margins (|u - ratio| of the acceptance tests, distance of u_resample to a CDF
@@ -710,4 +739,25 @@ def test_fp8_lm_head_batched_draft_steps(batch):
         # and the quantised head is a usable stand-in for the bf16 one (3 fraction bits, averaged over 512 terms)
         z_bf16 = O.lm_head(head_cpu, h)
         assert np.max(np.abs(z_ref - z_bf16)) < 0.1 * np.max(np.abs(z_bf16))
+    beagle_check_device(head_gpu.ctx)
+
+
+def test_bounded_wait_runs_out_and_is_reported_once():
+    """The device error path without any fault or hang: a one-CTA kernel polls, with a short limit, a barrier that nothing
+    completes and no copy targets; it gives up, raises the context's error word and returns.  beagle_check_device then
+    reports BEAGLE_ERR_DEVICE exactly once, and the context keeps working (a draft step still matches the oracle)."""
+    from paper_2505_24544_b200.binding import BeagleError, beagle_check_device, beagle_selftest_wait_timeout
+    w = SMALL_GQA.scaled(batch=2, gamma=2)
+    head_gpu, head_cpu, _ = build(w, max_ctx=64)
+    rng = WL.data_rng(w, 321)
+    seqs = prefill_both(head_gpu, head_cpu, w, rng, [0, 1], [20, 33])
+    beagle_check_device(head_gpu.ctx)                       # nothing raised so far
+    beagle_selftest_wait_timeout(head_gpu.ctx)
+    with pytest.raises(BeagleError) as e:
+        beagle_check_device(head_gpu.ctx)
+    assert e.value.status == 7 and "bounded wait" in str(e.value)
+    beagle_check_device(head_gpu.ctx)                       # reported once, then clear
+    first = WL.make_tokens(w, rng, (2,))
+    _, _, err = run_chain_parity(head_gpu, head_cpu, w, [0, 1], seqs, first, w.gamma)
+    assert err <= 2e-2 + 1e-2 * 20
     beagle_check_device(head_gpu.ctx)
