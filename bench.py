@@ -788,6 +788,7 @@ def main():
     ap.add_argument("--only-block", action="store_true", help="diagnostic: time only the block-attention forward (C5 shape)")
     ap.add_argument("--block-batch", type=int, default=0, help="sequences of the block forward (default: the workload's 8)")
     ap.add_argument("--only-legs", action="store_true", help="diagnostic: only the prefill and verify-from-logits legs of the headline workload")
+    ap.add_argument("--legs-batch", type=int, default=0, help="with --only-legs: cut the workload down to this many sequences (profiler captures)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -825,6 +826,8 @@ def main():
         return
 
     w = WL.WORKLOADS[args.workload]
+    if args.only_legs and args.legs_batch > 0:
+        w = w.scaled(batch=min(w.batch, args.legs_batch))
     iters = args.steps + args.warmup
     extra = iters * (w.gamma + 1) + 64
     max_draft = 64          # chain depth <= 8; the draft tree (depth 6, top-10) keeps 51 draft states
@@ -838,7 +841,7 @@ def main():
     if args.only_legs:
         out = {"prefill": {w.name: bench_prefill(scn, peaks)}, "verify_greedy_logits": {w.name: bench_verify_greedy_logits(head, w, peaks)}}
         w3 = WL.WORKLOADS["c3_llama3_8b_b1"]
-        if w.name == HEADLINE:
+        if w.name == HEADLINE and args.legs_batch == 0:
             scn3 = ServeScenario(head, w3, iters, device)
             out["prefill"][w3.name] = bench_prefill(scn3, peaks)
             out["verify_greedy_logits"][w3.name] = bench_verify_greedy_logits(head, w3, peaks)

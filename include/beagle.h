@@ -22,10 +22,17 @@
  *     cudaStream_t (as void*; NULL = the legacy default stream).
  *   - dtype 0 = fp32, 1 = bf16 is the storage type of weights, states, cache and hidden outputs;
  *     accumulation, softmax and logits are fp32.  Weights are row-major [out, in].
- *   - Calls only enqueue work on the stream and return; they never synchronise.  Argument, shape,
- *     capacity and state errors are detected on the host before anything is launched and leave
- *     the context unchanged.  No call aborts, throws or traps.
- *   - A context is not thread-safe; use one per stream.
+ *   - Calls only enqueue work on the stream and return; they never synchronise -- with one exception:
+ *     the FIRST call on a context that launches anything zeroes a few device words of the workspace
+ *     (an error word, completion counters), builds the rotary table if that option is on, and waits
+ *     for that once, so that later calls may use any stream.  That first call must be made outside
+ *     stream capture (inside one it returns BEAGLE_ERR_STATE and launches nothing); from the second
+ *     call on the entry points are capturable.  Argument, shape, capacity and state errors are
+ *     detected on the host before anything is launched and leave the context unchanged.  No call
+ *     aborts, throws or traps.
+ *   - A context belongs to the device that was current when it was created, and every call on it
+ *     must be made with that device current.  Several contexts, on one or on several devices, may
+ *     live in one process.  A context is not thread-safe; use one per stream.
  */
 #ifndef BEAGLE_H
 #define BEAGLE_H
@@ -112,7 +119,7 @@ beagle_status beagle_create(const beagle_config* cfg, const beagle_weights* weig
 beagle_status beagle_destroy(beagle_ctx* ctx);
 
 /* Key/value projection and cache append over TRUE states (Eq. 2 first line; Section 4.1, cache
- * paragraph: "reset the cache to true states at the end of the iteration").  For each b < batch:
+ * paragraph: after every iteration the cache is cut back to the true states).  For each b < batch:
  * the draft tail of slot seq_slot[b] is dropped, then new_len[b] rows of `hidden_dev` are projected
  * with W_k, W_v and appended.  hidden_dev is packed row-major [sum(new_len), d] in the storage type,
  * sequences in call order.  seq_slot and new_len are HOST arrays; slots must be distinct.
@@ -251,7 +258,7 @@ beagle_status beagle_verify_sample(beagle_ctx* ctx, int32_t batch, int32_t gamma
                                    float temperature, const float* u_accept_dev, const float* u_resample_dev,
                                    int32_t* accept_len_dev, int32_t* out_tokens_dev, void* stream);
 
-/* Dynamic draft tree for one sequence (the "dynamic draft attention tree" of the experimental setup, i.e. the
+/* Dynamic draft tree for one sequence (the draft tree of the experimental setup, Section 5.1, i.e. the
  * method of EAGLE-2 with depth = 1 + `depth`, `topk` children per node and `n_candidates` nodes kept; the paper's
  * runs use 6, 10 and 60).  The root token *root_token_dev (the target's last token) is forwarded over the slot's true
  * states; its topk most likely next tokens become the first frontier, each scored by its log-probability.  `depth`

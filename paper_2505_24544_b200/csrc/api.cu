@@ -137,6 +137,9 @@ beagle_status check_config(const beagle_config* c) {
     const int vec = c->dtype == BEAGLE_BF16 ? 8 : 4;
     const int lpk = c->head_dim / vec;
     if (c->head_dim % vec || (lpk != 4 && lpk != 8 && lpk != 16 && lpk != 32)) return BEAGLE_ERR_SHAPE;
+    // the widest rows (32 pieces of 16 bytes) with eight grouped query heads would need more static shared memory than
+    // a decode-attention CTA has (bf16, head_dim 256, Hq / Hkv = 8): no kernel serves that shape
+    if (lpk == 32 && g * c->head_dim > 1024) return BEAGLE_ERR_SHAPE;
     return BEAGLE_OK;
 }
 

@@ -37,7 +37,7 @@ __global__ void __launch_bounds__(256) embed_norm_kernel(const int32_t* tokens, 
         row = src + (size_t)r * d;
     } else {
         int tok = tokens != nullptr ? tokens[r] : last_token[meta.slot[r]];
-        (void)BEAGLE_IN_BOUNDS(tok >= 0 && tok < vocab && BEAGLE_SLOT_OK(meta.slot[r]));
+        (void)BEAGLE_IN_BOUNDS(tok >= 0 && tok < vocab && (tokens != nullptr || BEAGLE_SLOT_OK(meta.slot[r])));
         tok = min(max(tok, 0), vocab - 1);      // ids are validated by contract; never read out of range
         row = embed + (size_t)tok * d;
     }
@@ -123,7 +123,9 @@ int launch_embed_norm(int dtype, const int32_t* tokens, const int32_t* last_toke
 // (or one row of each of W / W2 in the gated mode) and streams them once per group of NB batch
 // rows with 16-byte loads; the activations are re-read through L1.
 // ------------------------------------------------------------------------------------------------
-template <typename T, int NB, int MODE>
+// HALVES (K/V append of a narrow projection, e.g. 8 K/V heads): the warp owns ONE weight row and its two streams are the
+// row's halves, which doubles the CTAs of a grid that would otherwise leave most SMs without work.
+template <typename T, int NB, int MODE, bool HALVES = false>
 __global__ void __launch_bounds__(256) stream_proj_kernel(const GemvArgs a) {
     constexpr int VEC = VecOf<T>::N;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -131,10 +133,17 @@ __global__ void __launch_bounds__(256) stream_proj_kernel(const GemvArgs a) {
     const T* W = reinterpret_cast<const T*>(a.W);
     const T* W2 = reinterpret_cast<const T*>(a.W2);
     const T* Wsel = (MODE == GEMV_KV && blockIdx.y == 1) ? W2 : W;
+    const int klen = HALVES ? a.K / 2 : a.K;     // elements each of the warp's two streams covers
     int n0, n1;
     bool v0, v1;
     const T *w0, *w1;
-    if (MODE == GEMV_SILU_MUL) {
+    if (HALVES) {
+        n0 = n1 = unit;
+        v0 = unit < a.N;
+        v1 = false;                              // (the second accumulator is folded into the first below)
+        w0 = Wsel + (size_t)(v0 ? unit : 0) * a.K;
+        w1 = w0 + klen;
+    } else if (MODE == GEMV_SILU_MUL) {
         n0 = n1 = unit;
         v0 = v1 = unit < a.N;
         const int nn = v0 ? unit : 0;
@@ -157,7 +166,7 @@ __global__ void __launch_bounds__(256) stream_proj_kernel(const GemvArgs a) {
     // this one still streams slow the chain down (releasing before the wait: -3.7 % drafted tokens/s).
     if (lane < 16) {                            // the first 2 KB of each row (bf16; 4 KB in fp32, every other line)
         const int k = lane * 64;
-        if (k < a.K) { prefetch_l2(w0 + k); prefetch_l2(w1 + k); }
+        if (k < klen) { prefetch_l2(w0 + k); prefetch_l2(w1 + k); }
     }
     pdl_wait();
 
@@ -173,7 +182,7 @@ __global__ void __launch_bounds__(256) stream_proj_kernel(const GemvArgs a) {
         for (int j = 0; j < NB; ++j) { acc0[j] = 0.f; acc1[j] = 0.f; }
 
 #pragma unroll 4
-        for (int k = lane * VEC; k < a.K; k += 32 * VEC) {
+        for (int k = lane * VEC; k < klen; k += 32 * VEC) {
             float wf0[VEC], wf1[VEC];
             unpack16<T>(ld_stream16(w0 + k), wf0);
             unpack16<T>(ld_stream16(w1 + k), wf1);
@@ -181,17 +190,28 @@ __global__ void __launch_bounds__(256) stream_proj_kernel(const GemvArgs a) {
             for (int j = 0; j < NB; ++j) {
                 float xf[VEC];
                 unpack16<T>(ld_act16(xp[j] + k), xf);      // activations: written by the previous kernel of the chain
+                if (HALVES) {
+                    float xg[VEC];
+                    unpack16<T>(ld_act16(xp[j] + klen + k), xg);
 #pragma unroll
-                for (int v = 0; v < VEC; ++v) {
-                    acc0[j] = fmaf(wf0[v], xf[v], acc0[j]);
-                    acc1[j] = fmaf(wf1[v], xf[v], acc1[j]);
+                    for (int v = 0; v < VEC; ++v) {
+                        acc0[j] = fmaf(wf0[v], xf[v], acc0[j]);
+                        acc1[j] = fmaf(wf1[v], xg[v], acc1[j]);
+                    }
+                } else {
+#pragma unroll
+                    for (int v = 0; v < VEC; ++v) {
+                        acc0[j] = fmaf(wf0[v], xf[v], acc0[j]);
+                        acc1[j] = fmaf(wf1[v], xf[v], acc1[j]);
+                    }
                 }
             }
         }
 #pragma unroll
         for (int j = 0; j < NB; ++j) {
+            if (HALVES) acc0[j] += acc1[j];
             acc0[j] = warp_sum(acc0[j]);
-            acc1[j] = warp_sum(acc1[j]);
+            if (!HALVES) acc1[j] = warp_sum(acc1[j]);
         }
 
         if (MODE == GEMV_LOGITS) {
@@ -249,9 +269,19 @@ int gemv_grid_blocks(int mode, int N) {
     const int units = (mode == GEMV_SILU_MUL) ? N : (N + 1) / 2;
     return (units + 7) / 8;
 }
+// K/V append of a narrow projection: two-rows-per-warp CTAs would number fewer than two per SM (148 SMs)
+static bool kv_use_halves(const GemvArgs& a, int vec) { return 2 * gemv_grid_blocks(GEMV_KV, a.N) < 296 && a.K % (2 * vec) == 0; }
 
 template <typename T, int MODE>
 static void gemv_dispatch_nb(const GemvArgs& a, dim3 grid, cudaStream_t stream) {
+    if (MODE == GEMV_KV && kv_use_halves(a, VecOf<T>::N)) {
+        grid.x = (a.N + 7) / 8;                  // one row per warp
+        if (a.B <= 1) launch_pdl(stream_proj_kernel<T, 1, GEMV_KV, true>, grid, dim3(256), 0, stream, a);
+        else if (a.B <= 2) launch_pdl(stream_proj_kernel<T, 2, GEMV_KV, true>, grid, dim3(256), 0, stream, a);
+        else if (a.B <= 4) launch_pdl(stream_proj_kernel<T, 4, GEMV_KV, true>, grid, dim3(256), 0, stream, a);
+        else launch_pdl(stream_proj_kernel<T, 8, GEMV_KV, true>, grid, dim3(256), 0, stream, a);
+        return;
+    }
     if (a.B <= 1) launch_pdl(stream_proj_kernel<T, 1, MODE>, grid, dim3(256), 0, stream, a);
     else if (a.B <= 2) launch_pdl(stream_proj_kernel<T, 2, MODE>, grid, dim3(256), 0, stream, a);
     else if (a.B <= 4) launch_pdl(stream_proj_kernel<T, 4, MODE>, grid, dim3(256), 0, stream, a);

@@ -56,6 +56,11 @@ def test_query_sizes_and_shape_validation(lib):
     assert lib.beagle_query_sizes(C.byref(bad), C.byref(kv), C.byref(ws)) == 2
     bad = good_config(); bad.head_dim = 100
     assert lib.beagle_query_sizes(C.byref(bad), C.byref(kv), C.byref(ws)) == 2
+    bad = good_config(); bad.head_dim = 256; bad.n_q_heads = 64; bad.n_kv_heads = 8       # bf16, 256-wide heads, 8 grouped heads: no kernel
+    kv_, ws_ = C.c_size_t(), C.c_size_t()
+    assert lib.beagle_query_sizes(C.byref(bad), C.byref(kv_), C.byref(ws_)) == 2
+    ok = good_config(); ok.head_dim = 256; ok.n_q_heads = 32; ok.n_kv_heads = 8
+    assert lib.beagle_query_sizes(C.byref(ok), C.byref(kv_), C.byref(ws_)) == 0
     bad = good_config(); bad.dtype = 7
     assert lib.beagle_query_sizes(C.byref(bad), C.byref(kv), C.byref(ws)) == 1
     # rotary option: a base below 1 (or negative) is rejected; a valid one adds the (cos, sin) table to the workspace

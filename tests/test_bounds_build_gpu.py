@@ -22,7 +22,7 @@ def test_small_parity_cases_pass_under_the_bounds_checking_build():
     from paper_2505_24544_b200 import build
     lib = build.build(checked=True)
     env = dict(os.environ, BEAGLE_LIBRARY=lib)
-    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join("tests", "test_parity_gpu.py"), "-x", "-q", "-m", "gpu"],
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join("tests", "test_parity_gpu.py"), "-x", "-m", "gpu"],
                        cwd=ROOT, env=env, capture_output=True, text=True, timeout=1500)
     tail = r.stdout[-3000:] + r.stderr[-1000:]
     assert "bounds-checking build" in r.stdout, tail          # the child really loaded the checked library

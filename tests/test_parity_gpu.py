@@ -7,7 +7,7 @@ import torch
 
 import oracle as O
 from paper_2505_24544_b200 import workloads as WL
-from parity_utils import assert_close, check_tokens, oracle_head, run_chain_parity, to_dev
+from parity_utils import assert_close, cache_rows_parity, check_tokens, oracle_head, run_chain_parity, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -760,4 +760,53 @@ def test_bounded_wait_runs_out_and_is_reported_once():
     first = WL.make_tokens(w, rng, (2,))
     _, _, err = run_chain_parity(head_gpu, head_cpu, w, [0, 1], seqs, first, w.gamma)
     assert err <= 2e-2 + 1e-2 * 20
+    beagle_check_device(head_gpu.ctx)
+
+
+def test_first_call_inside_stream_capture_is_refused():
+    """A context's first launching call zeroes device words and waits for that; inside a stream capture that work would only be
+    recorded, so the call is refused with BEAGLE_ERR_STATE and nothing is launched.  After one ordinary call the same
+    sequence captures and replays."""
+    from paper_2505_24544_b200 import binding as B
+    w = SMALL_GQA.scaled(batch=2, gamma=2)
+    head_gpu, head_cpu, _ = build(w, max_ctx=64)
+    rng = WL.data_rng(w, 99)
+    hidden = to_dev(WL.make_hidden(w, rng, 30), w.dtype)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with pytest.raises(B.BeagleError) as e:
+        with torch.cuda.graph(g, stream=side):
+            head_gpu.prefill_kv([0, 1], [10, 20], hidden)
+    assert e.value.status == 4 and "capture" in str(e.value)
+    assert head_gpu.slot_lengths(0) == (0, 0) and head_gpu.launch_count == 0
+    torch.cuda.synchronize()
+    head_gpu.prefill_kv([0, 1], [10, 20], hidden)            # the ordinary first call
+    assert head_gpu.slot_lengths(1) == (20, 0)
+    B.beagle_check_device(head_gpu.ctx)
+
+
+@pytest.mark.parametrize("w", [SMALL_GQA, SMALL_MHA], ids=lambda w: w.name)
+def test_dense_prefill_every_cache_row_across_tile_sequence_and_head_boundaries(w):
+    """The tensor-core prefill (more than 512 rows: one GEMM over W_k and W_v side by side, cache rows written whole) on a
+    ragged batch whose sequence boundaries fall inside the 128-row tiles; with 64-wide heads a 128-column tile holds two
+    K/V heads.  EVERY cache row of every sequence is compared with the oracle's projection, then a second call appends
+    another 600 rows behind the first ones (positions that do not start at zero) and is checked the same way."""
+    w = w.scaled(batch=5)
+    head_gpu, head_cpu, _ = build(w, max_slots=6, max_ctx=1000)
+    rng = WL.data_rng(w, 512)
+    slots = [4, 0, 3, 1, 5]
+    base = {s: 0 for s in slots}
+    for lengths in ([100, 130, 7, 300, 200], [129, 1, 255, 90, 125]):
+        assert sum(lengths) > 512
+        hidden = WL.make_hidden(w, rng, sum(lengths))
+        head_gpu.prefill_kv(slots, lengths, to_dev(hidden, w.dtype))
+        torch.cuda.synchronize()
+        r = 0
+        for s, n in zip(slots, lengths):
+            cache_rows_parity(head_gpu, head_cpu, w, s, base[s], hidden[r:r + n], f"slot {s} rows {base[s]}..{base[s] + n}")
+            r += n
+            base[s] += n
+            assert head_gpu.slot_lengths(s) == (base[s], 0)
+    from paper_2505_24544_b200.binding import beagle_check_device
     beagle_check_device(head_gpu.ctx)
