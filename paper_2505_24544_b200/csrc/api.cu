@@ -504,8 +504,9 @@ beagle_status beagle_check_device(beagle_ctx* ctx, void* stream_) {
     if (cudaMemcpy(&word, ctx->dev_error, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
         return fail(ctx, BEAGLE_ERR_CUDA, "check_device: %s", cudaGetErrorString(cudaGetLastError()));
     if (word != 0) {
-        // reported once: the word is cleared so that the context stays usable and a later check speaks of later kernels
-        if (cudaMemset(ctx->dev_error, 0, sizeof(int)) != cudaSuccess)
+        // reported once: the word is cleared so that the context stays usable and a later check speaks of later kernels; the
+        // counters behind it are cleared too, since a kernel that gave up may have left its tickets half-way
+        if (cudaMemset(ctx->dev_error, 0, dev_words_bytes(ctx->cfg)) != cudaSuccess)
             return fail(ctx, BEAGLE_ERR_CUDA, "check_device: %s", cudaGetErrorString(cudaGetLastError()));
         return fail(ctx, BEAGLE_ERR_DEVICE, word == 2 ? "a kernel's index check failed (bounds-checking build): the access was skipped"
                                                       : "a kernel gave up on a bounded wait (pipeline barrier never completed)");
