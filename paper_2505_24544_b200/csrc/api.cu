@@ -1463,7 +1463,7 @@ beagle_status beagle_verify_sample(beagle_ctx* ctx, int32_t batch, int32_t gamma
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     StageTimer timer_(ctx, ST_VERIFY, stream);
     ctx->launches += launch_verify_sample(logits_dtype, draft_tokens_dev, draft_logits_dev, target_logits_dev, batch, gamma, ctx->cfg.vocab,
-                                          temperature, u_accept_dev, u_resample_dev, ctx->vs_scratch, accept_len_dev, out_tokens_dev, stream);
+                                          temperature, u_accept_dev, u_resample_dev, ctx->vs_scratch, accept_len_dev, out_tokens_dev, ctx->sm_count, stream);
     return cuda_ok(ctx, "verify_sample");
 }
 

@@ -27,10 +27,10 @@ struct VsScratch {
 
 // One launch covers the target rows (type T, blockIdx.y < rows_p) and the draft rows (fp32).
 template <typename T, typename U>
-__device__ __forceinline__ void lse_scan_row(const U* __restrict__ z, int V, int split, float inv_t, bool base_aligned, size_t row_elems,
-                                             float& m, float& s) {
+__device__ __forceinline__ void lse_scan_row(const U* __restrict__ z, int V, int split, int nsplit, float inv_t, bool base_aligned,
+                                             size_t row_elems, float& m, float& s) {
     constexpr int VEC = VecOf<U>::N;
-    int per = (V + kLseSplit - 1) / kLseSplit;
+    int per = (V + nsplit - 1) / nsplit;
     per = (per + VEC - 1) / VEC * VEC;
     const int lo = split * per, hi = min(V, lo + per);
     auto add = [&](float v) {
@@ -40,7 +40,30 @@ __device__ __forceinline__ void lse_scan_row(const U* __restrict__ z, int V, int
         else s += __expf(v - m);
     };
     if (base_aligned && row_elems % VEC == 0) {
-        for (int i = lo + threadIdx.x * VEC; i < hi; i += blockDim.x * VEC) {
+        int i = lo + threadIdx.x * VEC;
+        const int stride = blockDim.x * VEC;
+        for (; i + 3 * stride + VEC <= hi; i += 4 * stride) {          // four independent 16-byte loads in flight per thread
+            uint4 u[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) u[j] = ld_stream16(z + i + j * stride);
+            float f[4][VEC];
+            float vm = -INFINITY;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                unpack16<U>(u[j], f[j]);
+#pragma unroll
+                for (int v = 0; v < VEC; ++v) vm = fmaxf(vm, f[j][v]);
+            }
+            vm *= inv_t;
+            if (vm > m) { s *= __expf(m - vm); m = vm; }           // one rescale per 64 bytes; m = -inf: s stays 0
+            if (m != -INFINITY) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+#pragma unroll
+                    for (int v = 0; v < VEC; ++v) s += __expf(f[j][v] * inv_t - m);
+            }
+        }
+        for (; i < hi; i += stride) {
             if (i + VEC <= hi) {
                 float f[VEC];
                 unpack16<U>(ld_stream16(z + i), f);
@@ -65,16 +88,18 @@ __device__ __forceinline__ void lse_scan_row(const U* __restrict__ z, int V, int
 template <typename T>
 __global__ void __launch_bounds__(256) vs_lse_partial_kernel(const T* __restrict__ zp, int rows_p, const float* __restrict__ zq, int V,
                                                             float inv_t, float2* __restrict__ part_p, float2* __restrict__ part_q) {
-    const int split = blockIdx.x;
+    // gridDim.x <= kLseSplit slices per row: the grid is sized to about one resident wave (every further CTA costs more in
+    // launch, first-load latency and reduction than its shorter slice saves); the unused partial slots are filled with "no mass"
+    const int split = blockIdx.x, nsplit = gridDim.x;
     int row = blockIdx.y;
     float m = -INFINITY, s = 0.f;
     float2* part;
     if (row < rows_p) {
-        lse_scan_row<T, T>(zp + (size_t)row * V, V, split, inv_t, (reinterpret_cast<uintptr_t>(zp) & 15) == 0, (size_t)row * V, m, s);
+        lse_scan_row<T, T>(zp + (size_t)row * V, V, split, nsplit, inv_t, (reinterpret_cast<uintptr_t>(zp) & 15) == 0, (size_t)row * V, m, s);
         part = part_p;
     } else {
         row -= rows_p;
-        lse_scan_row<T, float>(zq + (size_t)row * V, V, split, inv_t, (reinterpret_cast<uintptr_t>(zq) & 15) == 0, (size_t)row * V, m, s);
+        lse_scan_row<T, float>(zq + (size_t)row * V, V, split, nsplit, inv_t, (reinterpret_cast<uintptr_t>(zq) & 15) == 0, (size_t)row * V, m, s);
         part = part_q;
     }
     // merge (m, s) pairs: warp, then CTA, always in the same order
@@ -96,6 +121,8 @@ __global__ void __launch_bounds__(256) vs_lse_partial_kernel(const T* __restrict
             M = M2;
         }
         part[(size_t)row * kLseSplit + split] = make_float2(M, S);
+        if (split == 0)
+            for (int e = nsplit; e < kLseSplit; ++e) part[(size_t)row * kLseSplit + e] = make_float2(-INFINITY, 0.f);
     }
 }
 
@@ -290,10 +317,20 @@ VsScratch carve(void* scratch, int B, int gamma) {
 
 template <typename T>
 int run_verify_sample(const int32_t* draft, const float* zq, const T* zp, int B, int gamma, int V, float temperature, const float* u_accept,
-                      const float* u_resample, void* scratch, int32_t* accept_len, int32_t* out_tokens, cudaStream_t stream) {
+                      const float* u_resample, void* scratch, int32_t* accept_len, int32_t* out_tokens, int sm_count, cudaStream_t stream) {
     const VsScratch sc = carve(scratch, B, gamma);
     const float inv_t = 1.0f / temperature;
-    vs_lse_partial_kernel<T><<<dim3(kLseSplit, B * (gamma + 1) + gamma * B), 256, 0, stream>>>(zp, B * (gamma + 1), zq, V, inv_t, sc.lse_p, sc.lse_q);
+    const int lse_rows = B * (gamma + 1) + gamma * B;
+    static int per_sm = 0;                                        // resident CTAs of this instantiation per SM (same on every B200)
+    if (per_sm == 0 && (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, vs_lse_partial_kernel<T>, 256, 0) != cudaSuccess || per_sm < 1)) {
+        cudaGetLastError();
+        per_sm = 4;
+    }
+    int nsplit = (per_sm * sm_count) / lse_rows;                  // one resident wave ...
+    const int cap = (V + 4095) / 4096;                            // ... of slices no shorter than 4096 logits
+    nsplit = nsplit < cap ? nsplit : cap;
+    nsplit = nsplit < 1 ? 1 : (nsplit > kLseSplit ? kLseSplit : nsplit);
+    vs_lse_partial_kernel<T><<<dim3(nsplit, lse_rows), 256, 0, stream>>>(zp, B * (gamma + 1), zq, V, inv_t, sc.lse_p, sc.lse_q);
     const int n = 1;
     vs_accept_kernel<T><<<(B + 3) / 4, 128, 0, stream>>>(draft, zq, zp, B, gamma, V, inv_t, u_accept, sc, accept_len, out_tokens);
     vs_residual_kernel<T><<<dim3(kChunks, B), 256, 0, stream>>>(zq, zp, B, gamma, V, inv_t, accept_len, sc);
@@ -310,13 +347,13 @@ size_t verify_sample_scratch_bytes(int max_batch, int max_gamma) {
 
 int launch_verify_sample(int logits_dtype, const int32_t* draft, const float* draft_logits, const void* target_logits, int B, int gamma, int V,
                          float temperature, const float* u_accept, const float* u_resample, void* scratch, int32_t* accept_len,
-                         int32_t* out_tokens, cudaStream_t stream) {
+                         int32_t* out_tokens, int sm_count, cudaStream_t stream) {
     if (B <= 0) return 0;
     return logits_dtype == 0
         ? run_verify_sample<float>(draft, draft_logits, static_cast<const float*>(target_logits), B, gamma, V, temperature, u_accept,
-                                   u_resample, scratch, accept_len, out_tokens, stream)
+                                   u_resample, scratch, accept_len, out_tokens, sm_count, stream)
         : run_verify_sample<bf16>(draft, draft_logits, static_cast<const bf16*>(target_logits), B, gamma, V, temperature, u_accept,
-                                  u_resample, scratch, accept_len, out_tokens, stream);
+                                  u_resample, scratch, accept_len, out_tokens, sm_count, stream);
 }
 
 }  // namespace beagle
