@@ -181,11 +181,11 @@ __global__ void __launch_bounds__(256) stream_proj_kernel(const GemvArgs a) {
 #pragma unroll
         for (int j = 0; j < NB; ++j) { acc0[j] = 0.f; acc1[j] = 0.f; }
 
-#pragma unroll 4
-        for (int k = lane * VEC; k < klen; k += 32 * VEC) {
+        // one step of both streams against the NB activation rows
+        auto consume = [&](const uint4& ua, const uint4& ub, int k) {
             float wf0[VEC], wf1[VEC];
-            unpack16<T>(ld_stream16(w0 + k), wf0);
-            unpack16<T>(ld_stream16(w1 + k), wf1);
+            unpack16<T>(ua, wf0);
+            unpack16<T>(ub, wf1);
 #pragma unroll
             for (int j = 0; j < NB; ++j) {
                 float xf[VEC];
@@ -206,6 +206,29 @@ __global__ void __launch_bounds__(256) stream_proj_kernel(const GemvArgs a) {
                     }
                 }
             }
+        };
+        if constexpr (MODE == GEMV_LOGITS && NB == 1) {
+            // The LM head at batch 1 is one long stream (0.26 - 1.05 GB): eight steps of both rows are requested before the first
+            // is consumed (16 loads of 16 bytes in flight per lane; measured 164 -> 153 us at V = 128256).  The shorter
+            // projections lose with this form (fewer resident CTAs, longer tails: down-projection 27 -> 33 us) and keep the loop below.
+            constexpr int U = 8;
+            for (int k0 = lane * VEC; k0 < klen; k0 += U * 32 * VEC) {
+                uint4 wa[U], wb[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int k = k0 + u * 32 * VEC;
+                    if (k < klen) { wa[u] = ld_stream16(w0 + k); wb[u] = ld_stream16(w1 + k); }
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int k = k0 + u * 32 * VEC;
+                    if (k >= klen) break;
+                    consume(wa[u], wb[u], k);
+                }
+            }
+        } else {
+#pragma unroll 4
+            for (int k = lane * VEC; k < klen; k += 32 * VEC) consume(ld_stream16(w0 + k), ld_stream16(w1 + k), k);
         }
 #pragma unroll
         for (int j = 0; j < NB; ++j) {
