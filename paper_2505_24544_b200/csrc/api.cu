@@ -312,7 +312,7 @@ int dense_gemm(beagle_ctx* ctx, int epi, const GemmArgs& a, cudaStream_t stream)
         const int rc = tc_gemm(ctx->tc, epi, t, stream);
         if (rc >= 0) return rc;
     }
-    if (epi == GEMM_ARGMAX_KEYS || epi == GEMM_CE || epi == GEMM_DLOGITS || epi == GEMM_KV_CACHE_PAIR) return -1;
+    if (epi == GEMM_ARGMAX_KEYS || epi == GEMM_CE || epi == GEMM_DLOGITS || epi == GEMM_KV_CACHE_PAIR || a.a_mn || a.b_mn) return -1;
     return launch_gemm_simt(ctx->cfg.dtype, epi, a, stream);
 }
 
@@ -1244,6 +1244,15 @@ beagle_status beagle_block_grad(beagle_ctx* ctx, int32_t batch, int32_t S, const
     };
     // dX = dY W: A = dY [M, n_out_pad], "weight" = W^T [n_in, n_out_pad] (transposed here, padded columns zero)
     auto dx_gemm = [&](int epi, const void* dYm, int ldy, const void* W, int n_out, int n_in, void* out, const void* resid) -> int {
+        if (ctx->tc != nullptr) {
+            // tensor cores: the weight [n_out, n_in] is read as it lies, as an MN-major operand (no transposed copy)
+            memset(&g, 0, sizeof(g));
+            g.M = M; g.A = dYm; g.lda = ldy; g.K = n_out; g.W = W; g.ldw = n_in; g.b_mn = 1; g.N = n_in; g.C = out; g.ldc = n_in;
+            g.R = resid; g.ldr = n_in;
+            StageTimer timer_(ctx, ST_BWD_DX, stream);
+            const int r = dense_gemm(ctx, epi, g, stream);
+            if (r > 0) { ctx->launches += r; return r; }
+        }
         const int np = (n_out + 7) / 8 * 8;
         transpose(W, n_out, n_in, n_in, WT, np, 0, np);
         memset(&g, 0, sizeof(g));
@@ -1255,6 +1264,16 @@ beagle_status beagle_block_grad(beagle_ctx* ctx, int32_t batch, int32_t S, const
         return r;
     };
     // dW = dY^T X: A = dY^T [n_out, K], "weight" = X^T [n_in, K], K = Mp (or 2 Mp with two row blocks side by side), fp32 out
+    // dW = dY^T X on the tensor cores without transposed copies: both operands MN-major, contraction over the M rows
+    auto dw_gemm_mn = [&](const void* dYm, int ldy, int n_out, const void* Xm, int ldx, int n_in, float* out) -> int {
+        if (ctx->tc == nullptr) return -1;
+        memset(&g, 0, sizeof(g));
+        g.M = n_out; g.A = dYm; g.lda = ldy; g.a_mn = 1; g.K = M; g.W = Xm; g.ldw = ldx; g.b_mn = 1; g.N = n_in; g.C = out; g.ldc = n_in;
+        StageTimer timer_(ctx, ST_BWD_DW, stream);
+        const int r = dense_gemm(ctx, GEMM_F32, g, stream);
+        if (r > 0) ctx->launches += r;
+        return r;
+    };
     auto dw_gemm = [&](int n_out, int n_in, int Kc, float* out) -> int {
         memset(&g, 0, sizeof(g));
         g.M = n_out; g.A = TA; g.lda = Kc; g.K = Kc; g.W = TB; g.N = n_in; g.C = out; g.ldc = n_in; g.w_transient = 1;
@@ -1309,14 +1328,14 @@ beagle_status beagle_block_grad(beagle_ctx* ctx, int32_t batch, int32_t S, const
     }
     // ---- LM head: dh = dz W_lm + dh0;  dW_lm = dz^T h
     BEAGLE_NEED(dx_gemm(GEMM_RESID, DZ, Vp, ctx->w.w_lm, V, d, DH, DH0), "dh");
-    if (grads->w_lm != nullptr) {
+    if (grads->w_lm != nullptr && dw_gemm_mn(DZ, Vp, V, H, d, d, grads->w_lm) < 0) {
         transpose(DZ, M, V, Vp, TA, Mp, 0, Mp);
         transpose(H, M, d, d, TB, Mp, 0, Mp);
         BEAGLE_NEED(dw_gemm(V, d, Mp, grads->w_lm), "dW_lm");
     }
     // ---- MLP: h = y + W_down act
     BEAGLE_NEED(dx_gemm(GEMM_STORE, DH, d, ctx->w.w_down, d, m, DACT, nullptr), "dact");
-    if (grads->w_down != nullptr) {
+    if (grads->w_down != nullptr && dw_gemm_mn(DH, d, d, ACT, m, m, grads->w_down) < 0) {
         transpose(DH, M, d, d, TA, Mp, 0, Mp);
         transpose(ACT, M, m, m, TB, Mp, 0, Mp);
         BEAGLE_NEED(dw_gemm(d, m, Mp, grads->w_down), "dW_down");
@@ -1328,12 +1347,15 @@ beagle_status beagle_block_grad(beagle_ctx* ctx, int32_t batch, int32_t S, const
     BEAGLE_NEED(dx_gemm(GEMM_STORE, G, m, ctx->w.w_gate, m, d, DYN, nullptr), "dyn (gate)");
     BEAGLE_NEED(dx_gemm(GEMM_RESID, U, m, ctx->w.w_up, m, d, DYN, DYN), "dyn (up)");
     if (grads->w_gate != nullptr || grads->w_up != nullptr) {
-        transpose(Yn, M, d, d, TB, Mp, 0, Mp);
-        if (grads->w_gate != nullptr) {
+        bool yn_t = false;          // Yn^T made (only the path with transposed copies needs it)
+        if (grads->w_gate != nullptr && dw_gemm_mn(G, m, m, Yn, d, d, grads->w_gate) < 0) {
+            transpose(Yn, M, d, d, TB, Mp, 0, Mp);
+            yn_t = true;
             transpose(G, M, m, m, TA, Mp, 0, Mp);
             BEAGLE_NEED(dw_gemm(m, d, Mp, grads->w_gate), "dW_gate");
         }
-        if (grads->w_up != nullptr) {
+        if (grads->w_up != nullptr && dw_gemm_mn(U, m, m, Yn, d, d, grads->w_up) < 0) {
+            if (!yn_t) transpose(Yn, M, d, d, TB, Mp, 0, Mp);
             transpose(U, M, m, m, TA, Mp, 0, Mp);
             BEAGLE_NEED(dw_gemm(m, d, Mp, grads->w_up), "dW_up");
         }
@@ -1346,7 +1368,7 @@ beagle_status beagle_block_grad(beagle_ctx* ctx, int32_t batch, int32_t S, const
     }
     // ---- output projection: y = W_O o + x
     BEAGLE_NEED(dx_gemm(GEMM_STORE, DY, d, ctx->w.w_o, d, qd, DO, nullptr), "do");
-    if (grads->w_o != nullptr) {
+    if (grads->w_o != nullptr && dw_gemm_mn(DY, d, d, O, qd, qd, grads->w_o) < 0) {
         transpose(DY, M, d, d, TA, Mp, 0, Mp);
         transpose(O, M, qd, qd, TB, Mp, 0, Mp);
         BEAGLE_NEED(dw_gemm(d, qd, Mp, grads->w_o), "dW_o");
@@ -1382,12 +1404,19 @@ beagle_status beagle_block_grad(beagle_ctx* ctx, int32_t batch, int32_t S, const
         if (sim_steps > 1) ctx->launches += launch_rope_rows(dt, DKP, M, c.n_kv_heads, c.head_dim, S, 0, 1, rope, stream);
     }
     // ---- projections: dW_q = dq^T xn;  dW_k = dk_true^T h_true + dk_pred^T h_hat (same for V)
-    if (grads->w_q != nullptr) {
+    if (grads->w_q != nullptr && dw_gemm_mn(DQ, qd, qd, Xn, d, d, grads->w_q) < 0) {
         transpose(DQ, M, qd, qd, TA, Mp, 0, Mp);
         transpose(Xn, M, d, d, TB, Mp, 0, Mp);
         BEAGLE_NEED(dw_gemm(qd, d, Mp, grads->w_q), "dW_q");
     }
-    if (grads->w_k != nullptr || grads->w_v != nullptr) {
+    // (under simulation the contraction runs over two row blocks, true and predicted: that case keeps the transposed copies)
+    bool kv_done = false;
+    if (sim_steps == 1 && ctx->tc != nullptr) {
+        kv_done = true;
+        if (grads->w_k != nullptr) kv_done = kv_done && dw_gemm_mn(DKT, kd, kd, hidden_dev, d, d, grads->w_k) > 0;
+        if (kv_done && grads->w_v != nullptr) kv_done = dw_gemm_mn(DVT, kd, kd, hidden_dev, d, d, grads->w_v) > 0;
+    }
+    if (!kv_done && (grads->w_k != nullptr || grads->w_v != nullptr)) {
         const int Kc = sim_steps > 1 ? 2 * Mp : Mp;
         transpose(hidden_dev, M, d, d, TB, Kc, 0, Mp);
         if (sim_steps > 1) transpose(H, M, d, d, TB, Kc, Mp, Mp);

@@ -59,7 +59,7 @@ struct TcSmem {
     static constexpr int kBytes = kStages * kStageBytes + kStagingBytes + 1024 /*align*/ + 256 /*barriers*/;
 };
 
-template <int BN, bool DUAL, int EPI>
+template <int BN, bool DUAL, int EPI, bool AMN = false, bool BMN = false>
 __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA,
                                                             const __grid_constant__ CUtensorMap tmB,
                                                             const __grid_constant__ CUtensorMap tmB2, const TcArgs args) {
@@ -124,8 +124,18 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
                     const uint32_t sa = smem_base + s * SM::kStageBytes, sb = sa + kABytes;
                     mbar_expect_tx(bar_full + 8 * s, kABytes + kBBytes * (DUAL ? 2 : 1));
                     const int kc = kb * BK;
-                    tma_load_2d(sa, &tmA, bar_full + 8 * s, kc, ta * BM);
-                    tma_load_2d(sb, &tmB, bar_full + 8 * s, kc, tb * BN);
+                    if (AMN) {      // the operand is stored [k][m]: one box of 64 k-rows x 64 m per 64 rows of the tile
+#pragma unroll
+                        for (int i = 0; i < BM / 64; ++i) tma_load_2d(sa + i * (BK * 128), &tmA, bar_full + 8 * s, ta * BM + 64 * i, kc);
+                    } else {
+                        tma_load_2d(sa, &tmA, bar_full + 8 * s, kc, ta * BM);
+                    }
+                    if (BMN) {
+#pragma unroll
+                        for (int i = 0; i < BN / 64; ++i) tma_load_2d(sb + i * (BK * 128), &tmB, bar_full + 8 * s, tb * BN + 64 * i, kc);
+                    } else {
+                        tma_load_2d(sb, &tmB, bar_full + 8 * s, kc, tb * BN);
+                    }
                     if (DUAL) tma_load_2d(sb + kBBytes, &tmB2, bar_full + 8 * s, kc, tb * BN);
                     ++issued;
                 }
@@ -145,7 +155,7 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
         if (lane == 0) {
             // gate and up tiles sit back to back in the stage (256 rows of 128 bytes), so one MMA of N = 2*BN
             // fills both accumulators and reads the A tile once
-            constexpr uint32_t idesc = make_idesc(BM, DUAL ? 2 * BN : BN);
+            constexpr uint32_t idesc = make_idesc_major(BM, DUAL ? 2 * BN : BN, AMN, BMN);
             bool ok = true;
             int consumed = 0, it = 0;
             for (int t = blockIdx.x; t < ntiles && ok; t += gridDim.x, ++it) {
@@ -162,12 +172,15 @@ __global__ void __launch_bounds__(kTcThreads) tc_gemm_kernel(const __grid_consta
                     if (!ok) break;
                     fence_after();
                     const uint32_t sa = smem_base + s * SM::kStageBytes, sb = sa + kABytes;
-                    const uint64_t da = umma_desc(sa), db = umma_desc(sb);
+                    const uint64_t da = AMN ? umma_desc_mn(sa, BK * 128) : umma_desc(sa);
+                    const uint64_t db = BMN ? umma_desc_mn(sb, BK * 128) : umma_desc(sb);
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; ++k) {
                         const uint32_t acc = (kb > 0 || k > 0) ? 1u : 0u;
-                        const uint64_t koff = static_cast<uint64_t>((k * UMMA_K * 2) >> 4);   // advance inside the swizzle atom
-                        umma_bf16(tacc, da + koff, db + koff, idesc, acc);
+                        // K-major: advance inside the swizzle atom (32 bytes per step); MN-major: 16 rows of 128 bytes per step
+                        const uint64_t koff_a = static_cast<uint64_t>((AMN ? k * UMMA_K * 128 : k * UMMA_K * 2) >> 4);
+                        const uint64_t koff_b = static_cast<uint64_t>((BMN ? k * UMMA_K * 128 : k * UMMA_K * 2) >> 4);
+                        umma_bf16(tacc, da + koff_a, db + koff_b, idesc, acc);
                     }
                     umma_commit(bar_empty + 8 * s);   // frees the stage once these MMAs have read it
                     ++consumed;
@@ -465,6 +478,18 @@ bool tc_encode_map(TcPlan* p, CUtensorMap* out, const void* base, long long rows
     return r == CUDA_SUCCESS;
 }
 
+// An MN-major operand: stored [krows, feat] row-major (row stride ld elements); box = 64 features x 64 k-rows.
+bool tc_encode_map_mn(TcPlan* p, CUtensorMap* out, const void* base, long long feat, long long krows, long long ld) {
+    cuuint64_t dims[2] = {(cuuint64_t)feat, (cuuint64_t)krows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {64u, (cuuint32_t)BK};
+    cuuint32_t estr[2] = {1, 1};
+    const CUresult r = p->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 bool tc_encode_map_u8(TcPlan* p, CUtensorMap* out, const void* base, long long rows, long long K, long long ld, int box_rows) {
     cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)ld};
@@ -496,13 +521,13 @@ const CUtensorMap* tc_weight_map(TcPlan* p, const void* W, int rows, int K, int 
 
 namespace {
 
-template <int BN, bool DUAL, int EPI>
+template <int BN, bool DUAL, int EPI, bool AMN = false, bool BMN = false>
 int launch_tc(const CUtensorMap& a, const CUtensorMap& b, const CUtensorMap& b2, const TcArgs& args, dim3 grid, cudaStream_t stream) {
     using SM = TcSmem<BN, DUAL, EPI>;
     static PerDeviceOnce smem_attr;
-    if (!smem_attr.ensure([] { return cudaFuncSetAttribute(tc_gemm_kernel<BN, DUAL, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kBytes) == cudaSuccess; }))
+    if (!smem_attr.ensure([] { return cudaFuncSetAttribute(tc_gemm_kernel<BN, DUAL, EPI, AMN, BMN>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kBytes) == cudaSuccess; }))
         return -1;
-    tc_gemm_kernel<BN, DUAL, EPI><<<grid, kTcThreads, SM::kBytes, stream>>>(a, b, b2, args);
+    tc_gemm_kernel<BN, DUAL, EPI, AMN, BMN><<<grid, kTcThreads, SM::kBytes, stream>>>(a, b, b2, args);
     return 1;
 }
 
@@ -537,15 +562,20 @@ void tc_plan_destroy(TcPlan* plan) { delete plan; }
 
 int tc_gemm(TcPlan* p, int epi, const GemmArgs& g, cudaStream_t stream) {
     if (p == nullptr) return -1;
-    if (g.K % 8 || g.lda % 8) return -1;                       // TMA: 16-byte row pitch
+    if (g.lda % 8 || (!g.a_mn && !g.b_mn && g.K % 8)) return -1;   // TMA: 16-byte row pitch
     if (reinterpret_cast<uintptr_t>(g.A) & 15) return -1;
+    if ((g.a_mn || g.b_mn) && epi != GEMM_STORE && epi != GEMM_RESID && epi != GEMM_F32) return -1;
+    if (g.a_mn && !g.b_mn) return -1;                              // the forms in use: W transposed, or both
     const bool dual = (epi == GEMM_SILU_MUL || epi == GEMM_KV_CACHE_PAIR);
     const int BN = dual ? 128 : 256;
     CUtensorMap mapA;
-    if (!tc_encode_map(p, &mapA, g.A, g.M, g.K, g.lda, BM)) return -1;
+    if (g.a_mn ? !tc_encode_map_mn(p, &mapA, g.A, g.M, g.K, g.lda) : !tc_encode_map(p, &mapA, g.A, g.M, g.K, g.lda, BM)) return -1;
     CUtensorMap transient;
     const CUtensorMap* mapB;
-    if (g.w_transient) {
+    if (g.b_mn) {
+        if ((reinterpret_cast<uintptr_t>(g.W) & 15) || g.ldw % 8 || !tc_encode_map_mn(p, &transient, g.W, g.N, g.K, g.ldw)) return -1;
+        mapB = &transient;
+    } else if (g.w_transient) {
         if (dual || (reinterpret_cast<uintptr_t>(g.W) & 15) || !tc_encode_map(p, &transient, g.W, g.N, g.K, g.K, BN)) return -1;
         mapB = &transient;
     } else {
@@ -571,6 +601,12 @@ int tc_gemm(TcPlan* p, int epi, const GemmArgs& g, cudaStream_t stream) {
         return -1;
     const int ntiles = a.tiles_a * a.tiles_b;
     dim3 grid(ntiles < p->sm_count ? ntiles : p->sm_count, 1, 1);        // persistent: one CTA per SM
+    if (g.b_mn) {
+        if (g.a_mn) return epi == GEMM_F32 ? launch_tc<256, false, TC_F32, true, true>(mapA, *mapB, *mapB, a, grid, stream) : -1;
+        if (epi == GEMM_STORE) return launch_tc<256, false, TC_STORE, false, true>(mapA, *mapB, *mapB, a, grid, stream);
+        if (epi == GEMM_RESID) return launch_tc<256, false, TC_RESID, false, true>(mapA, *mapB, *mapB, a, grid, stream);
+        return -1;
+    }
     switch (epi) {
         case GEMM_STORE: return launch_tc<256, false, TC_STORE>(mapA, *mapB, *mapB, a, grid, stream);
         case GEMM_RESID: return launch_tc<256, false, TC_RESID>(mapA, *mapB, *mapB, a, grid, stream);

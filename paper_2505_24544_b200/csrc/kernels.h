@@ -156,6 +156,9 @@ struct GemmArgs {
     const float* row_coef;          // GEMM_DLOGITS: [M] loss weight of the row times the loss scale
     int* error_word;                // device word set to 1 when a bounded wait ran out
     int w_transient;                // W is a workspace buffer (its tensor map is not cached by pointer)
+    // Transposed operands (tensor-core path only, GEMM_STORE / GEMM_RESID / GEMM_F32): a_mn: A is given as [K, M] row-major
+    // (row stride lda), i.e. the product is A^T W^T; b_mn: W is given as [K, N] row-major (row stride ldw).
+    int a_mn, b_mn, ldw;
     SeqRows rows;
 };
 int launch_gemm_simt(int dtype, int epi, const GemmArgs& a, cudaStream_t stream);

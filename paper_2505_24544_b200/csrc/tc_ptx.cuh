@@ -94,6 +94,23 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
 __host__ __device__ constexpr uint32_t make_idesc(int m, int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(m >> 4) << 24);
 }
+// The same with the operands' major-ness chosen: an MN-major operand is stored with its M (or N) index contiguous, i.e. it
+// is the transpose of what the K-major form expects (bits 15 / 16 of the descriptor).
+__host__ __device__ constexpr uint32_t make_idesc_major(int m, int n, bool a_mn, bool b_mn) {
+    return make_idesc(m, n) | (a_mn ? (1u << 15) : 0u) | (b_mn ? (1u << 16) : 0u);
+}
+// Shared-memory descriptor of an MN-major bf16 operand tile with 128-byte swizzle: rows are k indices, each row holds 64
+// consecutive M (or N) indices (128 bytes); 8-row groups are 1024 bytes apart (stride offset), the next 64 M / N indices start
+// `mn_chunk_bytes` further on (leading offset).  One MMA (K = 16) reads 16 rows: advance the start address by 2048 bytes.
+__device__ __forceinline__ uint64_t umma_desc_mn(uint32_t smem_addr, uint32_t mn_chunk_bytes) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
+    d |= static_cast<uint64_t>(mn_chunk_bytes >> 4) << 16;     // leading-dimension byte offset: between 64-index chunks
+    d |= static_cast<uint64_t>(1024u >> 4) << 32;              // stride between 8-row (k) groups
+    d |= static_cast<uint64_t>(1) << 46;
+    d |= static_cast<uint64_t>(2) << 61;                       // 128-byte swizzle
+    return d;
+}
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
