@@ -208,8 +208,7 @@ BlockLayout block_layout(const beagle_config& c, int batch, int S) {
     L.x = take(M * d * elt); L.xn = take(M * d * elt); L.q = take(M * qd * elt);
     L.kt = take(M * kd * elt); L.vt = take(M * kd * elt); L.kp = take(M * kd * elt); L.vp = take(M * kd * elt);
     L.Sp = (S + 7) / 8 * 8;
-    const size_t vT = c.dtype == BEAGLE_BF16 ? kd * (size_t)batch * L.Sp * elt : 0;       // V^T for the tcgen05 attention
-    L.vtT = take(vT); L.vpT = take(vT);
+    L.vtT = take(0); L.vpT = take(0);          // (transposed values: no longer made)
     L.o = take(M * qd * elt); L.y = take(M * d * elt); L.yn = take(M * d * elt);
     L.act = take(M * m * elt); L.h = take(M * d * elt);
     L.lm_chunk_rows = (int)(M < (size_t)kLmChunkRows ? M : (size_t)kLmChunkRows);
@@ -1038,17 +1037,9 @@ static beagle_status block_forward_impl(beagle_ctx* ctx, int32_t batch, int32_t 
             if (ctx->tc != nullptr) {       // bf16, head_dim 64 / 128: tensor-core tiles
                     float* lse2 = (loss != nullptr && step == sim_steps) ? loss->lse2 : nullptr;
                 if (c.head_dim == 64 || c.head_dim == 128) {
-                    // tcgen05 path: it consumes the values transposed (keys contiguous), one padded column block per sequence
-                    void *VtT = ws + L.vtT, *VpT = ws + L.vpT;
-                    const int ldT = batch * L.Sp;
-                    int nt = 0;
-                    if (step == 1)
-                        nt += launch_transpose_pad_batched(dt, Vt, S, ctx->kd, ctx->kd, (size_t)S * ctx->kd, VtT, ldT, 0, L.Sp, L.Sp, batch, stream);
-                    if (step > 1)
-                        nt += launch_transpose_pad_batched(dt, Vp, S, ctx->kd, ctx->kd, (size_t)S * ctx->kd, VpT, ldT, 0, L.Sp, L.Sp, batch, stream);
-                    rc = tc_attn_block_umma(ctx->tc, Q, Kt, VtT, Kp, step > 1 ? VpT : VtT, batch, S, L.Sp, c.n_q_heads, c.n_kv_heads, c.head_dim,
+                    // tcgen05 path: the values are read as they lie (MN-major operand of P V)
+                    rc = tc_attn_block_umma(ctx->tc, Q, Kt, Vt, Kp, step > 1 ? Vp : Vt, batch, S, c.n_q_heads, c.n_kv_heads, c.head_dim,
                                             block, offset, step, O, ctx->dev_error, stream, lse2);
-                    if (rc >= 0) rc += nt; else ctx->launches += nt;
                 }
                 if (rc >= 0 && lse2 != nullptr) loss->lse2_written = true;
             }

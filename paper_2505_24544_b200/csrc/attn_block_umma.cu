@@ -12,10 +12,10 @@
 // Recomputing S (a third of the work again) removes the running-maximum rescale of O, which on this
 // architecture would mean reading and rewriting the TMEM accumulator for every tile or holding O
 // in 128 registers per thread; with O resident in TMEM two CTAs fit an SM and overlap each other's
-// softmax with MMAs.  V is consumed as V^T (keys contiguous), the only B-operand form used here, so
-// the caller passes a transposed copy.
+// softmax with MMAs.  V is read as it lies ([key][head_dim]: the B operand of P V in its MN-major form),
+// so no transposed copy of the values is made.
 //
-// Roles: warp 0 = TMA producer (Q once; K tiles in a two-stage ring, V^T tile single-buffered),
+// Roles: warp 0 = TMA producer (Q once; K tiles in a two-stage ring, V tile single-buffered),
 // warp 1 = MMA issuer and TMEM owner (two S buffers of 64 columns + the O accumulator), warps 2-5 =
 // softmax (warp w owns TMEM lanes 32 (w % 4) ..).  Every wait is bounded; a wait that runs out
 // raises the error word, the CTA drains and frees its TMEM.
@@ -50,7 +50,7 @@ template <int DH>
 struct UmmaAttnSmem {
     static constexpr int kQ = kUQ * DH * 2;             // DH/64 tiles of [128 x 64]
     static constexpr int kK = kUKey * DH * 2;           // DH/64 tiles of [64 keys x 64]
-    static constexpr int kV = DH * kUKey * 2;           // [DH rows x 64 keys]
+    static constexpr int kV = DH * kUKey * 2;           // DH/64 blocks of [64 keys x 64 dims]
     static constexpr int kP = kUQ * kUKey * 2;          // [128 x 64 keys]
     static constexpr int kBytes = kQ + 2 * kK + kV + kP + 1024 /*align*/ + 128 /*barriers*/;
 };
@@ -58,10 +58,9 @@ struct UmmaAttnSmem {
 template <int DH>
 __global__ void __launch_bounds__(kUThreads, 2) attn_block_umma_kernel(const __grid_constant__ CUtensorMap tmQ,
                                                                      const __grid_constant__ CUtensorMap tmKt,
-                                                                     const __grid_constant__ CUtensorMap tmVtT,
+                                                                     const __grid_constant__ CUtensorMap tmVt,
                                                                      const __grid_constant__ CUtensorMap tmKp,
-                                                                     const __grid_constant__ CUtensorMap tmVpT, const UmmaAttnArgs a,
-                                                                     const int Sp) {
+                                                                     const __grid_constant__ CUtensorMap tmVp, const UmmaAttnArgs a) {
     using SM = UmmaAttnSmem<DH>;
     constexpr int kHalves = DH / 64;
     constexpr uint32_t kTmemCols = 256;                  // S buffers at columns 0 and 64, O at 128 .. 128 + DH
@@ -83,7 +82,6 @@ __global__ void __launch_bounds__(kUThreads, 2) attn_block_umma_kernel(const __g
     const int kvh = h / (a.Hq / a.Hkv);
     const int q0 = qtile * kUQ;
     const int row_base = b * a.S;                               // rows of Q / K in the packed [B*S, .] matrices
-    const int col_base = b * Sp;                                // columns of this sequence in the transposed V
 
     // key tiles this CTA visits (identical in every role)
     const int p_last = min(q0 + kUQ, a.S);
@@ -144,7 +142,10 @@ __global__ void __launch_bounds__(kUThreads, 2) attn_block_umma_kernel(const __g
                     ok = mbar_wait(v_empty, (t2 & 1) ^ 1, s_abort);
                     if (!ok) break;
                     mbar_expect_tx(v_full, SM::kV);
-                    tma_load_2d(sV, pred ? &tmVpT : &tmVtT, v_full, col_base + kt * kUKey, kvh * DH);
+                    // values as they lie, [key][head_dim]: an MN-major B operand, one box of 64 keys x 64 dims per 64 dims
+#pragma unroll
+                    for (int hf = 0; hf < kHalves; ++hf)
+                        tma_load_2d(sV + hf * (kUKey * 128), pred ? &tmVp : &tmVt, v_full, kvh * DH + hf * 64, row_base + kt * kUKey);
                     ++v_issued;
                 }
             }
@@ -159,7 +160,7 @@ __global__ void __launch_bounds__(kUThreads, 2) attn_block_umma_kernel(const __g
     } else if (warp == 1) {
         // ---------------- MMA issuer
         if (lane == 0 && n_iter > 0) {
-            constexpr uint32_t idesc_s = make_idesc(kUQ, kUKey), idesc_o = make_idesc(kUQ, DH);
+            constexpr uint32_t idesc_s = make_idesc(kUQ, kUKey), idesc_o = make_idesc_major(kUQ, DH, false, true);
             bool ok = mbar_wait(q_full, 0, s_abort);
             auto issue_s = [&](int j) {
                 const int st = j & 1;
@@ -189,11 +190,12 @@ __global__ void __launch_bounds__(kUThreads, 2) attn_block_umma_kernel(const __g
                     if (ok) ok = mbar_wait(v_full, t2 & 1, s_abort);
                     if (!ok) break;
                     fence_after();
-                    const uint64_t dp = umma_desc(sP), dv = umma_desc(sV);
+                    const uint64_t dp = umma_desc(sP), dv = umma_desc_mn(sV, kUKey * 128);
 #pragma unroll
                     for (int k = 0; k < kUKey / UMMA_K; ++k) {
-                        const uint64_t koff = static_cast<uint64_t>((k * UMMA_K * 2) >> 4);
-                        umma_bf16(tmem_base + 2 * kUKey, dp + koff, dv + koff, idesc_o, (t2 > 0 || k > 0) ? 1u : 0u);
+                        const uint64_t koff_p = static_cast<uint64_t>((k * UMMA_K * 2) >> 4);      // P: K-major, 32 bytes per step
+                        const uint64_t koff_v = static_cast<uint64_t>((k * UMMA_K * 128) >> 4);    // V: 16 key rows of 128 bytes per step
+                        umma_bf16(tmem_base + 2 * kUKey, dp + koff_p, dv + koff_v, idesc_o, (t2 > 0 || k > 0) ? 1u : 0u);
                     }
                     umma_commit(v_empty);
                     umma_commit(p_empty);
@@ -335,27 +337,27 @@ __global__ void __launch_bounds__(kUThreads, 2) attn_block_umma_kernel(const __g
 }
 
 template <int DH>
-int launch_umma_attn(const CUtensorMap* maps, const UmmaAttnArgs& a, int Sp, dim3 grid, cudaStream_t stream) {
+int launch_umma_attn(const CUtensorMap* maps, const UmmaAttnArgs& a, dim3 grid, cudaStream_t stream) {
     using SM = UmmaAttnSmem<DH>;
     static PerDeviceOnce smem_attr;
     if (!smem_attr.ensure([] { return cudaFuncSetAttribute(attn_block_umma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, SM::kBytes) == cudaSuccess; }))
         return -1;
-    attn_block_umma_kernel<DH><<<grid, kUThreads, SM::kBytes, stream>>>(maps[0], maps[1], maps[2], maps[3], maps[4], a, Sp);
+    attn_block_umma_kernel<DH><<<grid, kUThreads, SM::kBytes, stream>>>(maps[0], maps[1], maps[2], maps[3], maps[4], a);
     return 1;
 }
 
 }  // namespace
 
-int tc_attn_block_umma(TcPlan* p, const void* Q, const void* Kt, const void* VtT, const void* Kp, const void* VpT, int B, int S, int Sp, int Hq,
+int tc_attn_block_umma(TcPlan* p, const void* Q, const void* Kt, const void* Vt, const void* Kp, const void* Vp, int B, int S, int Hq,
                        int Hkv, int dh, int block, int offset, int step, void* O, int* error_word, cudaStream_t stream, float* lse2) {
-    if (p == nullptr || (dh != 64 && dh != 128) || B <= 0 || S <= 0 || B > 65535 || Hq > 65535 || (Sp & 7) || Sp < S) return -1;
+    if (p == nullptr || (dh != 64 && dh != 128) || B <= 0 || S <= 0 || B > 65535 || Hq > 65535) return -1;
     const long long rows = (long long)B * S;
     CUtensorMap maps[5];
     if (!tc_encode_map(p, &maps[0], Q, rows, (long long)Hq * dh, (long long)Hq * dh, kUQ)) return -1;
     if (!tc_encode_map(p, &maps[1], Kt, rows, (long long)Hkv * dh, (long long)Hkv * dh, kUKey)) return -1;
-    if (!tc_encode_map(p, &maps[2], VtT, (long long)Hkv * dh, (long long)B * Sp, (long long)B * Sp, dh)) return -1;
+    if (!tc_encode_map_mn(p, &maps[2], Vt, (long long)Hkv * dh, rows, (long long)Hkv * dh)) return -1;
     if (!tc_encode_map(p, &maps[3], Kp, rows, (long long)Hkv * dh, (long long)Hkv * dh, kUKey)) return -1;
-    if (!tc_encode_map(p, &maps[4], VpT, (long long)Hkv * dh, (long long)B * Sp, (long long)B * Sp, dh)) return -1;
+    if (!tc_encode_map_mn(p, &maps[4], Vp, (long long)Hkv * dh, rows, (long long)Hkv * dh)) return -1;
     UmmaAttnArgs a;
     a.S = S; a.Hq = Hq; a.Hkv = Hkv; a.block = block; a.offset = offset; a.step = step;
     a.scale_log2 = 1.4426950408889634f / sqrtf((float)dh);
@@ -363,7 +365,7 @@ int tc_attn_block_umma(TcPlan* p, const void* Q, const void* Kt, const void* VtT
     a.lse2 = lse2;
     a.error_word = error_word;
     dim3 grid((S + kUQ - 1) / kUQ, Hq, B);
-    return dh == 128 ? launch_umma_attn<128>(maps, a, Sp, grid, stream) : launch_umma_attn<64>(maps, a, Sp, grid, stream);
+    return dh == 128 ? launch_umma_attn<128>(maps, a, grid, stream) : launch_umma_attn<64>(maps, a, grid, stream);
 }
 
 }  // namespace beagle

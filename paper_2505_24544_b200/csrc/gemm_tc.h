@@ -72,10 +72,9 @@ int tc_attn_chunk(void);
 
 // ---- block-masked cross-attention of the multi-token forward (bf16, head_dim 64 or 128) -------
 // Same contract as launch_attn_block, on tcgen05 (both products as tcgen05.mma, accumulators in tensor memory); -1 when not
-// covered (caller falls back).  VtT / VpT: the values TRANSPOSED, [Hkv*dh, B*Sp] with sequence b's position j at column
-// b*Sp + j, Sp >= S a multiple of 8 (padding columns finite).  lse2 (optional, fp32 [B*S, Hq]): base-2 log-sum-exp of every
-// row's scaled scores, for the backward below.
-int tc_attn_block_umma(TcPlan* plan, const void* Q, const void* Kt, const void* VtT, const void* Kp, const void* VpT, int B, int S, int Sp, int Hq,
+// covered (caller falls back).  Vt / Vp are read as they lie ([B*S, Hkv*dh]).  lse2 (optional, fp32 [B*S, Hq]): base-2
+// log-sum-exp of every row's scaled scores, for the backward below.
+int tc_attn_block_umma(TcPlan* plan, const void* Q, const void* Kt, const void* Vt, const void* Kp, const void* Vp, int B, int S, int Hq,
                        int Hkv, int dh, int block, int offset, int step, void* O, int* error_word, cudaStream_t stream, float* lse2 = nullptr);
 // Attention backward on tcgen05 (same contract as launch_attn_block_bwd, bf16, head_dim 64 / 128).  QT / dOT: [Hq*dh, B*Sp],
 // KtT / KpT: [Hkv*dh, B*Sp] transposed copies (sequence b's position j at column b*Sp + j, Sp a multiple of 8); delta: fp32

@@ -27,6 +27,8 @@ struct TcPlan {
 // K-major bf16 matrix [rows, K] (row stride ld elements), box = 64 columns x box_rows rows,
 // 128-byte swizzle, out-of-range elements read as zero.
 bool tc_encode_map(TcPlan* p, CUtensorMap* out, const void* base, long long rows, long long K, long long ld, int box_rows);
+// An MN-major bf16 operand: stored [krows, feat] row-major (row stride ld elements); box = 64 features x 64 k-rows.
+bool tc_encode_map_mn(TcPlan* p, CUtensorMap* out, const void* base, long long feat, long long krows, long long ld);
 // The same for a K-major matrix of bytes (FP8): box = 128 columns x box_rows rows.
 bool tc_encode_map_u8(TcPlan* p, CUtensorMap* out, const void* base, long long rows, long long K, long long ld, int box_rows);
 const CUtensorMap* tc_weight_map_u8(TcPlan* p, const void* W, int rows, int K, int box_rows);
