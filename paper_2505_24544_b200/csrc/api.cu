@@ -254,8 +254,7 @@ GradLayout grad_layout(const beagle_config& c, int batch, int S) {
     // one transposed weight at a time: [in, out] (hidden, mlp_dim and head_dim are multiples of 8; the vocabulary is padded)
     L.wt = take(max2(d * (size_t)L.Vp, max2(m, qd) * d) * elt);
     // transposed copies for the tcgen05 attention backward (bf16 only)
-    const size_t colsT = c.dtype == BEAGLE_BF16 ? (size_t)batch * L.fwd.Sp : 0;
-    L.qT = take(qd * colsT * elt); L.doT = take(qd * colsT * elt); L.ktT = take(kd * colsT * elt); L.kpT = take(kd * colsT * elt);
+    L.qT = take(0); L.doT = take(0); L.ktT = take(0); L.kpT = take(0);      // (transposed copies for the attention backward: no longer made)
     L.lse = take(M * c.n_q_heads * sizeof(float)); L.delta = take(M * c.n_q_heads * sizeof(float));
     L.stats = take(M * 4 * sizeof(float)); L.coef = take(M * sizeof(float)); L.vrow = take(M * sizeof(float));
     L.dgpart = take((size_t)rmsnorm_bwd_parts((int)M) * d * sizeof(float));
@@ -1368,16 +1367,8 @@ beagle_status beagle_block_grad(beagle_ctx* ctx, int32_t batch, int32_t S, const
     {
         StageTimer timer_(ctx, ST_BWD_ATTN, stream);
         rc = -1;
-        if (spec.lse2_written) {     // bf16, head_dim 64 / 128: tcgen05, from the forward's log-sum-exp and transposed copies of Q, dO, K
-            const int Sp = F.Sp, ldT = batch * Sp;
-            void *QT = ws + L.qT, *DOT = ws + L.doT, *KTT = ws + L.ktT, *KPT = ws + L.kpT;
-            int nt = 0;
-            nt += launch_transpose_pad_batched(dt, Q, S, qd, qd, (size_t)S * qd, QT, ldT, 0, Sp, Sp, batch, stream);
-            nt += launch_transpose_pad_batched(dt, DO, S, qd, qd, (size_t)S * qd, DOT, ldT, 0, Sp, Sp, batch, stream);
-            nt += launch_transpose_pad_batched(dt, Kt, S, kd, kd, (size_t)S * kd, KTT, ldT, 0, Sp, Sp, batch, stream);
-            if (sim_steps > 1) nt += launch_transpose_pad_batched(dt, Kp, S, kd, kd, (size_t)S * kd, KPT, ldT, 0, Sp, Sp, batch, stream);
-            ctx->launches += nt;
-            rc = tc_attn_block_bwd_umma(ctx->tc, Q, Kt, Vt, Kp, Vp_, O, DO, spec.lse2, QT, DOT, KTT, sim_steps > 1 ? KPT : KTT, batch, S, Sp,
+        if (spec.lse2_written) {     // bf16, head_dim 64 / 128: tcgen05, from the forward's log-sum-exp
+            rc = tc_attn_block_bwd_umma(ctx->tc, Q, Kt, Vt, Kp, Vp_, O, DO, spec.lse2, batch, S,
                                         c.n_q_heads, c.n_kv_heads, c.head_dim, block, offset, sim_steps, reinterpret_cast<float*>(ws + L.delta), DQ,
                                         DKT, DVT, DKP, DVP, ctx->dev_error, stream);
         }

@@ -11,8 +11,8 @@
 //     and  dV += P^T dO,  dK += dS^T Q  accumulate in tensor memory over all tiles;
 //   * query side: one CTA = 128 queries of one (sequence, query head); Q and dO stay in shared memory,
 //     key tiles (64 keys) are streamed:  S = Q K^T, dP = dO V^T, dS -> shared memory, dQ += dS K.
-// The accumulating products contract over the streamed dimension, so their B operands are consumed
-// transposed (Q^T, dO^T, K^T with the streamed index contiguous): the caller passes transposed copies.
+// The accumulating products contract over the streamed dimension: their B operands (Q, dO, K tiles as they lie,
+// [streamed index][head_dim]) are read in the MN-major form, so no transposed copy of any tensor is needed.
 // Roles per CTA: warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner, warps 2-5 = one thread
 // per tile row.  Every wait is bounded.
 #include <cstring>
@@ -32,7 +32,7 @@ constexpr int kBS = 64;           // streamed tile (queries on the key side, key
 constexpr int kBwdThreads = 320;   // warp 0 producer, warp 1 MMA issuer, warps 2-9: two threads per tile row (32 streamed columns each)
 
 struct UBwdArgs {
-    int S, Sp, Hq, Hkv, block, offset, step;
+    int S, Hq, Hkv, block, offset, step;
     float scale_log2, scale;
     const float* lse2;      // [B*S, Hq]
     const float* delta;     // [B*S, Hq]
@@ -107,7 +107,7 @@ __device__ __forceinline__ void store_acc_row(uint32_t taddr, float scale, bf16*
 template <int DH>
 struct UBwdKvSmem {
     static constexpr int kRes = kBM * DH * 2;           // K (or V) of the CTA's 128 keys
-    static constexpr int kTile = kBS * DH * 2;          // a 64-query tile of Q / dO, or of Q^T / dO^T
+    static constexpr int kTile = kBS * DH * 2;          // a 64-query tile of Q / dO
     static constexpr int kOp = kBM * kBS * 2;           // P^T / dS^T operand tile
     static constexpr int kBytes = 2 * kRes + 4 * kTile + 2 * kTile + 2 * kOp + 1024 + 128;
 };
@@ -118,9 +118,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kv_umma_kernel(const 
                                                                         const __grid_constant__ CUtensorMap tmKp128,
                                                                         const __grid_constant__ CUtensorMap tmVp128,
                                                                         const __grid_constant__ CUtensorMap tmQ64,
-                                                                        const __grid_constant__ CUtensorMap tmdO64,
-                                                                        const __grid_constant__ CUtensorMap tmQT,
-                                                                        const __grid_constant__ CUtensorMap tmdOT, const UBwdArgs a,
+                                                                        const __grid_constant__ CUtensorMap tmdO64, const UBwdArgs a,
                                                                         const int nz) {
     using SM = UBwdKvSmem<DH>;
     constexpr int kHalves = DH / 64;
@@ -148,7 +146,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kv_umma_kernel(const 
     const int b = blockIdx.z / nz, pred = blockIdx.z % nz;
     const int G = a.Hq / a.Hkv;
     const int kt0 = kt * kBM;
-    const int row_base = b * a.S, col_base = b * a.Sp;
+    const int row_base = b * a.S;
     const int n_qtiles = (a.S + kBS - 1) / kBS;
 
     // query tiles that read keys of this tile
@@ -206,8 +204,12 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kv_umma_kernel(const 
                 ok = mbar_wait(t_empty, (j & 1) ^ 1, s_abort);
                 if (!ok) { issued = j + 1; break; }
                 mbar_expect_tx(t_full, 2 * SM::kTile);
-                tma_load_2d(sQT, &tmQT, t_full, col_base + qt * kBS, h * DH);
-                tma_load_2d(sdOT, &tmdOT, t_full, col_base + qt * kBS, h * DH);
+                // the same two tiles once more for the accumulating products, which read them as MN-major operands
+#pragma unroll
+                for (int hf = 0; hf < kHalves; ++hf) {
+                    tma_load_2d(sQT + hf * (kBS * 128), &tmQ64, t_full, h * DH + hf * 64, row_base + qt * kBS);
+                    tma_load_2d(sdOT + hf * (kBS * 128), &tmdO64, t_full, h * DH + hf * 64, row_base + qt * kBS);
+                }
                 issued = j + 1;
             }
             if (*s_abort) {      // copies already requested still land: bounded wait for the latest of each buffer
@@ -219,7 +221,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kv_umma_kernel(const 
     } else if (warp == 1) {
         // ---------------- MMA issuer
         if (lane == 0 && J > 0) {
-            constexpr uint32_t idesc_s = make_idesc(kBM, kBS), idesc_o = make_idesc(kBM, DH);
+            constexpr uint32_t idesc_s = make_idesc(kBM, kBS), idesc_o = make_idesc_major(kBM, DH, false, true);
             bool ok = mbar_wait(kv_full, 0, s_abort);
             auto issue_s = [&](int j) {
                 const int st = j & 1;
@@ -251,12 +253,14 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kv_umma_kernel(const 
                 if (ok) ok = mbar_wait(t_full, j & 1, s_abort);
                 if (!ok) break;
                 fence_after();
-                const uint64_t dpt = umma_desc(sPT), ddot = umma_desc(sdOT), dst = umma_desc(sdST), dqt = umma_desc(sQT);
+                // dO and Q tiles as they lie ([query][head_dim]): MN-major B operands, 16 query rows of 128 bytes per step
+                const uint64_t dpt = umma_desc(sPT), ddot = umma_desc_mn(sdOT, kBS * 128), dst = umma_desc(sdST), dqt = umma_desc_mn(sQT, kBS * 128);
 #pragma unroll
                 for (int k = 0; k < kBS / UMMA_K; ++k) {
                     const uint64_t koff = static_cast<uint64_t>((k * UMMA_K * 2) >> 4);
-                    umma_bf16(tmem_base + 256, dpt + koff, ddot + koff, idesc_o, (j > 0 || k > 0) ? 1u : 0u);           // dV += P^T dO
-                    umma_bf16(tmem_base + 256 + DH, dst + koff, dqt + koff, idesc_o, (j > 0 || k > 0) ? 1u : 0u);      // dK += dS^T Q
+                    const uint64_t koff_mn = static_cast<uint64_t>((k * UMMA_K * 128) >> 4);
+                    umma_bf16(tmem_base + 256, dpt + koff, ddot + koff_mn, idesc_o, (j > 0 || k > 0) ? 1u : 0u);           // dV += P^T dO
+                    umma_bf16(tmem_base + 256 + DH, dst + koff, dqt + koff_mn, idesc_o, (j > 0 || k > 0) ? 1u : 0u);      // dK += dS^T Q
                 }
                 umma_commit(t_empty);
                 umma_commit(p_empty);
@@ -371,7 +375,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kv_umma_kernel(const 
 template <int DH>
 struct UBwdQSmem {
     static constexpr int kRes = kBM * DH * 2;           // Q (or dO) of the CTA's 128 queries
-    static constexpr int kTile = kBS * DH * 2;          // a 64-key tile of K / V, or of K^T
+    static constexpr int kTile = kBS * DH * 2;          // a 64-key tile of K / V
     static constexpr int kOp = kBM * kBS * 2;           // dS operand tile
     static constexpr int kBytes = 2 * kRes + 4 * kTile + kTile + kOp + 1024 + 128;
 };
@@ -382,9 +386,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_q_umma_kernel(const _
                                                                        const __grid_constant__ CUtensorMap tmK64,
                                                                        const __grid_constant__ CUtensorMap tmV64,
                                                                        const __grid_constant__ CUtensorMap tmKp64,
-                                                                       const __grid_constant__ CUtensorMap tmVp64,
-                                                                       const __grid_constant__ CUtensorMap tmKT,
-                                                                       const __grid_constant__ CUtensorMap tmKpT, const UBwdArgs a) {
+                                                                       const __grid_constant__ CUtensorMap tmVp64, const UBwdArgs a) {
     using SM = UBwdQSmem<DH>;
     constexpr int kHalves = DH / 64;
     constexpr uint32_t kTmemCols = 512;
@@ -407,7 +409,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_q_umma_kernel(const _
     const int h = blockIdx.y, b = blockIdx.z;
     const int kvh = h / (a.Hq / a.Hkv);
     const int q0 = qtile * kBM;
-    const int row_base = b * a.S, col_base = b * a.Sp;
+    const int row_base = b * a.S;
 
     const int p_last = min(q0 + kBM, a.S);
     const int n_max = nvis(p_last, a.block, a.offset);
@@ -468,7 +470,9 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_q_umma_kernel(const _
                 ok = mbar_wait(t_empty, (j & 1) ^ 1, s_abort);
                 if (!ok) break;
                 mbar_expect_tx(t_full, SM::kTile);
-                tma_load_2d(sKT, pred ? &tmKpT : &tmKT, t_full, col_base + kt * kBS, kvh * DH);
+#pragma unroll
+                for (int hf = 0; hf < kHalves; ++hf)      // the K tile once more, read by dQ += dS K as an MN-major operand
+                    tma_load_2d(sKT + hf * (kBS * 128), pred ? &tmKp64 : &tmK64, t_full, kvh * DH + hf * 64, row_base + kt * kBS);
             }
             if (*s_abort) {
                 for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(q_full, 0); ++i) {}
@@ -479,7 +483,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_q_umma_kernel(const _
     } else if (warp == 1) {
         // ---------------- MMA issuer
         if (lane == 0 && J > 0) {
-            constexpr uint32_t idesc_s = make_idesc(kBM, kBS), idesc_o = make_idesc(kBM, DH);
+            constexpr uint32_t idesc_s = make_idesc(kBM, kBS), idesc_o = make_idesc_major(kBM, DH, false, true);
             bool ok = mbar_wait(q_full, 0, s_abort);
             auto issue_s = [&](int j) {
                 const int st = j & 1;
@@ -511,11 +515,12 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_q_umma_kernel(const _
                 if (ok) ok = mbar_wait(t_full, j & 1, s_abort);
                 if (!ok) break;
                 fence_after();
-                const uint64_t dds = umma_desc(sdS), dkt = umma_desc(sKT);
+                const uint64_t dds = umma_desc(sdS), dkt = umma_desc_mn(sKT, kBS * 128);
 #pragma unroll
                 for (int k = 0; k < kBS / UMMA_K; ++k) {
                     const uint64_t koff = static_cast<uint64_t>((k * UMMA_K * 2) >> 4);
-                    umma_bf16(tmem_base + 256, dds + koff, dkt + koff, idesc_o, (j > 0 || k > 0) ? 1u : 0u);   // dQ += dS K
+                    const uint64_t koff_mn = static_cast<uint64_t>((k * UMMA_K * 128) >> 4);
+                    umma_bf16(tmem_base + 256, dds + koff, dkt + koff_mn, idesc_o, (j > 0 || k > 0) ? 1u : 0u);   // dQ += dS K
                 }
                 umma_commit(t_empty);
                 umma_commit(p_empty);
@@ -610,22 +615,21 @@ int launch_ubwd(const CUtensorMap* m, const UBwdArgs& a, int B, int nz, cudaStre
         }))
         return -1;
     const int tiles = (a.S + kBM - 1) / kBM;
-    // maps: 0 Q128, 1 dO128, 2 Q64, 3 dO64, 4 K128, 5 V128, 6 Kp128, 7 Vp128, 8 K64, 9 V64, 10 Kp64, 11 Vp64, 12 QT, 13 dOT, 14 KT, 15 KpT
-    attn_bwd_q_umma_kernel<DH><<<dim3(tiles, a.Hq, B), kBwdThreads, UBwdQSmem<DH>::kBytes, stream>>>(m[0], m[1], m[8], m[9], m[10], m[11], m[14], m[15], a);
-    attn_bwd_kv_umma_kernel<DH><<<dim3(tiles, a.Hkv, B * nz), kBwdThreads, UBwdKvSmem<DH>::kBytes, stream>>>(m[4], m[5], m[6], m[7], m[2], m[3], m[12],
-                                                                                                             m[13], a, nz);
+    // maps: 0 Q128, 1 dO128, 2 Q64, 3 dO64, 4 K128, 5 V128, 6 Kp128, 7 Vp128, 8 K64, 9 V64, 10 Kp64, 11 Vp64
+    attn_bwd_q_umma_kernel<DH><<<dim3(tiles, a.Hq, B), kBwdThreads, UBwdQSmem<DH>::kBytes, stream>>>(m[0], m[1], m[8], m[9], m[10], m[11], a);
+    attn_bwd_kv_umma_kernel<DH><<<dim3(tiles, a.Hkv, B * nz), kBwdThreads, UBwdKvSmem<DH>::kBytes, stream>>>(m[4], m[5], m[6], m[7], m[2], m[3], a, nz);
     return 2;
 }
 
 }  // namespace
 
 int tc_attn_block_bwd_umma(TcPlan* p, const void* Q, const void* Kt, const void* Vt, const void* Kp, const void* Vp, const void* O, const void* dO,
-                           const float* lse2, const void* QT, const void* dOT, const void* KtT, const void* KpT, int B, int S, int Sp, int Hq,
+                           const float* lse2, int B, int S, int Hq,
                            int Hkv, int dh, int block, int offset, int step, float* delta, void* dQ, void* dKt, void* dVt, void* dKp, void* dVp,
                            int* error_word, cudaStream_t stream) {
-    if (p == nullptr || (dh != 64 && dh != 128) || B <= 0 || S <= 0 || 2 * B > 65535 || Hq > 65535 || (Sp & 7) || Sp < S) return -1;
-    const long long rows = (long long)B * S, qd = (long long)Hq * dh, kd = (long long)Hkv * dh, colsT = (long long)B * Sp;
-    CUtensorMap m[16];
+    if (p == nullptr || (dh != 64 && dh != 128) || B <= 0 || S <= 0 || 2 * B > 65535 || Hq > 65535) return -1;
+    const long long rows = (long long)B * S, qd = (long long)Hq * dh, kd = (long long)Hkv * dh;
+    CUtensorMap m[12];
     bool okm = true;
     okm = okm && tc_encode_map(p, &m[0], Q, rows, qd, qd, kBM) && tc_encode_map(p, &m[1], dO, rows, qd, qd, kBM);
     okm = okm && tc_encode_map(p, &m[2], Q, rows, qd, qd, kBS) && tc_encode_map(p, &m[3], dO, rows, qd, qd, kBS);
@@ -634,11 +638,9 @@ int tc_attn_block_bwd_umma(TcPlan* p, const void* Q, const void* Kt, const void*
         okm = okm && tc_encode_map(p, &m[4 + i], kv[i], rows, kd, kd, kBM);
         okm = okm && tc_encode_map(p, &m[8 + i], kv[i], rows, kd, kd, kBS);
     }
-    okm = okm && tc_encode_map(p, &m[12], QT, qd, colsT, colsT, dh) && tc_encode_map(p, &m[13], dOT, qd, colsT, colsT, dh);
-    okm = okm && tc_encode_map(p, &m[14], KtT, kd, colsT, colsT, dh) && tc_encode_map(p, &m[15], KpT, kd, colsT, colsT, dh);
     if (!okm) return -1;
     UBwdArgs a;
-    a.S = S; a.Sp = Sp; a.Hq = Hq; a.Hkv = Hkv; a.block = block; a.offset = offset; a.step = step;
+    a.S = S; a.Hq = Hq; a.Hkv = Hkv; a.block = block; a.offset = offset; a.step = step;
     a.scale = 1.0f / sqrtf((float)dh);
     a.scale_log2 = 1.4426950408889634f * a.scale;
     a.lse2 = lse2; a.delta = delta;

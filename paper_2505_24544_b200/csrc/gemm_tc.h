@@ -76,12 +76,9 @@ int tc_attn_chunk(void);
 // log-sum-exp of every row's scaled scores, for the backward below.
 int tc_attn_block_umma(TcPlan* plan, const void* Q, const void* Kt, const void* Vt, const void* Kp, const void* Vp, int B, int S, int Hq,
                        int Hkv, int dh, int block, int offset, int step, void* O, int* error_word, cudaStream_t stream, float* lse2 = nullptr);
-// Attention backward on tcgen05 (same contract as launch_attn_block_bwd, bf16, head_dim 64 / 128).  QT / dOT: [Hq*dh, B*Sp],
-// KtT / KpT: [Hkv*dh, B*Sp] transposed copies (sequence b's position j at column b*Sp + j, Sp a multiple of 8); delta: fp32
-// [B*S, Hq] scratch.
+// Attention backward on tcgen05 (same contract as launch_attn_block_bwd, bf16, head_dim 64 / 128); delta: fp32 [B*S, Hq] scratch.
 int tc_attn_block_bwd_umma(TcPlan* plan, const void* Q, const void* Kt, const void* Vt, const void* Kp, const void* Vp, const void* O,
-                           const void* dO, const float* lse2, const void* QT, const void* dOT, const void* KtT, const void* KpT, int B, int S,
-                           int Sp, int Hq, int Hkv, int dh, int block, int offset, int step, float* delta, void* dQ, void* dKt, void* dVt,
-                           void* dKp, void* dVp, int* error_word, cudaStream_t stream);
+                           const void* dO, const float* lse2, int B, int S, int Hq, int Hkv, int dh, int block, int offset, int step,
+                           float* delta, void* dQ, void* dKt, void* dVt, void* dKp, void* dVp, int* error_word, cudaStream_t stream);
 
 }  // namespace beagle
