@@ -891,6 +891,9 @@ def main():
                    "hidden": w.hidden, "heads": [w.n_q_heads, w.n_kv_heads, w.head_dim], "mlp": w.mlp_dim, "vocab": w.vocab,
                    "step": STEP_TEXT,
                    "l2": "inputs larger than L2 (weights %.2f GB + K/V per draft step)" % (step_bytes(w, mean_ctx) / 1e9),
+                   "weights": "row-major as the caller gave them + tile-major copies of the eight projection matrices, made once at load "
+                              "(beagle_pack_weights, %.2f GB), which the draft steps of this batch size stream"
+                              % ((head.ctx.packed_buf.numel() if head.ctx.packed_buf is not None else 0) / 1e9),
                    "mean_tau": scn.mean_tau, "parallelism": "replicas" if world > 1 else "single"},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps},
         "gpu_launches": launches,

@@ -157,6 +157,24 @@ beagle_status beagle_slot_lengths(const beagle_ctx* ctx, int32_t slot, int32_t* 
 beagle_status beagle_quantize_rows_e4m3(const void* src_dev, int32_t dtype, int64_t rows, int32_t cols, void* q_out_dev,
                                         float* scale_out_dev, void* stream);
 
+/* Tile-major copies of the projection weights for draft steps of 9..64 rows (a re-layout of the same numbers; not part
+ * of the paper; bf16 configurations).  Those steps stream every weight matrix once per call in tiles of 128 output rows
+ * x 128 bytes of the reduction; in the row-major layout a tile is 128 pieces 2*in bytes apart, in the packed layout it
+ * is one contiguous run of 16 KB and the tiles a thread block reads follow one another, which the memory system serves
+ * faster.  Results are bit-identical with and without the copies (same tiles, same order of accumulation).
+ *
+ * beagle_packed_weights_bytes: size of the buffer for w_q, w_k, w_v, w_o, w_gate, w_up, w_down, w_lm (and the FP8 LM
+ *   head bytes when with_fp8_lm_head != 0), each padded to whole tiles; 0 for an fp32 configuration.
+ * beagle_pack_weights: writes the copies of the context's CURRENT weights into packed_dev (device, 256-byte aligned,
+ *   at least that many bytes, owned by the caller, must outlive the context or the next call of this function) on
+ *   `stream`, and makes beagle_draft_step / beagle_draft_tree with 9..64 rows read them from then on.  Every other
+ *   path keeps reading the row-major weights, which must stay valid.  The copies do NOT follow later changes of the
+ *   weights: after an update in place call this again (same buffer allowed, once no earlier call still reads it).
+ *   packed_dev == NULL: back to the row-major weights.  An fp32 configuration accepts the call and does nothing.
+ * Errors: INVALID_ARG (NULL context / size pointer, misaligned buffer), CAPACITY (buffer too small), CUDA. */
+beagle_status beagle_packed_weights_bytes(const beagle_config* cfg, int32_t with_fp8_lm_head, size_t* bytes);
+beagle_status beagle_pack_weights(beagle_ctx* ctx, void* packed_dev, size_t bytes, void* stream);
+
 /* Workspace bytes of beagle_block_forward for `batch` sequences of S positions. */
 beagle_status beagle_block_workspace_bytes(const beagle_config* cfg, int32_t batch, int32_t S, size_t* bytes);
 

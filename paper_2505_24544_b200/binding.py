@@ -30,6 +30,7 @@ EXPORTED_SYMBOLS = (
     "beagle_profile_stage_name", "beagle_verify_greedy_static", "beagle_check_device", "beagle_selftest_wait_timeout",
     "beagle_workspace_buffer", "beagle_block_workspace_buffer", "beagle_verify_sample", "beagle_block_loss", "beagle_draft_tree", "beagle_verify_tree_greedy",
     "beagle_block_grad_workspace_bytes", "beagle_block_grad", "beagle_quantize_rows_e4m3",
+    "beagle_packed_weights_bytes", "beagle_pack_weights",
 )
 
 BUFFER_IDS = {"x": 0, "xn": 1, "q": 2, "o": 3, "y": 4, "yn": 5, "act": 6, "h": 7, "kt": 8, "vt": 9, "kp": 10, "vp": 11}
@@ -116,6 +117,10 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.beagle_verify_tree_greedy.restype = C.c_int
     lib.beagle_verify_sample.argtypes = [vp, i32, i32, vp, vp, vp, i32, C.c_float, vp, vp, vp, vp, vp]
     lib.beagle_verify_sample.restype = C.c_int
+    lib.beagle_packed_weights_bytes.argtypes = [C.POINTER(BeagleConfig), i32, szp]
+    lib.beagle_packed_weights_bytes.restype = C.c_int
+    lib.beagle_pack_weights.argtypes = [vp, vp, C.c_size_t, vp]
+    lib.beagle_pack_weights.restype = C.c_int
     lib.beagle_check_device.argtypes = [vp, vp]
     lib.beagle_check_device.restype = C.c_int
     lib.beagle_selftest_wait_timeout.argtypes = [vp, vp]
@@ -185,6 +190,7 @@ class Context:
         self.kv_buf = torch.empty(kv.value, dtype=torch.uint8, device=dev)
         self.ws_buf = torch.empty(ws.value, dtype=torch.uint8, device=dev)
         self.block_ws: Optional[torch.Tensor] = None
+        self.packed_buf: Optional[torch.Tensor] = None
         handle = C.c_void_p()
         st = self.lib.beagle_create(C.byref(cfg), C.byref(w), self.kv_buf.data_ptr(), kv.value, self.ws_buf.data_ptr(),
                                     ws.value, C.byref(handle))
@@ -433,6 +439,29 @@ def kv_cache_views(ctx: Context) -> Tuple[torch.Tensor, torch.Tensor]:
     return k, v
 
 
+def beagle_packed_weights_bytes(cfg: BeagleConfig, with_fp8_lm_head: bool) -> int:
+    n = C.c_size_t()
+    st = load_library().beagle_packed_weights_bytes(C.byref(cfg), int(bool(with_fp8_lm_head)), C.byref(n))
+    if st != 0:
+        raise BeagleError(st, "beagle_packed_weights_bytes rejected the configuration")
+    return int(n.value)
+
+
+def beagle_pack_weights(ctx: Context, enable: bool = True) -> None:
+    """Makes (or, enable=False, drops) the tile-major copies of the projection weights that draft steps of 9..64 rows stream.
+    Call again after changing the weights in place."""
+    if not enable:
+        ctx.check(ctx.lib.beagle_pack_weights(ctx.handle, None, 0, _stream()))
+        ctx.packed_buf = None
+        return
+    n = beagle_packed_weights_bytes(ctx.cfg, "w_lm_fp8" in ctx.weights)
+    if n == 0:
+        return
+    if ctx.packed_buf is None or ctx.packed_buf.numel() < n:
+        ctx.packed_buf = torch.empty(n, dtype=torch.uint8, device=ctx.kv_buf.device)
+    ctx.check(ctx.lib.beagle_pack_weights(ctx.handle, ctx.packed_buf.data_ptr(), n, _stream()))
+
+
 def beagle_selftest_wait_timeout(ctx: Context) -> None:
     """Launches the one-CTA kernel whose bounded wait runs out (test support for the device error path)."""
     ctx.check(ctx.lib.beagle_selftest_wait_timeout(ctx.handle, _stream()))
@@ -462,18 +491,24 @@ class BeagleHead:
 
     def __init__(self, *, hidden: int, n_q_heads: int, n_kv_heads: int, head_dim: int, mlp_dim: int, vocab: int,
                  dtype: str, weights: Dict[str, torch.Tensor], max_slots: int, max_ctx: int, max_draft: int,
-                 rms_eps: float = 1e-5, norm_q: bool = True, norm_mlp: bool = True, rope_theta: float = 0.0):
+                 rms_eps: float = 1e-5, norm_q: bool = True, norm_mlp: bool = True, rope_theta: float = 0.0,
+                 pack_weights: bool = True):
+        """pack_weights: bf16 heads keep tile-major copies of the projection weights for draft steps of 9..64 rows
+        (``beagle_pack_weights``; about the size of the weights without the embedding); after changing a weight tensor in
+        place call ``beagle_pack_weights(head.ctx)`` again."""
         code = {"fp32": BEAGLE_FP32, "bf16": BEAGLE_BF16}[dtype]
         self.cfg = BeagleConfig(hidden, n_q_heads, n_kv_heads, head_dim, mlp_dim, vocab, code, rms_eps, int(norm_q),
                                 int(norm_mlp), max_slots, max_ctx, max_draft, float(rope_theta))
         self.ctx = Context(self.cfg, weights)
+        if pack_weights:
+            beagle_pack_weights(self.ctx)
         self.weight_shapes = {n: tuple(weights[n].shape) for n in WEIGHT_NAMES}
         self.device = self.ctx.kv_buf.device
         self.dtype = torch_dtype(code)
 
     @classmethod
     def from_workload(cls, w, weights_np, device="cuda", max_slots=None, max_ctx=None, max_draft=None, rope_theta=0.0,
-                      fp8_lm_head=False) -> "BeagleHead":
+                      fp8_lm_head=False, pack_weights=True) -> "BeagleHead":
         """Uploads numpy float32 weights (already rounded to the storage type) and builds the head.
         fp8_lm_head: also make the FP8 copy of the LM head (used by draft steps of more than 8 rows)."""
         dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
@@ -483,7 +518,7 @@ class BeagleHead:
         return cls(hidden=w.hidden, n_q_heads=w.n_q_heads, n_kv_heads=w.n_kv_heads, head_dim=w.head_dim,
                    mlp_dim=w.mlp_dim, vocab=w.vocab, dtype=w.dtype, weights=weights,
                    max_slots=max_slots or w.batch, max_ctx=max_ctx or (w.ctx_max + 64),
-                   max_draft=max_draft or max(w.gamma, 1), rms_eps=w.rms_eps, rope_theta=rope_theta)
+                   max_draft=max_draft or max(w.gamma, 1), rms_eps=w.rms_eps, rope_theta=rope_theta, pack_weights=pack_weights)
 
     def prefill_kv(self, seq_slot, new_len, hidden):
         beagle_prefill_kv(self.ctx, seq_slot, new_len, hidden)

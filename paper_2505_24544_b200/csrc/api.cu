@@ -521,6 +521,62 @@ beagle_status beagle_selftest_wait_timeout(beagle_ctx* ctx, void* stream_) {
     return cuda_ok(ctx, "selftest_wait_timeout");
 }
 
+// The matrices that the 9..64-row serve path streams, in the order their tile-major copies lie in the caller's buffer.
+namespace {
+struct PackItem { const void* W; int N, K, elt_bytes; };
+int pack_items(const beagle_config& c, const beagle_weights* w, bool fp8, PackItem out[9]) {
+    const int qd = c.n_q_heads * c.head_dim, kd = c.n_kv_heads * c.head_dim;
+    int n = 0;
+    out[n++] = {w ? w->w_q : nullptr, qd, c.hidden, 2};
+    out[n++] = {w ? w->w_k : nullptr, kd, c.hidden, 2};
+    out[n++] = {w ? w->w_v : nullptr, kd, c.hidden, 2};
+    out[n++] = {w ? w->w_o : nullptr, c.hidden, qd, 2};
+    out[n++] = {w ? w->w_gate : nullptr, c.mlp_dim, c.hidden, 2};
+    out[n++] = {w ? w->w_up : nullptr, c.mlp_dim, c.hidden, 2};
+    out[n++] = {w ? w->w_down : nullptr, c.hidden, c.mlp_dim, 2};
+    out[n++] = {w ? w->w_lm : nullptr, c.vocab, c.hidden, 2};
+    if (fp8) out[n++] = {w ? w->w_lm_fp8 : nullptr, c.vocab, c.hidden, 1};
+    return n;
+}
+}  // namespace
+
+beagle_status beagle_packed_weights_bytes(const beagle_config* cfg, int32_t with_fp8_lm_head, size_t* bytes) {
+    if (bytes == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    *bytes = 0;
+    const beagle_status st = check_config(cfg);
+    if (st != BEAGLE_OK) return st;
+    if (cfg->dtype != BEAGLE_BF16) return BEAGLE_OK;
+    PackItem items[9];
+    const int n = pack_items(*cfg, nullptr, with_fp8_lm_head != 0, items);
+    size_t total = 0;
+    for (int i = 0; i < n; ++i) total += tc_skinny_packed_bytes(items[i].N, items[i].K, items[i].elt_bytes);
+    *bytes = total;
+    return BEAGLE_OK;
+}
+
+beagle_status beagle_pack_weights(beagle_ctx* ctx, void* packed_dev, size_t bytes, void* stream_) {
+    if (ctx == nullptr) return BEAGLE_ERR_INVALID_ARG;
+    if (ctx->tc == nullptr) return BEAGLE_OK;                          // fp32 configuration: nothing reads packed weights
+    tc_skinny_forget_packed(ctx->tc);
+    if (packed_dev == nullptr) return BEAGLE_OK;
+    if (reinterpret_cast<uintptr_t>(packed_dev) & (kAlign - 1)) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "packed weights buffer is not 256-byte aligned");
+    const bool fp8 = ctx->w.w_lm_fp8 != nullptr;
+    size_t need = 0;
+    beagle_packed_weights_bytes(&ctx->cfg, fp8 ? 1 : 0, &need);
+    if (bytes < need) return fail(ctx, BEAGLE_ERR_CAPACITY, "packed weights need %zu bytes, got %zu", need, bytes);
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    PackItem items[9];
+    const int n = pack_items(ctx->cfg, &ctx->w, fp8, items);
+    char* dst = static_cast<char*>(packed_dev);
+    for (int i = 0; i < n; ++i) {
+        // a matrix whose shape the tiled kernels do not take (row pitch not a multiple of 16 bytes) simply keeps its row-major form
+        const int r = tc_skinny_pack(ctx->tc, items[i].W, items[i].N, items[i].K, items[i].elt_bytes, dst, stream);
+        if (r > 0) ctx->launches += r;
+        dst += tc_skinny_packed_bytes(items[i].N, items[i].K, items[i].elt_bytes);
+    }
+    return cuda_ok(ctx, "pack_weights");
+}
+
 const char* beagle_last_error(const beagle_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
 int64_t beagle_launch_count(const beagle_ctx* ctx) { return ctx ? ctx->launches : 0; }
 

@@ -45,6 +45,7 @@ struct SkArgs {
     unsigned long long* keys; // [B][gridDim.x]
     const float* w_scale;     // FP8 LM head: per weight row
     const float* x_scale;     // FP8 LM head: per batch row
+    int packed;               // the weight maps describe tile-major copies: tile (ta, kb) is rows [(ta * kb_total + kb) * 128, +128)
     int* error_word;
 };
 
@@ -124,9 +125,11 @@ __device__ __forceinline__ void sk_body(const CUtensorMap* mapW, const CUtensorM
             // The weights do not depend on the previous kernel: fill the ring with weight tiles
             // while that kernel drains, then wait for it and add the activation tiles.
             const int npre = min(nkb, kStages);
+            // row-major weights: the tile's 128 rows, 128 bytes at column kb of each; packed: one contiguous tile of 16 KB
+            const int wx = args.packed ? 0 : BKE, wy0 = args.packed ? (ta * kb_total + kb0) * BM : ta * BM, wy = args.packed ? BM : 0;
             for (int kb = 0; kb < npre; ++kb) {
                 mbar_expect_tx(bar_full + 8 * kb, SM::kStageBytes);
-                tma_load_2d_hint(smem_base + kb * SM::kStageBytes, mapW, bar_full + 8 * kb, (kb0 + kb) * BKE, ta * BM, stream_once);
+                tma_load_2d_hint(smem_base + kb * SM::kStageBytes, mapW, bar_full + 8 * kb, (kb0 + kb) * wx, wy0 + kb * wy, stream_once);
             }
             pdl_wait();
             for (int kb = 0; kb < npre; ++kb)
@@ -139,7 +142,7 @@ __device__ __forceinline__ void sk_body(const CUtensorMap* mapW, const CUtensorM
                 const uint32_t sa = smem_base + s * SM::kStageBytes, sb = sa + kABytes;
                 mbar_expect_tx(bar_full + 8 * s, SM::kStageBytes);
                 const int kc = (kb0 + kb) * BKE;
-                tma_load_2d_hint(sa, mapW, bar_full + 8 * s, kc, ta * BM, stream_once);
+                tma_load_2d_hint(sa, mapW, bar_full + 8 * s, (kb0 + kb) * wx, wy0 + kb * wy, stream_once);
                 tma_load_2d_hint(sb, mapX, bar_full + 8 * s, kc, 0, keep);
                 ++issued;
             }
@@ -401,6 +404,22 @@ __global__ void __launch_bounds__(kFinThreads) tc_finish_kernel(const FinishArgs
     }
 }
 
+// ---------------------------------------------------------------------------------------------- tile-major weight copies
+// One thread per 16-byte piece of the destination: tile t = ta * kb_total + kb holds rows [128 ta, +128) x bytes [128 kb, +128)
+// of the source, row r of the tile at 128 r inside it; pieces outside the matrix are zero.
+__global__ void __launch_bounds__(256) pack_tiles_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, const int N,
+                                                         const long long row_bytes, const int kb_total, const long long pieces) {
+    const long long idx = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (idx >= pieces) return;
+    const int c = (int)(idx & 7), r = (int)((idx >> 3) & 127);
+    const long long t = idx >> 10;
+    const int kb = (int)(t % kb_total);
+    const long long row = (t / kb_total) * BM + r, byte = (long long)kb * 128 + c * 16;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (row < N && byte < row_bytes) v = src[(row * row_bytes + byte) >> 4];
+    dst[idx] = v;
+}
+
 struct SplitPlan { int tiles, kb_total, kb_per_split, splits; };
 SplitPlan split_plan(int N, int K, int nmat, bool allow_split) {
     SplitPlan s;
@@ -474,14 +493,61 @@ int launch_sk_qkv(const CUtensorMap& wq, const CUtensorMap& wk, const CUtensorMa
 
 }  // namespace
 
+size_t tc_skinny_packed_bytes(int N, int K, int elt_bytes) {
+    const size_t tiles = (N + BM - 1) / BM, kb_total = ((size_t)K * elt_bytes + 127) / 128;
+    return tiles * kb_total * (size_t)(BM * 128);
+}
+
+int tc_skinny_pack(TcPlan* p, const void* W, int N, int K, int elt_bytes, void* dst, cudaStream_t stream) {
+    if (p == nullptr || W == nullptr) return -1;
+    p->packed.erase(W);
+    if (dst == nullptr) return 0;
+    const long long row_bytes = (long long)K * elt_bytes;
+    if ((elt_bytes != 1 && elt_bytes != 2) || N <= 0 || K <= 0 || row_bytes % 16 || (reinterpret_cast<uintptr_t>(W) & 15) ||
+        (reinterpret_cast<uintptr_t>(dst) & 127))
+        return -1;
+    const int kb_total = (int)((row_bytes + 127) / 128);
+    const long long rows = (long long)((N + BM - 1) / BM) * kb_total * BM, pieces = rows * 8;
+    if (rows > 0x7fffffffLL) return -1;                    // the tile's first row is a 32-bit TMA coordinate
+    TcPlan::Packed e;
+    e.tiles = dst; e.N = N; e.K = K; e.elt_bytes = elt_bytes;
+    // the copy as a matrix of `rows` rows of 128 bytes: a box of 128 rows is one tile
+    const bool ok = elt_bytes == 2 ? tc_encode_map(p, &e.map, dst, rows, BK, BK, BM) : tc_encode_map_u8(p, &e.map, dst, rows, 128, 128, BM);
+    if (!ok) return -1;
+    pack_tiles_kernel<<<(unsigned)((pieces + 255) / 256), 256, 0, stream>>>(static_cast<const uint4*>(W), static_cast<uint4*>(dst), N, row_bytes,
+                                                                            kb_total, pieces);
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    p->packed.emplace(W, e);
+    return 1;
+}
+
+void tc_skinny_forget_packed(TcPlan* p) {
+    if (p != nullptr) p->packed.clear();
+}
+
+namespace {
+// The tile-major copy's map when W [N, K] has one, else nullptr.
+const CUtensorMap* packed_map(TcPlan* p, const void* W, int N, int K, int elt_bytes) {
+    auto it = p->packed.find(W);
+    if (it == p->packed.end() || it->second.N != N || it->second.K != K || it->second.elt_bytes != elt_bytes) return nullptr;
+    return &it->second.map;
+}
+}  // namespace
+
 int tc_skinny_qkv(TcPlan* p, const SkinnyArgs& q, const SkinnyArgs& kv, cudaStream_t stream) {
     if (p == nullptr || q.B <= 0 || q.B > kMaxCallBatch || kv.B != q.B || kv.K != q.K) return -1;
     if (q.K % 8 || q.ldx % 8 || kv.ldx % 8 || (q.N % 4) || (kv.N % 4) || (kv.dh % 4)) return -1;
     if ((reinterpret_cast<uintptr_t>(q.X) & 15) || (reinterpret_cast<uintptr_t>(kv.X) & 15)) return -1;
     const int bn = q.B <= 16 ? 16 : (q.B <= 32 ? 32 : 64);
-    const CUtensorMap* mapWq = tc_weight_map(p, q.W, q.N, q.K, BM);
-    const CUtensorMap* mapWk = tc_weight_map(p, kv.W, kv.N, kv.K, BM);
-    const CUtensorMap* mapWv = tc_weight_map(p, kv.W2, kv.N, kv.K, BM);
+    const CUtensorMap* mapWq = packed_map(p, q.W, q.N, q.K, 2);
+    const CUtensorMap* mapWk = packed_map(p, kv.W, kv.N, kv.K, 2);
+    const CUtensorMap* mapWv = packed_map(p, kv.W2, kv.N, kv.K, 2);
+    const bool packed = mapWq != nullptr && mapWk != nullptr && mapWv != nullptr;       // one flag for the launch: all three or none
+    if (!packed) {
+        mapWq = tc_weight_map(p, q.W, q.N, q.K, BM);
+        mapWk = tc_weight_map(p, kv.W, kv.N, kv.K, BM);
+        mapWv = tc_weight_map(p, kv.W2, kv.N, kv.K, BM);
+    }
     CUtensorMap mapXq, mapXkv;
     if (mapWq == nullptr || mapWk == nullptr || mapWv == nullptr || !tc_encode_map(p, &mapXq, q.X, q.B, q.K, q.ldx, bn) ||
         !tc_encode_map(p, &mapXkv, kv.X, kv.B, kv.K, kv.ldx, bn))
@@ -493,6 +559,7 @@ int tc_skinny_qkv(TcPlan* p, const SkinnyArgs& q, const SkinnyArgs& kv, cudaStre
     SkArgs a;
     memset(&a, 0, sizeof(a));
     a.N = q.N; a.K = q.K; a.B = q.B; a.nmat = 1; a.kb_per_split = (kb_total + cs - 1) / cs; a.error_word = q.error_word;
+    a.packed = packed ? 1 : 0;
     FinishArgs f;
     memset(&f, 0, sizeof(f));
     f.splits = cs; f.nmat = 1; f.B = q.B; f.N = q.N;
@@ -521,21 +588,29 @@ int tc_skinny(TcPlan* p, int mode, const SkinnyArgs& g, cudaStream_t stream) {
     if (mode == SK_KV && (g.dh % 4)) return -1;
     const int nmat = (mode == SK_SILU_MUL || mode == SK_KV) ? 2 : 1;
     const int bn = g.B <= 16 ? 16 : (g.B <= 32 ? 32 : 64);
-    const CUtensorMap* mapW = tc_weight_map(p, g.W, g.N, g.K, BM);
-    const CUtensorMap* mapW2 = nmat == 2 ? tc_weight_map(p, g.W2, g.N, g.K, BM) : mapW;
+    const CUtensorMap* mapW = packed_map(p, g.W, g.N, g.K, 2);
+    const CUtensorMap* mapW2 = nmat == 2 ? packed_map(p, g.W2, g.N, g.K, 2) : mapW;
+    const bool packed = mapW != nullptr && mapW2 != nullptr;
+    if (!packed) {
+        mapW = tc_weight_map(p, g.W, g.N, g.K, BM);
+        mapW2 = nmat == 2 ? tc_weight_map(p, g.W2, g.N, g.K, BM) : mapW;
+    }
     CUtensorMap mapX;
     if (mapW == nullptr || mapW2 == nullptr || !tc_encode_map(p, &mapX, g.X, g.B, g.K, g.ldx, bn)) return -1;
     const bool logits = (mode == SK_LOGITS);
     if (logits && g.W8 != nullptr) {
         // FP8 LM head: byte tensor maps (128 elements per swizzle row), scales applied in the epilogue
         if (g.K % 16 || g.X8 == nullptr || g.w_scale == nullptr || g.x_scale == nullptr || (reinterpret_cast<uintptr_t>(g.X8) & 15)) return -1;
-        const CUtensorMap* mapW8 = tc_weight_map_u8(p, g.W8, g.N, g.K, BM);
+        const CUtensorMap* mapW8 = packed_map(p, g.W8, g.N, g.K, 1);
+        const bool packed8 = mapW8 != nullptr;
+        if (!packed8) mapW8 = tc_weight_map_u8(p, g.W8, g.N, g.K, BM);
         CUtensorMap mapX8;
         if (mapW8 == nullptr || !tc_encode_map_u8(p, &mapX8, g.X8, g.B, g.K, g.K, bn)) return -1;
         SkArgs a8;
         memset(&a8, 0, sizeof(a8));
         a8.N = g.N; a8.K = g.K; a8.B = g.B; a8.nmat = 1; a8.kb_per_split = (g.K + 2 * BK - 1) / (2 * BK);
         a8.logits = g.logits; a8.keys = g.keys; a8.w_scale = g.w_scale; a8.x_scale = g.x_scale; a8.error_word = g.error_word;
+        a8.packed = packed8 ? 1 : 0;
         FinishArgs f8;
         memset(&f8, 0, sizeof(f8));
         const dim3 grid8((g.N + BM - 1) / BM, 1, 1);
@@ -550,6 +625,7 @@ int tc_skinny(TcPlan* p, int mode, const SkinnyArgs& g, cudaStream_t stream) {
     memset(&a, 0, sizeof(a));
     a.N = g.N; a.K = g.K; a.B = g.B; a.nmat = nmat; a.kb_per_split = sp.kb_per_split;
     a.partial = g.partial; a.logits = g.logits; a.keys = g.keys; a.error_word = g.error_word;
+    a.packed = packed ? 1 : 0;
     dim3 grid(sp.tiles, nmat, sp.splits);
     FinishArgs f;
     memset(&f, 0, sizeof(f));

@@ -57,6 +57,13 @@ int tc_skinny_qkv(TcPlan* plan, const SkinnyArgs& q, const SkinnyArgs& kv, cudaS
 // Bytes of fp32 partial sums a projection [N, K] with `nmat` weight matrices needs for 64 rows.
 size_t tc_skinny_partial_bytes(int N, int K, int nmat);
 int tc_skinny_key_tiles(int N);
+// Tile-major copy of a K-major weight matrix [N, K] (elt_bytes 2: bf16, 1: FP8 bytes) for the kernels above: tile (ta, kb) = rows
+// [128 ta, +128) x bytes [128 kb, +128) of the matrix, 16 KB contiguous, at ((ta * ceil(K * elt_bytes / 128)) + kb) * 16 KB; rows and
+// bytes past the matrix are zero.  tc_skinny_packed_bytes: size of the copy.  tc_skinny_pack: writes it (one launch) and registers
+// it, so that tc_skinny / tc_skinny_qkv given W read `dst` instead; dst == nullptr forgets W's copy.  Returns launches or -1.
+size_t tc_skinny_packed_bytes(int N, int K, int elt_bytes);
+int tc_skinny_pack(TcPlan* plan, const void* W, int N, int K, int elt_bytes, void* dst, cudaStream_t stream);
+void tc_skinny_forget_packed(TcPlan* plan);
 
 // ---- TMA-staged decode attention over the bf16 cache (head_dim 64 or 128) ----------------------
 // Binds the cache halves ([rows, head_dim] each); false when the shape is not covered.

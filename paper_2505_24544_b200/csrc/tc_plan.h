@@ -19,6 +19,8 @@ struct TcPlan {
     beagle_config cfg;
     beagle_weights w;
     std::map<std::pair<const void*, int>, CUtensorMap> weight_maps;   // (pointer, box rows) -> map
+    struct Packed { const void* tiles; int N, K, elt_bytes; CUtensorMap map; };
+    std::map<const void*, Packed> packed;                             // row-major weight pointer -> its tile-major copy
     int sm_count = 148;
     CUtensorMap cache_k, cache_v;      // the K/V cache as [rows, head_dim] for the staged decode attention
     bool cache_maps_ok = false;

@@ -82,6 +82,29 @@ def test_query_sizes_and_shape_validation(lib):
     assert lib.beagle_block_grad_workspace_bytes(C.byref(cfg), 1 << 13, 1 << 13, C.byref(g)) == 3       # more than 2^24 positions
 
 
+def test_packed_weights_bytes_counts_whole_tiles(lib):
+    """Tile-major copies: every matrix padded to tiles of 128 rows x 128 bytes (64 bf16 / 128 FP8 elements)."""
+    def tiles(n, k, elt):
+        return -(-n // 128) * -(-(k * elt) // 128) * 128 * 128
+    cfg = good_config()
+    n = C.c_size_t()
+    assert lib.beagle_packed_weights_bytes(C.byref(cfg), 0, C.byref(n)) == 0
+    want = 2 * tiles(4096, 4096, 2) + 2 * tiles(1024, 4096, 2) + 2 * tiles(14336, 4096, 2) + tiles(4096, 14336, 2) + tiles(128256, 4096, 2)
+    assert n.value == want
+    assert lib.beagle_packed_weights_bytes(C.byref(cfg), 1, C.byref(n)) == 0
+    assert n.value == want + tiles(128256, 4096, 1)
+    odd = good_config(); odd.hidden = 520; odd.mlp_dim = 1416; odd.vocab = 4099; odd.n_q_heads = 8; odd.n_kv_heads = 2; odd.head_dim = 64
+    assert lib.beagle_packed_weights_bytes(C.byref(odd), 0, C.byref(n)) == 0
+    assert n.value == (tiles(512, 520, 2) + 2 * tiles(128, 520, 2) + tiles(520, 512, 2) + 2 * tiles(1416, 520, 2) + tiles(520, 1416, 2)
+                       + tiles(4099, 520, 2))
+    fp32 = good_config(); fp32.dtype = 0
+    assert lib.beagle_packed_weights_bytes(C.byref(fp32), 0, C.byref(n)) == 0 and n.value == 0
+    assert lib.beagle_packed_weights_bytes(C.byref(cfg), 0, None) == 1
+    bad = good_config(); bad.n_kv_heads = 5
+    assert lib.beagle_packed_weights_bytes(C.byref(bad), 0, C.byref(n)) == 2
+    assert lib.beagle_pack_weights(None, None, 0, None) == 1
+
+
 def test_null_context_is_rejected(lib):
     assert lib.beagle_prefill_kv(None, 0, None, None, None, None) == 1
     assert lib.beagle_draft_step(None, 0, None, None, 1, None, 1, None, None, None) == 1

@@ -742,6 +742,59 @@ def test_fp8_lm_head_batched_draft_steps(batch):
     beagle_check_device(head_gpu.ctx)
 
 
+@pytest.mark.parametrize("batch,fp8", [(12, False), (33, False), (64, True)])
+def test_packed_weight_copies_give_the_same_bits_and_follow_a_repack(batch, fp8):
+    """The tile-major weight copies are a re-layout only: a chain of batched draft steps gives bit-identical logits,
+    states and tokens with and without them (sizes that leave ragged tiles in both directions: 1416 and 4099 rows, 520-
+    and 1416-element reductions); after a weight changes in place, a repack follows it and a head without copies agrees."""
+    from paper_2505_24544_b200.binding import (BeagleHead, beagle_pack_weights, beagle_packed_weights_bytes, beagle_check_device,
+                                               beagle_reset_slot)
+    w = SMALL_GQA.scaled(batch=batch, hidden=528 if fp8 else 520, ctx_min=3, ctx_max=150, gamma=3, seed=2011, mlp_dim=1416, vocab=4099)
+    weights = WL.make_weights(w)
+    heads = [BeagleHead.from_workload(w, weights, max_ctx=w.ctx_max + 64, fp8_lm_head=fp8, pack_weights=pk) for pk in (True, False)]
+    assert heads[0].ctx.packed_buf is not None and heads[1].ctx.packed_buf is None
+    assert heads[0].ctx.packed_buf.numel() == beagle_packed_weights_bytes(heads[0].cfg, fp8)
+    rng = WL.data_rng(w, batch)
+    lengths = WL.make_context_lengths(w, rng)
+    hidden = to_dev(WL.make_hidden(w, rng, int(np.sum(lengths))), w.dtype)
+    first = to_dev(WL.make_tokens(w, rng, (batch,)), w.dtype)
+    slots = list(range(batch))
+
+    def chain(head):
+        for slot in slots:
+            beagle_reset_slot(head.ctx, slot)
+        head.prefill_kv(slots, list(map(int, lengths)), hidden)
+        out = []
+        for step in range(3):
+            out.append(head.draft_step(slots, tokens_in=first if step == 0 else None, want_logits=True, want_hidden=True))
+        torch.cuda.synchronize()
+        return out
+
+    def same(a, b, what):
+        for step, (x, y) in enumerate(zip(a, b)):
+            for name, u, v in zip(("tokens", "logits", "hidden"), x, y):
+                assert torch.equal(u, v), f"{what}: step {step} {name} differ"
+
+    ref = chain(heads[1])
+    same(chain(heads[0]), ref, "packed vs row-major")
+    # a weight changes in place: the copies are stale until the repack, then both heads agree again
+    for head in heads:
+        head.ctx.weights["w_gate"].mul_(-0.5)
+        head.ctx.weights["w_lm"][::3].mul_(0.25)
+        if fp8:
+            head.ctx.weights["w_lm_fp8"][::5] ^= 0x80          # flips the sign of every fifth row's codes
+    ref2 = chain(heads[1])
+    assert not torch.equal(ref2[0][1], ref[0][1])
+    stale = chain(heads[0])
+    assert torch.equal(stale[0][1], ref[0][1]), "the copies do not follow the weights by themselves"
+    beagle_pack_weights(heads[0].ctx)
+    same(chain(heads[0]), ref2, "after repack")
+    beagle_pack_weights(heads[0].ctx, enable=False)
+    same(chain(heads[0]), ref2, "copies dropped")
+    for head in heads:
+        beagle_check_device(head.ctx)
+
+
 def test_bounded_wait_runs_out_and_is_reported_once():
     """The device error path without any fault or hang: a one-CTA kernel polls, with a short limit, a barrier that nothing
     completes and no copy targets; it gives up, raises the context's error word and returns.  beagle_check_device then
@@ -775,11 +828,12 @@ def test_first_call_inside_stream_capture_is_refused():
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
     g = torch.cuda.CUDAGraph()
+    launched = head_gpu.launch_count                         # the weight re-layout at construction
     with pytest.raises(B.BeagleError) as e:
         with torch.cuda.graph(g, stream=side):
             head_gpu.prefill_kv([0, 1], [10, 20], hidden)
     assert e.value.status == 4 and "capture" in str(e.value)
-    assert head_gpu.slot_lengths(0) == (0, 0) and head_gpu.launch_count == 0
+    assert head_gpu.slot_lengths(0) == (0, 0) and head_gpu.launch_count == launched
     torch.cuda.synchronize()
     head_gpu.prefill_kv([0, 1], [10, 20], hidden)            # the ordinary first call
     assert head_gpu.slot_lengths(1) == (20, 0)
