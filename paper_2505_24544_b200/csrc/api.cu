@@ -1665,7 +1665,7 @@ beagle_status beagle_draft_tree(beagle_ctx* ctx, int32_t slot, const int32_t* ro
             BEAGLE_TREE_SKINNY(SK_LOGITS, a, "LM head");
         }
         ctx->launches += launch_topk_logprob(ctx->tree_logits, rows, c.vocab, topk, T, stream);
-        ctx->launches += launch_tree_expand(T, topk, e, e == 0 ? 0 : topk + (e - 1) * topk * topk, stream);
+        ctx->launches += launch_tree_expand(T, c.vocab, topk, rows, e, e == 0 ? 0 : topk + (e - 1) * topk * topk, stream);
     }
 #undef BEAGLE_TREE_SKINNY
     ctx->launches += launch_tree_rerank(T, total, n_candidates, tree_tokens_dev, tree_parents_dev, tree_scores_dev, stream);

@@ -89,7 +89,6 @@ constexpr int kTreeMaxTopk = 16, kTreeMaxDepth = 8, kTreeMaxCandidates = 64;
 constexpr int kTreeMaxNodes = kTreeMaxTopk + kTreeMaxDepth * kTreeMaxTopk * kTreeMaxTopk;
 struct TreeArrays {
     int32_t* node_tok; int32_t* node_par; float* node_score;       // every node created, in creation order
-    int32_t* child_tok; float* child_lq;                           // [rows][k] of the last forward: k best children, log-probabilities
     int32_t* frontier_node; int32_t* frontier_tok;                 // [k] nodes to forward next and their tokens
     int32_t* frontier_anc;                                         // [k][kTreeMaxDepth + 1] tail positions of their ancestors' states
     float2* topk_lse; unsigned long long* topk_keys;               // per (row, vocabulary slice): (max, exp-sum) and the slice's k best keys
@@ -97,7 +96,7 @@ struct TreeArrays {
 size_t tree_arrays_bytes(int vocab);
 TreeArrays tree_arrays_carve(void* mem, int vocab);
 int launch_topk_logprob(const float* logits, int rows, int V, int k, const TreeArrays& t, cudaStream_t stream);
-int launch_tree_expand(const TreeArrays& t, int k, int level, int base, cudaStream_t stream);
+int launch_tree_expand(const TreeArrays& t, int V, int k, int rows, int level, int base, cudaStream_t stream);
 int launch_tree_rerank(const TreeArrays& t, int total, int n, int32_t* out_tok, int32_t* out_par, float* out_score, cudaStream_t stream);
 // Attention partial over each row's ancestor draft states, stored as split-KV chunk `chunk_idx` (bf16, dh 64 / 128).
 int launch_attn_tail(const void* q, const void* kcache, const void* vcache, const int32_t* anc, int nanc, int rows, int slot, int n_true, int Hq,
