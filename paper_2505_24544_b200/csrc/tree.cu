@@ -135,10 +135,17 @@ __global__ void __launch_bounds__(32 * kTreeMaxTopk) tree_expand_kernel(TreeArra
         const float lse = M + __logf(S);
         const unsigned long long* cand = t.topk_keys + (size_t)warp * nsplit * k;
         const int ncand = nsplit * k;
+        constexpr int kHeld = 16;                              // candidates a lane keeps in registers (512 per row: 32 slices of 16)
+        unsigned long long held[kHeld];
+#pragma unroll
+        for (int e = 0; e < kHeld; ++e) held[e] = lane + e * 32 < ncand ? cand[lane + e * 32] : 0ull;
         unsigned long long prev = ~0ull;
         for (int j = 0; j < k; ++j) {
             unsigned long long best = 0ull;
-            for (int i = lane; i < ncand; i += 32) {
+#pragma unroll
+            for (int e = 0; e < kHeld; ++e)
+                if (held[e] < prev && held[e] > best) best = held[e];
+            for (int i = lane + kHeld * 32; i < ncand; i += 32) {      // larger vocabularies: the rest from memory
                 const unsigned long long key = cand[i];
                 if (key < prev && key > best) best = key;
             }
