@@ -842,7 +842,8 @@ def main():
     sampler = ClockSampler(physical_gpu_index(local))
     scn = ServeScenario(head, w, iters, device)
     if args.only_legs:
-        out = {"prefill": {w.name: bench_prefill(scn, peaks)}, "verify_greedy_logits": {w.name: bench_verify_greedy_logits(head, w, peaks)}}
+        out = {"prefill": {w.name: bench_prefill(scn, peaks)}, "verify_greedy_logits": {w.name: bench_verify_greedy_logits(head, w, peaks)},
+               "verify_sample": bench_verify_sample(head, w, steps=20, warmup=3, peaks=peaks)}
         w3 = WL.WORKLOADS["c3_llama3_8b_b1"]
         if w.name == HEADLINE and args.legs_batch == 0:
             scn3 = ServeScenario(head, w3, iters, device)

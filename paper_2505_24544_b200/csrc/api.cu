@@ -1528,9 +1528,11 @@ beagle_status beagle_verify_sample(beagle_ctx* ctx, int32_t batch, int32_t gamma
         return fail(ctx, BEAGLE_ERR_INVALID_ARG, "verify_sample: NULL argument");
     if (logits_dtype != BEAGLE_FP32 && logits_dtype != BEAGLE_BF16) return fail(ctx, BEAGLE_ERR_INVALID_ARG, "verify_sample: unknown logits_dtype");
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const beagle_status st0 = device_setup_once(ctx, stream);          // the sequences' tickets must read zero
+    if (st0 != BEAGLE_OK) return st0;
     StageTimer timer_(ctx, ST_VERIFY, stream);
     ctx->launches += launch_verify_sample(logits_dtype, draft_tokens_dev, draft_logits_dev, target_logits_dev, batch, gamma, ctx->cfg.vocab,
-                                          temperature, u_accept_dev, u_resample_dev, ctx->vs_scratch, accept_len_dev, out_tokens_dev, ctx->sm_count, stream);
+                                          temperature, u_accept_dev, u_resample_dev, ctx->vs_scratch, verify_tickets(ctx), accept_len_dev, out_tokens_dev, ctx->sm_count, stream);
     return cuda_ok(ctx, "verify_sample");
 }
 

@@ -81,7 +81,7 @@ int launch_accept(const int32_t* draft, const int32_t* target_ids, int B, int ga
 // [gamma, B, V]; target_logits [B, gamma+1, V] fp32 or bf16.
 size_t verify_sample_scratch_bytes(int max_batch, int max_gamma);
 int launch_verify_sample(int logits_dtype, const int32_t* draft, const float* draft_logits, const void* target_logits, int B, int gamma, int V,
-                         float temperature, const float* u_accept, const float* u_resample, void* scratch, int32_t* accept_len,
+                         float temperature, const float* u_accept, const float* u_resample, void* scratch, int* tickets, int32_t* accept_len,
                          int32_t* out_tokens, int sm_count, cudaStream_t stream);
 
 // ---- dynamic-tree drafting: device-side bookkeeping -------------------------------------------
