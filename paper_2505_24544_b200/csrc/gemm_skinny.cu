@@ -205,17 +205,32 @@ __device__ __forceinline__ void sk_body(const CUtensorMap* mapW, const CUtensorM
                         for (int j = 0; j < 16; ++j)
                             if (c0 + j < args.B) dst[(size_t)(c0 + j) * args.N] = __uint_as_float(r[j]);
                     }
-                } else {
+                } else if (c0 < args.B) {
+                    // the 16 columns' keys first, then the five shuffle rounds over all of them at once: sixteen independent
+                    // chains per round instead of sixteen reductions one after the other (each a chain of five shuffle latencies)
+                    unsigned long long key[16];
+                    const float ws = FP8 ? (feat < args.N ? args.w_scale[feat] : 0.f) : 1.f;
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
                         const int col = c0 + j;
-                        if (col >= args.B) break;                         // uniform across the warp
+                        const bool live = col < args.B && feat < args.N;
                         float v = __uint_as_float(r[j]);
-                        if (FP8) v *= (feat < args.N ? args.w_scale[feat] : 0.f) * args.x_scale[col];
-                        unsigned long long key = feat < args.N ? argmax_key(v, feat) : 0ull;
-                        if (args.logits != nullptr && feat < args.N) args.logits[(size_t)col * args.N + feat] = v;
-                        key = warp_max_u64(key);
-                        if (lane == 0) s_keys[q * BN + col] = key;
+                        if (FP8) v *= ws * (col < args.B ? args.x_scale[col] : 0.f);
+                        if (live && args.logits != nullptr) args.logits[(size_t)col * args.N + feat] = v;
+                        key[j] = live ? argmax_key(v, feat) : 0ull;
+                    }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const unsigned long long other = __shfl_xor_sync(0xffffffffu, key[j], o);
+                            key[j] = other > key[j] ? other : key[j];
+                        }
+                    }
+                    if (lane == 0) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (c0 + j < args.B) s_keys[q * BN + c0 + j] = key[j];
                     }
                 }
             }
@@ -283,7 +298,7 @@ __device__ __forceinline__ void sk_body(const CUtensorMap* mapW, const CUtensorM
 }
 
 template <int BN, int VAR, bool FP8>
-__global__ void __launch_bounds__(kSkThreads) tc_skinny_kernel(const __grid_constant__ CUtensorMap tmW,
+__global__ void __launch_bounds__(kSkThreads, 3) tc_skinny_kernel(const __grid_constant__ CUtensorMap tmW,
                                                                const __grid_constant__ CUtensorMap tmW2,
                                                                const __grid_constant__ CUtensorMap tmX, const SkArgs args,
                                                                const FinishArgs fin, const int mode) {
