@@ -32,8 +32,7 @@ template <int BN>
 struct SkSmem {
     static constexpr int kStageBytes = kABytes + BN * BK * 2;
     static constexpr int kStages = 3;            // 54-72 KB per CTA: three CTAs per SM, so a dependent launch finds a free slot to prefetch in
-    static constexpr int kKeyBytes = 4 * BN * 8;
-    static constexpr int kBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/ + kKeyBytes;
+    static constexpr int kBytes = kStages * kStageBytes + 1024 /*align*/ + 256 /*barriers*/;   // 64 columns: 75 KB, still three CTAs per SM
 };
 
 struct SkArgs {
@@ -97,7 +96,7 @@ __device__ __forceinline__ void sk_body(const CUtensorMap* mapW, const CUtensorM
     const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * kStages, bar_acc = bar_empty + 8 * kStages;
     uint32_t* s_tmem = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 1);
     volatile int* s_abort = reinterpret_cast<volatile int*>(s_tmem + 1);
-    unsigned long long* s_keys = reinterpret_cast<unsigned long long*>(smem_gen + kStages * SM::kStageBytes + 256);
+    unsigned long long* s_keys = reinterpret_cast<unsigned long long*>(smem_gen);     // [4][BN], over the ring: it is idle once the accumulator is complete
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int BKE = FP8 ? 2 * BK : BK;        // elements per 128-byte row of a tile
