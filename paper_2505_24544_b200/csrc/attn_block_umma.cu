@@ -4,18 +4,20 @@
 // One CTA = 128 consecutive query positions of one (sequence, query head): the 128 rows of an MMA
 // tile, one TMEM lane and one softmax thread per query, so row maxima and row sums need no
 // cross-thread reduction.  Keys are walked in tiles of 64 (true tiles up to the largest n(p) of the
-// CTA, then the predicted band on the diagonal, as in the mma.sync kernel).  The walk is done twice:
-//   pass 1:  S = Q K^T per tile -> every row's maximum of the masked, scaled scores;
-//   pass 2:  S again -> P = exp2(S - max) rounded to bf16 (row sums over the rounded weights),
-//            written to shared memory in the MMA's operand layout -> O += P V accumulated in TMEM
-//            over all tiles, read once at the end, normalised and stored.
-// Recomputing S (a third of the work again) removes the running-maximum rescale of O, which on this
-// architecture would mean reading and rewriting the TMEM accumulator for every tile or holding O
-// in 128 registers per thread; with O resident in TMEM two CTAs fit an SM and overlap each other's
-// softmax with MMAs.  V is read as it lies ([key][head_dim]: the B operand of P V in its MN-major form),
-// so no transposed copy of the values is made.
+// CTA, then the predicted band on the diagonal, as in the mma.sync kernel), once:
+//   S = Q K^T per tile -> P = exp2(S - m) rounded to bf16 (row sums over the rounded weights), written to shared
+//   memory in the MMA's operand layout -> O += P V accumulated in TMEM over all tiles, read once at the end,
+//   normalised and stored.
+// m is the row's reference point, not its running maximum: it is set by the row's first visible tile and moves only when a
+// later tile exceeds it by more than 8 (a factor 256: harmless in bf16 and fp32).  Only then the accumulated O row and row sum
+// are scaled by 2^(m_old - m_new) -- a read-modify-write of the warp's O rows in tensor memory, which a running maximum would
+// ask for in almost every tile and which happens here a few times per row at most.  (An earlier form avoided the rescale by
+// walking the keys twice, maxima first: a third more MMA work and twice the softmax-side work.)  With O resident in TMEM two
+// CTAs fit an SM and overlap each other's softmax with MMAs.  V is read as it lies ([key][head_dim]: the B operand of P V in
+// its MN-major form), so no transposed copy of the values is made.
 //
-// Roles: warp 0 = TMA producer (Q once; K tiles in a two-stage ring, V tile single-buffered),
+// Roles: warp 0 = TMA producer (Q once; K and V tiles in two-stage rings of their own: a K slot is free once its S is
+// complete, a V slot once its P V is),
 // warp 1 = MMA issuer and TMEM owner (two S buffers of 64 columns + the O accumulator), warps 2-5 =
 // softmax (warp w owns TMEM lanes 32 (w % 4) ..).  Every wait is bounded; a wait that runs out
 // raises the error word, the CTA drains and frees its TMEM.
@@ -52,7 +54,10 @@ struct UmmaAttnSmem {
     static constexpr int kK = kUKey * DH * 2;           // DH/64 tiles of [64 keys x 64]
     static constexpr int kV = DH * kUKey * 2;           // DH/64 blocks of [64 keys x 64 dims]
     static constexpr int kP = kUQ * kUKey * 2;          // [128 x 64 keys]
-    static constexpr int kBytes = kQ + 2 * kK + kV + kP + 1024 /*align*/ + 128 /*barriers*/;
+    // Q, two K tiles, two V tiles, P, then 256 bytes of barriers and flags: 112.25 KB at head_dim 128, so that two CTAs share an
+    // SM.  No slack for alignment: the kernel checks that its dynamic shared memory starts on a 1 KB boundary (it does when the
+    // kernel has no static shared memory) and otherwise raises the error word instead of running.
+    static constexpr int kBytes = kQ + 2 * kK + 2 * kV + kP + 256;
 };
 
 template <int DH>
@@ -64,16 +69,21 @@ __global__ void __launch_bounds__(kUThreads, 2) attn_block_umma_kernel(const __g
     using SM = UmmaAttnSmem<DH>;
     constexpr int kHalves = DH / 64;
     constexpr uint32_t kTmemCols = 256;                  // S buffers at columns 0 and 64, O at 128 .. 128 + DH
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-    const uint32_t sQ = smem_base, sK = sQ + SM::kQ, sV = sK + 2 * SM::kK, sP = sV + SM::kV;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + SM::kQ + 2 * SM::kK + SM::kV + SM::kP);
+    constexpr float kSlack = 8.f;                        // how far a tile's maximum may exceed the row's reference point before it moves
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t smem_base = smem_u32(smem_raw);
+    if (smem_base & 1023u) {                                    // the swizzled tiles need 1 KB alignment: refuse rather than compute nonsense
+        if (threadIdx.x == 0 && a.error_word != nullptr) atomicExch(a.error_word, 1);
+        return;
+    }
+    uint8_t* smem_gen = smem_raw;
+    const uint32_t sQ = smem_base, sK = sQ + SM::kQ, sV = sK + 2 * SM::kK, sP = sV + 2 * SM::kV;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem_gen + SM::kQ + 2 * SM::kK + 2 * SM::kV + SM::kP);
     const uint32_t bar0 = smem_u32(bars);
-    const uint32_t q_full = bar0, k_full = bar0 + 8, k_empty = bar0 + 24, v_full = bar0 + 40, v_empty = bar0 + 48;
-    const uint32_t s_full = bar0 + 56, s_empty = bar0 + 72, p_full = bar0 + 88, p_empty = bar0 + 96, o_full = bar0 + 104;
-    __shared__ uint32_t s_tmem;
-    __shared__ int s_abort_word;
+    const uint32_t q_full = bar0, k_full = bar0 + 8, k_empty = bar0 + 24, v_full = bar0 + 40, v_empty = bar0 + 56;
+    const uint32_t s_full = bar0 + 72, s_empty = bar0 + 88, p_full = bar0 + 104, p_empty = bar0 + 112, o_full = bar0 + 120;
+    uint32_t& s_tmem = *reinterpret_cast<uint32_t*>(bars + 16);
+    int& s_abort_word = *reinterpret_cast<int*>(reinterpret_cast<uint8_t*>(bars + 16) + 4);
     volatile int* s_abort = &s_abort_word;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -92,11 +102,10 @@ __global__ void __launch_bounds__(kUThreads, 2) attn_block_umma_kernel(const __g
     const int band_hi = min(n_max + a.block - 1, a.S);
     const int n_pred_tiles = (a.step > 1 && band_hi > n_min) ? (band_hi + kUKey - 1) / kUKey - band_lo_tile : 0;
     const int n_iter = n_true_tiles + n_pred_tiles;
-    const int J = 2 * n_iter;                                   // pass 1 then pass 2 over the same tiles
+    const int J = n_iter;                                       // one pass over the key tiles
     auto tile_of = [&](int j, bool& pred, int& kt) {
-        const int t = j >= n_iter ? j - n_iter : j;
-        pred = t >= n_true_tiles;
-        kt = pred ? band_lo_tile + (t - n_true_tiles) : t;
+        pred = j >= n_true_tiles;
+        kt = pred ? band_lo_tile + (j - n_true_tiles) : j;
     };
 
     if (threadIdx.x == 0) {
@@ -104,8 +113,8 @@ __global__ void __launch_bounds__(kUThreads, 2) attn_block_umma_kernel(const __g
         for (int s = 0; s < 2; ++s) {
             mbar_init(k_full + 8 * s, 1); mbar_init(k_empty + 8 * s, 1);
             mbar_init(s_full + 8 * s, 1); mbar_init(s_empty + 8 * s, 4);
+            mbar_init(v_full + 8 * s, 1); mbar_init(v_empty + 8 * s, 1);
         }
-        mbar_init(v_full, 1); mbar_init(v_empty, 1);
         mbar_init(p_full, 4); mbar_init(p_empty, 1);
         mbar_init(o_full, 1);
         s_abort_word = 0;
@@ -137,24 +146,22 @@ __global__ void __launch_bounds__(kUThreads, 2) attn_block_umma_kernel(const __g
                     tma_load_2d(sK + st * SM::kK + hf * (kUKey * 128), pred ? &tmKp : &tmKt, k_full + 8 * st, kvh * DH + hf * 64,
                                 row_base + kt * kUKey);
                 ++k_issued;
-                if (j >= n_iter) {
-                    const int t2 = j - n_iter;
-                    ok = mbar_wait(v_empty, (t2 & 1) ^ 1, s_abort);
-                    if (!ok) break;
-                    mbar_expect_tx(v_full, SM::kV);
-                    // values as they lie, [key][head_dim]: an MN-major B operand, one box of 64 keys x 64 dims per 64 dims
+                ok = mbar_wait(v_empty + 8 * st, ((j >> 1) & 1) ^ 1, s_abort);
+                if (!ok) break;
+                mbar_expect_tx(v_full + 8 * st, SM::kV);
+                // values as they lie, [key][head_dim]: an MN-major B operand, one box of 64 keys x 64 dims per 64 dims
 #pragma unroll
-                    for (int hf = 0; hf < kHalves; ++hf)
-                        tma_load_2d(sV + hf * (kUKey * 128), pred ? &tmVp : &tmVt, v_full, kvh * DH + hf * 64, row_base + kt * kUKey);
-                    ++v_issued;
-                }
+                for (int hf = 0; hf < kHalves; ++hf)
+                    tma_load_2d(sV + st * SM::kV + hf * (kUKey * 128), pred ? &tmVp : &tmVt, v_full + 8 * st, kvh * DH + hf * 64,
+                                row_base + kt * kUKey);
+                ++v_issued;
             }
             if (*s_abort) {      // copies already requested still land: wait (bounded) for the last of each buffer
                 for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(q_full, 0); ++i) {}
                 for (int n = max(0, k_issued - 2); n < k_issued; ++n)
                     for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(k_full + 8 * (n & 1), (n >> 1) & 1); ++i) {}
-                if (v_issued > 0)
-                    for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(v_full, (v_issued - 1) & 1); ++i) {}
+                for (int n = max(0, v_issued - 2); n < v_issued; ++n)
+                    for (uint32_t i = 0; i < kSpinLimit && !mbar_try_wait(v_full + 8 * (n & 1), (n >> 1) & 1); ++i) {}
             }
         }
     } else if (warp == 1) {
@@ -184,20 +191,20 @@ __global__ void __launch_bounds__(kUThreads, 2) attn_block_umma_kernel(const __g
             issue_s(0);
             for (int j = 0; j < J && ok; ++j) {
                 if (j + 1 < J) issue_s(j + 1);               // S of the next tile runs under this tile's softmax
-                if (j >= n_iter && ok) {
-                    const int t2 = j - n_iter;
+                if (ok) {
+                    const int t2 = j;
                     ok = mbar_wait(p_full, t2 & 1, s_abort);
-                    if (ok) ok = mbar_wait(v_full, t2 & 1, s_abort);
+                    if (ok) ok = mbar_wait(v_full + 8 * (j & 1), (j >> 1) & 1, s_abort);
                     if (!ok) break;
                     fence_after();
-                    const uint64_t dp = umma_desc(sP), dv = umma_desc_mn(sV, kUKey * 128);
+                    const uint64_t dp = umma_desc(sP), dv = umma_desc_mn(sV + (j & 1) * SM::kV, kUKey * 128);
 #pragma unroll
                     for (int k = 0; k < kUKey / UMMA_K; ++k) {
                         const uint64_t koff_p = static_cast<uint64_t>((k * UMMA_K * 2) >> 4);      // P: K-major, 32 bytes per step
                         const uint64_t koff_v = static_cast<uint64_t>((k * UMMA_K * 128) >> 4);    // V: 16 key rows of 128 bytes per step
                         umma_bf16(tmem_base + 2 * kUKey, dp + koff_p, dv + koff_v, idesc_o, (t2 > 0 || k > 0) ? 1u : 0u);
                     }
-                    umma_commit(v_empty);
+                    umma_commit(v_empty + 8 * (j & 1));
                     umma_commit(p_empty);
                 }
             }
@@ -234,60 +241,78 @@ __global__ void __launch_bounds__(kUThreads, 2) attn_block_umma_kernel(const __g
             // visible keys of this row in this tile: [lo, hi) (true tiles: [0, n(p)); predicted band: [n(p), hi(p)))
             const bool full = valid && !pred && (kt0 + kUKey <= n_min);   // a tile below every n(p) of the CTA: no mask
             const int lo = pred ? n_row : 0, hi = pred ? hi_row : n_row;  // an invalid row has lo = hi = 0
-            if (j < n_iter) {
-                // pass 1: running maximum of the masked scores (the positive scale is applied to the maximum)
-                float mx = -INFINITY;
-                if (full) {
-#pragma unroll
-                    for (int c = 0; c < 4; ++c)
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) mx = fmaxf(mx, __uint_as_float(r[c][i]));
-                } else {
-#pragma unroll
-                    for (int c = 0; c < 4; ++c)
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const int key = kt0 + 16 * c + i;
-                            mx = fmaxf(mx, (key >= lo && key < hi) ? __uint_as_float(r[c][i]) : -INFINITY);
-                        }
-                }
-                m_row = fmaxf(m_row, mx * a.scale_log2);
-            } else {
-                // pass 2: P = exp2(S - max), rounded to bf16; the row sum is taken over the rounded weights
-                uint32_t pk[32];
-                const float neg_m = (m_row == -INFINITY) ? 0.f : -m_row;      // a row without keys has every weight masked below
-                float l0 = 0.f, l1 = 0.f;
+            // the tile's maximum of the masked scores (the positive scale is applied to the maximum)
+            float mx = -INFINITY;
+            if (full) {
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
 #pragma unroll
-                    for (int i = 0; i < 16; i += 2) {
-                        float p0 = exp2f(fmaf(__uint_as_float(r[c][i]), a.scale_log2, neg_m));
-                        float p1v = exp2f(fmaf(__uint_as_float(r[c][i + 1]), a.scale_log2, neg_m));
-                        if (!full) {
-                            const int key = kt0 + 16 * c + i;
-                            p0 = (key >= lo && key < hi) ? p0 : 0.f;
-                            p1v = (key + 1 >= lo && key + 1 < hi) ? p1v : 0.f;
-                        }
-                        const __nv_bfloat162 t = __floats2bfloat162_rn(p0, p1v);
-                        const uint32_t bits = *reinterpret_cast<const uint32_t*>(&t);
-                        l0 += __uint_as_float(bits << 16);
-                        l1 += __uint_as_float(bits & 0xffff0000u);
-                        pk[(16 * c + i) >> 1] = bits;
-                    }
-                l_row += l0 + l1;
-                const int t2 = j - n_iter;
-                if (ok) ok = mbar_wait(p_empty, (t2 & 1) ^ 1, s_abort);     // the previous tile's P V has read the buffer
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                // row `row` of the [128 x 64] operand tile: 16-byte chunk c at position c ^ (row & 7) (128-byte swizzle)
+                    for (int i = 0; i < 16; ++i) mx = fmaxf(mx, __uint_as_float(r[c][i]));
+            } else {
 #pragma unroll
-                for (int c = 0; c < 8; ++c)
-                    *reinterpret_cast<uint4*>(smem_gen + (sP - smem_base) + row * 128 + ((c ^ (row & 7)) << 4)) =
-                        make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-                fence_async_smem();                              // generic-proxy writes -> visible to the MMA's async proxy
-                __syncwarp();
-                if (lane == 0) mbar_arrive(p_full);
+                for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const int key = kt0 + 16 * c + i;
+                        mx = fmaxf(mx, (key >= lo && key < hi) ? __uint_as_float(r[c][i]) : -INFINITY);
+                    }
             }
+            mx *= a.scale_log2;
+            // The row's reference point m only moves when a tile exceeds it by more than kSlack (in log2 units): the weights stay
+            // below 2^kSlack, well inside bf16 and fp32, and the accumulated O row and row sum are then scaled by 2^(m_old - m_new).
+            // A row's first tile with a visible key sets m (nothing has been accumulated for that row: factor 1).
+            const float m_old = m_row;
+            const bool grow = mx > m_old + kSlack;
+            m_row = grow ? mx : m_old;
+            const float factor = (grow && m_old != -INFINITY) ? exp2f(m_old - m_row) : 1.f;
+            // P = exp2(S - m), rounded to bf16; the row sum is taken over the rounded weights
+            uint32_t pk[32];
+            const float neg_m = (m_row == -INFINITY) ? 0.f : -m_row;          // a row without keys has every weight masked below
+            float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+#pragma unroll
+                for (int i = 0; i < 16; i += 2) {
+                    float p0 = exp2f(fmaf(__uint_as_float(r[c][i]), a.scale_log2, neg_m));
+                    float p1v = exp2f(fmaf(__uint_as_float(r[c][i + 1]), a.scale_log2, neg_m));
+                    if (!full) {
+                        const int key = kt0 + 16 * c + i;
+                        p0 = (key >= lo && key < hi) ? p0 : 0.f;
+                        p1v = (key + 1 >= lo && key + 1 < hi) ? p1v : 0.f;
+                    }
+                    const __nv_bfloat162 t = __floats2bfloat162_rn(p0, p1v);
+                    const uint32_t bits = *reinterpret_cast<const uint32_t*>(&t);
+                    l0 += __uint_as_float(bits << 16);
+                    l1 += __uint_as_float(bits & 0xffff0000u);
+                    pk[(16 * c + i) >> 1] = bits;
+                }
+            l_row = fmaf(l_row, factor, l0 + l1);
+            if (ok) ok = mbar_wait(p_empty, (j & 1) ^ 1, s_abort);           // the previous tile's P V has completed: O and the P buffer are free
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            if (__any_sync(0xffffffffu, factor != 1.f)) {
+                // some row of this warp moved its reference point: scale the warp's 32 O rows in tensor memory (factor 1 elsewhere)
+                fence_after();
+#pragma unroll
+                for (int c0 = 0; c0 < DH; c0 += 16) {
+                    uint32_t ro[16];
+                    tmem_ld16(tmem_base + 2 * kUKey + c0 + lane_off, ro);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) ro[i] = __float_as_uint(__uint_as_float(ro[i]) * factor);
+                    tmem_st16(tmem_base + 2 * kUKey + c0 + lane_off, ro);
+                }
+                tmem_st_wait();
+                fence_before();
+            }
+            // row `row` of the [128 x 64] operand tile: 16-byte chunk c at position c ^ (row & 7) (128-byte swizzle)
+#pragma unroll
+            for (int c = 0; c < 8; ++c)
+                *reinterpret_cast<uint4*>(smem_gen + (sP - smem_base) + row * 128 + ((c ^ (row & 7)) << 4)) =
+                    make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+            fence_async_smem();                              // generic-proxy writes -> visible to the MMA's async proxy
+            __syncwarp();
+            if (lane == 0) mbar_arrive(p_full);
         }
         // ---- O from tensor memory, normalised, straight to global memory (one 2*DH-byte row per thread)
         if (n_iter > 0) {

@@ -247,6 +247,42 @@ def test_block_forward_bf16_head_dim_128(S, block, offset, sim_steps):
     beagle_check_device(head_gpu.ctx)
 
 
+def rising_score_inputs(w, head_cpu, S, rng, top=14.0):
+    """One repeated token and states h_j = a_j g + noise with g chosen so that query head 0's score of key j rises linearly
+    from 0 to `top` (natural units) along the sequence; the other heads get other slopes, some falling."""
+    tokens = np.full((1, S), int(WL.make_tokens(w, rng, (1,))[0]), dtype=np.int32)
+    dh = w.head_dim
+    q = O.rms_norm(O.embed_tokens(head_cpu, tokens[0][:1]), head_cpu.g_q, head_cpu.cfg.rms_eps)[0] @ head_cpu.w_q.T
+    g = head_cpu.w_k[:dh].T @ q[:dh]
+    gamma = np.linalg.norm(g)
+    g /= gamma
+    a = top * np.sqrt(dh) / gamma * np.arange(S) / (S - 1)
+    hidden = WL.round_to_storage((a[:, None] * g[None, :] + 0.5 * WL.make_hidden(w, rng, S)).reshape(-1), w.dtype).reshape(1, S, w.hidden)
+    k = hidden[0].astype(np.float64) @ head_cpu.w_k.T
+    G = w.n_q_heads // w.n_kv_heads
+    rise = np.array([(q[h * dh:(h + 1) * dh] @ (k[S - 8] - k[0])[(h // G) * dh:(h // G + 1) * dh]) / np.sqrt(dh) for h in range(w.n_q_heads)])
+    return tokens, hidden, rise * np.log2(np.e)
+
+
+@pytest.mark.parametrize("w,sim_steps", [(SMALL_MHA, 1), (SMALL_MHA, 3), (SMALL_GQA, 2)], ids=lambda v: getattr(v, "name", str(v)))
+def test_block_attention_when_later_keys_dominate(w, sim_steps):
+    """Scores that rise by 20 bits along the sequence for one query head (and fall for others): every row's largest scores lie in
+    its LAST key tiles, so a kernel that keeps a reference point per row and accumulates against it has to move that point, and
+    rescale what it has accumulated, several times per row.  Compared with the oracle in its bf16-storage mode (both sides then
+    hold the same rounded q, k, v: at scores this large the unrounded oracle differs by what rounding k alone does to the weights)."""
+    head_gpu, head_cpu, _ = build(w, max_slots=1, max_ctx=64)
+    S, block = 330, 4
+    tokens, hidden, rise_bits = rising_score_inputs(w, head_cpu, S, WL.data_rng(w, 4242 + sim_steps))
+    assert rise_bits.max() > 16, rise_bits                       # the premise: more than two moves of 8 bits for some head
+    logits, argmax, hid = head_gpu.block_forward(to_dev(tokens, w.dtype), to_dev(hidden, w.dtype), block, 0, sim_steps)
+    torch.cuda.synchronize()
+    ref = O.block_forward(head_cpu.with_storage("bf16"), tokens[0], hidden[0], block, 0, sim_steps)
+    assert_close(hid[0].float().cpu().numpy(), ref["hidden"], w.dtype, "hidden")
+    assert_close(logits[0].cpu().numpy(), ref["logits"], w.dtype, "logits")
+    from paper_2505_24544_b200.binding import beagle_check_device
+    beagle_check_device(head_gpu.ctx)
+
+
 @pytest.mark.parametrize("name,stage,sim_steps,soft", [("c1", "early", 1, True), ("c1", "late", 3, False), ("gqa", "early", 1, False),
                                                         ("gqa", "late", 4, True), ("mha", "late", 2, True)])
 def test_block_loss_forward(name, stage, sim_steps, soft):
