@@ -5,7 +5,7 @@
 // tile, one TMEM lane and one softmax thread per query, so row maxima and row sums need no
 // cross-thread reduction.  Keys are walked in tiles of 64 (true tiles up to the largest n(p) of the
 // CTA, then the predicted band on the diagonal, as in the mma.sync kernel), once:
-//   S = Q K^T per tile -> P = exp2(S - m) rounded to bf16 (row sums over the rounded weights), written to shared
+//   S = Q K^T per tile -> P = exp2(S - m) rounded to bf16 (row sums in fp32 over the unrounded weights), written to shared
 //   memory in the MMA's operand layout -> O += P V accumulated in TMEM over all tiles, read once at the end,
 //   normalised and stored.
 // m is the row's reference point, not its running maximum: it is set by the row's first visible tile and moves only when a
@@ -265,7 +265,7 @@ __global__ void __launch_bounds__(kUThreads, 2) attn_block_umma_kernel(const __g
             const bool grow = mx > m_old + kSlack;
             m_row = grow ? mx : m_old;
             const float factor = (grow && m_old != -INFINITY) ? exp2f(m_old - m_row) : 1.f;
-            // P = exp2(S - m), rounded to bf16; the row sum is taken over the rounded weights
+            // P = exp2(S - m), rounded to bf16 for the MMA; the row sum is taken over the unrounded weights (fp32)
             uint32_t pk[32];
             const float neg_m = (m_row == -INFINITY) ? 0.f : -m_row;          // a row without keys has every weight masked below
             float l0 = 0.f, l1 = 0.f;
@@ -281,10 +281,9 @@ __global__ void __launch_bounds__(kUThreads, 2) attn_block_umma_kernel(const __g
                         p1v = (key + 1 >= lo && key + 1 < hi) ? p1v : 0.f;
                     }
                     const __nv_bfloat162 t = __floats2bfloat162_rn(p0, p1v);
-                    const uint32_t bits = *reinterpret_cast<const uint32_t*>(&t);
-                    l0 += __uint_as_float(bits << 16);
-                    l1 += __uint_as_float(bits & 0xffff0000u);
-                    pk[(16 * c + i) >> 1] = bits;
+                    l0 += p0;
+                    l1 += p1v;
+                    pk[(16 * c + i) >> 1] = *reinterpret_cast<const uint32_t*>(&t);
                 }
             l_row = fmaf(l_row, factor, l0 + l1);
             if (ok) ok = mbar_wait(p_empty, (j & 1) ^ 1, s_abort);           // the previous tile's P V has completed: O and the P buffer are free

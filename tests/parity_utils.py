@@ -147,9 +147,11 @@ def check_tokens(gpu_tok: np.ndarray, ref_logits: np.ndarray, what: str):
             continue
         top = np.partition(flat[r], -2)[-2:]
         margin = top[1] - top[0]
-        second = [i for i in np.argsort(flat[r])[-2:]]
-        assert margin <= MARGIN and gt[r] in second, (
-            f"{what}: row {r}: gpu id {gt[r]}, oracle id {ref_ids[r]}, oracle top-2 margin {margin:.3e}")
+        # a different id is admissible only in a near tie, and only if the oracle itself puts it within the margin of its maximum
+        # (with three or more logits inside the margin the runner-up is not the only valid answer)
+        assert margin <= MARGIN and 0 <= gt[r] < flat.shape[1] and top[1] - flat[r][gt[r]] <= MARGIN, (
+            f"{what}: row {r}: gpu id {gt[r]} (oracle logit {flat[r][min(max(int(gt[r]), 0), flat.shape[1] - 1)]:.6f}), oracle id {ref_ids[r]} "
+            f"(logit {top[1]:.6f}), oracle top-2 margin {margin:.3e}")
     return ref_ids.reshape(ref_logits.shape[:-1])
 
 
