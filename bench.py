@@ -790,7 +790,7 @@ def main():
     ap.add_argument("--fp8-lm-head", action="store_true", help="diagnostic: the serve scenario with the optional FP8 LM head (not the headline arithmetic)")
     ap.add_argument("--only-block", action="store_true", help="diagnostic: time only the block-attention forward (C5 shape)")
     ap.add_argument("--block-batch", type=int, default=0, help="sequences of the block forward (default: the workload's 8)")
-    ap.add_argument("--only-legs", action="store_true", help="diagnostic: only the prefill and verify-from-logits legs of the headline workload")
+    ap.add_argument("--only-legs", action="store_true", help="diagnostic: only the prefill, verification and draft-tree legs of the headline workload")
     ap.add_argument("--legs-batch", type=int, default=0, help="with --only-legs: cut the workload down to this many sequences (profiler captures)")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -848,6 +848,7 @@ def main():
         if w.name == HEADLINE and args.legs_batch == 0:
             scn3 = ServeScenario(head, w3, iters, device)
             out["prefill"][w3.name] = bench_prefill(scn3, peaks)
+            out["draft_tree"] = bench_draft_tree(head, w3, scn3, steps=5, warmup=3, peaks=peaks)
             out["verify_greedy_logits"][w3.name] = bench_verify_greedy_logits(head, w3, peaks)
         if rank == 0:
             print(json.dumps(out), flush=True)
