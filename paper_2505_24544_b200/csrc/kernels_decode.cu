@@ -694,12 +694,13 @@ int launch_row_argmax(int logits_dtype, const void* logits, int rows, int V, uns
 // for that); measured at 32 x 7 x 128256 fp32 logits, more and smaller slices only add per-CTA cost.
 // ------------------------------------------------------------------------------------------------
 template <typename T>
-__global__ void __launch_bounds__(256, 8) verify_greedy_fused_kernel(const T* __restrict__ logits, int V, int nsplit, int per, int gamma,
-                                                                     const int32_t* __restrict__ draft,
-                                                                     unsigned long long* __restrict__ keys, int* __restrict__ tickets,
-                                                                     int32_t* __restrict__ accept_len, int32_t* __restrict__ out_tokens) {
+__global__ void __launch_bounds__(256, 8) verify_greedy_fused_kernel(const T* logits, int V, int nsplit, int per, int gamma,
+                                                                     const int32_t* draft, unsigned long long* keys, int* tickets,
+                                                                     int32_t* accept_len, int32_t* out_tokens) {
     constexpr int VEC = VecOf<T>::N;
     const int split = blockIdx.x, row = blockIdx.y;
+    pdl_launch_dependents();
+    pdl_wait();                      // the logits and the drafted tokens may be the output of the kernels before
     const int b = row / (gamma + 1);
     const T* z = logits + (size_t)row * V;
     const int lo = split * per, hi = min(V, lo + per);
@@ -724,7 +725,7 @@ __global__ void __launch_bounds__(256, 8) verify_greedy_fused_kernel(const T* __
         for (; i + 3 * 256 < nvec; i += 4 * 256) {       // four independent 16-byte loads in flight per thread
             uint4 u[4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) u[j] = ld_stream16(zb + (size_t)(i + j * 256) * VEC);
+            for (int j = 0; j < 4; ++j) u[j] = ld_act_stream16(zb + (size_t)(i + j * 256) * VEC);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 float f[VEC];
@@ -735,7 +736,7 @@ __global__ void __launch_bounds__(256, 8) verify_greedy_fused_kernel(const T* __
         }
         for (; i < nvec; i += 256) {
             float f[VEC];
-            unpack16<T>(ld_stream16(zb + (size_t)i * VEC), f);
+            unpack16<T>(ld_act_stream16(zb + (size_t)i * VEC), f);
 #pragma unroll
             for (int v = 0; v < VEC; ++v) take(f[v], body0 + i * VEC + v);
         }
@@ -803,9 +804,9 @@ int launch_verify_greedy_fused(int logits_dtype, const void* logits, int B, int 
     per = (per + vec - 1) / vec * vec;
     dim3 grid(nsplit, rows);
     if (logits_dtype == 0)
-        verify_greedy_fused_kernel<float><<<grid, 256, 0, stream>>>((const float*)logits, V, nsplit, per, gamma, draft, keys, tickets, accept_len, out_tokens);
+        launch_pdl(verify_greedy_fused_kernel<float>, grid, dim3(256), 0, stream, (const float*)logits, V, nsplit, per, gamma, draft, keys, tickets, accept_len, out_tokens);
     else
-        verify_greedy_fused_kernel<bf16><<<grid, 256, 0, stream>>>((const bf16*)logits, V, nsplit, per, gamma, draft, keys, tickets, accept_len, out_tokens);
+        launch_pdl(verify_greedy_fused_kernel<bf16>, grid, dim3(256), 0, stream, (const bf16*)logits, V, nsplit, per, gamma, draft, keys, tickets, accept_len, out_tokens);
     return 1;
 }
 
