@@ -376,6 +376,17 @@ def elt(w):
     return 2 if w.dtype == "bf16" else 4
 
 
+def workload_config(w: WL.Workload, parallelism: str) -> dict:
+    """The `config` object of a bench line: the workload and nothing that depends on the run, so that both arms print the same."""
+    e, d, qd, kd, m, V = elt(w), w.hidden, w.n_q_heads * w.head_dim, w.n_kv_heads * w.head_dim, w.mlp_dim, w.vocab
+    weights_gb = e * (2 * d * qd + 2 * d * kd + 3 * d * m + V * d) / 1e9
+    return {"workload": w.name, "batch": w.batch, "gamma": w.gamma, "ctx": [w.ctx_min, w.ctx_max],
+            "hidden": w.hidden, "heads": [w.n_q_heads, w.n_kv_heads, w.head_dim], "mlp": w.mlp_dim, "vocab": w.vocab,
+            "step": STEP_TEXT,
+            "l2": "inputs larger than L2: every draft step streams the head's %.2f GB of weights and the batch's K/V cache" % weights_gb,
+            "parallelism": parallelism}
+
+
 def step_bytes(w: WL.Workload, mean_ctx: float):
     """Algorithmic HBM bytes of one draft step of the whole batch (weights once + K/V per sequence)."""
     e, d, qd, kd, m, V = elt(w), w.hidden, w.n_q_heads * w.head_dim, w.n_kv_heads * w.head_dim, w.mlp_dim, w.vocab
@@ -510,9 +521,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
         "warmup": warm, "ms_per_step": 1e3 * sec / steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "batch": w.batch, "gamma": w.gamma, "ctx": [w.ctx_min, w.ctx_max],
-                   "hidden": w.hidden, "heads": [w.n_q_heads, w.n_kv_heads, w.head_dim], "mlp": w.mlp_dim, "vocab": w.vocab,
-                   "step": STEP_TEXT, "parallelism": "single", "sample": sample},
+        "config": workload_config(w, "single"),
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample, "nproc": os.cpu_count(),
                          "cpu_model": cpu_model()},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -889,14 +898,11 @@ def main():
         "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": ("bf16" if w.dtype == "bf16" else "f32") + ("+e4m3 LM head (diagnostic run, not the headline)" if args.fp8_lm_head else ""),
         "data": "synthetic",
-        "config": {"workload": w.name, "batch": w.batch, "gamma": w.gamma, "ctx": [w.ctx_min, w.ctx_max],
-                   "hidden": w.hidden, "heads": [w.n_q_heads, w.n_kv_heads, w.head_dim], "mlp": w.mlp_dim, "vocab": w.vocab,
-                   "step": STEP_TEXT,
-                   "l2": "inputs larger than L2 (weights %.2f GB + K/V per draft step)" % (step_bytes(w, mean_ctx) / 1e9),
-                   "weights": "row-major as the caller gave them + tile-major copies of the eight projection matrices, made once at load "
-                              "(beagle_pack_weights, %.2f GB), which the draft steps of this batch size stream"
-                              % ((head.ctx.packed_buf.numel() if head.ctx.packed_buf is not None else 0) / 1e9),
-                   "mean_tau": scn.mean_tau, "parallelism": "replicas" if world > 1 else "single"},
+        "config": workload_config(w, "replicas" if world > 1 else "single"),
+        "run": {"mean_tau": scn.mean_tau,
+                "weights": "row-major as the caller gave them + tile-major copies of the eight projection matrices, made once at load "
+                           "(beagle_pack_weights, %.2f GB), which the draft steps of this batch size stream"
+                           % ((head.ctx.packed_buf.numel() if head.ctx.packed_buf is not None else 0) / 1e9)},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms / args.steps},
         "gpu_launches": launches,
         "roofline": roofline,

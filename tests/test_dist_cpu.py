@@ -76,3 +76,9 @@ def test_reference_arm_prints_the_contract_line_on_a_small_workload():
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["value"] == line["value"]
     assert line["e2e"] == {"value": line["value"], "unit": line["unit"], "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
     assert line["config"]["workload"] == "c1_tiny_fp32" and line["higher_is_better"] is True
+    # `config` holds the workload only (what depends on the run sits elsewhere in the line), so the library's arm prints the same object
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2505_24544_b200 import workloads as WL
+    assert line["config"] == bench.workload_config(WL.WORKLOADS["c1_tiny_fp32"], "single")
+    assert set(line["config"]) == {"workload", "batch", "gamma", "ctx", "hidden", "heads", "mlp", "vocab", "step", "l2", "parallelism"}
