@@ -136,7 +136,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kv_umma_kernel(const 
     const uint32_t s_full = bar0 + 56, s_empty = bar0 + 72, p_full = bar0 + 88, p_empty = bar0 + 96, o_full = bar0 + 104;
     __shared__ uint32_t s_tmem;
     __shared__ int s_abort_word;
-    __shared__ float s_ls[2][kBS], s_dl[2][kBS];
+    __shared__ __align__(16) float s_ls[2][kBS], s_dl[2][kBS];     // read four columns at a time
     __shared__ int s_n[2][kBS], s_hi[2][kBS];
     volatile int* s_abort = &s_abort_word;
 
@@ -311,23 +311,30 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kv_umma_kernel(const 
 #pragma unroll
             for (int c = 0; c < 2; ++c) {
 #pragma unroll
-                for (int i = 0; i < 16; i += 2) {
-                    float pv[2], dv[2];
+                for (int i = 0; i < 16; i += 4) {
+                    // the four queries' log-sum-exp and delta with one 16-byte load each (the same words for every lane)
+                    const int col0 = 32 * half + 16 * c + i;
+                    const float4 ls4 = *reinterpret_cast<const float4*>(&s_ls[st][col0]);
+                    const float4 dl4 = *reinterpret_cast<const float4*>(&s_dl[st][col0]);
+                    const float lsv[4] = {ls4.x, ls4.y, ls4.z, ls4.w}, dlv[4] = {dl4.x, dl4.y, dl4.z, dl4.w};
+                    float pv[4], dv[4];
 #pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        const int col = 32 * half + 16 * c + i + u;
-                        float p = exp2f(fmaf(__uint_as_float(rs[c][i + u]), a.scale_log2, -s_ls[st][col]));
+                    for (int u = 0; u < 4; ++u) {
+                        float p = exp2f(fmaf(__uint_as_float(rs[c][i + u]), a.scale_log2, -lsv[u]));
                         if (!full) {
-                            const int n = s_n[st][col], hi = s_hi[st][col];
+                            const int n = s_n[st][col0 + u], hi = s_hi[st][col0 + u];
                             const bool vis = pred ? (key >= n && key < hi) : (key < n);
                             p = vis ? p : 0.f;
                         }
                         pv[u] = p;
-                        dv[u] = p * (__uint_as_float(rd[c][i + u]) - s_dl[st][col]);
+                        dv[u] = p * (__uint_as_float(rd[c][i + u]) - dlv[u]);
                     }
-                    const __nv_bfloat162 tp = __floats2bfloat162_rn(pv[0], pv[1]), td = __floats2bfloat162_rn(dv[0], dv[1]);
-                    pk_p[(16 * c + i) >> 1] = *reinterpret_cast<const uint32_t*>(&tp);
-                    pk_ds[(16 * c + i) >> 1] = *reinterpret_cast<const uint32_t*>(&td);
+#pragma unroll
+                    for (int u = 0; u < 4; u += 2) {
+                        const __nv_bfloat162 tp = __floats2bfloat162_rn(pv[u], pv[u + 1]), td = __floats2bfloat162_rn(dv[u], dv[u + 1]);
+                        pk_p[(16 * c + i + u) >> 1] = *reinterpret_cast<const uint32_t*>(&tp);
+                        pk_ds[(16 * c + i + u) >> 1] = *reinterpret_cast<const uint32_t*>(&td);
+                    }
                 }
             }
             if (ok) ok = mbar_wait(p_empty, (j & 1) ^ 1, s_abort);   // the previous tile's products have read the operand tiles
