@@ -667,6 +667,29 @@ def test_status_codes_for_capacity_and_state():
     torch.cuda.synchronize()
 
 
+def test_status_codes_of_pack_weights():
+    """Buffer too small: CAPACITY; misaligned: INVALID_ARG; an fp32 head accepts the call and needs no bytes."""
+    import ctypes as C
+    from paper_2505_24544_b200 import binding as B
+    w = SMALL_GQA.scaled(batch=12)
+    head, _, _ = build(w, pack_weights=False)
+    lib, n = head.ctx.lib, B.beagle_packed_weights_bytes(head.cfg, False)
+    assert n > 0 and head.ctx.packed_buf is None
+    buf = torch.empty(n + 512, dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    assert lib.beagle_pack_weights(head.ctx.handle, buf.data_ptr(), n - 1, stream) == 3
+    assert "packed weights need" in lib.beagle_last_error(head.ctx.handle).decode()
+    assert lib.beagle_pack_weights(head.ctx.handle, buf.data_ptr() + 16, n, stream) == 1
+    assert lib.beagle_pack_weights(head.ctx.handle, buf.data_ptr(), n, stream) == 0
+    assert lib.beagle_pack_weights(head.ctx.handle, None, 0, stream) == 0
+    torch.cuda.synchronize()
+    c1 = WL.WORKLOADS["c1_tiny_fp32"]
+    head32, _, _ = build(c1)
+    assert head32.ctx.packed_buf is None and B.beagle_packed_weights_bytes(head32.cfg, False) == 0
+    assert lib.beagle_pack_weights(head32.ctx.handle, buf.data_ptr(), n, stream) == 0
+    B.beagle_check_device(head.ctx)
+
+
 def test_status_codes_of_the_training_entry_points():
     """Argument errors of beagle_block_loss / beagle_block_grad are reported before any launch."""
     from paper_2505_24544_b200.binding import BeagleError
